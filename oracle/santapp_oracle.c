@@ -1,0 +1,542 @@
+/*
+ * SANTA++ decode attention — plain fp64 CPU oracle.
+ *
+ * TEST INFRASTRUCTURE, NOT PRODUCT CODE. This file is the slow, obviously
+ * correct restatement of what the paper's method computes. Only the test
+ * suite, the smoke check and the benchmark's cpu-baseline / reference arm may
+ * call it. It shares no code, tables or helpers with the CUDA path.
+ *
+ * Every function follows one passage of the paper, in the paper's order and
+ * notation, with no blocking, fusion or reordering:
+ *   orc_dense_head            full-cache attention, Eq. (method-attention)
+ *   orc_contiguous_parents    Algorithm 4 (contiguous parent partition)
+ *   orc_build_teams           Algorithm 2 (actual-key teams from parents)
+ *   orc_decode_head_given_gumbel / orc_decode_head
+ *                             Algorithm 1 (SANTA++ attention, one query head),
+ *                             routing weight Eq. (method-routing), inclusion
+ *                             correction Eq. (method-inclusion), estimator
+ *                             Eq. (method-estimate)
+ *   orc_philox4x32_10, orc_uniform_open, orc_gumbel, orc_team_word
+ *                             the reproducible Gumbel(0,1) stream (the paper
+ *                             only asks for independent Gumbel draws; the
+ *                             generator and its keying are this build's
+ *                             reading and are documented with the function)
+ *   orc_logical_access_*      logical KV-access counter, Eq. (qwen-logical-access)
+ *   orc_team_budget           selected-team count, Eq. (method-budget)
+ *
+ * Parity pins (tests marked "not gpu"): Philox words against an independent
+ * library generator; Gumbel law by Kolmogorov-Smirnov and moments; first-draw
+ * law and the every-key-its-own-team limit against softmax; K >= M against a
+ * library softmax; inclusion probabilities against exact enumeration of the
+ * successive-sampling law and against 1e5-draw frequencies; unbiasedness of
+ * the two unnormalised sums by quadrature and Monte Carlo; Algorithm 2 on
+ * hand-worked parents and duplicate keys; the accounting helpers against the
+ * figures the paper prints.
+ * Parity unpinned: nothing in this file. (Accuracy of the sampled output
+ * against dense attention on real model data is outside what can be pinned
+ * here; only the estimator identities are.)
+ *
+ * Build: gcc -O2 -ffp-contract=off -fPIC -shared [-fopenmp] (see build_oracle.py).
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+/* ------------------------------------------------------------------------- */
+/* Random stream                                                             */
+/* ------------------------------------------------------------------------- */
+
+/* Philox4x32 with 10 rounds (Salmon, Moraes, Dror, Shaw 2011): a 128-bit
+ * counter and a 64-bit key give four 32-bit words. Each round multiplies two
+ * counter words by fixed odd constants, swaps high/low halves into the other
+ * lanes and xors in the key; the key is advanced by Weyl constants between
+ * rounds. */
+void orc_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4])
+{
+    uint32_t c0 = ctr[0], c1 = ctr[1], c2 = ctr[2], c3 = ctr[3];
+    uint32_t k0 = key[0], k1 = key[1];
+    for (int round = 0; round < 10; ++round) {
+        uint64_t prod0 = (uint64_t)0xD2511F53u * (uint64_t)c0;
+        uint64_t prod1 = (uint64_t)0xCD9E8D57u * (uint64_t)c2;
+        uint32_t hi0 = (uint32_t)(prod0 >> 32), lo0 = (uint32_t)prod0;
+        uint32_t hi1 = (uint32_t)(prod1 >> 32), lo1 = (uint32_t)prod1;
+        uint32_t n0 = hi1 ^ c1 ^ k0;
+        uint32_t n1 = lo1;
+        uint32_t n2 = hi0 ^ c3 ^ k1;
+        uint32_t n3 = lo0;
+        c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+        k0 += 0x9E3779B9u;
+        k1 += 0xBB67AE85u;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+/* The 32-bit word that belongs to team g (0-based, local to its sequence and
+ * KV head) for query head `head` at decode step `step` on stream `stream`:
+ * key = (low, high) halves of the seed; counter = (g / 4, step, head, stream);
+ * word g mod 4 of the block. Heads that share a KV head differ in the counter,
+ * so their draws are independent, as the GQA rule of the Method section
+ * requires. */
+uint32_t orc_team_word(uint64_t seed, uint32_t step, uint32_t head, uint32_t stream, uint32_t g)
+{
+    uint32_t ctr[4] = { g >> 2, step, head, stream };
+    uint32_t key[2] = { (uint32_t)(seed & 0xFFFFFFFFu), (uint32_t)(seed >> 32) };
+    uint32_t out[4];
+    orc_philox4x32_10(ctr, key, out);
+    return out[g & 3u];
+}
+
+/* Uniform on the open interval: the centre of the x-th of 2^32 equal cells. */
+double orc_uniform_open(uint32_t x)
+{
+    return ((double)x + 0.5) * (1.0 / 4294967296.0);
+}
+
+/* Standard Gumbel by inversion of the CDF exp(-exp(-x)) quoted in the
+ * "Conditional inclusion correction" paragraph: G = -log(-log u). */
+double orc_gumbel(uint32_t x)
+{
+    return -log(-log(orc_uniform_open(x)));
+}
+
+void orc_gumbel_many(uint64_t seed, uint32_t step, uint32_t head, uint32_t stream,
+                     int32_t M, double *gumbel /* [M] */)
+{
+    for (int32_t g = 0; g < M; ++g)
+        gumbel[g] = orc_gumbel(orc_team_word(seed, step, head, stream, (uint32_t)g));
+}
+
+/* ------------------------------------------------------------------------- */
+/* Full-cache attention, Eq. (method-attention)                              */
+/* ------------------------------------------------------------------------- */
+
+static double dot(const double *a, const double *b, int d)
+{
+    double s = 0.0;
+    for (int j = 0; j < d; ++j) s += a[j] * b[j];
+    return s;
+}
+
+/* s_i = q.k_i * scale, Z = sum e^{s_i}, U = sum e^{s_i} v_i, o = U / Z over
+ * the n rows of (k, v). Evaluated with the usual max shift, which cancels in
+ * the ratio. */
+void orc_dense_head(int d, const double *q, int64_t n, const double *k, const double *v,
+                    double scale, double *o /* [d] */)
+{
+    double smax = -INFINITY;
+    for (int64_t i = 0; i < n; ++i) {
+        double s = dot(q, k + i * d, d) * scale;
+        if (s > smax) smax = s;
+    }
+    double Z = 0.0;
+    for (int j = 0; j < d; ++j) o[j] = 0.0;
+    for (int64_t i = 0; i < n; ++i) {
+        double s = dot(q, k + i * d, d) * scale;
+        double a = exp(s - smax);
+        Z += a;
+        for (int j = 0; j < d; ++j) o[j] += a * v[i * d + j];
+    }
+    for (int j = 0; j < d; ++j) o[j] /= Z;
+}
+
+/* Dense attention over prompt rows followed by suffix rows (two buffers). */
+void orc_dense_head_two(int d, const double *q,
+                        int64_t n, const double *k, const double *v,
+                        int64_t t, const double *ks, const double *vs,
+                        double scale, double *o /* [d] */)
+{
+    double smax = -INFINITY;
+    for (int64_t i = 0; i < n; ++i) { double s = dot(q, k + i * d, d) * scale; if (s > smax) smax = s; }
+    for (int64_t i = 0; i < t; ++i) { double s = dot(q, ks + i * d, d) * scale; if (s > smax) smax = s; }
+    double Z = 0.0;
+    for (int j = 0; j < d; ++j) o[j] = 0.0;
+    for (int64_t i = 0; i < n; ++i) {
+        double a = exp(dot(q, k + i * d, d) * scale - smax);
+        Z += a;
+        for (int j = 0; j < d; ++j) o[j] += a * v[i * d + j];
+    }
+    for (int64_t i = 0; i < t; ++i) {
+        double a = exp(dot(q, ks + i * d, d) * scale - smax);
+        Z += a;
+        for (int j = 0; j < d; ++j) o[j] += a * vs[i * d + j];
+    }
+    for (int j = 0; j < d; ++j) o[j] /= Z;
+}
+
+/* ------------------------------------------------------------------------- */
+/* Algorithm 4: contiguous parent partition                                  */
+/* ------------------------------------------------------------------------- */
+
+/* Parents are consecutive spans of P tokens; the last may be short. Writes
+ * parent_start[0..n_parents] (0-based, half-open) and returns n_parents =
+ * ceil(N / P). */
+int32_t orc_contiguous_parents(int32_t N, int32_t P, int32_t *parent_start)
+{
+    int32_t n_parents = (N + P - 1) / P;
+    for (int32_t u = 0; u < n_parents; ++u) parent_start[u] = u * P;
+    parent_start[n_parents] = N;
+    return n_parents;
+}
+
+/* ------------------------------------------------------------------------- */
+/* Algorithm 2: actual-key teams from a parent partition                     */
+/* ------------------------------------------------------------------------- */
+
+static double sqdist(const double *a, const double *b, int d)
+{
+    double s = 0.0;
+    for (int j = 0; j < d; ++j) { double e = a[j] - b[j]; s += e * e; }
+    return s;
+}
+
+/* keys: [N][d] prefill keys in token order. Parents are given as index lists:
+ * parent u holds tokens parent_member[parent_start[u] .. parent_start[u+1]),
+ * listed in increasing token index. R = maximum representatives per parent.
+ * Outputs (teams in emission order: parent by parent, representative-selection
+ * order inside a parent):
+ *   team_start[M+1], team_member[N]  members of team g in increasing token index
+ *   rep_row[M]                       token index of the representative of team g
+ * Returns M. Ties: representative choices go to the smallest token index,
+ * assignments to the earliest-selected representative ("Shared team
+ * construction" paragraph). */
+int32_t orc_build_teams(int32_t N, int d, const double *keys,
+                        int32_t n_parents, const int32_t *parent_start, const int32_t *parent_member,
+                        int32_t R,
+                        int32_t *team_start, int32_t *team_member, int32_t *rep_row)
+{
+    (void)N;
+    double *mu = (double *)malloc(sizeof(double) * (size_t)d);
+    int32_t M = 0, rows_out = 0;
+    team_start[0] = 0;
+    for (int32_t p = 0; p < n_parents; ++p) {
+        const int32_t *C = parent_member + parent_start[p];
+        int32_t nC = parent_start[p + 1] - parent_start[p];
+        int32_t r = R < nC ? R : nC;
+        /* parent mean */
+        for (int j = 0; j < d; ++j) mu[j] = 0.0;
+        for (int32_t a = 0; a < nC; ++a)
+            for (int j = 0; j < d; ++j) mu[j] += keys[(int64_t)C[a] * d + j];
+        for (int j = 0; j < d; ++j) mu[j] /= (double)nC;
+        /* first representative: the actual key nearest the mean */
+        int32_t *L = (int32_t *)malloc(sizeof(int32_t) * (size_t)r);      /* positions in C */
+        char *is_rep = (char *)calloc((size_t)nC, 1);
+        double best = INFINITY; int32_t arg = 0;
+        for (int32_t a = 0; a < nC; ++a) {
+            double dist = sqdist(keys + (int64_t)C[a] * d, mu, d);
+            if (dist < best) { best = dist; arg = a; }
+        }
+        L[0] = arg; is_rep[arg] = 1;
+        /* farthest-first: maximise the distance to the nearest chosen representative */
+        for (int32_t u = 1; u < r; ++u) {
+            double far = -INFINITY; int32_t farg = -1;
+            for (int32_t a = 0; a < nC; ++a) {
+                if (is_rep[a]) continue;
+                double nearest = INFINITY;
+                for (int32_t w = 0; w < u; ++w) {
+                    double dist = sqdist(keys + (int64_t)C[a] * d, keys + (int64_t)C[L[w]] * d, d);
+                    if (dist < nearest) nearest = dist;
+                }
+                if (nearest > far) { far = nearest; farg = a; }
+            }
+            L[u] = farg; is_rep[farg] = 1;
+        }
+        /* nearest-representative assignment, then representative self-ownership */
+        int32_t *b = (int32_t *)malloc(sizeof(int32_t) * (size_t)nC);
+        for (int32_t a = 0; a < nC; ++a) {
+            double nearest = INFINITY; int32_t owner = -1;
+            for (int32_t u = 0; u < r; ++u) {
+                double dist = sqdist(keys + (int64_t)C[a] * d, keys + (int64_t)C[L[u]] * d, d);
+                if (dist < nearest) { nearest = dist; owner = u; }
+            }
+            b[a] = owner;
+        }
+        for (int32_t u = 0; u < r; ++u) b[L[u]] = u;
+        /* emit the r teams of this parent */
+        for (int32_t u = 0; u < r; ++u) {
+            for (int32_t a = 0; a < nC; ++a)
+                if (b[a] == u) team_member[rows_out++] = C[a];
+            rep_row[M] = C[L[u]];
+            ++M;
+            team_start[M] = rows_out;
+        }
+        free(b); free(is_rep); free(L);
+    }
+    free(mu);
+    return M;
+}
+
+/* ------------------------------------------------------------------------- */
+/* Algorithm 1: SANTA++ attention for one query head                         */
+/* ------------------------------------------------------------------------- */
+
+typedef struct { double y; int32_t g; } orc_scored;
+
+/* Descending perturbed score; equal scores (a continuum-probability-zero event
+ * the paper does not order) go to the smaller team id. */
+static int cmp_scored(const void *pa, const void *pb)
+{
+    const orc_scored *a = (const orc_scored *)pa, *b = (const orc_scored *)pb;
+    if (a->y > b->y) return -1;
+    if (a->y < b->y) return 1;
+    return (a->g > b->g) - (a->g < b->g);
+}
+
+/*
+ * Inputs
+ *   q[d]; prompt rows k_cache/v_cache [N][d] in token order; team records as
+ *   CSR (team_start[M+1], team_member[*] token indices) plus the frozen
+ *   representative keys rep_key[M][d]; exact suffix ks/vs [t][d]; requested
+ *   team count K >= 1; the M Gumbel draws (unused when K >= M); scale = 1/sqrt(d).
+ * Outputs
+ *   o[d]          estimated attention output U^ / Z^
+ *   sel[Ke]       selected teams in descending perturbed score (Ke = min(K, M);
+ *                 0..M-1 in order when K >= M)
+ *   logc[Ke]      log of the conditional inclusion correction c_g (0 when K >= M)
+ *   tau_out       the (K+1)-st largest perturbed score (NaN when K >= M)
+ *   margin_out    Y_(K) - Y_(K+1), how far the draw is from a different set
+ *   phi_out[M], y_out[M]   routing logits and perturbed scores (nullable)
+ *   U_out[d], Z_out        the two unnormalised sums multiplied by e^{-shift}
+ *                          (nullable); shift = *shift_io if use_shift != 0,
+ *                          else the maximum corrected logit, written back
+ * Returns Ke.
+ */
+int32_t orc_decode_head_given_gumbel(
+    int d, const double *q,
+    int64_t N, const double *k_cache, const double *v_cache,
+    int32_t M, const int32_t *team_start, const int32_t *team_member, const double *rep_key,
+    int64_t t, const double *ks, const double *vs,
+    int32_t K, const double *gumbel, double scale,
+    double *o, int32_t *sel, double *logc, double *tau_out, double *margin_out,
+    double *phi_out, double *y_out, double *U_out, double *Z_out,
+    int use_shift, double *shift_io)
+{
+    (void)N;
+    int32_t Ke = K < M ? K : M;                         /* K <- min(K, M) */
+    double tau = NAN, margin = INFINITY;
+    double *c = (double *)malloc(sizeof(double) * (size_t)(Ke > 0 ? Ke : 1));
+    if (Ke == M) {
+        /* select every team with correction one; no draw is consumed */
+        for (int32_t g = 0; g < M; ++g) { sel[g] = g; c[g] = 1.0; }
+        if (phi_out || y_out)
+            for (int32_t g = 0; g < M; ++g) {
+                double n_g = (double)(team_start[g + 1] - team_start[g]);
+                double phi = log(n_g) + dot(q, rep_key + (int64_t)g * d, d) * scale;
+                if (phi_out) phi_out[g] = phi;
+                if (y_out) y_out[g] = NAN;
+            }
+    } else {
+        orc_scored *Y = (orc_scored *)malloc(sizeof(orc_scored) * (size_t)M);
+        double *phi = (double *)malloc(sizeof(double) * (size_t)M);
+        for (int32_t g = 0; g < M; ++g) {
+            double n_g = (double)(team_start[g + 1] - team_start[g]);
+            phi[g] = log(n_g) + dot(q, rep_key + (int64_t)g * d, d) * scale;   /* routing logit */
+            Y[g].y = phi[g] + gumbel[g];                                       /* perturbed score */
+            Y[g].g = g;
+            if (phi_out) phi_out[g] = phi[g];
+            if (y_out) y_out[g] = Y[g].y;
+        }
+        qsort(Y, (size_t)M, sizeof(orc_scored), cmp_scored);
+        for (int32_t a = 0; a < Ke; ++a) sel[a] = Y[a].g;      /* the K largest */
+        tau = Y[Ke].y;                                         /* the (K+1)-st largest */
+        margin = Y[Ke - 1].y - Y[Ke].y;
+        for (int32_t a = 0; a < Ke; ++a)
+            c[a] = -expm1(-exp(phi[sel[a]] - tau));            /* 1 - exp[-exp(phi - tau)] */
+        free(phi); free(Y);
+    }
+    for (int32_t a = 0; a < Ke; ++a) logc[a] = log(c[a]);
+
+    /* exact logits of every member of every selected team and of the suffix;
+     * one common shift so that the exponentials stay in range */
+    double shift;
+    if (use_shift) {
+        shift = *shift_io;
+    } else {
+        shift = -INFINITY;
+        for (int64_t i = 0; i < t; ++i) {
+            double s = dot(q, ks + i * d, d) * scale;
+            if (s > shift) shift = s;
+        }
+        for (int32_t a = 0; a < Ke; ++a) {
+            int32_t g = sel[a];
+            for (int32_t m = team_start[g]; m < team_start[g + 1]; ++m) {
+                double s = dot(q, k_cache + (int64_t)team_member[m] * d, d) * scale - logc[a];
+                if (s > shift) shift = s;
+            }
+        }
+        if (shift_io) *shift_io = shift;
+    }
+    double Zhat = 0.0;
+    double *Uhat = (double *)malloc(sizeof(double) * (size_t)d);
+    for (int j = 0; j < d; ++j) Uhat[j] = 0.0;
+    /* suffix rows: weight one */
+    for (int64_t i = 0; i < t; ++i) {
+        double a_i = exp(dot(q, ks + i * d, d) * scale - shift);
+        Zhat += a_i;
+        for (int j = 0; j < d; ++j) Uhat[j] += a_i * vs[i * d + j];
+    }
+    /* selected teams: team sums first, then divided by c_g */
+    double *Ug = (double *)malloc(sizeof(double) * (size_t)d);
+    for (int32_t a = 0; a < Ke; ++a) {
+        int32_t g = sel[a];
+        double Zg = 0.0;
+        for (int j = 0; j < d; ++j) Ug[j] = 0.0;
+        for (int32_t m = team_start[g]; m < team_start[g + 1]; ++m) {
+            int64_t i = team_member[m];
+            double a_i = exp(dot(q, k_cache + i * d, d) * scale - shift);
+            Zg += a_i;
+            for (int j = 0; j < d; ++j) Ug[j] += a_i * v_cache[i * d + j];
+        }
+        Zhat += Zg / c[a];
+        for (int j = 0; j < d; ++j) Uhat[j] += Ug[j] / c[a];
+    }
+    for (int j = 0; j < d; ++j) o[j] = Uhat[j] / Zhat;
+    if (U_out) for (int j = 0; j < d; ++j) U_out[j] = Uhat[j];
+    if (Z_out) *Z_out = Zhat;
+    if (tau_out) *tau_out = tau;
+    if (margin_out) *margin_out = margin;
+    free(Ug); free(Uhat); free(c);
+    return Ke;
+}
+
+/* Algorithm 1 with the Gumbel draws taken from the Philox stream keyed by
+ * (seed; step, head, stream). */
+int32_t orc_decode_head(
+    int d, const double *q,
+    int64_t N, const double *k_cache, const double *v_cache,
+    int32_t M, const int32_t *team_start, const int32_t *team_member, const double *rep_key,
+    int64_t t, const double *ks, const double *vs,
+    int32_t K, uint64_t seed, uint32_t step, uint32_t head, uint32_t stream, double scale,
+    double *o, int32_t *sel, double *logc, double *tau_out, double *margin_out)
+{
+    double *gumbel = (double *)malloc(sizeof(double) * (size_t)(M > 0 ? M : 1));
+    if (K < M) orc_gumbel_many(seed, step, head, stream, M, gumbel);
+    int32_t Ke = orc_decode_head_given_gumbel(d, q, N, k_cache, v_cache, M, team_start, team_member,
+                                              rep_key, t, ks, vs, K, gumbel, scale, o, sel, logc,
+                                              tau_out, margin_out, NULL, NULL, NULL, NULL, 0, NULL);
+    free(gumbel);
+    return Ke;
+}
+
+/*
+ * One decode step of one sequence under GQA: query head h uses KV head h / G
+ * (G = n_q_heads / n_kv_heads), shares that head's team records with its
+ * siblings, and samples on its own Philox counter. Buffers are per KV head,
+ * concatenated: k_cache/v_cache [n_kv][N][d], team_start [n_kv][M_max+1] with
+ * M[j] teams used, team_member [n_kv][N], rep_key [n_kv][M_max][d], suffix
+ * [n_kv][t][d]. Outputs per query head: o [n_q][d], sel/logc [n_q][K],
+ * tau/margin [n_q]. Heads are independent; OpenMP, when compiled in, runs
+ * them on separate threads without changing any result.
+ */
+void orc_decode_step(
+    int d, int32_t n_q, int32_t n_kv, const double *q /* [n_q][d] */,
+    int64_t N, const double *k_cache, const double *v_cache,
+    int32_t M_max, const int32_t *M, const int32_t *team_start, const int32_t *team_member,
+    const double *rep_key,
+    int64_t t, const double *ks, const double *vs,
+    int32_t K, uint64_t seed, uint32_t step, uint32_t stream, double scale,
+    double *o, int32_t *sel, double *logc, double *tau, double *margin, int32_t n_threads)
+{
+    int32_t G = n_q / n_kv;
+    (void)n_threads;
+#ifdef _OPENMP
+#pragma omp parallel for schedule(dynamic, 1) num_threads(n_threads > 0 ? n_threads : 1)
+#endif
+    for (int32_t h = 0; h < n_q; ++h) {
+        int32_t j = h / G;
+        orc_decode_head(d, q + (int64_t)h * d,
+                        N, k_cache + (int64_t)j * N * d, v_cache + (int64_t)j * N * d,
+                        M[j], team_start + (int64_t)j * (M_max + 1), team_member + (int64_t)j * N,
+                        rep_key + (int64_t)j * M_max * d,
+                        t, ks + (int64_t)j * t * d, vs + (int64_t)j * t * d,
+                        K, seed, step, (uint32_t)h, stream, scale,
+                        o + (int64_t)h * d, sel + (int64_t)h * K, logc + (int64_t)h * K,
+                        tau + h, margin + h);
+    }
+}
+
+/* Dense attention for every query head of one sequence (same buffer layout). */
+void orc_dense_step(
+    int d, int32_t n_q, int32_t n_kv, const double *q,
+    int64_t N, const double *k_cache, const double *v_cache,
+    int64_t t, const double *ks, const double *vs, double scale, double *o, int32_t n_threads)
+{
+    int32_t G = n_q / n_kv;
+    (void)n_threads;
+#ifdef _OPENMP
+#pragma omp parallel for schedule(dynamic, 1) num_threads(n_threads > 0 ? n_threads : 1)
+#endif
+    for (int32_t h = 0; h < n_q; ++h) {
+        int32_t j = h / G;
+        orc_dense_head_two(d, q + (int64_t)h * d,
+                           N, k_cache + (int64_t)j * N * d, v_cache + (int64_t)j * N * d,
+                           t, ks + (int64_t)j * t * d, vs + (int64_t)j * t * d, scale,
+                           o + (int64_t)h * d);
+    }
+}
+
+int32_t orc_has_openmp(void)
+{
+#ifdef _OPENMP
+    return 1;
+#else
+    return 0;
+#endif
+}
+
+/* ------------------------------------------------------------------------- */
+/* Accounting                                                                */
+/* ------------------------------------------------------------------------- */
+
+/* Eq. (method-budget): K = min{M, S / (P / R)}; R must divide P and P/R must
+ * divide S. Returns -1 when the divisibility rules fail. */
+int32_t orc_team_budget(int32_t M, int32_t S, int32_t P, int32_t R)
+{
+    if (P <= 0 || R <= 0 || S <= 0) return -1;
+    if (P % R != 0) return -1;
+    int32_t per = P / R;
+    if (S % per != 0) return -1;
+    int32_t K = S / per;
+    return K < M ? K : M;
+}
+
+/* Eq. (qwen-logical-access): for calls c with m_c representatives scanned,
+ * u_c distinct selected prompt rows (union over the heads of a KV head), e_c
+ * suffix rows and cache length N_c, KV% = 100 * sum[m + 2(u + e)] / sum[2 N].
+ * Arrays have n_calls entries. */
+double orc_logical_access_pct(int64_t n_calls, const int64_t *m, const int64_t *u,
+                              const int64_t *e, const int64_t *Ncache)
+{
+    double num = 0.0, den = 0.0;
+    for (int64_t c = 0; c < n_calls; ++c) {
+        num += (double)m[c] + 2.0 * ((double)u[c] + (double)e[c]);
+        den += 2.0 * (double)Ncache[c];
+    }
+    return 100.0 * num / den;
+}
+
+/* Number of distinct prompt rows read for one KV head: the union, over the
+ * n_heads query heads that share it, of the members of their selected teams. */
+int64_t orc_union_rows(int32_t M, const int32_t *team_start, int32_t n_heads, int32_t Ke,
+                       const int32_t *sel /* [n_heads][Ke] */)
+{
+    char *hit = (char *)calloc((size_t)(M > 0 ? M : 1), 1);
+    for (int32_t h = 0; h < n_heads; ++h)
+        for (int32_t a = 0; a < Ke; ++a) hit[sel[(int64_t)h * Ke + a]] = 1;
+    int64_t rows = 0;
+    for (int32_t g = 0; g < M; ++g)
+        if (hit[g]) rows += team_start[g + 1] - team_start[g];
+    free(hit);
+    return rows;
+}
+
+/* Bytes of keys and values a dense decode step streams for one layer:
+ * n_kv heads x N rows x d elements x (K and V) x bytes per element. */
+double orc_dense_kv_bytes(int64_t N, int32_t n_kv, int32_t d, int32_t bytes_per_el)
+{
+    return 2.0 * (double)n_kv * (double)N * (double)d * (double)bytes_per_el;
+}
