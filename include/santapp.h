@@ -1,0 +1,216 @@
+/*
+ * santapp.h — C ABI of the SANTA++ decode-attention library for NVIDIA B200 (sm_100a).
+ *
+ * Three operations, named after the paper's statement of the problem:
+ *
+ *   santapp_build_teams        once after prefill, per sequence and KV head: contiguous
+ *                              parent groups (Algorithm 4), actual-key representatives and
+ *                              nearest-representative teams (Algorithm 2), written out as a
+ *                              team-contiguous copy of K/V with CSR row offsets (the packed
+ *                              copy of the appendix "Triton decode kernels").
+ *   santapp_decode_attn        per generated token: SANTA++ attention for every query head
+ *                              (Algorithm 1) under the GQA rule of the Method section.
+ *   santapp_dense_decode_attn  full-cache attention, Eq. (method-attention), over the same
+ *                              buffers: the in-library dense baseline.
+ *
+ * Conventions
+ *   - "device" pointers address GPU global memory of the current device; "host" pointers
+ *     address CPU memory. The library allocates no device memory and keeps no state: the
+ *     caller owns every buffer, including workspaces, whose sizes come from the *_sizes /
+ *     *_workspace_bytes queries. Buffers must be 256-byte aligned.
+ *   - bf16 tensors are raw 16-bit patterns. head_dim is 128. Query head h uses KV head
+ *     h / (n_q_heads / n_kv_heads); at most 8 query heads per KV head.
+ *   - A batch holds n_seqs independent sequences of prompt length prompt_len[b] >= 1; prompt
+ *     rows of all sequences are concatenated: sequence b owns rows
+ *     [seq_row_off[b], seq_row_off[b+1]) of each KV head's plane.
+ *   - Team ids are local to a (sequence, KV head), numbered parent by parent and, inside a
+ *     parent, in representative-selection order (the emission order of Algorithm 2).
+ *   - Every call is asynchronous on `stream` (a cudaStream_t passed as void*; NULL is the
+ *     legacy default stream) and returns SANTAPP_OK or a negative santapp_status. No call
+ *     throws, aborts or traps. Argument errors are detected on the host before any launch.
+ *
+ * Random stream (the paper asks for independent Gumbel(0,1) draws; this is the library's
+ * realisation): Philox4x32-10 with key = (seed low 32 bits, seed high 32 bits) and counter
+ * (team_id / 4, step, query head index, stream_base + sequence index); team g takes word
+ * g mod 4; u = (word + 0.5) / 2^32; G = -log(-log u). The draw is a pure function of
+ * (seed, step, head, sequence stream, team), so a replayed step reproduces its sample.
+ */
+#ifndef SANTAPP_H
+#define SANTAPP_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum santapp_status {
+    SANTAPP_OK = 0,
+    SANTAPP_ERR_INVALID_ARG = -1,        /* null pointer, non-positive size, K < 1, R does not divide P, ... */
+    SANTAPP_ERR_UNSUPPORTED = -2,        /* head_dim != 128, group size > 8, parent_size > 512, too many teams */
+    SANTAPP_ERR_WORKSPACE_TOO_SMALL = -3,
+    SANTAPP_ERR_CUDA = -4                /* a CUDA runtime call or launch failed; see santapp_last_cuda_error */
+} santapp_status;
+
+typedef void *santapp_stream;            /* cudaStream_t */
+
+/* Problem geometry (host struct). */
+typedef struct santapp_geom {
+    int32_t n_seqs;            /* B: sequences in the batch                         */
+    int32_t n_q_heads;         /* Hq                                               */
+    int32_t n_kv_heads;        /* Hkv; must divide Hq                              */
+    int32_t head_dim;          /* d; 128                                           */
+    int32_t parent_size;       /* P: nominal parent size (Algorithm 4), <= 512      */
+    int32_t reps_per_parent;   /* R: maximum representatives per parent; divides P  */
+} santapp_geom;
+
+/* Sizes derived from the geometry and the prompt lengths (host struct, output). */
+typedef struct santapp_sizes {
+    int64_t rows_total;              /* sum_b prompt_len[b]                                          */
+    int64_t teams_total;             /* sum_b M_b, M_b = sum over parents of min(R, parent rows)     */
+    int32_t max_teams_per_seq;       /* max_b M_b                                                    */
+    int32_t max_rows_per_seq;        /* max_b prompt_len[b]                                          */
+    int64_t team_row_start_elems;    /* n_kv_heads * (teams_total + n_seqs) int32 elements           */
+    size_t build_workspace_bytes;    /* workspace santapp_build_teams needs                          */
+} santapp_sizes;
+
+/*
+ * Team records (Section "Preparing parent groups and teams"; packed layout of the appendix
+ * "Triton decode kernels"). All pointers are device pointers, caller-allocated. After
+ * santapp_build_teams they are immutable: memberships and representative keys stay fixed
+ * for the whole decode.
+ */
+typedef struct santapp_teams {
+    void *k_packed;            /* bf16 [n_kv_heads][rows_total][d]: each team's members occupy a
+                                  contiguous row range, teams in id order, members by token index   */
+    void *v_packed;            /* bf16, same layout                                                 */
+    void *rep_keys;            /* bf16 [n_kv_heads][teams_total][d]: frozen representative keys      */
+    int32_t *team_row_start;   /* int32 [n_kv_heads][teams_total + n_seqs]: for sequence b the
+                                  M_b + 1 CSR offsets start at element seq_team_off[b] + b; values
+                                  are row offsets local to the sequence (0 .. prompt_len[b])         */
+    int32_t *row_token;        /* int32 [n_kv_heads][rows_total]: prompt token index (local to its
+                                  sequence) of each packed row                                       */
+    int64_t *seq_row_off;      /* int64 [n_seqs + 1] device copy of the row offsets                  */
+    int64_t *seq_team_off;     /* int64 [n_seqs + 1] device copy of the team offsets                 */
+    int64_t rows_total;        /* host scalars, as in santapp_sizes                                  */
+    int64_t teams_total;
+    int32_t max_teams_per_seq;
+    int32_t max_rows_per_seq;
+} santapp_teams;
+
+/*
+ * Optional per-step diagnostics (device pointers, each may be NULL).
+ * With Ke = min(K, M_b): sel_idx/sel_logc hold Ke entries per head followed by -1 / 0 padding.
+ */
+typedef struct santapp_debug {
+    int32_t *sel_idx;          /* int32 [n_seqs][n_q_heads][K]: sampled team ids in descending
+                                  perturbed score; 0..M_b-1 when K >= M_b                            */
+    float *sel_logc;           /* fp32  [n_seqs][n_q_heads][K]: log c_g, Eq. (method-inclusion)      */
+    double *tau;               /* fp64  [n_seqs][n_q_heads]: (K+1)-st largest perturbed score; NaN
+                                  when K >= M_b                                                      */
+    int32_t *union_rows;       /* int32 [n_seqs][n_kv_heads]: distinct prompt rows read (u_c of the
+                                  logical-access counter)                                            */
+    int32_t *status;           /* int32 [1]: bit flags raised on the device (0 = clean);
+                                  bit 0: non-finite output                                           */
+} santapp_debug;
+
+/* Library version: major * 10000 + minor * 100 + patch. */
+int santapp_version(void);
+
+/* Text for a santapp_status value. The returned string is static. */
+const char *santapp_strerror(int status);
+
+/* Text of the last CUDA error a call on this thread ran into (static storage; "" if none). */
+const char *santapp_last_cuda_error(void);
+
+/*
+ * Sizes for a batch (Algorithm 4: sequence b has ceil(prompt_len[b] / P) parents; Algorithm 2:
+ * a parent of c rows yields min(R, c) teams).
+ *   geom             host, in
+ *   prompt_len_host  host int32 [n_seqs], in; every entry >= 1
+ *   out              host, out
+ */
+int santapp_build_teams_sizes(const santapp_geom *geom, const int32_t *prompt_len_host,
+                              santapp_sizes *out);
+
+/*
+ * Build the team records of one layer for every (sequence, KV head).
+ * Algorithm 4 (contiguous parents of P tokens, last one possibly short), then Algorithm 2 per
+ * parent: r = min(R, rows); first representative = the key nearest the parent mean; each later
+ * one = the key farthest from its nearest chosen representative; every key joins its nearest
+ * representative (squared Euclidean distance on the raw keys, evaluated in fp64); each
+ * representative owns its own row. Ties: representative choices go to the smaller token index,
+ * assignments to the earlier-selected representative.
+ *   k_prompt, v_prompt   device bf16 [n_kv_heads][rows_total][d], token order, in (not modified)
+ *   teams                host struct of device pointers, out: every array is overwritten; the
+ *                        host scalars are filled in
+ *   workspace            device, >= sizes.build_workspace_bytes; contents undefined afterwards
+ * The call copies the (n_seqs + 1)-entry offset tables to the device with cudaMemcpyAsync from
+ * pageable memory, which orders after prior work on `stream`; it is a preparation call, outside
+ * the per-token path.
+ */
+int santapp_build_teams(const santapp_geom *geom, const int32_t *prompt_len_host,
+                        const void *k_prompt, const void *v_prompt,
+                        santapp_teams *teams, void *workspace, size_t workspace_bytes,
+                        santapp_stream stream);
+
+/* Workspace bytes santapp_decode_attn needs for n_sample = K on these team records. */
+size_t santapp_decode_workspace_bytes(const santapp_geom *geom, const santapp_teams *teams,
+                                      int32_t n_sample);
+
+/*
+ * One decode step of SANTA++ attention for all sequences and query heads (Algorithm 1).
+ * Per query head h of sequence b, with the M_b teams of its KV head:
+ *   K <- min(n_sample, M_b). If K = M_b every team is read with c_g = 1 and nothing is drawn.
+ *   Otherwise phi_g = log n_g + q.l_g * scale (Eq. method-routing), Y_g = phi_g + Gumbel draw,
+ *   S = the K largest Y (ties to the smaller team id), tau = the (K+1)-st largest,
+ *   c_g = 1 - exp(-exp(phi_g - tau)) (Eq. method-inclusion); routing is evaluated in fp64.
+ *   out = U^ / Z^ of Eq. (method-estimate): every member of every selected team enters with
+ *   weight e^{s_i} / c_g, every suffix row with weight e^{s_i}, s_i = q.k_i * scale
+ *   (bf16 inputs, fp32 accumulation). Heads sharing a KV head sample independently; K/V rows
+ *   of the union of their selections are read once.
+ *   teams           host struct of device pointers, in
+ *   q               device bf16 [n_seqs][n_q_heads][d], in (unscaled, post-RoPE)
+ *   k_suffix,v_suffix device bf16 [n_seqs][n_kv_heads][suffix_cap][d], in: exact suffix of
+ *                   generated tokens; may be NULL when suffix_cap == 0
+ *   suffix_len_dev  device int32 [n_seqs], in: visible suffix rows per sequence (clamped to
+ *                   [0, suffix_cap]); NULL means 0 everywhere
+ *   n_sample        K >= 1
+ *   seed, step, stream_base   random-stream key and counters (see top of file)
+ *   scale           logit scale; 0 means 1 / sqrt(d)
+ *   out             device fp32 [n_seqs][n_q_heads][d], out
+ *   dbg             host struct of device pointers or NULL
+ *   workspace       device, >= santapp_decode_workspace_bytes(...); contents undefined on entry
+ *                   and on exit; must not be shared by calls that may overlap on the GPU
+ */
+int santapp_decode_attn(const santapp_geom *geom, const santapp_teams *teams, const void *q,
+                        const void *k_suffix, const void *v_suffix, const int32_t *suffix_len_dev,
+                        int32_t suffix_cap, int32_t n_sample, uint64_t seed, uint32_t step,
+                        uint32_t stream_base, float scale, float *out, const santapp_debug *dbg,
+                        void *workspace, size_t workspace_bytes, santapp_stream stream);
+
+/* Workspace bytes santapp_dense_decode_attn needs. */
+size_t santapp_dense_workspace_bytes(const santapp_geom *geom, const santapp_teams *teams);
+
+/*
+ * Dense decode attention, Eq. (method-attention), over all prompt rows (read from the packed
+ * copy; attention does not depend on row order) and the visible suffix, for all sequences and
+ * query heads. Arguments as in santapp_decode_attn.
+ */
+int santapp_dense_decode_attn(const santapp_geom *geom, const santapp_teams *teams, const void *q,
+                              const void *k_suffix, const void *v_suffix,
+                              const int32_t *suffix_len_dev, int32_t suffix_cap, float scale,
+                              float *out, void *workspace, size_t workspace_bytes,
+                              santapp_stream stream);
+
+/*
+ * Launch statistics of the most recent decode / dense call on this thread (host-side
+ * bookkeeping, no device access): number of kernels launched by that call.
+ */
+int santapp_last_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SANTAPP_H */

@@ -1,0 +1,272 @@
+"""ctypes binding of libsantapp.so: argument marshalling only.
+
+Every step of the path (team build, routing, sampling, exact attention, split-K
+merge) runs in the library's CUDA kernels. PyTorch is used for device memory and
+streams. There is no CPU fallback: if the library is missing or cannot be loaded
+the first call raises.
+
+The functions keep the names of the C entry points (include/santapp.h).
+"""
+import ctypes
+import os
+from dataclasses import dataclass
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libsantapp.so")
+
+SANTAPP_OK = 0
+SANTAPP_ERR_INVALID_ARG = -1
+SANTAPP_ERR_UNSUPPORTED = -2
+SANTAPP_ERR_WORKSPACE_TOO_SMALL = -3
+SANTAPP_ERR_CUDA = -4
+
+EXPORTS = [
+    "santapp_version", "santapp_strerror", "santapp_last_cuda_error", "santapp_build_teams_sizes",
+    "santapp_build_teams", "santapp_decode_workspace_bytes", "santapp_decode_attn",
+    "santapp_dense_workspace_bytes", "santapp_dense_decode_attn", "santapp_last_launch_count",
+]
+
+
+class SantappError(RuntimeError):
+    def __init__(self, status, detail=""):
+        self.status = status
+        super().__init__(f"santapp status {status}: {detail}")
+
+
+class CGeom(ctypes.Structure):
+    _fields_ = [("n_seqs", ctypes.c_int32), ("n_q_heads", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32),
+                ("head_dim", ctypes.c_int32), ("parent_size", ctypes.c_int32),
+                ("reps_per_parent", ctypes.c_int32)]
+
+
+class CSizes(ctypes.Structure):
+    _fields_ = [("rows_total", ctypes.c_int64), ("teams_total", ctypes.c_int64),
+                ("max_teams_per_seq", ctypes.c_int32), ("max_rows_per_seq", ctypes.c_int32),
+                ("team_row_start_elems", ctypes.c_int64), ("build_workspace_bytes", ctypes.c_size_t)]
+
+
+class CTeams(ctypes.Structure):
+    _fields_ = [("k_packed", ctypes.c_void_p), ("v_packed", ctypes.c_void_p), ("rep_keys", ctypes.c_void_p),
+                ("team_row_start", ctypes.c_void_p), ("row_token", ctypes.c_void_p),
+                ("seq_row_off", ctypes.c_void_p), ("seq_team_off", ctypes.c_void_p),
+                ("rows_total", ctypes.c_int64), ("teams_total", ctypes.c_int64),
+                ("max_teams_per_seq", ctypes.c_int32), ("max_rows_per_seq", ctypes.c_int32)]
+
+
+class CDebug(ctypes.Structure):
+    _fields_ = [("sel_idx", ctypes.c_void_p), ("sel_logc", ctypes.c_void_p), ("tau", ctypes.c_void_p),
+                ("union_rows", ctypes.c_void_p), ("status", ctypes.c_void_p)]
+
+
+_lib = None
+
+
+def load_library(path: Optional[str] = None):
+    """Load libsantapp.so and declare its signatures. Raises if it is missing."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    p = path or LIB_PATH
+    if not os.path.exists(p):
+        raise SantappError(SANTAPP_ERR_CUDA, f"{p} not found: build it with `python -m paper_2609_35629_b200.build` "
+                                             "(there is no CPU fallback)")
+    L = ctypes.CDLL(p)
+    vp, i32, u32, u64, f32, sz = (ctypes.c_void_p, ctypes.c_int32, ctypes.c_uint32, ctypes.c_uint64,
+                                  ctypes.c_float, ctypes.c_size_t)
+    L.santapp_version.restype = ctypes.c_int
+    L.santapp_strerror.argtypes = [ctypes.c_int]
+    L.santapp_strerror.restype = ctypes.c_char_p
+    L.santapp_last_cuda_error.restype = ctypes.c_char_p
+    L.santapp_last_launch_count.restype = ctypes.c_int
+    L.santapp_build_teams_sizes.argtypes = [ctypes.POINTER(CGeom), ctypes.POINTER(i32), ctypes.POINTER(CSizes)]
+    L.santapp_build_teams_sizes.restype = ctypes.c_int
+    L.santapp_build_teams.argtypes = [ctypes.POINTER(CGeom), ctypes.POINTER(i32), vp, vp,
+                                      ctypes.POINTER(CTeams), vp, sz, vp]
+    L.santapp_build_teams.restype = ctypes.c_int
+    L.santapp_decode_workspace_bytes.argtypes = [ctypes.POINTER(CGeom), ctypes.POINTER(CTeams), i32]
+    L.santapp_decode_workspace_bytes.restype = sz
+    L.santapp_dense_workspace_bytes.argtypes = [ctypes.POINTER(CGeom), ctypes.POINTER(CTeams)]
+    L.santapp_dense_workspace_bytes.restype = sz
+    L.santapp_decode_attn.argtypes = [ctypes.POINTER(CGeom), ctypes.POINTER(CTeams), vp, vp, vp, vp, i32, i32,
+                                      u64, u32, u32, f32, vp, ctypes.POINTER(CDebug), vp, sz, vp]
+    L.santapp_decode_attn.restype = ctypes.c_int
+    L.santapp_dense_decode_attn.argtypes = [ctypes.POINTER(CGeom), ctypes.POINTER(CTeams), vp, vp, vp, vp, i32,
+                                            f32, vp, vp, sz, vp]
+    L.santapp_dense_decode_attn.restype = ctypes.c_int
+    if path is None:
+        _lib = L
+    return L
+
+
+def _check(rc):
+    if rc != SANTAPP_OK:
+        L = load_library()
+        detail = L.santapp_strerror(rc).decode()
+        if rc == SANTAPP_ERR_CUDA:
+            detail += " — " + L.santapp_last_cuda_error().decode()
+        raise SantappError(rc, detail)
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    if t is None:
+        return None
+    if not t.is_cuda or not t.is_contiguous():
+        raise SantappError(SANTAPP_ERR_INVALID_ARG, "tensors must be contiguous CUDA tensors")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream_ptr(stream):
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+@dataclass
+class Geometry:
+    n_seqs: int
+    n_q_heads: int
+    n_kv_heads: int
+    head_dim: int = 128
+    parent_size: int = 512
+    reps_per_parent: int = 32
+
+    def c(self) -> CGeom:
+        return CGeom(self.n_seqs, self.n_q_heads, self.n_kv_heads, self.head_dim, self.parent_size,
+                     self.reps_per_parent)
+
+
+@dataclass
+class Sizes:
+    rows_total: int
+    teams_total: int
+    max_teams_per_seq: int
+    max_rows_per_seq: int
+    team_row_start_elems: int
+    build_workspace_bytes: int
+
+
+class Teams:
+    """Team records of one layer: device tensors plus the C struct that points at them."""
+
+    def __init__(self, geom: Geometry, sizes: Sizes, device):
+        d = geom.head_dim
+        kv = geom.n_kv_heads
+        self.geom = geom
+        self.sizes = sizes
+        self.k_packed = torch.empty((kv, sizes.rows_total, d), dtype=torch.bfloat16, device=device)
+        self.v_packed = torch.empty_like(self.k_packed)
+        self.rep_keys = torch.empty((kv, sizes.teams_total, d), dtype=torch.bfloat16, device=device)
+        self.team_row_start = torch.empty((kv, sizes.teams_total + geom.n_seqs), dtype=torch.int32, device=device)
+        self.row_token = torch.empty((kv, sizes.rows_total), dtype=torch.int32, device=device)
+        self.seq_row_off = torch.empty(geom.n_seqs + 1, dtype=torch.int64, device=device)
+        self.seq_team_off = torch.empty(geom.n_seqs + 1, dtype=torch.int64, device=device)
+        self.c = CTeams(self.k_packed.data_ptr(), self.v_packed.data_ptr(), self.rep_keys.data_ptr(),
+                        self.team_row_start.data_ptr(), self.row_token.data_ptr(),
+                        self.seq_row_off.data_ptr(), self.seq_team_off.data_ptr(),
+                        sizes.rows_total, sizes.teams_total, sizes.max_teams_per_seq, sizes.max_rows_per_seq)
+
+
+def santapp_version() -> int:
+    return load_library().santapp_version()
+
+
+def santapp_last_launch_count() -> int:
+    return load_library().santapp_last_launch_count()
+
+
+def santapp_build_teams_sizes(geom: Geometry, prompt_len) -> Sizes:
+    L = load_library()
+    n = len(prompt_len)
+    arr = (ctypes.c_int32 * n)(*[int(x) for x in prompt_len])
+    out = CSizes()
+    g = geom.c()
+    _check(L.santapp_build_teams_sizes(ctypes.byref(g), arr, ctypes.byref(out)))
+    return Sizes(out.rows_total, out.teams_total, out.max_teams_per_seq, out.max_rows_per_seq,
+                 out.team_row_start_elems, out.build_workspace_bytes)
+
+
+def santapp_build_teams(geom: Geometry, prompt_len, k_prompt: torch.Tensor, v_prompt: torch.Tensor,
+                        stream=None) -> Teams:
+    """k_prompt, v_prompt: bf16 CUDA tensors [n_kv_heads, rows_total, d] in token order."""
+    L = load_library()
+    sizes = santapp_build_teams_sizes(geom, prompt_len)
+    teams = Teams(geom, sizes, k_prompt.device)
+    ws = torch.empty(max(sizes.build_workspace_bytes, 256), dtype=torch.uint8, device=k_prompt.device)
+    n = len(prompt_len)
+    arr = (ctypes.c_int32 * n)(*[int(x) for x in prompt_len])
+    g = geom.c()
+    _check(L.santapp_build_teams(ctypes.byref(g), arr, _ptr(k_prompt), _ptr(v_prompt), ctypes.byref(teams.c),
+                                 _ptr(ws), ws.numel(), _stream_ptr(stream)))
+    teams._build_ws = ws      # keep alive until the stream has consumed it
+    return teams
+
+
+def santapp_decode_workspace_bytes(geom: Geometry, teams: Teams, n_sample: int) -> int:
+    g = geom.c()
+    return int(load_library().santapp_decode_workspace_bytes(ctypes.byref(g), ctypes.byref(teams.c), n_sample))
+
+
+def santapp_dense_workspace_bytes(geom: Geometry, teams: Teams) -> int:
+    g = geom.c()
+    return int(load_library().santapp_dense_workspace_bytes(ctypes.byref(g), ctypes.byref(teams.c)))
+
+
+class DebugBuffers:
+    """Optional per-step diagnostics (device tensors)."""
+
+    def __init__(self, geom: Geometry, n_sample: int, device):
+        B, Hq, Hkv = geom.n_seqs, geom.n_q_heads, geom.n_kv_heads
+        self.sel_idx = torch.full((B, Hq, n_sample), -1, dtype=torch.int32, device=device)
+        self.sel_logc = torch.zeros((B, Hq, n_sample), dtype=torch.float32, device=device)
+        self.tau = torch.zeros((B, Hq), dtype=torch.float64, device=device)
+        self.union_rows = torch.zeros((B, Hkv), dtype=torch.int32, device=device)
+        self.status = torch.zeros(1, dtype=torch.int32, device=device)
+        self.c = CDebug(self.sel_idx.data_ptr(), self.sel_logc.data_ptr(), self.tau.data_ptr(),
+                        self.union_rows.data_ptr(), self.status.data_ptr())
+
+
+def santapp_decode_attn(geom: Geometry, teams: Teams, q: torch.Tensor, k_suffix: Optional[torch.Tensor],
+                        v_suffix: Optional[torch.Tensor], suffix_len: Optional[torch.Tensor], n_sample: int,
+                        seed: int, step: int, stream_base: int = 0, scale: float = 0.0,
+                        out: Optional[torch.Tensor] = None, debug: Optional[DebugBuffers] = None,
+                        workspace: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """q bf16 [B, Hq, d]; k_suffix/v_suffix bf16 [B, Hkv, cap, d]; suffix_len int32 [B] (device)."""
+    L = load_library()
+    if out is None:
+        out = torch.empty((geom.n_seqs, geom.n_q_heads, geom.head_dim), dtype=torch.float32, device=q.device)
+    if workspace is None:
+        workspace = torch.empty(santapp_decode_workspace_bytes(geom, teams, n_sample), dtype=torch.uint8,
+                                device=q.device)
+    cap = 0 if k_suffix is None else int(k_suffix.shape[2])
+    g = geom.c()
+    _check(L.santapp_decode_attn(ctypes.byref(g), ctypes.byref(teams.c), _ptr(q), _ptr(k_suffix), _ptr(v_suffix),
+                                 _ptr(suffix_len), cap, n_sample, ctypes.c_uint64(seed), step, stream_base,
+                                 scale, _ptr(out), ctypes.byref(debug.c) if debug is not None else None,
+                                 _ptr(workspace), workspace.numel(), _stream_ptr(stream)))
+    return out
+
+
+def santapp_dense_decode_attn(geom: Geometry, teams: Teams, q: torch.Tensor, k_suffix: Optional[torch.Tensor],
+                              v_suffix: Optional[torch.Tensor], suffix_len: Optional[torch.Tensor],
+                              scale: float = 0.0, out: Optional[torch.Tensor] = None,
+                              workspace: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    L = load_library()
+    if out is None:
+        out = torch.empty((geom.n_seqs, geom.n_q_heads, geom.head_dim), dtype=torch.float32, device=q.device)
+    if workspace is None:
+        workspace = torch.empty(santapp_dense_workspace_bytes(geom, teams), dtype=torch.uint8, device=q.device)
+    cap = 0 if k_suffix is None else int(k_suffix.shape[2])
+    g = geom.c()
+    _check(L.santapp_dense_decode_attn(ctypes.byref(g), ctypes.byref(teams.c), _ptr(q), _ptr(k_suffix),
+                                       _ptr(v_suffix), _ptr(suffix_len), cap, scale, _ptr(out), _ptr(workspace),
+                                       workspace.numel(), _stream_ptr(stream)))
+    return out
+
+
+def bf16_bits_to_cuda(bits, device="cuda"):
+    """numpy uint16 bf16 bit patterns -> CUDA bfloat16 tensor (no value conversion)."""
+    import numpy as np
+    t = torch.from_numpy(np.ascontiguousarray(bits).view(np.int16))
+    return t.to(device).view(torch.bfloat16)

@@ -1,0 +1,386 @@
+// C ABI of the SANTA++ decode-attention library: argument checks, workspace carving, launches.
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <vector>
+
+#include "common.cuh"
+
+using namespace santapp;
+
+namespace {
+
+thread_local char g_cuda_error[256] = "";
+thread_local int g_launches = 0;
+
+int cuda_fail(cudaError_t err, const char *where)
+{
+    snprintf(g_cuda_error, sizeof(g_cuda_error), "%s: %s", where, cudaGetErrorString(err));
+    return SANTAPP_ERR_CUDA;
+}
+
+inline size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
+
+int check_geom(const santapp_geom *g)
+{
+    if (!g) return SANTAPP_ERR_INVALID_ARG;
+    if (g->n_seqs < 1 || g->n_q_heads < 1 || g->n_kv_heads < 1 || g->parent_size < 1 || g->reps_per_parent < 1)
+        return SANTAPP_ERR_INVALID_ARG;
+    if (g->n_q_heads % g->n_kv_heads != 0) return SANTAPP_ERR_INVALID_ARG;
+    if (g->parent_size % g->reps_per_parent != 0) return SANTAPP_ERR_INVALID_ARG;   // R divides P
+    if (g->head_dim != kHeadDim) return SANTAPP_ERR_UNSUPPORTED;
+    if (g->n_q_heads / g->n_kv_heads > kMaxGroup) return SANTAPP_ERR_UNSUPPORTED;
+    if (g->parent_size > kMaxParent) return SANTAPP_ERR_UNSUPPORTED;
+    return SANTAPP_OK;
+}
+
+int teams_in_sequence(int N, int P, int R)
+{
+    const int full = N / P, tail = N % P;
+    return full * (R < P ? R : P) + (tail ? (R < tail ? R : tail) : 0);
+}
+
+int check_teams(const santapp_geom *g, const santapp_teams *t)
+{
+    if (!t) return SANTAPP_ERR_INVALID_ARG;
+    if (!t->k_packed || !t->v_packed || !t->rep_keys || !t->team_row_start || !t->seq_row_off || !t->seq_team_off)
+        return SANTAPP_ERR_INVALID_ARG;
+    if (t->rows_total < g->n_seqs || t->teams_total < g->n_seqs || t->max_teams_per_seq < 1)
+        return SANTAPP_ERR_INVALID_ARG;
+    if (t->rows_total >= (int64_t)1 << 31) return SANTAPP_ERR_UNSUPPORTED;
+    if (t->max_teams_per_seq > kMaxTeamsPerSeq) return SANTAPP_ERR_UNSUPPORTED;
+    return SANTAPP_OK;
+}
+
+BatchView make_view(const santapp_geom *g, const santapp_teams *t)
+{
+    BatchView bv;
+    bv.n_seqs = g->n_seqs;
+    bv.n_q = g->n_q_heads;
+    bv.n_kv = g->n_kv_heads;
+    bv.group = g->n_q_heads / g->n_kv_heads;
+    bv.seq_row_off = t->seq_row_off;
+    bv.seq_team_off = t->seq_team_off;
+    bv.rows_total = t->rows_total;
+    bv.teams_total = t->teams_total;
+    return bv;
+}
+
+// Workspace layout shared by the sparse and the dense call. Offsets in bytes.
+struct DecodeLayout {
+    size_t ctl, y, sel_team, sel_logc, tau, seg_prefix, seg_row, seg_mask, seg_logc, pair_nseg, pair_rows,
+        pair_union, pair_prefix, partials, total;
+    int seg_cap, grid, n_pairs;
+};
+
+DecodeLayout decode_layout(const santapp_geom *g, const santapp_teams *t, int K, bool dense, int grid)
+{
+    DecodeLayout L;
+    const int G = g->n_q_heads / g->n_kv_heads;
+    L.n_pairs = g->n_seqs * g->n_kv_heads;
+    L.grid = grid;
+    int64_t cap = dense ? 1 : (int64_t)G * K;
+    if (cap > t->max_teams_per_seq) cap = t->max_teams_per_seq;
+    L.seg_cap = (int)cap + 1;                                   // + the suffix segment
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
+    L.ctl = take(sizeof(int32_t) * (2 * (size_t)L.n_pairs + 2));
+    L.y = take(dense ? 0 : sizeof(double) * (size_t)g->n_q_heads * (size_t)t->teams_total);
+    L.sel_team = take(dense ? 0 : sizeof(int32_t) * (size_t)g->n_seqs * g->n_q_heads * K);
+    L.sel_logc = take(dense ? 0 : sizeof(float) * (size_t)g->n_seqs * g->n_q_heads * K);
+    L.tau = take(dense ? 0 : sizeof(double) * (size_t)g->n_seqs * g->n_q_heads);
+    L.seg_prefix = take(sizeof(int32_t) * (size_t)L.n_pairs * (L.seg_cap + 1));
+    L.seg_row = take(sizeof(int32_t) * (size_t)L.n_pairs * L.seg_cap);
+    L.seg_mask = take(sizeof(uint32_t) * (size_t)L.n_pairs * L.seg_cap);
+    L.seg_logc = take(sizeof(float) * (size_t)L.n_pairs * L.seg_cap * G);
+    L.pair_nseg = take(sizeof(int32_t) * (size_t)L.n_pairs);
+    L.pair_rows = take(sizeof(int32_t) * (size_t)L.n_pairs);
+    L.pair_union = take(sizeof(int32_t) * (size_t)L.n_pairs);
+    L.pair_prefix = take(sizeof(int64_t) * ((size_t)L.n_pairs + 1));
+    L.partials = take(sizeof(float) * ((size_t)grid + L.n_pairs) * G * kPartialStride);
+    L.total = off;
+    return L;
+}
+
+void fill_plan(const DecodeLayout &L, char *ws, PlanView &plan, Control &ctl)
+{
+    int32_t *c = reinterpret_cast<int32_t *>(ws + L.ctl);
+    ctl.select_ticket = c;
+    ctl.attend_ticket = c + L.n_pairs;
+    ctl.plan_ticket = c + 2 * L.n_pairs;
+    plan.seg_cap = L.seg_cap;
+    plan.seg_prefix = reinterpret_cast<int32_t *>(ws + L.seg_prefix);
+    plan.seg_row = reinterpret_cast<int32_t *>(ws + L.seg_row);
+    plan.seg_mask = reinterpret_cast<uint32_t *>(ws + L.seg_mask);
+    plan.seg_logc = reinterpret_cast<float *>(ws + L.seg_logc);
+    plan.pair_nseg = reinterpret_cast<int32_t *>(ws + L.pair_nseg);
+    plan.pair_rows = reinterpret_cast<int32_t *>(ws + L.pair_rows);
+    plan.pair_union_rows = reinterpret_cast<int32_t *>(ws + L.pair_union);
+    plan.pair_row_prefix = reinterpret_cast<int64_t *>(ws + L.pair_prefix);
+}
+
+}  // namespace
+
+extern "C" {
+
+int santapp_version(void) { return 100; }
+
+const char *santapp_strerror(int status)
+{
+    switch (status) {
+        case SANTAPP_OK: return "ok";
+        case SANTAPP_ERR_INVALID_ARG: return "invalid argument";
+        case SANTAPP_ERR_UNSUPPORTED: return "unsupported configuration";
+        case SANTAPP_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+        case SANTAPP_ERR_CUDA: return "CUDA error";
+        default: return "unknown status";
+    }
+}
+
+const char *santapp_last_cuda_error(void) { return g_cuda_error; }
+
+int santapp_last_launch_count(void) { return g_launches; }
+
+int santapp_build_teams_sizes(const santapp_geom *geom, const int32_t *prompt_len_host, santapp_sizes *out)
+{
+    int rc = check_geom(geom);
+    if (rc != SANTAPP_OK) return rc;
+    if (!prompt_len_host || !out) return SANTAPP_ERR_INVALID_ARG;
+    memset(out, 0, sizeof(*out));
+    for (int b = 0; b < geom->n_seqs; ++b) {
+        const int N = prompt_len_host[b];
+        if (N < 1) return SANTAPP_ERR_INVALID_ARG;
+        const int M = teams_in_sequence(N, geom->parent_size, geom->reps_per_parent);
+        out->rows_total += N;
+        out->teams_total += M;
+        if (M > out->max_teams_per_seq) out->max_teams_per_seq = M;
+        if (N > out->max_rows_per_seq) out->max_rows_per_seq = N;
+    }
+    if (out->rows_total >= (int64_t)1 << 31) return SANTAPP_ERR_UNSUPPORTED;
+    out->team_row_start_elems = (int64_t)geom->n_kv_heads * (out->teams_total + geom->n_seqs);
+    out->build_workspace_bytes = align_up(sizeof(uint16_t) * (size_t)geom->n_kv_heads * (size_t)out->rows_total);
+    return SANTAPP_OK;
+}
+
+int santapp_build_teams(const santapp_geom *geom, const int32_t *prompt_len_host, const void *k_prompt,
+                        const void *v_prompt, santapp_teams *teams, void *workspace, size_t workspace_bytes,
+                        santapp_stream stream)
+{
+    santapp_sizes sz;
+    int rc = santapp_build_teams_sizes(geom, prompt_len_host, &sz);
+    if (rc != SANTAPP_OK) return rc;
+    if (!k_prompt || !v_prompt || !teams || !workspace) return SANTAPP_ERR_INVALID_ARG;
+    if (!teams->k_packed || !teams->v_packed || !teams->rep_keys || !teams->team_row_start || !teams->row_token
+        || !teams->seq_row_off || !teams->seq_team_off)
+        return SANTAPP_ERR_INVALID_ARG;
+    if (workspace_bytes < sz.build_workspace_bytes) return SANTAPP_ERR_WORKSPACE_TOO_SMALL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    g_cuda_error[0] = 0;
+
+    std::vector<int64_t> offs(2 * ((size_t)geom->n_seqs + 1));
+    int64_t *row_off = offs.data(), *team_off = offs.data() + geom->n_seqs + 1;
+    row_off[0] = team_off[0] = 0;
+    int max_parents = 0;
+    for (int b = 0; b < geom->n_seqs; ++b) {
+        const int N = prompt_len_host[b];
+        row_off[b + 1] = row_off[b] + N;
+        team_off[b + 1] = team_off[b] + teams_in_sequence(N, geom->parent_size, geom->reps_per_parent);
+        const int parents = (N + geom->parent_size - 1) / geom->parent_size;
+        if (parents > max_parents) max_parents = parents;
+    }
+    const size_t ob = sizeof(int64_t) * ((size_t)geom->n_seqs + 1);
+    cudaError_t err = cudaMemcpyAsync(teams->seq_row_off, row_off, ob, cudaMemcpyHostToDevice, s);
+    if (err != cudaSuccess) return cuda_fail(err, "copy seq_row_off");
+    err = cudaMemcpyAsync(teams->seq_team_off, team_off, ob, cudaMemcpyHostToDevice, s);
+    if (err != cudaSuccess) return cuda_fail(err, "copy seq_team_off");
+
+    teams->rows_total = sz.rows_total;
+    teams->teams_total = sz.teams_total;
+    teams->max_teams_per_seq = sz.max_teams_per_seq;
+    teams->max_rows_per_seq = sz.max_rows_per_seq;
+
+    BuildParams p;
+    p.bv = make_view(geom, teams);
+    p.parent_size = geom->parent_size;
+    p.reps = geom->reps_per_parent;
+    p.teams_per_full_parent = geom->reps_per_parent < geom->parent_size ? geom->reps_per_parent : geom->parent_size;
+    p.k_prompt = static_cast<const uint16_t *>(k_prompt);
+    p.v_prompt = static_cast<const uint16_t *>(v_prompt);
+    p.k_packed = static_cast<uint16_t *>(teams->k_packed);
+    p.v_packed = static_cast<uint16_t *>(teams->v_packed);
+    p.rep_keys = static_cast<uint16_t *>(teams->rep_keys);
+    p.team_row_start = teams->team_row_start;
+    p.row_token = teams->row_token;
+    p.owner = static_cast<uint16_t *>(workspace);
+    p.max_parents_per_seq = max_parents;
+    err = launch_build_teams(p, s);
+    if (err != cudaSuccess) return cuda_fail(err, "build_teams launch");
+    return SANTAPP_OK;
+}
+
+size_t santapp_decode_workspace_bytes(const santapp_geom *geom, const santapp_teams *teams, int32_t n_sample)
+{
+    if (check_geom(geom) != SANTAPP_OK || !teams || n_sample < 1 || n_sample > 256) return 0;
+    return decode_layout(geom, teams, n_sample, false, attend_grid_size()).total;
+}
+
+size_t santapp_dense_workspace_bytes(const santapp_geom *geom, const santapp_teams *teams)
+{
+    if (check_geom(geom) != SANTAPP_OK || !teams) return 0;
+    return decode_layout(geom, teams, 1, true, attend_grid_size()).total;
+}
+
+int santapp_decode_attn(const santapp_geom *geom, const santapp_teams *teams, const void *q, const void *k_suffix,
+                        const void *v_suffix, const int32_t *suffix_len_dev, int32_t suffix_cap, int32_t n_sample,
+                        uint64_t seed, uint32_t step, uint32_t stream_base, float scale, float *out,
+                        const santapp_debug *dbg, void *workspace, size_t workspace_bytes, santapp_stream stream)
+{
+    g_launches = 0;
+    int rc = check_geom(geom);
+    if (rc != SANTAPP_OK) return rc;
+    if ((rc = check_teams(geom, teams)) != SANTAPP_OK) return rc;
+    if (!q || !out || !workspace) return SANTAPP_ERR_INVALID_ARG;
+    if (n_sample < 1 || suffix_cap < 0) return SANTAPP_ERR_INVALID_ARG;
+    if (n_sample > 256) return SANTAPP_ERR_UNSUPPORTED;
+    if (suffix_cap > 0 && suffix_len_dev && (!k_suffix || !v_suffix)) return SANTAPP_ERR_INVALID_ARG;
+    if (!(scale >= 0.f) || isinf(scale)) return SANTAPP_ERR_INVALID_ARG;
+    if ((int64_t)geom->n_seqs * geom->n_kv_heads * (int64_t)suffix_cap >= (int64_t)1 << 31) return SANTAPP_ERR_UNSUPPORTED;
+    const int grid = attend_grid_size();
+    const DecodeLayout L = decode_layout(geom, teams, n_sample, false, grid);
+    if (workspace_bytes < L.total) return SANTAPP_ERR_WORKSPACE_TOO_SMALL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    g_cuda_error[0] = 0;
+    char *ws = static_cast<char *>(workspace);
+    const double sc = scale == 0.f ? 1.0 / sqrt((double)geom->head_dim) : (double)scale;
+
+    PlanView plan;
+    Control ctl;
+    fill_plan(L, ws, plan, ctl);
+
+    RouteParams rp;
+    rp.bv = make_view(geom, teams);
+    rp.rep_keys = static_cast<const uint16_t *>(teams->rep_keys);
+    rp.team_row_start = teams->team_row_start;
+    rp.q = static_cast<const uint16_t *>(q);
+    rp.y = reinterpret_cast<double *>(ws + L.y);
+    rp.n_sample = n_sample;
+    rp.seed_lo = (uint32_t)(seed & 0xFFFFFFFFull);
+    rp.seed_hi = (uint32_t)(seed >> 32);
+    rp.step = step;
+    rp.stream_base = stream_base;
+    rp.scale = sc;
+    rp.ctl = ctl;
+    rp.n_pairs = L.n_pairs;
+    rp.status = dbg ? dbg->status : nullptr;
+    cudaError_t err = launch_route_score(rp, teams->max_teams_per_seq, s);
+    if (err != cudaSuccess) return cuda_fail(err, "route_score launch");
+    ++g_launches;
+
+    SelectParams sp;
+    sp.bv = rp.bv;
+    sp.team_row_start = teams->team_row_start;
+    sp.y = rp.y;
+    sp.n_sample = n_sample;
+    sp.seed_lo = rp.seed_lo;
+    sp.seed_hi = rp.seed_hi;
+    sp.step = step;
+    sp.stream_base = stream_base;
+    sp.sel_team = reinterpret_cast<int32_t *>(ws + L.sel_team);
+    sp.sel_logc = reinterpret_cast<float *>(ws + L.sel_logc);
+    sp.tau = reinterpret_cast<double *>(ws + L.tau);
+    sp.suffix_len = suffix_len_dev;
+    sp.suffix_cap = suffix_cap;
+    sp.plan = plan;
+    sp.ctl = ctl;
+    sp.n_pairs = L.n_pairs;
+    sp.dbg_sel_idx = dbg ? dbg->sel_idx : nullptr;
+    sp.dbg_sel_logc = dbg ? dbg->sel_logc : nullptr;
+    sp.dbg_tau = dbg ? dbg->tau : nullptr;
+    sp.dbg_union_rows = dbg ? dbg->union_rows : nullptr;
+    err = launch_select_plan(sp, teams->max_teams_per_seq, s);
+    if (err != cudaSuccess) return cuda_fail(err, "select_plan launch");
+    ++g_launches;
+
+    AttendParams ap;
+    ap.bv = rp.bv;
+    ap.k_packed = static_cast<const uint16_t *>(teams->k_packed);
+    ap.v_packed = static_cast<const uint16_t *>(teams->v_packed);
+    ap.k_suffix = static_cast<const uint16_t *>(k_suffix);
+    ap.v_suffix = static_cast<const uint16_t *>(v_suffix);
+    ap.q = rp.q;
+    ap.qk_scale_log2 = (float)(sc * 1.4426950408889634);
+    ap.plan = plan;
+    ap.ctl = ctl;
+    ap.n_pairs = L.n_pairs;
+    ap.partials = reinterpret_cast<float *>(ws + L.partials);
+    ap.out = out;
+    ap.status = rp.status;
+    ap.min_rows_per_cta = 64;
+    err = launch_attend(ap, false, grid, s);
+    if (err != cudaSuccess) return cuda_fail(err, "attend launch");
+    ++g_launches;
+    return SANTAPP_OK;
+}
+
+int santapp_dense_decode_attn(const santapp_geom *geom, const santapp_teams *teams, const void *q,
+                              const void *k_suffix, const void *v_suffix, const int32_t *suffix_len_dev,
+                              int32_t suffix_cap, float scale, float *out, void *workspace, size_t workspace_bytes,
+                              santapp_stream stream)
+{
+    g_launches = 0;
+    int rc = check_geom(geom);
+    if (rc != SANTAPP_OK) return rc;
+    if ((rc = check_teams(geom, teams)) != SANTAPP_OK) return rc;
+    if (!q || !out || !workspace) return SANTAPP_ERR_INVALID_ARG;
+    if (suffix_cap < 0) return SANTAPP_ERR_INVALID_ARG;
+    if (suffix_cap > 0 && suffix_len_dev && (!k_suffix || !v_suffix)) return SANTAPP_ERR_INVALID_ARG;
+    if (!(scale >= 0.f) || isinf(scale)) return SANTAPP_ERR_INVALID_ARG;
+    if ((int64_t)geom->n_seqs * geom->n_kv_heads * (int64_t)suffix_cap >= (int64_t)1 << 31) return SANTAPP_ERR_UNSUPPORTED;
+    const int grid = attend_grid_size();
+    const DecodeLayout L = decode_layout(geom, teams, 1, true, grid);
+    if (workspace_bytes < L.total) return SANTAPP_ERR_WORKSPACE_TOO_SMALL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    g_cuda_error[0] = 0;
+    char *ws = static_cast<char *>(workspace);
+    const double sc = scale == 0.f ? 1.0 / sqrt((double)geom->head_dim) : (double)scale;
+
+    PlanView plan;
+    Control ctl;
+    fill_plan(L, ws, plan, ctl);
+
+    SelectParams sp;
+    memset(&sp, 0, sizeof(sp));
+    sp.bv = make_view(geom, teams);
+    sp.team_row_start = teams->team_row_start;
+    sp.suffix_len = suffix_len_dev;
+    sp.suffix_cap = suffix_cap;
+    sp.plan = plan;
+    sp.ctl = ctl;
+    sp.n_pairs = L.n_pairs;
+    cudaError_t err = launch_dense_plan(sp, s);
+    if (err != cudaSuccess) return cuda_fail(err, "dense_plan launch");
+    ++g_launches;
+
+    AttendParams ap;
+    ap.bv = sp.bv;
+    ap.k_packed = static_cast<const uint16_t *>(teams->k_packed);
+    ap.v_packed = static_cast<const uint16_t *>(teams->v_packed);
+    ap.k_suffix = static_cast<const uint16_t *>(k_suffix);
+    ap.v_suffix = static_cast<const uint16_t *>(v_suffix);
+    ap.q = static_cast<const uint16_t *>(q);
+    ap.qk_scale_log2 = (float)(sc * 1.4426950408889634);
+    ap.plan = plan;
+    ap.ctl = ctl;
+    ap.n_pairs = L.n_pairs;
+    ap.partials = reinterpret_cast<float *>(ws + L.partials);
+    ap.out = out;
+    ap.status = nullptr;
+    ap.min_rows_per_cta = 64;
+    err = launch_attend(ap, true, grid, s);
+    if (err != cudaSuccess) return cuda_fail(err, "attend launch");
+    ++g_launches;
+    return SANTAPP_OK;
+}
+
+}  // extern "C"

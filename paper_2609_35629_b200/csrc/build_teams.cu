@@ -1,0 +1,276 @@
+// santapp_build_teams: contiguous parents (Algorithm 4) and actual-key teams (Algorithm 2),
+// written as a team-contiguous copy of K/V with CSR offsets. Preparation path, run once after
+// prefill; distances are evaluated in fp64 in a fixed order (token index, then dimension) with
+// separate multiply and add, so that exact ties fall the way the paper's tie rules say.
+#include <limits.h>
+
+#include "common.cuh"
+
+namespace santapp {
+
+namespace {
+
+constexpr int kBuildThreads = 256;
+constexpr int kRowWords = 65;            // 64 data words + 1 pad word: conflict-free column walks
+
+struct ValIdx {
+    double v;
+    int i;
+};
+
+template <bool kMin>
+__device__ __forceinline__ ValIdx pick(const ValIdx &a, const ValIdx &b)
+{
+    bool take_b;
+    if (kMin) take_b = (b.v < a.v) || (b.v == a.v && b.i < a.i);
+    else      take_b = (b.v > a.v) || (b.v == a.v && b.i < a.i);
+    return take_b ? b : a;
+}
+
+// Block-wide arg-min / arg-max; ties go to the smaller index. Result valid in every thread.
+template <bool kMin>
+__device__ ValIdx block_arg(ValIdx x, ValIdx *scratch /* [33] */)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        ValIdx y;
+        y.v = __shfl_xor_sync(0xFFFFFFFFu, x.v, o);
+        y.i = __shfl_xor_sync(0xFFFFFFFFu, x.i, o);
+        x = pick<kMin>(x, y);
+    }
+    __syncthreads();
+    if (lane == 0) scratch[warp] = x;
+    __syncthreads();
+    if (warp == 0) {
+        ValIdx y = scratch[lane < n_warps ? lane : 0];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            ValIdx z;
+            z.v = __shfl_xor_sync(0xFFFFFFFFu, y.v, o);
+            z.i = __shfl_xor_sync(0xFFFFFFFFu, y.i, o);
+            y = pick<kMin>(y, z);
+        }
+        if (lane == 0) scratch[32] = y;
+    }
+    __syncthreads();
+    return scratch[32];
+}
+
+// Squared distance between row `i` (shared memory, bf16 words) and a reference vector in fp64,
+// summed over dimensions in increasing order, multiply and add rounded separately.
+__device__ __forceinline__ double sqdist_row_vec(const uint32_t *row, const double *ref)
+{
+    double s = 0.0;
+#pragma unroll 8
+    for (int w = 0; w < 64; ++w) {
+        const uint32_t word = row[w];
+        const double e0 = __dsub_rn((double)bf16_lo(word), ref[2 * w]);
+        const double e1 = __dsub_rn((double)bf16_hi(word), ref[2 * w + 1]);
+        s = __dadd_rn(s, __dmul_rn(e0, e0));
+        s = __dadd_rn(s, __dmul_rn(e1, e1));
+    }
+    return s;
+}
+
+__device__ __forceinline__ double sqdist_row_row(const uint32_t *row, const uint32_t *ref)
+{
+    double s = 0.0;
+#pragma unroll 8
+    for (int w = 0; w < 64; ++w) {
+        const uint32_t a = row[w], b = ref[w];
+        const double e0 = __dsub_rn((double)bf16_lo(a), (double)bf16_lo(b));
+        const double e1 = __dsub_rn((double)bf16_hi(a), (double)bf16_hi(b));
+        s = __dadd_rn(s, __dmul_rn(e0, e0));
+        s = __dadd_rn(s, __dmul_rn(e1, e1));
+    }
+    return s;
+}
+
+// One block per (parent, sequence, KV head): representatives, owners, team sizes.
+__global__ void __launch_bounds__(kBuildThreads)
+build_parent_kernel(BuildParams p)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const int parent = blockIdx.x, b = blockIdx.y, j = blockIdx.z;
+    const int64_t row0 = p.bv.seq_row_off[b];
+    const int N = (int)(p.bv.seq_row_off[b + 1] - row0);
+    const int P = p.parent_size;
+    const int first = parent * P;
+    if (first >= N) return;
+    const int nC = min(P, N - first);
+    const int r = min(p.reps, nC);
+    const int tid = threadIdx.x;
+
+    double *mu = reinterpret_cast<double *>(smem_raw);                    // [128]
+    double *mind = mu + kHeadDim;                                         // [P]
+    ValIdx *scratch = reinterpret_cast<ValIdx *>(mind + P);               // [33]
+    uint32_t *rows = reinterpret_cast<uint32_t *>(scratch + 33);          // [P][kRowWords]
+    int *owner = reinterpret_cast<int *>(rows + (size_t)P * kRowWords);   // [P]
+    int *count = owner + P;                                               // [P] (r used)
+    int *rep_of = count + P;                                              // [P] (r used): row inside parent
+    unsigned char *is_rep = reinterpret_cast<unsigned char *>(rep_of + P);  // [P]
+
+    const uint32_t *src = reinterpret_cast<const uint32_t *>(p.k_prompt)
+                          + ((size_t)j * p.bv.rows_total + row0 + first) * 64;
+    for (int e = tid; e < nC * 64; e += kBuildThreads) rows[(e >> 6) * kRowWords + (e & 63)] = src[e];
+    for (int i = tid; i < nC; i += kBuildThreads) { is_rep[i] = 0; count[i] = 0; }
+    __syncthreads();
+
+    // parent mean: rows added in token order, then one division
+    if (tid < kHeadDim) {
+        double s = 0.0;
+        const int w = tid >> 1;
+        const bool hi = tid & 1;
+        for (int i = 0; i < nC; ++i) {
+            const uint32_t word = rows[i * kRowWords + w];
+            s = __dadd_rn(s, (double)(hi ? bf16_hi(word) : bf16_lo(word)));
+        }
+        mu[tid] = __ddiv_rn(s, (double)nC);
+    }
+    __syncthreads();
+
+    // first representative: the actual key nearest the mean
+    {
+        ValIdx best = {INFINITY, INT_MAX};
+        for (int i = tid; i < nC; i += kBuildThreads) {
+            ValIdx c = {sqdist_row_vec(rows + i * kRowWords, mu), i};
+            best = pick<true>(best, c);
+        }
+        best = block_arg<true>(best, scratch);
+        if (tid == 0) { rep_of[0] = best.i; is_rep[best.i] = 1; }
+    }
+    __syncthreads();
+
+    // farthest-first representatives; the running (nearest distance, owner) pair is the
+    // nearest-representative assignment with ties going to the earlier-selected one
+    for (int i = tid; i < nC; i += kBuildThreads) { mind[i] = INFINITY; owner[i] = 0; }
+    for (int u = 0; u < r; ++u) {
+        const uint32_t *ref = rows + rep_of[u] * kRowWords;
+        ValIdx far = {-2.0, INT_MAX};
+        for (int i = tid; i < nC; i += kBuildThreads) {
+            const double dist = sqdist_row_row(rows + i * kRowWords, ref);
+            if (dist < mind[i]) { mind[i] = dist; owner[i] = u; }
+            ValIdx c = {is_rep[i] ? -1.0 : mind[i], i};
+            far = pick<false>(far, c);
+        }
+        if (u + 1 < r) {
+            far = block_arg<false>(far, scratch);
+            if (tid == 0) { rep_of[u + 1] = far.i; is_rep[far.i] = 1; }
+            __syncthreads();
+        }
+    }
+    __syncthreads();
+    // representative self-ownership
+    for (int u = tid; u < r; u += kBuildThreads) owner[rep_of[u]] = u;
+    __syncthreads();
+
+    for (int i = tid; i < nC; i += kBuildThreads) atomicAdd(&count[owner[i]], 1);
+    __syncthreads();
+
+    // outputs: owner per row, team sizes (scanned later), representative keys
+    uint16_t *owner_out = p.owner + (size_t)j * p.bv.rows_total + row0 + first;
+    for (int i = tid; i < nC; i += kBuildThreads) owner_out[i] = (uint16_t)owner[i];
+
+    const int64_t team0 = p.bv.seq_team_off[b];
+    const int team_local0 = parent * p.teams_per_full_parent;
+    int32_t *csr = p.team_row_start + (size_t)j * (p.bv.teams_total + p.bv.n_seqs) + team0 + b;
+    if (parent == 0 && tid == 0) csr[0] = 0;
+    for (int u = tid; u < r; u += kBuildThreads) csr[1 + team_local0 + u] = count[u];
+
+    uint32_t *rep_dst = reinterpret_cast<uint32_t *>(p.rep_keys)
+                        + ((size_t)j * p.bv.teams_total + team0 + team_local0) * 64;
+    for (int e = tid; e < r * 64; e += kBuildThreads)
+        rep_dst[e] = rows[rep_of[e >> 6] * kRowWords + (e & 63)];
+}
+
+// One block per (sequence, KV head): team sizes -> CSR row offsets (inclusive scan in place).
+__global__ void __launch_bounds__(kBuildThreads)
+scan_team_sizes_kernel(BuildParams p)
+{
+    __shared__ int scratch[33];
+    const int b = blockIdx.x, j = blockIdx.y;
+    const int64_t team0 = p.bv.seq_team_off[b];
+    const int M = (int)(p.bv.seq_team_off[b + 1] - team0);
+    int32_t *csr = p.team_row_start + (size_t)j * (p.bv.teams_total + p.bv.n_seqs) + team0 + b + 1;
+    int carry = 0;
+    for (int base = 0; base < M; base += kBuildThreads) {
+        const int g = base + threadIdx.x;
+        const int v = g < M ? csr[g] : 0;
+        int total;
+        const int excl = block_exclusive_scan(v, scratch, total);
+        if (g < M) csr[g] = carry + excl + v;
+        carry += total;
+    }
+}
+
+// One block per (parent, sequence, KV head): stable partition of the parent's rows by team and
+// copy of K/V rows into the packed layout.
+__global__ void __launch_bounds__(kBuildThreads)
+pack_parent_kernel(BuildParams p)
+{
+    __shared__ uint16_t owner[kMaxParent];
+    __shared__ int dest[kMaxParent];
+    const int parent = blockIdx.x, b = blockIdx.y, j = blockIdx.z;
+    const int64_t row0 = p.bv.seq_row_off[b];
+    const int N = (int)(p.bv.seq_row_off[b + 1] - row0);
+    const int P = p.parent_size;
+    const int first = parent * P;
+    if (first >= N) return;
+    const int nC = min(P, N - first);
+    const int tid = threadIdx.x;
+
+    const uint16_t *owner_in = p.owner + (size_t)j * p.bv.rows_total + row0 + first;
+    for (int i = tid; i < nC; i += kBuildThreads) owner[i] = owner_in[i];
+    __syncthreads();
+
+    const int64_t team0 = p.bv.seq_team_off[b];
+    const int32_t *csr = p.team_row_start + (size_t)j * (p.bv.teams_total + p.bv.n_seqs) + team0 + b;
+    const int team_local0 = parent * p.teams_per_full_parent;
+    for (int i = tid; i < nC; i += kBuildThreads) {
+        const int u = owner[i];
+        int rank = 0;
+        for (int a = 0; a < i; ++a) rank += (owner[a] == u);
+        dest[i] = csr[team_local0 + u] + rank;              // members in increasing token index
+    }
+    __syncthreads();
+
+    const size_t plane = (size_t)j * p.bv.rows_total + row0;
+    const uint2 *ksrc = reinterpret_cast<const uint2 *>(p.k_prompt) + (plane + first) * 32;
+    const uint2 *vsrc = reinterpret_cast<const uint2 *>(p.v_prompt) + (plane + first) * 32;
+    uint2 *kdst = reinterpret_cast<uint2 *>(p.k_packed) + plane * 32;
+    uint2 *vdst = reinterpret_cast<uint2 *>(p.v_packed) + plane * 32;
+    const int lane = tid & 31, warp = tid >> 5;
+    for (int i = warp; i < nC; i += kBuildThreads / 32) {
+        const size_t d = (size_t)dest[i] * 32 + lane;
+        kdst[d] = ksrc[(size_t)i * 32 + lane];
+        vdst[d] = vsrc[(size_t)i * 32 + lane];
+    }
+    int32_t *tok = p.row_token + plane;
+    for (int i = tid; i < nC; i += kBuildThreads) tok[dest[i]] = first + i;
+}
+
+size_t build_parent_smem(int P)
+{
+    return sizeof(double) * (kHeadDim + P) + sizeof(ValIdx) * 33 + sizeof(uint32_t) * (size_t)P * kRowWords
+           + sizeof(int) * 3 * (size_t)P + (size_t)P + 16;
+}
+
+}  // namespace
+
+cudaError_t launch_build_teams(const BuildParams &p, cudaStream_t s)
+{
+    const size_t smem = build_parent_smem(p.parent_size);
+    cudaError_t err = cudaFuncSetAttribute(build_parent_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           (int)smem);
+    if (err != cudaSuccess) return err;
+    dim3 grid(p.max_parents_per_seq, p.bv.n_seqs, p.bv.n_kv);
+    build_parent_kernel<<<grid, kBuildThreads, smem, s>>>(p);
+    if ((err = cudaGetLastError()) != cudaSuccess) return err;
+    scan_team_sizes_kernel<<<dim3(p.bv.n_seqs, p.bv.n_kv), kBuildThreads, 0, s>>>(p);
+    if ((err = cudaGetLastError()) != cudaSuccess) return err;
+    pack_parent_kernel<<<grid, kBuildThreads, 0, s>>>(p);
+    return cudaGetLastError();
+}
+
+}  // namespace santapp

@@ -1,0 +1,198 @@
+// Shared declarations of the SANTA++ decode-attention kernels (sm_100a).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "santapp.h"
+
+namespace santapp {
+
+constexpr int kHeadDim = 128;
+constexpr int kMaxGroup = 8;            // query heads per KV head
+constexpr int kMaxParent = 512;
+constexpr int kMaxTeamsPerSeq = 16384;  // selection keeps one 8-byte key per team in shared memory
+constexpr uint32_t kSrcSuffix = 0x80000000u;   // segment flag: rows live in the suffix buffers
+
+constexpr int kPartialStride = 132;     // floats per (slot, head): m, l, 2 pad, acc[128]
+
+// ---------------------------------------------------------------------------------------------
+// Device-side views. Plain structs passed by value to kernels.
+// ---------------------------------------------------------------------------------------------
+
+struct BatchView {
+    int n_seqs, n_q, n_kv, group;
+    const int64_t *seq_row_off;     // [n_seqs + 1]
+    const int64_t *seq_team_off;    // [n_seqs + 1]
+    int64_t rows_total, teams_total;
+};
+
+// Read plan of one (sequence, KV head) pair: the union of the teams its query heads selected,
+// in ascending team id, optionally followed by one suffix segment.
+struct PlanView {
+    int seg_cap;                    // segments reserved per pair
+    int32_t *seg_prefix;            // [n_pairs][seg_cap + 1] exclusive prefix of segment rows
+    int32_t *seg_row;               // [n_pairs][seg_cap] first row (global row of the KV plane, or
+                                    //   row of the suffix buffer when kSrcSuffix is set in seg_mask)
+    uint32_t *seg_mask;             // [n_pairs][seg_cap] bit h: head h of the group selected the team
+    float *seg_logc;                // [n_pairs][seg_cap][group] log2(e) * log c_g per selecting head
+    int32_t *pair_nseg;             // [n_pairs]
+    int32_t *pair_rows;             // [n_pairs] rows of the pair's plan (prompt union + suffix)
+    int32_t *pair_union_rows;       // [n_pairs] prompt rows only
+    int64_t *pair_row_prefix;       // [n_pairs + 1] exclusive prefix of pair_rows over pairs
+};
+
+struct Control {
+    int32_t *select_ticket;         // [n_pairs]
+    int32_t *plan_ticket;           // [1]
+    int32_t *attend_ticket;         // [n_pairs]
+};
+
+struct RouteParams {
+    BatchView bv;
+    const uint16_t *rep_keys;       // [n_kv][teams_total][128]
+    const int32_t *team_row_start;  // [n_kv][teams_total + n_seqs]
+    const uint16_t *q;              // [n_seqs][n_q][128]
+    double *y;                      // [n_q][teams_total] perturbed routing scores
+    int n_sample;
+    uint32_t seed_lo, seed_hi, step, stream_base;
+    double scale;
+    Control ctl;
+    int n_pairs;
+    int32_t *status;                // nullable
+};
+
+struct SelectParams {
+    BatchView bv;
+    const int32_t *team_row_start;
+    const double *y;
+    int n_sample;
+    uint32_t seed_lo, seed_hi, step, stream_base;
+    int32_t *sel_team;              // [n_seqs][n_q][n_sample]
+    float *sel_logc;                // [n_seqs][n_q][n_sample] natural log
+    double *tau;                    // [n_seqs][n_q]
+    const int32_t *suffix_len;      // nullable
+    int suffix_cap;
+    PlanView plan;
+    Control ctl;
+    int n_pairs;
+    // diagnostics (nullable)
+    int32_t *dbg_sel_idx;
+    float *dbg_sel_logc;
+    double *dbg_tau;
+    int32_t *dbg_union_rows;
+};
+
+struct AttendParams {
+    BatchView bv;
+    const uint16_t *k_packed, *v_packed;    // [n_kv][rows_total][128]
+    const uint16_t *k_suffix, *v_suffix;    // [n_seqs][n_kv][suffix_cap][128]
+    const uint16_t *q;
+    float qk_scale_log2;            // scale * log2(e)
+    PlanView plan;
+    Control ctl;
+    int n_pairs;
+    float *partials;                // [grid + n_pairs][group][kPartialStride]
+    float *out;                     // [n_seqs][n_q][128]
+    int32_t *status;                // nullable
+    int min_rows_per_cta;
+};
+
+// ---------------------------------------------------------------------------------------------
+// Host launchers (each returns the cudaError_t of its launches).
+// ---------------------------------------------------------------------------------------------
+cudaError_t launch_route_score(const RouteParams &p, int max_teams_per_seq, cudaStream_t s);
+cudaError_t launch_select_plan(const SelectParams &p, int max_teams_per_seq, cudaStream_t s);
+cudaError_t launch_dense_plan(const SelectParams &p, cudaStream_t s);
+cudaError_t launch_attend(const AttendParams &p, bool all_heads, int grid, cudaStream_t s);
+int attend_grid_size();
+
+struct BuildParams {
+    BatchView bv;
+    int parent_size, reps;
+    int teams_per_full_parent;              // min(R, P)
+    const uint16_t *k_prompt, *v_prompt;    // [n_kv][rows_total][128] token order
+    uint16_t *k_packed, *v_packed, *rep_keys;
+    int32_t *team_row_start, *row_token;
+    uint16_t *owner;                        // workspace [n_kv][rows_total]: team index inside the parent
+    int max_parents_per_seq;
+};
+cudaError_t launch_build_teams(const BuildParams &p, cudaStream_t s);
+
+// ---------------------------------------------------------------------------------------------
+// Device helpers
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
+__device__ __forceinline__ float bf16_to_float(uint16_t b) { return __uint_as_float(((uint32_t)b) << 16); }
+__device__ __forceinline__ double bf16_to_double(uint16_t b) { return (double)bf16_to_float(b); }
+
+// Philox4x32-10: 128-bit counter, 64-bit key, four 32-bit words.
+__device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint32_t k0, uint32_t k1)
+{
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        const uint32_t hi0 = __umulhi(0xD2511F53u, c.x), lo0 = 0xD2511F53u * c.x;
+        const uint32_t hi1 = __umulhi(0xCD9E8D57u, c.z), lo1 = 0xCD9E8D57u * c.z;
+        c = make_uint4(hi1 ^ c.y ^ k0, lo1, hi0 ^ c.w ^ k1, lo0);
+        k0 += 0x9E3779B9u;
+        k1 += 0xBB67AE85u;
+    }
+    return c;
+}
+
+// Gumbel(0,1) from a 32-bit word: u = (x + 0.5) / 2^32 in (0,1), G = -log(-log u), in fp64.
+__device__ __forceinline__ double gumbel_from_word(uint32_t x)
+{
+    const double u = ((double)x + 0.5) * (1.0 / 4294967296.0);
+    return -log(-log(u));
+}
+
+__device__ __forceinline__ uint32_t pick_word(const uint4 &w, int i)
+{
+    return i == 0 ? w.x : (i == 1 ? w.y : (i == 2 ? w.z : w.w));
+}
+
+// Order-preserving map from a double to an unsigned 64-bit key (larger double <=> larger key).
+__device__ __forceinline__ unsigned long long sortable_key(double v)
+{
+    const unsigned long long b = (unsigned long long)__double_as_longlong(v);
+    return (b & 0x8000000000000000ull) ? ~b : (b | 0x8000000000000000ull);
+}
+__device__ __forceinline__ double key_to_double(unsigned long long k)
+{
+    const unsigned long long b = (k & 0x8000000000000000ull) ? (k & 0x7FFFFFFFFFFFFFFFull) : ~k;
+    return __longlong_as_double((long long)b);
+}
+
+// Exclusive prefix sum of one int per thread over the block; returns the thread's offset and the
+// block total. `scratch` needs 33 ints of shared memory. blockDim.x is a multiple of 32, <= 1024.
+__device__ __forceinline__ int block_exclusive_scan(int v, int *scratch, int &total)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+    int incl = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if (lane >= o) incl += t;
+    }
+    __syncthreads();                       // scratch may still be read from a previous call
+    if (lane == 31) scratch[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        int w = lane < n_warps ? scratch[lane] : 0;
+        int wi = w;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int t = __shfl_up_sync(0xFFFFFFFFu, wi, o);
+            if (lane >= o) wi += t;
+        }
+        scratch[lane] = wi - w;            // exclusive offset of each warp
+        if (lane == 31) scratch[32] = wi;  // block total
+    }
+    __syncthreads();
+    total = scratch[32];
+    return scratch[warp] + incl - v;
+}
+
+}  // namespace santapp

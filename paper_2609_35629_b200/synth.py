@@ -182,6 +182,7 @@ def make_queries(spec: WorkloadSpec, data: LayerData, step: int) -> np.ndarray:
     q = np.empty((spec.n_seqs, spec.n_q_heads, d), dtype=np.float32)
     for b in range(spec.n_seqs):
         lo, hi = int(data.seq_row_off[b]), int(data.seq_row_off[b + 1])
+        keys_f32 = {}
         for h in range(spec.n_q_heads):
             j = h // G
             eps = rng.standard_normal(d, dtype=np.float32)
@@ -192,10 +193,12 @@ def make_queries(spec: WorkloadSpec, data: LayerData, step: int) -> np.ndarray:
             elif spec.query_kind == "concentrated":
                 if data.centres is None:
                     raise ValueError("concentrated queries need make_layer(..., keep_centres=True)")
+                if j not in keys_f32:
+                    keys_f32[j] = bf16_to_f32(data.k_prompt[j, lo:hi])
                 c = data.centres[j, int(rng.integers(0, spec.n_clusters))]
-                base = (c + np.float32(0.5) * eps).astype(np.float64)
-                logits = bf16_to_f64(data.k_prompt[j, lo:hi]) @ base / np.sqrt(d)
-                q[b, h] = (_bisect_alpha(logits, 64, 0.90) * base).astype(np.float32)
+                base = c + np.float32(0.5) * eps
+                logits = (keys_f32[j] @ base).astype(np.float64) / np.sqrt(d)
+                q[b, h] = np.float32(_bisect_alpha(logits, 64, 0.90)) * base
             else:
                 raise ValueError(spec.query_kind)
     return f32_to_bf16_bits(q)

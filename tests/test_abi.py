@@ -1,0 +1,98 @@
+"""The C-ABI library loads and exports every symbol include/santapp.h declares; host-side
+argument checks and size queries work without a GPU (no compute call is made here)."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2609_35629_b200 import binding as sp
+from paper_2609_35629_b200 import build as sp_build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    sp_build.build()
+    return sp.load_library()
+
+
+def test_header_symbols_are_exported(lib):
+    header = open(os.path.join(ROOT, "include", "santapp.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    declared = set(re.findall(r"\b(santapp_[a-z_]+)\s*\(", header))
+    assert declared, "no declarations found"
+    assert declared == set(sp.EXPORTS)
+    for name in declared:
+        assert hasattr(lib, name), f"{name} not exported"
+
+
+def test_version_and_strerror(lib):
+    assert lib.santapp_version() >= 100
+    assert lib.santapp_strerror(0) == b"ok"
+    assert b"invalid" in lib.santapp_strerror(sp.SANTAPP_ERR_INVALID_ARG)
+    assert b"workspace" in lib.santapp_strerror(sp.SANTAPP_ERR_WORKSPACE_TOO_SMALL)
+
+
+def test_sizes_follow_algorithms_4_and_2(lib):
+    g = sp.Geometry(3, 28, 4, 128, 512, 32)
+    s = sp.santapp_build_teams_sizes(g, [32768, 8192 + 100, 5])
+    # ceil(N/P) parents; a parent of c rows gives min(R, c) teams
+    assert s.rows_total == 32768 + 8292 + 5
+    assert s.teams_total == 64 * 32 + (16 * 32 + 32) + 5
+    assert s.max_teams_per_seq == 2048 and s.max_rows_per_seq == 32768
+    assert s.team_row_start_elems == 4 * (s.teams_total + 3)
+    assert s.build_workspace_bytes >= 2 * 4 * s.rows_total
+
+
+@pytest.mark.parametrize("kw,status", [
+    (dict(n_seqs=0), sp.SANTAPP_ERR_INVALID_ARG),
+    (dict(n_q_heads=30), sp.SANTAPP_ERR_INVALID_ARG),            # Hkv must divide Hq
+    (dict(reps_per_parent=7), sp.SANTAPP_ERR_INVALID_ARG),       # R must divide P
+    (dict(head_dim=64), sp.SANTAPP_ERR_UNSUPPORTED),
+    (dict(n_q_heads=36), sp.SANTAPP_ERR_UNSUPPORTED),            # 9 query heads per KV head
+    (dict(parent_size=1024), sp.SANTAPP_ERR_UNSUPPORTED),
+])
+def test_bad_geometry_is_rejected_on_the_host(lib, kw, status):
+    base = dict(n_seqs=1, n_q_heads=28, n_kv_heads=4, head_dim=128, parent_size=512, reps_per_parent=32)
+    base.update(kw)
+    with pytest.raises(sp.SantappError) as e:
+        sp.santapp_build_teams_sizes(sp.Geometry(**base), [1024] * max(base["n_seqs"], 1))
+    assert e.value.status == status
+
+
+def test_bad_prompt_length_is_rejected(lib):
+    with pytest.raises(sp.SantappError) as e:
+        sp.santapp_build_teams_sizes(sp.Geometry(2, 28, 4), [1024, 0])
+    assert e.value.status == sp.SANTAPP_ERR_INVALID_ARG
+
+
+def test_null_arguments_return_invalid_arg_without_touching_a_gpu(lib):
+    g = sp.Geometry(1, 28, 4).c()
+    t = sp.CTeams()                                                # all null
+    rc = lib.santapp_decode_attn(ctypes.byref(g), ctypes.byref(t), None, None, None, None, 0, 32, 0, 0, 0, 0.0,
+                                 None, None, None, 0, None)
+    assert rc == sp.SANTAPP_ERR_INVALID_ARG
+    rc = lib.santapp_dense_decode_attn(ctypes.byref(g), ctypes.byref(t), None, None, None, None, 0, 0.0, None,
+                                       None, 0, None)
+    assert rc == sp.SANTAPP_ERR_INVALID_ARG
+    rc = lib.santapp_build_teams(ctypes.byref(g), (ctypes.c_int32 * 1)(1024), None, None, ctypes.byref(t), None, 0,
+                                 None)
+    assert rc == sp.SANTAPP_ERR_INVALID_ARG
+
+
+def test_workspace_queries(lib):
+    g = sp.Geometry(1, 28, 4)
+    t = sp.CTeams(1, 1, 1, 1, 1, 1, 1, 32768, 8192, 2048, 32768)
+    ws32 = lib.santapp_decode_workspace_bytes(ctypes.byref(g.c()), ctypes.byref(t), 32)
+    ws64 = lib.santapp_decode_workspace_bytes(ctypes.byref(g.c()), ctypes.byref(t), 64)
+    wsd = lib.santapp_dense_workspace_bytes(ctypes.byref(g.c()), ctypes.byref(t))
+    assert 0 < wsd < ws32 < ws64 < 64 << 20
+    assert ws32 >= 8 * 28 * 8192                                    # the fp64 perturbed scores
+    assert lib.santapp_decode_workspace_bytes(ctypes.byref(g.c()), ctypes.byref(t), 0) == 0
+
+
+def test_missing_library_fails_loudly(tmp_path):
+    with pytest.raises(sp.SantappError):
+        sp.load_library(str(tmp_path / "libsantapp.so"))

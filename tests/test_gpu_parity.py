@@ -1,0 +1,235 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 oracle
+on the same seeded inputs.
+
+Bars (from the benchmark spec): sampled team indices bit-exact for the same
+seed; sparse outputs within 2e-3 * max|V|; dense outputs within 1e-3 * max|V|;
+team records identical (the builder evaluates distances in fp64 in the oracle's
+order, so even near-ties must fall the same way).
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import santapp_oracle as orc
+from paper_2609_35629_b200 import binding as sp
+from paper_2609_35629_b200 import synth
+
+import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+SPARSE_TOL = 2e-3
+DENSE_TOL = 1e-3
+
+_cache = {}
+
+
+def layer_for(name, spec_fn, **kw):
+    key = (name, tuple(sorted(kw.items())))
+    if key not in _cache:
+        spec = spec_fn(**kw)
+        data = synth.make_layer(spec, layer=0, keep_centres=(spec.query_kind == "concentrated"))
+        _cache[key] = pu.GpuLayer(spec, data)
+    return _cache[key]
+
+
+def check_team_records(layer, seqs=None, kv_heads=None):
+    spec = layer.spec
+    for b in (range(spec.n_seqs) if seqs is None else seqs):
+        r0, r1 = int(layer.seq_row_off[b]), int(layer.seq_row_off[b + 1])
+        for j in (range(spec.n_kv_heads) if kv_heads is None else kv_heads):
+            keys = synth.bf16_to_f64(layer.data.k_prompt[j, r0:r1])
+            ts_o, tm_o, rep_o = orc.build_teams_contiguous(keys, spec.parent_size, spec.reps_per_parent)
+            ts_g, tm_g, rep_g = layer.records(b, j)
+            assert np.array_equal(ts_g, ts_o)
+            assert np.array_equal(tm_g, tm_o)
+            assert np.array_equal(rep_g, keys[rep_o])                 # frozen representative keys
+            # packed rows are the member rows, K and V alike
+            assert np.array_equal(layer.k_packed_bits[j, r0:r1], layer.data.k_prompt[j, r0:r1][tm_g])
+            assert np.array_equal(layer.v_packed_bits[j, r0:r1], layer.data.v_prompt[j, r0:r1][tm_g])
+
+
+def check_sparse_step(layer, step, K, seed=1234, stream_base=0, suffix_len=None, seqs=None):
+    spec = layer.spec
+    q_bits = synth.make_queries(spec, layer.data, step)
+    sl = spec.suffix_len(step) if suffix_len is None else np.asarray(suffix_len, dtype=np.int32)
+    out, dbg = pu.gpu_step(layer, q_bits, sl, K, seed, step, stream_base)
+    ref = pu.oracle_step(layer, q_bits, sl, K, seed, step, stream_base, seqs=seqs)
+    assert int(dbg.status.item()) == 0
+    sel = dbg.sel_idx.cpu().numpy()
+    logc = dbg.sel_logc.cpu().numpy()
+    tau = dbg.tau.cpu().numpy()
+    union = dbg.union_rows.cpu().numpy()
+    vmax = pu.max_abs_v(layer)
+    worst = 0.0
+    for b, r in ref.items():
+        M = int(layer.seq_team_off[b + 1] - layer.seq_team_off[b])
+        Ke = min(K, M)
+        if Ke < M:
+            assert np.all(r.margin > 1e-9), "seeded workload too close to a selection boundary"
+        assert np.array_equal(sel[b, :, :Ke], r.sel[:, :Ke]), f"sampled teams differ (seq {b}, step {step})"
+        assert np.all(sel[b, :, Ke:] == -1)
+        assert np.allclose(logc[b, :, :Ke], r.logc[:, :Ke], rtol=0, atol=1e-5)
+        if Ke < M:
+            assert np.allclose(tau[b], r.tau, rtol=0, atol=1e-9)
+        else:
+            assert np.all(np.isnan(tau[b]))
+        for j in range(spec.n_kv_heads):
+            ts, _, _ = layer.records(b, j)
+            G = spec.group
+            assert union[b, j] == orc.union_rows(ts, r.sel[j * G:(j + 1) * G, :Ke])
+        err = np.abs(out[b] - r.o).max()
+        worst = max(worst, err)
+        assert err <= SPARSE_TOL * vmax, f"max |delta| {err} > {SPARSE_TOL} * {vmax}"
+    return worst
+
+
+def check_dense_step(layer, step, suffix_len=None, seqs=None):
+    spec = layer.spec
+    q_bits = synth.make_queries(spec, layer.data, step)
+    sl = spec.suffix_len(step) if suffix_len is None else np.asarray(suffix_len, dtype=np.int32)
+    out, _ = pu.gpu_step(layer, q_bits, sl, 0, 0, step, dense=True)
+    ref = pu.oracle_step(layer, q_bits, sl, 0, 0, step, dense=True, seqs=seqs)
+    vmax = pu.max_abs_v(layer)
+    for b, o in ref.items():
+        err = np.abs(out[b] - o).max()
+        assert err <= DENSE_TOL * vmax, f"dense max |delta| {err} > {DENSE_TOL} * {vmax}"
+
+
+# ---------------------------------------------------------------------------------------------
+
+def test_team_records_small_gqa_ragged_with_short_tail():
+    layer = layer_for("small", synth.spec_small_gqa)
+    check_team_records(layer)
+
+
+def test_team_records_tiny_config():
+    layer = layer_for("tiny", synth.spec_tiny)
+    check_team_records(layer)
+
+
+def test_team_records_duplicate_keys_and_singletons():
+    """Exact ties everywhere (all keys equal) and R = P (every key its own team)."""
+    spec = synth.spec_small_gqa(prompt=(300, 77), parent_size=64, reps=64)
+    data = synth.make_layer(spec)
+    layer = pu.GpuLayer(spec, data)
+    check_team_records(layer)
+    assert np.all(np.diff(layer.records(0, 0)[0]) == 1)
+    spec2 = synth.spec_small_gqa(prompt=(200, 130), parent_size=64, reps=8)
+    data2 = synth.make_layer(spec2)
+    data2.k_prompt[:] = data2.k_prompt[0, 0]                        # every key identical
+    layer2 = pu.GpuLayer(spec2, data2)
+    check_team_records(layer2)
+
+
+def test_decode_small_gqa_steps():
+    layer = layer_for("small", synth.spec_small_gqa)
+    for step in range(3):
+        check_sparse_step(layer, step, K=8)
+
+
+@pytest.mark.parametrize("K", [1, 2, 31, 33])
+def test_decode_small_gqa_budgets(K):
+    layer = layer_for("small", synth.spec_small_gqa)
+    check_sparse_step(layer, 1, K=K)
+
+
+def test_decode_k_at_least_m_equals_dense():
+    layer = layer_for("small", synth.spec_small_gqa)
+    spec = layer.spec
+    M_max = int(layer.teams.sizes.max_teams_per_seq)
+    step = 2
+    q_bits = synth.make_queries(spec, layer.data, step)
+    sl = spec.suffix_len(step)
+    check_sparse_step(layer, step, K=M_max)                          # all sequences: shortcut
+    out_s, _ = pu.gpu_step(layer, q_bits, sl, M_max, 5, step)
+    out_d, _ = pu.gpu_step(layer, q_bits, sl, 0, 0, step, dense=True)
+    assert np.abs(out_s - out_d).max() <= 1e-5 * pu.max_abs_v(layer)
+    # mixed: K between the two sequences' team counts -> one sampled, one dense
+    Ms = np.diff(layer.seq_team_off)
+    if Ms.min() < Ms.max():
+        check_sparse_step(layer, step, K=int(Ms.min()))
+
+
+def test_decode_suffix_edge_cases():
+    layer = layer_for("small", synth.spec_small_gqa)
+    check_sparse_step(layer, 0, K=8, suffix_len=[0, 0])
+    check_sparse_step(layer, 0, K=8, suffix_len=[layer.spec.suffix_cap, 1])
+    check_dense_step(layer, 0, suffix_len=[0, 0])
+    check_dense_step(layer, 0, suffix_len=[layer.spec.suffix_cap, 1])
+
+
+def test_decode_every_key_its_own_team():
+    spec = synth.spec_small_gqa(prompt=(256, 128), parent_size=32, reps=32, n_sample=16)
+    layer = pu.GpuLayer(spec, synth.make_layer(spec))
+    check_sparse_step(layer, 0, K=16)
+
+
+def test_decode_single_team_sequence():
+    """M = 1 for a sequence: K >= M, so the single team is always read."""
+    spec = synth.spec_small_gqa(prompt=(64, 700), parent_size=64, reps=1, n_sample=4)
+    layer = pu.GpuLayer(spec, synth.make_layer(spec))
+    check_sparse_step(layer, 0, K=4)
+    check_dense_step(layer, 0)
+
+
+def test_dense_small_gqa():
+    layer = layer_for("small", synth.spec_small_gqa)
+    for step in range(2):
+        check_dense_step(layer, step)
+
+
+def test_tiny_config_all_queries():
+    """Config 1: 1 head, 4096 keys + 16 suffix rows, 256 teams, 16 sampled, 32 queries."""
+    layer = layer_for("tiny", synth.spec_tiny)
+    for step in range(32):
+        check_sparse_step(layer, step, K=16, seed=0)
+    check_dense_step(layer, 0)
+
+
+def test_same_seed_same_bits_and_seed_changes_sample():
+    layer = layer_for("small", synth.spec_small_gqa)
+    spec = layer.spec
+    q_bits = synth.make_queries(spec, layer.data, 0)
+    sl = spec.suffix_len(0)
+    a, da = pu.gpu_step(layer, q_bits, sl, 8, 99, 0)
+    b, db = pu.gpu_step(layer, q_bits, sl, 8, 99, 0)
+    assert np.array_equal(da.sel_idx.cpu().numpy(), db.sel_idx.cpu().numpy())
+    assert np.abs(a - b).max() <= 1e-6 * pu.max_abs_v(layer)         # merge order may differ by rounding
+    c, dc = pu.gpu_step(layer, q_bits, sl, 8, 100, 0)
+    assert not np.array_equal(da.sel_idx.cpu().numpy(), dc.sel_idx.cpu().numpy())
+    d, dd = pu.gpu_step(layer, q_bits, sl, 8, 99, 1)
+    assert not np.array_equal(da.sel_idx.cpu().numpy(), dd.sel_idx.cpu().numpy())
+
+
+def test_ragged_batch_medium():
+    """Ragged CSR-of-CSR metadata: 6 sequences of different lengths, 31 sampled teams."""
+    spec = synth.spec_ragged(n_steps=2, n_seqs=6, lo=1024, hi=6144)
+    layer = pu.GpuLayer(spec, synth.make_layer(spec))
+    check_team_records(layer, seqs=[0, 5], kv_heads=[1])
+    check_sparse_step(layer, 0, K=31)
+    check_dense_step(layer, 1)
+
+
+def test_qwen_32k_full_size_batch1():
+    """Config 2 at full size (28 heads over 4 KV heads, 32K prompt, 2048 teams per KV head,
+    32 sampled teams): every head against the oracle, several steps; team records of one KV
+    head against the oracle's Algorithm 2."""
+    layer = layer_for("qwen_b1", synth.spec_qwen_b1)
+    check_team_records(layer, kv_heads=[2])
+    for step in (0, 7, 255):
+        check_sparse_step(layer, step, K=32)
+    check_sparse_step(layer, 3, K=32, suffix_len=[0])
+    check_sparse_step(layer, 4, K=31)
+    check_sparse_step(layer, 5, K=128)
+    check_dense_step(layer, 9)
+
+
+def test_qwen_32k_batch8_concentrated_sampled_sequences():
+    """Config 3 shape (8 sequences, 64 sampled teams, concentrated queries): the GPU runs the
+    whole batch, the oracle checks two of the sequences."""
+    layer = layer_for("qwen_b8", synth.spec_qwen_b8, n_steps=2)
+    check_sparse_step(layer, 0, K=64, seqs=[0, 5])
+    check_dense_step(layer, 1, seqs=[3])
