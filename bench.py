@@ -1,0 +1,520 @@
+#!/usr/bin/env python
+"""Benchmark of SANTA++ decode attention on B200.
+
+One "step" is one decode token through `--layers` independently seeded layers of the
+Qwen2.5-7B single-layer workload (batch 1, 28 query heads over 4 KV heads, head_dim 128,
+32K-token prompt, suffix growing to 256, parents of 512 with 32 representatives, 32 sampled
+teams): per layer, the whole hot path (representative scoring, Gumbel-top-K sampling, read
+plan, exact attention over the sampled teams and the suffix, split-K merge). The layers are
+visited round-robin so that every layer-step reads K/V from HBM, not from L2 (28 layers hold
+1.8 GiB of packed K/V against 126 MB of L2).
+
+Prints ONE JSON line (rank 0). `value` is microseconds per layer-step with all inputs resident
+in HBM, replayed from CUDA graphs; `e2e` is the same through host buffers (pinned host to
+device copies of the step's queries, new suffix rows and counters, device to host read of the
+outputs, inside the timed region).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--layers L]
+"""
+import argparse
+import json
+import math
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "decode_attn_us_per_layer_step"
+UNIT = "us"
+N_STEP_INPUTS = 8          # distinct (query, suffix length, step) inputs cycled through
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--layers", type=int, default=28)
+    ap.add_argument("--workload", default="qwen7b_b1_32k",
+                    choices=["qwen7b_b1_32k", "qwen7b_b8_32k", "ragged", "long_128k", "small_gqa"])
+    ap.add_argument("--n-sample", type=int, default=0, help="override K")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-stages", action="store_true")
+    return ap.parse_args()
+
+
+def make_spec(args, seed):
+    from paper_2609_35629_b200 import synth
+    if args.workload == "qwen7b_b1_32k":
+        spec = synth.spec_qwen_b1(seed=seed)
+    elif args.workload == "qwen7b_b8_32k":
+        spec = synth.spec_qwen_b8(seed=seed)
+    elif args.workload == "ragged":
+        spec = synth.spec_ragged(seed=seed)
+    elif args.workload == "long_128k":
+        spec = synth.spec_long(seed=seed)
+    else:
+        spec = synth.spec_small_gqa(seed=seed)
+    if args.n_sample:
+        spec.n_sample = args.n_sample
+    return spec
+
+
+def workload_text(spec, layers):
+    return (f"{spec.name}: {spec.n_seqs} seq x {spec.n_q_heads} q heads / {spec.n_kv_heads} KV heads, d={spec.head_dim}, "
+            f"prompt {min(spec.prompt_len)}..{max(spec.prompt_len)}, suffix cap {spec.suffix_cap}, "
+            f"P={spec.parent_size}, R={spec.reps_per_parent}, K={spec.n_sample}, {layers} layers round-robin")
+
+
+# -------------------------------------------------------------------------------------------
+# Clock sampling (read-only NVML queries)
+# -------------------------------------------------------------------------------------------
+class ClockSampler:
+    REASONS = {0x1: "gpu_idle", 0x2: "applications_clocks_setting", 0x4: "sw_power_cap", 0x8: "hw_slowdown",
+               0x10: "sync_boost", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+               0x80: "hw_power_brake_slowdown", 0x100: "display_clock_setting"}
+
+    def __init__(self, device_index):
+        self.samples, self.reason_bits, self.max_mhz = [], 0, None
+        self._stop = threading.Event()
+        self._thread = None
+        self.ok = False
+        try:
+            import pynvml
+            import torch
+            pynvml.nvmlInit()
+            try:
+                uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+                if not uuid.startswith("GPU-"):
+                    uuid = "GPU-" + uuid
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(uuid)
+            except Exception:
+                vis = os.environ.get("CUDA_VISIBLE_DEVICES", "")
+                ids = [x for x in vis.split(",") if x.strip() != ""]
+                phys = int(ids[device_index]) if ids and ids[device_index].isdigit() else device_index
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(phys)
+            self.nv = pynvml
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception as e:  # NVML unavailable: report that, do not guess
+            self.err = repr(e)
+
+    def _run(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                self.reason_bits |= int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+            except Exception:
+                pass
+            time.sleep(0.002)
+
+    def start(self):
+        if self.ok:
+            self._stop.clear()
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        if self._thread is not None:
+            self._stop.set()
+            self._thread.join()
+            self._thread = None
+
+    def summary(self):
+        if not self.ok or not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": ["nvml_unavailable"]}
+        reasons = [name for bit, name in self.REASONS.items() if self.reason_bits & bit and name != "gpu_idle"]
+        return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.max_mhz, "reasons": reasons,
+                "samples": len(self.samples)}
+
+
+# -------------------------------------------------------------------------------------------
+# The reference arm: the CPU oracle, as it stands, on the host cores
+# -------------------------------------------------------------------------------------------
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import santapp_oracle as orc
+    from paper_2609_35629_b200 import synth
+    spec = make_spec(args, seed=0)
+    cores = len(os.sched_getaffinity(0))
+    data = synth.make_layer(spec, layer=0, keep_centres=(spec.query_kind == "concentrated"))
+    scale = 1.0 / math.sqrt(spec.head_dim)
+    b = 0
+    r0, r1 = int(data.seq_row_off[b]), int(data.seq_row_off[b + 1])
+    k = synth.bf16_to_f64(data.k_prompt[:, r0:r1])
+    v = synth.bf16_to_f64(data.v_prompt[:, r0:r1])
+    recs = [orc.build_teams_contiguous(k[j], spec.parent_size, spec.reps_per_parent)
+            for j in range(spec.n_kv_heads)]
+    M = np.array([len(r[0]) - 1 for r in recs], dtype=np.int32)
+    ts = np.zeros((spec.n_kv_heads, int(M.max()) + 1), dtype=np.int32)
+    tm = np.zeros((spec.n_kv_heads, r1 - r0), dtype=np.int32)
+    rk = np.zeros((spec.n_kv_heads, int(M.max()), spec.head_dim))
+    for j, (s, m, rep) in enumerate(recs):
+        ts[j, :len(s)] = s
+        tm[j] = m
+        rk[j, :len(rep)] = k[j][rep]
+
+    def one(step):
+        q = synth.bf16_to_f64(synth.make_queries(spec, data, step)[b])
+        t = int(spec.suffix_len(step)[b])
+        ks = synth.bf16_to_f64(data.k_suffix[b, :, :t]) if t else None
+        vs = synth.bf16_to_f64(data.v_suffix[b, :, :t]) if t else None
+        t0 = time.perf_counter()
+        orc.decode_step(q, k, v, M, ts, tm, rk, ks, vs, spec.n_sample, 0, step, b, scale, n_threads=cores)
+        return time.perf_counter() - t0
+
+    for s in range(args.warmup):
+        one(s)
+    times = [one(args.warmup + s) for s in range(args.steps)]
+    us = 1e6 * float(np.sum(times)) / max(len(times), 1)
+    sample = (f"{args.steps} layer-steps of sequence 0 of layer 0 ({spec.n_q_heads} heads, {r1 - r0} prompt rows), "
+              f"fp64 oracle, OpenMP over heads")
+    line = {"impl": "reference", "metric": METRIC, "value": us, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": us / 1e3, "higher_is_better": False,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": workload_text(spec, 1)},
+            "cpu_baseline": {"value": us, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": us, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+# -------------------------------------------------------------------------------------------
+# Our arm
+# -------------------------------------------------------------------------------------------
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2609_35629_b200 import binding as sp
+    from paper_2609_35629_b200 import synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    sp.load_library()
+
+    # Independent replicas: every rank owns its own sequences (seed = rank); no exchange.
+    spec = make_spec(args, seed=rank)
+    L = args.layers
+    geom = sp.Geometry(spec.n_seqs, spec.n_q_heads, spec.n_kv_heads, spec.head_dim, spec.parent_size,
+                       spec.reps_per_parent)
+    K = spec.n_sample
+    B, Hq, Hkv, d = spec.n_seqs, spec.n_q_heads, spec.n_kv_heads, spec.head_dim
+    conc = spec.query_kind == "concentrated"
+
+    # ---- inputs: generated on the host (seeded), moved to HBM, teams built on the GPU ----
+    t_prep = time.perf_counter()
+    layers, host_layers = [], []
+    q_all = np.empty((N_STEP_INPUTS, L, B, Hq, d), dtype=np.uint16)
+    cap = max(spec.suffix_cap, 1)
+    ksuf_all = torch.empty((L, B, Hkv, cap, d), dtype=torch.bfloat16, device=dev)
+    vsuf_all = torch.empty_like(ksuf_all)
+    for l in range(L):
+        data = synth.make_layer(spec, layer=l, keep_centres=conc)
+        for s in range(N_STEP_INPUTS):
+            q_all[s, l] = synth.make_queries(spec, data, s)
+        k_prompt = sp.bf16_bits_to_cuda(data.k_prompt, dev)
+        v_prompt = sp.bf16_bits_to_cuda(data.v_prompt, dev)
+        teams = sp.santapp_build_teams(geom, spec.prompt_len, k_prompt, v_prompt)
+        torch.cuda.synchronize()
+        del k_prompt, v_prompt
+        ksuf_all[l].copy_(sp.bf16_bits_to_cuda(data.k_suffix, dev))
+        vsuf_all[l].copy_(sp.bf16_bits_to_cuda(data.v_suffix, dev))
+        layers.append(dict(teams=teams, k_suffix=ksuf_all[l], v_suffix=vsuf_all[l]))
+        if l == 0:
+            host_layers.append(data)
+    prep_s = time.perf_counter() - t_prep
+
+    # step s of the cycle uses decode step index (and suffix length) spread over the 256-step run
+    step_ids = [int(round(i * (spec.n_steps - 1) / max(N_STEP_INPUTS - 1, 1))) for i in range(N_STEP_INPUTS)]
+    sl_all = np.stack([spec.suffix_len(st) for st in step_ids]).astype(np.int32)        # [S, B]
+
+    # packed per-step inputs: [q bytes | suffix_len | step]
+    q_bytes = L * B * Hq * d * 2
+    in_bytes = q_bytes + 4 * B + 4
+    in_bytes_pad = (in_bytes + 255) // 256 * 256
+    inputs_host = torch.zeros((N_STEP_INPUTS, in_bytes_pad), dtype=torch.uint8).pin_memory()
+    for s in range(N_STEP_INPUTS):
+        row = inputs_host[s].numpy()
+        row[:q_bytes] = q_all[s].reshape(-1).view(np.uint8)
+        row[q_bytes:q_bytes + 4 * B] = sl_all[s].view(np.uint8)
+        row[q_bytes + 4 * B:in_bytes] = np.array([step_ids[s]], dtype=np.uint32).view(np.uint8)
+    inputs_dev = inputs_host.to(dev)
+    cur = torch.zeros(in_bytes_pad, dtype=torch.uint8, device=dev)
+    q_cur = cur[:q_bytes].view(torch.bfloat16).view(L, B, Hq, d)
+    sl_cur = cur[q_bytes:q_bytes + 4 * B].view(torch.int32)
+    step_cur = cur[q_bytes + 4 * B:in_bytes].view(torch.int32)
+    out = torch.zeros((L, B, Hq, d), dtype=torch.float32, device=dev)
+    out_dense = torch.zeros_like(out)
+    ws = [torch.empty(sp.santapp_decode_workspace_bytes(geom, layers[l]["teams"], K), dtype=torch.uint8, device=dev)
+          for l in range(L)]
+    wsd = torch.empty(sp.santapp_dense_workspace_bytes(geom, layers[0]["teams"]), dtype=torch.uint8, device=dev)
+    seed = 1234 + rank
+
+    def sparse_layer(l, debug=None):
+        ly = layers[l]
+        sp.santapp_decode_attn(geom, ly["teams"], q_cur[l], ly["k_suffix"], ly["v_suffix"], sl_cur, K, seed, 0,
+                               stream_base=l * B, out=out[l], debug=debug, workspace=ws[l], step_dev=step_cur)
+
+    def dense_layer(l):
+        ly = layers[l]
+        sp.santapp_dense_decode_attn(geom, ly["teams"], q_cur[l], ly["k_suffix"], ly["v_suffix"], sl_cur,
+                                     out=out_dense[l], workspace=wsd)
+
+    def set_inputs(s):
+        cur.copy_(inputs_dev[s], non_blocking=True)
+
+    # ---- accounting pass (eager): union rows per (input, layer) -> algorithmic bytes ----
+    dbg = sp.DebugBuffers(geom, K, dev)
+    union = np.zeros((N_STEP_INPUTS, L), dtype=np.int64)
+    M_total = int(layers[0]["teams"].sizes.teams_total)
+    N_total = int(layers[0]["teams"].sizes.rows_total)
+    for s in range(N_STEP_INPUTS):
+        set_inputs(s)
+        for l in range(L):
+            sparse_layer(l, debug=dbg)
+            torch.cuda.synchronize()
+            union[s, l] = int(dbg.union_rows.sum().item())
+            assert int(dbg.status.item()) == 0, "non-finite output"
+    launches_per_layer_step = sp.santapp_last_launch_count()
+    suffix_rows = sl_all.sum(axis=1).astype(np.int64) * Hkv                              # per input, per layer
+    row_bytes = 2 * d * 2                                                                # K row + V row, bf16
+    io_bytes = B * Hq * d * (2 + 4)                                                      # q in, out fp32
+    attend_bytes = row_bytes * (union + suffix_rows[:, None]) + io_bytes                 # [S, L]
+    route_bytes = Hkv * (M_total * d * 2 + (M_total + B) * 4)
+    sparse_bytes = attend_bytes + route_bytes
+    dense_bytes = row_bytes * (Hkv * N_total + suffix_rows) + io_bytes                   # [S]
+
+    # ---- graphs: one decode step = all layers ----
+    def capture(fn):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            for l in range(L):
+                fn(l)
+        return g
+
+    set_inputs(0)
+    for l in range(L):
+        dense_layer(l)
+    torch.cuda.synchronize()
+    g_sparse = capture(sparse_layer)
+    g_dense = capture(dense_layer)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    def timed(run_step, steps, warmup, sampler=None):
+        for i in range(warmup):
+            run_step(i)
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        if sampler:
+            sampler.start()
+        e0.record()
+        for i in range(steps):
+            run_step(warmup + i)
+        e1.record()
+        torch.cuda.synchronize()
+        if sampler:
+            sampler.stop()
+        ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ms], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        barrier()
+        return ms
+
+    def sparse_step(i):
+        set_inputs(i % N_STEP_INPUTS)
+        g_sparse.replay()
+
+    def dense_step(i):
+        set_inputs(i % N_STEP_INPUTS)
+        g_dense.replay()
+
+    Kst, W = args.steps, max(args.warmup, 3)
+    sampler = ClockSampler(local_rank)
+    ms_sparse = timed(sparse_step, Kst, W, sampler)
+    clocks = sampler.summary()
+    n_dense = max(min(Kst, 50), 3)
+    ms_dense = timed(dense_step, n_dense, 3)
+    us_layer = 1e3 * ms_sparse / (Kst * L * world)
+    us_layer_dense = 1e3 * ms_dense / (n_dense * L * world)
+
+    used = np.array([(W + i) % N_STEP_INPUTS for i in range(Kst)])
+    mean_sparse_bytes = float(sparse_bytes[used].mean())
+    mean_attend_bytes = float(attend_bytes[used].mean())
+    used_d = np.array([(3 + i) % N_STEP_INPUTS for i in range(n_dense)])
+    mean_dense_bytes = float(dense_bytes[used_d].mean())
+
+    # eager (no graph) timing of the same step, for reference
+    def eager_step(i):
+        set_inputs(i % N_STEP_INPUTS)
+        for l in range(L):
+            sparse_layer(l)
+    ms_eager = timed(eager_step, max(Kst // 10, 3), 3)
+    us_layer_eager = 1e3 * ms_eager / (max(Kst // 10, 3) * L * world)
+
+    # ---- isolated stages (graphs of one stage over all layers; plans and scores left in the
+    # per-layer workspaces by a full step with the same inputs) ----
+    stages = {}
+    if not args.no_stages:
+        set_inputs(1)
+        g_sparse.replay()
+        torch.cuda.synchronize()
+        for name, mask in (("route_score", sp.STAGE_ROUTE), ("select_plan", sp.STAGE_SELECT),
+                           ("attend", sp.STAGE_ATTEND)):
+            sp.santapp_set_stage_mask(mask)
+            g = capture(sparse_layer)
+            sp.santapp_set_stage_mask(sp.STAGE_ALL)
+            reps = max(Kst // 4, 10)
+            ms = timed(lambda i: g.replay(), reps, 3)
+            stages[name] = 1e3 * ms / (reps * L)
+        attend_bytes_1 = float(attend_bytes[1].mean())
+    peaks = {}
+    try:
+        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+    except Exception:
+        pass
+    peak_gbs = float(peaks.get("hbm_gbs", 6650.0))
+    peak_kind = "measured (MEASURED_PEAKS.json hbm_gbs)" if "hbm_gbs" in peaks else "fallback 6650 GB/s"
+    roofline = None
+    if stages:
+        achieved = attend_bytes_1 / (stages["attend"] * 1e-6) / 1e9
+        roofline = {"bound": "hbm", "kernel": "attend_kernel", "achieved": achieved, "peak": peak_gbs, "unit": "GB/s",
+                    "frac": achieved / peak_gbs, "traffic": None, "peak_kind": peak_kind,
+                    "algorithmic_bytes_per_launch": attend_bytes_1, "us_per_launch": stages["attend"]}
+
+    # ---- end to end through host buffers ----
+    e2e = None
+    if not args.no_e2e:
+        new_rows = torch.zeros((N_STEP_INPUTS, 2, B, L, Hkv, d), dtype=torch.bfloat16).pin_memory()
+        for s in range(N_STEP_INPUTS):
+            for b in range(B):
+                t = max(int(sl_all[s, b]) - 1, 0)
+                new_rows[s, 0, b] = ksuf_all[:, b, :, t].cpu()
+                new_rows[s, 1, b] = vsuf_all[:, b, :, t].cpu()
+        new_dev = torch.zeros((2, B, L, Hkv, d), dtype=torch.bfloat16, device=dev)
+        out_host = torch.zeros((L, B, Hq, d), dtype=torch.float32).pin_memory()
+
+        def e2e_step(i):
+            s = i % N_STEP_INPUTS
+            cur.copy_(inputs_host[s], non_blocking=True)             # queries, suffix lengths, step
+            new_dev.copy_(new_rows[s], non_blocking=True)            # the token's own K/V rows
+            for b in range(B):                                       # append them to every layer's suffix
+                t = max(int(sl_all[s, b]) - 1, 0)
+                ksuf_all[:, b, :, t].copy_(new_dev[0, b], non_blocking=True)
+                vsuf_all[:, b, :, t].copy_(new_dev[1, b], non_blocking=True)
+            g_sparse.replay()
+            out_host.copy_(out, non_blocking=True)
+            torch.cuda.current_stream().synchronize()                # the caller reads the result
+
+        n_e2e = max(Kst // 4, 5)
+        ms_e2e = timed(e2e_step, n_e2e, 3)
+        e2e = {"value": 1e3 * ms_e2e / (n_e2e * L * world), "unit": UNIT,
+               "h2d_bytes_per_step": int(in_bytes + new_rows[0].numel() * 2),
+               "d2h_bytes_per_step": int(out_host.numel() * 4)}
+
+    # ---- the oracle on the host cores, bounded sample ----
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu_baseline = cpu_baseline_leg(spec, host_layers[0], layers[0]["teams"], seed)
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": us_layer, "unit": UNIT, "n_gpus": world, "steps": Kst, "warmup": W,
+            "ms_per_step": ms_sparse / Kst, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": workload_text(spec, L), "l2": "inputs larger than L2: layers visited round-robin",
+                       "replay": "CUDA graph of one decode step over all layers", "replicas": world},
+            "clocks": clocks, "gpu_launches": int(Kst * L * launches_per_layer_step),
+            "e2e": e2e, "roofline": roofline, "cpu_baseline": cpu_baseline,
+            "layer_steps_per_s": 1e6 / us_layer, "tokens_per_s_attention_only": B * 1e6 / (us_layer * 28),
+            "us_per_layer_step_eager": us_layer_eager,
+            "dense_us_per_layer_step": us_layer_dense, "speedup_vs_dense": us_layer_dense / us_layer,
+            "bytes_per_layer_step": mean_sparse_bytes, "dense_bytes_per_layer_step": mean_dense_bytes,
+            "read_reduction": mean_dense_bytes / mean_sparse_bytes,
+            "achieved_gbs": mean_sparse_bytes / (us_layer * 1e-6) / 1e9,
+            "achieved_frac_of_peak": mean_sparse_bytes / (us_layer * 1e-6) / 1e9 / peak_gbs,
+            "dense_achieved_gbs": mean_dense_bytes / (us_layer_dense * 1e-6) / 1e9,
+            "dense_achieved_frac_of_peak": mean_dense_bytes / (us_layer_dense * 1e-6) / 1e9 / peak_gbs,
+            "attend_bytes_per_layer_step": mean_attend_bytes,
+            "logical_access_pct": 100.0 * float((M_total * Hkv + 2 * (union[used].mean() + suffix_rows[used].mean()))
+                                                / (2 * (Hkv * N_total + suffix_rows[used].mean()))),
+            "stage_us": stages, "prep_seconds": prep_s,
+        }
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def cpu_baseline_leg(spec, data, teams, seed):
+    """The fp64 oracle on sequence 0 of layer 0, using the GPU-built team records, timed on
+    all host cores for a bounded number of layer-steps."""
+    from oracle import santapp_oracle as orc
+    from paper_2609_35629_b200 import synth
+    cores = len(os.sched_getaffinity(0))
+    b = 0
+    r0, r1 = int(data.seq_row_off[b]), int(data.seq_row_off[b + 1])
+    n_kv, d = spec.n_kv_heads, spec.head_dim
+    trs = teams.team_row_start.cpu().numpy()
+    tok = teams.row_token.cpu().numpy()
+    import torch
+    rep_bits = teams.rep_keys.view(torch.int16).cpu().numpy().view(np.uint16)
+    to = teams.seq_team_off.cpu().numpy()
+    t0, t1 = int(to[b]), int(to[b + 1])
+    M = np.full(n_kv, t1 - t0, dtype=np.int32)
+    ts = np.ascontiguousarray(trs[:, t0 + b:t1 + b + 1])
+    tm = np.ascontiguousarray(tok[:, r0:r1])
+    rk = synth.bf16_to_f64(rep_bits[:, t0:t1])
+    k = synth.bf16_to_f64(data.k_prompt[:, r0:r1])
+    v = synth.bf16_to_f64(data.v_prompt[:, r0:r1])
+    scale = 1.0 / math.sqrt(d)
+    times, n = [], 0
+    budget = time.perf_counter() + 15.0
+    while time.perf_counter() < budget and n < 400:
+        step = n % spec.n_steps
+        q = synth.bf16_to_f64(synth.make_queries(spec, data, step % N_STEP_INPUTS)[b])
+        t = int(spec.suffix_len(step)[b])
+        ks = synth.bf16_to_f64(data.k_suffix[b, :, :t]) if t else None
+        vs = synth.bf16_to_f64(data.v_suffix[b, :, :t]) if t else None
+        s0 = time.perf_counter()
+        orc.decode_step(q, k, v, M, ts, tm, rk, ks, vs, spec.n_sample, seed, step, b, scale, n_threads=cores)
+        times.append(time.perf_counter() - s0)
+        n += 1
+    us = 1e6 * float(np.mean(times[1:] if len(times) > 1 else times))
+    return {"value": us, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"{n} layer-steps of sequence 0, layer 0 ({spec.n_q_heads} heads, {r1 - r0} prompt rows), "
+                      f"fp64 oracle with OpenMP over heads"}
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -178,6 +178,8 @@ size_t santapp_decode_workspace_bytes(const santapp_geom *geom, const santapp_te
  *                   [0, suffix_cap]); NULL means 0 everywhere
  *   n_sample        K >= 1
  *   seed, step, stream_base   random-stream key and counters (see top of file)
+ *   step_dev        device uint32 [1] or NULL: when given, its value is added to `step` on the
+ *                   device, so a captured CUDA graph can be replayed for successive tokens
  *   scale           logit scale; 0 means 1 / sqrt(d)
  *   out             device fp32 [n_seqs][n_q_heads][d], out
  *   dbg             host struct of device pointers or NULL
@@ -187,8 +189,9 @@ size_t santapp_decode_workspace_bytes(const santapp_geom *geom, const santapp_te
 int santapp_decode_attn(const santapp_geom *geom, const santapp_teams *teams, const void *q,
                         const void *k_suffix, const void *v_suffix, const int32_t *suffix_len_dev,
                         int32_t suffix_cap, int32_t n_sample, uint64_t seed, uint32_t step,
-                        uint32_t stream_base, float scale, float *out, const santapp_debug *dbg,
-                        void *workspace, size_t workspace_bytes, santapp_stream stream);
+                        const uint32_t *step_dev, uint32_t stream_base, float scale, float *out,
+                        const santapp_debug *dbg, void *workspace, size_t workspace_bytes,
+                        santapp_stream stream);
 
 /* Workspace bytes santapp_dense_decode_attn needs. */
 size_t santapp_dense_workspace_bytes(const santapp_geom *geom, const santapp_teams *teams);
@@ -209,6 +212,17 @@ int santapp_dense_decode_attn(const santapp_geom *geom, const santapp_teams *tea
  * bookkeeping, no device access): number of kernels launched by that call.
  */
 int santapp_last_launch_count(void);
+
+/*
+ * Diagnostic: choose which stages the following santapp_decode_attn calls on this thread
+ * launch, for timing one stage in isolation (the paper's "isolated-stage measurements").
+ * Bit 0: representative scoring and perturbation; bit 1: selection and read plan; bit 2: exact
+ * attention and merge. A stage that is skipped reuses what an earlier full call with the same
+ * arguments left in the same workspace. The default, and the only setting that computes a
+ * decode step, is SANTAPP_STAGE_ALL.
+ */
+enum { SANTAPP_STAGE_ROUTE = 1, SANTAPP_STAGE_SELECT = 2, SANTAPP_STAGE_ATTEND = 4, SANTAPP_STAGE_ALL = 7 };
+void santapp_set_stage_mask(int mask);
 
 #ifdef __cplusplus
 }

@@ -27,7 +27,10 @@ EXPORTS = [
     "santapp_version", "santapp_strerror", "santapp_last_cuda_error", "santapp_build_teams_sizes",
     "santapp_build_teams", "santapp_decode_workspace_bytes", "santapp_decode_attn",
     "santapp_dense_workspace_bytes", "santapp_dense_decode_attn", "santapp_last_launch_count",
+    "santapp_set_stage_mask",
 ]
+
+STAGE_ROUTE, STAGE_SELECT, STAGE_ATTEND, STAGE_ALL = 1, 2, 4, 7
 
 
 class SantappError(RuntimeError):
@@ -91,7 +94,9 @@ def load_library(path: Optional[str] = None):
     L.santapp_dense_workspace_bytes.argtypes = [ctypes.POINTER(CGeom), ctypes.POINTER(CTeams)]
     L.santapp_dense_workspace_bytes.restype = sz
     L.santapp_decode_attn.argtypes = [ctypes.POINTER(CGeom), ctypes.POINTER(CTeams), vp, vp, vp, vp, i32, i32,
-                                      u64, u32, u32, f32, vp, ctypes.POINTER(CDebug), vp, sz, vp]
+                                      u64, u32, vp, u32, f32, vp, ctypes.POINTER(CDebug), vp, sz, vp]
+    L.santapp_set_stage_mask.argtypes = [ctypes.c_int]
+    L.santapp_set_stage_mask.restype = None
     L.santapp_decode_attn.restype = ctypes.c_int
     L.santapp_dense_decode_attn.argtypes = [ctypes.POINTER(CGeom), ctypes.POINTER(CTeams), vp, vp, vp, vp, i32,
                                             f32, vp, vp, sz, vp]
@@ -176,6 +181,10 @@ def santapp_last_launch_count() -> int:
     return load_library().santapp_last_launch_count()
 
 
+def santapp_set_stage_mask(mask: int) -> None:
+    load_library().santapp_set_stage_mask(mask)
+
+
 def santapp_build_teams_sizes(geom: Geometry, prompt_len) -> Sizes:
     L = load_library()
     n = len(prompt_len)
@@ -231,8 +240,10 @@ def santapp_decode_attn(geom: Geometry, teams: Teams, q: torch.Tensor, k_suffix:
                         v_suffix: Optional[torch.Tensor], suffix_len: Optional[torch.Tensor], n_sample: int,
                         seed: int, step: int, stream_base: int = 0, scale: float = 0.0,
                         out: Optional[torch.Tensor] = None, debug: Optional[DebugBuffers] = None,
-                        workspace: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
-    """q bf16 [B, Hq, d]; k_suffix/v_suffix bf16 [B, Hkv, cap, d]; suffix_len int32 [B] (device)."""
+                        workspace: Optional[torch.Tensor] = None, stream=None,
+                        step_dev: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """q bf16 [B, Hq, d]; k_suffix/v_suffix bf16 [B, Hkv, cap, d]; suffix_len int32 [B] (device);
+    step_dev optional device int32/uint32 [1] added to `step` on the device."""
     L = load_library()
     if out is None:
         out = torch.empty((geom.n_seqs, geom.n_q_heads, geom.head_dim), dtype=torch.float32, device=q.device)
@@ -242,8 +253,8 @@ def santapp_decode_attn(geom: Geometry, teams: Teams, q: torch.Tensor, k_suffix:
     cap = 0 if k_suffix is None else int(k_suffix.shape[2])
     g = geom.c()
     _check(L.santapp_decode_attn(ctypes.byref(g), ctypes.byref(teams.c), _ptr(q), _ptr(k_suffix), _ptr(v_suffix),
-                                 _ptr(suffix_len), cap, n_sample, ctypes.c_uint64(seed), step, stream_base,
-                                 scale, _ptr(out), ctypes.byref(debug.c) if debug is not None else None,
+                                 _ptr(suffix_len), cap, n_sample, ctypes.c_uint64(seed), step, _ptr(step_dev),
+                                 stream_base, scale, _ptr(out), ctypes.byref(debug.c) if debug is not None else None,
                                  _ptr(workspace), workspace.numel(), _stream_ptr(stream)))
     return out
 

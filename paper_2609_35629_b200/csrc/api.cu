@@ -13,6 +13,7 @@ namespace {
 
 thread_local char g_cuda_error[256] = "";
 thread_local int g_launches = 0;
+thread_local int g_stage_mask = SANTAPP_STAGE_ALL;
 
 int cuda_fail(cudaError_t err, const char *where)
 {
@@ -142,6 +143,8 @@ const char *santapp_last_cuda_error(void) { return g_cuda_error; }
 
 int santapp_last_launch_count(void) { return g_launches; }
 
+void santapp_set_stage_mask(int mask) { g_stage_mask = mask & SANTAPP_STAGE_ALL; }
+
 int santapp_build_teams_sizes(const santapp_geom *geom, const int32_t *prompt_len_host, santapp_sizes *out)
 {
     int rc = check_geom(geom);
@@ -233,7 +236,8 @@ size_t santapp_dense_workspace_bytes(const santapp_geom *geom, const santapp_tea
 
 int santapp_decode_attn(const santapp_geom *geom, const santapp_teams *teams, const void *q, const void *k_suffix,
                         const void *v_suffix, const int32_t *suffix_len_dev, int32_t suffix_cap, int32_t n_sample,
-                        uint64_t seed, uint32_t step, uint32_t stream_base, float scale, float *out,
+                        uint64_t seed, uint32_t step, const uint32_t *step_dev, uint32_t stream_base, float scale,
+                        float *out,
                         const santapp_debug *dbg, void *workspace, size_t workspace_bytes, santapp_stream stream)
 {
     g_launches = 0;
@@ -268,14 +272,18 @@ int santapp_decode_attn(const santapp_geom *geom, const santapp_teams *teams, co
     rp.seed_lo = (uint32_t)(seed & 0xFFFFFFFFull);
     rp.seed_hi = (uint32_t)(seed >> 32);
     rp.step = step;
+    rp.step_dev = step_dev;
     rp.stream_base = stream_base;
     rp.scale = sc;
     rp.ctl = ctl;
     rp.n_pairs = L.n_pairs;
     rp.status = dbg ? dbg->status : nullptr;
-    cudaError_t err = launch_route_score(rp, teams->max_teams_per_seq, s);
-    if (err != cudaSuccess) return cuda_fail(err, "route_score launch");
-    ++g_launches;
+    cudaError_t err = cudaSuccess;
+    if (g_stage_mask & SANTAPP_STAGE_ROUTE) {
+        err = launch_route_score(rp, teams->max_teams_per_seq, s);
+        if (err != cudaSuccess) return cuda_fail(err, "route_score launch");
+        ++g_launches;
+    }
 
     SelectParams sp;
     sp.bv = rp.bv;
@@ -285,6 +293,7 @@ int santapp_decode_attn(const santapp_geom *geom, const santapp_teams *teams, co
     sp.seed_lo = rp.seed_lo;
     sp.seed_hi = rp.seed_hi;
     sp.step = step;
+    sp.step_dev = step_dev;
     sp.stream_base = stream_base;
     sp.sel_team = reinterpret_cast<int32_t *>(ws + L.sel_team);
     sp.sel_logc = reinterpret_cast<float *>(ws + L.sel_logc);
@@ -298,9 +307,11 @@ int santapp_decode_attn(const santapp_geom *geom, const santapp_teams *teams, co
     sp.dbg_sel_logc = dbg ? dbg->sel_logc : nullptr;
     sp.dbg_tau = dbg ? dbg->tau : nullptr;
     sp.dbg_union_rows = dbg ? dbg->union_rows : nullptr;
-    err = launch_select_plan(sp, teams->max_teams_per_seq, s);
-    if (err != cudaSuccess) return cuda_fail(err, "select_plan launch");
-    ++g_launches;
+    if (g_stage_mask & SANTAPP_STAGE_SELECT) {
+        err = launch_select_plan(sp, teams->max_teams_per_seq, s);
+        if (err != cudaSuccess) return cuda_fail(err, "select_plan launch");
+        ++g_launches;
+    }
 
     AttendParams ap;
     ap.bv = rp.bv;
@@ -317,9 +328,11 @@ int santapp_decode_attn(const santapp_geom *geom, const santapp_teams *teams, co
     ap.out = out;
     ap.status = rp.status;
     ap.min_rows_per_cta = 64;
-    err = launch_attend(ap, false, grid, s);
-    if (err != cudaSuccess) return cuda_fail(err, "attend launch");
-    ++g_launches;
+    if (g_stage_mask & SANTAPP_STAGE_ATTEND) {
+        err = launch_attend(ap, false, grid, s);
+        if (err != cudaSuccess) return cuda_fail(err, "attend launch");
+        ++g_launches;
+    }
     return SANTAPP_OK;
 }
 

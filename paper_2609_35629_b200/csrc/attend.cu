@@ -46,7 +46,7 @@ __global__ void __launch_bounds__(kAttendThreads, kAll ? 1 : 2)
 attend_kernel(AttendParams p)
 {
     __shared__ AttendShared<G> sh;
-    const int tid = threadIdx.x, lane = tid & 31;
+    const int tid = threadIdx.x;
     const int hw = tid >> 4, l16 = tid & 15;
 
     const int64_t total = p.plan.pair_row_prefix[p.n_pairs];
@@ -244,6 +244,7 @@ attend_kernel(AttendParams p)
         __syncthreads();
         if (sh.flag) {
             __threadfence();
+            if (tid == 0) p.ctl.attend_ticket[pair] = 0;              // every CTA of the pair has arrived
             const float *first = p.partials + (size_t)(c_lo + pair) * G * kPartialStride;
             // common scale per head, then weights per (slot, head)
             if (tid < G) {

@@ -56,6 +56,7 @@ struct RouteParams {
     double *y;                      // [n_q][teams_total] perturbed routing scores
     int n_sample;
     uint32_t seed_lo, seed_hi, step, stream_base;
+    const uint32_t *step_dev;       // nullable: added to step
     double scale;
     Control ctl;
     int n_pairs;
@@ -68,6 +69,7 @@ struct SelectParams {
     const double *y;
     int n_sample;
     uint32_t seed_lo, seed_hi, step, stream_base;
+    const uint32_t *step_dev;       // nullable: added to step
     int32_t *sel_team;              // [n_seqs][n_q][n_sample]
     float *sel_logc;                // [n_seqs][n_q][n_sample] natural log
     double *tau;                    // [n_seqs][n_q]

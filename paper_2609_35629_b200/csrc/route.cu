@@ -76,6 +76,7 @@ route_score_kernel(RouteParams p)
 
     const uint16_t *rep = p.rep_keys + ((size_t)j * p.bv.teams_total + team0) * kHeadDim;
     const int32_t *csr = p.team_row_start + (size_t)j * (p.bv.teams_total + p.bv.n_seqs) + team0 + b;
+    const uint32_t step = p.step + (p.step_dev ? *p.step_dev : 0u);
 
 #pragma unroll 1
     for (int it = 0; it < 2; ++it) {
@@ -113,7 +114,7 @@ route_score_kernel(RouteParams p)
             const double phi = log((double)n_g) + dot * p.scale;
             const uint32_t head = (uint32_t)(j * G + h);
             const uint4 words = philox4x32_10(
-                make_uint4((uint32_t)g >> 2, p.step, head, p.stream_base + (uint32_t)b), p.seed_lo, p.seed_hi);
+                make_uint4((uint32_t)g >> 2, step, head, p.stream_base + (uint32_t)b), p.seed_lo, p.seed_hi);
             const double y = phi + gumbel_from_word(pick_word(words, g & 3));
             p.y[(size_t)head * p.bv.teams_total + team0 + g] = y;
         }
@@ -166,6 +167,7 @@ __device__ void publish_pair_prefix(const SelectParams &p, int *flag_smem, int *
     __syncthreads();
     if (!*flag_smem) return;
     __threadfence();
+    if (threadIdx.x == 0) *p.ctl.plan_ticket = 0;                  // every pair has arrived
     int64_t carry = 0;
     for (int base = 0; base < p.n_pairs; base += (int)blockDim.x) {
         const int i = base + (int)threadIdx.x;
@@ -297,8 +299,9 @@ select_plan_kernel(SelectParams p)
                 rank += (ka > k) || (ka == k && cand_id[a] < id);
             }
             // phi = Y - G with the same draw the scorer used
+            const uint32_t step = p.step + (p.step_dev ? *p.step_dev : 0u);
             const uint4 words = philox4x32_10(
-                make_uint4((uint32_t)id >> 2, p.step, (uint32_t)head, p.stream_base + (uint32_t)b),
+                make_uint4((uint32_t)id >> 2, step, (uint32_t)head, p.stream_base + (uint32_t)b),
                 p.seed_lo, p.seed_hi);
             const double phi = key_to_double(k) - gumbel_from_word(pick_word(words, id & 3));
             const double x = phi - tau;
@@ -325,6 +328,7 @@ select_plan_kernel(SelectParams p)
     __syncthreads();
     if (!sh.is_last) return;
     __threadfence();
+    if (tid == 0) p.ctl.select_ticket[pair] = 0;                   // all G heads of the pair have arrived
 
     const int cap = p.plan.seg_cap;
     int32_t *seg_prefix = p.plan.seg_prefix + (size_t)pair * (cap + 1);
@@ -445,9 +449,13 @@ template <int G>
 cudaError_t launch_select_plan_g(const SelectParams &p, int max_teams, cudaStream_t s)
 {
     const size_t smem = sizeof(unsigned long long) * (size_t)max_teams + 64;
-    cudaError_t err = cudaFuncSetAttribute(select_plan_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                           (int)smem);
-    if (err != cudaSuccess) return err;
+    static thread_local size_t smem_set = 0;             // raise the limit once per thread and size
+    if (smem > smem_set) {
+        cudaError_t err = cudaFuncSetAttribute(select_plan_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                               (int)smem);
+        if (err != cudaSuccess) return err;
+        smem_set = smem;
+    }
     select_plan_kernel<G><<<dim3(G, p.n_pairs), kSelectThreads, smem, s>>>(p);
     return cudaGetLastError();
 }

@@ -71,8 +71,8 @@ def test_bad_prompt_length_is_rejected(lib):
 def test_null_arguments_return_invalid_arg_without_touching_a_gpu(lib):
     g = sp.Geometry(1, 28, 4).c()
     t = sp.CTeams()                                                # all null
-    rc = lib.santapp_decode_attn(ctypes.byref(g), ctypes.byref(t), None, None, None, None, 0, 32, 0, 0, 0, 0.0,
-                                 None, None, None, 0, None)
+    rc = lib.santapp_decode_attn(ctypes.byref(g), ctypes.byref(t), None, None, None, None, 0, 32, 0, 0, None, 0,
+                                 0.0, None, None, None, 0, None)
     assert rc == sp.SANTAPP_ERR_INVALID_ARG
     rc = lib.santapp_dense_decode_attn(ctypes.byref(g), ctypes.byref(t), None, None, None, None, 0, 0.0, None,
                                        None, 0, None)

@@ -233,3 +233,40 @@ def test_qwen_32k_batch8_concentrated_sampled_sequences():
     layer = layer_for("qwen_b8", synth.spec_qwen_b8, n_steps=2)
     check_sparse_step(layer, 0, K=64, seqs=[0, 5])
     check_dense_step(layer, 1, seqs=[3])
+
+
+def test_device_side_step_offset_equals_explicit_step():
+    """step = 3 with a device-side offset of 4 draws the same sample as step = 7."""
+    layer = layer_for("small", synth.spec_small_gqa)
+    spec = layer.spec
+    q = sp.bf16_bits_to_cuda(synth.make_queries(spec, layer.data, 0))
+    sl = torch.from_numpy(spec.suffix_len(0)).cuda()
+    d1 = sp.DebugBuffers(layer.geom, 8, "cuda")
+    d2 = sp.DebugBuffers(layer.geom, 8, "cuda")
+    off = torch.tensor([4], dtype=torch.int32, device="cuda")
+    o1 = sp.santapp_decode_attn(layer.geom, layer.teams, q, layer.k_suffix, layer.v_suffix, sl, 8, 11, 7, debug=d1)
+    o2 = sp.santapp_decode_attn(layer.geom, layer.teams, q, layer.k_suffix, layer.v_suffix, sl, 8, 11, 3, debug=d2,
+                                step_dev=off)
+    torch.cuda.synchronize()
+    assert torch.equal(d1.sel_idx, d2.sel_idx)
+    assert torch.allclose(o1, o2, rtol=0, atol=1e-6)
+
+
+def test_stage_mask_reruns_one_stage_on_the_same_workspace():
+    layer = layer_for("small", synth.spec_small_gqa)
+    spec = layer.spec
+    q = sp.bf16_bits_to_cuda(synth.make_queries(spec, layer.data, 1))
+    sl = torch.from_numpy(spec.suffix_len(1)).cuda()
+    ws = torch.empty(sp.santapp_decode_workspace_bytes(layer.geom, layer.teams, 8), dtype=torch.uint8, device="cuda")
+    args = (layer.geom, layer.teams, q, layer.k_suffix, layer.v_suffix, sl, 8, 5, 1)
+    full = sp.santapp_decode_attn(*args, workspace=ws).clone()
+    assert sp.santapp_last_launch_count() == 3
+    try:
+        for mask in (sp.STAGE_ATTEND, sp.STAGE_SELECT, sp.STAGE_ROUTE, sp.STAGE_ATTEND):
+            sp.santapp_set_stage_mask(mask)
+            again = sp.santapp_decode_attn(*args, workspace=ws)
+            assert sp.santapp_last_launch_count() == 1
+            torch.cuda.synchronize()
+            assert torch.allclose(full, again, rtol=0, atol=1e-6)
+    finally:
+        sp.santapp_set_stage_mask(sp.STAGE_ALL)
