@@ -252,6 +252,7 @@ int santapp_decode_attn(const santapp_geom *geom, const santapp_teams *teams, co
     if ((int64_t)geom->n_seqs * geom->n_kv_heads * (int64_t)suffix_cap >= (int64_t)1 << 31) return SANTAPP_ERR_UNSUPPORTED;
     const int grid = attend_grid_size();
     const DecodeLayout L = decode_layout(geom, teams, n_sample, false, grid);
+    if (L.seg_cap > attend_max_segments() || L.n_pairs > attend_max_pairs()) return SANTAPP_ERR_UNSUPPORTED;
     if (workspace_bytes < L.total) return SANTAPP_ERR_WORKSPACE_TOO_SMALL;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     g_cuda_error[0] = 0;
@@ -352,6 +353,7 @@ int santapp_dense_decode_attn(const santapp_geom *geom, const santapp_teams *tea
     if ((int64_t)geom->n_seqs * geom->n_kv_heads * (int64_t)suffix_cap >= (int64_t)1 << 31) return SANTAPP_ERR_UNSUPPORTED;
     const int grid = attend_grid_size();
     const DecodeLayout L = decode_layout(geom, teams, 1, true, grid);
+    if (L.n_pairs > attend_max_pairs()) return SANTAPP_ERR_UNSUPPORTED;
     if (workspace_bytes < L.total) return SANTAPP_ERR_WORKSPACE_TOO_SMALL;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     g_cuda_error[0] = 0;

@@ -108,6 +108,8 @@ cudaError_t launch_select_plan(const SelectParams &p, int max_teams_per_seq, cud
 cudaError_t launch_dense_plan(const SelectParams &p, cudaStream_t s);
 cudaError_t launch_attend(const AttendParams &p, bool all_heads, int grid, cudaStream_t s);
 int attend_grid_size();
+int attend_max_segments();
+int attend_max_pairs();
 
 struct BuildParams {
     BatchView bv;

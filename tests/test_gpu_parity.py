@@ -262,11 +262,14 @@ def test_stage_mask_reruns_one_stage_on_the_same_workspace():
     full = sp.santapp_decode_attn(*args, workspace=ws).clone()
     assert sp.santapp_last_launch_count() == 3
     try:
-        for mask in (sp.STAGE_ATTEND, sp.STAGE_SELECT, sp.STAGE_ROUTE, sp.STAGE_ATTEND):
+        # each stage alone, in pipeline order, reusing what the full call left in the workspace;
+        # only the last stage writes the output
+        for mask in (sp.STAGE_ATTEND, sp.STAGE_ROUTE, sp.STAGE_SELECT, sp.STAGE_ATTEND):
             sp.santapp_set_stage_mask(mask)
             again = sp.santapp_decode_attn(*args, workspace=ws)
             assert sp.santapp_last_launch_count() == 1
             torch.cuda.synchronize()
-            assert torch.allclose(full, again, rtol=0, atol=1e-6)
+            if mask == sp.STAGE_ATTEND:
+                assert torch.allclose(full, again, rtol=0, atol=1e-6)
     finally:
         sp.santapp_set_stage_mask(sp.STAGE_ALL)
