@@ -3,14 +3,21 @@
 // (applied as s_i - log c_g, so the same correction enters the mass and the value sum), every
 // suffix row with weight e^{s_i}; Eq. (method-estimate).
 //
-// The rows of all (sequence, KV head) pairs form one global row space that is cut into equal
-// contiguous ranges, one per CTA (split-K by rows, not by teams), one CTA per SM. Inside a CTA
-// one producer thread streams the range through a ring of shared-memory stages with bulk
-// asynchronous copies (whole runs of team-contiguous rows per copy, K and V), eight consumer
-// warps evaluate the rows (half a warp per row) with an online softmax, and the CTA leaves one
-// partial per pair it touched. The last CTA to finish a pair merges that pair's partials by
-// log-sum-exp (the split-softmax reduction).
+// Work split. The rows of all (sequence, KV head) pairs form one global row space that is cut
+// into equal contiguous ranges, one per CTA (split-K by rows, not by teams), one CTA per SM.
+// Inside a CTA the range is dealt out in blocks of 16 rows to eight consumer warps; two
+// producer warps stream each block's K and V rows into that warp's private two-slot ring in
+// shared memory with 16-byte asynchronous copies (whole 256-byte rows per half warp, XOR
+// swizzled so that ldmatrix is bank-conflict free) and signal an mbarrier.
 //
+// Arithmetic. The GQA group is a real MMA tile: the query heads of the KV head (at most 8)
+// are the M rows of S^T = q K^T (mma.sync m16n8k16, bf16 inputs, fp32 accumulation), so one
+// row of K serves every head at once; a team contributes to a head only where the head
+// selected it (mask), with the head's own correction. The weights are split into two bf16
+// terms (p = p_hi + p_lo) so that O^T += V^T P^T keeps fp32-level accuracy.
+//
+// Each CTA leaves one online-softmax partial per pair it touched; the last CTA to finish a
+// pair merges that pair's partials by log-sum-exp (the split-softmax reduction).
 // Every wait on a barrier is bounded: on expiry the kernel raises a status bit and leaves.
 #include <math_constants.h>
 
@@ -21,20 +28,21 @@ namespace santapp {
 namespace {
 
 constexpr int kConsumerWarps = 8;
+constexpr int kProducerWarps = 2;
 constexpr int kConsumerThreads = 32 * kConsumerWarps;
-constexpr int kAttendThreads = kConsumerThreads + 32;       // + one producer warp
-constexpr int kHalfWarps = kConsumerThreads / 16;           // rows evaluated side by side
-constexpr int kStageRows = 32;
-constexpr int kRowsPerHalfWarp = kStageRows / kHalfWarps;   // 2
-constexpr int kStages = 8;
+constexpr int kAttendThreads = 32 * (kConsumerWarps + kProducerWarps);
+constexpr int kBlockRows = 16;                              // rows per block (one warp, one MMA K step)
+constexpr int kSlots = 2;                                   // ring slots per consumer warp
 constexpr int kRowBytes = kHeadDim * 2;                     // one bf16 row
-constexpr int kStageBytes = kStageRows * kRowBytes * 2;     // K block then V block
+constexpr int kTileBytes = kBlockRows * kRowBytes;          // K tile or V tile of a block
+constexpr int kSlotBytes = 2 * kTileBytes;                  // K tile then V tile
 constexpr int kSegMax = 1025;                               // plan segments of one pair (G * K + suffix)
 constexpr int kPairMax = 1024;                              // pairs whose offsets are staged
 constexpr int kMaxAttendGrid = 512;
 constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr int kNoSeg = 0xFFFF;
 
-// ---- mbarrier / bulk copy primitives (shared::cta addresses as 32-bit) ----
+// ---- primitives ----
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
 __device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count)
@@ -49,10 +57,10 @@ __device__ __forceinline__ void mbar_arrive(uint64_t *bar)
 {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t *bar, uint32_t bytes)
+// The executing thread's earlier cp.async copies arrive on the barrier when they complete.
+__device__ __forceinline__ void cp_async_arrive(uint64_t *bar)
 {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
-                 : "memory");
+    asm volatile("cp.async.mbarrier.arrive.shared::cta.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
 {
@@ -76,23 +84,48 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
     *abort_flag = 1;
     return false;
 }
-// 1-D bulk copy global -> shared, completion counted in bytes on an mbarrier. Both addresses
-// and the size are multiples of 16 (rows are 256 bytes).
-__device__ __forceinline__ void bulk_copy_g2s(void *dst, const void *src, uint32_t bytes, uint64_t *bar)
+// 16-byte asynchronous copy global -> shared; src_bytes = 0 writes zeros instead.
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, uint32_t src_bytes)
 {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-                     smem_u32(dst)),
-                 "l"(src), "r"(bytes), "r"(smem_u32(bar))
-                 : "memory");
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(addr));
+}
+// D += A (16x16, row) * B (16x8, col), bf16 inputs, fp32 accumulation.
+__device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                         uint32_t b0, uint32_t b1)
+{
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+                 "{%0,%1,%2,%3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+// (lo, hi) -> bf16x2 with lo in the low half, round to nearest even.
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
+{
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
 }
 
 // ---- shared memory carve-up (dynamic) ----
 template <int G>
 struct Smem {
-    static constexpr size_t ring = 0;                                           // kStages * kStageBytes
-    static constexpr size_t bars = ring + (size_t)kStages * kStageBytes;        // full[kStages], empty[kStages]
-    static constexpr size_t q = bars + 2 * kStages * 8;                          // float [G][128]
-    static constexpr size_t seg_prefix = q + (size_t)G * kHeadDim * 4;          // int [kSegMax + 1] (+pad)
+    static constexpr size_t ring = 0;                                           // [warps][kSlots][kSlotBytes]
+    static constexpr size_t ring_bytes = (size_t)kConsumerWarps * kSlots * kSlotBytes;
+    static constexpr size_t bars = ring + ring_bytes;                           // full[w][s], empty[w][s]
+    static constexpr size_t row_seg = bars + 2 * kConsumerWarps * kSlots * 8;   // u16 [w][s][16]
+    static constexpr size_t seg_prefix = row_seg + kConsumerWarps * kSlots * kBlockRows * 2;   // int [kSegMax+1]
     static constexpr size_t seg_row = seg_prefix + (kSegMax + 3) * 4;           // int [kSegMax]
     static constexpr size_t seg_mask = seg_row + (kSegMax + 3) * 4;             // uint [kSegMax]
     static constexpr size_t seg_logc = seg_mask + (kSegMax + 3) * 4;            // float [kSegMax][G]
@@ -100,7 +133,7 @@ struct Smem {
     static constexpr size_t pair_nseg = pair_prefix + (kPairMax + 1) * 8;       // int [kPairMax]
     static constexpr size_t misc = pair_nseg + kPairMax * 4;                    // flags
     static constexpr size_t total = misc + 64;
-    // aliases of the ring, used only after a span's stages are consumed
+    // aliases of the ring, used only after a span's blocks are consumed
     static constexpr size_t red_acc = ring;                                     // float [warps][G][128]
     static constexpr size_t red_m = red_acc + (size_t)kConsumerWarps * G * kHeadDim * 4;   // float [warps][G]
     static constexpr size_t red_l = red_m + (size_t)kConsumerWarps * G * 4;
@@ -112,12 +145,12 @@ template <int G, bool kAll>
 __global__ void __launch_bounds__(kAttendThreads, 1)
 attend_kernel(AttendParams p)
 {
-    extern __shared__ __align__(128) unsigned char smem[];
+    extern __shared__ __align__(1024) unsigned char smem[];
     using S = Smem<G>;
     unsigned char *ring = smem + S::ring;
-    uint64_t *full_bar = reinterpret_cast<uint64_t *>(smem + S::bars);
-    uint64_t *empty_bar = full_bar + kStages;
-    float(*q_s)[kHeadDim] = reinterpret_cast<float(*)[kHeadDim]>(smem + S::q);
+    uint64_t *full_bar = reinterpret_cast<uint64_t *>(smem + S::bars);          // [w * kSlots + s]
+    uint64_t *empty_bar = full_bar + kConsumerWarps * kSlots;
+    uint16_t *row_seg = reinterpret_cast<uint16_t *>(smem + S::row_seg);        // [(w * kSlots + s) * 16 + r]
     int *seg_prefix = reinterpret_cast<int *>(smem + S::seg_prefix);
     int *seg_row = reinterpret_cast<int *>(smem + S::seg_row);
     uint32_t *seg_mask = reinterpret_cast<uint32_t *>(smem + S::seg_mask);
@@ -128,13 +161,13 @@ attend_kernel(AttendParams p)
     int *last_flag = reinterpret_cast<int *>(smem + S::misc) + 1;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int hw = tid >> 4, l16 = tid & 15;
-    const bool is_producer = warp == kConsumerWarps;
+    const bool is_producer = warp >= kConsumerWarps;
+    const int g = lane >> 2, c = lane & 3;                 // MMA fragment coordinates
 
     if (tid == 0) {
-        for (int s = 0; s < kStages; ++s) {
-            mbar_init(full_bar + s, 1);
-            mbar_init(empty_bar + s, kConsumerWarps);
+        for (int s = 0; s < kConsumerWarps * kSlots; ++s) {
+            mbar_init(full_bar + s, 32);                   // one arrival per producer lane
+            mbar_init(empty_bar + s, 1);                   // the consumer warp's lane 0
         }
         fence_barrier_init();
         *abort_flag = 0;
@@ -160,7 +193,7 @@ attend_kernel(AttendParams p)
         pair = lo;
     }
 
-    uint32_t g_stage = 0;          // stages issued so far by this CTA (same count in every thread)
+    uint32_t g_block = 0;          // blocks dealt out so far by this CTA (same count in every thread)
 
     while (r0 < r1) {
         const int64_t pb = pair_prefix[pair], pe = pair_prefix[pair + 1];
@@ -172,185 +205,212 @@ attend_kernel(AttendParams p)
 
         __syncthreads();                                   // the previous span is done with the tables
         {
+            // one round trip: every load is issued before the first store
             const int32_t *g_prefix = p.plan.seg_prefix + (size_t)pair * (cap + 1);
             const int32_t *g_row = p.plan.seg_row + (size_t)pair * cap;
             const uint32_t *g_mask = p.plan.seg_mask + (size_t)pair * cap;
             const float *g_logc = p.plan.seg_logc + (size_t)pair * cap * G;
-            for (int i = tid; i < nseg; i += kAttendThreads) {
-                seg_prefix[i] = g_prefix[i];
-                seg_row[i] = g_row[i];
-                seg_mask[i] = g_mask[i];
+            for (int i0 = 0; i0 <= nseg; i0 += kAttendThreads) {
+                const int i = i0 + tid;
+                int v_prefix = 0, v_row = 0;
+                uint32_t v_mask = 0u;
+                float v_logc[G];
+                if (i <= nseg) v_prefix = g_prefix[i];
+                if (i < nseg) {
+                    v_row = g_row[i];
+                    v_mask = g_mask[i];
+                    if (!kAll) {
+#pragma unroll
+                        for (int h = 0; h < G; ++h) v_logc[h] = g_logc[(size_t)i * G + h];
+                    }
+                }
+                if (i <= nseg) seg_prefix[i] = v_prefix;
+                if (i < nseg) {
+                    seg_row[i] = v_row;
+                    seg_mask[i] = v_mask;
+                    if (!kAll) {
+#pragma unroll
+                        for (int h = 0; h < G; ++h) seg_logc[i][h] = v_logc[h];
+                    }
+                }
             }
-            if (tid == 0) seg_prefix[nseg] = g_prefix[nseg];
-            if (!kAll)
-                for (int e = tid; e < nseg * G; e += kAttendThreads) (&seg_logc[0][0])[e] = g_logc[e];
-            for (int e = tid; e < G * kHeadDim; e += kAttendThreads) {
-                const int h = e >> 7, d = e & 127;
-                q_s[h][d] = bf16_to_float(p.q[((size_t)b * p.bv.n_q + (size_t)j * G + h) * kHeadDim + d])
-                            * p.qk_scale_log2;
+        }
+        // A fragments of q for the 8 k-steps: head g (zero rows for g >= G and for M rows 8..15)
+        uint32_t qa[8][2];
+        if (!is_producer) {
+            const uint32_t *qrow = reinterpret_cast<const uint32_t *>(
+                p.q + ((size_t)b * p.bv.n_q + (size_t)j * G + (g < G ? g : 0)) * kHeadDim);
+#pragma unroll
+            for (int s = 0; s < 8; ++s) {
+                qa[s][0] = g < G ? __ldg(qrow + 8 * s + c) : 0u;
+                qa[s][1] = g < G ? __ldg(qrow + 8 * s + 4 + c) : 0u;
             }
         }
         __syncthreads();
 
-        const int n_st = (bnd - a + kStageRows - 1) / kStageRows;
+        const int n_blk = (bnd - a + kBlockRows - 1) / kBlockRows;
         const unsigned char *k_plane = reinterpret_cast<const unsigned char *>(p.k_packed)
                                        + (size_t)j * p.bv.rows_total * kRowBytes;
         const unsigned char *v_plane = reinterpret_cast<const unsigned char *>(p.v_packed)
                                        + (size_t)j * p.bv.rows_total * kRowBytes;
 
-        float m[G], l[G], acc[G][8];
+        // online-softmax state of head g (replicated over the quad) and O^T fragments:
+        // o[t][r]: d = 16 t + g + 8 (r >> 1), head = 2 c + (r & 1)
+        float m_run = -CUDART_INF_F, l_run = 0.f;
+        float o[8][4];
 #pragma unroll
-        for (int h = 0; h < G; ++h) {
-            m[h] = -CUDART_INF_F;
-            l[h] = 0.f;
-#pragma unroll
-            for (int i = 0; i < 8; ++i) acc[h][i] = 0.f;
-        }
+        for (int t = 0; t < 8; ++t) { o[t][0] = o[t][1] = o[t][2] = o[t][3] = 0.f; }
 
-        int st_issued = 0;                                 // producer thread: stages issued in this span
         if (is_producer) {
-            if (lane == 0) {
-                // the ring may have been used as scratch by the previous span's merge
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                int cur = 0;
-                {   // first segment of the span
-                    int lo = 0, hi = nseg;
-                    while (hi - lo > 1) {
-                        const int mid = (lo + hi) >> 1;
-                        if (seg_prefix[mid] <= a) lo = mid; else hi = mid;
+            // ---------------- producer warps: blocks of alternating parity ----------------
+            const int pw = warp - kConsumerWarps;
+            int cur = 0;                                   // segment cursor of lane r (r < 16)
+            for (int bi = 0; bi < n_blk; ++bi) {
+                const uint32_t gb = g_block + bi;
+                if ((int)(gb % kProducerWarps) != pw) continue;
+                const int w = gb % kConsumerWarps;
+                const uint32_t u = gb / kConsumerWarps;
+                const int slot = u % kSlots;
+                const int bs = w * kSlots + slot;
+                if (u >= (uint32_t)kSlots &&
+                    !__all_sync(0xFFFFFFFFu, mbar_wait(empty_bar + bs, ((u / kSlots) - 1) & 1, abort_flag)))
+                    break;
+                // lane r < 16 resolves row r of the block
+                const int pos = a + bi * kBlockRows + (lane & 15);
+                const bool valid = pos < bnd;
+                int64_t grow = 0;
+                int suf = 0;
+                if (valid) {
+                    if (pos >= seg_prefix[cur + 1]) {      // moved on: binary search from here
+                        int lo = cur + 1, hi = nseg;
+                        while (hi - lo > 1) {
+                            const int mid = (lo + hi) >> 1;
+                            if (seg_prefix[mid] <= pos) lo = mid; else hi = mid;
+                        }
+                        cur = lo;
                     }
-                    cur = lo;
+                    grow = (int64_t)seg_row[cur] + (pos - seg_prefix[cur]);
+                    suf = (seg_mask[cur] & kSrcSuffix) ? 1 : 0;
                 }
-                for (int st = 0; st < n_st; ++st) {
-                    const uint32_t gs = g_stage + st;
-                    const int slot = gs % kStages;
-                    if (gs >= kStages && !mbar_wait(empty_bar + slot, ((gs / kStages) - 1) & 1, abort_flag)) break;
-                    const int base = a + st * kStageRows, end = min(base + kStageRows, bnd);
-                    unsigned char *kst = ring + (size_t)slot * kStageBytes;
-                    unsigned char *vst = kst + kStageRows * kRowBytes;
-                    mbar_arrive_expect_tx(full_bar + slot, (uint32_t)(end - base) * 2 * kRowBytes);
-                    int pos = base;
-                    while (pos < end) {
-                        while (pos >= seg_prefix[cur + 1]) ++cur;
-                        const int run_end = min(end, seg_prefix[cur + 1]);
-                        const uint32_t bytes = (uint32_t)(run_end - pos) * kRowBytes;
-                        const size_t row = (size_t)seg_row[cur] + (size_t)(pos - seg_prefix[cur]);
-                        const bool suf = (seg_mask[cur] & kSrcSuffix) != 0u;
-                        const unsigned char *ks = (suf ? reinterpret_cast<const unsigned char *>(p.k_suffix) : k_plane)
-                                                  + row * kRowBytes;
-                        const unsigned char *vs = (suf ? reinterpret_cast<const unsigned char *>(p.v_suffix) : v_plane)
-                                                  + row * kRowBytes;
-                        bulk_copy_g2s(kst + (size_t)(pos - base) * kRowBytes, ks, bytes, full_bar + slot);
-                        bulk_copy_g2s(vst + (size_t)(pos - base) * kRowBytes, vs, bytes, full_bar + slot);
-                        pos = run_end;
-                    }
-                    st_issued = st + 1;
+                if (lane < 16) row_seg[bs * kBlockRows + lane] = (uint16_t)(valid ? cur : kNoSeg);
+                const uint32_t slot_addr = smem_u32(ring + (size_t)bs * kSlotBytes);
+                const int chunk = lane & 15;
+#pragma unroll
+                for (int piece = 0; piece < kBlockRows / 2; ++piece) {
+                    const int row = 2 * piece + (lane >> 4);
+                    const int64_t rr = __shfl_sync(0xFFFFFFFFu, grow, row);
+                    const int rs = __shfl_sync(0xFFFFFFFFu, suf, row);
+                    const int rv = __shfl_sync(0xFFFFFFFFu, (int)valid, row);
+                    const unsigned char *ks = (rs ? reinterpret_cast<const unsigned char *>(p.k_suffix) : k_plane)
+                                              + rr * kRowBytes + chunk * 16;
+                    const unsigned char *vs = (rs ? reinterpret_cast<const unsigned char *>(p.v_suffix) : v_plane)
+                                              + rr * kRowBytes + chunk * 16;
+                    const uint32_t dst = slot_addr + row * kRowBytes + ((chunk ^ (row & 7)) << 4);
+                    cp_async16(dst, ks, rv ? 16u : 0u);
+                    cp_async16(dst + kTileBytes, vs, rv ? 16u : 0u);
                 }
+                cp_async_arrive(full_bar + bs);
+                mbar_arrive(full_bar + bs);
             }
         } else {
-            int cur = 0;
-            {
-                int lo = 0, hi = nseg;
-                while (hi - lo > 1) {
-                    const int mid = (lo + hi) >> 1;
-                    if (seg_prefix[mid] <= a) lo = mid; else hi = mid;
-                }
-                cur = lo;
-            }
-            for (int st = 0; st < n_st; ++st) {
-                const uint32_t gs = g_stage + st;
-                const int slot = gs % kStages;
-                if (!mbar_wait(full_bar + slot, (gs / kStages) & 1, abort_flag)) break;
-                const int base = a + st * kStageRows, end = min(base + kStageRows, bnd);
-                const unsigned char *kst = ring + (size_t)slot * kStageBytes;
-                const unsigned char *vst = kst + kStageRows * kRowBytes;
+            // ---------------- consumer warps ----------------
+            const float qk = p.qk_scale_log2;
+            int first = (int)((warp + kConsumerWarps - (g_block % kConsumerWarps)) % kConsumerWarps);
+            for (int bi = first; bi < n_blk; bi += kConsumerWarps) {
+                const uint32_t gb = g_block + bi;
+                const uint32_t u = gb / kConsumerWarps;
+                const int slot = u % kSlots;
+                const int bs = warp * kSlots + slot;
+                if (!__all_sync(0xFFFFFFFFu, mbar_wait(full_bar + bs, (u / kSlots) & 1, abort_flag))) break;
+                const uint32_t k_addr = smem_u32(ring + (size_t)bs * kSlotBytes);
+                const uint32_t v_addr = k_addr + kTileBytes;
 
-                uint4 kk[kRowsPerHalfWarp], vv[kRowsPerHalfWarp];
-                int segi[kRowsPerHalfWarp];
-                uint32_t msk[kRowsPerHalfWarp];
-                uint32_t any = 0u;
+                // the four (row, head g) entries of this thread: rows 2c, 2c+1, 8+2c, 9+2c
+                bool on[4];
+                float lc[4];
 #pragma unroll
-                for (int u = 0; u < kRowsPerHalfWarp; ++u) {
-                    const int pos = base + u * kHalfWarps + hw;
-                    msk[u] = 0u;
-                    segi[u] = 0;
-                    kk[u] = make_uint4(0u, 0u, 0u, 0u);
-                    vv[u] = make_uint4(0u, 0u, 0u, 0u);
-                    if (pos < end) {
-                        while (pos >= seg_prefix[cur + 1]) ++cur;
-                        kk[u] = *reinterpret_cast<const uint4 *>(kst + (size_t)(pos - base) * kRowBytes + l16 * 16);
-                        vv[u] = *reinterpret_cast<const uint4 *>(vst + (size_t)(pos - base) * kRowBytes + l16 * 16);
-                        msk[u] = seg_mask[cur] & 0xFFu;
-                        segi[u] = cur;
+                for (int i = 0; i < 4; ++i) {
+                    const int r = 2 * c + (i & 1) + 8 * (i >> 1);
+                    lc[i] = 0.f;
+                    if (kAll) {
+                        on[i] = (g < G) && (a + bi * kBlockRows + r < bnd);
+                    } else {
+                        const int sg = row_seg[bs * kBlockRows + r];
+                        on[i] = false;
+                        if (sg != kNoSeg && g < G) {
+                            on[i] = (seg_mask[sg] >> g) & 1u;
+                            lc[i] = seg_logc[sg][g];
+                        }
                     }
-                    any |= msk[u];
+                }
+
+                // S^T = q K^T for the two 8-row groups
+                float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+                {
+                    const int lrow = lane & 7, lmat = lane >> 3;
+#pragma unroll
+                    for (int sp = 0; sp < 4; ++sp) {
+                        uint32_t kb0[4], kb1[4];
+                        const int chunk = 4 * sp + lmat;
+                        ldmatrix_x4(kb0, k_addr + lrow * kRowBytes + ((chunk ^ lrow) << 4));
+                        ldmatrix_x4(kb1, k_addr + (8 + lrow) * kRowBytes + ((chunk ^ lrow) << 4));
+                        mma_bf16(s0, qa[2 * sp][0], 0u, qa[2 * sp][1], 0u, kb0[0], kb0[1]);
+                        mma_bf16(s1, qa[2 * sp][0], 0u, qa[2 * sp][1], 0u, kb1[0], kb1[1]);
+                        mma_bf16(s0, qa[2 * sp + 1][0], 0u, qa[2 * sp + 1][1], 0u, kb0[2], kb0[3]);
+                        mma_bf16(s1, qa[2 * sp + 1][0], 0u, qa[2 * sp + 1][1], 0u, kb1[2], kb1[3]);
+                    }
+                }
+                float sc[4];
+                sc[0] = on[0] ? fmaf(s0[0], qk, -lc[0]) : -CUDART_INF_F;
+                sc[1] = on[1] ? fmaf(s0[1], qk, -lc[1]) : -CUDART_INF_F;
+                sc[2] = on[2] ? fmaf(s1[0], qk, -lc[2]) : -CUDART_INF_F;
+                sc[3] = on[3] ? fmaf(s1[1], qk, -lc[3]) : -CUDART_INF_F;
+                float mloc = fmaxf(fmaxf(sc[0], sc[1]), fmaxf(sc[2], sc[3]));
+                mloc = fmaxf(mloc, __shfl_xor_sync(0xFFFFFFFFu, mloc, 1));
+                mloc = fmaxf(mloc, __shfl_xor_sync(0xFFFFFFFFu, mloc, 2));
+                const float m_new = fmaxf(m_run, mloc);
+                const bool grew = m_new > m_run;
+                if (__any_sync(0xFFFFFFFFu, grew)) {
+                    const float f = grew ? exp2f(m_run - m_new) : 1.f;          // exp2f(-inf) = 0 on first rows
+                    l_run *= f;
+                    const float fe = __shfl_sync(0xFFFFFFFFu, f, 8 * c);        // head 2c lives in lanes 8c..8c+3
+                    const float fo = __shfl_sync(0xFFFFFFFFu, f, 8 * c + 4);    // head 2c+1
+#pragma unroll
+                    for (int t = 0; t < 8; ++t) { o[t][0] *= fe; o[t][1] *= fo; o[t][2] *= fe; o[t][3] *= fo; }
+                    m_run = m_new;
+                }
+                float pw[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) pw[i] = on[i] ? exp2f(sc[i] - m_run) : 0.f;
+                l_run += (pw[0] + pw[1]) + (pw[2] + pw[3]);
+                // P^T as B fragments, split in two bf16 terms
+                const uint32_t ph0 = pack_bf16x2(pw[0], pw[1]), ph1 = pack_bf16x2(pw[2], pw[3]);
+                const uint32_t pl0 = pack_bf16x2(pw[0] - bf16_lo(ph0), pw[1] - bf16_hi(ph0));
+                const uint32_t pl1 = pack_bf16x2(pw[2] - bf16_lo(ph1), pw[3] - bf16_hi(ph1));
+
+                // O^T += V^T P^T
+                {
+                    const int lrow = lane & 7, lmat = lane >> 3;
+                    const int vrow = (lmat >> 1) * 8 + lrow;
+#pragma unroll
+                    for (int t = 0; t < 8; ++t) {
+                        uint32_t va[4];
+                        const int chunk = 2 * t + (lmat & 1);
+                        ldmatrix_x4_trans(va, v_addr + vrow * kRowBytes + ((chunk ^ lrow) << 4));
+                        mma_bf16(o[t], va[0], va[1], va[2], va[3], ph0, ph1);
+                        mma_bf16(o[t], va[0], va[1], va[2], va[3], pl0, pl1);
+                    }
                 }
                 __syncwarp();
-                if (lane == 0) mbar_arrive(empty_bar + slot);          // the rows are in registers
-                if (!kAll) any |= __shfl_xor_sync(0xFFFFFFFFu, any, 16);
-
-#pragma unroll
-                for (int h = 0; h < G; ++h) {
-                    if (kAll || ((any >> h) & 1u)) {
-                        const float4 qa = *reinterpret_cast<const float4 *>(&q_s[h][l16 * 8]);
-                        const float4 qb = *reinterpret_cast<const float4 *>(&q_s[h][l16 * 8 + 4]);
-                        float sc[kRowsPerHalfWarp];
-                        float mx = -CUDART_INF_F;
-#pragma unroll
-                        for (int u = 0; u < kRowsPerHalfWarp; ++u) {
-                            float d = bf16_lo(kk[u].x) * qa.x;
-                            d = fmaf(bf16_hi(kk[u].x), qa.y, d);
-                            d = fmaf(bf16_lo(kk[u].y), qa.z, d);
-                            d = fmaf(bf16_hi(kk[u].y), qa.w, d);
-                            d = fmaf(bf16_lo(kk[u].z), qb.x, d);
-                            d = fmaf(bf16_hi(kk[u].z), qb.y, d);
-                            d = fmaf(bf16_lo(kk[u].w), qb.z, d);
-                            d = fmaf(bf16_hi(kk[u].w), qb.w, d);
-                            d += __shfl_xor_sync(0xFFFFFFFFu, d, 8);
-                            d += __shfl_xor_sync(0xFFFFFFFFu, d, 4);
-                            d += __shfl_xor_sync(0xFFFFFFFFu, d, 2);
-                            d += __shfl_xor_sync(0xFFFFFFFFu, d, 1);
-                            const bool on = (msk[u] >> h) & 1u;
-                            if (!kAll) d -= seg_logc[segi[u]][h];
-                            sc[u] = on ? d : -CUDART_INF_F;
-                            mx = fmaxf(mx, sc[u]);
-                        }
-                        if (mx > m[h]) {
-                            const float f = exp2f(m[h] - mx);          // 0 on the first rows
-                            l[h] *= f;
-#pragma unroll
-                            for (int i = 0; i < 8; ++i) acc[h][i] *= f;
-                            m[h] = mx;
-                        }
-#pragma unroll
-                        for (int u = 0; u < kRowsPerHalfWarp; ++u) {
-                            const bool on = (msk[u] >> h) & 1u;
-                            const float pw = on ? exp2f(sc[u] - m[h]) : 0.f;
-                            l[h] += pw;
-                            acc[h][0] = fmaf(pw, bf16_lo(vv[u].x), acc[h][0]);
-                            acc[h][1] = fmaf(pw, bf16_hi(vv[u].x), acc[h][1]);
-                            acc[h][2] = fmaf(pw, bf16_lo(vv[u].y), acc[h][2]);
-                            acc[h][3] = fmaf(pw, bf16_hi(vv[u].y), acc[h][3]);
-                            acc[h][4] = fmaf(pw, bf16_lo(vv[u].z), acc[h][4]);
-                            acc[h][5] = fmaf(pw, bf16_hi(vv[u].z), acc[h][5]);
-                            acc[h][6] = fmaf(pw, bf16_lo(vv[u].w), acc[h][6]);
-                            acc[h][7] = fmaf(pw, bf16_hi(vv[u].w), acc[h][7]);
-                        }
-                    }
-                }
+                if (lane == 0) mbar_arrive(empty_bar + bs);
             }
         }
-        g_stage += (uint32_t)n_st;
-        __syncthreads();                                   // every stage of the span is consumed
+        g_block += (uint32_t)n_blk;
+        __syncthreads();                                   // every block of the span is consumed
         if (*abort_flag) {
             // a bounded wait ran out: report, let copies already issued land, and leave
             if (tid == 0 && p.status) atomicOr(p.status, 2);
-            if (is_producer && lane == 0) {
-                const uint32_t issued = g_stage - (uint32_t)n_st + (uint32_t)st_issued;
-                for (uint32_t gs = issued > (uint32_t)kStages ? issued - kStages : 0u; gs < issued; ++gs)
-                    for (uint32_t it = 0; it < kSpinLimit; ++it)
-                        if (mbar_try_wait(full_bar + gs % kStages, (gs / kStages) & 1)) break;
-            }
+            if (is_producer) asm volatile("cp.async.wait_all;" ::: "memory");
             __syncthreads();
             return;
         }
@@ -360,24 +420,16 @@ attend_kernel(AttendParams p)
         float(*red_m)[G] = reinterpret_cast<float(*)[G]>(smem + S::red_m);
         float(*red_l)[G] = reinterpret_cast<float(*)[G]>(smem + S::red_l);
         if (!is_producer) {
+            l_run += __shfl_xor_sync(0xFFFFFFFFu, l_run, 1);
+            l_run += __shfl_xor_sync(0xFFFFFFFFu, l_run, 2);
+            if (c == 0 && g < G) { red_m[warp][g] = m_run; red_l[warp][g] = l_run; }
 #pragma unroll
-            for (int h = 0; h < G; ++h) {
-                const float mo = __shfl_xor_sync(0xFFFFFFFFu, m[h], 16);
-                const float mm = fmaxf(m[h], mo);
-                const float f = m[h] > -CUDART_INF_F ? exp2f(m[h] - mm) : 0.f;
-                float lh = l[h] * f;
-                lh += __shfl_xor_sync(0xFFFFFFFFu, lh, 16);
-                float av[8];
+            for (int t = 0; t < 8; ++t) {
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    av[i] = acc[h][i] * f;
-                    av[i] += __shfl_xor_sync(0xFFFFFFFFu, av[i], 16);
+                for (int r = 0; r < 4; ++r) {
+                    const int h = 2 * c + (r & 1), d = 16 * t + g + 8 * (r >> 1);
+                    if (h < G) red_acc[warp][h][d] = o[t][r];
                 }
-                if (lane < 16) {
-                    *reinterpret_cast<float4 *>(&red_acc[warp][h][l16 * 8]) = make_float4(av[0], av[1], av[2], av[3]);
-                    *reinterpret_cast<float4 *>(&red_acc[warp][h][l16 * 8 + 4]) = make_float4(av[4], av[5], av[6], av[7]);
-                }
-                if (lane == 0) { red_m[warp][h] = mm; red_l[warp][h] = lh; }
             }
         }
         __syncthreads();
@@ -417,26 +469,26 @@ attend_kernel(AttendParams p)
             if (warp < G) {
                 const int h = warp;
                 float mh = -CUDART_INF_F;
-                for (int c = lane; c < n_ctas; c += 32)
-                    mh = fmaxf(mh, __ldcg(first + ((size_t)c * G + h) * kPartialStride));
+                for (int cc = lane; cc < n_ctas; cc += 32)
+                    mh = fmaxf(mh, __ldcg(first + ((size_t)cc * G + h) * kPartialStride));
 #pragma unroll
-                for (int o = 16; o > 0; o >>= 1) mh = fmaxf(mh, __shfl_xor_sync(0xFFFFFFFFu, mh, o));
+                for (int off = 16; off > 0; off >>= 1) mh = fmaxf(mh, __shfl_xor_sync(0xFFFFFFFFu, mh, off));
                 float den = 0.f;
-                for (int c = lane; c < n_ctas; c += 32) {
-                    const float *pp = first + ((size_t)c * G + h) * kPartialStride;
+                for (int cc = lane; cc < n_ctas; cc += 32) {
+                    const float *pp = first + ((size_t)cc * G + h) * kPartialStride;
                     const float mj = __ldcg(pp);
                     const float wgt = mj > -CUDART_INF_F ? exp2f(mj - mh) : 0.f;
-                    wbuf[h][c] = wgt;
+                    wbuf[h][cc] = wgt;
                     den = fmaf(wgt, __ldcg(pp + 1), den);
                 }
 #pragma unroll
-                for (int o = 16; o > 0; o >>= 1) den += __shfl_xor_sync(0xFFFFFFFFu, den, o);
+                for (int off = 16; off > 0; off >>= 1) den += __shfl_xor_sync(0xFFFFFFFFu, den, off);
                 __syncwarp();
                 float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll 4
-                for (int c = 0; c < n_ctas; ++c) {
-                    const float wgt = wbuf[h][c];
-                    const float4 *pp = reinterpret_cast<const float4 *>(first + ((size_t)c * G + h) * kPartialStride + 4);
+#pragma unroll 8
+                for (int cc = 0; cc < n_ctas; ++cc) {
+                    const float wgt = wbuf[h][cc];
+                    const float4 *pp = reinterpret_cast<const float4 *>(first + ((size_t)cc * G + h) * kPartialStride + 4);
                     float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
                     if (wgt != 0.f) v = __ldcg(pp + lane);
                     num.x = fmaf(wgt, v.x, num.x);
@@ -445,9 +497,9 @@ attend_kernel(AttendParams p)
                     num.w = fmaf(wgt, v.w, num.w);
                 }
                 const float inv = 1.f / den;
-                const float4 o = make_float4(num.x * inv, num.y * inv, num.z * inv, num.w * inv);
-                *reinterpret_cast<float4 *>(p.out + ((size_t)b * p.bv.n_q + (size_t)j * G + h) * kHeadDim + lane * 4) = o;
-                if (p.status && !(isfinite(o.x) && isfinite(o.y) && isfinite(o.z) && isfinite(o.w)))
+                const float4 ov = make_float4(num.x * inv, num.y * inv, num.z * inv, num.w * inv);
+                *reinterpret_cast<float4 *>(p.out + ((size_t)b * p.bv.n_q + (size_t)j * G + h) * kHeadDim + lane * 4) = ov;
+                if (p.status && !(isfinite(ov.x) && isfinite(ov.y) && isfinite(ov.z) && isfinite(ov.w)))
                     atomicOr(p.status, 1);
             }
         }
