@@ -94,7 +94,7 @@ DecodeLayout decode_layout(const santapp_geom *g, const santapp_teams *t, int K,
     L.seg_prefix = take(sizeof(int32_t) * (size_t)L.n_pairs * (L.seg_cap + 1));
     L.seg_row = take(sizeof(int32_t) * (size_t)L.n_pairs * L.seg_cap);
     L.seg_mask = take(sizeof(uint32_t) * (size_t)L.n_pairs * L.seg_cap);
-    L.seg_logc = take(sizeof(float) * (size_t)L.n_pairs * L.seg_cap * G);
+    L.seg_logc = take(sizeof(float) * (size_t)L.n_pairs * L.seg_cap * kMaxGroup);
     L.pair_nseg = take(sizeof(int32_t) * (size_t)L.n_pairs);
     L.pair_rows = take(sizeof(int32_t) * (size_t)L.n_pairs);
     L.pair_union = take(sizeof(int32_t) * (size_t)L.n_pairs);

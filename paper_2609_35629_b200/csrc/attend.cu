@@ -5,10 +5,11 @@
 //
 // Work split. The rows of all (sequence, KV head) pairs form one global row space that is cut
 // into equal contiguous ranges, one per CTA (split-K by rows, not by teams), one CTA per SM.
-// Inside a CTA the range is dealt out in blocks of 16 rows to eight consumer warps; two
-// producer warps stream each block's K and V rows into that warp's private two-slot ring in
-// shared memory with 16-byte asynchronous copies (whole 256-byte rows per half warp, XOR
-// swizzled so that ldmatrix is bank-conflict free) and signal an mbarrier.
+// Inside a CTA each warp takes a contiguous run of 16-row blocks. A warp streams its own blocks
+// through a private two-slot ring in shared memory with 16-byte asynchronous copies (a whole
+// 256-byte row per half warp, XOR swizzled so that ldmatrix is bank-conflict free), one block
+// ahead of the one it is evaluating, together with the block's per-row head masks and
+// corrections; completion is tracked with cp.async groups, so the kernel has no spin-wait.
 //
 // Arithmetic. The GQA group is a real MMA tile: the query heads of the KV head (at most 8)
 // are the M rows of S^T = q K^T (mma.sync m16n8k16, bf16 inputs, fp32 accumulation), so one
@@ -17,8 +18,8 @@
 // terms (p = p_hi + p_lo) so that O^T += V^T P^T keeps fp32-level accuracy.
 //
 // Each CTA leaves one online-softmax partial per pair it touched; the last CTA to finish a
-// pair merges that pair's partials by log-sum-exp (the split-softmax reduction).
-// Every wait on a barrier is bounded: on expiry the kernel raises a status bit and leaves.
+// pair stages that pair's partials in shared memory and merges them by log-sum-exp (the
+// split-softmax reduction).
 #include <math_constants.h>
 
 #include "common.cuh"
@@ -27,67 +28,31 @@ namespace santapp {
 
 namespace {
 
-constexpr int kConsumerWarps = 8;
-constexpr int kProducerWarps = 2;
-constexpr int kConsumerThreads = 32 * kConsumerWarps;
-constexpr int kAttendThreads = 32 * (kConsumerWarps + kProducerWarps);
+constexpr int kWarps = 12;
+constexpr int kAttendThreads = 32 * kWarps;
 constexpr int kBlockRows = 16;                              // rows per block (one warp, one MMA K step)
-constexpr int kSlots = 2;                                   // ring slots per consumer warp
+constexpr int kSlots = 2;                                   // ring slots per warp
 constexpr int kRowBytes = kHeadDim * 2;                     // one bf16 row
 constexpr int kTileBytes = kBlockRows * kRowBytes;          // K tile or V tile of a block
 constexpr int kSlotBytes = 2 * kTileBytes;                  // K tile then V tile
 constexpr int kSegMax = 1025;                               // plan segments of one pair (G * K + suffix)
-constexpr int kPairMax = 1024;                              // pairs whose offsets are staged
+constexpr int kPairMax = 512;                               // pairs whose offsets are staged
 constexpr int kMaxAttendGrid = 512;
-constexpr uint32_t kSpinLimit = 1u << 22;
-constexpr int kNoSeg = 0xFFFF;
+constexpr uint32_t kNoRow = 0xFFFFFFFFu;
 
 // ---- primitives ----
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
-__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void fence_barrier_init()
-{
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t *bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-// The executing thread's earlier cp.async copies arrive on the barrier when they complete.
-__device__ __forceinline__ void cp_async_arrive(uint64_t *bar)
-{
-    asm volatile("cp.async.mbarrier.arrive.shared::cta.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-// Bounded wait. Returns false when the limit ran out or another thread already gave up.
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag)
-{
-    for (uint32_t it = 0; it < kSpinLimit; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 1023u) == 1023u && *abort_flag) return false;
-    }
-    *abort_flag = 1;
-    return false;
-}
 // 16-byte asynchronous copy global -> shared; src_bytes = 0 writes zeros instead.
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, uint32_t src_bytes)
 {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait_group()
+{
+    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
 }
 __device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr)
 {
@@ -122,23 +87,23 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
 template <int G>
 struct Smem {
     static constexpr size_t ring = 0;                                           // [warps][kSlots][kSlotBytes]
-    static constexpr size_t ring_bytes = (size_t)kConsumerWarps * kSlots * kSlotBytes;
-    static constexpr size_t bars = ring + ring_bytes;                           // full[w][s], empty[w][s]
-    static constexpr size_t row_seg = bars + 2 * kConsumerWarps * kSlots * 8;   // u16 [w][s][16]
-    static constexpr size_t seg_prefix = row_seg + kConsumerWarps * kSlots * kBlockRows * 2;   // int [kSegMax+1]
+    static constexpr size_t ring_bytes = (size_t)kWarps * kSlots * kSlotBytes;
+    static constexpr size_t logc_tab = ring + ring_bytes;                       // float [warps][kSlots][16][8]
+    static constexpr size_t mask_tab = logc_tab + (size_t)kWarps * kSlots * kBlockRows * kMaxGroup * 4;
+    static constexpr size_t seg_prefix = mask_tab + kWarps * kSlots * kBlockRows;   // int [kSegMax + 1]
     static constexpr size_t seg_row = seg_prefix + (kSegMax + 3) * 4;           // int [kSegMax]
     static constexpr size_t seg_mask = seg_row + (kSegMax + 3) * 4;             // uint [kSegMax]
-    static constexpr size_t seg_logc = seg_mask + (kSegMax + 3) * 4;            // float [kSegMax][G]
-    static constexpr size_t pair_prefix = (seg_logc + (size_t)kSegMax * G * 4 + 15) / 16 * 16;  // int64 [kPairMax+1]
+    static constexpr size_t pair_prefix = (seg_mask + (kSegMax + 3) * 4 + 15) / 16 * 16;   // int64 [kPairMax + 1]
     static constexpr size_t pair_nseg = pair_prefix + (kPairMax + 1) * 8;       // int [kPairMax]
     static constexpr size_t misc = pair_nseg + kPairMax * 4;                    // flags
     static constexpr size_t total = misc + 64;
     // aliases of the ring, used only after a span's blocks are consumed
     static constexpr size_t red_acc = ring;                                     // float [warps][G][128]
-    static constexpr size_t red_m = red_acc + (size_t)kConsumerWarps * G * kHeadDim * 4;   // float [warps][G]
-    static constexpr size_t red_l = red_m + (size_t)kConsumerWarps * G * 4;
-    static constexpr size_t wbuf = red_l + (size_t)kConsumerWarps * G * 4;      // float [G][kMaxAttendGrid]
-    static_assert(wbuf + (size_t)G * kMaxAttendGrid * 4 <= bars, "merge scratch must fit in the ring");
+    static constexpr size_t red_m = red_acc + (size_t)kWarps * G * kHeadDim * 4;   // float [warps][G]
+    static constexpr size_t red_l = red_m + (size_t)kWarps * G * 4;
+    static_assert(red_l + (size_t)kWarps * G * 4 <= ring_bytes, "merge scratch must fit in the ring");
+    static constexpr int merge_chunk = (int)(ring_bytes / ((size_t)G * kPartialStride * 4));   // partials staged at once
+    static_assert(total <= 227 * 1024, "shared memory budget");
 };
 
 template <int G, bool kAll>
@@ -147,31 +112,17 @@ attend_kernel(AttendParams p)
 {
     extern __shared__ __align__(1024) unsigned char smem[];
     using S = Smem<G>;
-    unsigned char *ring = smem + S::ring;
-    uint64_t *full_bar = reinterpret_cast<uint64_t *>(smem + S::bars);          // [w * kSlots + s]
-    uint64_t *empty_bar = full_bar + kConsumerWarps * kSlots;
-    uint16_t *row_seg = reinterpret_cast<uint16_t *>(smem + S::row_seg);        // [(w * kSlots + s) * 16 + r]
     int *seg_prefix = reinterpret_cast<int *>(smem + S::seg_prefix);
     int *seg_row = reinterpret_cast<int *>(smem + S::seg_row);
     uint32_t *seg_mask = reinterpret_cast<uint32_t *>(smem + S::seg_mask);
-    float(*seg_logc)[G] = reinterpret_cast<float(*)[G]>(smem + S::seg_logc);
     int64_t *pair_prefix = reinterpret_cast<int64_t *>(smem + S::pair_prefix);
     int *pair_nseg = reinterpret_cast<int *>(smem + S::pair_nseg);
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + S::misc);
-    int *last_flag = reinterpret_cast<int *>(smem + S::misc) + 1;
+    int *last_flag = reinterpret_cast<int *>(smem + S::misc);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const bool is_producer = warp >= kConsumerWarps;
     const int g = lane >> 2, c = lane & 3;                 // MMA fragment coordinates
+    const int hw = lane >> 4, chunk = lane & 15;           // copy coordinates: row parity, 16-byte chunk
 
-    if (tid == 0) {
-        for (int s = 0; s < kConsumerWarps * kSlots; ++s) {
-            mbar_init(full_bar + s, 32);                   // one arrival per producer lane
-            mbar_init(empty_bar + s, 1);                   // the consumer warp's lane 0
-        }
-        fence_barrier_init();
-        *abort_flag = 0;
-    }
     for (int i = tid; i <= p.n_pairs; i += kAttendThreads) pair_prefix[i] = p.plan.pair_row_prefix[i];
     for (int i = tid; i < p.n_pairs; i += kAttendThreads) pair_nseg[i] = p.plan.pair_nseg[i];
     __syncthreads();
@@ -193,7 +144,9 @@ attend_kernel(AttendParams p)
         pair = lo;
     }
 
-    uint32_t g_block = 0;          // blocks dealt out so far by this CTA (same count in every thread)
+    const uint32_t ring_w = smem_u32(smem + S::ring) + (uint32_t)warp * kSlots * kSlotBytes;
+    float *logc_w = reinterpret_cast<float *>(smem + S::logc_tab) + warp * kSlots * kBlockRows * kMaxGroup;
+    unsigned char *mask_w = smem + S::mask_tab + warp * kSlots * kBlockRows;
 
     while (r0 < r1) {
         const int64_t pb = pair_prefix[pair], pe = pair_prefix[pair + 1];
@@ -202,6 +155,7 @@ attend_kernel(AttendParams p)
         const int b = pair / p.bv.n_kv, j = pair - b * p.bv.n_kv;
         const int cap = p.plan.seg_cap;
         const int nseg = pair_nseg[pair];
+        const float *g_logc = p.plan.seg_logc + (size_t)pair * cap * kMaxGroup;
 
         __syncthreads();                                   // the previous span is done with the tables
         {
@@ -209,35 +163,19 @@ attend_kernel(AttendParams p)
             const int32_t *g_prefix = p.plan.seg_prefix + (size_t)pair * (cap + 1);
             const int32_t *g_row = p.plan.seg_row + (size_t)pair * cap;
             const uint32_t *g_mask = p.plan.seg_mask + (size_t)pair * cap;
-            const float *g_logc = p.plan.seg_logc + (size_t)pair * cap * G;
             for (int i0 = 0; i0 <= nseg; i0 += kAttendThreads) {
                 const int i = i0 + tid;
                 int v_prefix = 0, v_row = 0;
                 uint32_t v_mask = 0u;
-                float v_logc[G];
                 if (i <= nseg) v_prefix = g_prefix[i];
-                if (i < nseg) {
-                    v_row = g_row[i];
-                    v_mask = g_mask[i];
-                    if (!kAll) {
-#pragma unroll
-                        for (int h = 0; h < G; ++h) v_logc[h] = g_logc[(size_t)i * G + h];
-                    }
-                }
+                if (i < nseg) { v_row = g_row[i]; v_mask = g_mask[i]; }
                 if (i <= nseg) seg_prefix[i] = v_prefix;
-                if (i < nseg) {
-                    seg_row[i] = v_row;
-                    seg_mask[i] = v_mask;
-                    if (!kAll) {
-#pragma unroll
-                        for (int h = 0; h < G; ++h) seg_logc[i][h] = v_logc[h];
-                    }
-                }
+                if (i < nseg) { seg_row[i] = v_row; seg_mask[i] = v_mask; }
             }
         }
         // A fragments of q for the 8 k-steps: head g (zero rows for g >= G and for M rows 8..15)
         uint32_t qa[8][2];
-        if (!is_producer) {
+        {
             const uint32_t *qrow = reinterpret_cast<const uint32_t *>(
                 p.q + ((size_t)b * p.bv.n_q + (size_t)j * G + (g < G ? g : 0)) * kHeadDim);
 #pragma unroll
@@ -248,11 +186,72 @@ attend_kernel(AttendParams p)
         }
         __syncthreads();
 
-        const int n_blk = (bnd - a + kBlockRows - 1) / kBlockRows;
         const unsigned char *k_plane = reinterpret_cast<const unsigned char *>(p.k_packed)
                                        + (size_t)j * p.bv.rows_total * kRowBytes;
         const unsigned char *v_plane = reinterpret_cast<const unsigned char *>(p.v_packed)
                                        + (size_t)j * p.bv.rows_total * kRowBytes;
+        const unsigned char *k_suf = reinterpret_cast<const unsigned char *>(p.k_suffix);
+        const unsigned char *v_suf = reinterpret_cast<const unsigned char *>(p.v_suffix);
+
+        // this warp's contiguous run of blocks: [blk0, blk0 + nb)
+        const int n_blk = (bnd - a + kBlockRows - 1) / kBlockRows;
+        const int per = n_blk / kWarps, rem = n_blk - per * kWarps;
+        const int nb = per + (warp < rem ? 1 : 0);
+        const int blk0 = warp * per + min(warp, rem);
+
+        // segment cursor of row (lane & 15) of the current block; rows advance by 16 per block
+        int cur = 0;
+        if (nb > 0) {
+            const int pos = min(a + blk0 * kBlockRows + (lane & 15), bnd - 1);
+            int lo = 0, hi = nseg;
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                if (seg_prefix[mid] <= pos) lo = mid; else hi = mid;
+            }
+            cur = lo;
+        }
+
+        // Issue the copies of this warp's block i (if it exists) into ring slot i % kSlots and
+        // close a group: K and V rows, and for each row its head mask and corrections.
+        auto issue = [&](int i) {
+            if (i < nb) {
+                const int slot = i % kSlots;
+                const int pos0 = a + (blk0 + i) * kBlockRows;
+                const int r = lane & 15;
+                const int pos = pos0 + r;
+                uint32_t info = kNoRow;                    // row index in its buffer, bit 31: suffix buffer
+                if (pos < bnd) {
+                    while (pos >= seg_prefix[cur + 1]) ++cur;
+                    const uint32_t mk = seg_mask[cur];
+                    info = (uint32_t)(seg_row[cur] + (pos - seg_prefix[cur])) | (mk & kSrcSuffix);
+                    if (lane < 16) {
+                        mask_w[slot * kBlockRows + r] = (unsigned char)(mk & 0xFFu);
+                        if (!kAll) {
+                            const uint32_t dst = smem_u32(logc_w + (slot * kBlockRows + r) * kMaxGroup);
+                            cp_async16(dst, g_logc + (size_t)cur * kMaxGroup, 16u);
+                            cp_async16(dst + 16, g_logc + (size_t)cur * kMaxGroup + 4, 16u);
+                        }
+                    }
+                } else if (lane < 16) {
+                    mask_w[slot * kBlockRows + r] = 0;
+                }
+                const uint32_t k_dst = ring_w + slot * kSlotBytes;
+#pragma unroll
+                for (int piece = 0; piece < kBlockRows / 2; ++piece) {
+                    const int row = 2 * piece + hw;
+                    const uint32_t ri = __shfl_sync(0xFFFFFFFFu, info, row);
+                    const bool valid = ri != kNoRow;
+                    const size_t off = (size_t)(ri & 0x7FFFFFFFu) * kRowBytes + chunk * 16;
+                    const bool suf = (ri & kSrcSuffix) != 0u;
+                    const unsigned char *ks = valid ? (suf ? k_suf : k_plane) + off : k_plane;
+                    const unsigned char *vs = valid ? (suf ? v_suf : v_plane) + off : v_plane;
+                    const uint32_t dst = k_dst + row * kRowBytes + ((chunk ^ (row & 7)) << 4);
+                    cp_async16(dst, ks, valid ? 16u : 0u);
+                    cp_async16(dst + kTileBytes, vs, valid ? 16u : 0u);
+                }
+            }
+            cp_async_commit();
+        };
 
         // online-softmax state of head g (replicated over the quad) and O^T fragments:
         // o[t][r]: d = 16 t + g + 8 (r >> 1), head = 2 c + (r & 1)
@@ -260,169 +259,99 @@ attend_kernel(AttendParams p)
         float o[8][4];
 #pragma unroll
         for (int t = 0; t < 8; ++t) { o[t][0] = o[t][1] = o[t][2] = o[t][3] = 0.f; }
+        const float qk = p.qk_scale_log2;
 
-        if (is_producer) {
-            // ---------------- producer warps: blocks of alternating parity ----------------
-            const int pw = warp - kConsumerWarps;
-            int cur = 0;                                   // segment cursor of lane r (r < 16)
-            for (int bi = 0; bi < n_blk; ++bi) {
-                const uint32_t gb = g_block + bi;
-                if ((int)(gb % kProducerWarps) != pw) continue;
-                const int w = gb % kConsumerWarps;
-                const uint32_t u = gb / kConsumerWarps;
-                const int slot = u % kSlots;
-                const int bs = w * kSlots + slot;
-                if (u >= (uint32_t)kSlots &&
-                    !__all_sync(0xFFFFFFFFu, mbar_wait(empty_bar + bs, ((u / kSlots) - 1) & 1, abort_flag)))
-                    break;
-                // lane r < 16 resolves row r of the block
-                const int pos = a + bi * kBlockRows + (lane & 15);
-                const bool valid = pos < bnd;
-                int64_t grow = 0;
-                int suf = 0;
-                if (valid) {
-                    if (pos >= seg_prefix[cur + 1]) {      // moved on: binary search from here
-                        int lo = cur + 1, hi = nseg;
-                        while (hi - lo > 1) {
-                            const int mid = (lo + hi) >> 1;
-                            if (seg_prefix[mid] <= pos) lo = mid; else hi = mid;
-                        }
-                        cur = lo;
-                    }
-                    grow = (int64_t)seg_row[cur] + (pos - seg_prefix[cur]);
-                    suf = (seg_mask[cur] & kSrcSuffix) ? 1 : 0;
-                }
-                if (lane < 16) row_seg[bs * kBlockRows + lane] = (uint16_t)(valid ? cur : kNoSeg);
-                const uint32_t slot_addr = smem_u32(ring + (size_t)bs * kSlotBytes);
-                const int chunk = lane & 15;
+        issue(0);
+        for (int i = 0; i < nb; ++i) {
+            issue(i + 1);
+            cp_async_wait_group<1>();                      // block i has landed (this lane's copies)
+            __syncwarp();                                  // ... and every other lane's
+            const int slot = i % kSlots;
+            const uint32_t k_addr = ring_w + slot * kSlotBytes;
+            const uint32_t v_addr = k_addr + kTileBytes;
+
+            // the four (row, head g) entries of this thread: rows 2c, 2c+1, 8+2c, 9+2c
+            bool on[4];
+            float lc[4];
 #pragma unroll
-                for (int piece = 0; piece < kBlockRows / 2; ++piece) {
-                    const int row = 2 * piece + (lane >> 4);
-                    const int64_t rr = __shfl_sync(0xFFFFFFFFu, grow, row);
-                    const int rs = __shfl_sync(0xFFFFFFFFu, suf, row);
-                    const int rv = __shfl_sync(0xFFFFFFFFu, (int)valid, row);
-                    const unsigned char *ks = (rs ? reinterpret_cast<const unsigned char *>(p.k_suffix) : k_plane)
-                                              + rr * kRowBytes + chunk * 16;
-                    const unsigned char *vs = (rs ? reinterpret_cast<const unsigned char *>(p.v_suffix) : v_plane)
-                                              + rr * kRowBytes + chunk * 16;
-                    const uint32_t dst = slot_addr + row * kRowBytes + ((chunk ^ (row & 7)) << 4);
-                    cp_async16(dst, ks, rv ? 16u : 0u);
-                    cp_async16(dst + kTileBytes, vs, rv ? 16u : 0u);
-                }
-                cp_async_arrive(full_bar + bs);
-                mbar_arrive(full_bar + bs);
+            for (int e = 0; e < 4; ++e) {
+                const int r = 2 * c + (e & 1) + 8 * (e >> 1);
+                const uint32_t mk = mask_w[slot * kBlockRows + r];
+                on[e] = (g < G) && ((mk >> g) & 1u);
+                lc[e] = (!kAll && on[e]) ? logc_w[(slot * kBlockRows + r) * kMaxGroup + g] : 0.f;
             }
-        } else {
-            // ---------------- consumer warps ----------------
-            const float qk = p.qk_scale_log2;
-            int first = (int)((warp + kConsumerWarps - (g_block % kConsumerWarps)) % kConsumerWarps);
-            for (int bi = first; bi < n_blk; bi += kConsumerWarps) {
-                const uint32_t gb = g_block + bi;
-                const uint32_t u = gb / kConsumerWarps;
-                const int slot = u % kSlots;
-                const int bs = warp * kSlots + slot;
-                if (!__all_sync(0xFFFFFFFFu, mbar_wait(full_bar + bs, (u / kSlots) & 1, abort_flag))) break;
-                const uint32_t k_addr = smem_u32(ring + (size_t)bs * kSlotBytes);
-                const uint32_t v_addr = k_addr + kTileBytes;
 
-                // the four (row, head g) entries of this thread: rows 2c, 2c+1, 8+2c, 9+2c
-                bool on[4];
-                float lc[4];
+            // S^T = q K^T for the two 8-row groups, two accumulators each to shorten the chain
+            float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+            float s2[4] = {0.f, 0.f, 0.f, 0.f}, s3[4] = {0.f, 0.f, 0.f, 0.f};
+            {
+                const int lrow = lane & 7, lmat = lane >> 3;
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int r = 2 * c + (i & 1) + 8 * (i >> 1);
-                    lc[i] = 0.f;
-                    if (kAll) {
-                        on[i] = (g < G) && (a + bi * kBlockRows + r < bnd);
-                    } else {
-                        const int sg = row_seg[bs * kBlockRows + r];
-                        on[i] = false;
-                        if (sg != kNoSeg && g < G) {
-                            on[i] = (seg_mask[sg] >> g) & 1u;
-                            lc[i] = seg_logc[sg][g];
-                        }
-                    }
+                for (int sp = 0; sp < 4; ++sp) {
+                    uint32_t kb0[4], kb1[4];
+                    const int ch = 4 * sp + lmat;
+                    ldmatrix_x4(kb0, k_addr + lrow * kRowBytes + ((ch ^ lrow) << 4));
+                    ldmatrix_x4(kb1, k_addr + (8 + lrow) * kRowBytes + ((ch ^ lrow) << 4));
+                    mma_bf16(s0, qa[2 * sp][0], 0u, qa[2 * sp][1], 0u, kb0[0], kb0[1]);
+                    mma_bf16(s1, qa[2 * sp][0], 0u, qa[2 * sp][1], 0u, kb1[0], kb1[1]);
+                    mma_bf16(s2, qa[2 * sp + 1][0], 0u, qa[2 * sp + 1][1], 0u, kb0[2], kb0[3]);
+                    mma_bf16(s3, qa[2 * sp + 1][0], 0u, qa[2 * sp + 1][1], 0u, kb1[2], kb1[3]);
                 }
-
-                // S^T = q K^T for the two 8-row groups
-                float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
-                {
-                    const int lrow = lane & 7, lmat = lane >> 3;
-#pragma unroll
-                    for (int sp = 0; sp < 4; ++sp) {
-                        uint32_t kb0[4], kb1[4];
-                        const int chunk = 4 * sp + lmat;
-                        ldmatrix_x4(kb0, k_addr + lrow * kRowBytes + ((chunk ^ lrow) << 4));
-                        ldmatrix_x4(kb1, k_addr + (8 + lrow) * kRowBytes + ((chunk ^ lrow) << 4));
-                        mma_bf16(s0, qa[2 * sp][0], 0u, qa[2 * sp][1], 0u, kb0[0], kb0[1]);
-                        mma_bf16(s1, qa[2 * sp][0], 0u, qa[2 * sp][1], 0u, kb1[0], kb1[1]);
-                        mma_bf16(s0, qa[2 * sp + 1][0], 0u, qa[2 * sp + 1][1], 0u, kb0[2], kb0[3]);
-                        mma_bf16(s1, qa[2 * sp + 1][0], 0u, qa[2 * sp + 1][1], 0u, kb1[2], kb1[3]);
-                    }
-                }
-                float sc[4];
-                sc[0] = on[0] ? fmaf(s0[0], qk, -lc[0]) : -CUDART_INF_F;
-                sc[1] = on[1] ? fmaf(s0[1], qk, -lc[1]) : -CUDART_INF_F;
-                sc[2] = on[2] ? fmaf(s1[0], qk, -lc[2]) : -CUDART_INF_F;
-                sc[3] = on[3] ? fmaf(s1[1], qk, -lc[3]) : -CUDART_INF_F;
-                float mloc = fmaxf(fmaxf(sc[0], sc[1]), fmaxf(sc[2], sc[3]));
-                mloc = fmaxf(mloc, __shfl_xor_sync(0xFFFFFFFFu, mloc, 1));
-                mloc = fmaxf(mloc, __shfl_xor_sync(0xFFFFFFFFu, mloc, 2));
-                const float m_new = fmaxf(m_run, mloc);
-                const bool grew = m_new > m_run;
-                if (__any_sync(0xFFFFFFFFu, grew)) {
-                    const float f = grew ? exp2f(m_run - m_new) : 1.f;          // exp2f(-inf) = 0 on first rows
-                    l_run *= f;
-                    const float fe = __shfl_sync(0xFFFFFFFFu, f, 8 * c);        // head 2c lives in lanes 8c..8c+3
-                    const float fo = __shfl_sync(0xFFFFFFFFu, f, 8 * c + 4);    // head 2c+1
-#pragma unroll
-                    for (int t = 0; t < 8; ++t) { o[t][0] *= fe; o[t][1] *= fo; o[t][2] *= fe; o[t][3] *= fo; }
-                    m_run = m_new;
-                }
-                float pw[4];
-#pragma unroll
-                for (int i = 0; i < 4; ++i) pw[i] = on[i] ? exp2f(sc[i] - m_run) : 0.f;
-                l_run += (pw[0] + pw[1]) + (pw[2] + pw[3]);
-                // P^T as B fragments, split in two bf16 terms
-                const uint32_t ph0 = pack_bf16x2(pw[0], pw[1]), ph1 = pack_bf16x2(pw[2], pw[3]);
-                const uint32_t pl0 = pack_bf16x2(pw[0] - bf16_lo(ph0), pw[1] - bf16_hi(ph0));
-                const uint32_t pl1 = pack_bf16x2(pw[2] - bf16_lo(ph1), pw[3] - bf16_hi(ph1));
-
-                // O^T += V^T P^T
-                {
-                    const int lrow = lane & 7, lmat = lane >> 3;
-                    const int vrow = (lmat >> 1) * 8 + lrow;
-#pragma unroll
-                    for (int t = 0; t < 8; ++t) {
-                        uint32_t va[4];
-                        const int chunk = 2 * t + (lmat & 1);
-                        ldmatrix_x4_trans(va, v_addr + vrow * kRowBytes + ((chunk ^ lrow) << 4));
-                        mma_bf16(o[t], va[0], va[1], va[2], va[3], ph0, ph1);
-                        mma_bf16(o[t], va[0], va[1], va[2], va[3], pl0, pl1);
-                    }
-                }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(empty_bar + bs);
             }
+            float sc[4];
+            sc[0] = on[0] ? fmaf(s0[0] + s2[0], qk, -lc[0]) : -CUDART_INF_F;
+            sc[1] = on[1] ? fmaf(s0[1] + s2[1], qk, -lc[1]) : -CUDART_INF_F;
+            sc[2] = on[2] ? fmaf(s1[0] + s3[0], qk, -lc[2]) : -CUDART_INF_F;
+            sc[3] = on[3] ? fmaf(s1[1] + s3[1], qk, -lc[3]) : -CUDART_INF_F;
+            float mloc = fmaxf(fmaxf(sc[0], sc[1]), fmaxf(sc[2], sc[3]));
+            mloc = fmaxf(mloc, __shfl_xor_sync(0xFFFFFFFFu, mloc, 1));
+            mloc = fmaxf(mloc, __shfl_xor_sync(0xFFFFFFFFu, mloc, 2));
+            const float m_new = fmaxf(m_run, mloc);
+            const bool grew = m_new > m_run;
+            if (__any_sync(0xFFFFFFFFu, grew)) {
+                const float f = grew ? exp2f(m_run - m_new) : 1.f;              // exp2f(-inf) = 0 on first rows
+                l_run *= f;
+                const float fe = __shfl_sync(0xFFFFFFFFu, f, 8 * c);            // head 2c lives in lanes 8c..8c+3
+                const float fo = __shfl_sync(0xFFFFFFFFu, f, 8 * c + 4);        // head 2c+1
+#pragma unroll
+                for (int t = 0; t < 8; ++t) { o[t][0] *= fe; o[t][1] *= fo; o[t][2] *= fe; o[t][3] *= fo; }
+                m_run = m_new;
+            }
+            float pw[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) pw[e] = on[e] ? exp2f(sc[e] - m_run) : 0.f;
+            l_run += (pw[0] + pw[1]) + (pw[2] + pw[3]);
+            // P^T as B fragments, split in two bf16 terms
+            const uint32_t ph0 = pack_bf16x2(pw[0], pw[1]), ph1 = pack_bf16x2(pw[2], pw[3]);
+            const uint32_t pl0 = pack_bf16x2(pw[0] - bf16_lo(ph0), pw[1] - bf16_hi(ph0));
+            const uint32_t pl1 = pack_bf16x2(pw[2] - bf16_lo(ph1), pw[3] - bf16_hi(ph1));
+
+            // O^T += V^T P^T
+            {
+                const int lrow = lane & 7, lmat = lane >> 3;
+                const int vrow = (lmat >> 1) * 8 + lrow;
+#pragma unroll
+                for (int t = 0; t < 8; ++t) {
+                    uint32_t va[4];
+                    const int ch = 2 * t + (lmat & 1);
+                    ldmatrix_x4_trans(va, v_addr + vrow * kRowBytes + ((ch ^ lrow) << 4));
+                    mma_bf16(o[t], va[0], va[1], va[2], va[3], ph0, ph1);
+                    mma_bf16(o[t], va[0], va[1], va[2], va[3], pl0, pl1);
+                }
+            }
+            __syncwarp();                                  // the slot may be refilled by the next issue
         }
-        g_block += (uint32_t)n_blk;
+        cp_async_wait_group<0>();
         __syncthreads();                                   // every block of the span is consumed
-        if (*abort_flag) {
-            // a bounded wait ran out: report, let copies already issued land, and leave
-            if (tid == 0 && p.status) atomicOr(p.status, 2);
-            if (is_producer) asm volatile("cp.async.wait_all;" ::: "memory");
-            __syncthreads();
-            return;
-        }
 
-        // ---- merge the consumer warps into one partial (the ring is free: reuse it) ----
+        // ---- merge the warps into one partial (the ring is free: reuse it) ----
         float(*red_acc)[G][kHeadDim] = reinterpret_cast<float(*)[G][kHeadDim]>(smem + S::red_acc);
         float(*red_m)[G] = reinterpret_cast<float(*)[G]>(smem + S::red_m);
         float(*red_l)[G] = reinterpret_cast<float(*)[G]>(smem + S::red_l);
-        if (!is_producer) {
-            l_run += __shfl_xor_sync(0xFFFFFFFFu, l_run, 1);
-            l_run += __shfl_xor_sync(0xFFFFFFFFu, l_run, 2);
-            if (c == 0 && g < G) { red_m[warp][g] = m_run; red_l[warp][g] = l_run; }
+        l_run += __shfl_xor_sync(0xFFFFFFFFu, l_run, 1);
+        l_run += __shfl_xor_sync(0xFFFFFFFFu, l_run, 2);
+        if (c == 0 && g < G) { red_m[warp][g] = m_run; red_l[warp][g] = l_run; }
+        if (nb > 0) {
 #pragma unroll
             for (int t = 0; t < 8; ++t) {
 #pragma unroll
@@ -435,23 +364,23 @@ attend_kernel(AttendParams p)
         __syncthreads();
         const int slot_id = blockIdx.x + pair;
         float *part = p.partials + (size_t)slot_id * G * kPartialStride;
-        if (!is_producer) {
-            for (int e = tid; e < G * kHeadDim; e += kConsumerThreads) {
-                const int h = e >> 7, d = e & 127;
-                float mh = -CUDART_INF_F;
+        for (int e = tid; e < G * kHeadDim; e += kAttendThreads) {
+            const int h = e >> 7, d = e & 127;
+            float mh = -CUDART_INF_F;
 #pragma unroll
-                for (int w = 0; w < kConsumerWarps; ++w) mh = fmaxf(mh, red_m[w][h]);
-                float num = 0.f, den = 0.f;
+            for (int w = 0; w < kWarps; ++w) mh = fmaxf(mh, red_m[w][h]);
+            float num = 0.f, den = 0.f;
 #pragma unroll
-                for (int w = 0; w < kConsumerWarps; ++w) {
-                    const float mw = red_m[w][h];
-                    const float f = mw > -CUDART_INF_F ? exp2f(mw - mh) : 0.f;
+            for (int w = 0; w < kWarps; ++w) {
+                const float mw = red_m[w][h];
+                if (mw > -CUDART_INF_F) {                  // warps without rows for this head left no data
+                    const float f = exp2f(mw - mh);
                     num = fmaf(f, red_acc[w][h][d], num);
                     den = fmaf(f, red_l[w][h], den);
                 }
-                part[h * kPartialStride + 4 + d] = num;
-                if (d == 0) { part[h * kPartialStride] = mh; part[h * kPartialStride + 1] = den; }
             }
+            part[h * kPartialStride + 4 + d] = num;
+            if (d == 0) { part[h * kPartialStride] = mh; part[h * kPartialStride + 1] = den; }
         }
 
         // ---- last CTA of the pair: log-sum-exp merge of the pair's partials ----
@@ -464,40 +393,53 @@ attend_kernel(AttendParams p)
         if (*last_flag) {
             __threadfence();
             if (tid == 0) p.ctl.attend_ticket[pair] = 0;              // every CTA of the pair has arrived
+            // The pair's partials are contiguous in memory. Stage them in shared memory a chunk
+            // at a time with asynchronous copies, then merge from there: thread (h, lane) owns
+            // four output columns of head h.
             const float *first = p.partials + (size_t)(c_lo + pair) * G * kPartialStride;
-            float(*wbuf)[kMaxAttendGrid] = reinterpret_cast<float(*)[kMaxAttendGrid]>(smem + S::wbuf);
-            if (warp < G) {
-                const int h = warp;
-                float mh = -CUDART_INF_F;
-                for (int cc = lane; cc < n_ctas; cc += 32)
-                    mh = fmaxf(mh, __ldcg(first + ((size_t)cc * G + h) * kPartialStride));
-#pragma unroll
-                for (int off = 16; off > 0; off >>= 1) mh = fmaxf(mh, __shfl_xor_sync(0xFFFFFFFFu, mh, off));
-                float den = 0.f;
-                for (int cc = lane; cc < n_ctas; cc += 32) {
-                    const float *pp = first + ((size_t)cc * G + h) * kPartialStride;
-                    const float mj = __ldcg(pp);
-                    const float wgt = mj > -CUDART_INF_F ? exp2f(mj - mh) : 0.f;
-                    wbuf[h][cc] = wgt;
-                    den = fmaf(wgt, __ldcg(pp + 1), den);
+            float *stage = reinterpret_cast<float *>(smem + S::ring);
+            constexpr int kPer = G * kPartialStride;                   // floats per partial
+            const int h = tid >> 5;
+            float m_acc = -CUDART_INF_F, l_acc = 0.f;
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int c0 = 0; c0 < n_ctas; c0 += S::merge_chunk) {
+                const int nc = min(S::merge_chunk, n_ctas - c0);
+                __syncthreads();                           // the previous chunk has been read
+                const int n16 = nc * kPer / 4;             // 16-byte pieces
+                const float *src = first + (size_t)c0 * kPer;
+                for (int i = tid; i < n16; i += kAttendThreads)
+                    cp_async16(smem_u32(stage + 4 * i), src + 4 * i, 16u);
+                cp_async_commit();
+                cp_async_wait_group<0>();
+                __syncthreads();
+                if (h < G) {
+                    float mc = -CUDART_INF_F;
+                    for (int cc = 0; cc < nc; ++cc) mc = fmaxf(mc, stage[(cc * G + h) * kPartialStride]);
+                    const float m_new = fmaxf(m_acc, mc);
+                    if (m_new > -CUDART_INF_F) {
+                        const float f = m_acc > -CUDART_INF_F ? exp2f(m_acc - m_new) : 0.f;
+                        l_acc *= f;
+                        acc.x *= f; acc.y *= f; acc.z *= f; acc.w *= f;
+                        for (int cc = 0; cc < nc; ++cc) {
+                            const float *pp = stage + (cc * G + h) * kPartialStride;
+                            const float mj = pp[0];
+                            if (mj > -CUDART_INF_F) {
+                                const float wgt = exp2f(mj - m_new);
+                                const float4 v = *reinterpret_cast<const float4 *>(pp + 4 + lane * 4);
+                                l_acc = fmaf(wgt, pp[1], l_acc);
+                                acc.x = fmaf(wgt, v.x, acc.x);
+                                acc.y = fmaf(wgt, v.y, acc.y);
+                                acc.z = fmaf(wgt, v.z, acc.z);
+                                acc.w = fmaf(wgt, v.w, acc.w);
+                            }
+                        }
+                        m_acc = m_new;
+                    }
                 }
-#pragma unroll
-                for (int off = 16; off > 0; off >>= 1) den += __shfl_xor_sync(0xFFFFFFFFu, den, off);
-                __syncwarp();
-                float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll 8
-                for (int cc = 0; cc < n_ctas; ++cc) {
-                    const float wgt = wbuf[h][cc];
-                    const float4 *pp = reinterpret_cast<const float4 *>(first + ((size_t)cc * G + h) * kPartialStride + 4);
-                    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-                    if (wgt != 0.f) v = __ldcg(pp + lane);
-                    num.x = fmaf(wgt, v.x, num.x);
-                    num.y = fmaf(wgt, v.y, num.y);
-                    num.z = fmaf(wgt, v.z, num.z);
-                    num.w = fmaf(wgt, v.w, num.w);
-                }
-                const float inv = 1.f / den;
-                const float4 ov = make_float4(num.x * inv, num.y * inv, num.z * inv, num.w * inv);
+            }
+            if (h < G) {
+                const float inv = 1.f / l_acc;
+                const float4 ov = make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
                 *reinterpret_cast<float4 *>(p.out + ((size_t)b * p.bv.n_q + (size_t)j * G + h) * kHeadDim + lane * 4) = ov;
                 if (p.status && !(isfinite(ov.x) && isfinite(ov.y) && isfinite(ov.z) && isfinite(ov.w)))
                     atomicOr(p.status, 1);

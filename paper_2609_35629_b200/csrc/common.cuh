@@ -35,7 +35,7 @@ struct PlanView {
     int32_t *seg_row;               // [n_pairs][seg_cap] first row (global row of the KV plane, or
                                     //   row of the suffix buffer when kSrcSuffix is set in seg_mask)
     uint32_t *seg_mask;             // [n_pairs][seg_cap] bit h: head h of the group selected the team
-    float *seg_logc;                // [n_pairs][seg_cap][group] log2(e) * log c_g per selecting head
+    float *seg_logc;                // [n_pairs][seg_cap][kMaxGroup] log2(e) * log c_g per selecting head
     int32_t *pair_nseg;             // [n_pairs]
     int32_t *pair_rows;             // [n_pairs] rows of the pair's plan (prompt union + suffix)
     int32_t *pair_union_rows;       // [n_pairs] prompt rows only
