@@ -50,7 +50,8 @@ typedef enum santapp_status {
     SANTAPP_ERR_INVALID_ARG = -1,        /* null pointer, non-positive size, K < 1, R does not divide P, ... */
     SANTAPP_ERR_UNSUPPORTED = -2,        /* head_dim != 128, group size > 8, parent_size > 512, too many teams */
     SANTAPP_ERR_WORKSPACE_TOO_SMALL = -3,
-    SANTAPP_ERR_CUDA = -4                /* a CUDA runtime call or launch failed; see santapp_last_cuda_error */
+    SANTAPP_ERR_CUDA = -4,               /* a CUDA runtime call or launch failed; see santapp_last_cuda_error */
+    SANTAPP_ERR_STATIC_SCRATCH = -5      /* the problem needs more scratch than the built-in array holds */
 } santapp_status;
 
 typedef void *santapp_stream;            /* cudaStream_t */
@@ -206,6 +207,40 @@ int santapp_dense_decode_attn(const santapp_geom *geom, const santapp_teams *tea
                               const int32_t *suffix_len_dev, int32_t suffix_cap, float scale,
                               float *out, void *workspace, size_t workspace_bytes,
                               santapp_stream stream);
+
+/*
+ * Dense decode attention for callers that cannot hand the library a workspace. (The paper has
+ * no counterpart: this entry point exists for deployment reasons only.)
+ *
+ * Who needs it: code that has no way to obtain device memory at the point of the call. Examples
+ * are a serving loop whose device memory was handed over in full to another component's pool,
+ * a plug-in host that forbids CUDA allocation calls inside its callbacks, and latency-critical
+ * paths that must not run into the device-wide synchronisation an allocation can cause. For
+ * them the scratch memory santapp_dense_decode_attn would take as `workspace` lives inside the
+ * library: one array of SANTAPP_STATIC_SCRATCH_BYTES bytes in device global memory, part of
+ * the library image, so every GPU that loads the library holds it until the process exits.
+ * The call makes no allocation of any kind (no cudaMalloc, cudaFree, or allocating library
+ * routine); inputs and outputs are still the caller's buffers.
+ *
+ * Computes exactly what santapp_dense_decode_attn computes, with the same arguments minus the
+ * workspace pair.
+ *   - Limit: if santapp_dense_workspace_bytes(geom, teams) exceeds SANTAPP_STATIC_SCRATCH_BYTES
+ *     the call returns SANTAPP_ERR_STATIC_SCRATCH and launches nothing (the text of
+ *     santapp_last_cuda_error says how many bytes were needed). On a 148-SM GPU with 7 query
+ *     heads per KV head the 2 MiB array covers about 400 (sequence, KV head) pairs.
+ *   - Set-up: the first call on each device looks up the array's device address (the device
+ *     must be current, as for every call) and remembers it. Make that first call outside any
+ *     stream capture.
+ *   - Sharing: every call on a device uses the same array, which keeps whatever the previous
+ *     call left in it. Nothing in it has to be cleared between calls: the kernels initialise
+ *     every counter and table they read. Two calls that can overlap on the GPU (different
+ *     streams without an ordering between them) race on the array and must not be issued.
+ */
+#define SANTAPP_STATIC_SCRATCH_BYTES (2u << 20)
+int santapp_dense_decode_attn_noalloc(const santapp_geom *geom, const santapp_teams *teams,
+                                      const void *q, const void *k_suffix, const void *v_suffix,
+                                      const int32_t *suffix_len_dev, int32_t suffix_cap,
+                                      float scale, float *out, santapp_stream stream);
 
 /*
  * Launch statistics of the most recent decode / dense call on this thread (host-side

@@ -22,12 +22,14 @@ SANTAPP_ERR_INVALID_ARG = -1
 SANTAPP_ERR_UNSUPPORTED = -2
 SANTAPP_ERR_WORKSPACE_TOO_SMALL = -3
 SANTAPP_ERR_CUDA = -4
+SANTAPP_ERR_STATIC_SCRATCH = -5
+SANTAPP_STATIC_SCRATCH_BYTES = 2 << 20
 
 EXPORTS = [
     "santapp_version", "santapp_strerror", "santapp_last_cuda_error", "santapp_build_teams_sizes",
     "santapp_build_teams", "santapp_decode_workspace_bytes", "santapp_decode_attn",
     "santapp_dense_workspace_bytes", "santapp_dense_decode_attn", "santapp_last_launch_count",
-    "santapp_set_stage_mask",
+    "santapp_set_stage_mask", "santapp_dense_decode_attn_noalloc",
 ]
 
 STAGE_ROUTE, STAGE_SELECT, STAGE_ATTEND, STAGE_ALL = 1, 2, 4, 7
@@ -101,6 +103,9 @@ def load_library(path: Optional[str] = None):
     L.santapp_dense_decode_attn.argtypes = [ctypes.POINTER(CGeom), ctypes.POINTER(CTeams), vp, vp, vp, vp, i32,
                                             f32, vp, vp, sz, vp]
     L.santapp_dense_decode_attn.restype = ctypes.c_int
+    L.santapp_dense_decode_attn_noalloc.argtypes = [ctypes.POINTER(CGeom), ctypes.POINTER(CTeams), vp, vp, vp, vp,
+                                                    i32, f32, vp, vp]
+    L.santapp_dense_decode_attn_noalloc.restype = ctypes.c_int
     if path is None:
         _lib = L
     return L
@@ -110,7 +115,7 @@ def _check(rc):
     if rc != SANTAPP_OK:
         L = load_library()
         detail = L.santapp_strerror(rc).decode()
-        if rc == SANTAPP_ERR_CUDA:
+        if rc in (SANTAPP_ERR_CUDA, SANTAPP_ERR_STATIC_SCRATCH):
             detail += " — " + L.santapp_last_cuda_error().decode()
         raise SantappError(rc, detail)
 
@@ -273,6 +278,27 @@ def santapp_dense_decode_attn(geom: Geometry, teams: Teams, q: torch.Tensor, k_s
     _check(L.santapp_dense_decode_attn(ctypes.byref(g), ctypes.byref(teams.c), _ptr(q), _ptr(k_suffix),
                                        _ptr(v_suffix), _ptr(suffix_len), cap, scale, _ptr(out), _ptr(workspace),
                                        workspace.numel(), _stream_ptr(stream)))
+    return out
+
+
+def santapp_dense_decode_attn_noalloc(geom: Geometry, teams: Teams, q: torch.Tensor,
+                                      k_suffix: Optional[torch.Tensor], v_suffix: Optional[torch.Tensor],
+                                      suffix_len: Optional[torch.Tensor], scale: float = 0.0,
+                                      out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """Dense decode attention that takes no workspace: for callers that cannot allocate device
+    memory around the call, the scratch lives in a fixed array inside the library. Pass `out` to
+    keep the call itself free of any allocation; if it is omitted this wrapper (not the library)
+    creates the output tensor. Same result as santapp_dense_decode_attn. Calls share the array,
+    so do not let two of them overlap on the GPU; the first call on a device should come
+    before any stream capture."""
+    L = load_library()
+    if out is None:
+        out = torch.empty((geom.n_seqs, geom.n_q_heads, geom.head_dim), dtype=torch.float32, device=q.device)
+    cap = 0 if k_suffix is None else int(k_suffix.shape[2])
+    g = geom.c()
+    _check(L.santapp_dense_decode_attn_noalloc(ctypes.byref(g), ctypes.byref(teams.c), _ptr(q), _ptr(k_suffix),
+                                               _ptr(v_suffix), _ptr(suffix_len), cap, scale, _ptr(out),
+                                               _stream_ptr(stream)))
     return out
 
 

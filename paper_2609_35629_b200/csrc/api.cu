@@ -3,6 +3,7 @@
 #include <stdio.h>
 #include <string.h>
 
+#include <mutex>
 #include <vector>
 
 #include "common.cuh"
@@ -135,6 +136,7 @@ const char *santapp_strerror(int status)
         case SANTAPP_ERR_UNSUPPORTED: return "unsupported configuration";
         case SANTAPP_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
         case SANTAPP_ERR_CUDA: return "CUDA error";
+        case SANTAPP_ERR_STATIC_SCRATCH: return "problem needs more scratch than the built-in array holds";
         default: return "unknown status";
     }
 }
@@ -399,3 +401,53 @@ int santapp_dense_decode_attn(const santapp_geom *geom, const santapp_teams *tea
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------------------------
+// Dense decode attention without a caller-provided workspace.
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+// Scratch for santapp_dense_decode_attn_noalloc. In host code this name is only a handle for
+// the runtime's symbol lookup, never a device address; the address comes from
+// cudaGetSymbolAddress below.
+static __device__ __align__(256) unsigned char g_static_scratch[SANTAPP_STATIC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+void *g_static_scratch_addr[kMaxDevices];      // per device ordinal; null until looked up
+
+}  // namespace
+
+extern "C" int santapp_dense_decode_attn_noalloc(const santapp_geom *geom, const santapp_teams *teams,
+                                                 const void *q, const void *k_suffix, const void *v_suffix,
+                                                 const int32_t *suffix_len_dev, int32_t suffix_cap, float scale,
+                                                 float *out, santapp_stream stream)
+{
+    int rc = check_geom(geom);
+    if (rc != SANTAPP_OK) return rc;
+    if ((rc = check_teams(geom, teams)) != SANTAPP_OK) return rc;
+    const size_t need = santapp_dense_workspace_bytes(geom, teams);
+    if (need > (size_t)SANTAPP_STATIC_SCRATCH_BYTES) {
+        snprintf(g_cuda_error, sizeof(g_cuda_error), "built-in scratch holds %u bytes, this problem needs %zu",
+                 (unsigned)SANTAPP_STATIC_SCRATCH_BYTES, need);
+        return SANTAPP_ERR_STATIC_SCRATCH;
+    }
+    int dev = -1;
+    cudaError_t err = cudaGetDevice(&dev);
+    if (err != cudaSuccess) return cuda_fail(err, "cudaGetDevice");
+    if (dev < 0 || dev >= kMaxDevices) return SANTAPP_ERR_UNSUPPORTED;
+    void *scratch = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_static_mutex);
+        if (g_static_scratch_addr[dev] == nullptr) {
+            // once per device, with that device current
+            void *addr = nullptr;
+            err = cudaGetSymbolAddress(&addr, g_static_scratch);
+            if (err != cudaSuccess) return cuda_fail(err, "cudaGetSymbolAddress(static scratch)");
+            g_static_scratch_addr[dev] = addr;
+        }
+        scratch = g_static_scratch_addr[dev];
+    }
+    return santapp_dense_decode_attn(geom, teams, q, k_suffix, v_suffix, suffix_len_dev, suffix_cap, scale, out,
+                                     scratch, (size_t)SANTAPP_STATIC_SCRATCH_BYTES, stream);
+}
