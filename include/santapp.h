@@ -94,6 +94,8 @@ typedef struct santapp_teams {
                                   sequence) of each packed row                                       */
     int64_t *seq_row_off;      /* int64 [n_seqs + 1] device copy of the row offsets                  */
     int64_t *seq_team_off;     /* int64 [n_seqs + 1] device copy of the team offsets                 */
+    float *rep_abs_max;        /* fp32  [n_kv_heads][n_seqs]: largest |element| among the pair's
+                                  representative keys (bounds the fp32 routing pass)                 */
     int64_t rows_total;        /* host scalars, as in santapp_sizes                                  */
     int64_t teams_total;
     int32_t max_teams_per_seq;
@@ -166,7 +168,9 @@ size_t santapp_decode_workspace_bytes(const santapp_geom *geom, const santapp_te
  *   K <- min(n_sample, M_b). If K = M_b every team is read with c_g = 1 and nothing is drawn.
  *   Otherwise phi_g = log n_g + q.l_g * scale (Eq. method-routing), Y_g = phi_g + Gumbel draw,
  *   S = the K largest Y (ties to the smaller team id), tau = the (K+1)-st largest,
- *   c_g = 1 - exp(-exp(phi_g - tau)) (Eq. method-inclusion); routing is evaluated in fp64.
+ *   c_g = 1 - exp(-exp(phi_g - tau)) (Eq. method-inclusion). The sample is the fp64 one: an
+ *   fp32 pass over all teams only narrows the field to the teams whose exact fp64 score can
+ *   still be among the K+1 largest, and those are re-evaluated and ranked in fp64.
  *   out = U^ / Z^ of Eq. (method-estimate): every member of every selected team enters with
  *   weight e^{s_i} / c_g, every suffix row with weight e^{s_i}, s_i = q.k_i * scale
  *   (bf16 inputs, fp32 accumulation). Heads sharing a KV head sample independently; K/V rows
@@ -177,7 +181,7 @@ size_t santapp_decode_workspace_bytes(const santapp_geom *geom, const santapp_te
  *                   generated tokens; may be NULL when suffix_cap == 0
  *   suffix_len_dev  device int32 [n_seqs], in: visible suffix rows per sequence (clamped to
  *                   [0, suffix_cap]); NULL means 0 everywhere
- *   n_sample        K >= 1
+ *   n_sample        1 <= K <= 128, and (query heads per KV head) * min(K, M_b) <= 1024
  *   seed, step, stream_base   random-stream key and counters (see top of file)
  *   step_dev        device uint32 [1] or NULL: when given, its value is added to `step` on the
  *                   device, so a captured CUDA graph can be replayed for successive tokens
@@ -251,9 +255,10 @@ int santapp_last_launch_count(void);
 /*
  * Diagnostic: choose which stages the following santapp_decode_attn calls on this thread
  * launch, for timing one stage in isolation (the paper's "isolated-stage measurements").
- * Bit 0: representative scoring and perturbation; bit 1: selection and read plan; bit 2: exact
- * attention and merge. A stage that is skipped reuses what an earlier full call with the same
- * arguments left in the same workspace. The default, and the only setting that computes a
+ * Bit 0: representative scoring and perturbation; bit 1: selection and read plan (a kernel of
+ * its own only for batches of many (sequence, KV head) pairs; for few pairs that work is the
+ * first phase of the attention kernel); bit 2: exact attention and merge. A stage that is
+ * skipped reuses what an earlier full call with the same arguments left in the same workspace. The default, and the only setting that computes a
  * decode step, is SANTAPP_STAGE_ALL.
  */
 enum { SANTAPP_STAGE_ROUTE = 1, SANTAPP_STAGE_SELECT = 2, SANTAPP_STAGE_ATTEND = 4, SANTAPP_STAGE_ALL = 7 };

@@ -57,6 +57,7 @@ class CTeams(ctypes.Structure):
     _fields_ = [("k_packed", ctypes.c_void_p), ("v_packed", ctypes.c_void_p), ("rep_keys", ctypes.c_void_p),
                 ("team_row_start", ctypes.c_void_p), ("row_token", ctypes.c_void_p),
                 ("seq_row_off", ctypes.c_void_p), ("seq_team_off", ctypes.c_void_p),
+                ("rep_abs_max", ctypes.c_void_p),
                 ("rows_total", ctypes.c_int64), ("teams_total", ctypes.c_int64),
                 ("max_teams_per_seq", ctypes.c_int32), ("max_rows_per_seq", ctypes.c_int32)]
 
@@ -172,9 +173,10 @@ class Teams:
         self.row_token = torch.empty((kv, sizes.rows_total), dtype=torch.int32, device=device)
         self.seq_row_off = torch.empty(geom.n_seqs + 1, dtype=torch.int64, device=device)
         self.seq_team_off = torch.empty(geom.n_seqs + 1, dtype=torch.int64, device=device)
+        self.rep_abs_max = torch.empty((kv, geom.n_seqs), dtype=torch.float32, device=device)
         self.c = CTeams(self.k_packed.data_ptr(), self.v_packed.data_ptr(), self.rep_keys.data_ptr(),
                         self.team_row_start.data_ptr(), self.row_token.data_ptr(),
-                        self.seq_row_off.data_ptr(), self.seq_team_off.data_ptr(),
+                        self.seq_row_off.data_ptr(), self.seq_team_off.data_ptr(), self.rep_abs_max.data_ptr(),
                         sizes.rows_total, sizes.teams_total, sizes.max_teams_per_seq, sizes.max_rows_per_seq)
 
 

@@ -46,7 +46,8 @@ int teams_in_sequence(int N, int P, int R)
 int check_teams(const santapp_geom *g, const santapp_teams *t)
 {
     if (!t) return SANTAPP_ERR_INVALID_ARG;
-    if (!t->k_packed || !t->v_packed || !t->rep_keys || !t->team_row_start || !t->seq_row_off || !t->seq_team_off)
+    if (!t->k_packed || !t->v_packed || !t->rep_keys || !t->team_row_start || !t->seq_row_off || !t->seq_team_off
+        || !t->rep_abs_max)
         return SANTAPP_ERR_INVALID_ARG;
     if (t->rows_total < g->n_seqs || t->teams_total < g->n_seqs || t->max_teams_per_seq < 1)
         return SANTAPP_ERR_INVALID_ARG;
@@ -71,9 +72,9 @@ BatchView make_view(const santapp_geom *g, const santapp_teams *t)
 
 // Workspace layout shared by the sparse and the dense call. Offsets in bytes.
 struct DecodeLayout {
-    size_t ctl, y, sel_team, sel_logc, tau, seg_prefix, seg_row, seg_mask, seg_logc, pair_nseg, pair_rows,
-        pair_union, pair_prefix, partials, total;
-    int seg_cap, grid, n_pairs;
+    size_t ctl, y32, seg_prefix, seg_row, seg_mask, seg_logc, pair_nseg, pair_rows, pair_prefix, partials, total;
+    int seg_cap, grid, n_pairs, ctas_per_pair;
+    bool static_split;
 };
 
 DecodeLayout decode_layout(const santapp_geom *g, const santapp_teams *t, int K, bool dense, int grid)
@@ -82,23 +83,23 @@ DecodeLayout decode_layout(const santapp_geom *g, const santapp_teams *t, int K,
     const int G = g->n_q_heads / g->n_kv_heads;
     L.n_pairs = g->n_seqs * g->n_kv_heads;
     L.grid = grid;
+    // few pairs: a fixed number of CTAs per pair and the plan built inside the attention kernel;
+    // many pairs: equal row ranges over a plan in global memory
+    L.static_split = (int64_t)L.n_pairs * 9 <= grid;
+    L.ctas_per_pair = L.static_split ? grid / L.n_pairs : 1;
     int64_t cap = dense ? 1 : (int64_t)G * K;
     if (cap > t->max_teams_per_seq) cap = t->max_teams_per_seq;
     L.seg_cap = (int)cap + 1;                                   // + the suffix segment
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
-    L.ctl = take(sizeof(int32_t) * (2 * (size_t)L.n_pairs + 2));
-    L.y = take(dense ? 0 : sizeof(double) * (size_t)g->n_q_heads * (size_t)t->teams_total);
-    L.sel_team = take(dense ? 0 : sizeof(int32_t) * (size_t)g->n_seqs * g->n_q_heads * K);
-    L.sel_logc = take(dense ? 0 : sizeof(float) * (size_t)g->n_seqs * g->n_q_heads * K);
-    L.tau = take(dense ? 0 : sizeof(double) * (size_t)g->n_seqs * g->n_q_heads);
+    L.ctl = take(sizeof(int32_t) * ((size_t)L.n_pairs + 2));
+    L.y32 = take(dense ? 0 : sizeof(float) * (size_t)g->n_q_heads * (size_t)t->teams_total);
     L.seg_prefix = take(sizeof(int32_t) * (size_t)L.n_pairs * (L.seg_cap + 1));
     L.seg_row = take(sizeof(int32_t) * (size_t)L.n_pairs * L.seg_cap);
     L.seg_mask = take(sizeof(uint32_t) * (size_t)L.n_pairs * L.seg_cap);
     L.seg_logc = take(sizeof(float) * (size_t)L.n_pairs * L.seg_cap * kMaxGroup);
     L.pair_nseg = take(sizeof(int32_t) * (size_t)L.n_pairs);
     L.pair_rows = take(sizeof(int32_t) * (size_t)L.n_pairs);
-    L.pair_union = take(sizeof(int32_t) * (size_t)L.n_pairs);
     L.pair_prefix = take(sizeof(int64_t) * ((size_t)L.n_pairs + 1));
     L.partials = take(sizeof(float) * ((size_t)grid + L.n_pairs) * G * kPartialStride);
     L.total = off;
@@ -108,9 +109,8 @@ DecodeLayout decode_layout(const santapp_geom *g, const santapp_teams *t, int K,
 void fill_plan(const DecodeLayout &L, char *ws, PlanView &plan, Control &ctl)
 {
     int32_t *c = reinterpret_cast<int32_t *>(ws + L.ctl);
-    ctl.select_ticket = c;
-    ctl.attend_ticket = c + L.n_pairs;
-    ctl.plan_ticket = c + 2 * L.n_pairs;
+    ctl.attend_ticket = c;
+    ctl.plan_ticket = c + L.n_pairs;
     plan.seg_cap = L.seg_cap;
     plan.seg_prefix = reinterpret_cast<int32_t *>(ws + L.seg_prefix);
     plan.seg_row = reinterpret_cast<int32_t *>(ws + L.seg_row);
@@ -118,7 +118,7 @@ void fill_plan(const DecodeLayout &L, char *ws, PlanView &plan, Control &ctl)
     plan.seg_logc = reinterpret_cast<float *>(ws + L.seg_logc);
     plan.pair_nseg = reinterpret_cast<int32_t *>(ws + L.pair_nseg);
     plan.pair_rows = reinterpret_cast<int32_t *>(ws + L.pair_rows);
-    plan.pair_union_rows = reinterpret_cast<int32_t *>(ws + L.pair_union);
+    plan.pair_union_rows = nullptr;
     plan.pair_row_prefix = reinterpret_cast<int64_t *>(ws + L.pair_prefix);
 }
 
@@ -177,7 +177,7 @@ int santapp_build_teams(const santapp_geom *geom, const int32_t *prompt_len_host
     if (rc != SANTAPP_OK) return rc;
     if (!k_prompt || !v_prompt || !teams || !workspace) return SANTAPP_ERR_INVALID_ARG;
     if (!teams->k_packed || !teams->v_packed || !teams->rep_keys || !teams->team_row_start || !teams->row_token
-        || !teams->seq_row_off || !teams->seq_team_off)
+        || !teams->seq_row_off || !teams->seq_team_off || !teams->rep_abs_max)
         return SANTAPP_ERR_INVALID_ARG;
     if (workspace_bytes < sz.build_workspace_bytes) return SANTAPP_ERR_WORKSPACE_TOO_SMALL;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -221,12 +221,14 @@ int santapp_build_teams(const santapp_geom *geom, const int32_t *prompt_len_host
     p.max_parents_per_seq = max_parents;
     err = launch_build_teams(p, s);
     if (err != cudaSuccess) return cuda_fail(err, "build_teams launch");
+    err = launch_rep_abs_max(p.bv, p.rep_keys, teams->rep_abs_max, s);
+    if (err != cudaSuccess) return cuda_fail(err, "rep_abs_max launch");
     return SANTAPP_OK;
 }
 
 size_t santapp_decode_workspace_bytes(const santapp_geom *geom, const santapp_teams *teams, int32_t n_sample)
 {
-    if (check_geom(geom) != SANTAPP_OK || !teams || n_sample < 1 || n_sample > 256) return 0;
+    if (check_geom(geom) != SANTAPP_OK || !teams || n_sample < 1 || n_sample > 128) return 0;
     return decode_layout(geom, teams, n_sample, false, attend_grid_size()).total;
 }
 
@@ -248,7 +250,7 @@ int santapp_decode_attn(const santapp_geom *geom, const santapp_teams *teams, co
     if ((rc = check_teams(geom, teams)) != SANTAPP_OK) return rc;
     if (!q || !out || !workspace) return SANTAPP_ERR_INVALID_ARG;
     if (n_sample < 1 || suffix_cap < 0) return SANTAPP_ERR_INVALID_ARG;
-    if (n_sample > 256) return SANTAPP_ERR_UNSUPPORTED;
+    if (n_sample > 128) return SANTAPP_ERR_UNSUPPORTED;
     if (suffix_cap > 0 && suffix_len_dev && (!k_suffix || !v_suffix)) return SANTAPP_ERR_INVALID_ARG;
     if (!(scale >= 0.f) || isinf(scale)) return SANTAPP_ERR_INVALID_ARG;
     if ((int64_t)geom->n_seqs * geom->n_kv_heads * (int64_t)suffix_cap >= (int64_t)1 << 31) return SANTAPP_ERR_UNSUPPORTED;
@@ -265,12 +267,12 @@ int santapp_decode_attn(const santapp_geom *geom, const santapp_teams *teams, co
     Control ctl;
     fill_plan(L, ws, plan, ctl);
 
-    RouteParams rp;
+    ScoreParams rp;
     rp.bv = make_view(geom, teams);
     rp.rep_keys = static_cast<const uint16_t *>(teams->rep_keys);
     rp.team_row_start = teams->team_row_start;
     rp.q = static_cast<const uint16_t *>(q);
-    rp.y = reinterpret_cast<double *>(ws + L.y);
+    rp.y32 = reinterpret_cast<float *>(ws + L.y32);
     rp.n_sample = n_sample;
     rp.seed_lo = (uint32_t)(seed & 0xFFFFFFFFull);
     rp.seed_hi = (uint32_t)(seed >> 32);
@@ -283,36 +285,37 @@ int santapp_decode_attn(const santapp_geom *geom, const santapp_teams *teams, co
     rp.status = dbg ? dbg->status : nullptr;
     cudaError_t err = cudaSuccess;
     if (g_stage_mask & SANTAPP_STAGE_ROUTE) {
-        err = launch_route_score(rp, teams->max_teams_per_seq, s);
-        if (err != cudaSuccess) return cuda_fail(err, "route_score launch");
+        err = launch_score32(rp, teams->max_teams_per_seq, s);
+        if (err != cudaSuccess) return cuda_fail(err, "score launch");
         ++g_launches;
     }
 
-    SelectParams sp;
-    sp.bv = rp.bv;
-    sp.team_row_start = teams->team_row_start;
-    sp.y = rp.y;
-    sp.n_sample = n_sample;
-    sp.seed_lo = rp.seed_lo;
-    sp.seed_hi = rp.seed_hi;
-    sp.step = step;
-    sp.step_dev = step_dev;
-    sp.stream_base = stream_base;
-    sp.sel_team = reinterpret_cast<int32_t *>(ws + L.sel_team);
-    sp.sel_logc = reinterpret_cast<float *>(ws + L.sel_logc);
-    sp.tau = reinterpret_cast<double *>(ws + L.tau);
-    sp.suffix_len = suffix_len_dev;
-    sp.suffix_cap = suffix_cap;
-    sp.plan = plan;
-    sp.ctl = ctl;
-    sp.n_pairs = L.n_pairs;
-    sp.dbg_sel_idx = dbg ? dbg->sel_idx : nullptr;
-    sp.dbg_sel_logc = dbg ? dbg->sel_logc : nullptr;
-    sp.dbg_tau = dbg ? dbg->tau : nullptr;
-    sp.dbg_union_rows = dbg ? dbg->union_rows : nullptr;
-    if (g_stage_mask & SANTAPP_STAGE_SELECT) {
-        err = launch_select_plan(sp, teams->max_teams_per_seq, s);
-        if (err != cudaSuccess) return cuda_fail(err, "select_plan launch");
+    PlanParams pp;
+    pp.in.bv = rp.bv;
+    pp.in.y32 = rp.y32;
+    pp.in.rep_keys = rp.rep_keys;
+    pp.in.team_row_start = teams->team_row_start;
+    pp.in.rep_abs_max = teams->rep_abs_max;
+    pp.in.q = rp.q;
+    pp.in.n_sample = n_sample;
+    pp.in.seed_lo = rp.seed_lo;
+    pp.in.seed_hi = rp.seed_hi;
+    pp.in.step = step;
+    pp.in.step_dev = step_dev;
+    pp.in.stream_base = stream_base;
+    pp.in.scale = sc;
+    pp.in.suffix_len = suffix_len_dev;
+    pp.in.suffix_cap = suffix_cap;
+    pp.in.dbg_sel_idx = dbg ? dbg->sel_idx : nullptr;
+    pp.in.dbg_sel_logc = dbg ? dbg->sel_logc : nullptr;
+    pp.in.dbg_tau = dbg ? dbg->tau : nullptr;
+    pp.in.dbg_union_rows = dbg ? dbg->union_rows : nullptr;
+    pp.plan = plan;
+    pp.ctl = ctl;
+    pp.n_pairs = L.n_pairs;
+    if (!L.static_split && (g_stage_mask & SANTAPP_STAGE_SELECT)) {
+        err = launch_plan(pp, s);
+        if (err != cudaSuccess) return cuda_fail(err, "plan launch");
         ++g_launches;
     }
 
@@ -325,14 +328,17 @@ int santapp_decode_attn(const santapp_geom *geom, const santapp_teams *teams, co
     ap.q = rp.q;
     ap.qk_scale_log2 = (float)(sc * 1.4426950408889634);
     ap.plan = plan;
+    ap.in = pp.in;
     ap.ctl = ctl;
     ap.n_pairs = L.n_pairs;
     ap.partials = reinterpret_cast<float *>(ws + L.partials);
     ap.out = out;
     ap.status = rp.status;
     ap.min_rows_per_cta = 64;
+    ap.ctas_per_pair = L.ctas_per_pair;
     if (g_stage_mask & SANTAPP_STAGE_ATTEND) {
-        err = launch_attend(ap, false, grid, s);
+        const int launch_grid = L.static_split ? L.n_pairs * L.ctas_per_pair : grid;
+        err = launch_attend(ap, false, L.static_split, launch_grid, s);
         if (err != cudaSuccess) return cuda_fail(err, "attend launch");
         ++g_launches;
     }
@@ -366,21 +372,27 @@ int santapp_dense_decode_attn(const santapp_geom *geom, const santapp_teams *tea
     Control ctl;
     fill_plan(L, ws, plan, ctl);
 
-    SelectParams sp;
-    memset(&sp, 0, sizeof(sp));
-    sp.bv = make_view(geom, teams);
-    sp.team_row_start = teams->team_row_start;
-    sp.suffix_len = suffix_len_dev;
-    sp.suffix_cap = suffix_cap;
-    sp.plan = plan;
-    sp.ctl = ctl;
-    sp.n_pairs = L.n_pairs;
-    cudaError_t err = launch_dense_plan(sp, s);
-    if (err != cudaSuccess) return cuda_fail(err, "dense_plan launch");
-    ++g_launches;
+    PlanParams pp;
+    memset(&pp, 0, sizeof(pp));
+    pp.in.bv = make_view(geom, teams);
+    pp.in.suffix_len = suffix_len_dev;
+    pp.in.suffix_cap = suffix_cap;
+    pp.plan = plan;
+    pp.ctl = ctl;
+    pp.n_pairs = L.n_pairs;
+    cudaError_t err;
+    if (L.static_split) {
+        // the plan is trivial and built inside the kernel; only the merge tickets need clearing
+        err = cudaMemsetAsync(ctl.attend_ticket, 0, sizeof(int32_t) * (size_t)L.n_pairs, s);
+        if (err != cudaSuccess) return cuda_fail(err, "ticket memset");
+    } else {
+        err = launch_dense_plan(pp, s);
+        if (err != cudaSuccess) return cuda_fail(err, "dense_plan launch");
+        ++g_launches;
+    }
 
     AttendParams ap;
-    ap.bv = sp.bv;
+    ap.bv = pp.in.bv;
     ap.k_packed = static_cast<const uint16_t *>(teams->k_packed);
     ap.v_packed = static_cast<const uint16_t *>(teams->v_packed);
     ap.k_suffix = static_cast<const uint16_t *>(k_suffix);
@@ -388,13 +400,16 @@ int santapp_dense_decode_attn(const santapp_geom *geom, const santapp_teams *tea
     ap.q = static_cast<const uint16_t *>(q);
     ap.qk_scale_log2 = (float)(sc * 1.4426950408889634);
     ap.plan = plan;
+    ap.in = pp.in;
     ap.ctl = ctl;
     ap.n_pairs = L.n_pairs;
     ap.partials = reinterpret_cast<float *>(ws + L.partials);
     ap.out = out;
     ap.status = nullptr;
     ap.min_rows_per_cta = 64;
-    err = launch_attend(ap, true, grid, s);
+    ap.ctas_per_pair = L.ctas_per_pair;
+    const int launch_grid = L.static_split ? L.n_pairs * L.ctas_per_pair : grid;
+    err = launch_attend(ap, true, L.static_split, launch_grid, s);
     if (err != cudaSuccess) return cuda_fail(err, "attend launch");
     ++g_launches;
     return SANTAPP_OK;

@@ -3,13 +3,18 @@
 // (applied as s_i - log c_g, so the same correction enters the mass and the value sum), every
 // suffix row with weight e^{s_i}; Eq. (method-estimate).
 //
-// Work split. The rows of all (sequence, KV head) pairs form one global row space that is cut
-// into equal contiguous ranges, one per CTA (split-K by rows, not by teams), one CTA per SM.
-// Inside a CTA each warp takes a contiguous run of 16-row blocks. A warp streams its own blocks
-// through a private two-slot ring in shared memory with 16-byte asynchronous copies (a whole
-// 256-byte row per half warp, XOR swizzled so that ldmatrix is bank-conflict free), one block
-// ahead of the one it is evaluating, together with the block's per-row head masks and
-// corrections; completion is tracked with cp.async groups, so the kernel has no spin-wait.
+// Work split, two ways (split-K by rows, never by teams; one CTA per SM):
+//   static   a fixed number of CTAs per (sequence, KV head) pair. Every CTA of a pair first
+//            runs the pair's sampling and builds its read plan in shared memory (pairplan.cuh;
+//            the dense kernel's plan is trivial), then takes its share of the pair's rows. No
+//            plan kernel, no global plan: the shortest path for few pairs.
+//   dynamic  the rows of all pairs form one global row space cut into equal contiguous ranges;
+//            plans come from a plan kernel through global memory. Best balance for many pairs.
+// Inside a CTA each warp takes a contiguous run of 16-row blocks and streams them through a
+// private two-slot ring in shared memory with 16-byte asynchronous copies (a whole 256-byte row
+// per half warp, XOR swizzled so that ldmatrix is bank-conflict free), one block ahead of the one
+// it is evaluating, together with the block's per-row head masks and corrections; completion is
+// tracked with cp.async groups, so the kernel has no spin-wait.
 //
 // Arithmetic. The GQA group is a real MMA tile: the query heads of the KV head (at most 8)
 // are the M rows of S^T = q K^T (mma.sync m16n8k16, bf16 inputs, fp32 accumulation), so one
@@ -23,20 +28,20 @@
 #include <math_constants.h>
 
 #include "common.cuh"
+#include "pairplan.cuh"
 
 namespace santapp {
 
 namespace {
 
-constexpr int kWarps = 12;
-constexpr int kAttendThreads = 32 * kWarps;
+constexpr int kWarps = kPlanWarps;                          // 12
+constexpr int kAttendThreads = kPlanThreads;
 constexpr int kBlockRows = 16;                              // rows per block (one warp, one MMA K step)
 constexpr int kSlots = 2;                                   // ring slots per warp
 constexpr int kRowBytes = kHeadDim * 2;                     // one bf16 row
 constexpr int kTileBytes = kBlockRows * kRowBytes;          // K tile or V tile of a block
 constexpr int kSlotBytes = 2 * kTileBytes;                  // K tile then V tile
-constexpr int kSegMax = 1025;                               // plan segments of one pair (G * K + suffix)
-constexpr int kPairMax = 512;                               // pairs whose offsets are staged
+constexpr int kPairMax = 512;                               // pairs whose offsets are staged (dynamic split)
 constexpr int kMaxAttendGrid = 512;
 constexpr uint32_t kNoRow = 0xFFFFFFFFu;
 
@@ -97,7 +102,8 @@ struct Smem {
     static constexpr size_t pair_nseg = pair_prefix + (kPairMax + 1) * 8;       // int [kPairMax]
     static constexpr size_t misc = pair_nseg + kPairMax * 4;                    // flags
     static constexpr size_t total = misc + 64;
-    // aliases of the ring, used only after a span's blocks are consumed
+    // aliases of the ring: plan scratch before a pair's rows are streamed, merge scratch after
+    static_assert(sizeof(PlanScratch<G>) <= ring_bytes, "plan scratch must fit in the ring");
     static constexpr size_t red_acc = ring;                                     // float [warps][G][128]
     static constexpr size_t red_m = red_acc + (size_t)kWarps * G * kHeadDim * 4;   // float [warps][G]
     static constexpr size_t red_l = red_m + (size_t)kWarps * G * 4;
@@ -106,7 +112,7 @@ struct Smem {
     static_assert(total <= 227 * 1024, "shared memory budget");
 };
 
-template <int G, bool kAll>
+template <int G, bool kAll, bool kStatic>
 __global__ void __launch_bounds__(kAttendThreads, 1)
 attend_kernel(AttendParams p)
 {
@@ -117,25 +123,35 @@ attend_kernel(AttendParams p)
     uint32_t *seg_mask = reinterpret_cast<uint32_t *>(smem + S::seg_mask);
     int64_t *pair_prefix = reinterpret_cast<int64_t *>(smem + S::pair_prefix);
     int *pair_nseg = reinterpret_cast<int *>(smem + S::pair_nseg);
-    int *last_flag = reinterpret_cast<int *>(smem + S::misc);
+    int *misc = reinterpret_cast<int *>(smem + S::misc);
+    int *last_flag = misc;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = lane >> 2, c = lane & 3;                 // MMA fragment coordinates
     const int hw = lane >> 4, chunk = lane & 15;           // copy coordinates: row parity, 16-byte chunk
 
-    for (int i = tid; i <= p.n_pairs; i += kAttendThreads) pair_prefix[i] = p.plan.pair_row_prefix[i];
-    for (int i = tid; i < p.n_pairs; i += kAttendThreads) pair_nseg[i] = p.plan.pair_nseg[i];
-    __syncthreads();
+    const uint32_t ring_w = smem_u32(smem + S::ring) + (uint32_t)warp * kSlots * kSlotBytes;
+    float *logc_w = reinterpret_cast<float *>(smem + S::logc_tab) + warp * kSlots * kBlockRows * kMaxGroup;
+    unsigned char *mask_w = smem + S::mask_tab + warp * kSlots * kBlockRows;
+    const int cap = p.plan.seg_cap;
 
-    const int64_t total = pair_prefix[p.n_pairs];
-    int64_t rows_per_cta = (total + gridDim.x - 1) / gridDim.x;
-    if (rows_per_cta < p.min_rows_per_cta) rows_per_cta = p.min_rows_per_cta;
-    int64_t r0 = (int64_t)blockIdx.x * rows_per_cta;
-    if (r0 >= total) return;
-    const int64_t r1 = min(r0 + rows_per_cta, total);
-
-    int pair;
-    {
+    // ---- which (pair, row range) spans this CTA works on ----
+    int pair, sub = 0;
+    int64_t r0 = 0, r1 = 0, rows_per_cta = 0;              // dynamic split: global row range
+    if (kStatic) {
+        pair = blockIdx.x / p.ctas_per_pair;
+        sub = blockIdx.x - pair * p.ctas_per_pair;
+        if (pair >= p.n_pairs) return;
+    } else {
+        for (int i = tid; i <= p.n_pairs; i += kAttendThreads) pair_prefix[i] = p.plan.pair_row_prefix[i];
+        for (int i = tid; i < p.n_pairs; i += kAttendThreads) pair_nseg[i] = p.plan.pair_nseg[i];
+        __syncthreads();
+        const int64_t total = pair_prefix[p.n_pairs];
+        rows_per_cta = (total + gridDim.x - 1) / gridDim.x;
+        if (rows_per_cta < p.min_rows_per_cta) rows_per_cta = p.min_rows_per_cta;
+        r0 = (int64_t)blockIdx.x * rows_per_cta;
+        if (r0 >= total) return;
+        r1 = min(r0 + rows_per_cta, total);
         int lo = 0, hi = p.n_pairs;
         while (hi - lo > 1) {
             const int mid = (lo + hi) >> 1;
@@ -144,21 +160,69 @@ attend_kernel(AttendParams p)
         pair = lo;
     }
 
-    const uint32_t ring_w = smem_u32(smem + S::ring) + (uint32_t)warp * kSlots * kSlotBytes;
-    float *logc_w = reinterpret_cast<float *>(smem + S::logc_tab) + warp * kSlots * kBlockRows * kMaxGroup;
-    unsigned char *mask_w = smem + S::mask_tab + warp * kSlots * kBlockRows;
-
-    while (r0 < r1) {
-        const int64_t pb = pair_prefix[pair], pe = pair_prefix[pair + 1];
-        const int a = (int)(r0 - pb);
-        const int bnd = (int)(min(r1, pe) - pb);
+    while (true) {
+        int a, bnd, nseg, n_ctas, first_slot, slot_id;
+        int64_t pb = 0, pe = 0;
         const int b = pair / p.bv.n_kv, j = pair - b * p.bv.n_kv;
-        const int cap = p.plan.seg_cap;
-        const int nseg = pair_nseg[pair];
         const float *g_logc = p.plan.seg_logc + (size_t)pair * cap * kMaxGroup;
 
-        __syncthreads();                                   // the previous span is done with the tables
-        {
+        if (kStatic) {
+            int rows;
+            if (kAll) {
+                __syncthreads();
+                if (tid == 0) {
+                    const int64_t row0 = p.bv.seq_row_off[b];
+                    const int N = (int)(p.bv.seq_row_off[b + 1] - row0);
+                    int t = 0;
+                    if (p.in.suffix_len != nullptr && p.in.suffix_cap > 0)
+                        t = max(0, min(p.in.suffix_len[b], p.in.suffix_cap));
+                    const uint32_t all_heads = (1u << G) - 1u;
+                    seg_prefix[0] = 0;
+                    seg_row[0] = (int32_t)row0;
+                    seg_mask[0] = all_heads;
+                    int ns = 1, rw = N;
+                    if (t > 0) {
+                        seg_prefix[1] = rw;
+                        seg_row[1] = pair * p.in.suffix_cap;
+                        seg_mask[1] = all_heads | kSrcSuffix;
+                        rw += t;
+                        ns = 2;
+                    }
+                    seg_prefix[ns] = rw;
+                    misc[2] = ns;
+                    misc[3] = rw;
+                }
+                __syncthreads();
+                nseg = misc[2];
+                rows = misc[3];
+            } else {
+                PlanScratch<G> &scratch = *reinterpret_cast<PlanScratch<G> *>(smem + S::ring);
+                build_pair_plan<G>(p.in, pair, scratch, seg_prefix, seg_row, seg_mask,
+                                   p.plan.seg_logc + (size_t)pair * cap * kMaxGroup, nseg, rows, sub == 0);
+            }
+            const int per_cta = max((rows + p.ctas_per_pair - 1) / p.ctas_per_pair, p.min_rows_per_cta);
+            n_ctas = (rows + per_cta - 1) / per_cta;
+            a = sub * per_cta;
+            bnd = min(a + per_cta, rows);
+            first_slot = pair * p.ctas_per_pair;
+            slot_id = first_slot + sub;
+            if (a >= rows) {                               // more CTAs than this pair needs
+                if (p.ctas_per_pair > 1) return;
+                pair += gridDim.x;
+                if (pair >= p.n_pairs) return;
+                continue;
+            }
+        } else {
+            pb = pair_prefix[pair];
+            pe = pair_prefix[pair + 1];
+            a = (int)(r0 - pb);
+            bnd = (int)(min(r1, pe) - pb);
+            nseg = pair_nseg[pair];
+            const int c_lo = (int)(pb / rows_per_cta), c_hi = (int)((pe - 1) / rows_per_cta);
+            n_ctas = c_hi - c_lo + 1;
+            first_slot = c_lo + pair;
+            slot_id = blockIdx.x + pair;
+            __syncthreads();                               // the previous span is done with the tables
             // one round trip: every load is issued before the first store
             const int32_t *g_prefix = p.plan.seg_prefix + (size_t)pair * (cap + 1);
             const int32_t *g_row = p.plan.seg_row + (size_t)pair * cap;
@@ -362,7 +426,6 @@ attend_kernel(AttendParams p)
             }
         }
         __syncthreads();
-        const int slot_id = blockIdx.x + pair;
         float *part = p.partials + (size_t)slot_id * G * kPartialStride;
         for (int e = tid; e < G * kHeadDim; e += kAttendThreads) {
             const int h = e >> 7, d = e & 127;
@@ -384,8 +447,6 @@ attend_kernel(AttendParams p)
         }
 
         // ---- last CTA of the pair: log-sum-exp merge of the pair's partials ----
-        const int c_lo = (int)(pb / rows_per_cta), c_hi = (int)((pe - 1) / rows_per_cta);
-        const int n_ctas = c_hi - c_lo + 1;
         __threadfence();
         __syncthreads();
         if (tid == 0) *last_flag = (atomicAdd(p.ctl.attend_ticket + pair, 1) == n_ctas - 1);
@@ -396,7 +457,7 @@ attend_kernel(AttendParams p)
             // The pair's partials are contiguous in memory. Stage them in shared memory a chunk
             // at a time with asynchronous copies, then merge from there: thread (h, lane) owns
             // four output columns of head h.
-            const float *first = p.partials + (size_t)(c_lo + pair) * G * kPartialStride;
+            const float *first = p.partials + (size_t)first_slot * G * kPartialStride;
             float *stage = reinterpret_cast<float *>(smem + S::ring);
             constexpr int kPer = G * kPartialStride;                   // floats per partial
             const int h = tid >> 5;
@@ -445,26 +506,41 @@ attend_kernel(AttendParams p)
                     atomicOr(p.status, 1);
             }
         }
-        r0 = pb + bnd;
-        ++pair;
+
+        // ---- next span ----
+        if (kStatic) {
+            if (p.ctas_per_pair > 1) return;
+            pair += gridDim.x;                             // more pairs than CTAs: whole pairs, round robin
+            if (pair >= p.n_pairs) return;
+        } else {
+            r0 = pb + bnd;
+            if (r0 >= r1) return;
+            ++pair;
+        }
     }
 }
 
 template <int G>
-cudaError_t launch_attend_g(const AttendParams &p, bool all_heads, int grid, cudaStream_t s)
+cudaError_t launch_attend_g(const AttendParams &p, bool all_heads, bool static_split, int grid, cudaStream_t s)
 {
     const size_t smem = Smem<G>::total;
     static thread_local bool attr_set = false;
     if (!attr_set) {
-        cudaError_t err = cudaFuncSetAttribute(attend_kernel<G, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                               (int)smem);
-        if (err != cudaSuccess) return err;
-        err = cudaFuncSetAttribute(attend_kernel<G, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (err != cudaSuccess) return err;
+        const void *fns[4] = {(const void *)attend_kernel<G, true, true>, (const void *)attend_kernel<G, true, false>,
+                              (const void *)attend_kernel<G, false, true>, (const void *)attend_kernel<G, false, false>};
+        for (const void *fn : fns) {
+            cudaError_t err = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (err != cudaSuccess) return err;
+        }
         attr_set = true;
     }
-    if (all_heads) attend_kernel<G, true><<<grid, kAttendThreads, smem, s>>>(p);
-    else           attend_kernel<G, false><<<grid, kAttendThreads, smem, s>>>(p);
+    if (all_heads) {
+        if (static_split) attend_kernel<G, true, true><<<grid, kAttendThreads, smem, s>>>(p);
+        else              attend_kernel<G, true, false><<<grid, kAttendThreads, smem, s>>>(p);
+    } else {
+        if (static_split) attend_kernel<G, false, true><<<grid, kAttendThreads, smem, s>>>(p);
+        else              attend_kernel<G, false, false><<<grid, kAttendThreads, smem, s>>>(p);
+    }
     return cudaGetLastError();
 }
 
@@ -480,17 +556,17 @@ int attend_grid_size()
 int attend_max_segments() { return kSegMax; }
 int attend_max_pairs() { return kPairMax; }
 
-cudaError_t launch_attend(const AttendParams &p, bool all_heads, int grid, cudaStream_t s)
+cudaError_t launch_attend(const AttendParams &p, bool all_heads, bool static_split, int grid, cudaStream_t s)
 {
     switch (p.bv.group) {
-        case 1: return launch_attend_g<1>(p, all_heads, grid, s);
-        case 2: return launch_attend_g<2>(p, all_heads, grid, s);
-        case 3: return launch_attend_g<3>(p, all_heads, grid, s);
-        case 4: return launch_attend_g<4>(p, all_heads, grid, s);
-        case 5: return launch_attend_g<5>(p, all_heads, grid, s);
-        case 6: return launch_attend_g<6>(p, all_heads, grid, s);
-        case 7: return launch_attend_g<7>(p, all_heads, grid, s);
-        case 8: return launch_attend_g<8>(p, all_heads, grid, s);
+        case 1: return launch_attend_g<1>(p, all_heads, static_split, grid, s);
+        case 2: return launch_attend_g<2>(p, all_heads, static_split, grid, s);
+        case 3: return launch_attend_g<3>(p, all_heads, static_split, grid, s);
+        case 4: return launch_attend_g<4>(p, all_heads, static_split, grid, s);
+        case 5: return launch_attend_g<5>(p, all_heads, static_split, grid, s);
+        case 6: return launch_attend_g<6>(p, all_heads, static_split, grid, s);
+        case 7: return launch_attend_g<7>(p, all_heads, static_split, grid, s);
+        case 8: return launch_attend_g<8>(p, all_heads, static_split, grid, s);
         default: return cudaErrorInvalidValue;
     }
 }

@@ -43,17 +43,16 @@ struct PlanView {
 };
 
 struct Control {
-    int32_t *select_ticket;         // [n_pairs]
     int32_t *plan_ticket;           // [1]
     int32_t *attend_ticket;         // [n_pairs]
 };
 
-struct RouteParams {
+struct ScoreParams {
     BatchView bv;
     const uint16_t *rep_keys;       // [n_kv][teams_total][128]
     const int32_t *team_row_start;  // [n_kv][teams_total + n_seqs]
     const uint16_t *q;              // [n_seqs][n_q][128]
-    double *y;                      // [n_q][teams_total] perturbed routing scores
+    float *y32;                     // [n_q][teams_total] fp32 perturbed routing scores
     int n_sample;
     uint32_t seed_lo, seed_hi, step, stream_base;
     const uint32_t *step_dev;       // nullable: added to step
@@ -63,26 +62,32 @@ struct RouteParams {
     int32_t *status;                // nullable
 };
 
-struct SelectParams {
+// What the sampling step reads (see pairplan.cuh).
+struct PlanInputs {
     BatchView bv;
-    const int32_t *team_row_start;
-    const double *y;
+    const float *y32;               // [n_q][teams_total]
+    const uint16_t *rep_keys;       // [n_kv][teams_total][128]
+    const int32_t *team_row_start;  // [n_kv][teams_total + n_seqs]
+    const float *rep_abs_max;       // [n_kv][n_seqs]
+    const uint16_t *q;              // [n_seqs][n_q][128]
     int n_sample;
     uint32_t seed_lo, seed_hi, step, stream_base;
     const uint32_t *step_dev;       // nullable: added to step
-    int32_t *sel_team;              // [n_seqs][n_q][n_sample]
-    float *sel_logc;                // [n_seqs][n_q][n_sample] natural log
-    double *tau;                    // [n_seqs][n_q]
+    double scale;
     const int32_t *suffix_len;      // nullable
     int suffix_cap;
-    PlanView plan;
-    Control ctl;
-    int n_pairs;
     // diagnostics (nullable)
     int32_t *dbg_sel_idx;
     float *dbg_sel_logc;
     double *dbg_tau;
     int32_t *dbg_union_rows;
+};
+
+struct PlanParams {
+    PlanInputs in;
+    PlanView plan;
+    Control ctl;
+    int n_pairs;
 };
 
 struct AttendParams {
@@ -91,22 +96,27 @@ struct AttendParams {
     const uint16_t *k_suffix, *v_suffix;    // [n_seqs][n_kv][suffix_cap][128]
     const uint16_t *q;
     float qk_scale_log2;            // scale * log2(e)
-    PlanView plan;
+    PlanView plan;                  // plan in global memory (dynamic split); seg_logc in both modes
+    PlanInputs in;                  // static split: the plan is built inside the kernel
     Control ctl;
     int n_pairs;
-    float *partials;                // [grid + n_pairs][group][kPartialStride]
+    float *partials;                // [slots][group][kPartialStride]
     float *out;                     // [n_seqs][n_q][128]
     int32_t *status;                // nullable
     int min_rows_per_cta;
+    int ctas_per_pair;              // static split: CTAs that share one (sequence, KV head) pair
 };
 
 // ---------------------------------------------------------------------------------------------
 // Host launchers (each returns the cudaError_t of its launches).
 // ---------------------------------------------------------------------------------------------
-cudaError_t launch_route_score(const RouteParams &p, int max_teams_per_seq, cudaStream_t s);
-cudaError_t launch_select_plan(const SelectParams &p, int max_teams_per_seq, cudaStream_t s);
-cudaError_t launch_dense_plan(const SelectParams &p, cudaStream_t s);
-cudaError_t launch_attend(const AttendParams &p, bool all_heads, int grid, cudaStream_t s);
+cudaError_t launch_score32(const ScoreParams &p, int max_teams_per_seq, cudaStream_t s);
+cudaError_t launch_rep_abs_max(const BatchView &bv, const uint16_t *rep_keys, float *rep_abs_max, cudaStream_t s);
+cudaError_t launch_plan(const PlanParams &p, cudaStream_t s);
+cudaError_t launch_dense_plan(const PlanParams &p, cudaStream_t s);
+// split: 0 = rows of all pairs cut into equal ranges (plan read from global memory),
+//        1 = a fixed number of CTAs per pair (plan built in the kernel; dense: trivial plan)
+cudaError_t launch_attend(const AttendParams &p, bool all_heads, bool static_split, int grid, cudaStream_t s);
 int attend_grid_size();
 int attend_max_segments();
 int attend_max_pairs();

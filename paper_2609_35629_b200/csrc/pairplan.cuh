@@ -1,0 +1,384 @@
+// Sampling and read plan of one (sequence, KV head) pair, as a block-wide device function
+// (Algorithm 1: Gumbel-top-K over the perturbed routing scores, the conditional inclusion
+// correction of Eq. method-inclusion, and the GQA union of the heads' selections).
+//
+// The scorer leaves fp32 perturbed scores Y32 for every (head, team) together with a bound E on
+// |Y32 - Y| against the exact fp64 score Y. The sample must be the fp64 one, so per head:
+//   1. a lower bound t on the (K+1)-st largest Y32 (tournament over per-lane maxima);
+//   2. every team with Y32 >= t - 2E is a candidate: that set contains the K+1 largest exact
+//      scores (if K+1 teams have Y32 >= t they have Y >= t - E, so the (K+1)-st largest Y is at
+//      least t - E, and a team with Y above that has Y32 >= t - 2E);
+//   3. the candidates are re-evaluated exactly in fp64 (dot product of bf16 values, log n_g,
+//      Gumbel from the same Philox word) and ranked by (Y descending, team id ascending);
+//   4. the K largest are the sample, the next one is tau, c_g = 1 - exp(-exp(phi_g - tau)).
+// Candidates are processed at most kCandCap at a time with a running top-(K+1) list, so any
+// number of candidates is handled in bounded shared memory.
+// The plan is the union of the heads' samples in team order with head masks, per-head
+// log2(e) * log c_g, segment row prefix, and the exact suffix as a last segment.
+#pragma once
+
+#include <math_constants.h>
+
+#include "common.cuh"
+
+namespace santapp {
+
+constexpr int kPlanThreads = 384;       // block size of every kernel that builds a pair plan
+constexpr int kPlanWarps = kPlanThreads / 32;
+constexpr int kCandCap = 512;           // candidates of one head refined at a time
+constexpr int kListCap = 132;           // running top list: K + 1 <= 129 entries
+constexpr int kTopR = 7;                // per-lane maxima kept for the lower bound
+constexpr int kEntCap = 1024;           // G * K entries of a plan
+constexpr int kSegMax = 1025;           // segments of a plan (entries + suffix)
+constexpr int kBitmapWords = kMaxTeamsPerSeq / 32;
+
+struct HeadScratch {
+    int n_cand, n_list, n_ranges, range_len;
+    float t_lo;                         // candidate threshold on Y32 (lower bound minus guard)
+    float pad[3];
+    int cand_id[kCandCap];
+    double cand_y[kCandCap];
+    double cand_phi[kCandCap];
+    int list_id[2][kListCap];
+    double list_y[2][kListCap];
+    double list_phi[2][kListCap];
+};
+
+template <int G>
+struct PlanScratch {
+    double q64[G][kHeadDim];
+    HeadScratch head[G];
+    int ent_key[kEntCap];               // team * 8 + head
+    float ent_logc[kEntCap];
+    uint32_t bitmap[kBitmapWords];
+    int wprefix[kBitmapWords];
+    int seg_rows[kSegMax];
+    int scan[33];
+    double tau[kMaxGroup];
+    int misc[8];
+};
+
+// Guard on |Y32 - Y|: tensor-core accumulation of exact bf16 products, fp32 log / Gumbel.
+__device__ __forceinline__ float score_guard(double scale, double q_l1, float k_abs_max)
+{
+    return (float)(2.5e-4 * scale * q_l1 * (double)k_abs_max + 1e-3);
+}
+
+// Sorted insert into a descending list of kTopR values.
+__device__ __forceinline__ void top_insert(float (&top)[kTopR], float v)
+{
+    if (v > top[kTopR - 1]) {
+        top[kTopR - 1] = v;
+#pragma unroll
+        for (int i = kTopR - 1; i > 0; --i) {
+            if (top[i] > top[i - 1]) { const float t = top[i]; top[i] = top[i - 1]; top[i - 1] = t; }
+        }
+    }
+}
+
+// Warp: lower bound on the `need`-th largest of y[0..M): every lane keeps its kTopR largest,
+// then `need` rounds of "pop the largest head" over the lanes. -inf when M is too small.
+__device__ inline float warp_lower_bound(const float *y, int M, int need, int lane)
+{
+    float top[kTopR];
+#pragma unroll
+    for (int i = 0; i < kTopR; ++i) top[i] = -CUDART_INF_F;
+    for (int g = lane; g < M; g += 32) top_insert(top, __ldg(y + g));
+    float popped = -CUDART_INF_F;
+    for (int it = 0; it < need; ++it) {
+        float best = top[0];
+        int who = lane;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float ob = __shfl_xor_sync(0xFFFFFFFFu, best, o);
+            const int ow = __shfl_xor_sync(0xFFFFFFFFu, who, o);
+            if (ob > best || (ob == best && ow < who)) { best = ob; who = ow; }
+        }
+        popped = best;
+        if (lane == who) {
+#pragma unroll
+            for (int i = 0; i < kTopR - 1; ++i) top[i] = top[i + 1];
+            top[kTopR - 1] = -CUDART_INF_F;
+        }
+    }
+    return popped;
+}
+
+// Warp: append the teams of [lo, hi) with y >= t_lo to the head's candidate list, in team order.
+__device__ inline void warp_append_candidates(const float *y, int lo, int hi, float t_lo, HeadScratch &hs, int lane)
+{
+    int base = 0;
+    for (int g0 = lo; g0 < hi; g0 += 32) {
+        const int g = g0 + lane;
+        const bool take = g < hi && __ldg(y + g) >= t_lo;
+        const uint32_t bal = __ballot_sync(0xFFFFFFFFu, take);
+        if (take) {
+            const int slot = base + __popc(bal & ((1u << lane) - 1u));
+            if (slot < kCandCap) hs.cand_id[slot] = g;
+        }
+        base += __popc(bal);
+    }
+    if (lane == 0) hs.n_cand = base < kCandCap ? base : kCandCap;
+}
+
+// Block: plan of `pair` into shared-memory tables (seg_prefix[nseg+1], seg_row, seg_mask) and the
+// pair's log c table in global memory (g_logc [kSegMax][8]). All threads call; blockDim.x ==
+// kPlanThreads. Returns the number of segments in nseg_out and of rows in rows_out.
+template <int G>
+__device__ void build_pair_plan(const PlanInputs &in, int pair, PlanScratch<G> &sc, int *seg_prefix, int *seg_row,
+                                uint32_t *seg_mask, float *g_logc, int &nseg_out, int &rows_out, bool write_debug)
+{
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int b = pair / in.bv.n_kv, j = pair - b * in.bv.n_kv;
+    const int64_t team0 = in.bv.seq_team_off[b];
+    const int M = (int)(in.bv.seq_team_off[b + 1] - team0);
+    const int64_t row0 = in.bv.seq_row_off[b];
+    const int N = (int)(in.bv.seq_row_off[b + 1] - row0);
+    const int K = in.n_sample;
+    const int Ke = min(K, M);
+    int t_suffix = 0;
+    if (in.suffix_len != nullptr && in.suffix_cap > 0) t_suffix = max(0, min(in.suffix_len[b], in.suffix_cap));
+    const uint32_t all_heads = (1u << G) - 1u;
+    const float kLog2e = 1.4426950408889634f;
+    const size_t head0 = (size_t)b * in.bv.n_q + (size_t)j * G;       // first query head of the pair
+
+    __syncthreads();                                                  // scratch and tables are free
+    if (Ke == M) {
+        // every team is read with correction one; nothing is drawn
+        if (tid == 0) {
+            seg_prefix[0] = 0;
+            seg_row[0] = (int32_t)row0;
+            seg_mask[0] = all_heads;
+            int nseg = 1, rows = N;
+            if (t_suffix > 0) {
+                seg_prefix[1] = rows;
+                seg_row[1] = pair * in.suffix_cap;
+                seg_mask[1] = all_heads | kSrcSuffix;
+                rows += t_suffix;
+                nseg = 2;
+            }
+            seg_prefix[nseg] = rows;
+            sc.misc[0] = nseg;
+            sc.misc[1] = rows;
+            if (write_debug && in.dbg_union_rows) in.dbg_union_rows[pair] = N;
+        }
+        if (tid < 2 * kMaxGroup) g_logc[tid] = 0.f;
+        if (write_debug) {
+            for (int e = tid; e < G * K; e += kPlanThreads) {
+                const int h = e / K, a = e - h * K;
+                if (in.dbg_sel_idx) in.dbg_sel_idx[(head0 + h) * K + a] = a < M ? a : -1;
+                if (in.dbg_sel_logc) in.dbg_sel_logc[(head0 + h) * K + a] = 0.f;
+            }
+            if (tid < G && in.dbg_tau) in.dbg_tau[head0 + tid] = __longlong_as_double(0x7FF8000000000000ll);
+        }
+        __threadfence_block();
+        __syncthreads();
+        nseg_out = sc.misc[0];
+        rows_out = sc.misc[1];
+        return;
+    }
+
+    const uint32_t step = in.step + (in.step_dev ? *in.step_dev : 0u);
+    const uint16_t *rep = in.rep_keys + ((size_t)j * in.bv.teams_total + team0) * kHeadDim;
+    const int32_t *csr = in.team_row_start + (size_t)j * (in.bv.teams_total + in.bv.n_seqs) + team0 + b;
+
+    // ---- queries in fp64, guard per head, candidate thresholds ----
+    for (int e = tid; e < G * kHeadDim; e += kPlanThreads)
+        sc.q64[e >> 7][e & 127] = bf16_to_double(in.q[(head0 + (e >> 7)) * kHeadDim + (e & 127)]);
+    __syncthreads();
+    if (warp < G) {
+        const int h = warp;
+        HeadScratch &hs = sc.head[h];
+        double l1 = 0.0;
+        for (int d = lane; d < kHeadDim; d += 32) l1 += fabs(sc.q64[h][d]);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) l1 += __shfl_xor_sync(0xFFFFFFFFu, l1, o);
+        const float guard = score_guard(in.scale, l1, in.rep_abs_max[(size_t)j * in.bv.n_seqs + b]);
+        const float *y = in.y32 + ((size_t)j * G + h) * in.bv.teams_total + team0;
+        const float t_lb = warp_lower_bound(y, M, Ke + 1, lane);
+        const float t_lo = t_lb - 2.f * guard;
+        // how many candidates: one pass if they fit, else ranges of kCandCap teams
+        int cnt = 0;
+        for (int g = lane; g < M; g += 32) cnt += __ldg(y + g) >= t_lo;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xFFFFFFFFu, cnt, o);
+        if (lane == 0) {
+            hs.t_lo = t_lo;
+            hs.n_list = 0;
+            hs.range_len = cnt <= kCandCap ? M : kCandCap;
+            hs.n_ranges = cnt <= kCandCap ? 1 : (M + kCandCap - 1) / kCandCap;
+        }
+    }
+    __syncthreads();
+    int n_iter = 1;
+#pragma unroll
+    for (int h = 0; h < G; ++h) n_iter = max(n_iter, sc.head[h].n_ranges);
+
+    int cur = 0;                                                      // which list buffer is current
+    for (int it = 0; it < n_iter; ++it) {
+        // a. candidates of this range
+        if (warp < G) {
+            HeadScratch &hs = sc.head[warp];
+            if (it < hs.n_ranges) {
+                const float *y = in.y32 + ((size_t)j * G + warp) * in.bv.teams_total + team0;
+                const int lo = it * hs.range_len, hi = min(M, lo + hs.range_len);
+                warp_append_candidates(y, lo, hi, hs.t_lo, hs, lane);
+            } else if (lane == 0) {
+                hs.n_cand = 0;
+            }
+        }
+        __syncthreads();
+        // b. exact scores of the candidates (all heads, one thread per candidate)
+        int n_tot = 0, cand_off[G + 1];
+#pragma unroll
+        for (int h = 0; h < G; ++h) { cand_off[h] = n_tot; n_tot += sc.head[h].n_cand; }
+        cand_off[G] = n_tot;
+        for (int e = tid; e < n_tot; e += kPlanThreads) {
+            int h = 0;
+#pragma unroll
+            for (int hh = 1; hh < G; ++hh) h += (e >= cand_off[hh]);
+            HeadScratch &hs = sc.head[h];
+            const int i = e - cand_off[h];
+            const int id = hs.cand_id[i];
+            const uint4 *kr = reinterpret_cast<const uint4 *>(rep + (size_t)id * kHeadDim);
+            const double *qh = sc.q64[h];
+            double dot = 0.0;
+#pragma unroll 4
+            for (int c4 = 0; c4 < 16; ++c4) {
+                const uint4 w = __ldg(kr + c4);
+                const double *qq = qh + c4 * 8;
+                dot = fma((double)bf16_lo(w.x), qq[0], dot);
+                dot = fma((double)bf16_hi(w.x), qq[1], dot);
+                dot = fma((double)bf16_lo(w.y), qq[2], dot);
+                dot = fma((double)bf16_hi(w.y), qq[3], dot);
+                dot = fma((double)bf16_lo(w.z), qq[4], dot);
+                dot = fma((double)bf16_hi(w.z), qq[5], dot);
+                dot = fma((double)bf16_lo(w.w), qq[6], dot);
+                dot = fma((double)bf16_hi(w.w), qq[7], dot);
+            }
+            const int n_g = csr[id + 1] - csr[id];
+            const double phi = log((double)n_g) + dot * in.scale;
+            const uint4 words = philox4x32_10(
+                make_uint4((uint32_t)id >> 2, step, (uint32_t)(j * G + h), in.stream_base + (uint32_t)b),
+                in.seed_lo, in.seed_hi);
+            hs.cand_phi[i] = phi;
+            hs.cand_y[i] = phi + gumbel_from_word(pick_word(words, id & 3));
+        }
+        __syncthreads();
+        // c. merge with the running list: keep the Ke + 1 largest by (Y descending, id ascending)
+        int ent_off[G + 1], e_tot = 0;
+#pragma unroll
+        for (int h = 0; h < G; ++h) { ent_off[h] = e_tot; e_tot += sc.head[h].n_list + sc.head[h].n_cand; }
+        ent_off[G] = e_tot;
+        for (int e = tid; e < e_tot; e += kPlanThreads) {
+            int h = 0;
+#pragma unroll
+            for (int hh = 1; hh < G; ++hh) h += (e >= ent_off[hh]);
+            HeadScratch &hs = sc.head[h];
+            const int i = e - ent_off[h];
+            const int nl = hs.n_list, nc = hs.n_cand;
+            double y, phi;
+            int id;
+            if (i < nl) { y = hs.list_y[cur][i]; phi = hs.list_phi[cur][i]; id = hs.list_id[cur][i]; }
+            else { y = hs.cand_y[i - nl]; phi = hs.cand_phi[i - nl]; id = hs.cand_id[i - nl]; }
+            int rank = 0;
+            for (int a = 0; a < nl; ++a) {
+                const double ya = hs.list_y[cur][a];
+                rank += (ya > y) || (ya == y && hs.list_id[cur][a] < id);
+            }
+            for (int a = 0; a < nc; ++a) {
+                const double ya = hs.cand_y[a];
+                rank += (ya > y) || (ya == y && hs.cand_id[a] < id);
+            }
+            if (rank <= Ke) {
+                hs.list_y[cur ^ 1][rank] = y;
+                hs.list_phi[cur ^ 1][rank] = phi;
+                hs.list_id[cur ^ 1][rank] = id;
+            }
+        }
+        __syncthreads();
+        if (tid < G) sc.head[tid].n_list = min(Ke + 1, sc.head[tid].n_list + sc.head[tid].n_cand);
+        cur ^= 1;
+        __syncthreads();
+    }
+
+    // ---- corrections, diagnostics, plan entries ----
+    for (int e = tid; e < G * Ke; e += kPlanThreads) {
+        const int h = e / Ke, a = e - h * Ke;
+        const HeadScratch &hs = sc.head[h];
+        const double tau = hs.list_y[cur][Ke];
+        const double c = -expm1(-exp(hs.list_phi[cur][a] - tau));     // 1 - exp(-exp(phi - tau))
+        const float logc = (float)log(c);
+        const int id = hs.list_id[cur][a];
+        sc.ent_key[e] = id * kMaxGroup + h;
+        sc.ent_logc[e] = logc;
+        if (write_debug) {
+            if (in.dbg_sel_idx) in.dbg_sel_idx[(head0 + h) * K + a] = id;
+            if (in.dbg_sel_logc) in.dbg_sel_logc[(head0 + h) * K + a] = logc;
+            if (a == 0 && in.dbg_tau) in.dbg_tau[head0 + h] = tau;
+        }
+    }
+    for (int i = tid; i < (M + 31) / 32; i += kPlanThreads) sc.bitmap[i] = 0u;
+    for (int i = tid; i < kSegMax; i += kPlanThreads) seg_mask[i] = 0u;
+    __syncthreads();
+    const int E = G * Ke;
+    for (int e = tid; e < E; e += kPlanThreads) {
+        const int team = sc.ent_key[e] >> 3;
+        atomicOr(&sc.bitmap[team >> 5], 1u << (team & 31));
+    }
+    __syncthreads();
+    // word prefix of the bitmap -> segment index of a team = teams selected before it
+    {
+        const int n_words = (M + 31) / 32;
+        const int per = (n_words + kPlanThreads - 1) / kPlanThreads;
+        const int lo = min(tid * per, n_words), hi = min(lo + per, n_words);
+        int sum = 0;
+        for (int w = lo; w < hi; ++w) sum += __popc(sc.bitmap[w]);
+        int total;
+        int run = block_exclusive_scan(sum, sc.scan, total);
+        for (int w = lo; w < hi; ++w) { sc.wprefix[w] = run; run += __popc(sc.bitmap[w]); }
+        if (tid == 0) sc.misc[0] = total;                             // segments of the prompt
+    }
+    __syncthreads();
+    const int nseg_prompt = sc.misc[0];
+    for (int e = tid; e < E; e += kPlanThreads) {
+        const int team = sc.ent_key[e] >> 3, h = sc.ent_key[e] & 7;
+        const int seg = sc.wprefix[team >> 5] + __popc(sc.bitmap[team >> 5] & ((1u << (team & 31)) - 1u));
+        atomicOr(&seg_mask[seg], 1u << h);
+        g_logc[(size_t)seg * kMaxGroup + h] = kLog2e * sc.ent_logc[e];
+        const int r_lo = csr[team];
+        seg_row[seg] = (int32_t)(row0 + r_lo);                        // same value from every selecting head
+        sc.seg_rows[seg] = csr[team + 1] - r_lo;
+    }
+    __syncthreads();
+    {
+        const int per = (nseg_prompt + kPlanThreads - 1) / kPlanThreads;
+        const int lo = min(tid * per, nseg_prompt), hi = min(lo + per, nseg_prompt);
+        int sum = 0;
+        for (int s = lo; s < hi; ++s) sum += sc.seg_rows[s];
+        int total;
+        int run = block_exclusive_scan(sum, sc.scan, total);
+        for (int s = lo; s < hi; ++s) { seg_prefix[s] = run; run += sc.seg_rows[s]; }
+        if (tid == 0) {
+            int nseg = nseg_prompt, rows = total;
+            if (write_debug && in.dbg_union_rows) in.dbg_union_rows[pair] = total;
+            if (t_suffix > 0) {
+                seg_prefix[nseg] = rows;
+                seg_row[nseg] = pair * in.suffix_cap;
+                seg_mask[nseg] = all_heads | kSrcSuffix;
+                rows += t_suffix;
+                ++nseg;
+            }
+            seg_prefix[nseg] = rows;
+            sc.misc[0] = nseg;
+            sc.misc[1] = rows;
+        }
+        if (t_suffix > 0 && tid < kMaxGroup) g_logc[(size_t)nseg_prompt * kMaxGroup + tid] = 0.f;
+    }
+    __threadfence_block();
+    __syncthreads();
+    nseg_out = sc.misc[0];
+    rows_out = sc.misc[1];
+}
+
+}  // namespace santapp
