@@ -72,8 +72,8 @@ BatchView make_view(const santapp_geom *g, const santapp_teams *t)
 
 // Workspace layout shared by the sparse and the dense call. Offsets in bytes.
 struct DecodeLayout {
-    size_t ctl, y32, seg_prefix, seg_row, seg_mask, seg_logc, pair_nseg, pair_rows, pair_prefix, partials, total;
-    int seg_cap, grid, n_pairs, ctas_per_pair;
+    size_t ctl, y32, ymax, seg_prefix, seg_row, seg_mask, seg_logc, pair_nseg, pair_rows, pair_prefix, partials, total;
+    int seg_cap, grid, n_pairs, ctas_per_pair, ymax_stride;
     bool static_split;
 };
 
@@ -94,6 +94,8 @@ DecodeLayout decode_layout(const santapp_geom *g, const santapp_teams *t, int K,
     auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
     L.ctl = take(sizeof(int32_t) * ((size_t)L.n_pairs + 2));
     L.y32 = take(dense ? 0 : sizeof(float) * (size_t)g->n_q_heads * (size_t)t->teams_total);
+    L.ymax_stride = (int)(t->teams_total / 16 + g->n_seqs + 1);
+    L.ymax = take(dense ? 0 : sizeof(float) * (size_t)g->n_q_heads * (size_t)L.ymax_stride);
     L.seg_prefix = take(sizeof(int32_t) * (size_t)L.n_pairs * (L.seg_cap + 1));
     L.seg_row = take(sizeof(int32_t) * (size_t)L.n_pairs * L.seg_cap);
     L.seg_mask = take(sizeof(uint32_t) * (size_t)L.n_pairs * L.seg_cap);
@@ -273,6 +275,8 @@ int santapp_decode_attn(const santapp_geom *geom, const santapp_teams *teams, co
     rp.team_row_start = teams->team_row_start;
     rp.q = static_cast<const uint16_t *>(q);
     rp.y32 = reinterpret_cast<float *>(ws + L.y32);
+    rp.ymax = reinterpret_cast<float *>(ws + L.ymax);
+    rp.ymax_stride = L.ymax_stride;
     rp.n_sample = n_sample;
     rp.seed_lo = (uint32_t)(seed & 0xFFFFFFFFull);
     rp.seed_hi = (uint32_t)(seed >> 32);
@@ -293,6 +297,8 @@ int santapp_decode_attn(const santapp_geom *geom, const santapp_teams *teams, co
     PlanParams pp;
     pp.in.bv = rp.bv;
     pp.in.y32 = rp.y32;
+    pp.in.ymax = rp.ymax;
+    pp.in.ymax_stride = L.ymax_stride;
     pp.in.rep_keys = rp.rep_keys;
     pp.in.team_row_start = teams->team_row_start;
     pp.in.rep_abs_max = teams->rep_abs_max;

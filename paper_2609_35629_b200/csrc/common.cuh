@@ -53,6 +53,9 @@ struct ScoreParams {
     const int32_t *team_row_start;  // [n_kv][teams_total + n_seqs]
     const uint16_t *q;              // [n_seqs][n_q][128]
     float *y32;                     // [n_q][teams_total] fp32 perturbed routing scores
+    float *ymax;                    // [n_q][ymax_stride] largest score of each 16-team block: sequence b's
+                                    //   blocks start at seq_team_off[b] / 16 + b
+    int ymax_stride;
     int n_sample;
     uint32_t seed_lo, seed_hi, step, stream_base;
     const uint32_t *step_dev;       // nullable: added to step
@@ -66,6 +69,8 @@ struct ScoreParams {
 struct PlanInputs {
     BatchView bv;
     const float *y32;               // [n_q][teams_total]
+    const float *ymax;              // [n_q][ymax_stride], see ScoreParams
+    int ymax_stride;
     const uint16_t *rep_keys;       // [n_kv][teams_total][128]
     const int32_t *team_row_start;  // [n_kv][teams_total + n_seqs]
     const float *rep_abs_max;       // [n_kv][n_seqs]

@@ -4,7 +4,7 @@
 //
 // The scorer leaves fp32 perturbed scores Y32 for every (head, team) together with a bound E on
 // |Y32 - Y| against the exact fp64 score Y. The sample must be the fp64 one, so per head:
-//   1. a lower bound t on the (K+1)-st largest Y32 (tournament over per-lane maxima);
+//   1. a lower bound t on the (K+1)-st largest Y32 (from the maxima of 16-team blocks);
 //   2. every team with Y32 >= t - 2E is a candidate: that set contains the K+1 largest exact
 //      scores (if K+1 teams have Y32 >= t they have Y >= t - E, so the (K+1)-st largest Y is at
 //      least t - E, and a team with Y above that has Y32 >= t - 2E);
@@ -27,7 +27,7 @@ constexpr int kPlanThreads = 384;       // block size of every kernel that build
 constexpr int kPlanWarps = kPlanThreads / 32;
 constexpr int kCandCap = 512;           // candidates of one head refined at a time
 constexpr int kListCap = 132;           // running top list: K + 1 <= 129 entries
-constexpr int kTopR = 7;                // per-lane maxima kept for the lower bound
+constexpr int kTopR = 8;                // per-lane maxima kept for the lower bound (4 used for K + 1 <= 96)
 constexpr int kEntCap = 1024;           // G * K entries of a plan
 constexpr int kSegMax = 1025;           // segments of a plan (entries + suffix)
 constexpr int kBitmapWords = kMaxTeamsPerSeq / 32;
@@ -36,6 +36,7 @@ struct HeadScratch {
     int n_cand, n_list, n_ranges, range_len;
     float t_lo;                         // candidate threshold on Y32 (lower bound minus guard)
     float pad[3];
+    float bound_vals[32 * kTopR];       // per-lane largest block maxima, for the lower bound
     int cand_id[kCandCap];
     double cand_y[kCandCap];
     double cand_phi[kCandCap];
@@ -76,56 +77,87 @@ __device__ __forceinline__ void top_insert(float (&top)[kTopR], float v)
     }
 }
 
-// Warp: lower bound on the `need`-th largest of y[0..M): every lane keeps its kTopR largest,
-// then `need` rounds of "pop the largest head" over the lanes. -inf when M is too small.
-__device__ inline float warp_lower_bound(const float *y, int M, int need, int lane)
+// Warp: lower bound on the `need`-th largest score of a head from the maxima of its 16-team
+// blocks. Every lane keeps the R largest block maxima it sees (R = 4, or 8 for large `need`);
+// the kept values go to shared memory and every lane counts, for each of its own values, how
+// many kept values are larger. A value with at least need - 1 larger ones is, with them, `need`
+// distinct teams' scores, hence at most the `need`-th largest score; the largest such value is
+// returned (-inf when there are too few values).
+__device__ __forceinline__ float warp_lower_bound(const float *ym, int nblk, int need, int lane, float *vals)
 {
+    const int R = need <= 96 ? 4 : kTopR;
     float top[kTopR];
 #pragma unroll
     for (int i = 0; i < kTopR; ++i) top[i] = -CUDART_INF_F;
-    for (int g = lane; g < M; g += 32) top_insert(top, __ldg(y + g));
-    float popped = -CUDART_INF_F;
-    for (int it = 0; it < need; ++it) {
-        float best = top[0];
-        int who = lane;
+    for (int i0 = lane; i0 < nblk; i0 += 128) {
+        float v[4];
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            const float ob = __shfl_xor_sync(0xFFFFFFFFu, best, o);
-            const int ow = __shfl_xor_sync(0xFFFFFFFFu, who, o);
-            if (ob > best || (ob == best && ow < who)) { best = ob; who = ow; }
-        }
-        popped = best;
-        if (lane == who) {
+        for (int k = 0; k < 4; ++k) v[k] = (i0 + 32 * k < nblk) ? __ldg(ym + i0 + 32 * k) : -CUDART_INF_F;
 #pragma unroll
-            for (int i = 0; i < kTopR - 1; ++i) top[i] = top[i + 1];
-            top[kTopR - 1] = -CUDART_INF_F;
+        for (int k = 0; k < 4; ++k) top_insert(top, v[k]);
+    }
+#pragma unroll
+    for (int i = 0; i < kTopR; ++i)
+        if (i < R) vals[lane * R + i] = top[i];
+    __syncwarp();
+    int larger[kTopR];
+#pragma unroll
+    for (int i = 0; i < kTopR; ++i) larger[i] = 0;
+    for (int a4 = 0; a4 < 8 * R; ++a4) {
+        const float4 w = *reinterpret_cast<const float4 *>(vals + 4 * a4);     // same address in every lane
+#pragma unroll
+        for (int i = 0; i < kTopR; ++i) {
+            if (i < R) larger[i] += (w.x > top[i]) + (w.y > top[i]) + (w.z > top[i]) + (w.w > top[i]);
         }
     }
-    return popped;
+    float best = -CUDART_INF_F;
+#pragma unroll
+    for (int i = 0; i < kTopR; ++i)
+        if (i < R && larger[i] >= need - 1) best = fmaxf(best, top[i]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) best = fmaxf(best, __shfl_xor_sync(0xFFFFFFFFu, best, o));
+    __syncwarp();
+    return best;
 }
 
-// Warp: append the teams of [lo, hi) with y >= t_lo to the head's candidate list, in team order.
-__device__ inline void warp_append_candidates(const float *y, int lo, int hi, float t_lo, HeadScratch &hs, int lane)
+// Warp: append the teams of blocks [blk_lo, blk_hi) with y >= t_lo to the head's candidate list
+// (any order; the exact ranking does not depend on it). hs.n_cand counts every hit, also those
+// beyond kCandCap, so the caller can tell an overflow.
+__device__ __forceinline__ void warp_append_blocks(const float *y, const float *ym, int blk_lo, int blk_hi, int M, float t_lo,
+                                          HeadScratch &hs, int lane)
 {
-    int base = 0;
-    for (int g0 = lo; g0 < hi; g0 += 32) {
-        const int g = g0 + lane;
-        const bool take = g < hi && __ldg(y + g) >= t_lo;
-        const uint32_t bal = __ballot_sync(0xFFFFFFFFu, take);
-        if (take) {
-            const int slot = base + __popc(bal & ((1u << lane) - 1u));
-            if (slot < kCandCap) hs.cand_id[slot] = g;
+    // four blocks per lane at a time: block maxima first, then the scores of the blocks that can
+    // hold a candidate, all loads of a batch in flight together
+    for (int blk0 = blk_lo + lane; blk0 < blk_hi; blk0 += 128) {
+        bool hit[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) hit[k] = (blk0 + 32 * k < blk_hi) && (__ldg(ym + blk0 + 32 * k) >= t_lo);
+        float v[4][16];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const int g0 = (blk0 + 32 * k) * 16;
+#pragma unroll
+            for (int i = 0; i < 16; ++i) v[k][i] = (hit[k] && g0 + i < M) ? __ldg(y + g0 + i) : -CUDART_INF_F;
         }
-        base += __popc(bal);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const int g0 = (blk0 + 32 * k) * 16;
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                if (hit[k] && g0 + i < M && v[k][i] >= t_lo) {
+                    const int slot = atomicAdd(&hs.n_cand, 1);
+                    if (slot < kCandCap) hs.cand_id[slot] = g0 + i;
+                }
+            }
+        }
     }
-    if (lane == 0) hs.n_cand = base < kCandCap ? base : kCandCap;
 }
 
 // Block: plan of `pair` into shared-memory tables (seg_prefix[nseg+1], seg_row, seg_mask) and the
 // pair's log c table in global memory (g_logc [kSegMax][8]). All threads call; blockDim.x ==
 // kPlanThreads. Returns the number of segments in nseg_out and of rows in rows_out.
 template <int G>
-__device__ void build_pair_plan(const PlanInputs &in, int pair, PlanScratch<G> &sc, int *seg_prefix, int *seg_row,
+__device__ __forceinline__ void build_pair_plan(const PlanInputs &in, int pair, PlanScratch<G> &sc, int *seg_prefix, int *seg_row,
                                 uint32_t *seg_mask, float *g_logc, int &nseg_out, int &rows_out, bool write_debug)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -195,18 +227,21 @@ __device__ void build_pair_plan(const PlanInputs &in, int pair, PlanScratch<G> &
         for (int o = 16; o > 0; o >>= 1) l1 += __shfl_xor_sync(0xFFFFFFFFu, l1, o);
         const float guard = score_guard(in.scale, l1, in.rep_abs_max[(size_t)j * in.bv.n_seqs + b]);
         const float *y = in.y32 + ((size_t)j * G + h) * in.bv.teams_total + team0;
-        const float t_lb = warp_lower_bound(y, M, Ke + 1, lane);
+        const float *ym = in.ymax + ((size_t)j * G + h) * in.ymax_stride + (team0 >> 4) + b;
+        const int nblk = (M + 15) >> 4;
+        const float t_lb = warp_lower_bound(ym, nblk, Ke + 1, lane, hs.bound_vals);
         const float t_lo = t_lb - 2.f * guard;
-        // how many candidates: one pass if they fit, else ranges of kCandCap teams
-        int cnt = 0;
-        for (int g = lane; g < M; g += 32) cnt += __ldg(y + g) >= t_lo;
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xFFFFFFFFu, cnt, o);
+        // candidates in one go if they fit, else ranges of kCandCap teams in the loop below
+        if (lane == 0) hs.n_cand = 0;
+        __syncwarp();
+        warp_append_blocks(y, ym, 0, nblk, M, t_lo, hs, lane);
+        __syncwarp();
         if (lane == 0) {
+            const bool fits = hs.n_cand <= kCandCap;
             hs.t_lo = t_lo;
             hs.n_list = 0;
-            hs.range_len = cnt <= kCandCap ? M : kCandCap;
-            hs.n_ranges = cnt <= kCandCap ? 1 : (M + kCandCap - 1) / kCandCap;
+            hs.range_len = fits ? M : kCandCap;
+            hs.n_ranges = fits ? 1 : (M + kCandCap - 1) / kCandCap;
         }
     }
     __syncthreads();
@@ -219,12 +254,15 @@ __device__ void build_pair_plan(const PlanInputs &in, int pair, PlanScratch<G> &
         // a. candidates of this range
         if (warp < G) {
             HeadScratch &hs = sc.head[warp];
-            if (it < hs.n_ranges) {
+            if (hs.n_ranges > 1 && it < hs.n_ranges) {
                 const float *y = in.y32 + ((size_t)j * G + warp) * in.bv.teams_total + team0;
-                const int lo = it * hs.range_len, hi = min(M, lo + hs.range_len);
-                warp_append_candidates(y, lo, hi, hs.t_lo, hs, lane);
-            } else if (lane == 0) {
-                hs.n_cand = 0;
+                const float *ym = in.ymax + ((size_t)j * G + warp) * in.ymax_stride + (team0 >> 4) + b;
+                const int blk_lo = it * (kCandCap / 16), blk_hi = min((M + 15) >> 4, blk_lo + kCandCap / 16);
+                if (lane == 0) hs.n_cand = 0;
+                __syncwarp();
+                warp_append_blocks(y, ym, blk_lo, blk_hi, M, hs.t_lo, hs, lane);
+            } else if (it > 0 && lane == 0) {
+                hs.n_cand = 0;                                     // single range: done in iteration 0
             }
         }
         __syncthreads();
@@ -234,29 +272,38 @@ __device__ void build_pair_plan(const PlanInputs &in, int pair, PlanScratch<G> &
         for (int h = 0; h < G; ++h) { cand_off[h] = n_tot; n_tot += sc.head[h].n_cand; }
         cand_off[G] = n_tot;
         for (int e = tid; e < n_tot; e += kPlanThreads) {
-            int h = 0;
+            int h = 0, off = 0;
 #pragma unroll
-            for (int hh = 1; hh < G; ++hh) h += (e >= cand_off[hh]);
+            for (int hh = 1; hh < G; ++hh) {
+                const bool ge = e >= cand_off[hh];
+                h += ge;
+                off = ge ? cand_off[hh] : off;
+            }
             HeadScratch &hs = sc.head[h];
-            const int i = e - cand_off[h];
+            const int i = e - off;
             const int id = hs.cand_id[i];
             const uint4 *kr = reinterpret_cast<const uint4 *>(rep + (size_t)id * kHeadDim);
             const double *qh = sc.q64[h];
-            double dot = 0.0;
-#pragma unroll 4
+            const int r_lo = csr[id], r_hi = csr[id + 1];
+            uint4 kw[16];
+#pragma unroll
+            for (int c4 = 0; c4 < 16; ++c4) kw[c4] = __ldg(kr + c4);
+            double d0 = 0.0, d1 = 0.0, d2 = 0.0, d3 = 0.0;            // four chains, summed at the end
+#pragma unroll
             for (int c4 = 0; c4 < 16; ++c4) {
-                const uint4 w = __ldg(kr + c4);
+                const uint4 w = kw[c4];
                 const double *qq = qh + c4 * 8;
-                dot = fma((double)bf16_lo(w.x), qq[0], dot);
-                dot = fma((double)bf16_hi(w.x), qq[1], dot);
-                dot = fma((double)bf16_lo(w.y), qq[2], dot);
-                dot = fma((double)bf16_hi(w.y), qq[3], dot);
-                dot = fma((double)bf16_lo(w.z), qq[4], dot);
-                dot = fma((double)bf16_hi(w.z), qq[5], dot);
-                dot = fma((double)bf16_lo(w.w), qq[6], dot);
-                dot = fma((double)bf16_hi(w.w), qq[7], dot);
+                d0 = fma((double)bf16_lo(w.x), qq[0], d0);
+                d1 = fma((double)bf16_hi(w.x), qq[1], d1);
+                d2 = fma((double)bf16_lo(w.y), qq[2], d2);
+                d3 = fma((double)bf16_hi(w.y), qq[3], d3);
+                d0 = fma((double)bf16_lo(w.z), qq[4], d0);
+                d1 = fma((double)bf16_hi(w.z), qq[5], d1);
+                d2 = fma((double)bf16_lo(w.w), qq[6], d2);
+                d3 = fma((double)bf16_hi(w.w), qq[7], d3);
             }
-            const int n_g = csr[id + 1] - csr[id];
+            const double dot = (d0 + d1) + (d2 + d3);
+            const int n_g = r_hi - r_lo;
             const double phi = log((double)n_g) + dot * in.scale;
             const uint4 words = philox4x32_10(
                 make_uint4((uint32_t)id >> 2, step, (uint32_t)(j * G + h), in.stream_base + (uint32_t)b),
@@ -271,21 +318,27 @@ __device__ void build_pair_plan(const PlanInputs &in, int pair, PlanScratch<G> &
         for (int h = 0; h < G; ++h) { ent_off[h] = e_tot; e_tot += sc.head[h].n_list + sc.head[h].n_cand; }
         ent_off[G] = e_tot;
         for (int e = tid; e < e_tot; e += kPlanThreads) {
-            int h = 0;
+            int h = 0, off = 0;
 #pragma unroll
-            for (int hh = 1; hh < G; ++hh) h += (e >= ent_off[hh]);
+            for (int hh = 1; hh < G; ++hh) {
+                const bool ge = e >= ent_off[hh];
+                h += ge;
+                off = ge ? ent_off[hh] : off;
+            }
             HeadScratch &hs = sc.head[h];
-            const int i = e - ent_off[h];
+            const int i = e - off;
             const int nl = hs.n_list, nc = hs.n_cand;
             double y, phi;
             int id;
             if (i < nl) { y = hs.list_y[cur][i]; phi = hs.list_phi[cur][i]; id = hs.list_id[cur][i]; }
             else { y = hs.cand_y[i - nl]; phi = hs.cand_phi[i - nl]; id = hs.cand_id[i - nl]; }
             int rank = 0;
+#pragma unroll 4
             for (int a = 0; a < nl; ++a) {
                 const double ya = hs.list_y[cur][a];
                 rank += (ya > y) || (ya == y && hs.list_id[cur][a] < id);
             }
+#pragma unroll 4
             for (int a = 0; a < nc; ++a) {
                 const double ya = hs.cand_y[a];
                 rank += (ya > y) || (ya == y && hs.cand_id[a] < id);

@@ -104,8 +104,9 @@ score32_kernel(ScoreParams p)
         }
     }
     // acc[t][0], acc[t][1]: head g, teams base + 8 t + 2c, + 1
+    float blk_max = -INFINITY;
+    const uint32_t head = (uint32_t)(j * G + (g < G ? g : 0));
     if (g < G) {
-        const uint32_t head = (uint32_t)(j * G + g);
         float *y = p.y32 + (size_t)head * p.bv.teams_total + team0;
 #pragma unroll
         for (int t = 0; t < 2; ++t) {
@@ -114,15 +115,25 @@ score32_kernel(ScoreParams p)
                 const uint4 words = philox4x32_10(
                     make_uint4((uint32_t)t0 >> 2, step, head, p.stream_base + (uint32_t)b), p.seed_lo, p.seed_hi);
                 const int r0 = csr[t0], r1 = csr[t0 + 1];
-                y[t0] = logf((float)(r1 - r0)) + acc[t][0] * scale + gumbel32_from_word(pick_word(words, t0 & 3));
+                const float y0 = logf((float)(r1 - r0)) + acc[t][0] * scale
+                                 + gumbel32_from_word(pick_word(words, t0 & 3));
+                y[t0] = y0;
+                blk_max = fmaxf(blk_max, y0);
                 if (t0 + 1 < M) {
                     const int r2 = csr[t0 + 2];
-                    y[t0 + 1] = logf((float)(r2 - r1)) + acc[t][1] * scale
-                                + gumbel32_from_word(pick_word(words, (t0 & 3) + 1));
+                    const float y1 = logf((float)(r2 - r1)) + acc[t][1] * scale
+                                     + gumbel32_from_word(pick_word(words, (t0 & 3) + 1));
+                    y[t0 + 1] = y1;
+                    blk_max = fmaxf(blk_max, y1);
                 }
             }
         }
     }
+    // largest score of the warp's 16-team block, per head (the quad of a head holds its 16 scores)
+    blk_max = fmaxf(blk_max, __shfl_xor_sync(0xFFFFFFFFu, blk_max, 1));
+    blk_max = fmaxf(blk_max, __shfl_xor_sync(0xFFFFFFFFu, blk_max, 2));
+    if (g < G && c == 0)
+        p.ymax[(size_t)head * p.ymax_stride + (size_t)(team0 >> 4) + b + (base >> 4)] = blk_max;
 }
 
 // One block per (sequence, KV head): largest |element| among the pair's representative keys.
