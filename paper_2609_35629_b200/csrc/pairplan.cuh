@@ -27,18 +27,17 @@ constexpr int kPlanThreads = 384;       // block size of every kernel that build
 constexpr int kPlanWarps = kPlanThreads / 32;
 constexpr int kCandCap = 512;           // candidates of one head refined at a time
 constexpr int kListCap = 132;           // running top list: K + 1 <= 129 entries
-constexpr int kTopR = 8;                // per-lane maxima kept for the lower bound (4 used for K + 1 <= 96)
 constexpr int kEntCap = 1024;           // G * K entries of a plan
 constexpr int kSegMax = 1025;           // segments of a plan (entries + suffix)
 constexpr int kBitmapWords = kMaxTeamsPerSeq / 32;
 
-struct HeadScratch {
+struct alignas(16) HeadScratch {
     int n_cand, n_list, n_ranges, range_len;
     float t_lo;                         // candidate threshold on Y32 (lower bound minus guard)
     float pad[3];
-    float bound_vals[32 * kTopR];       // per-lane largest block maxima, for the lower bound
+    int hist[256];                      // block maxima by distance from the largest, for the lower bound
     int cand_id[kCandCap];
-    double cand_y[kCandCap];
+    double cand_y[kCandCap + 2];          // read in pairs: an odd count is padded with -inf
     double cand_phi[kCandCap];
     int list_id[2][kListCap];
     double list_y[2][kListCap];
@@ -46,7 +45,7 @@ struct HeadScratch {
 };
 
 template <int G>
-struct PlanScratch {
+struct alignas(16) PlanScratch {
     double q64[G][kHeadDim];
     HeadScratch head[G];
     int ent_key[kEntCap];               // team * 8 + head
@@ -65,59 +64,71 @@ __device__ __forceinline__ float score_guard(double scale, double q_l1, float k_
     return (float)(2.5e-4 * scale * q_l1 * (double)k_abs_max + 1e-3);
 }
 
-// Sorted insert into a descending list of kTopR values.
-__device__ __forceinline__ void top_insert(float (&top)[kTopR], float v)
-{
-    if (v > top[kTopR - 1]) {
-        top[kTopR - 1] = v;
-#pragma unroll
-        for (int i = kTopR - 1; i > 0; --i) {
-            if (top[i] > top[i - 1]) { const float t = top[i]; top[i] = top[i - 1]; top[i - 1] = t; }
-        }
-    }
-}
-
 // Warp: lower bound on the `need`-th largest score of a head from the maxima of its 16-team
-// blocks. Every lane keeps the R largest block maxima it sees (R = 4, or 8 for large `need`);
-// the kept values go to shared memory and every lane counts, for each of its own values, how
-// many kept values are larger. A value with at least need - 1 larger ones is, with them, `need`
-// distinct teams' scores, hence at most the `need`-th largest score; the largest such value is
-// returned (-inf when there are too few values).
-__device__ __forceinline__ float warp_lower_bound(const float *ym, int nblk, int need, int lane, float *vals)
+// blocks, by histograms: a block maximum v falls in global bin floor((top - v) * 4) counted down
+// from the largest maximum `top`; one pass counts a window of 255 consecutive bins. The first
+// bin at which the running count of block maxima reaches `need` has `need` distinct teams'
+// scores above its lower edge, so that edge is at most the `need`-th largest score. Windows
+// further down are visited only when an outlier at the top leaves the first one short.
+// -inf when there are fewer than `need` blocks.
+__device__ __forceinline__ float warp_lower_bound(const float *ym, int nblk, int need, int lane, int *hist)
 {
-    const int R = need <= 96 ? 4 : kTopR;
-    float top[kTopR];
-#pragma unroll
-    for (int i = 0; i < kTopR; ++i) top[i] = -CUDART_INF_F;
+    constexpr float kInvWidth = 4.f;
+    constexpr int kWindow = 255;
+    if (nblk < need) return -CUDART_INF_F;
+    float top = -CUDART_INF_F;
     for (int i0 = lane; i0 < nblk; i0 += 128) {
         float v[4];
 #pragma unroll
         for (int k = 0; k < 4; ++k) v[k] = (i0 + 32 * k < nblk) ? __ldg(ym + i0 + 32 * k) : -CUDART_INF_F;
-#pragma unroll
-        for (int k = 0; k < 4; ++k) top_insert(top, v[k]);
+        top = fmaxf(top, fmaxf(fmaxf(v[0], v[1]), fmaxf(v[2], v[3])));
     }
 #pragma unroll
-    for (int i = 0; i < kTopR; ++i)
-        if (i < R) vals[lane * R + i] = top[i];
-    __syncwarp();
-    int larger[kTopR];
+    for (int o = 16; o > 0; o >>= 1) top = fmaxf(top, __shfl_xor_sync(0xFFFFFFFFu, top, o));
+    int above = 0;                                             // maxima in the windows already passed
+    for (int win = 0; win < 16 * kWindow; win += kWindow) {   // 1020 units below the top, then give up
 #pragma unroll
-    for (int i = 0; i < kTopR; ++i) larger[i] = 0;
-    for (int a4 = 0; a4 < 8 * R; ++a4) {
-        const float4 w = *reinterpret_cast<const float4 *>(vals + 4 * a4);     // same address in every lane
+        for (int i = 0; i < 8; ++i) hist[lane * 8 + i] = 0;
+        __syncwarp();
+        for (int i0 = lane; i0 < nblk; i0 += 128) {
 #pragma unroll
-        for (int i = 0; i < kTopR; ++i) {
-            if (i < R) larger[i] += (w.x > top[i]) + (w.y > top[i]) + (w.z > top[i]) + (w.w > top[i]);
+            for (int k = 0; k < 4; ++k) {
+                if (i0 + 32 * k < nblk) {
+                    const float d = (top - __ldg(ym + i0 + 32 * k)) * kInvWidth;   // cached by the first pass
+                    const int gb = d >= 1073741824.f ? (1 << 30) : (int)d;         // global bin, the same in every pass
+                    if (gb >= win) atomicAdd(&hist[min(gb - win, kWindow)], 1);
+                }
+            }
         }
+        __syncwarp();
+        // lane l owns bins 8 l .. 8 l + 7 of the window; bin 255 holds everything below it
+        int local[8], sum = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { local[i] = hist[lane * 8 + i]; sum += local[i]; }
+        int incl = sum;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+            if (lane >= o) incl += t;
+        }
+        int bin = 256;                                         // first bin whose running count reaches need
+        int acc = above + incl - sum;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            acc += local[i];
+            if (acc >= need && bin == 256) bin = lane * 8 + i;
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) bin = min(bin, __shfl_xor_sync(0xFFFFFFFFu, bin, o));
+        const int below = __shfl_sync(0xFFFFFFFFu, local[7], 31);
+        const int total = __shfl_sync(0xFFFFFFFFu, incl, 31);
+        __syncwarp();
+        if (bin < kWindow)                                     // lower edge, minus the rounding of the binning
+            return top - (float)(win + bin + 1) * (1.f / kInvWidth) * (1.f + 1e-6f) - 1e-4f;
+        if (below == 0) break;
+        above += total - below;
     }
-    float best = -CUDART_INF_F;
-#pragma unroll
-    for (int i = 0; i < kTopR; ++i)
-        if (i < R && larger[i] >= need - 1) best = fmaxf(best, top[i]);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) best = fmaxf(best, __shfl_xor_sync(0xFFFFFFFFu, best, o));
-    __syncwarp();
-    return best;
+    return -CUDART_INF_F;
 }
 
 // Warp: append the teams of blocks [blk_lo, blk_hi) with y >= t_lo to the head's candidate list
@@ -151,6 +162,60 @@ __device__ __forceinline__ void warp_append_blocks(const float *y, const float *
             }
         }
     }
+}
+
+// Warp: candidates of a whole head in two steps: the blocks whose maximum reaches t_lo are
+// listed first (ballot compaction over the block maxima, which the bound left in cache), then
+// the scores of the listed blocks are fetched as independent 16-byte loads, several per lane in
+// flight. Returns false when more than kCandCap blocks qualify (the caller then walks ranges).
+__device__ __forceinline__ bool warp_append_listed(const float *y, const float *ym, int nblk, int M, float t_lo,
+                                                   HeadScratch &hs, int lane)
+{
+    int *blk_list = reinterpret_cast<int *>(hs.cand_y);        // free until the exact scores are written
+    int n_blk = 0;
+    for (int i0 = 0; i0 < nblk; i0 += 32) {
+        const int blk = i0 + lane;
+        const bool hit = blk < nblk && __ldg(ym + blk) >= t_lo;
+        const unsigned m = __ballot_sync(0xFFFFFFFFu, hit);
+        if (hit) {
+            const int slot = n_blk + __popc(m & ((1u << lane) - 1u));
+            if (slot < kCandCap) blk_list[slot] = blk;
+        }
+        n_blk += __popc(m);
+    }
+    if (n_blk > kCandCap) return false;
+    __syncwarp();
+    const int n_item = n_blk * 4;                              // (listed block, quarter of its 16 scores)
+    for (int it0 = lane; it0 < n_item; it0 += 128) {
+        float4 v[4];
+        int g0[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const int it = it0 + 32 * k;
+            g0[k] = -1;
+            if (it < n_item) {
+                g0[k] = blk_list[it >> 2] * 16 + (it & 3) * 4;
+                // rows of Y32 start at multiples of 4 teams only when team0 does; load scalars otherwise
+                v[k].x = g0[k] < M ? __ldg(y + g0[k]) : -CUDART_INF_F;
+                v[k].y = g0[k] + 1 < M ? __ldg(y + g0[k] + 1) : -CUDART_INF_F;
+                v[k].z = g0[k] + 2 < M ? __ldg(y + g0[k] + 2) : -CUDART_INF_F;
+                v[k].w = g0[k] + 3 < M ? __ldg(y + g0[k] + 3) : -CUDART_INF_F;
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            if (g0[k] < 0) continue;
+            const float vv[4] = {v[k].x, v[k].y, v[k].z, v[k].w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                if (g0[k] + i < M && vv[i] >= t_lo) {
+                    const int slot = atomicAdd(&hs.n_cand, 1);
+                    if (slot < kCandCap) hs.cand_id[slot] = g0[k] + i;
+                }
+            }
+        }
+    }
+    return true;
 }
 
 // Block: plan of `pair` into shared-memory tables (seg_prefix[nseg+1], seg_row, seg_mask) and the
@@ -214,30 +279,30 @@ __device__ __forceinline__ void build_pair_plan(const PlanInputs &in, int pair, 
     const uint16_t *rep = in.rep_keys + ((size_t)j * in.bv.teams_total + team0) * kHeadDim;
     const int32_t *csr = in.team_row_start + (size_t)j * (in.bv.teams_total + in.bv.n_seqs) + team0 + b;
 
-    // ---- queries in fp64, guard per head, candidate thresholds ----
-    for (int e = tid; e < G * kHeadDim; e += kPlanThreads)
-        sc.q64[e >> 7][e & 127] = bf16_to_double(in.q[(head0 + (e >> 7)) * kHeadDim + (e & 127)]);
-    __syncthreads();
-    if (warp < G) {
+    // ---- queries in fp64 (idle warps), guard per head and candidate thresholds (one warp per head) ----
+    if (warp >= G) {
+        for (int e = tid - 32 * G; e < G * kHeadDim; e += kPlanThreads - 32 * G)
+            sc.q64[e >> 7][e & 127] = bf16_to_double(in.q[(head0 + (e >> 7)) * kHeadDim + (e & 127)]);
+    } else {
         const int h = warp;
         HeadScratch &hs = sc.head[h];
-        double l1 = 0.0;
-        for (int d = lane; d < kHeadDim; d += 32) l1 += fabs(sc.q64[h][d]);
+        float l1 = 0.f;
+        for (int d = lane; d < kHeadDim; d += 32) l1 += fabsf(bf16_to_float(in.q[(head0 + h) * kHeadDim + d]));
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) l1 += __shfl_xor_sync(0xFFFFFFFFu, l1, o);
-        const float guard = score_guard(in.scale, l1, in.rep_abs_max[(size_t)j * in.bv.n_seqs + b]);
+        const float guard = score_guard(in.scale, (double)l1 * 1.001, in.rep_abs_max[(size_t)j * in.bv.n_seqs + b]);
         const float *y = in.y32 + ((size_t)j * G + h) * in.bv.teams_total + team0;
         const float *ym = in.ymax + ((size_t)j * G + h) * in.ymax_stride + (team0 >> 4) + b;
         const int nblk = (M + 15) >> 4;
-        const float t_lb = warp_lower_bound(ym, nblk, Ke + 1, lane, hs.bound_vals);
+        const float t_lb = warp_lower_bound(ym, nblk, Ke + 1, lane, hs.hist);
         const float t_lo = t_lb - 2.f * guard;
         // candidates in one go if they fit, else ranges of kCandCap teams in the loop below
         if (lane == 0) hs.n_cand = 0;
         __syncwarp();
-        warp_append_blocks(y, ym, 0, nblk, M, t_lo, hs, lane);
+        const bool listed = warp_append_listed(y, ym, nblk, M, t_lo, hs, lane);
         __syncwarp();
         if (lane == 0) {
-            const bool fits = hs.n_cand <= kCandCap;
+            const bool fits = listed && hs.n_cand <= kCandCap;
             hs.t_lo = t_lo;
             hs.n_list = 0;
             hs.range_len = fits ? M : kCandCap;
@@ -310,6 +375,7 @@ __device__ __forceinline__ void build_pair_plan(const PlanInputs &in, int pair, 
                 in.seed_lo, in.seed_hi);
             hs.cand_phi[i] = phi;
             hs.cand_y[i] = phi + gumbel_from_word(pick_word(words, id & 3));
+            if (i == hs.n_cand - 1) hs.cand_y[i + 1] = -CUDART_INF;
         }
         __syncthreads();
         // c. merge with the running list: keep the Ke + 1 largest by (Y descending, id ascending)
@@ -332,16 +398,26 @@ __device__ __forceinline__ void build_pair_plan(const PlanInputs &in, int pair, 
             int id;
             if (i < nl) { y = hs.list_y[cur][i]; phi = hs.list_phi[cur][i]; id = hs.list_id[cur][i]; }
             else { y = hs.cand_y[i - nl]; phi = hs.cand_phi[i - nl]; id = hs.cand_id[i - nl]; }
-            int rank = 0;
-#pragma unroll 4
-            for (int a = 0; a < nl; ++a) {
-                const double ya = hs.list_y[cur][a];
-                rank += (ya > y) || (ya == y && hs.list_id[cur][a] < id);
+            // rank = entries ahead in (Y descending, id ascending); scores are compared two at a
+            // time, and ids are looked at only when some other entry has exactly the same score
+            int rank = 0, same = 0;
+            const double2 *ly = reinterpret_cast<const double2 *>(hs.list_y[cur]);
+            const double2 *cy = reinterpret_cast<const double2 *>(hs.cand_y);
+#pragma unroll 2
+            for (int a = 0; a < (nl + 1) >> 1; ++a) {
+                const double2 w = ly[a];
+                rank += (w.x > y) + (w.y > y);
+                same += (w.x == y) + (w.y == y);
             }
-#pragma unroll 4
-            for (int a = 0; a < nc; ++a) {
-                const double ya = hs.cand_y[a];
-                rank += (ya > y) || (ya == y && hs.cand_id[a] < id);
+#pragma unroll 2
+            for (int a = 0; a < (nc + 1) >> 1; ++a) {
+                const double2 w = cy[a];
+                rank += (w.x > y) + (w.y > y);
+                same += (w.x == y) + (w.y == y);
+            }
+            if (same > 1) {
+                for (int a = 0; a < nl; ++a) rank += (hs.list_y[cur][a] == y && hs.list_id[cur][a] < id);
+                for (int a = 0; a < nc; ++a) rank += (hs.cand_y[a] == y && hs.cand_id[a] < id);
             }
             if (rank <= Ke) {
                 hs.list_y[cur ^ 1][rank] = y;
@@ -350,7 +426,11 @@ __device__ __forceinline__ void build_pair_plan(const PlanInputs &in, int pair, 
             }
         }
         __syncthreads();
-        if (tid < G) sc.head[tid].n_list = min(Ke + 1, sc.head[tid].n_list + sc.head[tid].n_cand);
+        if (tid < G) {
+            const int n_new = min(Ke + 1, sc.head[tid].n_list + sc.head[tid].n_cand);
+            sc.head[tid].n_list = n_new;
+            sc.head[tid].list_y[cur ^ 1][n_new] = -CUDART_INF;
+        }
         cur ^= 1;
         __syncthreads();
     }
