@@ -28,70 +28,75 @@ __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint3
                  : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1));
 }
 
-// Gumbel(0,1) in fp32 from a 32-bit word: u = (x + 0.5) / 2^32, G = -log(-log u). The upper half
-// of the range goes through log1p so that -log u keeps its relative accuracy as u -> 1.
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait_group()
+{
+    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
+constexpr int kScoreStages = 3;                                 // tiles in flight per warp (pipelined variant)
+constexpr int kScoreKeyRingBytes = kScoreStages * (kScoreThreads / 32) * 4096;
+constexpr int kScoreRingBytes = kScoreKeyRingBytes + kScoreStages * (kScoreThreads / 32) * 128;   // + row offsets
+
+// Gumbel(0,1) in fp32 from a 32-bit word: u = (x + 0.5) / 2^32, G = -log(-log u), to an absolute
+// error well inside the additive term of the guard (see score_guard in pairplan.cuh).
+// Lower half of the range (u <= 1/2): -log u >= 0.69 from the fast logarithm (3 ulp there).
+// Upper half: u = 1 - z with z = (2^32 - x - 0.5) / 2^32 in (0, 1/2]; -log(1 - z) from four series
+// terms when z < 2^-6 (relative truncation z^4 / 5 < 1.2e-8), else from the fast logarithm, whose
+// absolute error 2^-21.4 is then below 2.3e-5 of the result. The outer logarithm sees values in
+// (1e-10, 23) where the fast logarithm is accurate to 3 ulp or 2^-21.4 absolute.
 __device__ __forceinline__ float gumbel32_from_word(uint32_t x)
 {
     float nl;
     if (x >= 0x80000000u) {
-        const float w = (float)(0xFFFFFFFFu - x) + 0.5f;              // 2^32 - x - 0.5
-        nl = -log1pf(-w * 2.3283064365386963e-10f);
+        const float z = ((float)(0xFFFFFFFFu - x) + 0.5f) * 2.3283064365386963e-10f;
+        nl = z < 0.015625f ? z * (1.f + z * (0.5f + z * (0.33333334f + z * 0.25f))) : -__logf(1.f - z);
     } else {
-        nl = -logf(((float)x + 0.5f) * 2.3283064365386963e-10f);
+        nl = -__logf(((float)x + 0.5f) * 2.3283064365386963e-10f);
     }
-    return -logf(nl);
+    return -__logf(nl);
 }
 
+// A fragments of q for the GQA group of (b, j): k-step s of thread column c covers dims
+// (c + 4 (s / 2)) * 8 + 4 (s % 2) + {0,1} (a0) and + {2,3} (a2); the B fragments use the same
+// permutation of the 128 dims, so a lane feeds the tensor core the 16-byte pieces c, c+4, c+8,
+// c+12 of a key row exactly as they lie in memory.
 template <int G>
-__global__ void __launch_bounds__(kScoreThreads)
-score32_kernel(ScoreParams p)
+__device__ __forceinline__ void load_q_fragments(const ScoreParams &p, int b, int j, int g, int c, uint32_t (&qa)[8][2])
 {
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int g = lane >> 2, c = lane & 3;
-    const int pair = blockIdx.y;
-    const int b = pair / p.bv.n_kv, j = pair - b * p.bv.n_kv;
-
-    // The first block clears the tickets the later kernels of this call count on.
-    if (blockIdx.x == 0 && blockIdx.y == 0) {
-        for (int i = tid; i < p.n_pairs; i += kScoreThreads) p.ctl.attend_ticket[i] = 0;
-        if (tid == 0) {
-            *p.ctl.plan_ticket = 0;
-            if (p.status) *p.status = 0;
-        }
-    }
-
-    const int64_t team0 = p.bv.seq_team_off[b];
-    const int M = (int)(p.bv.seq_team_off[b + 1] - team0);
-    if (p.n_sample >= M) return;                       // every team is read; nothing is drawn
-    const int base = blockIdx.x * kScoreTeamsPerCta + warp * kScoreTeamsPerWarp;
-    if (base >= M) return;
-
-    // A fragments of q: k-step s of thread column c covers dims (c + 4 (s / 2)) * 8 + 4 (s % 2) + {0,1}
-    // (a0) and + {2,3} (a2); the B fragments below use the same permutation of the 128 dims.
-    uint32_t qa[8][2];
-    {
-        const uint32_t *qrow = reinterpret_cast<const uint32_t *>(
-            p.q + ((size_t)b * p.bv.n_q + (size_t)j * G + (g < G ? g : 0)) * kHeadDim);
+    const uint32_t *qrow = reinterpret_cast<const uint32_t *>(
+        p.q + ((size_t)b * p.bv.n_q + (size_t)j * G + (g < G ? g : 0)) * kHeadDim);
 #pragma unroll
-        for (int s = 0; s < 8; ++s) {
-            const int w = (c + 4 * (s >> 1)) * 4 + 2 * (s & 1);
-            qa[s][0] = g < G ? __ldg(qrow + w) : 0u;
-            qa[s][1] = g < G ? __ldg(qrow + w + 1) : 0u;
-        }
+    for (int s = 0; s < 8; ++s) {
+        const int w = (c + 4 * (s >> 1)) * 4 + 2 * (s & 1);
+        qa[s][0] = g < G ? __ldg(qrow + w) : 0u;
+        qa[s][1] = g < G ? __ldg(qrow + w + 1) : 0u;
     }
-    const uint16_t *rep = p.rep_keys + ((size_t)j * p.bv.teams_total + team0) * kHeadDim;
-    const int32_t *csr = p.team_row_start + (size_t)j * (p.bv.teams_total + p.bv.n_seqs) + team0 + b;
-    const uint32_t step = p.step + (p.step_dev ? *p.step_dev : 0u);
-    const float scale = (float)p.scale;
+}
 
-    // two n-tiles of 8 teams; B row n = team base + 8 tile + g, this lane holds chunks c, c+4, c+8, c+12
-    uint4 kb[2][4];
+// Scores of one tile of 16 teams (two n-tiles of 8; B row n = team base + 8 t + g) from the key
+// pieces kb of this lane: writes Y32 for the G heads and the tile's maximum per head.
+// csr_tile points at the 17 row offsets of the tile's teams (global or shared memory).
+template <int G>
+__device__ __forceinline__ void score_tile(const ScoreParams &p, int b, int j, int64_t team0, int M, int base,
+                                           const int32_t *csr_tile, const uint4 (&kb)[2][4], const uint32_t (&qa)[8][2],
+                                           uint32_t step, float scale, int g, int c)
+{
+    const uint32_t head = (uint32_t)(j * G + (g < G ? g : 0));
+    float *y = p.y32 + (size_t)head * p.bv.teams_total + team0;
+    // team sizes of this lane's four teams (teams base + 8 t + 2 c, + 1)
+    int n_team[2][2];
 #pragma unroll
     for (int t = 0; t < 2; ++t) {
-        const int team = min(base + 8 * t + g, M - 1);
-        const uint4 *row = reinterpret_cast<const uint4 *>(rep + (size_t)team * kHeadDim);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) kb[t][i] = __ldg(row + c + 4 * i);
+        const int t0 = base + 8 * t + 2 * c, o = 8 * t + 2 * c;
+        const int r0 = t0 < M ? csr_tile[o] : 0, r1 = t0 < M ? csr_tile[o + 1] : 1, r2 = t0 + 1 < M ? csr_tile[o + 2] : 2;
+        n_team[t][0] = r1 - r0;
+        n_team[t][1] = r2 - r1;
     }
     float acc[2][4];
 #pragma unroll
@@ -103,37 +108,205 @@ score32_kernel(ScoreParams p)
             mma_bf16_16816(acc[t], qa[2 * i + 1][0], qa[2 * i + 1][1], kb[t][i].z, kb[t][i].w);
         }
     }
-    // acc[t][0], acc[t][1]: head g, teams base + 8 t + 2c, + 1
+    // One Philox block covers four consecutive teams of a head: teams base + 8 t + {0..3} belong
+    // to thread columns 0 and 1, + {4..7} to columns 2 and 3. The even column computes the block
+    // of n-tile 0, the odd one that of n-tile 1, and the two exchange halves.
+    const int my_t = c & 1;
+    const uint4 words = philox4x32_10(
+        make_uint4((uint32_t)(base + 8 * my_t + 4 * (c >> 1)) >> 2, step, head, p.stream_base + (uint32_t)b),
+        p.seed_lo, p.seed_hi);
+    // this lane needs words {2 (c & 1), 2 (c & 1) + 1} of both n-tiles' blocks
+    uint32_t w[2][2];
+    {
+        const uint32_t give0 = (c & 1) ? words.x : words.z, give1 = (c & 1) ? words.y : words.w;
+        const uint32_t got0 = __shfl_xor_sync(0xFFFFFFFFu, give0, 1), got1 = __shfl_xor_sync(0xFFFFFFFFu, give1, 1);
+        const uint32_t keep0 = (c & 1) ? words.z : words.x, keep1 = (c & 1) ? words.w : words.y;
+        w[0][0] = my_t ? got0 : keep0;
+        w[0][1] = my_t ? got1 : keep1;
+        w[1][0] = my_t ? keep0 : got0;
+        w[1][1] = my_t ? keep1 : got1;
+    }
+    // acc[t][0], acc[t][1]: head g, teams base + 8 t + 2 c, + 1
     float blk_max = -INFINITY;
-    const uint32_t head = (uint32_t)(j * G + (g < G ? g : 0));
     if (g < G) {
-        float *y = p.y32 + (size_t)head * p.bv.teams_total + team0;
 #pragma unroll
         for (int t = 0; t < 2; ++t) {
-            const int t0 = base + 8 * t + 2 * c;                      // even team id: both share a Philox block
-            if (t0 < M) {
-                const uint4 words = philox4x32_10(
-                    make_uint4((uint32_t)t0 >> 2, step, head, p.stream_base + (uint32_t)b), p.seed_lo, p.seed_hi);
-                const int r0 = csr[t0], r1 = csr[t0 + 1];
-                const float y0 = logf((float)(r1 - r0)) + acc[t][0] * scale
-                                 + gumbel32_from_word(pick_word(words, t0 & 3));
-                y[t0] = y0;
-                blk_max = fmaxf(blk_max, y0);
-                if (t0 + 1 < M) {
-                    const int r2 = csr[t0 + 2];
-                    const float y1 = logf((float)(r2 - r1)) + acc[t][1] * scale
-                                     + gumbel32_from_word(pick_word(words, (t0 & 3) + 1));
-                    y[t0 + 1] = y1;
-                    blk_max = fmaxf(blk_max, y1);
-                }
-            }
+            const int t0 = base + 8 * t + 2 * c;
+            const float y0 = __logf((float)n_team[t][0]) + acc[t][0] * scale + gumbel32_from_word(w[t][0]);
+            const float y1 = __logf((float)n_team[t][1]) + acc[t][1] * scale + gumbel32_from_word(w[t][1]);
+            if (t0 < M) { y[t0] = y0; blk_max = fmaxf(blk_max, y0); }
+            if (t0 + 1 < M) { y[t0 + 1] = y1; blk_max = fmaxf(blk_max, y1); }
         }
     }
-    // largest score of the warp's 16-team block, per head (the quad of a head holds its 16 scores)
+    // largest score of the 16-team block, per head (the quad of a head holds its 16 scores)
     blk_max = fmaxf(blk_max, __shfl_xor_sync(0xFFFFFFFFu, blk_max, 1));
     blk_max = fmaxf(blk_max, __shfl_xor_sync(0xFFFFFFFFu, blk_max, 2));
     if (g < G && c == 0)
         p.ymax[(size_t)head * p.ymax_stride + (size_t)(team0 >> 4) + b + (base >> 4)] = blk_max;
+}
+
+__device__ __forceinline__ void clear_control(const ScoreParams &p, int tid)
+{
+    // The first block clears the tickets the later kernels of this call count on.
+    for (int i = tid; i < p.n_pairs; i += kScoreThreads) p.ctl.attend_ticket[i] = 0;
+    if (tid == 0) {
+        *p.ctl.plan_ticket = 0;
+        if (p.status) *p.status = 0;
+    }
+}
+
+// Small grids: one warp per tile of 16 teams, keys straight into registers (the shortest path).
+template <int G>
+__global__ void __launch_bounds__(kScoreThreads, 2)
+score32_kernel(ScoreParams p)
+{
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int g = lane >> 2, c = lane & 3;
+    const int pair = blockIdx.y;
+    const int b = pair / p.bv.n_kv, j = pair - b * p.bv.n_kv;
+    if (blockIdx.x == 0 && blockIdx.y == 0) clear_control(p, tid);
+
+    const int64_t team0 = p.bv.seq_team_off[b];
+    const int M = (int)(p.bv.seq_team_off[b + 1] - team0);
+    if (p.n_sample >= M) return;                       // every team is read; nothing is drawn
+    const int base = (blockIdx.x * (kScoreThreads / 32) + warp) * kScoreTeamsPerWarp;
+    if (base >= M) return;
+    uint32_t qa[8][2];
+    load_q_fragments<G>(p, b, j, g, c, qa);
+    const uint16_t *rep = p.rep_keys + ((size_t)j * p.bv.teams_total + team0) * kHeadDim;
+    uint4 kb[2][4];
+#pragma unroll
+    for (int t = 0; t < 2; ++t) {
+        const uint4 *row = reinterpret_cast<const uint4 *>(rep + (size_t)min(base + 8 * t + g, M - 1) * kHeadDim);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) kb[t][i] = __ldg(row + c + 4 * i);
+    }
+    const uint32_t step = p.step + (p.step_dev ? *p.step_dev : 0u);
+    const int32_t *csr = p.team_row_start + (size_t)j * (p.bv.teams_total + p.bv.n_seqs) + team0 + b;
+    score_tile<G>(p, b, j, team0, M, base, csr + base, kb, qa, step, (float)p.scale, g, c);
+}
+
+// Where a tile index of the flat kernel lies: tiles are the slots of the block-maximum table,
+// n_kv * ymax_stride of them; sequence b owns slots [(seq_team_off[b] >> 4) + b, ... + ceil(M / 16)),
+// the few slots between sequences are empty.
+struct TileCursor {
+    int j, s;                       // KV head and slot of the current tile
+    int b, slot_lo, slot_hi, M;     // sequence owning the slot range [slot_lo, slot_hi)
+    int64_t team0;
+};
+
+__device__ __forceinline__ TileCursor cursor_at(const ScoreParams &p, long long ti)
+{
+    TileCursor cur;
+    cur.j = (int)(ti / p.ymax_stride);
+    cur.s = (int)(ti - (long long)cur.j * p.ymax_stride);
+    cur.b = 0; cur.slot_lo = 0; cur.slot_hi = 0; cur.M = 0; cur.team0 = 0;      // empty range: located on first use
+    return cur;
+}
+
+// Tile under the cursor: true with its first team in `base` when it has teams to score.
+__device__ __forceinline__ bool locate_tile(const ScoreParams &p, TileCursor &cur, int &base)
+{
+    const int s = cur.s;
+    if (s < cur.slot_lo || s >= cur.slot_hi) {
+        int lo = 0, hi = p.bv.n_seqs - 1;              // largest b with start(b) <= s
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if ((int)(p.bv.seq_team_off[mid] >> 4) + mid <= s) lo = mid; else hi = mid - 1;
+        }
+        cur.b = lo;
+        cur.team0 = p.bv.seq_team_off[lo];
+        const int64_t next0 = p.bv.seq_team_off[lo + 1];
+        cur.M = (int)(next0 - cur.team0);
+        cur.slot_lo = (int)(cur.team0 >> 4) + lo;
+        cur.slot_hi = lo + 1 < p.bv.n_seqs ? (int)(next0 >> 4) + lo + 1 : p.ymax_stride;
+    }
+    base = (s - cur.slot_lo) * 16;
+    return base < cur.M && p.n_sample < cur.M;
+}
+
+__device__ __forceinline__ void advance(const ScoreParams &p, TileCursor &cur)
+{
+    if (++cur.s == p.ymax_stride) { cur.s = 0; ++cur.j; cur.slot_lo = cur.slot_hi = 0; }
+}
+
+// Large grids: two resident blocks per SM, every warp walks an equal contiguous share of all
+// tiles. The keys of the next kScoreStages tiles are in flight as cp.async copies into slots
+// private to each lane (a lane copies exactly the pieces it later feeds to the tensor core, so
+// no barrier is needed).
+template <int G>
+__global__ void __launch_bounds__(kScoreThreads, 2)
+score32_flat_kernel(ScoreParams p)
+{
+    extern __shared__ uint4 score_ring[];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int g = lane >> 2, c = lane & 3;
+    if (blockIdx.x == 0) clear_control(p, tid);
+
+    const long long n_tiles = (long long)p.bv.n_kv * p.ymax_stride;
+    const long long n_warps = (long long)gridDim.x * (kScoreThreads / 32), gw = (long long)blockIdx.x * (kScoreThreads / 32) + warp;
+    const long long t_lo = gw * n_tiles / n_warps, t_hi = (gw + 1) * n_tiles / n_warps;
+    const uint32_t step = p.step + (p.step_dev ? *p.step_dev : 0u);
+    const float scale = (float)p.scale;
+
+    // slot of piece (t, i) of stage s: [warp][s][t * 4 + i][lane]
+    auto slot = [&](int s, int t, int i) { return score_ring + ((warp * kScoreStages + s) * 8 + t * 4 + i) * 32 + lane; };
+    // the tile's 17 row offsets, copied by lanes 0..16: [warp][s][32]
+    int32_t *csr_ring = reinterpret_cast<int32_t *>(reinterpret_cast<unsigned char *>(score_ring) + kScoreKeyRingBytes)
+                        + warp * kScoreStages * 32;
+    TileCursor ahead = cursor_at(p, t_lo), here = ahead;
+    long long t_ahead = t_lo;                                   // tile index under `ahead`
+    auto issue_tile = [&](int s) {
+        int base;
+        if (t_ahead < t_hi && locate_tile(p, ahead, base)) {
+            const uint16_t *rep = p.rep_keys + ((size_t)ahead.j * p.bv.teams_total + ahead.team0) * kHeadDim;
+#pragma unroll
+            for (int t = 0; t < 2; ++t) {
+                const uint4 *row = reinterpret_cast<const uint4 *>(rep + (size_t)min(base + 8 * t + g, ahead.M - 1) * kHeadDim);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) cp_async16((uint32_t)__cvta_generic_to_shared(slot(s, t, i)), row + c + 4 * i);
+            }
+            if (lane <= 16 && base + lane <= ahead.M) {
+                const int32_t *csr = p.team_row_start + (size_t)ahead.j * (p.bv.teams_total + p.bv.n_seqs) + ahead.team0
+                                     + ahead.b + base + lane;
+                asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"((uint32_t)__cvta_generic_to_shared(
+                                 csr_ring + s * 32 + lane)), "l"(csr) : "memory");
+            }
+        }
+        cp_async_commit();                                       // one group per tile, empty or not
+        ++t_ahead;
+        advance(p, ahead);
+    };
+#pragma unroll
+    for (int s = 0; s < kScoreStages; ++s) issue_tile(s);
+
+    uint32_t qa[8][2];
+    int q_b = -1, q_j = -1;
+    int stage = 0;
+    for (long long ti = t_lo; ti < t_hi; ++ti) {
+        cp_async_wait_group<kScoreStages - 1>();                 // this lane's pieces of tile ti have landed
+        __syncwarp();                                            // the row offsets come from other lanes
+        int base;
+        if (locate_tile(p, here, base)) {
+            if (here.b != q_b || here.j != q_j) {
+                load_q_fragments<G>(p, here.b, here.j, g, c, qa);
+                q_b = here.b;
+                q_j = here.j;
+            }
+            uint4 kb[2][4];
+#pragma unroll
+            for (int t = 0; t < 2; ++t)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) kb[t][i] = *slot(stage, t, i);
+            score_tile<G>(p, here.b, here.j, here.team0, here.M, base, csr_ring + stage * 32, kb, qa, step, scale, g, c);
+        }
+        __syncwarp();                                            // every lane is done with the stage's row offsets
+        // refill the stage just consumed (its pieces are in registers and already used above)
+        issue_tile(stage);
+        advance(p, here);
+        stage = stage + 1 == kScoreStages ? 0 : stage + 1;
+    }
+    cp_async_wait_group<0>();
 }
 
 // One block per (sequence, KV head): largest |element| among the pair's representative keys.
@@ -163,8 +336,20 @@ rep_abs_max_kernel(BatchView bv, const uint16_t *rep_keys, float *rep_abs_max)
 template <int G>
 cudaError_t launch_score32_g(const ScoreParams &p, int max_teams, cudaStream_t s)
 {
-    dim3 grid((max_teams + kScoreTeamsPerCta - 1) / kScoreTeamsPerCta, p.n_pairs);
-    score32_kernel<G><<<grid, kScoreThreads, 0, s>>>(p);
+    const long long ctas1 = (long long)((max_teams + kScoreTeamsPerCta - 1) / kScoreTeamsPerCta) * p.n_pairs;
+    if (ctas1 < 2 * 148) {
+        dim3 grid((max_teams + kScoreTeamsPerCta - 1) / kScoreTeamsPerCta, p.n_pairs);
+        score32_kernel<G><<<grid, kScoreThreads, 0, s>>>(p);
+        return cudaGetLastError();
+    }
+    static bool configured = false;                              // per template instance; idempotent
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(score32_flat_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             kScoreRingBytes);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    score32_flat_kernel<G><<<2 * attend_grid_size(), kScoreThreads, kScoreRingBytes, s>>>(p);
     return cudaGetLastError();
 }
 
