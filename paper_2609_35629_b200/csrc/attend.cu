@@ -103,7 +103,7 @@ struct Smem {
     static constexpr size_t misc = pair_nseg + kPairMax * 4;                    // flags
     static constexpr size_t total = misc + 64;
     // aliases of the ring: plan scratch before a pair's rows are streamed, merge scratch after
-    static_assert(sizeof(PlanScratch<G>) <= ring_bytes, "plan scratch must fit in the ring");
+    static_assert(sizeof(PlanScratch) <= ring_bytes, "plan scratch must fit in the ring");
     static constexpr size_t red_acc = ring;                                     // float [warps][G][128]
     static constexpr size_t red_m = red_acc + (size_t)kWarps * G * kHeadDim * 4;   // float [warps][G]
     static constexpr size_t red_l = red_m + (size_t)kWarps * G * 4;
@@ -196,7 +196,7 @@ attend_kernel(AttendParams p)
                 nseg = misc[2];
                 rows = misc[3];
             } else {
-                PlanScratch<G> &scratch = *reinterpret_cast<PlanScratch<G> *>(smem + S::ring);
+                PlanScratch &scratch = *reinterpret_cast<PlanScratch *>(smem + S::ring);
                 build_pair_plan<G>(p.in, pair, scratch, seg_prefix, seg_row, seg_mask,
                                    p.plan.seg_logc + (size_t)pair * cap * kMaxGroup, nseg, rows, sub == 0);
             }

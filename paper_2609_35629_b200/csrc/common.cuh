@@ -65,7 +65,7 @@ struct ScoreParams {
     int32_t *status;                // nullable
 };
 
-// What the sampling step reads (see pairplan.cuh).
+// What the sampling step (headplan.cu) and the union step (pairplan.cuh) read and write.
 struct PlanInputs {
     BatchView bv;
     const float *y32;               // [n_q][teams_total]
@@ -81,6 +81,8 @@ struct PlanInputs {
     double scale;
     const int32_t *suffix_len;      // nullable
     int suffix_cap;
+    int32_t *sel_team;              // [n_seqs][n_q][n_sample] sampled teams of each head, descending score
+    float *sel_logc;                // [n_seqs][n_q][n_sample] log c_g of each
     // diagnostics (nullable)
     int32_t *dbg_sel_idx;
     float *dbg_sel_logc;
@@ -117,6 +119,7 @@ struct AttendParams {
 // ---------------------------------------------------------------------------------------------
 cudaError_t launch_score32(const ScoreParams &p, int max_teams_per_seq, cudaStream_t s);
 cudaError_t launch_rep_abs_max(const BatchView &bv, const uint16_t *rep_keys, float *rep_abs_max, cudaStream_t s);
+cudaError_t launch_headplan(const PlanInputs &in, cudaStream_t s);
 cudaError_t launch_plan(const PlanParams &p, cudaStream_t s);
 cudaError_t launch_dense_plan(const PlanParams &p, cudaStream_t s);
 // split: 0 = rows of all pairs cut into equal ranges (plan read from global memory),

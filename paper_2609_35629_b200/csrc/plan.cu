@@ -1,5 +1,5 @@
 // Read plans in global memory, for the attention kernel's equal-range split:
-//   plan_kernel        one block per (sequence, KV head) pair: sampling and plan of the pair
+//   plan_kernel        one block per (sequence, KV head) pair: union of the heads' samples
 //                      (pairplan.cuh), copied out to the workspace; the last block to finish turns
 //                      the pairs' row counts into the global row prefix.
 //   dense_plan_kernel  the trivial plan that reads every prompt row and the suffix.
@@ -34,7 +34,7 @@ __device__ void publish_pair_prefix(const PlanParams &p, int *flag_smem, int *sc
 
 template <int G>
 struct PlanKernelSmem {
-    PlanScratch<G> scratch;
+    PlanScratch scratch;
     int seg_prefix[kSegMax + 3];
     int seg_row[kSegMax + 3];
     uint32_t seg_mask[kSegMax + 3];
