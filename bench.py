@@ -196,21 +196,18 @@ def run_ours(args):
     import torch
     import torch.distributed as dist
     from paper_2609_35629_b200 import binding as sp
-    from paper_2609_35629_b200 import synth
+    from paper_2609_35629_b200 import replicas, synth
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, world, local_rank = replicas.env_rank_world()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
+    replicas.init_replicas("nccl", dev)
     sp.load_library()
 
     # Independent replicas: every rank owns its own sequences (seed = rank); no exchange.
-    spec = make_spec(args, seed=rank)
+    spec = make_spec(args, seed=replicas.replica_seed(0, rank))
     L = args.layers
     geom = sp.Geometry(spec.n_seqs, spec.n_q_heads, spec.n_kv_heads, spec.head_dim, spec.parent_size,
                        spec.reps_per_parent)
@@ -265,7 +262,7 @@ def run_ours(args):
     ws = [torch.empty(sp.santapp_decode_workspace_bytes(geom, layers[l]["teams"], K), dtype=torch.uint8, device=dev)
           for l in range(L)]
     wsd = torch.empty(sp.santapp_dense_workspace_bytes(geom, layers[0]["teams"]), dtype=torch.uint8, device=dev)
-    seed = 1234 + rank
+    seed = replicas.replica_seed(1234, rank)
 
     def sparse_layer(l, debug=None):
         ly = layers[l]
@@ -317,10 +314,7 @@ def run_ours(args):
     g_dense = capture(dense_layer)
 
     def barrier():
-        torch.cuda.synchronize()
-        if world > 1:
-            dist.barrier()
-            torch.cuda.synchronize()
+        replicas.barrier(dev)
 
     def timed(run_step, steps, warmup, sampler=None):
         for i in range(warmup):
@@ -336,11 +330,7 @@ def run_ours(args):
         torch.cuda.synchronize()
         if sampler:
             sampler.stop()
-        ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
+        ms = replicas.max_over_ranks(e0.elapsed_time(e1), dev)
         barrier()
         return ms
 
@@ -358,8 +348,8 @@ def run_ours(args):
     clocks = sampler.summary()
     n_dense = max(min(Kst, 50), 3)
     ms_dense = timed(dense_step, n_dense, 3)
-    us_layer = 1e3 * ms_sparse / (Kst * L * world)
-    us_layer_dense = 1e3 * ms_dense / (n_dense * L * world)
+    us_layer = replicas.us_per_layer_step(ms_sparse, Kst, L, world)
+    us_layer_dense = replicas.us_per_layer_step(ms_dense, n_dense, L, world)
 
     used = np.array([(W + i) % N_STEP_INPUTS for i in range(Kst)])
     mean_sparse_bytes = float(sparse_bytes[used].mean())
@@ -373,7 +363,7 @@ def run_ours(args):
         for l in range(L):
             sparse_layer(l)
     ms_eager = timed(eager_step, max(Kst // 10, 3), 3)
-    us_layer_eager = 1e3 * ms_eager / (max(Kst // 10, 3) * L * world)
+    us_layer_eager = replicas.us_per_layer_step(ms_eager, max(Kst // 10, 3), L, world)
 
     # ---- isolated stages (graphs of one stage over all layers; plans and scores left in the
     # per-layer workspaces by a full step with the same inputs) ----
@@ -389,7 +379,7 @@ def run_ours(args):
             sp.santapp_set_stage_mask(sp.STAGE_ALL)
             reps = max(Kst // 4, 10)
             ms = timed(lambda i: g.replay(), reps, 3)
-            stages[name] = 1e3 * ms / (reps * L)
+            stages[name] = 1e3 * ms / (reps * L)                       # per launch on one GPU (slowest rank)
         attend_bytes_1 = float(attend_bytes[1].mean())
     peaks = {}
     try:
@@ -431,7 +421,7 @@ def run_ours(args):
 
         n_e2e = max(Kst // 4, 5)
         ms_e2e = timed(e2e_step, n_e2e, 3)
-        e2e = {"value": 1e3 * ms_e2e / (n_e2e * L * world), "unit": UNIT,
+        e2e = {"value": replicas.us_per_layer_step(ms_e2e, n_e2e, L, world), "unit": UNIT,
                "h2d_bytes_per_step": int(in_bytes + new_rows[0].numel() * 2),
                "d2h_bytes_per_step": int(out_host.numel() * 4)}
 
