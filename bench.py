@@ -34,6 +34,12 @@ METRIC = "decode_attn_us_per_layer_step"
 UNIT = "us"
 N_STEP_INPUTS = 8          # distinct (query, suffix length, step) inputs cycled through
 
+# DRAM bytes (read + write) of one attend_kernel launch from an ncu capture of the same per-launch
+# work (summaries under profiles/, named for the kernel and workload); None where none was taken.
+NCU_TRAFFIC_BYTES = {
+    "qwen7b_b1_32k": 34.51e6,      # profiles/attend_kernel_qwen7b_b1_32k.md
+}
+
 
 def parse_args():
     ap = argparse.ArgumentParser()
@@ -392,7 +398,9 @@ def run_ours(args):
     if stages:
         achieved = attend_bytes_1 / (stages["attend"] * 1e-6) / 1e9
         roofline = {"bound": "hbm", "kernel": "attend_kernel", "achieved": achieved, "peak": peak_gbs, "unit": "GB/s",
-                    "frac": achieved / peak_gbs, "traffic": None, "peak_kind": peak_kind,
+                    "frac": achieved / peak_gbs,
+                    "traffic": NCU_TRAFFIC_BYTES.get(spec.name) if not args.n_sample else None,
+                    "peak_kind": peak_kind,
                     "algorithmic_bytes_per_launch": attend_bytes_1, "us_per_launch": stages["attend"]}
 
     # ---- end to end through host buffers ----
@@ -481,8 +489,8 @@ def cpu_baseline_leg(spec, data, teams, seed):
     v = synth.bf16_to_f64(data.v_prompt[:, r0:r1])
     scale = 1.0 / math.sqrt(d)
     times, n = [], 0
-    budget = time.perf_counter() + 15.0
-    while time.perf_counter() < budget and n < 400:
+    budget = time.perf_counter() + 12.0
+    while time.perf_counter() < budget and n < 4000:
         step = n % spec.n_steps
         q = synth.bf16_to_f64(synth.make_queries(spec, data, step % N_STEP_INPUTS)[b])
         t = int(spec.suffix_len(step)[b])
