@@ -255,11 +255,12 @@ int santapp_last_launch_count(void);
 /*
  * Diagnostic: choose which stages the following santapp_decode_attn calls on this thread
  * launch, for timing one stage in isolation (the paper's "isolated-stage measurements").
- * Bit 0: representative scoring and perturbation; bit 1: selection and read plan (a kernel of
- * its own only for batches of many (sequence, KV head) pairs; for few pairs that work is the
- * first phase of the attention kernel); bit 2: exact attention and merge. A stage that is
- * skipped reuses what an earlier full call with the same arguments left in the same workspace. The default, and the only setting that computes a
- * decode step, is SANTAPP_STAGE_ALL.
+ * Bit 0: representative scoring and perturbation; bit 1: sampling per query head, and the
+ * read plans as a kernel of their own for batches of many (sequence, KV head) pairs (for few
+ * pairs the union of the heads' samples is the first phase of the attention kernel);
+ * bit 2: exact attention and merge. A stage that is skipped reuses what an earlier full call
+ * with the same arguments left in the same workspace. The default, and the only setting that
+ * computes a decode step, is SANTAPP_STAGE_ALL.
  */
 enum { SANTAPP_STAGE_ROUTE = 1, SANTAPP_STAGE_SELECT = 2, SANTAPP_STAGE_ATTEND = 4, SANTAPP_STAGE_ALL = 7 };
 void santapp_set_stage_mask(int mask);
