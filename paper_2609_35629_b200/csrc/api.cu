@@ -72,7 +72,7 @@ BatchView make_view(const santapp_geom *g, const santapp_teams *t)
 
 // Workspace layout shared by the sparse and the dense call. Offsets in bytes.
 struct DecodeLayout {
-    size_t ctl, y32, ymax, sel_team, sel_logc, seg_prefix, seg_row, seg_mask, seg_logc, pair_nseg, pair_rows, pair_prefix, partials, total;
+    size_t ctl, y32, ymax, sel_team, sel_logc, sel_rows, seg_prefix, seg_row, seg_mask, seg_logc, pair_nseg, pair_rows, pair_prefix, partials, total;
     int seg_cap, grid, n_pairs, ctas_per_pair, ymax_stride;
     bool static_split;
 };
@@ -98,6 +98,7 @@ DecodeLayout decode_layout(const santapp_geom *g, const santapp_teams *t, int K,
     L.ymax = take(dense ? 0 : sizeof(float) * (size_t)g->n_q_heads * (size_t)L.ymax_stride);
     L.sel_team = take(dense ? 0 : sizeof(int32_t) * (size_t)g->n_seqs * g->n_q_heads * K);
     L.sel_logc = take(dense ? 0 : sizeof(float) * (size_t)g->n_seqs * g->n_q_heads * K);
+    L.sel_rows = take(dense ? 0 : sizeof(int2) * (size_t)g->n_seqs * g->n_q_heads * K);
     L.seg_prefix = take(sizeof(int32_t) * (size_t)L.n_pairs * (L.seg_cap + 1));
     L.seg_row = take(sizeof(int32_t) * (size_t)L.n_pairs * L.seg_cap);
     L.seg_mask = take(sizeof(uint32_t) * (size_t)L.n_pairs * L.seg_cap);
@@ -316,6 +317,7 @@ int santapp_decode_attn(const santapp_geom *geom, const santapp_teams *teams, co
     pp.in.suffix_cap = suffix_cap;
     pp.in.sel_team = reinterpret_cast<int32_t *>(ws + L.sel_team);
     pp.in.sel_logc = reinterpret_cast<float *>(ws + L.sel_logc);
+    pp.in.sel_rows = reinterpret_cast<int2 *>(ws + L.sel_rows);
     pp.in.dbg_sel_idx = dbg ? dbg->sel_idx : nullptr;
     pp.in.dbg_sel_logc = dbg ? dbg->sel_logc : nullptr;
     pp.in.dbg_tau = dbg ? dbg->tau : nullptr;

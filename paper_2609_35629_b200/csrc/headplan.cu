@@ -13,7 +13,7 @@
 //   4. the K largest are the sample, the next one is tau, c_g = 1 - exp(-exp(phi_g - tau)).
 // At most kCandCap candidates are held at a time; when more qualify the teams are walked in ranges
 // of kCandCap with a running top-(K+1) list, so any number of candidates fits in shared memory.
-// Output per head: the K sampled team ids in descending Y, and log c_g for each.
+// Output per head: the K sampled team ids in descending Y, log c_g and the packed row range of each.
 #include <math_constants.h>
 
 #include "common.cuh"
@@ -22,12 +22,10 @@ namespace santapp {
 
 namespace {
 
-constexpr int kHeadThreads = 256;
-constexpr int kHeadWarps = kHeadThreads / 32;
+constexpr int kMaxHeadWarps = 8;         // blocks of 256 threads, or 128 when many heads share the GPU
 constexpr int kCandCap = 512;           // candidates refined at a time
 constexpr int kListCap = 132;           // running top list: K + 1 <= 129 entries (+ one pad)
 constexpr int kDotLanes = 8;            // threads that share one candidate's dot product
-constexpr int kDotWarps = 4;            // warps 0..3 compute dot products, the others the Gumbel terms
 constexpr int kWindow = 255;            // histogram bins per pass of the bound
 
 struct alignas(16) HeadSmem {
@@ -39,8 +37,10 @@ struct alignas(16) HeadSmem {
     double list_phi[2][kListCap];
     int list_id[2][kListCap];
     int cand_id[kCandCap];
+    int2 cand_rows[kCandCap];           // first packed row (local to the sequence) and size of the candidate's team
+    int2 list_rows[2][kListCap];
     int hist[256];
-    float red_max[kHeadWarps], red_sum[kHeadWarps];
+    float red_max[kMaxHeadWarps], red_sum[kMaxHeadWarps];
     int n_blk, n_cand, bound_bin, bound_below, bound_total;
 };
 
@@ -51,9 +51,12 @@ __device__ __forceinline__ float score_guard(double scale, double q_l1, float k_
     return (float)(2.5e-4 * scale * q_l1 * (double)k_abs_max + 1e-3);
 }
 
+// The first half of the block's warps compute dot products, the second half the Gumbel terms.
+template <int kHeadThreads>
 __global__ void __launch_bounds__(kHeadThreads)
 headplan_kernel(PlanInputs in)
 {
+    constexpr int kHeadWarps = kHeadThreads / 32, kDotWarps = kHeadWarps / 2;
     __shared__ HeadSmem sm;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int hq = blockIdx.x;                                        // (sequence, query head)
@@ -104,7 +107,7 @@ headplan_kernel(PlanInputs in)
     if (nblk >= need) {
         int above = 0;
         for (int win = 0; win < 16 * kWindow; win += kWindow) {      // 1020 units below the top, then give up
-            sm.hist[tid] = 0;
+            for (int i = tid; i < 256; i += kHeadThreads) sm.hist[i] = 0;
             __syncthreads();
             for (int i = tid; i < nblk; i += kHeadThreads) {
                 const float d = (top - __ldg(ym + i)) * 4.f;
@@ -187,7 +190,7 @@ headplan_kernel(PlanInputs in)
         }
         const int n_cand = sm.n_cand;
 
-        // ---- 3a. exact terms: dot products on warps 0..3 (8 lanes per candidate, 16 dims each),
+        // ---- 3a. exact terms: dot products on the first half of the warps (8 lanes per candidate, 16 dims each),
         //          log n_g and the Gumbel term on the other warps (one thread per candidate) ----
         if (warp < kDotWarps) {
             const int sub = lane & (kDotLanes - 1);
@@ -224,7 +227,9 @@ headplan_kernel(PlanInputs in)
         } else {
             for (int i = tid - kDotWarps * 32; i < n_cand; i += kHeadThreads - kDotWarps * 32) {
                 const int id = sm.cand_id[i];
-                const int n_g = csr[id + 1] - csr[id];
+                const int r_lo = csr[id];
+                const int n_g = csr[id + 1] - r_lo;
+                sm.cand_rows[i] = make_int2(r_lo, n_g);
                 const uint4 words = philox4x32_10(
                     make_uint4((uint32_t)id >> 2, step, (uint32_t)hh, in.stream_base + (uint32_t)b), in.seed_lo, in.seed_hi);
                 sm.cand_g[i] = gumbel_from_word(pick_word(words, id & 3));
@@ -244,8 +249,9 @@ headplan_kernel(PlanInputs in)
         for (int e = tid; e < n_list + n_cand; e += kHeadThreads) {
             double y, phi;
             int id;
-            if (e < n_list) { y = sm.list_y[cur][e]; phi = sm.list_phi[cur][e]; id = sm.list_id[cur][e]; }
-            else { y = sm.cand_y[e - n_list]; phi = sm.cand_phi[e - n_list]; id = sm.cand_id[e - n_list]; }
+            int2 rows;
+            if (e < n_list) { y = sm.list_y[cur][e]; phi = sm.list_phi[cur][e]; id = sm.list_id[cur][e]; rows = sm.list_rows[cur][e]; }
+            else { y = sm.cand_y[e - n_list]; phi = sm.cand_phi[e - n_list]; id = sm.cand_id[e - n_list]; rows = sm.cand_rows[e - n_list]; }
             // rank = entries ahead of this one; scores are compared two at a time, ids are looked at
             // only when some other entry has exactly the same score
             int rank = 0, same = 0;
@@ -271,6 +277,7 @@ headplan_kernel(PlanInputs in)
                 sm.list_y[cur ^ 1][rank] = y;
                 sm.list_phi[cur ^ 1][rank] = phi;
                 sm.list_id[cur ^ 1][rank] = id;
+                sm.list_rows[cur ^ 1][rank] = rows;
             }
         }
         n_list = min(K + 1, n_list + n_cand);
@@ -287,6 +294,7 @@ headplan_kernel(PlanInputs in)
         const int id = sm.list_id[cur][a];
         in.sel_team[(size_t)hq * K + a] = id;
         in.sel_logc[(size_t)hq * K + a] = logc;
+        in.sel_rows[(size_t)hq * K + a] = sm.list_rows[cur][a];
         if (in.dbg_sel_idx) in.dbg_sel_idx[(size_t)hq * K + a] = id;
         if (in.dbg_sel_logc) in.dbg_sel_logc[(size_t)hq * K + a] = logc;
     }
@@ -297,7 +305,11 @@ headplan_kernel(PlanInputs in)
 
 cudaError_t launch_headplan(const PlanInputs &in, cudaStream_t s)
 {
-    headplan_kernel<<<in.bv.n_seqs * in.bv.n_q, kHeadThreads, 0, s>>>(in);
+    // 256 threads per head while every head's block is resident at once (4 per SM by registers),
+    // else 128 threads so that twice as many fit
+    const int n_heads = in.bv.n_seqs * in.bv.n_q;
+    if (n_heads <= 4 * attend_grid_size()) headplan_kernel<256><<<n_heads, 256, 0, s>>>(in);
+    else                                   headplan_kernel<128><<<n_heads, 128, 0, s>>>(in);
     return cudaGetLastError();
 }
 

@@ -19,6 +19,7 @@ constexpr int kBitmapWords = kMaxTeamsPerSeq / 32;
 struct alignas(16) PlanScratch {
     int ent_key[kEntCap];               // team * 8 + head
     float ent_logc[kEntCap];
+    int2 ent_rows[kEntCap];             // first packed row (local to the sequence) and row count of the team
     uint32_t bitmap[kBitmapWords];
     int wprefix[kBitmapWords];
     int seg_rows[kSegMax];
@@ -83,13 +84,12 @@ __device__ __forceinline__ void build_pair_plan(const PlanInputs &in, int pair, 
         return;
     }
 
-    const int32_t *csr = in.team_row_start + (size_t)j * (in.bv.teams_total + in.bv.n_seqs) + team0 + b;
-
     // ---- the heads' samples ----
     for (int e = tid; e < G * Ke; e += kPlanThreads) {
         const int h = e / Ke, a = e - h * Ke;
         sc.ent_key[e] = in.sel_team[(head0 + h) * K + a] * kMaxGroup + h;
         sc.ent_logc[e] = in.sel_logc[(head0 + h) * K + a];
+        sc.ent_rows[e] = in.sel_rows[(head0 + h) * K + a];
     }
     for (int i = tid; i < (M + 31) / 32; i += kPlanThreads) sc.bitmap[i] = 0u;
     for (int i = tid; i <= G * Ke; i += kPlanThreads) seg_mask[i] = 0u;
@@ -119,9 +119,8 @@ __device__ __forceinline__ void build_pair_plan(const PlanInputs &in, int pair, 
         const int seg = sc.wprefix[team >> 5] + __popc(sc.bitmap[team >> 5] & ((1u << (team & 31)) - 1u));
         atomicOr(&seg_mask[seg], 1u << h);
         g_logc[(size_t)seg * kMaxGroup + h] = kLog2e * sc.ent_logc[e];
-        const int r_lo = csr[team];
-        seg_row[seg] = (int32_t)(row0 + r_lo);                        // same value from every selecting head
-        sc.seg_rows[seg] = csr[team + 1] - r_lo;
+        seg_row[seg] = (int32_t)(row0 + sc.ent_rows[e].x);            // same value from every selecting head
+        sc.seg_rows[seg] = sc.ent_rows[e].y;
     }
     __syncthreads();
     {
