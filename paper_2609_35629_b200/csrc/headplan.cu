@@ -53,7 +53,7 @@ __device__ __forceinline__ float score_guard(double scale, double q_l1, float k_
 
 // The first half of the block's warps compute dot products, the second half the Gumbel terms.
 template <int kHeadThreads>
-__global__ void __launch_bounds__(kHeadThreads)
+__global__ void __launch_bounds__(kHeadThreads, 1024 / kHeadThreads)
 headplan_kernel(PlanInputs in)
 {
     constexpr int kHeadWarps = kHeadThreads / 32, kDotWarps = kHeadWarps / 2;
@@ -159,16 +159,25 @@ headplan_kernel(PlanInputs in)
     __syncthreads();
     const int n_blk = sm.n_blk;
     if (n_blk <= kCandCap) {
-        for (int it = tid; it < n_blk * 4; it += kHeadThreads) {     // (listed block, quarter of its 16 scores)
-            const int g0 = blk_list[it >> 2] * 16 + (it & 3) * 4;
-            float v[4];
+        // (listed block, quarter of its 16 scores) items, two per thread in flight
+        for (int it0 = tid; it0 < n_blk * 4; it0 += 2 * kHeadThreads) {
+            float v[2][4];
+            int g0[2];
 #pragma unroll
-            for (int i = 0; i < 4; ++i) v[i] = g0 + i < M ? __ldg(y32 + g0 + i) : -CUDART_INF_F;
+            for (int u = 0; u < 2; ++u) {
+                const int it = it0 + u * kHeadThreads;
+                g0[u] = it < n_blk * 4 ? blk_list[it >> 2] * 16 + (it & 3) * 4 : M;
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                if (g0 + i < M && v[i] >= t_lo) {
-                    const int slot = atomicAdd(&sm.n_cand, 1);
-                    if (slot < kCandCap) sm.cand_id[slot] = g0 + i;
+                for (int i = 0; i < 4; ++i) v[u][i] = g0[u] + i < M ? __ldg(y32 + g0[u] + i) : -CUDART_INF_F;
+            }
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    if (g0[u] + i < M && v[u][i] >= t_lo) {
+                        const int slot = atomicAdd(&sm.n_cand, 1);
+                        if (slot < kCandCap) sm.cand_id[slot] = g0[u] + i;
+                    }
                 }
             }
         }
@@ -195,12 +204,27 @@ headplan_kernel(PlanInputs in)
         if (warp < kDotWarps) {
             const int sub = lane & (kDotLanes - 1);
             const double *qs = sm.q64[sub];
-            for (int c0 = 0; c0 < n_cand; c0 += kDotWarps * 32 / kDotLanes) {
-                const int cand = c0 + (tid >> 3);
-                double d0 = 0.0, d1 = 0.0;
-                if (cand < n_cand) {
-                    const uint4 *kr = reinterpret_cast<const uint4 *>(rep + (size_t)sm.cand_id[cand] * kHeadDim) + sub * 2;
-                    const uint4 w0 = __ldg(kr), w1 = __ldg(kr + 1);
+            // four candidates per thread group at a time: all their key pieces are requested before
+            // the first product, so a chunk costs one memory round trip
+            constexpr int kPerPass = kDotWarps * 32 / kDotLanes, kChunk = 4;
+            for (int c0 = 0; c0 < n_cand; c0 += kPerPass * kChunk) {
+                uint4 w[kChunk][2];
+#pragma unroll
+                for (int u = 0; u < kChunk; ++u) {
+                    const int cand = c0 + u * kPerPass + (tid >> 3);
+                    if (cand < n_cand) {
+                        const uint4 *kr = reinterpret_cast<const uint4 *>(rep + (size_t)sm.cand_id[cand] * kHeadDim) + sub * 2;
+                        w[u][0] = __ldg(kr);
+                        w[u][1] = __ldg(kr + 1);
+                    } else {
+                        w[u][0] = w[u][1] = make_uint4(0u, 0u, 0u, 0u);
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < kChunk; ++u) {
+                    const int cand = c0 + u * kPerPass + (tid >> 3);
+                    const uint4 w0 = w[u][0], w1 = w[u][1];
+                    double d0 = 0.0, d1 = 0.0;
                     d0 = fma((double)bf16_lo(w0.x), qs[0], d0);
                     d1 = fma((double)bf16_hi(w0.x), qs[1], d1);
                     d0 = fma((double)bf16_lo(w0.y), qs[2], d0);
@@ -217,12 +241,12 @@ headplan_kernel(PlanInputs in)
                     d1 = fma((double)bf16_hi(w1.z), qs[13], d1);
                     d0 = fma((double)bf16_lo(w1.w), qs[14], d0);
                     d1 = fma((double)bf16_hi(w1.w), qs[15], d1);
+                    double d = d0 + d1;
+                    d += __shfl_xor_sync(0xFFFFFFFFu, d, 1);
+                    d += __shfl_xor_sync(0xFFFFFFFFu, d, 2);
+                    d += __shfl_xor_sync(0xFFFFFFFFu, d, 4);
+                    if (cand < n_cand && sub == 0) sm.cand_y[cand] = d;
                 }
-                double d = d0 + d1;
-                d += __shfl_xor_sync(0xFFFFFFFFu, d, 1);
-                d += __shfl_xor_sync(0xFFFFFFFFu, d, 2);
-                d += __shfl_xor_sync(0xFFFFFFFFu, d, 4);
-                if (cand < n_cand && sub == 0) sm.cand_y[cand] = d;
             }
         } else {
             for (int i = tid - kDotWarps * 32; i < n_cand; i += kHeadThreads - kDotWarps * 32) {
