@@ -146,7 +146,10 @@ attend_kernel(AttendParams p)
         for (int i = tid; i <= p.n_pairs; i += kAttendThreads) pair_prefix[i] = p.plan.pair_row_prefix[i];
         for (int i = tid; i < p.n_pairs; i += kAttendThreads) pair_nseg[i] = p.plan.pair_nseg[i];
         __syncthreads();
-        const int64_t total = pair_prefix[p.n_pairs];
+        // Rows of all pairs laid end to end, with a gap of span_penalty_rows after every pair: a CTA
+        // whose range crosses from one pair into the next pays the fixed cost of a second span
+        // (tables, pipeline refill, merge) out of its row budget, so ranges cost about equal time.
+        const int64_t total = pair_prefix[p.n_pairs] + (int64_t)p.span_penalty_rows * (p.n_pairs - 1);
         rows_per_cta = (total + gridDim.x - 1) / gridDim.x;
         if (rows_per_cta < p.min_rows_per_cta) rows_per_cta = p.min_rows_per_cta;
         r0 = (int64_t)blockIdx.x * rows_per_cta;
@@ -155,7 +158,7 @@ attend_kernel(AttendParams p)
         int lo = 0, hi = p.n_pairs;
         while (hi - lo > 1) {
             const int mid = (lo + hi) >> 1;
-            if (pair_prefix[mid] <= r0) lo = mid; else hi = mid;
+            if (pair_prefix[mid] + (int64_t)p.span_penalty_rows * mid <= r0) lo = mid; else hi = mid;
         }
         pair = lo;
     }
@@ -213,10 +216,17 @@ attend_kernel(AttendParams p)
                 continue;
             }
         } else {
-            pb = pair_prefix[pair];
-            pe = pair_prefix[pair + 1];
-            a = (int)(r0 - pb);
+            // this pair's rows occupy [pb, pe) of the padded row line
+            pb = pair_prefix[pair] + (int64_t)p.span_penalty_rows * pair;
+            pe = pb + (pair_prefix[pair + 1] - pair_prefix[pair]);
+            a = (int)(max(r0, pb) - pb);
             bnd = (int)(min(r1, pe) - pb);
+            if (a >= bnd) {                                // the range starts in the gap behind this pair
+                r0 = pe + p.span_penalty_rows;
+                if (r0 >= r1 || pair + 1 >= p.n_pairs) return;
+                ++pair;
+                continue;
+            }
             nseg = pair_nseg[pair];
             const int c_lo = (int)(pb / rows_per_cta), c_hi = (int)((pe - 1) / rows_per_cta);
             n_ctas = c_hi - c_lo + 1;
@@ -513,8 +523,9 @@ attend_kernel(AttendParams p)
             pair += gridDim.x;                             // more pairs than CTAs: whole pairs, round robin
             if (pair >= p.n_pairs) return;
         } else {
-            r0 = pb + bnd;
-            if (r0 >= r1) return;
+            if (pb + bnd < pe) return;                     // the range ended inside this pair
+            r0 = pe + p.span_penalty_rows;                 // first row of the next pair
+            if (r0 >= r1 || pair + 1 >= p.n_pairs) return;
             ++pair;
         }
     }

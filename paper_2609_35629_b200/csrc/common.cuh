@@ -112,6 +112,7 @@ struct AttendParams {
     float *out;                     // [n_seqs][n_q][128]
     int32_t *status;                // nullable
     int min_rows_per_cta;
+    int span_penalty_rows;          // equal-range split: rows a second span costs a CTA (see attend.cu)
     int ctas_per_pair;              // static split: CTAs that share one (sequence, KV head) pair
 };
 
