@@ -49,7 +49,7 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--layers", type=int, default=28)
     ap.add_argument("--workload", default="qwen7b_b1_32k",
-                    choices=["qwen7b_b1_32k", "qwen7b_b8_32k", "ragged", "long_128k", "small_gqa"])
+                    choices=["qwen7b_b1_32k", "qwen7b_b8_32k", "ragged", "long_128k", "paper_point_32k", "small_gqa"])
     ap.add_argument("--n-sample", type=int, default=0, help="override K")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -67,6 +67,8 @@ def make_spec(args, seed):
         spec = synth.spec_ragged(seed=seed)
     elif args.workload == "long_128k":
         spec = synth.spec_long(seed=seed)
+    elif args.workload == "paper_point_32k":
+        spec = synth.spec_paper_point(seed=seed)
     else:
         spec = synth.spec_small_gqa(seed=seed)
     if args.n_sample:

@@ -16,10 +16,9 @@ constexpr int kEntCap = 1024;           // G * K entries of a plan
 constexpr int kSegMax = 1025;           // segments of a plan (entries + suffix)
 constexpr int kBitmapWords = kMaxTeamsPerSeq / 32;
 
+constexpr int kEntPerThread = (kEntCap + kPlanThreads - 1) / kPlanThreads;   // entries a thread keeps in registers
+
 struct alignas(16) PlanScratch {
-    int ent_key[kEntCap];               // team * 8 + head
-    float ent_logc[kEntCap];
-    int2 ent_rows[kEntCap];             // first packed row (local to the sequence) and row count of the team
     uint32_t bitmap[kBitmapWords];
     int wprefix[kBitmapWords];
     int seg_rows[kSegMax];
@@ -84,56 +83,83 @@ __device__ __forceinline__ void build_pair_plan(const PlanInputs &in, int pair, 
         return;
     }
 
-    // ---- the heads' samples ----
-    for (int e = tid; e < G * Ke; e += kPlanThreads) {
-        const int h = e / Ke, a = e - h * Ke;
-        sc.ent_key[e] = in.sel_team[(head0 + h) * K + a] * kMaxGroup + h;
-        sc.ent_logc[e] = in.sel_logc[(head0 + h) * K + a];
-        sc.ent_rows[e] = in.sel_rows[(head0 + h) * K + a];
-    }
-    for (int i = tid; i < (M + 31) / 32; i += kPlanThreads) sc.bitmap[i] = 0u;
-    for (int i = tid; i <= G * Ke; i += kPlanThreads) seg_mask[i] = 0u;
-    __syncthreads();
+    // ---- the heads' samples: each thread keeps its entries in registers ----
     const int E = G * Ke;
-    for (int e = tid; e < E; e += kPlanThreads) {
-        const int team = sc.ent_key[e] >> 3;
-        atomicOr(&sc.bitmap[team >> 5], 1u << (team & 31));
+    const int n_words = (M + 31) / 32;
+    int ent_key[kEntPerThread];                                       // team * 8 + head, -1: none
+    float ent_logc[kEntPerThread];
+    int2 ent_rows[kEntPerThread];
+#pragma unroll
+    for (int u = 0; u < kEntPerThread; ++u) {
+        const int e = tid + u * kPlanThreads;
+        ent_key[u] = -1;
+        if (e < E) {
+            const int h = e / Ke, a = e - h * Ke;
+            const size_t at = (head0 + h) * K + a;
+            ent_key[u] = in.sel_team[at] * kMaxGroup + h;
+            ent_logc[u] = in.sel_logc[at];
+            ent_rows[u] = in.sel_rows[at];
+        }
+    }
+    for (int i = tid; i < n_words; i += kPlanThreads) sc.bitmap[i] = 0u;
+    for (int i = tid; i <= E; i += kPlanThreads) seg_mask[i] = 0u;
+    __syncthreads();
+#pragma unroll
+    for (int u = 0; u < kEntPerThread; ++u) {
+        if (ent_key[u] >= 0) {
+            const int team = ent_key[u] >> 3;
+            atomicOr(&sc.bitmap[team >> 5], 1u << (team & 31));
+        }
     }
     __syncthreads();
-    // word prefix of the bitmap -> segment index of a team = teams selected before it
-    {
-        const int n_words = (M + 31) / 32;
-        const int per = (n_words + kPlanThreads - 1) / kPlanThreads;
+    // word prefix of the bitmap (one warp): segment index of a team = selected teams before it
+    if (tid < 32) {
+        const int per = (n_words + 31) >> 5;
         const int lo = min(tid * per, n_words), hi = min(lo + per, n_words);
         int sum = 0;
         for (int w = lo; w < hi; ++w) sum += __popc(sc.bitmap[w]);
-        int total;
-        int run = block_exclusive_scan(sum, sc.scan, total);
+        int incl = sum;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+            if (tid >= o) incl += t;
+        }
+        int run = incl - sum;
         for (int w = lo; w < hi; ++w) { sc.wprefix[w] = run; run += __popc(sc.bitmap[w]); }
-        if (tid == 0) sc.misc[0] = total;                             // segments of the prompt
+        if (tid == 31) sc.misc[0] = incl;                             // segments of the prompt
     }
     __syncthreads();
     const int nseg_prompt = sc.misc[0];
-    for (int e = tid; e < E; e += kPlanThreads) {
-        const int team = sc.ent_key[e] >> 3, h = sc.ent_key[e] & 7;
-        const int seg = sc.wprefix[team >> 5] + __popc(sc.bitmap[team >> 5] & ((1u << (team & 31)) - 1u));
-        atomicOr(&seg_mask[seg], 1u << h);
-        g_logc[(size_t)seg * kMaxGroup + h] = kLog2e * sc.ent_logc[e];
-        seg_row[seg] = (int32_t)(row0 + sc.ent_rows[e].x);            // same value from every selecting head
-        sc.seg_rows[seg] = sc.ent_rows[e].y;
+#pragma unroll
+    for (int u = 0; u < kEntPerThread; ++u) {
+        if (ent_key[u] >= 0) {
+            const int team = ent_key[u] >> 3, h = ent_key[u] & 7;
+            const int seg = sc.wprefix[team >> 5] + __popc(sc.bitmap[team >> 5] & ((1u << (team & 31)) - 1u));
+            atomicOr(&seg_mask[seg], 1u << h);
+            g_logc[(size_t)seg * kMaxGroup + h] = kLog2e * ent_logc[u];
+            seg_row[seg] = (int32_t)(row0 + ent_rows[u].x);           // same value from every selecting head
+            sc.seg_rows[seg] = ent_rows[u].y;
+        }
     }
+    if (t_suffix > 0 && tid >= 32 && tid < 32 + kMaxGroup) g_logc[(size_t)nseg_prompt * kMaxGroup + (tid - 32)] = 0.f;
     __syncthreads();
-    {
-        const int per = (nseg_prompt + kPlanThreads - 1) / kPlanThreads;
+    // row prefix of the segments (one warp), then the suffix segment
+    if (tid < 32) {
+        const int per = (nseg_prompt + 31) >> 5;
         const int lo = min(tid * per, nseg_prompt), hi = min(lo + per, nseg_prompt);
         int sum = 0;
-        for (int s = lo; s < hi; ++s) sum += sc.seg_rows[s];
-        int total;
-        int run = block_exclusive_scan(sum, sc.scan, total);
-        for (int s = lo; s < hi; ++s) { seg_prefix[s] = run; run += sc.seg_rows[s]; }
-        if (tid == 0) {
-            int nseg = nseg_prompt, rows = total;
-            if (write_debug && in.dbg_union_rows) in.dbg_union_rows[pair] = total;
+        for (int sg = lo; sg < hi; ++sg) sum += sc.seg_rows[sg];
+        int incl = sum;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+            if (tid >= o) incl += t;
+        }
+        int run = incl - sum;
+        for (int sg = lo; sg < hi; ++sg) { seg_prefix[sg] = run; run += sc.seg_rows[sg]; }
+        if (tid == 31) {
+            int nseg = nseg_prompt, rows = incl;
+            if (write_debug && in.dbg_union_rows) in.dbg_union_rows[pair] = incl;
             if (t_suffix > 0) {
                 seg_prefix[nseg] = rows;
                 seg_row[nseg] = pair * in.suffix_cap;
@@ -145,7 +171,6 @@ __device__ __forceinline__ void build_pair_plan(const PlanInputs &in, int pair, 
             sc.misc[0] = nseg;
             sc.misc[1] = rows;
         }
-        if (t_suffix > 0 && tid < kMaxGroup) g_logc[(size_t)nseg_prompt * kMaxGroup + tid] = 0.f;
     }
     __threadfence_block();
     __syncthreads();

@@ -115,6 +115,12 @@ def spec_long(seed: int = 0, n_sample: int = 32, n_seqs: int = 4, prompt: int = 
                         16, [0] * n_seqs, 0, seed=seed)
 
 
+def spec_paper_point(seed: int = 0, n_steps: int = 256, prompt: int = 32768) -> WorkloadSpec:
+    """The paper's own operating point on the Qwen2.5-7B head layout: contiguous parents of 16 keys
+    with 4 representatives (about N / 4 teams of about 4 rows), 31 sampled teams, batch 1, no suffix."""
+    return WorkloadSpec("paper_point_32k", 1, 28, 4, [prompt], 2048, 16, 4, 31, n_steps, 16, [0], 0, seed=seed)
+
+
 def spec_small_gqa(seed: int = 0, n_seqs: int = 2, prompt=(1536, 1000), n_sample: int = 8,
                    parent_size: int = 128, reps: int = 8, n_steps: int = 3, suffix0=(5, 0)
                    ) -> WorkloadSpec:

@@ -227,6 +227,16 @@ def test_qwen_32k_full_size_batch1():
     check_dense_step(layer, 9)
 
 
+def test_paper_operating_point_32k():
+    """Parents of 16 keys with 4 representatives at 32K (8192 teams of about 4 rows per KV head),
+    31 sampled teams, no suffix: routing reads an eighth of the dense bytes, gathers are tiny."""
+    layer = layer_for("paper_point", synth.spec_paper_point)
+    check_team_records(layer, kv_heads=[1])
+    for step in (0, 9):
+        check_sparse_step(layer, step, K=31)
+    check_dense_step(layer, 2)
+
+
 def test_qwen_32k_batch8_concentrated_sampled_sequences():
     """Config 3 shape (8 sequences, 64 sampled teams, concentrated queries): the GPU runs the
     whole batch, the oracle checks two of the sequences."""
