@@ -104,8 +104,10 @@ struct Smem {
     static constexpr size_t total = misc + 64;
     // aliases of the ring: plan scratch before a pair's rows are streamed, merge scratch after
     static_assert(sizeof(PlanScratch) <= ring_bytes, "plan scratch must fit in the ring");
-    static constexpr size_t red_acc = ring;                                     // float [warps][G][128]
-    static constexpr size_t red_m = red_acc + (size_t)kWarps * G * kHeadDim * 4;   // float [warps][G]
+    static constexpr int red_pitch = kHeadDim + 4;                              // floats per (warp, head) row: the 4 extra
+                                                                                //   spread the heads of a store over the banks
+    static constexpr size_t red_acc = ring;                                     // float [warps][G][red_pitch]
+    static constexpr size_t red_m = red_acc + (size_t)kWarps * G * red_pitch * 4;  // float [warps][G]
     static constexpr size_t red_l = red_m + (size_t)kWarps * G * 4;
     static_assert(red_l + (size_t)kWarps * G * 4 <= ring_bytes, "merge scratch must fit in the ring");
     static constexpr int merge_chunk = (int)(ring_bytes / ((size_t)G * kPartialStride * 4));   // partials staged at once
@@ -419,7 +421,7 @@ attend_kernel(AttendParams p)
         __syncthreads();                                   // every block of the span is consumed
 
         // ---- merge the warps into one partial (the ring is free: reuse it) ----
-        float(*red_acc)[G][kHeadDim] = reinterpret_cast<float(*)[G][kHeadDim]>(smem + S::red_acc);
+        float(*red_acc)[G][S::red_pitch] = reinterpret_cast<float(*)[G][S::red_pitch]>(smem + S::red_acc);
         float(*red_m)[G] = reinterpret_cast<float(*)[G]>(smem + S::red_m);
         float(*red_l)[G] = reinterpret_cast<float(*)[G]>(smem + S::red_l);
         l_run += __shfl_xor_sync(0xFFFFFFFFu, l_run, 1);
@@ -436,24 +438,30 @@ attend_kernel(AttendParams p)
             }
         }
         __syncthreads();
+        // thread (h, lane) merges four output columns of head h over the warps
         float *part = p.partials + (size_t)slot_id * G * kPartialStride;
-        for (int e = tid; e < G * kHeadDim; e += kAttendThreads) {
-            const int h = e >> 7, d = e & 127;
+        if (warp < G) {
+            const int h = warp;
             float mh = -CUDART_INF_F;
 #pragma unroll
             for (int w = 0; w < kWarps; ++w) mh = fmaxf(mh, red_m[w][h]);
-            float num = 0.f, den = 0.f;
+            float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
+            float den = 0.f;
 #pragma unroll
             for (int w = 0; w < kWarps; ++w) {
                 const float mw = red_m[w][h];
                 if (mw > -CUDART_INF_F) {                  // warps without rows for this head left no data
                     const float f = exp2f(mw - mh);
-                    num = fmaf(f, red_acc[w][h][d], num);
+                    const float4 v = *reinterpret_cast<const float4 *>(&red_acc[w][h][4 * lane]);
+                    num.x = fmaf(f, v.x, num.x);
+                    num.y = fmaf(f, v.y, num.y);
+                    num.z = fmaf(f, v.z, num.z);
+                    num.w = fmaf(f, v.w, num.w);
                     den = fmaf(f, red_l[w][h], den);
                 }
             }
-            part[h * kPartialStride + 4 + d] = num;
-            if (d == 0) { part[h * kPartialStride] = mh; part[h * kPartialStride + 1] = den; }
+            *reinterpret_cast<float4 *>(part + h * kPartialStride + 4 + 4 * lane) = num;
+            if (lane == 0) { part[h * kPartialStride] = mh; part[h * kPartialStride + 1] = den; }
         }
 
         // ---- last CTA of the pair: log-sum-exp merge of the pair's partials ----
