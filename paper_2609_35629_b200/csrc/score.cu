@@ -52,13 +52,13 @@ constexpr int kScoreRingBytes = kScoreKeyRingBytes + kScoreStages * (kScoreThrea
 // (1e-10, 23) where the fast logarithm is accurate to 3 ulp or 2^-21.4 absolute.
 __device__ __forceinline__ float gumbel32_from_word(uint32_t x)
 {
-    float nl;
-    if (x >= 0x80000000u) {
-        const float z = ((float)(0xFFFFFFFFu - x) + 0.5f) * 2.3283064365386963e-10f;
-        nl = z < 0.015625f ? z * (1.f + z * (0.5f + z * (0.33333334f + z * 0.25f))) : -__logf(1.f - z);
-    } else {
-        nl = -__logf(((float)x + 0.5f) * 2.3283064365386963e-10f);
-    }
+    // straight-line: both halves are evaluated and one is selected, so lanes never diverge
+    const bool upper = x >= 0x80000000u;
+    const float u = ((float)x + 0.5f) * 2.3283064365386963e-10f;
+    const float z = ((float)(~x) + 0.5f) * 2.3283064365386963e-10f;      // 1 - u
+    const float by_log = -__logf(upper ? 1.f - z : u);
+    const float by_series = z * (1.f + z * (0.5f + z * (0.33333334f + z * 0.25f)));
+    const float nl = (upper && z < 0.015625f) ? by_series : by_log;
     return -__logf(nl);
 }
 
