@@ -115,7 +115,9 @@ typedef struct santapp_debug {
     int32_t *union_rows;       /* int32 [n_seqs][n_kv_heads]: distinct prompt rows read (u_c of the
                                   logical-access counter)                                            */
     int32_t *status;           /* int32 [1]: bit flags raised on the device (0 = clean);
-                                  bit 0: non-finite output                                           */
+                                  bit 0: non-finite output; bit 1: a head had fewer than K + 1
+                                  comparable routing scores (non-finite q or keys): its sample was
+                                  completed with arbitrary teams, the output is meaningless        */
 } santapp_debug;
 
 /* Library version: major * 10000 + minor * 100 + patch. */

@@ -318,6 +318,7 @@ int santapp_decode_attn(const santapp_geom *geom, const santapp_teams *teams, co
     pp.in.sel_team = reinterpret_cast<int32_t *>(ws + L.sel_team);
     pp.in.sel_logc = reinterpret_cast<float *>(ws + L.sel_logc);
     pp.in.sel_rows = reinterpret_cast<int2 *>(ws + L.sel_rows);
+    pp.in.status = dbg ? dbg->status : nullptr;
     pp.in.dbg_sel_idx = dbg ? dbg->sel_idx : nullptr;
     pp.in.dbg_sel_logc = dbg ? dbg->sel_logc : nullptr;
     pp.in.dbg_tau = dbg ? dbg->tau : nullptr;

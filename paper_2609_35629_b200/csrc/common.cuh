@@ -85,6 +85,7 @@ struct PlanInputs {
     float *sel_logc;                // [n_seqs][n_q][n_sample] log c_g of each
     int2 *sel_rows;                 // [n_seqs][n_q][n_sample] first packed row (local to the sequence), row count
     // diagnostics (nullable)
+    int32_t *status;
     int32_t *dbg_sel_idx;
     float *dbg_sel_logc;
     double *dbg_tau;

@@ -311,14 +311,29 @@ headplan_kernel(PlanInputs in)
     }
 
     // ---- 4. corrections ----
-    const double tau = sm.list_y[cur][K];
+    // Fewer than K + 1 ranked teams can only mean scores that do not compare (non-finite inputs):
+    // the sample is completed with the first teams so that every index handed on is valid, and
+    // the status word says so.
+    const bool short_list = n_list < K + 1;
+    const double tau = short_list ? __longlong_as_double(0x7FF8000000000000ll) : sm.list_y[cur][K];
+    if (short_list && tid == 0 && in.status) atomicOr(in.status, 2);
     for (int a = tid; a < K; a += kHeadThreads) {
-        const double c = -expm1(-exp(sm.list_phi[cur][a] - tau));         // 1 - exp(-exp(phi - tau))
-        const float logc = (float)log(c);
-        const int id = sm.list_id[cur][a];
+        int id;
+        float logc;
+        int2 rows;
+        if (a < n_list && !short_list) {
+            const double c = -expm1(-exp(sm.list_phi[cur][a] - tau));     // 1 - exp(-exp(phi - tau))
+            logc = (float)log(c);
+            id = sm.list_id[cur][a];
+            rows = sm.list_rows[cur][a];
+        } else {
+            id = a;                                                       // K < M: a valid team
+            logc = 0.f;
+            rows = make_int2(csr[a], csr[a + 1] - csr[a]);
+        }
         in.sel_team[(size_t)hq * K + a] = id;
         in.sel_logc[(size_t)hq * K + a] = logc;
-        in.sel_rows[(size_t)hq * K + a] = sm.list_rows[cur][a];
+        in.sel_rows[(size_t)hq * K + a] = rows;
         if (in.dbg_sel_idx) in.dbg_sel_idx[(size_t)hq * K + a] = id;
         if (in.dbg_sel_logc) in.dbg_sel_logc[(size_t)hq * K + a] = logc;
     }

@@ -311,6 +311,27 @@ def test_decode_many_short_sequences():
     check_dense_step(layer, 0)
 
 
+def test_non_finite_query_raises_status_bits_and_leaves_the_library_usable():
+    """A NaN query makes every routing score of its head incomparable: the call must finish, say so
+    in the status word (bit 1: sample completed arbitrarily; bit 0: non-finite output), hand on only
+    valid team ids, and the next clean call must be unaffected."""
+    layer = layer_for("small", synth.spec_small_gqa)
+    spec = layer.spec
+    q_bits = synth.make_queries(spec, layer.data, 0).copy()
+    q_bits[0, 3, :] = 0x7FC0                                          # bf16 NaN in every dim of one head
+    sl = spec.suffix_len(0)
+    out, dbg = pu.gpu_step(layer, q_bits, sl, 8, 5, 0)
+    status = int(dbg.status.item())
+    assert status & 2 and status & 1
+    sel = dbg.sel_idx.cpu().numpy()
+    Ms = np.diff(layer.seq_team_off)
+    for b in range(spec.n_seqs):
+        assert sel[b].min() >= 0 and sel[b].max() < Ms[b]
+    assert np.isnan(out[0, 3]).all()
+    assert np.isfinite(out[1]).all()                                  # other sequences are untouched
+    check_sparse_step(layer, 0, K=8)                                  # and a clean call still matches the oracle
+
+
 def test_device_side_step_offset_equals_explicit_step():
     """step = 3 with a device-side offset of 4 draws the same sample as step = 7."""
     layer = layer_for("small", synth.spec_small_gqa)
