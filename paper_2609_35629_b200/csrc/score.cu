@@ -41,7 +41,9 @@ __device__ __forceinline__ void cp_async_wait_group()
 
 constexpr int kScoreStages = 3;                                 // tiles in flight per warp (pipelined variant)
 constexpr int kScoreKeyRingBytes = kScoreStages * (kScoreThreads / 32) * 4096;
-constexpr int kScoreRingBytes = kScoreKeyRingBytes + kScoreStages * (kScoreThreads / 32) * 128;   // + row offsets
+constexpr int kScoreCsrRingBytes = kScoreStages * (kScoreThreads / 32) * 128;                       // row offsets
+constexpr int kSeqTableCap = 2048;                              // sequences whose first tile slot is kept in shared memory
+constexpr int kScoreRingBytes = kScoreKeyRingBytes + kScoreCsrRingBytes + (kSeqTableCap + 1) * 4;
 
 // Gumbel(0,1) in fp32 from a 32-bit word: u = (x + 0.5) / 2^32, G = -log(-log u), to an absolute
 // error well inside the additive term of the guard (see score_guard in pairplan.cuh).
@@ -205,14 +207,17 @@ __device__ __forceinline__ TileCursor cursor_at(const ScoreParams &p, long long 
 }
 
 // Tile under the cursor: true with its first team in `base` when it has teams to score.
-__device__ __forceinline__ bool locate_tile(const ScoreParams &p, TileCursor &cur, int &base)
+// seq_slot: first slot of every sequence in shared memory (nullptr: read the offsets from global
+// memory instead, for batches beyond kSeqTableCap).
+__device__ __forceinline__ bool locate_tile(const ScoreParams &p, const int *seq_slot, TileCursor &cur, int &base)
 {
     const int s = cur.s;
     if (s < cur.slot_lo || s >= cur.slot_hi) {
         int lo = 0, hi = p.bv.n_seqs - 1;              // largest b with start(b) <= s
         while (lo < hi) {
             const int mid = (lo + hi + 1) >> 1;
-            if ((int)(p.bv.seq_team_off[mid] >> 4) + mid <= s) lo = mid; else hi = mid - 1;
+            const int start = seq_slot ? seq_slot[mid] : (int)(p.bv.seq_team_off[mid] >> 4) + mid;
+            if (start <= s) lo = mid; else hi = mid - 1;
         }
         cur.b = lo;
         cur.team0 = p.bv.seq_team_off[lo];
@@ -254,11 +259,20 @@ score32_flat_kernel(ScoreParams p)
     // the tile's 17 row offsets, copied by lanes 0..16: [warp][s][32]
     int32_t *csr_ring = reinterpret_cast<int32_t *>(reinterpret_cast<unsigned char *>(score_ring) + kScoreKeyRingBytes)
                         + warp * kScoreStages * 32;
+    // first slot of every sequence, for the searches of locate_tile
+    int *seq_slot = reinterpret_cast<int *>(reinterpret_cast<unsigned char *>(score_ring) + kScoreKeyRingBytes
+                                            + kScoreCsrRingBytes);
+    if (p.bv.n_seqs <= kSeqTableCap) {
+        for (int i = tid; i < p.bv.n_seqs; i += kScoreThreads) seq_slot[i] = (int)(p.bv.seq_team_off[i] >> 4) + i;
+        __syncthreads();
+    } else {
+        seq_slot = nullptr;
+    }
     TileCursor ahead = cursor_at(p, t_lo), here = ahead;
     long long t_ahead = t_lo;                                   // tile index under `ahead`
     auto issue_tile = [&](int s) {
         int base;
-        if (t_ahead < t_hi && locate_tile(p, ahead, base)) {
+        if (t_ahead < t_hi && locate_tile(p, seq_slot, ahead, base)) {
             const uint16_t *rep = p.rep_keys + ((size_t)ahead.j * p.bv.teams_total + ahead.team0) * kHeadDim;
 #pragma unroll
             for (int t = 0; t < 2; ++t) {
@@ -287,7 +301,7 @@ score32_flat_kernel(ScoreParams p)
         cp_async_wait_group<kScoreStages - 1>();                 // this lane's pieces of tile ti have landed
         __syncwarp();                                            // the row offsets come from other lanes
         int base;
-        if (locate_tile(p, here, base)) {
+        if (locate_tile(p, seq_slot, here, base)) {
             if (here.b != q_b || here.j != q_j) {
                 load_q_fragments<G>(p, here.b, here.j, g, c, qa);
                 q_b = here.b;
