@@ -311,6 +311,17 @@ def test_decode_many_short_sequences():
     check_dense_step(layer, 0)
 
 
+@pytest.mark.parametrize("n_q,n_kv", [(32, 4), (8, 2), (6, 6), (3, 1)])
+def test_decode_other_group_sizes(n_q, n_kv):
+    """GQA groups of 8, 4, 1 and 3 query heads per KV head (the tensor-core tile holds up to 8)."""
+    import dataclasses
+    spec = dataclasses.replace(synth.spec_small_gqa(prompt=(1100, 640)), n_q_heads=n_q, n_kv_heads=n_kv)
+    layer = pu.GpuLayer(spec, synth.make_layer(spec))
+    check_sparse_step(layer, 0, K=8)
+    check_sparse_step(layer, 1, K=33)
+    check_dense_step(layer, 0)
+
+
 def test_non_finite_query_raises_status_bits_and_leaves_the_library_usable():
     """A NaN query makes every routing score of its head incomparable: the call must finish, say so
     in the status word (bit 1: sample completed arbitrarily; bit 0: non-finite output), hand on only
