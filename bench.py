@@ -503,9 +503,40 @@ def cpu_baseline_leg(spec, data, teams, seed):
         times.append(time.perf_counter() - s0)
         n += 1
     us = 1e6 * float(np.mean(times[1:] if len(times) > 1 else times))
+
+    # beside it, a few layer-steps each of: the oracle on one thread, and the oracle's dense
+    # attention (all prompt rows) on all cores and on one thread
+    def few(fn, reps):
+        took = []
+        for i in range(reps):
+            s0 = time.perf_counter()
+            fn(i)
+            took.append(time.perf_counter() - s0)
+        return 1e6 * float(np.mean(took))
+
+    def inputs(i):
+        step = i % spec.n_steps
+        q = synth.bf16_to_f64(synth.make_queries(spec, data, step % N_STEP_INPUTS)[b])
+        t = int(spec.suffix_len(step)[b])
+        ks = synth.bf16_to_f64(data.k_suffix[b, :, :t]) if t else None
+        vs = synth.bf16_to_f64(data.v_suffix[b, :, :t]) if t else None
+        return q, ks, vs, step
+
+    def sparse_1(i):
+        q, ks, vs, step = inputs(i)
+        orc.decode_step(q, k, v, M, ts, tm, rk, ks, vs, spec.n_sample, seed, step, b, scale, n_threads=1)
+
+    def dense_n(threads):
+        def run(i):
+            q, ks, vs, _ = inputs(i)
+            orc.dense_step(q, k, v, ks, vs, scale, n_threads=threads)
+        return run
+
+    extra = {"sparse_1_thread_us": few(sparse_1, 3), "dense_all_cores_us": few(dense_n(cores), 5),
+             "dense_1_thread_us": few(dense_n(1), 2)}
     return {"value": us, "unit": UNIT, "cores": cores, "kind": "oracle",
             "sample": f"{n} layer-steps of sequence 0, layer 0 ({spec.n_q_heads} heads, {r1 - r0} prompt rows), "
-                      f"fp64 oracle with OpenMP over heads"}
+                      f"fp64 oracle with OpenMP over heads", **extra}
 
 
 def main():
