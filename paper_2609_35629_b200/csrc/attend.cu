@@ -170,6 +170,18 @@ attend_kernel(AttendParams p)
         int64_t pb = 0, pe = 0;
         const int b = pair / p.bv.n_kv, j = pair - b * p.bv.n_kv;
         const float *g_logc = p.plan.seg_logc + (size_t)pair * cap * kMaxGroup;
+        // A fragments of q for the 8 k-steps: head g (zero rows for g >= G and for M rows 8..15);
+        // requested first, so that they arrive while the plan is being set up
+        uint32_t qa[8][2];
+        {
+            const uint32_t *qrow = reinterpret_cast<const uint32_t *>(
+                p.q + ((size_t)b * p.bv.n_q + (size_t)j * G + (g < G ? g : 0)) * kHeadDim);
+#pragma unroll
+            for (int s = 0; s < 8; ++s) {
+                qa[s][0] = g < G ? __ldg(qrow + 8 * s + c) : 0u;
+                qa[s][1] = g < G ? __ldg(qrow + 8 * s + 4 + c) : 0u;
+            }
+        }
 
         if (kStatic) {
             int rows;
@@ -247,17 +259,6 @@ attend_kernel(AttendParams p)
                 if (i < nseg) { v_row = g_row[i]; v_mask = g_mask[i]; }
                 if (i <= nseg) seg_prefix[i] = v_prefix;
                 if (i < nseg) { seg_row[i] = v_row; seg_mask[i] = v_mask; }
-            }
-        }
-        // A fragments of q for the 8 k-steps: head g (zero rows for g >= G and for M rows 8..15)
-        uint32_t qa[8][2];
-        {
-            const uint32_t *qrow = reinterpret_cast<const uint32_t *>(
-                p.q + ((size_t)b * p.bv.n_q + (size_t)j * G + (g < G ? g : 0)) * kHeadDim);
-#pragma unroll
-            for (int s = 0; s < 8; ++s) {
-                qa[s][0] = g < G ? __ldg(qrow + 8 * s + c) : 0u;
-                qa[s][1] = g < G ? __ldg(qrow + 8 * s + 4 + c) : 0u;
             }
         }
         __syncthreads();

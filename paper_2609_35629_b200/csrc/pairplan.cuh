@@ -35,17 +35,36 @@ __device__ __forceinline__ void build_pair_plan(const PlanInputs &in, int pair, 
 {
     const int tid = threadIdx.x;
     const int b = pair / in.bv.n_kv, j = pair - b * in.bv.n_kv;
+    const int K = in.n_sample;
+    const size_t head0 = (size_t)b * in.bv.n_q + (size_t)j * G;       // first query head of the pair
+    // The heads' samples, requested before anything else so that they travel together with the
+    // sequence offsets: each thread keeps its entries in registers. (When every team is read,
+    // K >= M, nothing was sampled and the values are not used.)
+    int ent_team[kEntPerThread];
+    float ent_logc[kEntPerThread];
+    int2 ent_rows[kEntPerThread];
+#pragma unroll
+    for (int u = 0; u < kEntPerThread; ++u) {
+        const int e = tid + u * kPlanThreads;
+        ent_team[u] = 0;
+        ent_logc[u] = 0.f;
+        ent_rows[u] = make_int2(0, 0);
+        if (e < G * K) {                                              // entry e: head e / K, rank e % K
+            const size_t at = head0 * K + e;
+            ent_team[u] = in.sel_team[at];
+            ent_logc[u] = in.sel_logc[at];
+            ent_rows[u] = in.sel_rows[at];
+        }
+    }
     const int64_t team0 = in.bv.seq_team_off[b];
     const int M = (int)(in.bv.seq_team_off[b + 1] - team0);
     const int64_t row0 = in.bv.seq_row_off[b];
     const int N = (int)(in.bv.seq_row_off[b + 1] - row0);
-    const int K = in.n_sample;
     const int Ke = min(K, M);
     int t_suffix = 0;
     if (in.suffix_len != nullptr && in.suffix_cap > 0) t_suffix = max(0, min(in.suffix_len[b], in.suffix_cap));
     const uint32_t all_heads = (1u << G) - 1u;
     const float kLog2e = 1.4426950408889634f;
-    const size_t head0 = (size_t)b * in.bv.n_q + (size_t)j * G;       // first query head of the pair
 
     __syncthreads();                                                  // scratch and tables are free
     if (Ke == M) {
@@ -83,23 +102,14 @@ __device__ __forceinline__ void build_pair_plan(const PlanInputs &in, int pair, 
         return;
     }
 
-    // ---- the heads' samples: each thread keeps its entries in registers ----
-    const int E = G * Ke;
+    // ---- here K < M, so every head has exactly K sampled teams ----
+    const int E = G * K;
     const int n_words = (M + 31) / 32;
     int ent_key[kEntPerThread];                                       // team * 8 + head, -1: none
-    float ent_logc[kEntPerThread];
-    int2 ent_rows[kEntPerThread];
 #pragma unroll
     for (int u = 0; u < kEntPerThread; ++u) {
         const int e = tid + u * kPlanThreads;
-        ent_key[u] = -1;
-        if (e < E) {
-            const int h = e / Ke, a = e - h * Ke;
-            const size_t at = (head0 + h) * K + a;
-            ent_key[u] = in.sel_team[at] * kMaxGroup + h;
-            ent_logc[u] = in.sel_logc[at];
-            ent_rows[u] = in.sel_rows[at];
-        }
+        ent_key[u] = e < E ? ent_team[u] * kMaxGroup + e / K : -1;
     }
     for (int i = tid; i < n_words; i += kPlanThreads) sc.bitmap[i] = 0u;
     for (int i = tid; i <= E; i += kPlanThreads) seg_mask[i] = 0u;
