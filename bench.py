@@ -534,6 +534,15 @@ def cpu_baseline_leg(spec, data, teams, seed):
 
     extra = {"sparse_1_thread_us": few(sparse_1, 3), "dense_all_cores_us": few(dense_n(cores), 5),
              "dense_1_thread_us": few(dense_n(1), 2)}
+    # routing agreement with dense attention over the prompt (Eq. diagnostic-kl), no sampling involved:
+    # mean over the heads of two of the step inputs
+    kls = []
+    for i in range(2):
+        q, _, _, _ = inputs(i * 100)
+        for h in range(spec.n_q_heads):
+            j = h // spec.group
+            kls.append(orc.routing_kl(q[h], k[j], ts[j], tm[j], rk[j], scale))
+    extra["routing_kl_nats_mean"] = float(np.mean(kls))
     return {"value": us, "unit": UNIT, "cores": cores, "kind": "oracle",
             "sample": f"{n} layer-steps of sequence 0, layer 0 ({spec.n_q_heads} heads, {r1 - r0} prompt rows), "
                       f"fp64 oracle with OpenMP over heads", **extra}

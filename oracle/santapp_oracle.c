@@ -23,6 +23,7 @@
  *                             reading and are documented with the function)
  *   orc_logical_access_*      logical KV-access counter, Eq. (qwen-logical-access)
  *   orc_team_budget           selected-team count, Eq. (method-budget)
+ *   orc_routing_kl            routing-agreement diagnostic, Eq. (diagnostic-kl)
  *
  * Parity pins (tests marked "not gpu"): Philox words against an independent
  * library generator; Gumbel law by Kolmogorov-Smirnov and moments; first-draw
@@ -31,7 +32,9 @@
  * successive-sampling law and against 1e5-draw frequencies; unbiasedness of
  * the two unnormalised sums by quadrature and Monte Carlo; Algorithm 2 on
  * hand-worked parents and duplicate keys; the accounting helpers against the
- * figures the paper prints.
+ * figures the paper prints; the routing KL against its closed forms (zero for
+ * singleton teams, log N - H(p) for one team holding every key) and against a
+ * numpy re-evaluation of the defining sum.
  * Parity unpinned: nothing in this file. (Accuracy of the sampled output
  * against dense attention on real model data is outside what can be pinned
  * here; only the estimator identities are.)
@@ -539,4 +542,50 @@ int64_t orc_union_rows(int32_t M, const int32_t *team_start, int32_t n_heads, in
 double orc_dense_kv_bytes(int64_t N, int32_t n_kv, int32_t d, int32_t bytes_per_el)
 {
     return 2.0 * (double)n_kv * (double)N * (double)d * (double)bytes_per_el;
+}
+
+/* Eq. (diagnostic-kl): agreement of the routing proposal with dense attention over
+ * the N prompt tokens, for one query head; no sampling is involved.
+ *   p_i  = dense attention weight of token i among the prompt tokens (softmax of
+ *          q.k_i * scale over i = 1..N),
+ *   P(g) = softmax over teams of log n_g + q.l_g * scale (l_g the routing key),
+ *   q_i  = P(g(i)) / n_g(i)  (a team's probability spread equally over its members),
+ *   KL(p || q) = sum_i p_i log(p_i / q_i), natural logarithm (nats).
+ * Tokens with p_i = 0 in floating point contribute 0 (the limit of x log x).
+ * team_start[M+1], team_member[N] (members of team g are team_member[team_start[g] ..
+ * team_start[g+1])), rep_key[M][d]. */
+double orc_routing_kl(int d, const double *q, int64_t N, const double *k, int32_t M,
+                      const int32_t *team_start, const int32_t *team_member,
+                      const double *rep_key, double scale)
+{
+    double *s = (double *)malloc(sizeof(double) * (size_t)N);
+    double *phi = (double *)malloc(sizeof(double) * (size_t)M);
+    double smax = -INFINITY, pmax = -INFINITY;
+    for (int64_t i = 0; i < N; ++i) {
+        s[i] = dot(q, k + i * d, d) * scale;
+        if (s[i] > smax) smax = s[i];
+    }
+    for (int32_t g = 0; g < M; ++g) {
+        int32_t n_g = team_start[g + 1] - team_start[g];
+        phi[g] = log((double)n_g) + dot(q, rep_key + (int64_t)g * d, d) * scale;
+        if (phi[g] > pmax) pmax = phi[g];
+    }
+    double Z = 0.0, Zr = 0.0;
+    for (int64_t i = 0; i < N; ++i) Z += exp(s[i] - smax);
+    for (int32_t g = 0; g < M; ++g) Zr += exp(phi[g] - pmax);
+    double kl = 0.0;
+    for (int32_t g = 0; g < M; ++g) {
+        int32_t n_g = team_start[g + 1] - team_start[g];
+        /* log q_i for the members of g */
+        double log_q = (phi[g] - pmax) - log(Zr) - log((double)n_g);
+        for (int32_t a = team_start[g]; a < team_start[g + 1]; ++a) {
+            int64_t i = team_member[a];
+            double log_p = (s[i] - smax) - log(Z);
+            double p = exp(log_p);
+            if (p > 0.0) kl += p * (log_p - log_q);
+        }
+    }
+    free(s);
+    free(phi);
+    return kl;
 }

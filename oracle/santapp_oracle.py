@@ -81,6 +81,8 @@ def lib():
         L.orc_union_rows.restype = _c.c_int64
         L.orc_dense_kv_bytes.argtypes = [_c.c_int64, _c.c_int32, _c.c_int32, _c.c_int32]
         L.orc_dense_kv_bytes.restype = _c.c_double
+        L.orc_routing_kl.argtypes = [_c.c_int, _f64p, _c.c_int64, _f64p, _c.c_int32, _i32p, _i32p, _f64p, _c.c_double]
+        L.orc_routing_kl.restype = _c.c_double
         _lib = L
     return _lib
 
@@ -299,3 +301,12 @@ def union_rows(team_start, sel):
 
 def dense_kv_bytes(N, n_kv, d, bytes_per_el):
     return float(lib().orc_dense_kv_bytes(N, n_kv, d, bytes_per_el))
+
+
+def routing_kl(q, k, team_start, team_member, rep_key, scale):
+    """KL(p || q) in nats between dense attention over the prompt and the routing proposal spread
+    over team members (Eq. diagnostic-kl), for one query head."""
+    q, k, rep_key = _f64(q), _f64(k), _f64(rep_key)
+    team_start, team_member = _i32(team_start), _i32(team_member)
+    return float(lib().orc_routing_kl(q.shape[0], q, k.shape[0], k, team_start.shape[0] - 1, team_start,
+                                      team_member, rep_key, scale))
