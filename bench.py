@@ -37,7 +37,7 @@ N_STEP_INPUTS = 8          # distinct (query, suffix length, step) inputs cycled
 # DRAM bytes (read + write) of one attend_kernel launch from an ncu capture of the same per-launch
 # work (summaries under profiles/, named for the kernel and workload); None where none was taken.
 NCU_TRAFFIC_BYTES = {
-    "qwen7b_b1_32k": 34.51e6,      # profiles/attend_kernel_qwen7b_b1_32k.md
+    "qwen7b_b1_32k": 34.61e6,      # profiles/attend_kernel_qwen7b_b1_32k.md (mean of two launches)
 }
 
 
