@@ -12,7 +12,9 @@ visited round-robin so that every layer-step reads K/V from HBM, not from L2 (28
 Prints ONE JSON line (rank 0). `value` is microseconds per layer-step with all inputs resident
 in HBM, replayed from CUDA graphs; `e2e` is the same through host buffers (pinned host to
 device copies of the step's queries, new suffix rows and counters, device to host read of the
-outputs, inside the timed region).
+outputs, inside the timed region). With the default workload the line also carries `batched`:
+the same measurement on the ragged 32-sequence batch (two layers, a few steps), the size at which
+the operator is bandwidth-bound rather than latency-bound (`--no-batched` skips it).
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--layers L]
 """
@@ -54,6 +56,7 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-stages", action="store_true")
+    ap.add_argument("--no-batched", action="store_true", help="skip the extra bandwidth-bound workload")
     return ap.parse_args()
 
 
@@ -204,7 +207,7 @@ def run_ours(args):
     import torch
     import torch.distributed as dist
     from paper_2609_35629_b200 import binding as sp
-    from paper_2609_35629_b200 import replicas, synth
+    from paper_2609_35629_b200 import replicas
 
     rank, world, local_rank = replicas.env_rank_world()
     if not torch.cuda.is_available():
@@ -214,9 +217,37 @@ def run_ours(args):
     replicas.init_replicas("nccl", dev)
     sp.load_library()
 
+    line = measure_workload(args, args.workload, args.layers, args.steps, args.warmup, dev,
+                            want_e2e=not args.no_e2e, want_cpu=not args.no_cpu_baseline, want_stages=not args.no_stages)
+    # Beside the headline workload (batch 1, latency-bound on this GPU), the same measurement on a
+    # batch large enough to be bandwidth-bound: the ragged serving batch, two layers.
+    if args.workload == "qwen7b_b1_32k" and not args.no_batched and not args.n_sample:
+        import gc
+        gc.collect()
+        torch.cuda.empty_cache()
+        big = measure_workload(args, "ragged", 2, 10, 3, dev, want_e2e=False, want_cpu=False, want_stages=True)
+        if rank == 0:
+            keep = ("value", "unit", "dense_us_per_layer_step", "speedup_vs_dense", "read_reduction",
+                    "achieved_frac_of_peak", "dense_achieved_frac_of_peak", "roofline", "stage_us", "steps", "warmup")
+            line["batched"] = {"workload": big["config"]["workload"], **{k: big[k] for k in keep}}
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def measure_workload(args, workload, n_layers, n_steps, n_warmup, dev, want_e2e, want_cpu, want_stages):
+    """One workload end to end: inputs, team build, graphs, timed runs. Returns the JSON line as a
+    dict on rank 0 (None elsewhere)."""
+    import torch
+    from paper_2609_35629_b200 import binding as sp
+    from paper_2609_35629_b200 import replicas, synth
+
+    rank, world, local_rank = replicas.env_rank_world()
+    wl_args = argparse.Namespace(**{**vars(args), "workload": workload})
     # Independent replicas: every rank owns its own sequences (seed = rank); no exchange.
-    spec = make_spec(args, seed=replicas.replica_seed(0, rank))
-    L = args.layers
+    spec = make_spec(wl_args, seed=replicas.replica_seed(0, rank))
+    L = n_layers
     geom = sp.Geometry(spec.n_seqs, spec.n_q_heads, spec.n_kv_heads, spec.head_dim, spec.parent_size,
                        spec.reps_per_parent)
     K = spec.n_sample
@@ -350,7 +381,7 @@ def run_ours(args):
         set_inputs(i % N_STEP_INPUTS)
         g_dense.replay()
 
-    Kst, W = args.steps, max(args.warmup, 3)
+    Kst, W = n_steps, max(n_warmup, 3)
     sampler = ClockSampler(local_rank)
     ms_sparse = timed(sparse_step, Kst, W, sampler)
     clocks = sampler.summary()
@@ -376,7 +407,7 @@ def run_ours(args):
     # ---- isolated stages (graphs of one stage over all layers; plans and scores left in the
     # per-layer workspaces by a full step with the same inputs) ----
     stages = {}
-    if not args.no_stages:
+    if want_stages:
         set_inputs(1)
         g_sparse.replay()
         torch.cuda.synchronize()
@@ -407,7 +438,7 @@ def run_ours(args):
 
     # ---- end to end through host buffers ----
     e2e = None
-    if not args.no_e2e:
+    if want_e2e:
         new_rows = torch.zeros((N_STEP_INPUTS, 2, B, L, Hkv, d), dtype=torch.bfloat16).pin_memory()
         for s in range(N_STEP_INPUTS):
             for b in range(B):
@@ -437,7 +468,7 @@ def run_ours(args):
 
     # ---- the oracle on the host cores, bounded sample ----
     cpu_baseline = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    if rank == 0 and world == 1 and want_cpu:
         cpu_baseline = cpu_baseline_leg(spec, host_layers[0], layers[0]["teams"], seed)
 
     if rank == 0:
@@ -463,9 +494,8 @@ def run_ours(args):
                                                 / (2 * (Hkv * N_total + suffix_rows[used].mean()))),
             "stage_us": stages, "prep_seconds": prep_s,
         }
-        print(json.dumps(line), flush=True)
-    if world > 1:
-        dist.destroy_process_group()
+        return line
+    return None
 
 
 def cpu_baseline_leg(spec, data, teams, seed):
