@@ -40,6 +40,8 @@ N_STEP_INPUTS = 8          # distinct (query, suffix length, step) inputs cycled
 # work (summaries under profiles/, named for the kernel and workload); None where none was taken.
 NCU_TRAFFIC_BYTES = {
     "qwen7b_b1_32k": 34.61e6,      # profiles/attend_kernel_qwen7b_b1_32k.md (mean of two launches)
+    "qwen7b_b8_32k": 409.0e6,      # profiles/attend_kernel_qwen7b_b8_32k.md
+    "ragged": 1036.2e6,            # profiles/all_kernels_ragged.md (mean of two launches)
 }
 
 
