@@ -17,7 +17,9 @@
  *   - "device" pointers address GPU global memory of the current device; "host" pointers
  *     address CPU memory. The library allocates no device memory and keeps no state: the
  *     caller owns every buffer, including workspaces, whose sizes come from the *_sizes /
- *     *_workspace_bytes queries. Buffers must be 256-byte aligned.
+ *     *_workspace_bytes queries. Buffers should be 256-byte aligned; a bf16 / fp32 array or a
+ *     workspace that is not at least 16-byte aligned (64-bit offset arrays: 8, 32-bit tables: 4)
+ *     is refused with SANTAPP_ERR_INVALID_ARG.
  *   - bf16 tensors are raw 16-bit patterns. head_dim is 128. Query head h uses KV head
  *     h / (n_q_heads / n_kv_heads); at most 8 query heads per KV head.
  *   - A batch holds n_seqs independent sequences of prompt length prompt_len[b] >= 1; prompt

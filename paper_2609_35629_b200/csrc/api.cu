@@ -24,6 +24,10 @@ int cuda_fail(cudaError_t err, const char *where)
 
 inline size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
 
+// Device arrays are read and written 16 bytes at a time (8 for the 64-bit offsets, 4 for the 32-bit
+// tables): a pointer that is not aligned accordingly would fault on the device, so it is refused here.
+inline bool misaligned(const void *p, size_t a) { return p != nullptr && (reinterpret_cast<uintptr_t>(p) % a) != 0; }
+
 int check_geom(const santapp_geom *g)
 {
     if (!g) return SANTAPP_ERR_INVALID_ARG;
@@ -48,6 +52,10 @@ int check_teams(const santapp_geom *g, const santapp_teams *t)
     if (!t) return SANTAPP_ERR_INVALID_ARG;
     if (!t->k_packed || !t->v_packed || !t->rep_keys || !t->team_row_start || !t->seq_row_off || !t->seq_team_off
         || !t->rep_abs_max)
+        return SANTAPP_ERR_INVALID_ARG;
+    if (misaligned(t->k_packed, 16) || misaligned(t->v_packed, 16) || misaligned(t->rep_keys, 16)
+        || misaligned(t->team_row_start, 4) || misaligned(t->row_token, 4) || misaligned(t->seq_row_off, 8)
+        || misaligned(t->seq_team_off, 8) || misaligned(t->rep_abs_max, 4))
         return SANTAPP_ERR_INVALID_ARG;
     if (t->rows_total < g->n_seqs || t->teams_total < g->n_seqs || t->max_teams_per_seq < 1)
         return SANTAPP_ERR_INVALID_ARG;
@@ -184,6 +192,11 @@ int santapp_build_teams(const santapp_geom *geom, const int32_t *prompt_len_host
     if (!teams->k_packed || !teams->v_packed || !teams->rep_keys || !teams->team_row_start || !teams->row_token
         || !teams->seq_row_off || !teams->seq_team_off || !teams->rep_abs_max)
         return SANTAPP_ERR_INVALID_ARG;
+    if (misaligned(k_prompt, 16) || misaligned(v_prompt, 16) || misaligned(workspace, 16)
+        || misaligned(teams->k_packed, 16) || misaligned(teams->v_packed, 16) || misaligned(teams->rep_keys, 16)
+        || misaligned(teams->team_row_start, 4) || misaligned(teams->row_token, 4) || misaligned(teams->seq_row_off, 8)
+        || misaligned(teams->seq_team_off, 8) || misaligned(teams->rep_abs_max, 4))
+        return SANTAPP_ERR_INVALID_ARG;
     if (workspace_bytes < sz.build_workspace_bytes) return SANTAPP_ERR_WORKSPACE_TOO_SMALL;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     g_cuda_error[0] = 0;
@@ -254,6 +267,9 @@ int santapp_decode_attn(const santapp_geom *geom, const santapp_teams *teams, co
     if (rc != SANTAPP_OK) return rc;
     if ((rc = check_teams(geom, teams)) != SANTAPP_OK) return rc;
     if (!q || !out || !workspace) return SANTAPP_ERR_INVALID_ARG;
+    if (misaligned(q, 16) || misaligned(out, 16) || misaligned(workspace, 16) || misaligned(k_suffix, 16)
+        || misaligned(v_suffix, 16) || misaligned(suffix_len_dev, 4))
+        return SANTAPP_ERR_INVALID_ARG;
     if (n_sample < 1 || suffix_cap < 0) return SANTAPP_ERR_INVALID_ARG;
     if (n_sample > 128) return SANTAPP_ERR_UNSUPPORTED;
     if (suffix_cap > 0 && suffix_len_dev && (!k_suffix || !v_suffix)) return SANTAPP_ERR_INVALID_ARG;
@@ -374,6 +390,9 @@ int santapp_dense_decode_attn(const santapp_geom *geom, const santapp_teams *tea
     if (rc != SANTAPP_OK) return rc;
     if ((rc = check_teams(geom, teams)) != SANTAPP_OK) return rc;
     if (!q || !out || !workspace) return SANTAPP_ERR_INVALID_ARG;
+    if (misaligned(q, 16) || misaligned(out, 16) || misaligned(workspace, 16) || misaligned(k_suffix, 16)
+        || misaligned(v_suffix, 16) || misaligned(suffix_len_dev, 4))
+        return SANTAPP_ERR_INVALID_ARG;
     if (suffix_cap < 0) return SANTAPP_ERR_INVALID_ARG;
     if (suffix_cap > 0 && suffix_len_dev && (!k_suffix || !v_suffix)) return SANTAPP_ERR_INVALID_ARG;
     if (!(scale >= 0.f) || isinf(scale)) return SANTAPP_ERR_INVALID_ARG;

@@ -544,16 +544,12 @@ template <int G>
 cudaError_t launch_attend_g(const AttendParams &p, bool all_heads, bool static_split, int grid, cudaStream_t s)
 {
     const size_t smem = Smem<G>::total;
-    static thread_local bool attr_set = false;
-    if (!attr_set) {
-        const void *fns[4] = {(const void *)attend_kernel<G, true, true>, (const void *)attend_kernel<G, true, false>,
-                              (const void *)attend_kernel<G, false, true>, (const void *)attend_kernel<G, false, false>};
-        for (const void *fn : fns) {
-            cudaError_t err = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-            if (err != cudaSuccess) return err;
-        }
-        attr_set = true;
-    }
+    static std::atomic<unsigned long long> done[4];
+    const void *fns[4] = {(const void *)attend_kernel<G, true, true>, (const void *)attend_kernel<G, true, false>,
+                          (const void *)attend_kernel<G, false, true>, (const void *)attend_kernel<G, false, false>};
+    const int which = (all_heads ? 0 : 2) + (static_split ? 0 : 1);
+    cudaError_t err = ensure_dynamic_smem(fns[which], (int)smem, done[which]);
+    if (err != cudaSuccess) return err;
     if (all_heads) {
         if (static_split) attend_kernel<G, true, true><<<grid, kAttendThreads, smem, s>>>(p);
         else              attend_kernel<G, true, false><<<grid, kAttendThreads, smem, s>>>(p);

@@ -4,6 +4,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "santapp.h"
 
 namespace santapp {
@@ -116,6 +118,21 @@ struct AttendParams {
     int span_penalty_rows;          // equal-range split: rows a second span costs a CTA (see attend.cu)
     int ctas_per_pair;              // static split: CTAs that share one (sequence, KV head) pair
 };
+
+// Kernels that need more than the default dynamic shared memory opt in once per device (the
+// attribute belongs to the device's context). `done` has one bit per device ordinal below 64;
+// higher ordinals simply set the attribute on every call.
+inline cudaError_t ensure_dynamic_smem(const void *fn, int bytes, std::atomic<unsigned long long> &done)
+{
+    int dev = 0;
+    cudaError_t err = cudaGetDevice(&dev);
+    if (err != cudaSuccess) return err;
+    const unsigned long long bit = dev < 64 ? 1ull << dev : 0ull;
+    if (bit && (done.load(std::memory_order_acquire) & bit)) return cudaSuccess;
+    err = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (err == cudaSuccess && bit) done.fetch_or(bit, std::memory_order_release);
+    return err;
+}
 
 // ---------------------------------------------------------------------------------------------
 // Host launchers (each returns the cudaError_t of its launches).

@@ -101,12 +101,9 @@ template <int G>
 cudaError_t launch_plan_g(const PlanParams &p, cudaStream_t s)
 {
     const size_t smem = sizeof(PlanKernelSmem<G>);
-    static thread_local bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t err = cudaFuncSetAttribute(plan_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (err != cudaSuccess) return err;
-        attr_set = true;
-    }
+    static std::atomic<unsigned long long> done;
+    cudaError_t err = ensure_dynamic_smem((const void *)plan_kernel<G>, (int)smem, done);
+    if (err != cudaSuccess) return err;
     plan_kernel<G><<<p.n_pairs, kPlanThreads, smem, s>>>(p);
     return cudaGetLastError();
 }

@@ -356,13 +356,9 @@ cudaError_t launch_score32_g(const ScoreParams &p, int max_teams, cudaStream_t s
         score32_kernel<G><<<grid, kScoreThreads, 0, s>>>(p);
         return cudaGetLastError();
     }
-    static bool configured = false;                              // per template instance; idempotent
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(score32_flat_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             kScoreRingBytes);
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
+    static std::atomic<unsigned long long> done;
+    cudaError_t e = ensure_dynamic_smem((const void *)score32_flat_kernel<G>, kScoreRingBytes, done);
+    if (e != cudaSuccess) return e;
     score32_flat_kernel<G><<<2 * attend_grid_size(), kScoreThreads, kScoreRingBytes, s>>>(p);
     return cudaGetLastError();
 }

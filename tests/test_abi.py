@@ -82,6 +82,27 @@ def test_null_arguments_return_invalid_arg_without_touching_a_gpu(lib):
     assert rc == sp.SANTAPP_ERR_INVALID_ARG
 
 
+def test_misaligned_pointers_are_refused_on_the_host(lib):
+    """Device arrays are accessed 16 bytes at a time; a pointer that would fault there is refused
+    before any launch (fake addresses: nothing is dereferenced)."""
+    g = sp.Geometry(1, 28, 4).c()
+    A = 0x10000                                                     # an aligned fake address
+    t = sp.CTeams(A, A, A, A, A, A, A, A, 32768, 2048, 2048, 32768)
+    args = dict(q=A, out=A, ws=A)
+
+    def decode(q=A, out=A, ws=A, teams=t):
+        return lib.santapp_decode_attn(ctypes.byref(g), ctypes.byref(teams), q, None, None, None, 0, 32, 0, 0, None,
+                                       0, 0.0, out, None, ws, 0, None)
+
+    assert decode(q=A + 2) == sp.SANTAPP_ERR_INVALID_ARG
+    assert decode(out=A + 4) == sp.SANTAPP_ERR_INVALID_ARG
+    assert decode(ws=A + 8) == sp.SANTAPP_ERR_INVALID_ARG
+    bad = sp.CTeams(A + 2, A, A, A, A, A, A, A, 32768, 2048, 2048, 32768)
+    assert decode(teams=bad) == sp.SANTAPP_ERR_INVALID_ARG
+    # aligned pointers pass the checks and fail later only because the workspace is too small
+    assert decode() == sp.SANTAPP_ERR_WORKSPACE_TOO_SMALL
+
+
 def test_workspace_queries(lib):
     g = sp.Geometry(1, 28, 4)
     t = sp.CTeams(1, 1, 1, 1, 1, 1, 1, 1, 32768, 8192, 2048, 32768)
