@@ -110,7 +110,8 @@ struct Smem {
     static constexpr size_t red_m = red_acc + (size_t)kWarps * G * red_pitch * 4;  // float [warps][G]
     static constexpr size_t red_l = red_m + (size_t)kWarps * G * 4;
     static_assert(red_l + (size_t)kWarps * G * 4 <= ring_bytes, "merge scratch must fit in the ring");
-    static constexpr int merge_chunk = (int)(ring_bytes / ((size_t)G * kPartialStride * 4));   // partials staged at once
+    static constexpr int merge_fit = (int)(ring_bytes / ((size_t)G * kPartialStride * 4));
+    static constexpr int merge_chunk = merge_fit < 64 ? merge_fit : 64;         // partials staged at once (two per lane)
     static_assert(total <= 227 * 1024, "shared memory budget");
 };
 
@@ -493,25 +494,48 @@ attend_kernel(AttendParams p)
                 cp_async_wait_group<0>();
                 __syncthreads();
                 if (h < G) {
-                    float mc = -CUDART_INF_F;
-                    for (int cc = 0; cc < nc; ++cc) mc = fmaxf(mc, stage[(cc * G + h) * kPartialStride]);
+                    // this warp's head: lane l holds the maxima and sums of partials l and l + 32
+                    float mv[2], lv[2];
+#pragma unroll
+                    for (int u = 0; u < 2; ++u) {
+                        const int cc = lane + 32 * u;
+                        mv[u] = cc < nc ? stage[(cc * G + h) * kPartialStride] : -CUDART_INF_F;
+                        lv[u] = cc < nc ? stage[(cc * G + h) * kPartialStride + 1] : 0.f;
+                    }
+                    float mc = fmaxf(mv[0], mv[1]);
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) mc = fmaxf(mc, __shfl_xor_sync(0xFFFFFFFFu, mc, o));
                     const float m_new = fmaxf(m_acc, mc);
                     if (m_new > -CUDART_INF_F) {
                         const float f = m_acc > -CUDART_INF_F ? exp2f(m_acc - m_new) : 0.f;
-                        l_acc *= f;
                         acc.x *= f; acc.y *= f; acc.z *= f; acc.w *= f;
-                        for (int cc = 0; cc < nc; ++cc) {
-                            const float *pp = stage + (cc * G + h) * kPartialStride;
-                            const float mj = pp[0];
-                            if (mj > -CUDART_INF_F) {
-                                const float wgt = exp2f(mj - m_new);
-                                const float4 v = *reinterpret_cast<const float4 *>(pp + 4 + lane * 4);
-                                l_acc = fmaf(wgt, pp[1], l_acc);
-                                acc.x = fmaf(wgt, v.x, acc.x);
-                                acc.y = fmaf(wgt, v.y, acc.y);
-                                acc.z = fmaf(wgt, v.z, acc.z);
-                                acc.w = fmaf(wgt, v.w, acc.w);
-                            }
+                        // one weight per partial, computed once and handed round by shuffle
+                        float w[2];
+#pragma unroll
+                        for (int u = 0; u < 2; ++u) w[u] = mv[u] > -CUDART_INF_F ? exp2f(mv[u] - m_new) : 0.f;
+                        float lsum = fmaf(w[0], lv[0], w[1] * lv[1]);
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) lsum += __shfl_xor_sync(0xFFFFFFFFu, lsum, o);
+                        l_acc = fmaf(l_acc, f, lsum);
+                        const float *col = stage + h * kPartialStride + 4 + lane * 4;
+                        const int n_lo = min(nc, 32);
+#pragma unroll 4
+                        for (int cc = 0; cc < n_lo; ++cc) {
+                            const float wgt = __shfl_sync(0xFFFFFFFFu, w[0], cc);
+                            const float4 v = *reinterpret_cast<const float4 *>(col + (size_t)cc * kPer);
+                            acc.x = fmaf(wgt, v.x, acc.x);
+                            acc.y = fmaf(wgt, v.y, acc.y);
+                            acc.z = fmaf(wgt, v.z, acc.z);
+                            acc.w = fmaf(wgt, v.w, acc.w);
+                        }
+#pragma unroll 4
+                        for (int cc = 32; cc < nc; ++cc) {
+                            const float wgt = __shfl_sync(0xFFFFFFFFu, w[1], cc - 32);
+                            const float4 v = *reinterpret_cast<const float4 *>(col + (size_t)cc * kPer);
+                            acc.x = fmaf(wgt, v.x, acc.x);
+                            acc.y = fmaf(wgt, v.y, acc.y);
+                            acc.z = fmaf(wgt, v.z, acc.z);
+                            acc.w = fmaf(wgt, v.w, acc.w);
                         }
                         m_acc = m_new;
                     }
