@@ -55,6 +55,8 @@ def parse_args():
     ap.add_argument("--workload", default="qwen7b_b1_32k",
                     choices=["qwen7b_b1_32k", "qwen7b_b8_32k", "ragged", "long_128k", "paper_point_32k", "small_gqa"])
     ap.add_argument("--n-sample", type=int, default=0, help="override K")
+    ap.add_argument("--key-layout", default="iid", choices=["iid", "runs"],
+                    help="cluster of each prompt row: independent draws, or geometric runs (positional locality)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-stages", action="store_true")
@@ -78,13 +80,15 @@ def make_spec(args, seed):
         spec = synth.spec_small_gqa(seed=seed)
     if args.n_sample:
         spec.n_sample = args.n_sample
+    spec.key_layout = args.key_layout
     return spec
 
 
 def workload_text(spec, layers):
     return (f"{spec.name}: {spec.n_seqs} seq x {spec.n_q_heads} q heads / {spec.n_kv_heads} KV heads, d={spec.head_dim}, "
             f"prompt {min(spec.prompt_len)}..{max(spec.prompt_len)}, suffix cap {spec.suffix_cap}, "
-            f"P={spec.parent_size}, R={spec.reps_per_parent}, K={spec.n_sample}, {layers} layers round-robin")
+            f"P={spec.parent_size}, R={spec.reps_per_parent}, K={spec.n_sample}, keys {spec.key_layout}, "
+            f"{layers} layers round-robin")
 
 
 # -------------------------------------------------------------------------------------------
@@ -223,7 +227,7 @@ def run_ours(args):
                             want_e2e=not args.no_e2e, want_cpu=not args.no_cpu_baseline, want_stages=not args.no_stages)
     # Beside the headline workload (batch 1, latency-bound on this GPU), the same measurement on a
     # batch large enough to be bandwidth-bound: the ragged serving batch, two layers.
-    if args.workload == "qwen7b_b1_32k" and not args.no_batched and not args.n_sample:
+    if args.workload == "qwen7b_b1_32k" and not args.no_batched and not args.n_sample and args.key_layout == "iid":
         import gc
         gc.collect()
         torch.cuda.empty_cache()
@@ -434,7 +438,7 @@ def measure_workload(args, workload, n_layers, n_steps, n_warmup, dev, want_e2e,
         achieved = attend_bytes_1 / (stages["attend"] * 1e-6) / 1e9
         roofline = {"bound": "hbm", "kernel": "attend_kernel", "achieved": achieved, "peak": peak_gbs, "unit": "GB/s",
                     "frac": achieved / peak_gbs,
-                    "traffic": NCU_TRAFFIC_BYTES.get(spec.name) if not args.n_sample else None,
+                    "traffic": NCU_TRAFFIC_BYTES.get(spec.name) if not args.n_sample and spec.key_layout == "iid" else None,
                     "peak_kind": peak_kind,
                     "algorithmic_bytes_per_launch": attend_bytes_1, "us_per_launch": stages["attend"]}
 

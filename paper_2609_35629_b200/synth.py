@@ -62,6 +62,8 @@ class WorkloadSpec:
     suffix_len0: List[int]           # suffix length at step 0, per sequence
     suffix_growth: int               # rows appended per step
     query_kind: str = "noisy_copy"   # or "concentrated"
+    key_layout: str = "iid"          # cluster of each prompt row: "iid", or "runs" (geometric runs of one
+                                     # cluster, mean length rows / clusters: positional locality)
     head_dim: int = HEAD_DIM
     seed: int = 0
 
@@ -143,9 +145,20 @@ class LayerData:
     centres: Optional[np.ndarray] = field(default=None, repr=False)   # [n_kv, n_clusters, d] float32
 
 
-def _clustered_rows(rng, n_rows, centres, sigma=0.3):
+def _clustered_rows(rng, n_rows, centres, sigma=0.3, layout="iid"):
     n_clusters, d = centres.shape
-    which = rng.integers(0, n_clusters, size=n_rows)
+    if layout == "iid":
+        which = rng.integers(0, n_clusters, size=n_rows)
+    elif layout == "runs":
+        mean_run = max(n_rows / n_clusters, 1.0)
+        lengths = np.empty(0, dtype=np.int64)
+        while lengths.sum() < n_rows:
+            more = rng.geometric(1.0 / mean_run, size=int(1.5 * n_rows / mean_run) + 8)
+            lengths = np.concatenate([lengths, more])
+        ids = rng.integers(0, n_clusters, size=lengths.shape[0])
+        which = np.repeat(ids, lengths)[:n_rows]
+    else:
+        raise ValueError(layout)
     eps = rng.standard_normal((n_rows, d), dtype=np.float32)
     return centres[which] + np.float32(sigma) * eps
 
@@ -167,7 +180,7 @@ def make_layer(spec: WorkloadSpec, layer: int = 0, keep_centres: bool = False) -
         centres_all[j] = centres
         for b in range(spec.n_seqs):
             n = spec.prompt_len[b]
-            k = _clustered_rows(rng, n, centres)
+            k = _clustered_rows(rng, n, centres, layout=spec.key_layout)
             k[: min(4, n)] *= np.float32(4.0)        # sink keys
             v = rng.standard_normal((n, d), dtype=np.float32)
             k_prompt[j, off[b]:off[b + 1]] = f32_to_bf16_bits(k)

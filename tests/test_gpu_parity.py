@@ -227,6 +227,18 @@ def test_qwen_32k_full_size_batch1():
     check_dense_step(layer, 9)
 
 
+def test_keys_in_runs_variant():
+    """Cluster ids in geometric runs (positional locality): smaller, more even teams than with
+    independent draws; same method, same bars."""
+    import dataclasses
+    spec = dataclasses.replace(synth.spec_small_gqa(prompt=(2048, 1500)), key_layout="runs")
+    layer = pu.GpuLayer(spec, synth.make_layer(spec))
+    check_team_records(layer, kv_heads=[0])
+    for step in range(2):
+        check_sparse_step(layer, step, K=8)
+    check_dense_step(layer, 0)
+
+
 def test_paper_operating_point_32k():
     """Parents of 16 keys with 4 representatives at 32K (8192 teams of about 4 rows per KV head),
     31 sampled teams, no suffix: routing reads an eighth of the dense bytes, gathers are tiny."""

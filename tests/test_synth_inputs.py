@@ -1,0 +1,59 @@
+"""The seeded input generators (no method arithmetic): determinism, the two key layouts, the bf16
+helpers and the suffix schedule."""
+import dataclasses
+
+import numpy as np
+
+from paper_2609_35629_b200 import synth
+
+
+def test_layers_are_reproducible_and_seeded():
+    spec = synth.spec_small_gqa()
+    a, b = synth.make_layer(spec, layer=1), synth.make_layer(spec, layer=1)
+    assert np.array_equal(a.k_prompt, b.k_prompt) and np.array_equal(a.v_suffix, b.v_suffix)
+    c = synth.make_layer(spec, layer=2)
+    assert not np.array_equal(a.k_prompt, c.k_prompt)
+    d = synth.make_layer(synth.spec_small_gqa(seed=1), layer=1)
+    assert not np.array_equal(a.k_prompt, d.k_prompt)
+    q0, q1 = synth.make_queries(spec, a, 0), synth.make_queries(spec, a, 1)
+    assert np.array_equal(q0, synth.make_queries(spec, a, 0)) and not np.array_equal(q0, q1)
+
+
+def test_bf16_helpers_round_to_nearest_even_and_widen_exactly():
+    x = np.array([1.0, 1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -8, -2.5, 0.0, 3.0e38], dtype=np.float32)
+    bits = synth.f32_to_bf16_bits(x)
+    back = synth.bf16_to_f32(bits)
+    assert back[0] == 1.0 and back[1] == 1.0                       # tie to even (down)
+    assert back[2] == np.float32(1.0 + 2.0 ** -6)                  # tie to even (up)
+    assert back[3] == -2.5 and back[4] == 0.0
+    assert np.array_equal(synth.bf16_to_f64(bits), back.astype(np.float64))
+    assert np.array_equal(synth.f32_to_bf16_bits(back), bits)      # idempotent
+
+
+def _run_lengths(which):
+    edges = np.flatnonzero(np.diff(which) != 0)
+    return np.diff(np.concatenate([[-1], edges, [len(which) - 1]]))
+
+
+def test_key_layouts():
+    """"iid": every row draws its cluster independently; "runs": geometric runs of one cluster
+    with mean length rows / clusters. Recover the cluster of each row by nearest centre."""
+    base = synth.spec_small_gqa(n_seqs=1, prompt=(4096,), suffix0=(0,))
+    for layout, lo, hi in (("iid", 1.0, 1.1), ("runs", 0.6 * 4096 / 32, 1.6 * 4096 / 32)):
+        spec = dataclasses.replace(base, key_layout=layout)
+        data = synth.make_layer(spec, keep_centres=True)
+        k = synth.bf16_to_f32(data.k_prompt[0])[4:]                # skip the scaled sink rows
+        c = data.centres[0]
+        d2 = (k * k).sum(1)[:, None] - 2.0 * k @ c.T + (c * c).sum(1)[None, :]
+        which = d2.argmin(1)
+        mean_run = _run_lengths(which).mean()
+        assert lo <= mean_run <= hi, (layout, mean_run)
+    # the default layout is the independent one, and its data do not depend on the new field
+    assert base.key_layout == "iid"
+
+
+def test_suffix_schedule():
+    spec = synth.spec_qwen_b1()
+    assert spec.suffix_len(0)[0] == 1 and spec.suffix_len(10)[0] == 11
+    assert spec.suffix_len(10_000)[0] == spec.suffix_cap            # clamps at the capacity
+    assert synth.spec_paper_point().suffix_len(5)[0] == 0
