@@ -418,7 +418,7 @@ def measure_workload(args, workload, n_layers, n_steps, n_warmup, dev, want_e2e,
         g_sparse.replay()
         torch.cuda.synchronize()
         for name, mask in (("route_score", sp.STAGE_ROUTE), ("select_plan", sp.STAGE_SELECT),
-                           ("attend", sp.STAGE_ATTEND)):
+                           ("route_and_select", sp.STAGE_ROUTE | sp.STAGE_SELECT), ("attend", sp.STAGE_ATTEND)):
             sp.santapp_set_stage_mask(mask)
             g = capture(sparse_layer)
             sp.santapp_set_stage_mask(sp.STAGE_ALL)
