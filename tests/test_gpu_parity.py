@@ -355,6 +355,28 @@ def test_non_finite_query_raises_status_bits_and_leaves_the_library_usable():
     check_sparse_step(layer, 0, K=8)                                  # and a clean call still matches the oracle
 
 
+def test_ragged_batch_full_size_sampled_sequences():
+    """Config 4 at full size (32 sequences of 8K to 64K tokens, suffixes up to 1024 rows, 31 sampled
+    teams): the GPU runs the whole batch, the oracle checks the shortest, the longest and one more."""
+    layer = layer_for("ragged_full", synth.spec_ragged)
+    lens = np.asarray(layer.spec.prompt_len)
+    seqs = sorted({int(lens.argmin()), int(lens.argmax()), 17})
+    check_sparse_step(layer, 0, K=31, seqs=seqs)
+    check_sparse_step(layer, 127, K=31, seqs=seqs[:1])
+    check_dense_step(layer, 3, seqs=seqs[-1:])
+    _cache.pop(("ragged_full", ()), None)                              # 2 GB of device memory
+
+
+def test_long_context_128k_sampled_sequence():
+    """Config 5 shape (4 sequences of 131072 tokens, 8192 teams per KV head): budgets 16 and 128,
+    one sequence against the oracle."""
+    layer = layer_for("long", synth.spec_long)
+    check_sparse_step(layer, 0, K=16, seqs=[2])
+    check_sparse_step(layer, 1, K=128, seqs=[0])
+    check_dense_step(layer, 0, seqs=[3])
+    _cache.pop(("long", ()), None)
+
+
 def test_device_side_step_offset_equals_explicit_step():
     """step = 3 with a device-side offset of 4 draws the same sample as step = 7."""
     layer = layer_for("small", synth.spec_small_gqa)
