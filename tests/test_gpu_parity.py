@@ -153,6 +153,24 @@ def test_decode_k_at_least_m_equals_dense():
         check_sparse_step(layer, step, K=int(Ms.min()))
 
 
+def test_decode_one_team_left_out():
+    """K = M - 1, the smallest sampled case: tau is the single excluded team's score."""
+    layer = layer_for("small", synth.spec_small_gqa)
+    Ms = np.diff(layer.seq_team_off)
+    check_sparse_step(layer, 0, K=int(Ms.min()) - 1)
+    check_sparse_step(layer, 1, K=int(Ms.max()) - 1)                 # the shorter sequence takes every team
+
+
+def test_decode_large_logits():
+    """Queries scaled up sixteen-fold: logits in the hundreds, softmax weights and corrections at
+    the ends of their ranges; the log-sum-exp bookkeeping must hold."""
+    layer = layer_for("small", synth.spec_small_gqa)
+    spec = layer.spec
+    q_bits = synth.make_queries(spec, layer.data, 2)
+    big = synth.f32_to_bf16_bits(16.0 * synth.bf16_to_f32(q_bits))
+    _check_with_queries(layer, big, K=8, step=2)
+
+
 def test_decode_suffix_edge_cases():
     layer = layer_for("small", synth.spec_small_gqa)
     check_sparse_step(layer, 0, K=8, suffix_len=[0, 0])
