@@ -41,7 +41,7 @@ constexpr int kSlots = 2;                                   // ring slots per wa
 constexpr int kRowBytes = kHeadDim * 2;                     // one bf16 row
 constexpr int kTileBytes = kBlockRows * kRowBytes;          // K tile or V tile of a block
 constexpr int kSlotBytes = 2 * kTileBytes;                  // K tile then V tile
-constexpr int kPairMax = 512;                               // pairs whose offsets are staged (dynamic split)
+constexpr int kPairMax = 512;                               // pairs whose offsets are staged at a time (dynamic split)
 constexpr int kMaxAttendGrid = 512;
 constexpr uint32_t kNoRow = 0xFFFFFFFFu;
 
@@ -140,29 +140,44 @@ attend_kernel(AttendParams p)
 
     // ---- which (pair, row range) spans this CTA works on ----
     int pair, sub = 0;
+    int pair_base = 0;                                     // first pair of the staged window (dynamic split)
+    auto stage_pairs = [&](int base) {                     // all threads: stage pairs [base, base + kPairMax]
+        __syncthreads();
+        const int n = min(kPairMax, p.n_pairs - base);
+        for (int i = tid; i <= n; i += kAttendThreads) pair_prefix[i] = p.plan.pair_row_prefix[base + i];
+        for (int i = tid; i < n; i += kAttendThreads) pair_nseg[i] = p.plan.pair_nseg[base + i];
+        __syncthreads();
+        pair_base = base;
+    };
     int64_t r0 = 0, r1 = 0, rows_per_cta = 0;              // dynamic split: global row range
     if (kStatic) {
         pair = blockIdx.x / p.ctas_per_pair;
         sub = blockIdx.x - pair * p.ctas_per_pair;
         if (pair >= p.n_pairs) return;
     } else {
-        for (int i = tid; i <= p.n_pairs; i += kAttendThreads) pair_prefix[i] = p.plan.pair_row_prefix[i];
-        for (int i = tid; i < p.n_pairs; i += kAttendThreads) pair_nseg[i] = p.plan.pair_nseg[i];
-        __syncthreads();
+        // pair_prefix / pair_nseg hold a window of kPairMax pairs starting at pair_base; batches of up
+        // to kPairMax pairs are staged whole, before anything else is waited for
+        const bool windowed = p.n_pairs > kPairMax;
+        if (!windowed) stage_pairs(0);
+        const int64_t all_rows = windowed ? p.plan.pair_row_prefix[p.n_pairs] : pair_prefix[p.n_pairs];
         // Rows of all pairs laid end to end, with a gap of span_penalty_rows after every pair: a CTA
         // whose range crosses from one pair into the next pays the fixed cost of a second span
         // (tables, pipeline refill, merge) out of its row budget, so ranges cost about equal time.
-        const int64_t total = pair_prefix[p.n_pairs] + (int64_t)p.span_penalty_rows * (p.n_pairs - 1);
+        const int64_t total = all_rows + (int64_t)p.span_penalty_rows * (p.n_pairs - 1);
         rows_per_cta = (total + gridDim.x - 1) / gridDim.x;
         if (rows_per_cta < p.min_rows_per_cta) rows_per_cta = p.min_rows_per_cta;
         r0 = (int64_t)blockIdx.x * rows_per_cta;
         if (r0 >= total) return;
         r1 = min(r0 + rows_per_cta, total);
+        // first pair of the range: the largest i with prefix[i] + penalty * i <= r0
         int lo = 0, hi = p.n_pairs;
         while (hi - lo > 1) {
             const int mid = (lo + hi) >> 1;
-            if (pair_prefix[mid] + (int64_t)p.span_penalty_rows * mid <= r0) lo = mid; else hi = mid;
+            const int64_t start = (windowed ? p.plan.pair_row_prefix[mid] : pair_prefix[mid])
+                                  + (int64_t)p.span_penalty_rows * mid;
+            if (start <= r0) lo = mid; else hi = mid;
         }
+        if (windowed) stage_pairs(lo);
         pair = lo;
     }
 
@@ -232,8 +247,9 @@ attend_kernel(AttendParams p)
             }
         } else {
             // this pair's rows occupy [pb, pe) of the padded row line
-            pb = pair_prefix[pair] + (int64_t)p.span_penalty_rows * pair;
-            pe = pb + (pair_prefix[pair + 1] - pair_prefix[pair]);
+            if (pair - pair_base >= kPairMax) stage_pairs(pair);           // walked off the staged window
+            pb = pair_prefix[pair - pair_base] + (int64_t)p.span_penalty_rows * pair;
+            pe = pb + (pair_prefix[pair - pair_base + 1] - pair_prefix[pair - pair_base]);
             a = (int)(max(r0, pb) - pb);
             bnd = (int)(min(r1, pe) - pb);
             if (a >= bnd) {                                // the range starts in the gap behind this pair
@@ -242,7 +258,7 @@ attend_kernel(AttendParams p)
                 ++pair;
                 continue;
             }
-            nseg = pair_nseg[pair];
+            nseg = pair_nseg[pair - pair_base];
             const int c_lo = (int)(pb / rows_per_cta), c_hi = (int)((pe - 1) / rows_per_cta);
             n_ctas = c_hi - c_lo + 1;
             first_slot = c_lo + pair;
@@ -594,7 +610,7 @@ int attend_grid_size()
 }
 
 int attend_max_segments() { return kSegMax; }
-int attend_max_pairs() { return kPairMax; }
+int attend_max_pairs() { return 1 << 16; }
 
 cudaError_t launch_attend(const AttendParams &p, bool all_heads, bool static_split, int grid, cudaStream_t s)
 {

@@ -395,6 +395,18 @@ def test_long_context_128k_sampled_sequence():
     _cache.pop(("long", ()), None)
 
 
+def test_decode_more_pairs_than_one_window():
+    """160 short sequences = 640 (sequence, KV head) pairs, more than the attention kernel stages at
+    a time; the oracle checks the first, the last and two in between."""
+    n = 160
+    spec = synth.spec_small_gqa(n_seqs=n, prompt=tuple(192 + 64 * (i % 3) for i in range(n)), parent_size=64, reps=8,
+                                n_sample=8, suffix0=tuple(i % 3 for i in range(n)))
+    layer = pu.GpuLayer(spec, synth.make_layer(spec))
+    seqs = [0, 53, 106, n - 1]
+    check_sparse_step(layer, 0, K=8, seqs=seqs)
+    check_dense_step(layer, 1, seqs=seqs)
+
+
 def test_device_side_step_offset_equals_explicit_step():
     """step = 3 with a device-side offset of 4 draws the same sample as step = 7."""
     layer = layer_for("small", synth.spec_small_gqa)
