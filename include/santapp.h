@@ -187,7 +187,7 @@ size_t santapp_decode_workspace_bytes(const santapp_geom *geom, const santapp_te
  *                   [0, suffix_cap]); NULL means 0 everywhere
  *   n_sample        1 <= K <= 128, and (query heads per KV head) * min(K, M_b) <= 1024
  *                   (SANTAPP_ERR_UNSUPPORTED beyond; likewise for more than 65536 (sequence, KV
- *                   head) pairs in one call or more than 16384 teams in a sequence)
+ *                   head) pairs in one call or more than 65536 teams in a sequence)
  *   seed, step, stream_base   random-stream key and counters (see top of file)
  *   step_dev        device uint32 [1] or NULL: when given, its value is added to `step` on the
  *                   device, so a captured CUDA graph can be replayed for successive tokens

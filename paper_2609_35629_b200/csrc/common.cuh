@@ -13,7 +13,7 @@ namespace santapp {
 constexpr int kHeadDim = 128;
 constexpr int kMaxGroup = 8;            // query heads per KV head
 constexpr int kMaxParent = 512;
-constexpr int kMaxTeamsPerSeq = 16384;  // selection keeps one 8-byte key per team in shared memory
+constexpr int kMaxTeamsPerSeq = 65536;  // the union plan keeps one bit and a prefix word per 32 teams in shared memory
 constexpr uint32_t kSrcSuffix = 0x80000000u;   // segment flag: rows live in the suffix buffers
 
 constexpr int kPartialStride = 132;     // floats per (slot, head): m, l, 2 pad, acc[128]

@@ -267,6 +267,14 @@ def test_paper_operating_point_32k():
     check_dense_step(layer, 2)
 
 
+def test_paper_operating_point_128k():
+    """The same operating point at 131072 tokens: 32768 teams per KV head."""
+    spec = synth.spec_paper_point(prompt=131072)
+    layer = pu.GpuLayer(spec, synth.make_layer(spec))
+    check_sparse_step(layer, 0, K=31)
+    check_dense_step(layer, 1)
+
+
 def test_qwen_32k_batch8_concentrated_sampled_sequences():
     """Config 3 shape (8 sequences, 64 sampled teams, concentrated queries): the GPU runs the
     whole batch, the oracle checks two of the sequences."""
