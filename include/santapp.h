@@ -119,7 +119,9 @@ typedef struct santapp_debug {
     int32_t *status;           /* int32 [1]: bit flags raised on the device (0 = clean);
                                   bit 0: non-finite output; bit 1: a head had fewer than K + 1
                                   comparable routing scores (non-finite q or keys): its sample was
-                                  completed with arbitrary teams, the output is meaningless        */
+                                  completed with arbitrary teams, the output is meaningless;
+                                  bit 2: a bounded wait for an asynchronous copy expired in the
+                                  scorer (never expected; the step's result is not valid)           */
 } santapp_debug;
 
 /* Library version: major * 10000 + minor * 100 + patch. */

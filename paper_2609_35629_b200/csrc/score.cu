@@ -6,9 +6,11 @@
 // itself is decided in fp64 there.
 //
 // The GQA group is the M tile of S^T = q K^T (mma.sync m16n8k16, bf16 inputs, fp32
-// accumulation). Lanes load 16-byte pieces of the representative keys straight from global
-// memory; the contraction index is permuted consistently on both operands, so no shared memory
-// staging is needed.
+// accumulation). A lane feeds the tensor core 16-byte pieces of the representative keys exactly
+// as they lie in memory: the contraction index is permuted consistently on both operands, so
+// no transpose is needed. Small grids load the pieces straight from global memory; large grids
+// stream whole tiles (16 keys = one contiguous 4 KB run) into shared memory with bulk
+// asynchronous copies that complete on mbarriers, three tiles ahead.
 #include "common.cuh"
 
 namespace santapp {
@@ -28,10 +30,6 @@ __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint3
                  : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1));
 }
 
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src)
-{
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
-}
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait_group()
@@ -39,11 +37,37 @@ __device__ __forceinline__ void cp_async_wait_group()
     asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
 }
 
+// Bulk asynchronous copy (the TMA engine's untiled form) of a contiguous run of bytes into shared
+// memory, completion counted in bytes on an mbarrier; addresses and size are multiples of 16.
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_copy_to_shared(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+
 constexpr int kScoreStages = 3;                                 // tiles in flight per warp (pipelined variant)
 constexpr int kScoreKeyRingBytes = kScoreStages * (kScoreThreads / 32) * 4096;
 constexpr int kScoreCsrRingBytes = kScoreStages * (kScoreThreads / 32) * 128;                       // row offsets
 constexpr int kSeqTableCap = 2048;                              // sequences whose first tile slot is kept in shared memory
-constexpr int kScoreRingBytes = kScoreKeyRingBytes + kScoreCsrRingBytes + (kSeqTableCap + 1) * 4;
+constexpr int kScoreSeqTableBytes = ((kSeqTableCap + 1) * 4 + 15) / 16 * 16;
+constexpr int kScoreBarrierBytes = kScoreStages * (kScoreThreads / 32) * 8;                         // one mbarrier per (warp, stage)
+constexpr int kScoreRingBytes = kScoreKeyRingBytes + kScoreCsrRingBytes + kScoreSeqTableBytes + kScoreBarrierBytes;
+constexpr int kScoreWaitPolls = 1 << 22;                        // bound on the polls of one mbarrier wait
 
 // Gumbel(0,1) in fp32 from a 32-bit word: u = (x + 0.5) / 2^32, G = -log(-log u), to an absolute
 // error well inside the additive term of the guard (see score_guard in pairplan.cuh).
@@ -236,9 +260,10 @@ __device__ __forceinline__ void advance(const ScoreParams &p, TileCursor &cur)
 }
 
 // Large grids: two resident blocks per SM, every warp walks an equal contiguous share of all
-// tiles. The keys of the next kScoreStages tiles are in flight as cp.async copies into slots
-// private to each lane (a lane copies exactly the pieces it later feeds to the tensor core, so
-// no barrier is needed).
+// tiles. The keys of the next kScoreStages tiles are in flight: lane 0 issues one bulk copy per
+// tile (16 keys are one contiguous run) that completes on the stage's mbarrier; the tile's 17 row
+// offsets travel as per-lane 4-byte cp.async copies (their address is only 4-byte aligned).
+// Every wait on an mbarrier is bounded; on expiry the warp raises status bit 2 and stops.
 template <int G>
 __global__ void __launch_bounds__(kScoreThreads, 2)
 score32_flat_kernel(ScoreParams p)
@@ -254,14 +279,24 @@ score32_flat_kernel(ScoreParams p)
     const uint32_t step = p.step + (p.step_dev ? *p.step_dev : 0u);
     const float scale = (float)p.scale;
 
-    // slot of piece (t, i) of stage s: [warp][s][t * 4 + i][lane]
-    auto slot = [&](int s, int t, int i) { return score_ring + ((warp * kScoreStages + s) * 8 + t * 4 + i) * 32 + lane; };
+    // keys of the tile in stage s: [warp][s] 16 rows of 256 bytes, as in global memory
+    auto tile_of = [&](int s) { return score_ring + (warp * kScoreStages + s) * 256; };
+    // completion barrier of stage s, initialised by lane 0
+    const uint32_t bars = (uint32_t)__cvta_generic_to_shared(reinterpret_cast<unsigned char *>(score_ring) + kScoreKeyRingBytes
+                                                             + kScoreCsrRingBytes + kScoreSeqTableBytes)
+                          + (uint32_t)warp * kScoreStages * 8;
+    if (lane == 0) {
+#pragma unroll
+        for (int s = 0; s < kScoreStages; ++s) mbar_init(bars + 8 * s, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
     // the tile's 17 row offsets, copied by lanes 0..16: [warp][s][32]
     int32_t *csr_ring = reinterpret_cast<int32_t *>(reinterpret_cast<unsigned char *>(score_ring) + kScoreKeyRingBytes)
                         + warp * kScoreStages * 32;
     // first slot of every sequence, for the searches of locate_tile
     int *seq_slot = reinterpret_cast<int *>(reinterpret_cast<unsigned char *>(score_ring) + kScoreKeyRingBytes
-                                            + kScoreCsrRingBytes);
+                                            + kScoreCsrRingBytes);       // kScoreSeqTableBytes
     if (p.bv.n_seqs <= kSeqTableCap) {
         for (int i = tid; i < p.bv.n_seqs; i += kScoreThreads) seq_slot[i] = (int)(p.bv.seq_team_off[i] >> 4) + i;
         __syncthreads();
@@ -273,12 +308,12 @@ score32_flat_kernel(ScoreParams p)
     auto issue_tile = [&](int s) {
         int base;
         if (t_ahead < t_hi && locate_tile(p, seq_slot, ahead, base)) {
-            const uint16_t *rep = p.rep_keys + ((size_t)ahead.j * p.bv.teams_total + ahead.team0) * kHeadDim;
-#pragma unroll
-            for (int t = 0; t < 2; ++t) {
-                const uint4 *row = reinterpret_cast<const uint4 *>(rep + (size_t)min(base + 8 * t + g, ahead.M - 1) * kHeadDim);
-#pragma unroll
-                for (int i = 0; i < 4; ++i) cp_async16((uint32_t)__cvta_generic_to_shared(slot(s, t, i)), row + c + 4 * i);
+            // the tile's keys are one contiguous run: a single bulk copy by lane 0
+            if (lane == 0) {
+                const uint16_t *src = p.rep_keys + ((size_t)ahead.j * p.bv.teams_total + ahead.team0 + base) * kHeadDim;
+                const uint32_t bytes = (uint32_t)min(kScoreTeamsPerWarp, ahead.M - base) * kHeadDim * 2;
+                mbar_expect_tx(bars + 8 * s, bytes);
+                bulk_copy_to_shared((uint32_t)__cvta_generic_to_shared(tile_of(s)), src, bytes, bars + 8 * s);
             }
             if (lane <= 16 && base + lane <= ahead.M) {
                 const int32_t *csr = p.team_row_start + (size_t)ahead.j * (p.bv.teams_total + p.bv.n_seqs) + ahead.team0
@@ -297,11 +332,22 @@ score32_flat_kernel(ScoreParams p)
     uint32_t qa[8][2];
     int q_b = -1, q_j = -1;
     int stage = 0;
+    uint32_t phases = 0u;                                        // bit s: parity of the next completion of stage s
     for (long long ti = t_lo; ti < t_hi; ++ti) {
-        cp_async_wait_group<kScoreStages - 1>();                 // this lane's pieces of tile ti have landed
+        cp_async_wait_group<kScoreStages - 1>();                 // this lane's row offset of tile ti has landed
         __syncwarp();                                            // the row offsets come from other lanes
         int base;
         if (locate_tile(p, seq_slot, here, base)) {
+            // wait for the tile's keys; the wait is bounded: on expiry the kernel flags it and stops
+            int polls = 0;
+            while (!mbar_try_wait(bars + 8 * stage, (phases >> stage) & 1u)) {
+                if (++polls >= kScoreWaitPolls) break;
+            }
+            if (polls >= kScoreWaitPolls) {
+                if (lane == 0 && p.status) atomicOr(p.status, 4);
+                break;
+            }
+            phases ^= 1u << stage;
             if (here.b != q_b || here.j != q_j) {
                 load_q_fragments<G>(p, here.b, here.j, g, c, qa);
                 q_b = here.b;
@@ -311,7 +357,7 @@ score32_flat_kernel(ScoreParams p)
 #pragma unroll
             for (int t = 0; t < 2; ++t)
 #pragma unroll
-                for (int i = 0; i < 4; ++i) kb[t][i] = *slot(stage, t, i);
+                for (int i = 0; i < 4; ++i) kb[t][i] = tile_of(stage)[(8 * t + g) * 16 + c + 4 * i];
             score_tile<G>(p, here.b, here.j, here.team0, here.M, base, csr_ring + stage * 32, kb, qa, step, scale, g, c);
         }
         __syncwarp();                                            // every lane is done with the stage's row offsets
