@@ -511,6 +511,7 @@ def measure_workload(args, workload, n_layers, n_steps, n_warmup, dev, want_e2e,
             "read_reduction": mean_dense_bytes / mean_sparse_bytes,
             "achieved_gbs": mean_sparse_bytes / (us_layer * 1e-6) / 1e9,
             "achieved_frac_of_peak": mean_sparse_bytes / (us_layer * 1e-6) / 1e9 / peak_gbs,
+            "achieved_frac_of_nominal_8tbs": mean_sparse_bytes / (us_layer * 1e-6) / 8e12,
             "dense_achieved_gbs": mean_dense_bytes / (us_layer_dense * 1e-6) / 1e9,
             "dense_achieved_frac_of_peak": mean_dense_bytes / (us_layer_dense * 1e-6) / 1e9 / peak_gbs,
             "attend_bytes_per_layer_step": mean_attend_bytes,
