@@ -24,6 +24,8 @@
  *   orc_logical_access_*      logical KV-access counter, Eq. (qwen-logical-access)
  *   orc_team_budget           selected-team count, Eq. (method-budget)
  *   orc_routing_kl            routing-agreement diagnostic, Eq. (diagnostic-kl)
+ *   orc_group_mean_keys       centroid-guided baseline of the routing diagnostic: one group per
+ *                             parent, routed by the arithmetic mean of its keys
  *
  * Parity pins (tests marked "not gpu"): Philox words against an independent
  * library generator; Gumbel law by Kolmogorov-Smirnov and moments; first-draw
@@ -588,4 +590,33 @@ double orc_routing_kl(int d, const double *q, int64_t N, const double *k, int32_
     free(s);
     free(phi);
     return kl;
+}
+
+/* Centroid-guided baseline (Section "How closely routing follows dense attention" and the
+ * appendix on the KL variants): every group is routed by the arithmetic mean of its keys
+ * instead of an actual key; the routing logit still adds log n_g, sampling, correction and
+ * estimator are unchanged. The paper forms the groups by k-means; here the groups are the
+ * contiguous parents of Algorithm 4 (k-means parents are not built in this library).
+ * For parent u: mean_u = (sum over its tokens in index order of k_i) / |C_u| in fp64, then
+ * stored as a bf16 value like every other routing key: fp64 -> fp32 (round to nearest) ->
+ * bf16 (round to nearest even). out_mean[n_parents][d] receives those values widened back to
+ * fp64. Returns n_parents. */
+int32_t orc_group_mean_keys(int32_t N, int d, const double *keys, int32_t P, double *out_mean)
+{
+    int32_t n_parents = (N + P - 1) / P;
+    for (int32_t u = 0; u < n_parents; ++u) {
+        int32_t lo = u * P, hi = (u + 1) * P < N ? (u + 1) * P : N;
+        for (int j = 0; j < d; ++j) {
+            double sum = 0.0;
+            for (int32_t i = lo; i < hi; ++i) sum += keys[(int64_t)i * d + j];
+            float f = (float)(sum / (double)(hi - lo));
+            uint32_t bits;
+            memcpy(&bits, &f, sizeof bits);
+            uint32_t rounded = (bits + 0x7FFFu + ((bits >> 16) & 1u)) & 0xFFFF0000u;
+            float back;
+            memcpy(&back, &rounded, sizeof back);
+            out_mean[(int64_t)u * d + j] = (double)back;
+        }
+    }
+    return n_parents;
 }

@@ -83,6 +83,8 @@ def lib():
         L.orc_dense_kv_bytes.restype = _c.c_double
         L.orc_routing_kl.argtypes = [_c.c_int, _f64p, _c.c_int64, _f64p, _c.c_int32, _i32p, _i32p, _f64p, _c.c_double]
         L.orc_routing_kl.restype = _c.c_double
+        L.orc_group_mean_keys.argtypes = [_c.c_int32, _c.c_int, _f64p, _c.c_int32, _f64p]
+        L.orc_group_mean_keys.restype = _c.c_int32
         _lib = L
     return _lib
 
@@ -310,3 +312,16 @@ def routing_kl(q, k, team_start, team_member, rep_key, scale):
     team_start, team_member = _i32(team_start), _i32(team_member)
     return float(lib().orc_routing_kl(q.shape[0], q, k.shape[0], k, team_start.shape[0] - 1, team_start,
                                       team_member, rep_key, scale))
+
+
+def group_mean_keys(keys, P):
+    """Centroid-guided baseline on contiguous parents: (team_start, team_member, mean_key) with one
+    group per parent, members in token order, and the parent's arithmetic-mean key rounded to a
+    bf16 value as its routing key."""
+    keys = _f64(keys)
+    N, d = keys.shape
+    n_parents = (N + P - 1) // P
+    mean = np.zeros((n_parents, d))
+    got = lib().orc_group_mean_keys(N, d, keys, P, mean)
+    assert got == n_parents
+    return contiguous_parents(N, P), np.arange(N, dtype=np.int32), mean

@@ -1,0 +1,53 @@
+"""Pins for the oracle's centroid-guided grouping (one group per contiguous parent, routed by the
+arithmetic mean of its keys, stored as a bf16 value)."""
+import numpy as np
+
+from oracle import santapp_oracle as orc
+from paper_2609_35629_b200 import synth
+
+
+def test_hand_worked_parents():
+    k = np.arange(24, dtype=np.float64).reshape(6, 4)                # rows 0..5, parents of 4: {0..3}, {4, 5}
+    ts, tm, mean = orc.group_mean_keys(k, 4)
+    assert ts.tolist() == [0, 4, 6] and tm.tolist() == list(range(6))
+    assert np.array_equal(mean, np.array([[6., 7., 8., 9.], [18., 19., 20., 21.]]))
+
+
+def test_groups_of_one_key_are_the_keys():
+    """P = 1: the mean of a single bf16 key is the key itself, so the variant coincides with
+    every-key-its-own-team routing (the SANTA limit) and its routing KL is zero."""
+    rng = np.random.default_rng(0)
+    k = synth.bf16_to_f64(synth.f32_to_bf16_bits(rng.normal(size=(50, 16)).astype(np.float32)))
+    ts, tm, mean = orc.group_mean_keys(k, 1)
+    assert np.array_equal(mean, k) and ts.tolist() == list(range(51))
+    q = rng.normal(size=16)
+    assert abs(orc.routing_kl(q, k, ts, tm, mean, 0.25)) < 1e-12
+
+
+def test_mean_is_rounded_to_a_bf16_value_to_nearest():
+    rng = np.random.default_rng(1)
+    k = synth.bf16_to_f64(synth.f32_to_bf16_bits(rng.normal(size=(37, 8)).astype(np.float32)))
+    P = 10
+    ts, tm, mean = orc.group_mean_keys(k, P)
+    assert ts.tolist() == [0, 10, 20, 30, 37]
+    for u in range(4):
+        exact = k[ts[u]:ts[u + 1]].mean(axis=0)
+        # a bf16 value: its float32 bit pattern has a zero low half
+        bits = mean[u].astype(np.float32).view(np.uint32)
+        assert np.all(bits & 0xFFFF == 0) and np.array_equal(mean[u].astype(np.float32).astype(np.float64), mean[u])
+        # nearest: within half a unit in the last place (8 significant bits) of the exact mean
+        assert np.all(np.abs(mean[u] - exact) <= 2.0 ** -8 * np.abs(exact) + 1e-300)
+        # and equal to the independent rounding helper of the input generators
+        want = synth.bf16_to_f64(synth.f32_to_bf16_bits(exact.astype(np.float32)))
+        assert np.array_equal(mean[u], want)
+
+
+def test_decode_with_mean_keys_keeps_the_dense_limit():
+    """Algorithm 1 does not care what the routing key is: with K >= M it still returns dense attention."""
+    rng = np.random.default_rng(2)
+    k = synth.bf16_to_f64(synth.f32_to_bf16_bits(rng.normal(size=(64, 16)).astype(np.float32)))
+    v = rng.normal(size=(64, 16))
+    q = rng.normal(size=16)
+    ts, tm, mean = orc.group_mean_keys(k, 8)
+    r = orc.decode_head_given_gumbel(q, k, v, ts, tm, mean, None, None, 8, None, 0.25)
+    assert np.allclose(r.o, orc.dense_head(q, k, v, 0.25), rtol=0, atol=1e-12)
