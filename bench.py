@@ -590,14 +590,19 @@ def cpu_baseline_leg(spec, data, teams, seed):
     extra = {"sparse_1_thread_us": few(sparse_1, 3), "dense_all_cores_us": few(dense_n(cores), 5),
              "dense_1_thread_us": few(dense_n(1), 2)}
     # routing agreement with dense attention over the prompt (Eq. diagnostic-kl), no sampling involved:
-    # mean over the heads of two of the step inputs
-    kls = []
+    # mean over the heads of two of the step inputs, for the workload's teams and for the
+    # centroid-guided baseline (groups of 4 and of 16 contiguous keys routed by their mean key)
+    variants = {"teams": [(ts[j], tm[j], rk[j]) for j in range(n_kv)]}
+    for size in (4, 16):
+        variants[f"centroid_groups_of_{size}"] = [orc.group_mean_keys(k[j], size) for j in range(n_kv)]
+    kls = {name: [] for name in variants}
     for i in range(2):
         q, _, _, _ = inputs(i * 100)
         for h in range(spec.n_q_heads):
             j = h // spec.group
-            kls.append(orc.routing_kl(q[h], k[j], ts[j], tm[j], rk[j], scale))
-    extra["routing_kl_nats_mean"] = float(np.mean(kls))
+            for name, recs in variants.items():
+                kls[name].append(orc.routing_kl(q[h], k[j], recs[j][0], recs[j][1], recs[j][2], scale))
+    extra["routing_kl_nats_mean"] = {name: float(np.mean(v)) for name, v in kls.items()}
     return {"value": us, "unit": UNIT, "cores": cores, "kind": "oracle",
             "sample": f"{n} layer-steps of sequence 0, layer 0 ({spec.n_q_heads} heads, {r1 - r0} prompt rows), "
                       f"fp64 oracle with OpenMP over heads", **extra}

@@ -164,6 +164,23 @@ int santapp_build_teams(const santapp_geom *geom, const int32_t *prompt_len_host
                         santapp_teams *teams, void *workspace, size_t workspace_bytes,
                         santapp_stream stream);
 
+/*
+ * Centroid-guided grouping, the baseline the paper's routing diagnostic compares the team variant
+ * with (Section "How closely routing follows dense attention"; appendix on the KL variants): one
+ * group per parent, routed by the arithmetic mean of its keys instead of an actual key; routing
+ * logit, sampling, correction and estimator are those of Algorithm 1, so the records are consumed by
+ * santapp_decode_attn unchanged. The paper forms the groups by k-means; this call uses the
+ * contiguous parents of Algorithm 4 (group size = geom->parent_size, last one possibly short).
+ * The mean of a parent is the fp64 sum of its keys in token order divided by their number, stored
+ * as bf16 (fp64 to fp32 to nearest, fp32 to bf16 to nearest even). Rows keep their token order.
+ * geom->reps_per_parent must be 1 (sizes then come from santapp_build_teams_sizes as usual).
+ * Arguments, ownership and errors as for santapp_build_teams.
+ */
+int santapp_build_groups_mean(const santapp_geom *geom, const int32_t *prompt_len_host,
+                              const void *k_prompt, const void *v_prompt,
+                              santapp_teams *teams, void *workspace, size_t workspace_bytes,
+                              santapp_stream stream);
+
 /* Workspace bytes santapp_decode_attn needs for n_sample = K on these team records. */
 size_t santapp_decode_workspace_bytes(const santapp_geom *geom, const santapp_teams *teams,
                                       int32_t n_sample);

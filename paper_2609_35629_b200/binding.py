@@ -29,7 +29,7 @@ EXPORTS = [
     "santapp_version", "santapp_strerror", "santapp_last_cuda_error", "santapp_build_teams_sizes",
     "santapp_build_teams", "santapp_decode_workspace_bytes", "santapp_decode_attn",
     "santapp_dense_workspace_bytes", "santapp_dense_decode_attn", "santapp_last_launch_count",
-    "santapp_set_stage_mask", "santapp_dense_decode_attn_noalloc",
+    "santapp_set_stage_mask", "santapp_dense_decode_attn_noalloc", "santapp_build_groups_mean",
 ]
 
 STAGE_ROUTE, STAGE_SELECT, STAGE_ATTEND, STAGE_ALL = 1, 2, 4, 7
@@ -92,6 +92,8 @@ def load_library(path: Optional[str] = None):
     L.santapp_build_teams.argtypes = [ctypes.POINTER(CGeom), ctypes.POINTER(i32), vp, vp,
                                       ctypes.POINTER(CTeams), vp, sz, vp]
     L.santapp_build_teams.restype = ctypes.c_int
+    L.santapp_build_groups_mean.argtypes = L.santapp_build_teams.argtypes
+    L.santapp_build_groups_mean.restype = ctypes.c_int
     L.santapp_decode_workspace_bytes.argtypes = [ctypes.POINTER(CGeom), ctypes.POINTER(CTeams), i32]
     L.santapp_decode_workspace_bytes.restype = sz
     L.santapp_dense_workspace_bytes.argtypes = [ctypes.POINTER(CGeom), ctypes.POINTER(CTeams)]
@@ -203,8 +205,15 @@ def santapp_build_teams_sizes(geom: Geometry, prompt_len) -> Sizes:
                  out.team_row_start_elems, out.build_workspace_bytes)
 
 
+def santapp_build_groups_mean(geom: Geometry, prompt_len, k_prompt: torch.Tensor, v_prompt: torch.Tensor,
+                              stream=None) -> Teams:
+    """Centroid-guided grouping: one group per contiguous parent, routed by its mean key
+    (geom.reps_per_parent must be 1). Arguments as for santapp_build_teams."""
+    return santapp_build_teams(geom, prompt_len, k_prompt, v_prompt, stream, _entry="santapp_build_groups_mean")
+
+
 def santapp_build_teams(geom: Geometry, prompt_len, k_prompt: torch.Tensor, v_prompt: torch.Tensor,
-                        stream=None) -> Teams:
+                        stream=None, _entry: str = "santapp_build_teams") -> Teams:
     """k_prompt, v_prompt: bf16 CUDA tensors [n_kv_heads, rows_total, d] in token order."""
     L = load_library()
     sizes = santapp_build_teams_sizes(geom, prompt_len)
@@ -213,8 +222,8 @@ def santapp_build_teams(geom: Geometry, prompt_len, k_prompt: torch.Tensor, v_pr
     n = len(prompt_len)
     arr = (ctypes.c_int32 * n)(*[int(x) for x in prompt_len])
     g = geom.c()
-    _check(L.santapp_build_teams(ctypes.byref(g), arr, _ptr(k_prompt), _ptr(v_prompt), ctypes.byref(teams.c),
-                                 _ptr(ws), ws.numel(), _stream_ptr(stream)))
+    _check(getattr(L, _entry)(ctypes.byref(g), arr, _ptr(k_prompt), _ptr(v_prompt), ctypes.byref(teams.c),
+                              _ptr(ws), ws.numel(), _stream_ptr(stream)))
     teams._build_ws = ws      # keep alive until the stream has consumed it
     return teams
 

@@ -181,9 +181,14 @@ int santapp_build_teams_sizes(const santapp_geom *geom, const int32_t *prompt_le
     return SANTAPP_OK;
 }
 
-int santapp_build_teams(const santapp_geom *geom, const int32_t *prompt_len_host, const void *k_prompt,
-                        const void *v_prompt, santapp_teams *teams, void *workspace, size_t workspace_bytes,
-                        santapp_stream stream)
+}  // extern "C"
+
+namespace {
+
+// Both builders: checks, offset tables, host scalars, then the kernels of the chosen grouping.
+int build_records(const santapp_geom *geom, const int32_t *prompt_len_host, const void *k_prompt,
+                  const void *v_prompt, santapp_teams *teams, void *workspace, size_t workspace_bytes,
+                  santapp_stream stream, bool mean_groups)
 {
     santapp_sizes sz;
     int rc = santapp_build_teams_sizes(geom, prompt_len_host, &sz);
@@ -237,11 +242,30 @@ int santapp_build_teams(const santapp_geom *geom, const int32_t *prompt_len_host
     p.row_token = teams->row_token;
     p.owner = static_cast<uint16_t *>(workspace);
     p.max_parents_per_seq = max_parents;
-    err = launch_build_teams(p, s);
-    if (err != cudaSuccess) return cuda_fail(err, "build_teams launch");
+    err = mean_groups ? launch_build_groups_mean(p, s) : launch_build_teams(p, s);
+    if (err != cudaSuccess) return cuda_fail(err, "build launch");
     err = launch_rep_abs_max(p.bv, p.rep_keys, teams->rep_abs_max, s);
     if (err != cudaSuccess) return cuda_fail(err, "rep_abs_max launch");
     return SANTAPP_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int santapp_build_teams(const santapp_geom *geom, const int32_t *prompt_len_host, const void *k_prompt,
+                        const void *v_prompt, santapp_teams *teams, void *workspace, size_t workspace_bytes,
+                        santapp_stream stream)
+{
+    return build_records(geom, prompt_len_host, k_prompt, v_prompt, teams, workspace, workspace_bytes, stream, false);
+}
+
+int santapp_build_groups_mean(const santapp_geom *geom, const int32_t *prompt_len_host, const void *k_prompt,
+                              const void *v_prompt, santapp_teams *teams, void *workspace, size_t workspace_bytes,
+                              santapp_stream stream)
+{
+    if (geom && geom->reps_per_parent != 1) return SANTAPP_ERR_INVALID_ARG;    // one group per parent
+    return build_records(geom, prompt_len_host, k_prompt, v_prompt, teams, workspace, workspace_bytes, stream, true);
 }
 
 size_t santapp_decode_workspace_bytes(const santapp_geom *geom, const santapp_teams *teams, int32_t n_sample)

@@ -256,7 +256,53 @@ size_t build_parent_smem(int P)
            + sizeof(int) * 3 * (size_t)P + (size_t)P + 16;
 }
 
+// Centroid-guided baseline of the paper's routing diagnostic, on the contiguous parents of
+// Algorithm 4: one group per parent, routed by the arithmetic mean of its keys. A block per
+// (parent, sequence, KV head), a thread per dimension: the mean is the fp64 sum in token order
+// divided by the count, stored like every routing key as bf16 (fp64 -> fp32 to nearest, then
+// fp32 -> bf16 to nearest even). Rows keep their token order, so the packed copies are copies.
+__global__ void __launch_bounds__(kHeadDim)
+group_mean_kernel(BuildParams p)
+{
+    const int parent = blockIdx.x, b = blockIdx.y, j = blockIdx.z, d = threadIdx.x;
+    const int64_t row0 = p.bv.seq_row_off[b];
+    const int N = (int)(p.bv.seq_row_off[b + 1] - row0);
+    const int n_parents = (N + p.parent_size - 1) / p.parent_size;
+    if (parent >= n_parents) return;
+    const int lo = parent * p.parent_size, hi = min(lo + p.parent_size, N);
+    const size_t plane = (size_t)j * p.bv.rows_total + (size_t)row0;
+    const uint16_t *k = p.k_prompt + plane * kHeadDim;
+    double sum = 0.0;
+    for (int i = lo; i < hi; ++i) sum = __dadd_rn(sum, bf16_to_double(k[(size_t)i * kHeadDim + d]));
+    const float f = __double2float_rn(__ddiv_rn(sum, (double)(hi - lo)));
+    const uint32_t bits = __float_as_uint(f);
+    const int64_t team0 = p.bv.seq_team_off[b];                     // one team per parent
+    p.rep_keys[((size_t)j * p.bv.teams_total + (size_t)team0 + parent) * kHeadDim + d] =
+        (uint16_t)((bits + 0x7FFFu + ((bits >> 16) & 1u)) >> 16);
+    int32_t *csr = p.team_row_start + (size_t)j * (p.bv.teams_total + p.bv.n_seqs) + team0 + b;
+    if (d == 0) {
+        csr[parent] = lo;
+        if (parent == n_parents - 1) csr[n_parents] = N;
+    }
+    for (int i = lo + d; i < hi; i += kHeadDim) p.row_token[plane + i] = i;
+    const uint4 *ks = reinterpret_cast<const uint4 *>(p.k_prompt + (plane + lo) * kHeadDim);
+    const uint4 *vs = reinterpret_cast<const uint4 *>(p.v_prompt + (plane + lo) * kHeadDim);
+    uint4 *kd = reinterpret_cast<uint4 *>(p.k_packed + (plane + lo) * kHeadDim);
+    uint4 *vd = reinterpret_cast<uint4 *>(p.v_packed + (plane + lo) * kHeadDim);
+    for (int idx = d; idx < (hi - lo) * (kHeadDim / 8); idx += kHeadDim) {
+        kd[idx] = ks[idx];
+        vd[idx] = vs[idx];
+    }
+}
+
 }  // namespace
+
+cudaError_t launch_build_groups_mean(const BuildParams &p, cudaStream_t s)
+{
+    dim3 grid(p.max_parents_per_seq, p.bv.n_seqs, p.bv.n_kv);
+    group_mean_kernel<<<grid, kHeadDim, 0, s>>>(p);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_build_teams(const BuildParams &p, cudaStream_t s)
 {

@@ -160,6 +160,7 @@ struct BuildParams {
     int max_parents_per_seq;
 };
 cudaError_t launch_build_teams(const BuildParams &p, cudaStream_t s);
+cudaError_t launch_build_groups_mean(const BuildParams &p, cudaStream_t s);
 
 // ---------------------------------------------------------------------------------------------
 // Device helpers

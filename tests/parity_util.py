@@ -23,14 +23,14 @@ def geometry(spec: synth.WorkloadSpec) -> sp.Geometry:
 class GpuLayer:
     """One layer's buffers on the GPU plus host copies of the team records."""
 
-    def __init__(self, spec, data, device="cuda"):
+    def __init__(self, spec, data, device="cuda", builder=None):
         self.spec, self.data = spec, data
         self.geom = geometry(spec)
         self.k_prompt = sp.bf16_bits_to_cuda(data.k_prompt, device)
         self.v_prompt = sp.bf16_bits_to_cuda(data.v_prompt, device)
         self.k_suffix = sp.bf16_bits_to_cuda(data.k_suffix, device)
         self.v_suffix = sp.bf16_bits_to_cuda(data.v_suffix, device)
-        self.teams = sp.santapp_build_teams(self.geom, spec.prompt_len, self.k_prompt, self.v_prompt)
+        self.teams = (builder or sp.santapp_build_teams)(self.geom, spec.prompt_len, self.k_prompt, self.v_prompt)
         torch.cuda.synchronize()
         t = self.teams
         self.team_row_start = t.team_row_start.cpu().numpy()

@@ -257,6 +257,32 @@ def test_keys_in_runs_variant():
     check_dense_step(layer, 0)
 
 
+def test_centroid_guided_groups():
+    """Groups routed by their mean key (one group per contiguous parent): records equal to the
+    oracle's, bit for bit, and a decode step on them matches the oracle like any other."""
+    import dataclasses
+    spec = dataclasses.replace(synth.spec_small_gqa(prompt=(2048, 1100)), parent_size=16, reps_per_parent=1,
+                               n_sample=24)
+    data = synth.make_layer(spec)
+    layer = pu.GpuLayer(spec, data, builder=sp.santapp_build_groups_mean)
+    for b in range(spec.n_seqs):
+        r0, r1 = int(layer.seq_row_off[b]), int(layer.seq_row_off[b + 1])
+        for j in range(spec.n_kv_heads):
+            ts_o, tm_o, mean_o = orc.group_mean_keys(synth.bf16_to_f64(data.k_prompt[j, r0:r1]), spec.parent_size)
+            ts_g, tm_g, rep_g = layer.records(b, j)
+            assert np.array_equal(ts_g, ts_o) and np.array_equal(tm_g, tm_o)
+            assert np.array_equal(rep_g, mean_o)
+            assert np.array_equal(layer.k_packed_bits[j, r0:r1], data.k_prompt[j, r0:r1])
+            assert np.array_equal(layer.v_packed_bits[j, r0:r1], data.v_prompt[j, r0:r1])
+    for step in range(2):
+        check_sparse_step(layer, step, K=24)
+    check_dense_step(layer, 0)
+    # the builder insists on one group per parent
+    bad = sp.Geometry(spec.n_seqs, spec.n_q_heads, spec.n_kv_heads, spec.head_dim, 16, 4)
+    with pytest.raises(sp.SantappError):
+        sp.santapp_build_groups_mean(bad, spec.prompt_len, layer.k_prompt, layer.v_prompt)
+
+
 def test_paper_operating_point_32k():
     """Parents of 16 keys with 4 representatives at 32K (8192 teams of about 4 rows per KV head),
     31 sampled teams, no suffix: routing reads an eighth of the dense bytes, gathers are tiny."""
