@@ -153,6 +153,57 @@ def test_decode_k_at_least_m_equals_dense():
         check_sparse_step(layer, step, K=int(Ms.min()))
 
 
+def test_stream_base_and_64_bit_seed():
+    """The sequence stream is stream_base + sequence index, and both halves of the seed key the draw."""
+    layer = layer_for("small", synth.spec_small_gqa)
+    check_sparse_step(layer, 1, K=8, seed=(0xDEADBEEF << 32) | 0x12345678, stream_base=7)
+    spec = layer.spec
+    q_bits = synth.make_queries(spec, layer.data, 1)
+    sl = spec.suffix_len(1)
+    _, d0 = pu.gpu_step(layer, q_bits, sl, 8, 5, 1, stream_base=0)
+    _, d1 = pu.gpu_step(layer, q_bits, sl, 8, 5, 1, stream_base=1)
+    _, d2 = pu.gpu_step(layer, q_bits, sl, 8, 5 | (1 << 40), 1, stream_base=0)
+    s0, s1, s2 = (d.sel_idx.cpu().numpy() for d in (d0, d1, d2))
+    assert not np.array_equal(s0, s1) and not np.array_equal(s0, s2)
+
+
+def test_scale_override():
+    """An explicit logit scale replaces 1 / sqrt(d) in routing and in attention alike."""
+    layer = layer_for("small", synth.spec_small_gqa)
+    spec = layer.spec
+    q_bits = synth.make_queries(spec, layer.data, 0)
+    sl = spec.suffix_len(0)
+    scale = 0.05
+    q = sp.bf16_bits_to_cuda(q_bits)
+    dbg = sp.DebugBuffers(layer.geom, 8, "cuda")
+    out = sp.santapp_decode_attn(layer.geom, layer.teams, q, layer.k_suffix, layer.v_suffix,
+                                 torch.from_numpy(sl).cuda(), 8, 3, 0, scale=scale, debug=dbg).cpu().numpy()
+    dense = sp.santapp_dense_decode_attn(layer.geom, layer.teams, q, layer.k_suffix, layer.v_suffix,
+                                         torch.from_numpy(sl).cuda(), scale=scale).cpu().numpy()
+    vmax = pu.max_abs_v(layer)
+    for b in range(spec.n_seqs):
+        oi = layer.oracle_inputs(b)
+        t = int(sl[b])
+        ks = synth.bf16_to_f64(layer.data.k_suffix[b, :, :t]) if t else None
+        vs = synth.bf16_to_f64(layer.data.v_suffix[b, :, :t]) if t else None
+        qf = synth.bf16_to_f64(q_bits[b])
+        # float32(0.05) is what the library receives
+        r = orc.decode_step(qf, oi["k"], oi["v"], oi["M"], oi["ts"], oi["tm"], oi["rk"], ks, vs, 8, 3, 0, b,
+                            float(np.float32(scale)))
+        assert np.array_equal(dbg.sel_idx.cpu().numpy()[b], r.sel)
+        assert np.abs(out[b] - r.o).max() <= SPARSE_TOL * vmax
+        o_d = orc.dense_step(qf, oi["k"], oi["v"], ks, vs, float(np.float32(scale)))
+        assert np.abs(dense[b] - o_d).max() <= DENSE_TOL * vmax
+
+
+@pytest.mark.parametrize("P,R", [(512, 64), (32, 2), (64, 64), (100, 10)])
+def test_team_records_other_parent_shapes(P, R):
+    spec = synth.spec_small_gqa(prompt=(1300, 700), parent_size=P, reps=R)
+    layer = pu.GpuLayer(spec, synth.make_layer(spec))
+    check_team_records(layer, kv_heads=[0, 3])
+    check_sparse_step(layer, 0, K=4)
+
+
 def test_decode_one_team_left_out():
     """K = M - 1, the smallest sampled case: tau is the single excluded team's score."""
     layer = layer_for("small", synth.spec_small_gqa)
