@@ -26,6 +26,10 @@
  *   orc_routing_kl            routing-agreement diagnostic, Eq. (diagnostic-kl)
  *   orc_group_mean_keys       centroid-guided baseline of the routing diagnostic: one group per
  *                             parent, routed by the arithmetic mean of its keys
+ *   orc_kmeans_parent_count, orc_nearest_centre_parents
+ *                             Algorithm 3 without the fit: the number of centres, and the
+ *                             nearest-centre partition with empty parents omitted (the
+ *                             centres are an input)
  *
  * Parity pins (tests marked "not gpu"): Philox words against an independent
  * library generator; Gumbel law by Kolmogorov-Smirnov and moments; first-draw
@@ -36,7 +40,8 @@
  * hand-worked parents and duplicate keys; the accounting helpers against the
  * figures the paper prints; the routing KL against its closed forms (zero for
  * singleton teams, log N - H(p) for one team holding every key) and against a
- * numpy re-evaluation of the defining sum.
+ * numpy re-evaluation of the defining sum; the nearest-centre partition against a library
+ * vector quantiser, hand-worked ties and empty centres, and brute force over all labellings.
  * Parity unpinned: nothing in this file. (Accuracy of the sampled output
  * against dense attention on real model data is outside what can be pinned
  * here; only the estimator identities are.)
@@ -617,6 +622,52 @@ int32_t orc_group_mean_keys(int32_t N, int d, const double *keys, int32_t P, dou
             memcpy(&back, &rounded, sizeof back);
             out_mean[(int64_t)u * d + j] = (double)back;
         }
+    }
+    return n_parents;
+}
+
+/* ------------------------------------------------------------------------- */
+/* Algorithm 3: parents from fitted centres                                  */
+/* ------------------------------------------------------------------------- */
+
+/* First line of Algorithm 3: the number of centres requested from the fit,
+ * M_parent = min(N, max(2, floor(N / P))), for N >= 2. */
+int32_t orc_kmeans_parent_count(int32_t N, int32_t P)
+{
+    int32_t m = N / P;
+    if (m < 2) m = 2;
+    if (m > N) m = N;
+    return m;
+}
+
+/* Last two lines of Algorithm 3. The centres mu_u are an input (the fit that
+ * produces them, MiniBatchKMeans with the paper's settings, is a library
+ * routine outside this file). Every key joins its nearest centre in squared
+ * Euclidean distance, ties going to the smaller centre index; parents without
+ * a key are omitted, the others keep the order of their centres.
+ *   keys[N][d], centres[n_centres][d]
+ *   label[N]                          centre index of each token
+ *   parent_start[n_parents + 1], parent_member[N]   index lists, tokens increasing
+ * Returns the number of non-empty parents. */
+int32_t orc_nearest_centre_parents(int32_t N, int d, const double *keys,
+                                   int32_t n_centres, const double *centres,
+                                   int32_t *label, int32_t *parent_start, int32_t *parent_member)
+{
+    for (int32_t i = 0; i < N; ++i) {
+        double best = INFINITY; int32_t arg = 0;
+        for (int32_t u = 0; u < n_centres; ++u) {
+            double dist = sqdist(keys + (int64_t)i * d, centres + (int64_t)u * d, d);
+            if (dist < best) { best = dist; arg = u; }
+        }
+        label[i] = arg;
+    }
+    int32_t n_parents = 0, filled = 0;
+    parent_start[0] = 0;
+    for (int32_t u = 0; u < n_centres; ++u) {
+        int32_t before = filled;
+        for (int32_t i = 0; i < N; ++i)
+            if (label[i] == u) parent_member[filled++] = i;
+        if (filled > before) parent_start[++n_parents] = filled;
     }
     return n_parents;
 }

@@ -85,6 +85,10 @@ def lib():
         L.orc_routing_kl.restype = _c.c_double
         L.orc_group_mean_keys.argtypes = [_c.c_int32, _c.c_int, _f64p, _c.c_int32, _f64p]
         L.orc_group_mean_keys.restype = _c.c_int32
+        L.orc_kmeans_parent_count.argtypes = [_c.c_int32, _c.c_int32]
+        L.orc_kmeans_parent_count.restype = _c.c_int32
+        L.orc_nearest_centre_parents.argtypes = [_c.c_int32, _c.c_int, _f64p, _c.c_int32, _f64p, _i32p, _i32p, _i32p]
+        L.orc_nearest_centre_parents.restype = _c.c_int32
         _lib = L
     return _lib
 
@@ -325,3 +329,21 @@ def group_mean_keys(keys, P):
     got = lib().orc_group_mean_keys(N, d, keys, P, mean)
     assert got == n_parents
     return contiguous_parents(N, P), np.arange(N, dtype=np.int32), mean
+
+
+def kmeans_parent_count(N, P):
+    """First line of Algorithm 3: min(N, max(2, N // P))."""
+    return int(lib().orc_kmeans_parent_count(N, P))
+
+
+def nearest_centre_parents(keys, centres):
+    """Last two lines of Algorithm 3 for given centres. Returns (label[N], parent_start, parent_member):
+    nearest centre per token (ties to the smaller centre index) and the non-empty parents as index
+    lists in centre order, tokens increasing."""
+    keys, centres = _f64(keys), _f64(centres)
+    N, d = keys.shape
+    label = np.zeros(N, dtype=np.int32)
+    parent_start = np.zeros(centres.shape[0] + 1, dtype=np.int32)
+    parent_member = np.zeros(N, dtype=np.int32)
+    n = lib().orc_nearest_centre_parents(N, d, keys, centres.shape[0], centres, label, parent_start, parent_member)
+    return label, parent_start[: n + 1].copy(), parent_member
