@@ -98,6 +98,14 @@ typedef struct santapp_teams {
     int64_t *seq_team_off;     /* int64 [n_seqs + 1] device copy of the team offsets                 */
     float *rep_abs_max;        /* fp32  [n_kv_heads][n_seqs]: largest |element| among the pair's
                                   representative keys (bounds the fp32 routing pass)                 */
+    int32_t *team_count;       /* int32 [n_kv_heads][n_seqs], or NULL: the number of teams M of each
+                                  (sequence, KV head). The offsets above reserve the same number of
+                                  team slots for every KV head of a sequence; a pair whose parents
+                                  yield fewer teams (santapp_build_teams_parents) uses the first M
+                                  slots, and the slots behind them are empty teams (row offset =
+                                  prompt length, representative key zero) that the decode ignores.
+                                  NULL means every slot holds a team. Written by every builder
+                                  when not NULL.                                                    */
     int64_t rows_total;        /* host scalars, as in santapp_sizes                                  */
     int64_t teams_total;
     int32_t max_teams_per_seq;
@@ -180,6 +188,58 @@ int santapp_build_groups_mean(const santapp_geom *geom, const int32_t *prompt_le
                               const void *k_prompt, const void *v_prompt,
                               santapp_teams *teams, void *workspace, size_t workspace_bytes,
                               santapp_stream stream);
+
+/*
+ * Algorithm 3 (global k-means parents), first line: the number of centres to fit for a prompt of
+ * prompt_len >= 2 keys and nominal parent size P: min(prompt_len, max(2, prompt_len / P)).
+ * Returns 0 for arguments outside that range. Host arithmetic only.
+ */
+int32_t santapp_kmeans_parent_count(int32_t prompt_len, int32_t parent_size);
+
+/*
+ * Algorithm 3, the assignment that follows the fit: every key joins its nearest centre, squared
+ * Euclidean distance evaluated in fp64 on the raw keys, ties going to the smaller centre index.
+ * The centres are an input: fitting them (minibatch k-means with the paper's settings) is left to
+ * the caller's clustering routine.
+ *   n_centres_host   host int32 [n_seqs], in: centres of sequence b (>= 1), the same for every KV head
+ *   k_prompt         device bf16 [n_kv_heads][rows_total][d], token order, in
+ *   centres          device fp32 [n_kv_heads][sum_b n_centres[b]][d], in: sequence b's centres
+ *                    start at the sum of the earlier sequences' counts
+ *   parent_of        device int32 [n_kv_heads][rows_total], out: centre index (local to the
+ *                    sequence) of each token; a centre that attracts no token simply does not occur
+ *   workspace        device, >= santapp_assign_parents_workspace_bytes(geom) (offset tables)
+ */
+size_t santapp_assign_parents_workspace_bytes(const santapp_geom *geom);
+int santapp_assign_parents(const santapp_geom *geom, const int32_t *prompt_len_host,
+                           const int32_t *n_centres_host, const void *k_prompt, const float *centres,
+                           int32_t *parent_of, void *workspace, size_t workspace_bytes,
+                           santapp_stream stream);
+
+/*
+ * Sizes for team records built from an arbitrary parent partition: sequence b, whose tokens carry
+ * parent labels in [0, n_parents[b]), gets min(prompt_len[b], n_parents[b] * R) team slots per KV
+ * head (a parent of c tokens yields min(R, c) teams; empty parents yield none).
+ * geom->parent_size is not used by the parent-based calls beyond the general checks.
+ */
+int santapp_parent_teams_sizes(const santapp_geom *geom, const int32_t *prompt_len_host,
+                               const int32_t *n_parents_host, santapp_sizes *out);
+
+/*
+ * Build the team records of one layer from a given parent partition (the partition Algorithm 3
+ * returns, or any other): Algorithm 2 on parents of any size. Parents are ordered by label, labels
+ * without a token are omitted, and each (sequence, KV head) has its own partition, so the number of
+ * teams may differ between the KV heads of a sequence: teams->team_count (required here) receives
+ * it, and unused slots are left as empty teams.
+ *   n_parents_host   host int32 [n_seqs], in: size of sequence b's label range (>= 1)
+ *   parent_of        device int32 [n_kv_heads][rows_total], in: label of each token, local to its
+ *                    sequence; values outside [0, n_parents[b]) are clamped into the range
+ *   teams, workspace as for santapp_build_teams, with sizes from santapp_parent_teams_sizes
+ * Arithmetic, tie rules and the packed layout are those of santapp_build_teams.
+ */
+int santapp_build_teams_parents(const santapp_geom *geom, const int32_t *prompt_len_host,
+                                const int32_t *n_parents_host, const void *k_prompt,
+                                const void *v_prompt, const int32_t *parent_of, santapp_teams *teams,
+                                void *workspace, size_t workspace_bytes, santapp_stream stream);
 
 /* Workspace bytes santapp_decode_attn needs for n_sample = K on these team records. */
 size_t santapp_decode_workspace_bytes(const santapp_geom *geom, const santapp_teams *teams,

@@ -30,6 +30,8 @@ EXPORTS = [
     "santapp_build_teams", "santapp_decode_workspace_bytes", "santapp_decode_attn",
     "santapp_dense_workspace_bytes", "santapp_dense_decode_attn", "santapp_last_launch_count",
     "santapp_set_stage_mask", "santapp_dense_decode_attn_noalloc", "santapp_build_groups_mean",
+    "santapp_kmeans_parent_count", "santapp_assign_parents_workspace_bytes", "santapp_assign_parents",
+    "santapp_parent_teams_sizes", "santapp_build_teams_parents",
 ]
 
 STAGE_ROUTE, STAGE_SELECT, STAGE_ATTEND, STAGE_ALL = 1, 2, 4, 7
@@ -57,7 +59,7 @@ class CTeams(ctypes.Structure):
     _fields_ = [("k_packed", ctypes.c_void_p), ("v_packed", ctypes.c_void_p), ("rep_keys", ctypes.c_void_p),
                 ("team_row_start", ctypes.c_void_p), ("row_token", ctypes.c_void_p),
                 ("seq_row_off", ctypes.c_void_p), ("seq_team_off", ctypes.c_void_p),
-                ("rep_abs_max", ctypes.c_void_p),
+                ("rep_abs_max", ctypes.c_void_p), ("team_count", ctypes.c_void_p),
                 ("rows_total", ctypes.c_int64), ("teams_total", ctypes.c_int64),
                 ("max_teams_per_seq", ctypes.c_int32), ("max_rows_per_seq", ctypes.c_int32)]
 
@@ -94,6 +96,19 @@ def load_library(path: Optional[str] = None):
     L.santapp_build_teams.restype = ctypes.c_int
     L.santapp_build_groups_mean.argtypes = L.santapp_build_teams.argtypes
     L.santapp_build_groups_mean.restype = ctypes.c_int
+    L.santapp_kmeans_parent_count.argtypes = [i32, i32]
+    L.santapp_kmeans_parent_count.restype = i32
+    L.santapp_assign_parents_workspace_bytes.argtypes = [ctypes.POINTER(CGeom)]
+    L.santapp_assign_parents_workspace_bytes.restype = sz
+    L.santapp_assign_parents.argtypes = [ctypes.POINTER(CGeom), ctypes.POINTER(i32), ctypes.POINTER(i32), vp, vp, vp,
+                                         vp, sz, vp]
+    L.santapp_assign_parents.restype = ctypes.c_int
+    L.santapp_parent_teams_sizes.argtypes = [ctypes.POINTER(CGeom), ctypes.POINTER(i32), ctypes.POINTER(i32),
+                                             ctypes.POINTER(CSizes)]
+    L.santapp_parent_teams_sizes.restype = ctypes.c_int
+    L.santapp_build_teams_parents.argtypes = [ctypes.POINTER(CGeom), ctypes.POINTER(i32), ctypes.POINTER(i32), vp, vp,
+                                              vp, ctypes.POINTER(CTeams), vp, sz, vp]
+    L.santapp_build_teams_parents.restype = ctypes.c_int
     L.santapp_decode_workspace_bytes.argtypes = [ctypes.POINTER(CGeom), ctypes.POINTER(CTeams), i32]
     L.santapp_decode_workspace_bytes.restype = sz
     L.santapp_dense_workspace_bytes.argtypes = [ctypes.POINTER(CGeom), ctypes.POINTER(CTeams)]
@@ -176,10 +191,11 @@ class Teams:
         self.seq_row_off = torch.empty(geom.n_seqs + 1, dtype=torch.int64, device=device)
         self.seq_team_off = torch.empty(geom.n_seqs + 1, dtype=torch.int64, device=device)
         self.rep_abs_max = torch.empty((kv, geom.n_seqs), dtype=torch.float32, device=device)
+        self.team_count = torch.empty((kv, geom.n_seqs), dtype=torch.int32, device=device)
         self.c = CTeams(self.k_packed.data_ptr(), self.v_packed.data_ptr(), self.rep_keys.data_ptr(),
                         self.team_row_start.data_ptr(), self.row_token.data_ptr(),
                         self.seq_row_off.data_ptr(), self.seq_team_off.data_ptr(), self.rep_abs_max.data_ptr(),
-                        sizes.rows_total, sizes.teams_total, sizes.max_teams_per_seq, sizes.max_rows_per_seq)
+                        self.team_count.data_ptr(), sizes.rows_total, sizes.teams_total, sizes.max_teams_per_seq, sizes.max_rows_per_seq)
 
 
 def santapp_version() -> int:
@@ -224,6 +240,59 @@ def santapp_build_teams(geom: Geometry, prompt_len, k_prompt: torch.Tensor, v_pr
     g = geom.c()
     _check(getattr(L, _entry)(ctypes.byref(g), arr, _ptr(k_prompt), _ptr(v_prompt), ctypes.byref(teams.c),
                               _ptr(ws), ws.numel(), _stream_ptr(stream)))
+    teams._build_ws = ws      # keep alive until the stream has consumed it
+    return teams
+
+
+def _i32_array(values):
+    return (ctypes.c_int32 * len(values))(*[int(x) for x in values])
+
+
+def santapp_kmeans_parent_count(prompt_len: int, parent_size: int) -> int:
+    """First line of Algorithm 3: min(N, max(2, N // P)); 0 for N < 2 or P < 1."""
+    return int(load_library().santapp_kmeans_parent_count(int(prompt_len), int(parent_size)))
+
+
+def santapp_assign_parents(geom: Geometry, prompt_len, n_centres, k_prompt: torch.Tensor, centres: torch.Tensor,
+                           stream=None) -> torch.Tensor:
+    """Nearest-centre label of every token. centres: fp32 CUDA tensor [n_kv_heads, sum(n_centres), d].
+    Returns int32 [n_kv_heads, rows_total]."""
+    L = load_library()
+    g = geom.c()
+    if centres.dtype != torch.float32:
+        raise SantappError(SANTAPP_ERR_INVALID_ARG, "centres must be float32")
+    parent_of = torch.empty((geom.n_kv_heads, k_prompt.shape[1]), dtype=torch.int32, device=k_prompt.device)
+    ws = torch.empty(max(int(L.santapp_assign_parents_workspace_bytes(ctypes.byref(g))), 256), dtype=torch.uint8,
+                     device=k_prompt.device)
+    _check(L.santapp_assign_parents(ctypes.byref(g), _i32_array(prompt_len), _i32_array(n_centres), _ptr(k_prompt),
+                                    _ptr(centres), _ptr(parent_of), _ptr(ws), ws.numel(), _stream_ptr(stream)))
+    parent_of._ws = ws
+    return parent_of
+
+
+def santapp_parent_teams_sizes(geom: Geometry, prompt_len, n_parents) -> Sizes:
+    L = load_library()
+    out = CSizes()
+    g = geom.c()
+    _check(L.santapp_parent_teams_sizes(ctypes.byref(g), _i32_array(prompt_len), _i32_array(n_parents),
+                                        ctypes.byref(out)))
+    return Sizes(out.rows_total, out.teams_total, out.max_teams_per_seq, out.max_rows_per_seq,
+                 out.team_row_start_elems, out.build_workspace_bytes)
+
+
+def santapp_build_teams_parents(geom: Geometry, prompt_len, n_parents, k_prompt: torch.Tensor,
+                                v_prompt: torch.Tensor, parent_of: torch.Tensor, stream=None) -> Teams:
+    """Team records from a parent label per token (int32 CUDA tensor [n_kv_heads, rows_total])."""
+    L = load_library()
+    sizes = santapp_parent_teams_sizes(geom, prompt_len, n_parents)
+    teams = Teams(geom, sizes, k_prompt.device)
+    ws = torch.empty(max(sizes.build_workspace_bytes, 256), dtype=torch.uint8, device=k_prompt.device)
+    g = geom.c()
+    if parent_of.dtype != torch.int32:
+        raise SantappError(SANTAPP_ERR_INVALID_ARG, "parent_of must be int32")
+    _check(L.santapp_build_teams_parents(ctypes.byref(g), _i32_array(prompt_len), _i32_array(n_parents),
+                                         _ptr(k_prompt), _ptr(v_prompt), _ptr(parent_of), ctypes.byref(teams.c),
+                                         _ptr(ws), ws.numel(), _stream_ptr(stream)))
     teams._build_ws = ws      # keep alive until the stream has consumed it
     return teams
 

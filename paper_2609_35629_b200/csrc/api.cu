@@ -55,7 +55,7 @@ int check_teams(const santapp_geom *g, const santapp_teams *t)
         return SANTAPP_ERR_INVALID_ARG;
     if (misaligned(t->k_packed, 16) || misaligned(t->v_packed, 16) || misaligned(t->rep_keys, 16)
         || misaligned(t->team_row_start, 4) || misaligned(t->row_token, 4) || misaligned(t->seq_row_off, 8)
-        || misaligned(t->seq_team_off, 8) || misaligned(t->rep_abs_max, 4))
+        || misaligned(t->seq_team_off, 8) || misaligned(t->rep_abs_max, 4) || misaligned(t->team_count, 4))
         return SANTAPP_ERR_INVALID_ARG;
     if (t->rows_total < g->n_seqs || t->teams_total < g->n_seqs || t->max_teams_per_seq < 1)
         return SANTAPP_ERR_INVALID_ARG;
@@ -73,6 +73,7 @@ BatchView make_view(const santapp_geom *g, const santapp_teams *t)
     bv.group = g->n_q_heads / g->n_kv_heads;
     bv.seq_row_off = t->seq_row_off;
     bv.seq_team_off = t->seq_team_off;
+    bv.team_count = t->team_count;
     bv.rows_total = t->rows_total;
     bv.teams_total = t->teams_total;
     return bv;
@@ -200,7 +201,8 @@ int build_records(const santapp_geom *geom, const int32_t *prompt_len_host, cons
     if (misaligned(k_prompt, 16) || misaligned(v_prompt, 16) || misaligned(workspace, 16)
         || misaligned(teams->k_packed, 16) || misaligned(teams->v_packed, 16) || misaligned(teams->rep_keys, 16)
         || misaligned(teams->team_row_start, 4) || misaligned(teams->row_token, 4) || misaligned(teams->seq_row_off, 8)
-        || misaligned(teams->seq_team_off, 8) || misaligned(teams->rep_abs_max, 4))
+        || misaligned(teams->seq_team_off, 8) || misaligned(teams->rep_abs_max, 4)
+        || misaligned(teams->team_count, 4))
         return SANTAPP_ERR_INVALID_ARG;
     if (workspace_bytes < sz.build_workspace_bytes) return SANTAPP_ERR_WORKSPACE_TOO_SMALL;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -240,6 +242,7 @@ int build_records(const santapp_geom *geom, const int32_t *prompt_len_host, cons
     p.rep_keys = static_cast<uint16_t *>(teams->rep_keys);
     p.team_row_start = teams->team_row_start;
     p.row_token = teams->row_token;
+    p.team_count = teams->team_count;
     p.owner = static_cast<uint16_t *>(workspace);
     p.max_parents_per_seq = max_parents;
     err = mean_groups ? launch_build_groups_mean(p, s) : launch_build_teams(p, s);
@@ -250,6 +253,212 @@ int build_records(const santapp_geom *geom, const int32_t *prompt_len_host, cons
 }
 
 }  // namespace
+
+namespace {
+
+// Workspace of santapp_build_teams_parents. Offsets in bytes.
+struct ParentLayout {
+    size_t label_off, parent_start, parent_cursor, parent_team_base, members, team_of, mind, owner, is_rep,
+        team_cursor, dest, total;
+};
+
+ParentLayout parent_layout(int n_seqs, int n_kv, int64_t rows_total, int64_t labels_total, int64_t teams_total)
+{
+    ParentLayout L;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
+    const size_t H = (size_t)n_kv, R = (size_t)rows_total, Lt = (size_t)labels_total;
+    L.label_off = take(sizeof(int64_t) * ((size_t)n_seqs + 1));
+    L.parent_start = take(sizeof(int32_t) * H * (Lt + (size_t)n_seqs));
+    L.parent_cursor = take(sizeof(int32_t) * H * Lt);
+    L.parent_team_base = take(sizeof(int32_t) * H * Lt);
+    L.members = take(sizeof(int32_t) * H * R);
+    L.team_of = take(sizeof(int32_t) * H * R);
+    L.mind = take(sizeof(double) * H * R);
+    L.owner = take(sizeof(int32_t) * H * R);
+    L.is_rep = take(H * R);
+    L.team_cursor = take(sizeof(int32_t) * H * (size_t)teams_total);
+    L.dest = take(sizeof(int32_t) * H * R);
+    L.total = off;
+    return L;
+}
+
+}  // namespace
+
+extern "C" {
+
+int32_t santapp_kmeans_parent_count(int32_t prompt_len, int32_t parent_size)
+{
+    if (prompt_len < 2 || parent_size < 1) return 0;
+    int32_t m = prompt_len / parent_size;
+    if (m < 2) m = 2;
+    if (m > prompt_len) m = prompt_len;
+    return m;
+}
+
+size_t santapp_assign_parents_workspace_bytes(const santapp_geom *geom)
+{
+    if (check_geom(geom) != SANTAPP_OK) return 0;
+    return 2 * align_up(sizeof(int64_t) * ((size_t)geom->n_seqs + 1));
+}
+
+int santapp_assign_parents(const santapp_geom *geom, const int32_t *prompt_len_host, const int32_t *n_centres_host,
+                           const void *k_prompt, const float *centres, int32_t *parent_of, void *workspace,
+                           size_t workspace_bytes, santapp_stream stream)
+{
+    int rc = check_geom(geom);
+    if (rc != SANTAPP_OK) return rc;
+    if (!prompt_len_host || !n_centres_host || !k_prompt || !centres || !parent_of || !workspace)
+        return SANTAPP_ERR_INVALID_ARG;
+    if (misaligned(k_prompt, 16) || misaligned(centres, 4) || misaligned(parent_of, 4) || misaligned(workspace, 16))
+        return SANTAPP_ERR_INVALID_ARG;
+    if (workspace_bytes < santapp_assign_parents_workspace_bytes(geom)) return SANTAPP_ERR_WORKSPACE_TOO_SMALL;
+    std::vector<int64_t> offs(2 * ((size_t)geom->n_seqs + 1));
+    int64_t *row_off = offs.data(), *cen_off = offs.data() + geom->n_seqs + 1;
+    row_off[0] = cen_off[0] = 0;
+    int max_rows = 0;
+    for (int b = 0; b < geom->n_seqs; ++b) {
+        if (prompt_len_host[b] < 1 || n_centres_host[b] < 1) return SANTAPP_ERR_INVALID_ARG;
+        row_off[b + 1] = row_off[b] + prompt_len_host[b];
+        cen_off[b + 1] = cen_off[b] + n_centres_host[b];
+        if (prompt_len_host[b] > max_rows) max_rows = prompt_len_host[b];
+    }
+    if (row_off[geom->n_seqs] >= (int64_t)1 << 31) return SANTAPP_ERR_UNSUPPORTED;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    g_cuda_error[0] = 0;
+    const size_t ob = sizeof(int64_t) * ((size_t)geom->n_seqs + 1);
+    unsigned char *ws = static_cast<unsigned char *>(workspace);
+    int64_t *d_row_off = reinterpret_cast<int64_t *>(ws);
+    int64_t *d_cen_off = reinterpret_cast<int64_t *>(ws + align_up(ob));
+    cudaError_t err = cudaMemcpyAsync(d_row_off, row_off, ob, cudaMemcpyHostToDevice, s);
+    if (err != cudaSuccess) return cuda_fail(err, "copy row offsets");
+    err = cudaMemcpyAsync(d_cen_off, cen_off, ob, cudaMemcpyHostToDevice, s);
+    if (err != cudaSuccess) return cuda_fail(err, "copy centre offsets");
+    AssignParams p;
+    p.n_seqs = geom->n_seqs;
+    p.n_kv = geom->n_kv_heads;
+    p.max_rows_per_seq = max_rows;
+    p.rows_total = row_off[geom->n_seqs];
+    p.centres_total = cen_off[geom->n_seqs];
+    p.seq_row_off = d_row_off;
+    p.seq_centre_off = d_cen_off;
+    p.k_prompt = static_cast<const uint16_t *>(k_prompt);
+    p.centres = centres;
+    p.parent_of = parent_of;
+    err = launch_assign_parents(p, s);
+    if (err != cudaSuccess) return cuda_fail(err, "assign_parents launch");
+    return SANTAPP_OK;
+}
+
+int santapp_parent_teams_sizes(const santapp_geom *geom, const int32_t *prompt_len_host, const int32_t *n_parents_host,
+                               santapp_sizes *out)
+{
+    int rc = check_geom(geom);
+    if (rc != SANTAPP_OK) return rc;
+    if (!prompt_len_host || !n_parents_host || !out) return SANTAPP_ERR_INVALID_ARG;
+    memset(out, 0, sizeof(*out));
+    int64_t labels_total = 0;
+    for (int b = 0; b < geom->n_seqs; ++b) {
+        const int N = prompt_len_host[b];
+        if (N < 1 || n_parents_host[b] < 1) return SANTAPP_ERR_INVALID_ARG;
+        const int64_t want = (int64_t)n_parents_host[b] * geom->reps_per_parent;
+        const int M = (int)(want < N ? want : N);
+        labels_total += n_parents_host[b];
+        out->rows_total += N;
+        out->teams_total += M;
+        if (M > out->max_teams_per_seq) out->max_teams_per_seq = M;
+        if (N > out->max_rows_per_seq) out->max_rows_per_seq = N;
+    }
+    if (out->rows_total >= (int64_t)1 << 31 || labels_total >= (int64_t)1 << 31) return SANTAPP_ERR_UNSUPPORTED;
+    out->team_row_start_elems = (int64_t)geom->n_kv_heads * (out->teams_total + geom->n_seqs);
+    out->build_workspace_bytes =
+        parent_layout(geom->n_seqs, geom->n_kv_heads, out->rows_total, labels_total, out->teams_total).total;
+    return SANTAPP_OK;
+}
+
+int santapp_build_teams_parents(const santapp_geom *geom, const int32_t *prompt_len_host, const int32_t *n_parents_host,
+                                const void *k_prompt, const void *v_prompt, const int32_t *parent_of,
+                                santapp_teams *teams, void *workspace, size_t workspace_bytes, santapp_stream stream)
+{
+    santapp_sizes sz;
+    int rc = santapp_parent_teams_sizes(geom, prompt_len_host, n_parents_host, &sz);
+    if (rc != SANTAPP_OK) return rc;
+    if (!k_prompt || !v_prompt || !parent_of || !teams || !workspace) return SANTAPP_ERR_INVALID_ARG;
+    if (!teams->k_packed || !teams->v_packed || !teams->rep_keys || !teams->team_row_start || !teams->row_token
+        || !teams->seq_row_off || !teams->seq_team_off || !teams->rep_abs_max || !teams->team_count)
+        return SANTAPP_ERR_INVALID_ARG;
+    if (misaligned(k_prompt, 16) || misaligned(v_prompt, 16) || misaligned(workspace, 16) || misaligned(parent_of, 4)
+        || misaligned(teams->k_packed, 16) || misaligned(teams->v_packed, 16) || misaligned(teams->rep_keys, 16)
+        || misaligned(teams->team_row_start, 4) || misaligned(teams->row_token, 4) || misaligned(teams->seq_row_off, 8)
+        || misaligned(teams->seq_team_off, 8) || misaligned(teams->rep_abs_max, 4)
+        || misaligned(teams->team_count, 4))
+        return SANTAPP_ERR_INVALID_ARG;
+    if (workspace_bytes < sz.build_workspace_bytes) return SANTAPP_ERR_WORKSPACE_TOO_SMALL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    g_cuda_error[0] = 0;
+
+    const int B = geom->n_seqs;
+    std::vector<int64_t> offs(3 * ((size_t)B + 1));
+    int64_t *row_off = offs.data(), *team_off = row_off + B + 1, *label_off = team_off + B + 1;
+    row_off[0] = team_off[0] = label_off[0] = 0;
+    int max_labels = 0;
+    for (int b = 0; b < B; ++b) {
+        const int N = prompt_len_host[b];
+        const int64_t want = (int64_t)n_parents_host[b] * geom->reps_per_parent;
+        row_off[b + 1] = row_off[b] + N;
+        team_off[b + 1] = team_off[b] + (want < N ? want : N);
+        label_off[b + 1] = label_off[b] + n_parents_host[b];
+        if (n_parents_host[b] > max_labels) max_labels = n_parents_host[b];
+    }
+    const ParentLayout L = parent_layout(B, geom->n_kv_heads, sz.rows_total, label_off[B], sz.teams_total);
+    unsigned char *ws = static_cast<unsigned char *>(workspace);
+    const size_t ob = sizeof(int64_t) * ((size_t)B + 1);
+    cudaError_t err = cudaMemcpyAsync(teams->seq_row_off, row_off, ob, cudaMemcpyHostToDevice, s);
+    if (err != cudaSuccess) return cuda_fail(err, "copy seq_row_off");
+    err = cudaMemcpyAsync(teams->seq_team_off, team_off, ob, cudaMemcpyHostToDevice, s);
+    if (err != cudaSuccess) return cuda_fail(err, "copy seq_team_off");
+    err = cudaMemcpyAsync(ws + L.label_off, label_off, ob, cudaMemcpyHostToDevice, s);
+    if (err != cudaSuccess) return cuda_fail(err, "copy label offsets");
+
+    teams->rows_total = sz.rows_total;
+    teams->teams_total = sz.teams_total;
+    teams->max_teams_per_seq = sz.max_teams_per_seq;
+    teams->max_rows_per_seq = sz.max_rows_per_seq;
+
+    ParentBuildParams p;
+    p.bv = make_view(geom, teams);
+    p.reps = geom->reps_per_parent;
+    p.max_labels_per_seq = max_labels;
+    p.max_rows_per_seq = sz.max_rows_per_seq;
+    p.labels_total = label_off[B];
+    p.k_prompt = static_cast<const uint16_t *>(k_prompt);
+    p.v_prompt = static_cast<const uint16_t *>(v_prompt);
+    p.parent_of = parent_of;
+    p.seq_label_off = reinterpret_cast<const int64_t *>(ws + L.label_off);
+    p.k_packed = static_cast<uint16_t *>(teams->k_packed);
+    p.v_packed = static_cast<uint16_t *>(teams->v_packed);
+    p.rep_keys = static_cast<uint16_t *>(teams->rep_keys);
+    p.team_row_start = teams->team_row_start;
+    p.row_token = teams->row_token;
+    p.team_count = teams->team_count;
+    p.parent_start = reinterpret_cast<int32_t *>(ws + L.parent_start);
+    p.parent_cursor = reinterpret_cast<int32_t *>(ws + L.parent_cursor);
+    p.parent_team_base = reinterpret_cast<int32_t *>(ws + L.parent_team_base);
+    p.members = reinterpret_cast<int32_t *>(ws + L.members);
+    p.team_of = reinterpret_cast<int32_t *>(ws + L.team_of);
+    p.mind = reinterpret_cast<double *>(ws + L.mind);
+    p.owner = reinterpret_cast<int32_t *>(ws + L.owner);
+    p.is_rep = ws + L.is_rep;
+    p.team_cursor = reinterpret_cast<int32_t *>(ws + L.team_cursor);
+    p.dest = reinterpret_cast<int32_t *>(ws + L.dest);
+    err = launch_build_teams_parents(p, s);
+    if (err != cudaSuccess) return cuda_fail(err, "build_teams_parents launch");
+    err = launch_rep_abs_max(p.bv, p.rep_keys, teams->rep_abs_max, s);
+    if (err != cudaSuccess) return cuda_fail(err, "rep_abs_max launch");
+    return SANTAPP_OK;
+}
+
+}  // extern "C"
 
 extern "C" {
 

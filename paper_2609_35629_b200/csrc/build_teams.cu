@@ -4,6 +4,7 @@
 // separate multiply and add, so that exact ties fall the way the paper's tie rules say.
 #include <limits.h>
 
+#include "build_util.cuh"
 #include "common.cuh"
 
 namespace santapp {
@@ -12,50 +13,6 @@ namespace {
 
 constexpr int kBuildThreads = 256;
 constexpr int kRowWords = 65;            // 64 data words + 1 pad word: conflict-free column walks
-
-struct ValIdx {
-    double v;
-    int i;
-};
-
-template <bool kMin>
-__device__ __forceinline__ ValIdx pick(const ValIdx &a, const ValIdx &b)
-{
-    bool take_b;
-    if (kMin) take_b = (b.v < a.v) || (b.v == a.v && b.i < a.i);
-    else      take_b = (b.v > a.v) || (b.v == a.v && b.i < a.i);
-    return take_b ? b : a;
-}
-
-// Block-wide arg-min / arg-max; ties go to the smaller index. Result valid in every thread.
-template <bool kMin>
-__device__ ValIdx block_arg(ValIdx x, ValIdx *scratch /* [33] */)
-{
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        ValIdx y;
-        y.v = __shfl_xor_sync(0xFFFFFFFFu, x.v, o);
-        y.i = __shfl_xor_sync(0xFFFFFFFFu, x.i, o);
-        x = pick<kMin>(x, y);
-    }
-    __syncthreads();
-    if (lane == 0) scratch[warp] = x;
-    __syncthreads();
-    if (warp == 0) {
-        ValIdx y = scratch[lane < n_warps ? lane : 0];
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            ValIdx z;
-            z.v = __shfl_xor_sync(0xFFFFFFFFu, y.v, o);
-            z.i = __shfl_xor_sync(0xFFFFFFFFu, y.i, o);
-            y = pick<kMin>(y, z);
-        }
-        if (lane == 0) scratch[32] = y;
-    }
-    __syncthreads();
-    return scratch[32];
-}
 
 // Squared distance between row `i` (shared memory, bf16 words) and a reference vector in fp64,
 // summed over dimensions in increasing order, multiply and add rounded separately.
@@ -193,6 +150,7 @@ scan_team_sizes_kernel(BuildParams p)
     const int64_t team0 = p.bv.seq_team_off[b];
     const int M = (int)(p.bv.seq_team_off[b + 1] - team0);
     int32_t *csr = p.team_row_start + (size_t)j * (p.bv.teams_total + p.bv.n_seqs) + team0 + b + 1;
+    if (threadIdx.x == 0 && p.team_count) p.team_count[(size_t)j * p.bv.n_seqs + b] = M;   // every slot is a team
     int carry = 0;
     for (int base = 0; base < M; base += kBuildThreads) {
         const int g = base + threadIdx.x;
@@ -283,6 +241,7 @@ group_mean_kernel(BuildParams p)
     if (d == 0) {
         csr[parent] = lo;
         if (parent == n_parents - 1) csr[n_parents] = N;
+        if (parent == 0 && p.team_count) p.team_count[(size_t)j * p.bv.n_seqs + b] = n_parents;
     }
     for (int i = lo + d; i < hi; i += kHeadDim) p.row_token[plane + i] = i;
     const uint4 *ks = reinterpret_cast<const uint4 *>(p.k_prompt + (plane + lo) * kHeadDim);

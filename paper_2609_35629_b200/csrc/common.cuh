@@ -25,9 +25,17 @@ constexpr int kPartialStride = 132;     // floats per (slot, head): m, l, 2 pad,
 struct BatchView {
     int n_seqs, n_q, n_kv, group;
     const int64_t *seq_row_off;     // [n_seqs + 1]
-    const int64_t *seq_team_off;    // [n_seqs + 1]
+    const int64_t *seq_team_off;    // [n_seqs + 1] team slots of each sequence
+    const int32_t *team_count;      // [n_kv][n_seqs] teams a pair really has, or null: every slot is a team
     int64_t rows_total, teams_total;
 };
+
+// Teams of (sequence b, KV head j): the first `pair_team_count` slots of the sequence's range.
+__device__ __forceinline__ int pair_team_count(const BatchView &bv, int b, int j)
+{
+    return bv.team_count ? bv.team_count[(size_t)j * bv.n_seqs + b]
+                         : (int)(bv.seq_team_off[b + 1] - bv.seq_team_off[b]);
+}
 
 // Read plan of one (sequence, KV head) pair: the union of the teams its query heads selected,
 // in ascending team id, optionally followed by one suffix segment.
@@ -156,11 +164,48 @@ struct BuildParams {
     const uint16_t *k_prompt, *v_prompt;    // [n_kv][rows_total][128] token order
     uint16_t *k_packed, *v_packed, *rep_keys;
     int32_t *team_row_start, *row_token;
+    int32_t *team_count;                    // [n_kv][n_seqs] or null
     uint16_t *owner;                        // workspace [n_kv][rows_total]: team index inside the parent
     int max_parents_per_seq;
 };
 cudaError_t launch_build_teams(const BuildParams &p, cudaStream_t s);
 cudaError_t launch_build_groups_mean(const BuildParams &p, cudaStream_t s);
+
+// Nearest-centre assignment (last step of Algorithm 3).
+struct AssignParams {
+    int n_seqs, n_kv, max_rows_per_seq;
+    int64_t rows_total, centres_total;
+    const int64_t *seq_row_off;             // device [n_seqs + 1]
+    const int64_t *seq_centre_off;          // device [n_seqs + 1]
+    const uint16_t *k_prompt;               // [n_kv][rows_total][128]
+    const float *centres;                   // [n_kv][centres_total][128]
+    int32_t *parent_of;                     // [n_kv][rows_total] out
+};
+cudaError_t launch_assign_parents(const AssignParams &p, cudaStream_t s);
+
+// Team records from an arbitrary parent partition given as one label per token.
+struct ParentBuildParams {
+    BatchView bv;                           // seq_team_off: team slots per sequence
+    int reps, max_labels_per_seq, max_rows_per_seq;
+    int64_t labels_total;
+    const uint16_t *k_prompt, *v_prompt;    // [n_kv][rows_total][128] token order
+    const int32_t *parent_of;               // [n_kv][rows_total] label of each token
+    const int64_t *seq_label_off;           // device [n_seqs + 1]
+    uint16_t *k_packed, *v_packed, *rep_keys;
+    int32_t *team_row_start, *row_token, *team_count;
+    // workspace
+    int32_t *parent_start;                  // [n_kv][labels_total + n_seqs] member-list offsets
+    int32_t *parent_cursor;                 // [n_kv][labels_total] counts, then scatter cursors
+    int32_t *parent_team_base;              // [n_kv][labels_total] first team of each parent
+    int32_t *members;                       // [n_kv][rows_total] tokens ordered by (label, index)
+    int32_t *team_of;                       // [n_kv][rows_total] team of each token
+    double *mind;                           // [n_kv][rows_total] distance to the nearest representative
+    int32_t *owner;                         // [n_kv][rows_total] its rank inside the parent
+    unsigned char *is_rep;                  // [n_kv][rows_total]
+    int32_t *team_cursor;                   // [n_kv][teams_total]
+    int32_t *dest;                          // [n_kv][rows_total] packed position of each token
+};
+cudaError_t launch_build_teams_parents(const ParentBuildParams &p, cudaStream_t s);
 
 // ---------------------------------------------------------------------------------------------
 // Device helpers

@@ -63,7 +63,7 @@ headplan_kernel(PlanInputs in)
     const int b = hq / in.bv.n_q, hh = hq - b * in.bv.n_q;            // hh = j * G + h
     const int j = hh / in.bv.group;
     const int64_t team0 = in.bv.seq_team_off[b];
-    const int M = (int)(in.bv.seq_team_off[b + 1] - team0);
+    const int M = pair_team_count(in.bv, b, j);
     const int K = in.n_sample;
     if (K >= M) return;                                               // every team is read with c = 1: nothing is drawn
 

@@ -56,8 +56,7 @@ __device__ __forceinline__ void build_pair_plan(const PlanInputs &in, int pair, 
             ent_rows[u] = in.sel_rows[at];
         }
     }
-    const int64_t team0 = in.bv.seq_team_off[b];
-    const int M = (int)(in.bv.seq_team_off[b + 1] - team0);
+    const int M = pair_team_count(in.bv, b, j);
     const int64_t row0 = in.bv.seq_row_off[b];
     const int N = (int)(in.bv.seq_row_off[b + 1] - row0);
     const int Ke = min(K, M);

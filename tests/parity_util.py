@@ -40,10 +40,12 @@ class GpuLayer:
         self.v_packed_bits = t.v_packed.view(torch.int16).cpu().numpy().view(np.uint16)
         self.seq_row_off = t.seq_row_off.cpu().numpy()
         self.seq_team_off = t.seq_team_off.cpu().numpy()
+        self.team_count = t.team_count.cpu().numpy()
 
     def records(self, b, j):
         """(team_start[M+1], team_member[N], rep_key[M, d] fp64) of sequence b, KV head j."""
-        t0, t1 = int(self.seq_team_off[b]), int(self.seq_team_off[b + 1])
+        t0 = int(self.seq_team_off[b])
+        t1 = t0 + int(self.team_count[j, b])          # the pair's teams; later slots of the sequence are empty
         r0, r1 = int(self.seq_row_off[b]), int(self.seq_row_off[b + 1])
         ts = self.team_row_start[j, t0 + b: t1 + b + 1].astype(np.int32)
         tm = self.row_token[j, r0:r1].astype(np.int32)

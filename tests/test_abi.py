@@ -87,7 +87,7 @@ def test_misaligned_pointers_are_refused_on_the_host(lib):
     before any launch (fake addresses: nothing is dereferenced)."""
     g = sp.Geometry(1, 28, 4).c()
     A = 0x10000                                                     # an aligned fake address
-    t = sp.CTeams(A, A, A, A, A, A, A, A, 32768, 2048, 2048, 32768)
+    t = sp.CTeams(A, A, A, A, A, A, A, A, A, 32768, 2048, 2048, 32768)
     args = dict(q=A, out=A, ws=A)
 
     def decode(q=A, out=A, ws=A, teams=t):
@@ -97,7 +97,7 @@ def test_misaligned_pointers_are_refused_on_the_host(lib):
     assert decode(q=A + 2) == sp.SANTAPP_ERR_INVALID_ARG
     assert decode(out=A + 4) == sp.SANTAPP_ERR_INVALID_ARG
     assert decode(ws=A + 8) == sp.SANTAPP_ERR_INVALID_ARG
-    bad = sp.CTeams(A + 2, A, A, A, A, A, A, A, 32768, 2048, 2048, 32768)
+    bad = sp.CTeams(A + 2, A, A, A, A, A, A, A, A, 32768, 2048, 2048, 32768)
     assert decode(teams=bad) == sp.SANTAPP_ERR_INVALID_ARG
     # aligned pointers pass the checks and fail later only because the workspace is too small
     assert decode() == sp.SANTAPP_ERR_WORKSPACE_TOO_SMALL
@@ -105,7 +105,7 @@ def test_misaligned_pointers_are_refused_on_the_host(lib):
 
 def test_workspace_queries(lib):
     g = sp.Geometry(1, 28, 4)
-    t = sp.CTeams(1, 1, 1, 1, 1, 1, 1, 1, 32768, 8192, 2048, 32768)
+    t = sp.CTeams(1, 1, 1, 1, 1, 1, 1, 1, 0, 32768, 8192, 2048, 32768)
     ws32 = lib.santapp_decode_workspace_bytes(ctypes.byref(g.c()), ctypes.byref(t), 32)
     ws64 = lib.santapp_decode_workspace_bytes(ctypes.byref(g.c()), ctypes.byref(t), 64)
     wsd = lib.santapp_dense_workspace_bytes(ctypes.byref(g.c()), ctypes.byref(t))
@@ -117,3 +117,39 @@ def test_workspace_queries(lib):
 def test_missing_library_fails_loudly(tmp_path):
     with pytest.raises(sp.SantappError):
         sp.load_library(str(tmp_path / "libsantapp.so"))
+
+
+@pytest.mark.parametrize("N,P,want", [(32768, 512, 64), (1000, 16, 62), (3, 16, 2), (5, 1, 5), (1, 16, 0), (8, 0, 0)])
+def test_kmeans_parent_count_is_the_first_line_of_algorithm_3(lib, N, P, want):
+    assert sp.santapp_kmeans_parent_count(N, P) == want
+
+
+def test_parent_teams_sizes(lib):
+    g = sp.Geometry(2, 28, 4, 128, 16, 4)
+    sz = sp.santapp_parent_teams_sizes(g, [1000, 10], [62, 5])
+    assert sz.rows_total == 1010
+    assert sz.teams_total == 62 * 4 + 10              # min(N, parents * R) slots per sequence
+    assert sz.max_teams_per_seq == 248 and sz.max_rows_per_seq == 1000
+    assert sz.team_row_start_elems == 4 * (sz.teams_total + 2)
+    assert sz.build_workspace_bytes > 25 * 4 * 1010
+    with pytest.raises(sp.SantappError) as e:
+        sp.santapp_parent_teams_sizes(g, [1000, 10], [62, 0])
+    assert e.value.status == sp.SANTAPP_ERR_INVALID_ARG
+
+
+def test_parent_calls_refuse_null_and_misaligned_arguments(lib):
+    g = sp.Geometry(1, 28, 4).c()
+    n = (ctypes.c_int32 * 1)(1024)
+    c = (ctypes.c_int32 * 1)(2)
+    A = 0x10000
+    t = sp.CTeams(A, A, A, A, A, A, A, A, A, 0, 0, 0, 0)
+    assert lib.santapp_assign_parents(ctypes.byref(g), n, c, None, A, A, A, 1 << 20, None) == sp.SANTAPP_ERR_INVALID_ARG
+    assert lib.santapp_assign_parents(ctypes.byref(g), n, c, A + 2, A, A, A, 1 << 20, None) == sp.SANTAPP_ERR_INVALID_ARG
+    assert lib.santapp_assign_parents(ctypes.byref(g), n, c, A, A, A, A, 8, None) == sp.SANTAPP_ERR_WORKSPACE_TOO_SMALL
+    assert lib.santapp_build_teams_parents(ctypes.byref(g), n, c, A, A, None, ctypes.byref(t), A, 1 << 30,
+                                           None) == sp.SANTAPP_ERR_INVALID_ARG
+    no_count = sp.CTeams(A, A, A, A, A, A, A, A, 0, 0, 0, 0, 0)
+    assert lib.santapp_build_teams_parents(ctypes.byref(g), n, c, A, A, A, ctypes.byref(no_count), A, 1 << 30,
+                                           None) == sp.SANTAPP_ERR_INVALID_ARG
+    assert lib.santapp_build_teams_parents(ctypes.byref(g), n, c, A, A, A, ctypes.byref(t), A, 16,
+                                           None) == sp.SANTAPP_ERR_WORKSPACE_TOO_SMALL

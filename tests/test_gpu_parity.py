@@ -64,22 +64,23 @@ def check_sparse_step(layer, step, K, seed=1234, stream_base=0, suffix_len=None,
     union = dbg.union_rows.cpu().numpy()
     vmax = pu.max_abs_v(layer)
     worst = 0.0
+    G = spec.group
     for b, r in ref.items():
-        M = int(layer.seq_team_off[b + 1] - layer.seq_team_off[b])
-        Ke = min(K, M)
-        if Ke < M:
-            assert np.all(r.margin > 1e-9), "seeded workload too close to a selection boundary"
-        assert np.array_equal(sel[b, :, :Ke], r.sel[:, :Ke]), f"sampled teams differ (seq {b}, step {step})"
-        assert np.all(sel[b, :, Ke:] == -1)
-        assert np.allclose(logc[b, :, :Ke], r.logc[:, :Ke], rtol=0, atol=1e-5)
-        if Ke < M:
-            assert np.allclose(tau[b], r.tau, rtol=0, atol=1e-9)
-        else:
-            assert np.all(np.isnan(tau[b]))
         for j in range(spec.n_kv_heads):
             ts, _, _ = layer.records(b, j)
-            G = spec.group
-            assert union[b, j] == orc.union_rows(ts, r.sel[j * G:(j + 1) * G, :Ke])
+            M = len(ts) - 1                                           # teams of this (sequence, KV head)
+            Ke = min(K, M)
+            hs = slice(j * G, (j + 1) * G)
+            if Ke < M:
+                assert np.all(r.margin[hs] > 1e-9), "seeded workload too close to a selection boundary"
+            assert np.array_equal(sel[b, hs, :Ke], r.sel[hs, :Ke]), f"sampled teams differ (seq {b}, step {step})"
+            assert np.all(sel[b, hs, Ke:] == -1)
+            assert np.allclose(logc[b, hs, :Ke], r.logc[hs, :Ke], rtol=0, atol=1e-5)
+            if Ke < M:
+                assert np.allclose(tau[b, hs], r.tau[hs], rtol=0, atol=1e-9)
+            else:
+                assert np.all(np.isnan(tau[b, hs]))
+            assert union[b, j] == orc.union_rows(ts, r.sel[hs, :Ke])
         err = np.abs(out[b] - r.o).max()
         worst = max(worst, err)
         assert err <= SPARSE_TOL * vmax, f"max |delta| {err} > {SPARSE_TOL} * {vmax}"
