@@ -57,6 +57,9 @@ def parse_args():
     ap.add_argument("--n-sample", type=int, default=0, help="override K")
     ap.add_argument("--key-layout", default="iid", choices=["iid", "runs"],
                     help="cluster of each prompt row: independent draws, or geometric runs (positional locality)")
+    ap.add_argument("--parents", default="contiguous", choices=["contiguous", "centres"],
+                    help="contiguous: Algorithm 4; centres: the partition Algorithm 3 returns when the fit "
+                         "recovers the centres the synthetic keys were drawn around")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-stages", action="store_true")
@@ -81,6 +84,7 @@ def make_spec(args, seed):
     if args.n_sample:
         spec.n_sample = args.n_sample
     spec.key_layout = args.key_layout
+    spec.parents = getattr(args, "parents", "contiguous")
     return spec
 
 
@@ -88,7 +92,7 @@ def workload_text(spec, layers):
     return (f"{spec.name}: {spec.n_seqs} seq x {spec.n_q_heads} q heads / {spec.n_kv_heads} KV heads, d={spec.head_dim}, "
             f"prompt {min(spec.prompt_len)}..{max(spec.prompt_len)}, suffix cap {spec.suffix_cap}, "
             f"P={spec.parent_size}, R={spec.reps_per_parent}, K={spec.n_sample}, keys {spec.key_layout}, "
-            f"{layers} layers round-robin")
+            f"{getattr(spec, 'parents', 'contiguous')} parents, {layers} layers round-robin")
 
 
 # -------------------------------------------------------------------------------------------
@@ -269,13 +273,26 @@ def measure_workload(args, workload, n_layers, n_steps, n_warmup, dev, want_e2e,
     ksuf_all = torch.empty((L, B, Hkv, cap, d), dtype=torch.bfloat16, device=dev)
     vsuf_all = torch.empty_like(ksuf_all)
     for l in range(L):
-        data = synth.make_layer(spec, layer=l, keep_centres=conc)
+        by_centres = spec.parents == "centres"
+        data = synth.make_layer(spec, layer=l, keep_centres=conc or by_centres)
         for s in range(N_STEP_INPUTS):
             q_all[s, l] = synth.make_queries(spec, data, s)
         k_prompt = sp.bf16_bits_to_cuda(data.k_prompt, dev)
         v_prompt = sp.bf16_bits_to_cuda(data.v_prompt, dev)
-        teams = sp.santapp_build_teams(geom, spec.prompt_len, k_prompt, v_prompt)
+        if by_centres:
+            # Algorithm 3 with the fit replaced by its ideal outcome on these keys: the centres the
+            # rows were drawn around, as many as its first line asks for
+            n_cen = [min(sp.santapp_kmeans_parent_count(n, spec.parent_size), spec.n_clusters) for n in spec.prompt_len]
+            cen = np.concatenate([data.centres[:, :n] for n in n_cen], axis=1)
+            t_build = time.perf_counter()
+            parent_of = sp.santapp_assign_parents(geom, spec.prompt_len, n_cen, k_prompt,
+                                                  torch.from_numpy(np.ascontiguousarray(cen)).to(dev))
+            teams = sp.santapp_build_teams_parents(geom, spec.prompt_len, n_cen, k_prompt, v_prompt, parent_of)
+        else:
+            t_build = time.perf_counter()
+            teams = sp.santapp_build_teams(geom, spec.prompt_len, k_prompt, v_prompt)
         torch.cuda.synchronize()
+        build_ms = 1e3 * (time.perf_counter() - t_build)
         del k_prompt, v_prompt
         ksuf_all[l].copy_(sp.bf16_bits_to_cuda(data.k_suffix, dev))
         vsuf_all[l].copy_(sp.bf16_bits_to_cuda(data.v_suffix, dev))
@@ -326,7 +343,8 @@ def measure_workload(args, workload, n_layers, n_steps, n_warmup, dev, want_e2e,
     # ---- accounting pass (eager): union rows per (input, layer) -> algorithmic bytes ----
     dbg = sp.DebugBuffers(geom, K, dev)
     union = np.zeros((N_STEP_INPUTS, L), dtype=np.int64)
-    M_total = int(layers[0]["teams"].sizes.teams_total)
+    M_total = int(layers[0]["teams"].sizes.teams_total)                  # team slots per KV head (all are read)
+    teams_real = int(layers[0]["teams"].team_count.sum().item())         # teams over all KV heads
     N_total = int(layers[0]["teams"].sizes.rows_total)
     for s in range(N_STEP_INPUTS):
         set_inputs(s)
@@ -456,7 +474,8 @@ def measure_workload(args, workload, n_layers, n_steps, n_warmup, dev, want_e2e,
         achieved = attend_bytes_1 / (stages["attend"] * 1e-6) / 1e9
         roofline = {"bound": "hbm", "kernel": "attend_kernel", "achieved": achieved, "peak": peak_gbs, "unit": "GB/s",
                     "frac": achieved / peak_gbs,
-                    "traffic": NCU_TRAFFIC_BYTES.get(spec.name) if not args.n_sample and spec.key_layout == "iid" else None,
+                    "traffic": (NCU_TRAFFIC_BYTES.get(spec.name)
+                                if not args.n_sample and spec.key_layout == "iid" and spec.parents == "contiguous" else None),
                     "peak_kind": peak_kind,
                     "algorithmic_bytes_per_launch": attend_bytes_1, "us_per_launch": stages["attend"]}
 
@@ -515,9 +534,9 @@ def measure_workload(args, workload, n_layers, n_steps, n_warmup, dev, want_e2e,
             "dense_achieved_gbs": mean_dense_bytes / (us_layer_dense * 1e-6) / 1e9,
             "dense_achieved_frac_of_peak": mean_dense_bytes / (us_layer_dense * 1e-6) / 1e9 / peak_gbs,
             "attend_bytes_per_layer_step": mean_attend_bytes,
-            "logical_access_pct": 100.0 * float((M_total * Hkv + 2 * (union[used].mean() + suffix_rows[used].mean()))
+            "logical_access_pct": 100.0 * float((teams_real + 2 * (union[used].mean() + suffix_rows[used].mean()))
                                                 / (2 * (Hkv * N_total + suffix_rows[used].mean()))),
-            "stage_us": stages, "paired_rounds": rounds, "prep_seconds": prep_s,
+            "stage_us": stages, "paired_rounds": rounds, "prep_seconds": prep_s, "team_build_ms_last_layer": build_ms,
         }
         return line
     return None
@@ -538,7 +557,7 @@ def cpu_baseline_leg(spec, data, teams, seed):
     rep_bits = teams.rep_keys.view(torch.int16).cpu().numpy().view(np.uint16)
     to = teams.seq_team_off.cpu().numpy()
     t0, t1 = int(to[b]), int(to[b + 1])
-    M = np.full(n_kv, t1 - t0, dtype=np.int32)
+    M = np.ascontiguousarray(teams.team_count.cpu().numpy()[:, b], dtype=np.int32)     # teams of each KV head
     ts = np.ascontiguousarray(trs[:, t0 + b:t1 + b + 1])
     tm = np.ascontiguousarray(tok[:, r0:r1])
     rk = synth.bf16_to_f64(rep_bits[:, t0:t1])

@@ -172,3 +172,41 @@ def test_contiguous_builder_reports_every_slot_as_a_team():
     layer = pu.GpuLayer(spec, synth.make_layer(spec, layer=0))
     want = np.diff(layer.seq_team_off).astype(np.int32)
     assert np.array_equal(layer.team_count, np.tile(want, (spec.n_kv_heads, 1)))
+
+
+def _centre_layer(spec):
+    """The configuration `bench.py --parents centres` times: as many of the generating centres as the
+    first line of Algorithm 3 asks for, assignment and records built on the GPU."""
+    data = synth.make_layer(spec, layer=0, keep_centres=True)
+    n_cen = [min(sp.santapp_kmeans_parent_count(n, spec.parent_size), spec.n_clusters) for n in spec.prompt_len]
+    cen = np.ascontiguousarray(np.concatenate([data.centres[:, :n] for n in n_cen], axis=1))
+    labels = _labels_gpu(spec, data, n_cen, cen)
+    return _layer_from_labels(spec, data, labels, n_cen), labels, n_cen, cen
+
+
+def test_centre_parents_32k_full_size():
+    """Config 2's shape with parents from centres instead of contiguous spans: labels and records of
+    one KV head against the oracle, then decode steps of every head."""
+    spec = synth.spec_qwen_b1()
+    layer, labels, n_cen, cen = _centre_layer(spec)
+    j = 1
+    keys = synth.bf16_to_f64(layer.data.k_prompt[j])
+    want, ps, pm = orc.nearest_centre_parents(keys, cen[j].astype(np.float64))
+    assert np.array_equal(labels[j], want)
+    ts_o, tm_o, rep_o = orc.build_teams(keys, ps, pm, spec.reps_per_parent)
+    ts_g, tm_g, rep_g = layer.records(0, j)
+    assert np.array_equal(ts_g, ts_o) and np.array_equal(tm_g, tm_o) and np.array_equal(rep_g, keys[rep_o])
+    sizes = np.diff(ps)
+    assert sizes.max() > spec.parent_size                      # parents larger than any contiguous one
+    for step in (0, 255):
+        check_sparse_step(layer, step, K=32)
+    check_dense_step(layer, 3)
+
+
+def test_centre_parents_paper_point_32k():
+    """The paper's operating point (P = 16, R = 4, K = 31) on centre parents: 2048 parents of uneven
+    size, a different team count for every KV head."""
+    spec = synth.spec_paper_point()
+    layer, _, _, _ = _centre_layer(spec)
+    assert len({int(c) for c in layer.team_count[:, 0]}) > 1
+    check_sparse_step(layer, 0, K=31)
