@@ -58,6 +58,12 @@ typedef enum santapp_status {
 
 typedef void *santapp_stream;            /* cudaStream_t */
 
+/* 16-bit element type of the inputs. Wherever this header says "bf16" for q, K, V, the suffix or
+ * the representative keys, the tensor holds raw 16-bit patterns of this type. Outputs are fp32 and
+ * every accumulation is fp32 or fp64 for both. The paper's own runs use fp16 inputs
+ * (Appendix "Kernel evaluation protocol and profiling"); santapp_build_groups_mean takes bf16 only. */
+typedef enum santapp_elem { SANTAPP_BF16 = 0, SANTAPP_FP16 = 1 } santapp_elem;
+
 /* Problem geometry (host struct). */
 typedef struct santapp_geom {
     int32_t n_seqs;            /* B: sequences in the batch                         */
@@ -66,6 +72,7 @@ typedef struct santapp_geom {
     int32_t head_dim;          /* d; 128                                           */
     int32_t parent_size;       /* P: nominal parent size (Algorithm 4), <= 512      */
     int32_t reps_per_parent;   /* R: maximum representatives per parent; divides P  */
+    int32_t elem_type;         /* santapp_elem of q, K, V and the representative keys */
 } santapp_geom;
 
 /* Sizes derived from the geometry and the prompt lengths (host struct, output). */

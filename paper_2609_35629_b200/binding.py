@@ -24,6 +24,7 @@ SANTAPP_ERR_WORKSPACE_TOO_SMALL = -3
 SANTAPP_ERR_CUDA = -4
 SANTAPP_ERR_STATIC_SCRATCH = -5
 SANTAPP_STATIC_SCRATCH_BYTES = 2 << 20
+SANTAPP_BF16, SANTAPP_FP16 = 0, 1
 
 EXPORTS = [
     "santapp_version", "santapp_strerror", "santapp_last_cuda_error", "santapp_build_teams_sizes",
@@ -46,7 +47,7 @@ class SantappError(RuntimeError):
 class CGeom(ctypes.Structure):
     _fields_ = [("n_seqs", ctypes.c_int32), ("n_q_heads", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32),
                 ("head_dim", ctypes.c_int32), ("parent_size", ctypes.c_int32),
-                ("reps_per_parent", ctypes.c_int32)]
+                ("reps_per_parent", ctypes.c_int32), ("elem_type", ctypes.c_int32)]
 
 
 class CSizes(ctypes.Structure):
@@ -159,10 +160,15 @@ class Geometry:
     head_dim: int = 128
     parent_size: int = 512
     reps_per_parent: int = 32
+    elem_type: int = 0               # SANTAPP_BF16; 1 = SANTAPP_FP16
 
     def c(self) -> CGeom:
         return CGeom(self.n_seqs, self.n_q_heads, self.n_kv_heads, self.head_dim, self.parent_size,
-                     self.reps_per_parent)
+                     self.reps_per_parent, self.elem_type)
+
+    @property
+    def torch_dtype(self):
+        return torch.float16 if self.elem_type == SANTAPP_FP16 else torch.bfloat16
 
 
 @dataclass
@@ -183,9 +189,9 @@ class Teams:
         kv = geom.n_kv_heads
         self.geom = geom
         self.sizes = sizes
-        self.k_packed = torch.empty((kv, sizes.rows_total, d), dtype=torch.bfloat16, device=device)
+        self.k_packed = torch.empty((kv, sizes.rows_total, d), dtype=geom.torch_dtype, device=device)
         self.v_packed = torch.empty_like(self.k_packed)
-        self.rep_keys = torch.empty((kv, sizes.teams_total, d), dtype=torch.bfloat16, device=device)
+        self.rep_keys = torch.empty((kv, sizes.teams_total, d), dtype=geom.torch_dtype, device=device)
         self.team_row_start = torch.empty((kv, sizes.teams_total + geom.n_seqs), dtype=torch.int32, device=device)
         self.row_token = torch.empty((kv, sizes.rows_total), dtype=torch.int32, device=device)
         self.seq_row_off = torch.empty(geom.n_seqs + 1, dtype=torch.int64, device=device)
@@ -382,8 +388,8 @@ def santapp_dense_decode_attn_noalloc(geom: Geometry, teams: Teams, q: torch.Ten
     return out
 
 
-def bf16_bits_to_cuda(bits, device="cuda"):
-    """numpy uint16 bf16 bit patterns -> CUDA bfloat16 tensor (no value conversion)."""
+def bf16_bits_to_cuda(bits, device="cuda", dtype=torch.bfloat16):
+    """numpy uint16 bit patterns -> CUDA tensor of the 16-bit `dtype` (no value conversion)."""
     import numpy as np
     t = torch.from_numpy(np.ascontiguousarray(bits).view(np.int16))
-    return t.to(device).view(torch.bfloat16)
+    return t.to(device).view(dtype)

@@ -34,6 +34,7 @@ int check_geom(const santapp_geom *g)
     if (g->n_seqs < 1 || g->n_q_heads < 1 || g->n_kv_heads < 1 || g->parent_size < 1 || g->reps_per_parent < 1)
         return SANTAPP_ERR_INVALID_ARG;
     if (g->n_q_heads % g->n_kv_heads != 0) return SANTAPP_ERR_INVALID_ARG;
+    if (g->elem_type != SANTAPP_BF16 && g->elem_type != SANTAPP_FP16) return SANTAPP_ERR_INVALID_ARG;
     if (g->parent_size % g->reps_per_parent != 0) return SANTAPP_ERR_INVALID_ARG;   // R divides P
     if (g->head_dim != kHeadDim) return SANTAPP_ERR_UNSUPPORTED;
     if (g->n_q_heads / g->n_kv_heads > kMaxGroup) return SANTAPP_ERR_UNSUPPORTED;
@@ -74,6 +75,7 @@ BatchView make_view(const santapp_geom *g, const santapp_teams *t)
     bv.seq_row_off = t->seq_row_off;
     bv.seq_team_off = t->seq_team_off;
     bv.team_count = t->team_count;
+    bv.elem = g->elem_type;
     bv.rows_total = t->rows_total;
     bv.teams_total = t->teams_total;
     return bv;
@@ -337,6 +339,7 @@ int santapp_assign_parents(const santapp_geom *geom, const int32_t *prompt_len_h
     AssignParams p;
     p.n_seqs = geom->n_seqs;
     p.n_kv = geom->n_kv_heads;
+    p.elem = geom->elem_type;
     p.max_rows_per_seq = max_rows;
     p.rows_total = row_off[geom->n_seqs];
     p.centres_total = cen_off[geom->n_seqs];
@@ -474,6 +477,7 @@ int santapp_build_groups_mean(const santapp_geom *geom, const int32_t *prompt_le
                               santapp_stream stream)
 {
     if (geom && geom->reps_per_parent != 1) return SANTAPP_ERR_INVALID_ARG;    // one group per parent
+    if (geom && geom->elem_type != SANTAPP_BF16) return SANTAPP_ERR_UNSUPPORTED;
     return build_records(geom, prompt_len_host, k_prompt, v_prompt, teams, workspace, workspace_bytes, stream, true);
 }
 

@@ -71,22 +71,38 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t add
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
                  : "r"(addr));
 }
-// D += A (16x16, row) * B (16x8, col), bf16 inputs, fp32 accumulation.
-__device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
-                                         uint32_t b0, uint32_t b1)
+// D += A (16x16, row) * B (16x8, col), bf16 (or fp16) inputs, fp32 accumulation.
+template <bool kHalf>
+__device__ __forceinline__ void mma_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                          uint32_t b0, uint32_t b1)
 {
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
-                 "{%0,%1,%2,%3};"
-                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+    if constexpr (kHalf)
+        asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+                     "{%0,%1,%2,%3};"
+                     : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                     : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+    else
+        asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+                     "{%0,%1,%2,%3};"
+                     : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                     : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
-// (lo, hi) -> bf16x2 with lo in the low half, round to nearest even.
-__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
+// (lo, hi) -> two 16-bit elements with lo in the low half, round to nearest even.
+template <bool kHalf>
+__device__ __forceinline__ uint32_t pack_x2(float lo, float hi)
 {
     uint32_t r;
-    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    if constexpr (kHalf) asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    else                 asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
     return r;
 }
+// fp16 holds nothing below 2^-24, so the weights of rows that follow a much larger score in the
+// same warp's stream would vanish when they are rounded for the value product (a bounded loss: a
+// warp streams at most a few thousand rows). With fp16 inputs the weights (and with them the
+// running sum and the accumulators, consistently, so the factor cancels in U / Z and in every
+// merge) are carried multiplied by 2^15: the largest is 32768, the smallest kept 2^-39 of the
+// running maximum. bf16 has the exponent range of fp32 and needs no such shift.
+template <bool kHalf> constexpr float kWeightShift = kHalf ? 15.f : 0.f;
 
 // ---- shared memory carve-up (dynamic) ----
 template <int G>
@@ -115,7 +131,7 @@ struct Smem {
     static_assert(total <= 227 * 1024, "shared memory budget");
 };
 
-template <int G, bool kAll, bool kStatic>
+template <int G, bool kAll, bool kStatic, bool kHalf>
 __global__ void __launch_bounds__(kAttendThreads, 1)
 attend_kernel(AttendParams p)
 {
@@ -386,10 +402,10 @@ attend_kernel(AttendParams p)
                     const int ch = 4 * sp + lmat;
                     ldmatrix_x4(kb0, k_addr + lrow * kRowBytes + ((ch ^ lrow) << 4));
                     ldmatrix_x4(kb1, k_addr + (8 + lrow) * kRowBytes + ((ch ^ lrow) << 4));
-                    mma_bf16(s0, qa[2 * sp][0], 0u, qa[2 * sp][1], 0u, kb0[0], kb0[1]);
-                    mma_bf16(s1, qa[2 * sp][0], 0u, qa[2 * sp][1], 0u, kb1[0], kb1[1]);
-                    mma_bf16(s2, qa[2 * sp + 1][0], 0u, qa[2 * sp + 1][1], 0u, kb0[2], kb0[3]);
-                    mma_bf16(s3, qa[2 * sp + 1][0], 0u, qa[2 * sp + 1][1], 0u, kb1[2], kb1[3]);
+                    mma_16816<kHalf>(s0, qa[2 * sp][0], 0u, qa[2 * sp][1], 0u, kb0[0], kb0[1]);
+                    mma_16816<kHalf>(s1, qa[2 * sp][0], 0u, qa[2 * sp][1], 0u, kb1[0], kb1[1]);
+                    mma_16816<kHalf>(s2, qa[2 * sp + 1][0], 0u, qa[2 * sp + 1][1], 0u, kb0[2], kb0[3]);
+                    mma_16816<kHalf>(s3, qa[2 * sp + 1][0], 0u, qa[2 * sp + 1][1], 0u, kb1[2], kb1[3]);
                 }
             }
             float sc[4];
@@ -413,12 +429,12 @@ attend_kernel(AttendParams p)
             }
             float pw[4];
 #pragma unroll
-            for (int e = 0; e < 4; ++e) pw[e] = on[e] ? exp2f(sc[e] - m_run) : 0.f;
+            for (int e = 0; e < 4; ++e) pw[e] = on[e] ? exp2f(sc[e] - m_run + kWeightShift<kHalf>) : 0.f;
             l_run += (pw[0] + pw[1]) + (pw[2] + pw[3]);
             // P^T as B fragments, split in two bf16 terms
-            const uint32_t ph0 = pack_bf16x2(pw[0], pw[1]), ph1 = pack_bf16x2(pw[2], pw[3]);
-            const uint32_t pl0 = pack_bf16x2(pw[0] - bf16_lo(ph0), pw[1] - bf16_hi(ph0));
-            const uint32_t pl1 = pack_bf16x2(pw[2] - bf16_lo(ph1), pw[3] - bf16_hi(ph1));
+            const uint32_t ph0 = pack_x2<kHalf>(pw[0], pw[1]), ph1 = pack_x2<kHalf>(pw[2], pw[3]);
+            const uint32_t pl0 = pack_x2<kHalf>(pw[0] - elem_lo<kHalf>(ph0), pw[1] - elem_hi<kHalf>(ph0));
+            const uint32_t pl1 = pack_x2<kHalf>(pw[2] - elem_lo<kHalf>(ph1), pw[3] - elem_hi<kHalf>(ph1));
 
             // O^T += V^T P^T
             {
@@ -429,8 +445,8 @@ attend_kernel(AttendParams p)
                     uint32_t va[4];
                     const int ch = 2 * t + (lmat & 1);
                     ldmatrix_x4_trans(va, v_addr + vrow * kRowBytes + ((ch ^ lrow) << 4));
-                    mma_bf16(o[t], va[0], va[1], va[2], va[3], ph0, ph1);
-                    mma_bf16(o[t], va[0], va[1], va[2], va[3], pl0, pl1);
+                    mma_16816<kHalf>(o[t], va[0], va[1], va[2], va[3], ph0, ph1);
+                    mma_16816<kHalf>(o[t], va[0], va[1], va[2], va[3], pl0, pl1);
                 }
             }
             __syncwarp();                                  // the slot may be refilled by the next issue
@@ -580,22 +596,22 @@ attend_kernel(AttendParams p)
     }
 }
 
-template <int G>
+template <int G, bool kHalf>
 cudaError_t launch_attend_g(const AttendParams &p, bool all_heads, bool static_split, int grid, cudaStream_t s)
 {
     const size_t smem = Smem<G>::total;
     static std::atomic<unsigned long long> done[4];
-    const void *fns[4] = {(const void *)attend_kernel<G, true, true>, (const void *)attend_kernel<G, true, false>,
-                          (const void *)attend_kernel<G, false, true>, (const void *)attend_kernel<G, false, false>};
+    const void *fns[4] = {(const void *)attend_kernel<G, true, true, kHalf>, (const void *)attend_kernel<G, true, false, kHalf>,
+                          (const void *)attend_kernel<G, false, true, kHalf>, (const void *)attend_kernel<G, false, false, kHalf>};
     const int which = (all_heads ? 0 : 2) + (static_split ? 0 : 1);
     cudaError_t err = ensure_dynamic_smem(fns[which], (int)smem, done[which]);
     if (err != cudaSuccess) return err;
     if (all_heads) {
-        if (static_split) attend_kernel<G, true, true><<<grid, kAttendThreads, smem, s>>>(p);
-        else              attend_kernel<G, true, false><<<grid, kAttendThreads, smem, s>>>(p);
+        if (static_split) attend_kernel<G, true, true, kHalf><<<grid, kAttendThreads, smem, s>>>(p);
+        else              attend_kernel<G, true, false, kHalf><<<grid, kAttendThreads, smem, s>>>(p);
     } else {
-        if (static_split) attend_kernel<G, false, true><<<grid, kAttendThreads, smem, s>>>(p);
-        else              attend_kernel<G, false, false><<<grid, kAttendThreads, smem, s>>>(p);
+        if (static_split) attend_kernel<G, false, true, kHalf><<<grid, kAttendThreads, smem, s>>>(p);
+        else              attend_kernel<G, false, false, kHalf><<<grid, kAttendThreads, smem, s>>>(p);
     }
     return cudaGetLastError();
 }
@@ -615,14 +631,22 @@ int attend_max_pairs() { return 1 << 16; }
 cudaError_t launch_attend(const AttendParams &p, bool all_heads, bool static_split, int grid, cudaStream_t s)
 {
     switch (p.bv.group) {
-        case 1: return launch_attend_g<1>(p, all_heads, static_split, grid, s);
-        case 2: return launch_attend_g<2>(p, all_heads, static_split, grid, s);
-        case 3: return launch_attend_g<3>(p, all_heads, static_split, grid, s);
-        case 4: return launch_attend_g<4>(p, all_heads, static_split, grid, s);
-        case 5: return launch_attend_g<5>(p, all_heads, static_split, grid, s);
-        case 6: return launch_attend_g<6>(p, all_heads, static_split, grid, s);
-        case 7: return launch_attend_g<7>(p, all_heads, static_split, grid, s);
-        case 8: return launch_attend_g<8>(p, all_heads, static_split, grid, s);
+        case 1: return p.bv.elem ? launch_attend_g<1, true>(p, all_heads, static_split, grid, s)
+                                 : launch_attend_g<1, false>(p, all_heads, static_split, grid, s);
+        case 2: return p.bv.elem ? launch_attend_g<2, true>(p, all_heads, static_split, grid, s)
+                                 : launch_attend_g<2, false>(p, all_heads, static_split, grid, s);
+        case 3: return p.bv.elem ? launch_attend_g<3, true>(p, all_heads, static_split, grid, s)
+                                 : launch_attend_g<3, false>(p, all_heads, static_split, grid, s);
+        case 4: return p.bv.elem ? launch_attend_g<4, true>(p, all_heads, static_split, grid, s)
+                                 : launch_attend_g<4, false>(p, all_heads, static_split, grid, s);
+        case 5: return p.bv.elem ? launch_attend_g<5, true>(p, all_heads, static_split, grid, s)
+                                 : launch_attend_g<5, false>(p, all_heads, static_split, grid, s);
+        case 6: return p.bv.elem ? launch_attend_g<6, true>(p, all_heads, static_split, grid, s)
+                                 : launch_attend_g<6, false>(p, all_heads, static_split, grid, s);
+        case 7: return p.bv.elem ? launch_attend_g<7, true>(p, all_heads, static_split, grid, s)
+                                 : launch_attend_g<7, false>(p, all_heads, static_split, grid, s);
+        case 8: return p.bv.elem ? launch_attend_g<8, true>(p, all_heads, static_split, grid, s)
+                                 : launch_attend_g<8, false>(p, all_heads, static_split, grid, s);
         default: return cudaErrorInvalidValue;
     }
 }

@@ -25,6 +25,7 @@ __device__ __forceinline__ int clamp_label(int v, int n) { return min(max(v, 0),
 constexpr int kAssignThreads = 128;
 constexpr int kCentreTile = 16;
 
+template <bool kHalf>
 __global__ void __launch_bounds__(kAssignThreads)
 assign_parents_kernel(AssignParams p)
 {
@@ -60,8 +61,8 @@ assign_parents_kernel(AssignParams p)
             double s = 0.0;
 #pragma unroll
             for (int w = 0; w < 64; ++w) {
-                const double e0 = __dsub_rn((double)bf16_lo(kw[w]), c[t][2 * w]);
-                const double e1 = __dsub_rn((double)bf16_hi(kw[w]), c[t][2 * w + 1]);
+                const double e0 = __dsub_rn((double)elem_lo<kHalf>(kw[w]), c[t][2 * w]);
+                const double e1 = __dsub_rn((double)elem_hi<kHalf>(kw[w]), c[t][2 * w + 1]);
                 s = __dadd_rn(s, __dmul_rn(e0, e0));
                 s = __dadd_rn(s, __dmul_rn(e1, e1));
             }
@@ -155,6 +156,7 @@ stable_scatter_kernel(const int32_t *labels, int32_t *cursors, int32_t *out, con
     }
 }
 
+template <bool kHalf>
 __device__ __forceinline__ double sqdist_grow_vec(const uint4 *row, const double *ref)
 {
     double s = 0.0;
@@ -164,8 +166,8 @@ __device__ __forceinline__ double sqdist_grow_vec(const uint4 *row, const double
         const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
 #pragma unroll
         for (int t = 0; t < 4; ++t) {
-            const double e0 = __dsub_rn((double)bf16_lo(w[t]), ref[8 * q + 2 * t]);
-            const double e1 = __dsub_rn((double)bf16_hi(w[t]), ref[8 * q + 2 * t + 1]);
+            const double e0 = __dsub_rn((double)elem_lo<kHalf>(w[t]), ref[8 * q + 2 * t]);
+            const double e1 = __dsub_rn((double)elem_hi<kHalf>(w[t]), ref[8 * q + 2 * t + 1]);
             s = __dadd_rn(s, __dmul_rn(e0, e0));
             s = __dadd_rn(s, __dmul_rn(e1, e1));
         }
@@ -173,6 +175,7 @@ __device__ __forceinline__ double sqdist_grow_vec(const uint4 *row, const double
     return s;
 }
 
+template <bool kHalf>
 __device__ __forceinline__ double sqdist_grow_row(const uint4 *row, const uint32_t *ref)
 {
     double s = 0.0;
@@ -183,8 +186,8 @@ __device__ __forceinline__ double sqdist_grow_row(const uint4 *row, const uint32
 #pragma unroll
         for (int t = 0; t < 4; ++t) {
             const uint32_t r = ref[4 * q + t];
-            const double e0 = __dsub_rn((double)bf16_lo(w[t]), (double)bf16_lo(r));
-            const double e1 = __dsub_rn((double)bf16_hi(w[t]), (double)bf16_hi(r));
+            const double e0 = __dsub_rn((double)elem_lo<kHalf>(w[t]), (double)elem_lo<kHalf>(r));
+            const double e1 = __dsub_rn((double)elem_hi<kHalf>(w[t]), (double)elem_hi<kHalf>(r));
             s = __dadd_rn(s, __dmul_rn(e0, e0));
             s = __dadd_rn(s, __dmul_rn(e1, e1));
         }
@@ -194,6 +197,7 @@ __device__ __forceinline__ double sqdist_grow_row(const uint4 *row, const uint32
 
 // Algorithm 2 for one parent of any size. One block per (label, sequence, KV head); the parent's
 // tokens are read through its member list, and the per-member state lives in global memory.
+template <bool kHalf>
 __global__ void __launch_bounds__(kThreads)
 build_parent_general_kernel(ParentBuildParams p)
 {
@@ -226,7 +230,7 @@ build_parent_general_kernel(ParentBuildParams p)
     if (tid < kHeadDim) {
         const uint16_t *col = p.k_prompt + plane * kHeadDim + tid;
         double s = 0.0;
-        for (int i = 0; i < nC; ++i) s = __dadd_rn(s, bf16_to_double(col[(size_t)mem[i] * kHeadDim]));
+        for (int i = 0; i < nC; ++i) s = __dadd_rn(s, elem_to_double<kHalf>(col[(size_t)mem[i] * kHeadDim]));
         mu[tid] = __ddiv_rn(s, (double)nC);
     }
     __syncthreads();
@@ -235,7 +239,7 @@ build_parent_general_kernel(ParentBuildParams p)
     {
         ValIdx best = {INFINITY, INT_MAX};
         for (int i = tid; i < nC; i += kThreads) {
-            ValIdx c = {sqdist_grow_vec(kbase + (size_t)mem[i] * 16, mu), i};
+            ValIdx c = {sqdist_grow_vec<kHalf>(kbase + (size_t)mem[i] * 16, mu), i};
             best = pick<true>(best, c);
         }
         best = block_arg<true>(best, scratch);
@@ -250,7 +254,7 @@ build_parent_general_kernel(ParentBuildParams p)
         __syncthreads();
         ValIdx far = {-2.0, INT_MAX};
         for (int i = tid; i < nC; i += kThreads) {
-            const double dist = sqdist_grow_row(kbase + (size_t)mem[i] * 16, ref);
+            const double dist = sqdist_grow_row<kHalf>(kbase + (size_t)mem[i] * 16, ref);
             double m = mind[i];
             if (dist < m) { m = dist; mind[i] = dist; owner[i] = u; }
             ValIdx c = {is_rep[i] ? -1.0 : m, i};
@@ -334,7 +338,8 @@ pack_rows_kernel(ParentBuildParams p)
 cudaError_t launch_assign_parents(const AssignParams &p, cudaStream_t s)
 {
     dim3 grid((p.max_rows_per_seq + kAssignThreads - 1) / kAssignThreads, p.n_seqs, p.n_kv);
-    assign_parents_kernel<<<grid, kAssignThreads, 0, s>>>(p);
+    if (p.elem) assign_parents_kernel<true><<<grid, kAssignThreads, 0, s>>>(p);
+    else        assign_parents_kernel<false><<<grid, kAssignThreads, 0, s>>>(p);
     return cudaGetLastError();
 }
 
@@ -353,7 +358,8 @@ cudaError_t launch_build_teams_parents(const ParentBuildParams &p, cudaStream_t 
     stable_scatter_kernel<true><<<dim3(B, H), 32, 0, s>>>(p.parent_of, p.parent_cursor, p.members, p.bv.seq_row_off,
                                                           p.seq_label_off, p.bv.rows_total, p.labels_total);
     if ((err = cudaGetLastError()) != cudaSuccess) return err;
-    build_parent_general_kernel<<<dim3(p.max_labels_per_seq, B, H), kThreads, 0, s>>>(p);
+    if (p.bv.elem) build_parent_general_kernel<true><<<dim3(p.max_labels_per_seq, B, H), kThreads, 0, s>>>(p);
+    else           build_parent_general_kernel<false><<<dim3(p.max_labels_per_seq, B, H), kThreads, 0, s>>>(p);
     if ((err = cudaGetLastError()) != cudaSuccess) return err;
     scan_teams_kernel<<<dim3(B, H), kThreads, 0, s>>>(p);
     if ((err = cudaGetLastError()) != cudaSuccess) return err;

@@ -16,28 +16,30 @@ constexpr int kRowWords = 65;            // 64 data words + 1 pad word: conflict
 
 // Squared distance between row `i` (shared memory, bf16 words) and a reference vector in fp64,
 // summed over dimensions in increasing order, multiply and add rounded separately.
+template <bool kHalf>
 __device__ __forceinline__ double sqdist_row_vec(const uint32_t *row, const double *ref)
 {
     double s = 0.0;
 #pragma unroll 8
     for (int w = 0; w < 64; ++w) {
         const uint32_t word = row[w];
-        const double e0 = __dsub_rn((double)bf16_lo(word), ref[2 * w]);
-        const double e1 = __dsub_rn((double)bf16_hi(word), ref[2 * w + 1]);
+        const double e0 = __dsub_rn((double)elem_lo<kHalf>(word), ref[2 * w]);
+        const double e1 = __dsub_rn((double)elem_hi<kHalf>(word), ref[2 * w + 1]);
         s = __dadd_rn(s, __dmul_rn(e0, e0));
         s = __dadd_rn(s, __dmul_rn(e1, e1));
     }
     return s;
 }
 
+template <bool kHalf>
 __device__ __forceinline__ double sqdist_row_row(const uint32_t *row, const uint32_t *ref)
 {
     double s = 0.0;
 #pragma unroll 8
     for (int w = 0; w < 64; ++w) {
         const uint32_t a = row[w], b = ref[w];
-        const double e0 = __dsub_rn((double)bf16_lo(a), (double)bf16_lo(b));
-        const double e1 = __dsub_rn((double)bf16_hi(a), (double)bf16_hi(b));
+        const double e0 = __dsub_rn((double)elem_lo<kHalf>(a), (double)elem_lo<kHalf>(b));
+        const double e1 = __dsub_rn((double)elem_hi<kHalf>(a), (double)elem_hi<kHalf>(b));
         s = __dadd_rn(s, __dmul_rn(e0, e0));
         s = __dadd_rn(s, __dmul_rn(e1, e1));
     }
@@ -45,6 +47,7 @@ __device__ __forceinline__ double sqdist_row_row(const uint32_t *row, const uint
 }
 
 // One block per (parent, sequence, KV head): representatives, owners, team sizes.
+template <bool kHalf>
 __global__ void __launch_bounds__(kBuildThreads)
 build_parent_kernel(BuildParams p)
 {
@@ -81,7 +84,7 @@ build_parent_kernel(BuildParams p)
         const bool hi = tid & 1;
         for (int i = 0; i < nC; ++i) {
             const uint32_t word = rows[i * kRowWords + w];
-            s = __dadd_rn(s, (double)(hi ? bf16_hi(word) : bf16_lo(word)));
+            s = __dadd_rn(s, (double)(hi ? elem_hi<kHalf>(word) : elem_lo<kHalf>(word)));
         }
         mu[tid] = __ddiv_rn(s, (double)nC);
     }
@@ -91,7 +94,7 @@ build_parent_kernel(BuildParams p)
     {
         ValIdx best = {INFINITY, INT_MAX};
         for (int i = tid; i < nC; i += kBuildThreads) {
-            ValIdx c = {sqdist_row_vec(rows + i * kRowWords, mu), i};
+            ValIdx c = {sqdist_row_vec<kHalf>(rows + i * kRowWords, mu), i};
             best = pick<true>(best, c);
         }
         best = block_arg<true>(best, scratch);
@@ -106,7 +109,7 @@ build_parent_kernel(BuildParams p)
         const uint32_t *ref = rows + rep_of[u] * kRowWords;
         ValIdx far = {-2.0, INT_MAX};
         for (int i = tid; i < nC; i += kBuildThreads) {
-            const double dist = sqdist_row_row(rows + i * kRowWords, ref);
+            const double dist = sqdist_row_row<kHalf>(rows + i * kRowWords, ref);
             if (dist < mind[i]) { mind[i] = dist; owner[i] = u; }
             ValIdx c = {is_rep[i] ? -1.0 : mind[i], i};
             far = pick<false>(far, c);
@@ -266,11 +269,12 @@ cudaError_t launch_build_groups_mean(const BuildParams &p, cudaStream_t s)
 cudaError_t launch_build_teams(const BuildParams &p, cudaStream_t s)
 {
     const size_t smem = build_parent_smem(p.parent_size);
-    cudaError_t err = cudaFuncSetAttribute(build_parent_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                           (int)smem);
+    cudaError_t err = cudaFuncSetAttribute(p.bv.elem ? build_parent_kernel<true> : build_parent_kernel<false>,
+                                           cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (err != cudaSuccess) return err;
     dim3 grid(p.max_parents_per_seq, p.bv.n_seqs, p.bv.n_kv);
-    build_parent_kernel<<<grid, kBuildThreads, smem, s>>>(p);
+    if (p.bv.elem) build_parent_kernel<true><<<grid, kBuildThreads, smem, s>>>(p);
+    else           build_parent_kernel<false><<<grid, kBuildThreads, smem, s>>>(p);
     if ((err = cudaGetLastError()) != cudaSuccess) return err;
     scan_team_sizes_kernel<<<dim3(p.bv.n_seqs, p.bv.n_kv), kBuildThreads, 0, s>>>(p);
     if ((err = cudaGetLastError()) != cudaSuccess) return err;

@@ -1,6 +1,7 @@
 // Shared declarations of the SANTA++ decode-attention kernels (sm_100a).
 #pragma once
 
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -28,6 +29,7 @@ struct BatchView {
     const int64_t *seq_team_off;    // [n_seqs + 1] team slots of each sequence
     const int32_t *team_count;      // [n_kv][n_seqs] teams a pair really has, or null: every slot is a team
     int64_t rows_total, teams_total;
+    int elem;                       // element type of q / K / V / representative keys: 0 bf16, 1 fp16
 };
 
 // Teams of (sequence b, KV head j): the first `pair_team_count` slots of the sequence's range.
@@ -173,7 +175,7 @@ cudaError_t launch_build_groups_mean(const BuildParams &p, cudaStream_t s);
 
 // Nearest-centre assignment (last step of Algorithm 3).
 struct AssignParams {
-    int n_seqs, n_kv, max_rows_per_seq;
+    int n_seqs, n_kv, max_rows_per_seq, elem;
     int64_t rows_total, centres_total;
     const int64_t *seq_row_off;             // device [n_seqs + 1]
     const int64_t *seq_centre_off;          // device [n_seqs + 1]
@@ -214,6 +216,28 @@ __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w 
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
 __device__ __forceinline__ float bf16_to_float(uint16_t b) { return __uint_as_float(((uint32_t)b) << 16); }
 __device__ __forceinline__ double bf16_to_double(uint16_t b) { return (double)bf16_to_float(b); }
+
+// The same three conversions for either 16-bit element type (kHalf: IEEE fp16, else bf16).
+template <bool kHalf>
+__device__ __forceinline__ float elem_to_float(uint16_t b)
+{
+    if constexpr (kHalf) return __half2float(__ushort_as_half(b));
+    else return bf16_to_float(b);
+}
+template <bool kHalf>
+__device__ __forceinline__ float elem_lo(uint32_t w)
+{
+    if constexpr (kHalf) return __half2float(__ushort_as_half((unsigned short)(w & 0xFFFFu)));
+    else return bf16_lo(w);
+}
+template <bool kHalf>
+__device__ __forceinline__ float elem_hi(uint32_t w)
+{
+    if constexpr (kHalf) return __half2float(__ushort_as_half((unsigned short)(w >> 16)));
+    else return bf16_hi(w);
+}
+template <bool kHalf>
+__device__ __forceinline__ double elem_to_double(uint16_t b) { return (double)elem_to_float<kHalf>(b); }
 
 // Philox4x32-10: 128-bit counter, 64-bit key, four 32-bit words.
 __device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint32_t k0, uint32_t k1)

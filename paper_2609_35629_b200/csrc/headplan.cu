@@ -52,7 +52,7 @@ __device__ __forceinline__ float score_guard(double scale, double q_l1, float k_
 }
 
 // The first half of the block's warps compute dot products, the second half the Gumbel terms.
-template <int kHeadThreads>
+template <int kHeadThreads, bool kHalf>
 __global__ void __launch_bounds__(kHeadThreads, 1024 / kHeadThreads)
 headplan_kernel(PlanInputs in)
 {
@@ -79,7 +79,7 @@ headplan_kernel(PlanInputs in)
     {
         float a = 0.f, top = -CUDART_INF_F;
         if (tid < kHeadDim) {
-            const float v = bf16_to_float(in.q[(size_t)hq * kHeadDim + tid]);
+            const float v = elem_to_float<kHalf>(in.q[(size_t)hq * kHeadDim + tid]);
             sm.q64[tid >> 4][tid & 15] = (double)v;
             a = fabsf(v);
         }
@@ -225,22 +225,22 @@ headplan_kernel(PlanInputs in)
                     const int cand = c0 + u * kPerPass + (tid >> 3);
                     const uint4 w0 = w[u][0], w1 = w[u][1];
                     double d0 = 0.0, d1 = 0.0;
-                    d0 = fma((double)bf16_lo(w0.x), qs[0], d0);
-                    d1 = fma((double)bf16_hi(w0.x), qs[1], d1);
-                    d0 = fma((double)bf16_lo(w0.y), qs[2], d0);
-                    d1 = fma((double)bf16_hi(w0.y), qs[3], d1);
-                    d0 = fma((double)bf16_lo(w0.z), qs[4], d0);
-                    d1 = fma((double)bf16_hi(w0.z), qs[5], d1);
-                    d0 = fma((double)bf16_lo(w0.w), qs[6], d0);
-                    d1 = fma((double)bf16_hi(w0.w), qs[7], d1);
-                    d0 = fma((double)bf16_lo(w1.x), qs[8], d0);
-                    d1 = fma((double)bf16_hi(w1.x), qs[9], d1);
-                    d0 = fma((double)bf16_lo(w1.y), qs[10], d0);
-                    d1 = fma((double)bf16_hi(w1.y), qs[11], d1);
-                    d0 = fma((double)bf16_lo(w1.z), qs[12], d0);
-                    d1 = fma((double)bf16_hi(w1.z), qs[13], d1);
-                    d0 = fma((double)bf16_lo(w1.w), qs[14], d0);
-                    d1 = fma((double)bf16_hi(w1.w), qs[15], d1);
+                    d0 = fma((double)elem_lo<kHalf>(w0.x), qs[0], d0);
+                    d1 = fma((double)elem_hi<kHalf>(w0.x), qs[1], d1);
+                    d0 = fma((double)elem_lo<kHalf>(w0.y), qs[2], d0);
+                    d1 = fma((double)elem_hi<kHalf>(w0.y), qs[3], d1);
+                    d0 = fma((double)elem_lo<kHalf>(w0.z), qs[4], d0);
+                    d1 = fma((double)elem_hi<kHalf>(w0.z), qs[5], d1);
+                    d0 = fma((double)elem_lo<kHalf>(w0.w), qs[6], d0);
+                    d1 = fma((double)elem_hi<kHalf>(w0.w), qs[7], d1);
+                    d0 = fma((double)elem_lo<kHalf>(w1.x), qs[8], d0);
+                    d1 = fma((double)elem_hi<kHalf>(w1.x), qs[9], d1);
+                    d0 = fma((double)elem_lo<kHalf>(w1.y), qs[10], d0);
+                    d1 = fma((double)elem_hi<kHalf>(w1.y), qs[11], d1);
+                    d0 = fma((double)elem_lo<kHalf>(w1.z), qs[12], d0);
+                    d1 = fma((double)elem_hi<kHalf>(w1.z), qs[13], d1);
+                    d0 = fma((double)elem_lo<kHalf>(w1.w), qs[14], d0);
+                    d1 = fma((double)elem_hi<kHalf>(w1.w), qs[15], d1);
                     double d = d0 + d1;
                     d += __shfl_xor_sync(0xFFFFFFFFu, d, 1);
                     d += __shfl_xor_sync(0xFFFFFFFFu, d, 2);
@@ -347,8 +347,14 @@ cudaError_t launch_headplan(const PlanInputs &in, cudaStream_t s)
     // 256 threads per head while every head's block is resident at once (4 per SM by registers),
     // else 128 threads so that twice as many fit
     const int n_heads = in.bv.n_seqs * in.bv.n_q;
-    if (n_heads <= 4 * attend_grid_size()) headplan_kernel<256><<<n_heads, 256, 0, s>>>(in);
-    else                                   headplan_kernel<128><<<n_heads, 128, 0, s>>>(in);
+    const bool wide = n_heads <= 4 * attend_grid_size();
+    if (in.bv.elem) {
+        if (wide) headplan_kernel<256, true><<<n_heads, 256, 0, s>>>(in);
+        else      headplan_kernel<128, true><<<n_heads, 128, 0, s>>>(in);
+    } else {
+        if (wide) headplan_kernel<256, false><<<n_heads, 256, 0, s>>>(in);
+        else      headplan_kernel<128, false><<<n_heads, 128, 0, s>>>(in);
+    }
     return cudaGetLastError();
 }
 

@@ -21,13 +21,20 @@ constexpr int kScoreThreads = 256;
 constexpr int kScoreTeamsPerWarp = 16;
 constexpr int kScoreTeamsPerCta = kScoreTeamsPerWarp * (kScoreThreads / 32);
 
-__device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1)
+template <bool kHalf>
+__device__ __forceinline__ void mma_16816(float (&d)[4], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1)
 {
     // A rows 8..15 are zero (a1 = a3 = 0): only heads 0..7 exist
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
-                 "{%0,%1,%2,%3};"
-                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-                 : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1));
+    if constexpr (kHalf)
+        asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+                     "{%0,%1,%2,%3};"
+                     : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                     : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1));
+    else
+        asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+                     "{%0,%1,%2,%3};"
+                     : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                     : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1));
 }
 
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
@@ -108,7 +115,7 @@ __device__ __forceinline__ void load_q_fragments(const ScoreParams &p, int b, in
 // Scores of one tile of 16 teams (two n-tiles of 8; B row n = team base + 8 t + g) from the key
 // pieces kb of this lane: writes Y32 for the G heads and the tile's maximum per head.
 // csr_tile points at the 17 row offsets of the tile's teams (global or shared memory).
-template <int G>
+template <int G, bool kHalf>
 __device__ __forceinline__ void score_tile(const ScoreParams &p, int b, int j, int64_t team0, int M, int base,
                                            const int32_t *csr_tile, const uint4 (&kb)[2][4], const uint32_t (&qa)[8][2],
                                            uint32_t step, float scale, int g, int c)
@@ -130,8 +137,8 @@ __device__ __forceinline__ void score_tile(const ScoreParams &p, int b, int j, i
         acc[t][0] = acc[t][1] = acc[t][2] = acc[t][3] = 0.f;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            mma_bf16_16816(acc[t], qa[2 * i][0], qa[2 * i][1], kb[t][i].x, kb[t][i].y);
-            mma_bf16_16816(acc[t], qa[2 * i + 1][0], qa[2 * i + 1][1], kb[t][i].z, kb[t][i].w);
+            mma_16816<kHalf>(acc[t], qa[2 * i][0], qa[2 * i][1], kb[t][i].x, kb[t][i].y);
+            mma_16816<kHalf>(acc[t], qa[2 * i + 1][0], qa[2 * i + 1][1], kb[t][i].z, kb[t][i].w);
         }
     }
     // One Philox block covers four consecutive teams of a head: teams base + 8 t + {0..3} belong
@@ -182,7 +189,7 @@ __device__ __forceinline__ void clear_control(const ScoreParams &p, int tid)
 }
 
 // Small grids: one warp per tile of 16 teams, keys straight into registers (the shortest path).
-template <int G>
+template <int G, bool kHalf>
 __global__ void __launch_bounds__(kScoreThreads, 2)
 score32_kernel(ScoreParams p)
 {
@@ -209,7 +216,7 @@ score32_kernel(ScoreParams p)
     }
     const uint32_t step = p.step + (p.step_dev ? *p.step_dev : 0u);
     const int32_t *csr = p.team_row_start + (size_t)j * (p.bv.teams_total + p.bv.n_seqs) + team0 + b;
-    score_tile<G>(p, b, j, team0, M, base, csr + base, kb, qa, step, (float)p.scale, g, c);
+    score_tile<G, kHalf>(p, b, j, team0, M, base, csr + base, kb, qa, step, (float)p.scale, g, c);
 }
 
 // Where a tile index of the flat kernel lies: tiles are the slots of the block-maximum table,
@@ -264,7 +271,7 @@ __device__ __forceinline__ void advance(const ScoreParams &p, TileCursor &cur)
 // tile (16 keys are one contiguous run) that completes on the stage's mbarrier; the tile's 17 row
 // offsets travel as per-lane 4-byte cp.async copies (their address is only 4-byte aligned).
 // Every wait on an mbarrier is bounded; on expiry the warp raises status bit 2 and stops.
-template <int G>
+template <int G, bool kHalf>
 __global__ void __launch_bounds__(kScoreThreads, 2)
 score32_flat_kernel(ScoreParams p)
 {
@@ -358,7 +365,7 @@ score32_flat_kernel(ScoreParams p)
             for (int t = 0; t < 2; ++t)
 #pragma unroll
                 for (int i = 0; i < 4; ++i) kb[t][i] = tile_of(stage)[(8 * t + g) * 16 + c + 4 * i];
-            score_tile<G>(p, here.b, here.j, here.team0, here.M, base, csr_ring + stage * 32, kb, qa, step, scale, g, c);
+            score_tile<G, kHalf>(p, here.b, here.j, here.team0, here.M, base, csr_ring + stage * 32, kb, qa, step, scale, g, c);
         }
         __syncwarp();                                            // every lane is done with the stage's row offsets
         // refill the stage just consumed (its pieces are in registers and already used above)
@@ -378,7 +385,7 @@ rep_abs_max_kernel(BatchView bv, const uint16_t *rep_keys, float *rep_abs_max)
     const int64_t team0 = bv.seq_team_off[b];
     const int64_t n = (bv.seq_team_off[b + 1] - team0) * kHeadDim / 2;     // 32-bit words
     const uint32_t *w = reinterpret_cast<const uint32_t *>(rep_keys + ((size_t)j * bv.teams_total + team0) * kHeadDim);
-    uint32_t m = 0u;                                                        // bf16 magnitudes order like integers
+    uint32_t m = 0u;                                       // bf16 and fp16 magnitudes order like integers
     for (int64_t i = threadIdx.x; i < n; i += blockDim.x) {
         const uint32_t v = w[i];
         m = max(m, max(v & 0x7FFFu, (v >> 16) & 0x7FFFu));
@@ -389,23 +396,23 @@ rep_abs_max_kernel(BatchView bv, const uint16_t *rep_keys, float *rep_abs_max)
     __syncthreads();
     if (threadIdx.x == 0) {
         for (int i = 1; i < 8; ++i) m = max(m, red[i]);
-        rep_abs_max[(size_t)j * bv.n_seqs + b] = __uint_as_float(m << 16);
+        rep_abs_max[(size_t)j * bv.n_seqs + b] = bv.elem ? elem_to_float<true>((uint16_t)m) : __uint_as_float(m << 16);
     }
 }
 
-template <int G>
+template <int G, bool kHalf>
 cudaError_t launch_score32_g(const ScoreParams &p, int max_teams, cudaStream_t s)
 {
     const long long ctas1 = (long long)((max_teams + kScoreTeamsPerCta - 1) / kScoreTeamsPerCta) * p.n_pairs;
     if (ctas1 < 2 * 148) {
         dim3 grid((max_teams + kScoreTeamsPerCta - 1) / kScoreTeamsPerCta, p.n_pairs);
-        score32_kernel<G><<<grid, kScoreThreads, 0, s>>>(p);
+        score32_kernel<G, kHalf><<<grid, kScoreThreads, 0, s>>>(p);
         return cudaGetLastError();
     }
     static std::atomic<unsigned long long> done;
-    cudaError_t e = ensure_dynamic_smem((const void *)score32_flat_kernel<G>, kScoreRingBytes, done);
+    cudaError_t e = ensure_dynamic_smem((const void *)score32_flat_kernel<G, kHalf>, kScoreRingBytes, done);
     if (e != cudaSuccess) return e;
-    score32_flat_kernel<G><<<2 * attend_grid_size(), kScoreThreads, kScoreRingBytes, s>>>(p);
+    score32_flat_kernel<G, kHalf><<<2 * attend_grid_size(), kScoreThreads, kScoreRingBytes, s>>>(p);
     return cudaGetLastError();
 }
 
@@ -414,14 +421,22 @@ cudaError_t launch_score32_g(const ScoreParams &p, int max_teams, cudaStream_t s
 cudaError_t launch_score32(const ScoreParams &p, int max_teams_per_seq, cudaStream_t s)
 {
     switch (p.bv.group) {
-        case 1: return launch_score32_g<1>(p, max_teams_per_seq, s);
-        case 2: return launch_score32_g<2>(p, max_teams_per_seq, s);
-        case 3: return launch_score32_g<3>(p, max_teams_per_seq, s);
-        case 4: return launch_score32_g<4>(p, max_teams_per_seq, s);
-        case 5: return launch_score32_g<5>(p, max_teams_per_seq, s);
-        case 6: return launch_score32_g<6>(p, max_teams_per_seq, s);
-        case 7: return launch_score32_g<7>(p, max_teams_per_seq, s);
-        case 8: return launch_score32_g<8>(p, max_teams_per_seq, s);
+        case 1: return p.bv.elem ? launch_score32_g<1, true>(p, max_teams_per_seq, s)
+                                 : launch_score32_g<1, false>(p, max_teams_per_seq, s);
+        case 2: return p.bv.elem ? launch_score32_g<2, true>(p, max_teams_per_seq, s)
+                                 : launch_score32_g<2, false>(p, max_teams_per_seq, s);
+        case 3: return p.bv.elem ? launch_score32_g<3, true>(p, max_teams_per_seq, s)
+                                 : launch_score32_g<3, false>(p, max_teams_per_seq, s);
+        case 4: return p.bv.elem ? launch_score32_g<4, true>(p, max_teams_per_seq, s)
+                                 : launch_score32_g<4, false>(p, max_teams_per_seq, s);
+        case 5: return p.bv.elem ? launch_score32_g<5, true>(p, max_teams_per_seq, s)
+                                 : launch_score32_g<5, false>(p, max_teams_per_seq, s);
+        case 6: return p.bv.elem ? launch_score32_g<6, true>(p, max_teams_per_seq, s)
+                                 : launch_score32_g<6, false>(p, max_teams_per_seq, s);
+        case 7: return p.bv.elem ? launch_score32_g<7, true>(p, max_teams_per_seq, s)
+                                 : launch_score32_g<7, false>(p, max_teams_per_seq, s);
+        case 8: return p.bv.elem ? launch_score32_g<8, true>(p, max_teams_per_seq, s)
+                                 : launch_score32_g<8, false>(p, max_teams_per_seq, s);
         default: return cudaErrorInvalidValue;
     }
 }

@@ -46,6 +46,24 @@ def bf16_to_f64(bits: np.ndarray) -> np.ndarray:
     return bf16_to_f32(bits).astype(np.float64)
 
 
+def round_bits(x: np.ndarray, elem: str = "bf16") -> np.ndarray:
+    """Round float32 to the 16-bit element type (nearest even); returns uint16 bit patterns."""
+    if elem == "fp16":
+        return np.ascontiguousarray(x, dtype=np.float32).astype(np.float16).view(np.uint16)
+    return f32_to_bf16_bits(x)
+
+
+def to_f32(bits: np.ndarray, elem: str = "bf16") -> np.ndarray:
+    if elem == "fp16":
+        return np.ascontiguousarray(bits, dtype=np.uint16).view(np.float16).astype(np.float32)
+    return bf16_to_f32(bits)
+
+
+def to_f64(bits: np.ndarray, elem: str = "bf16") -> np.ndarray:
+    """Exact widening of 16-bit patterns of the given element type to float64."""
+    return to_f32(bits, elem).astype(np.float64)
+
+
 @dataclass
 class WorkloadSpec:
     name: str
@@ -66,6 +84,7 @@ class WorkloadSpec:
                                      # cluster, mean length rows / clusters: positional locality)
     head_dim: int = HEAD_DIM
     seed: int = 0
+    elem: str = "bf16"               # 16-bit element type the draws are rounded to: "bf16" or "fp16"
 
     @property
     def group(self) -> int:
@@ -183,12 +202,12 @@ def make_layer(spec: WorkloadSpec, layer: int = 0, keep_centres: bool = False) -
             k = _clustered_rows(rng, n, centres, layout=spec.key_layout)
             k[: min(4, n)] *= np.float32(4.0)        # sink keys
             v = rng.standard_normal((n, d), dtype=np.float32)
-            k_prompt[j, off[b]:off[b + 1]] = f32_to_bf16_bits(k)
-            v_prompt[j, off[b]:off[b + 1]] = f32_to_bf16_bits(v)
+            k_prompt[j, off[b]:off[b + 1]] = round_bits(k, spec.elem)
+            v_prompt[j, off[b]:off[b + 1]] = round_bits(v, spec.elem)
             ks = _clustered_rows(rng, cap, centres)
             vs = rng.standard_normal((cap, d), dtype=np.float32)
-            k_suffix[b, j] = f32_to_bf16_bits(ks)
-            v_suffix[b, j] = f32_to_bf16_bits(vs)
+            k_suffix[b, j] = round_bits(ks, spec.elem)
+            v_suffix[b, j] = round_bits(vs, spec.elem)
     return LayerData(spec, layer, k_prompt, v_prompt, k_suffix, v_suffix, off,
                      centres_all if keep_centres else None)
 
@@ -207,20 +226,20 @@ def make_queries(spec: WorkloadSpec, data: LayerData, step: int) -> np.ndarray:
             eps = rng.standard_normal(d, dtype=np.float32)
             if spec.query_kind == "noisy_copy":
                 row = int(rng.integers(lo, hi))
-                kj = bf16_to_f32(data.k_prompt[j, row])
+                kj = to_f32(data.k_prompt[j, row], spec.elem)
                 q[b, h] = np.float32(2.0) * (kj + np.float32(0.5) * eps)
             elif spec.query_kind == "concentrated":
                 if data.centres is None:
                     raise ValueError("concentrated queries need make_layer(..., keep_centres=True)")
                 if j not in keys_f32:
-                    keys_f32[j] = bf16_to_f32(data.k_prompt[j, lo:hi])
+                    keys_f32[j] = to_f32(data.k_prompt[j, lo:hi], spec.elem)
                 c = data.centres[j, int(rng.integers(0, spec.n_clusters))]
                 base = c + np.float32(0.5) * eps
                 logits = (keys_f32[j] @ base).astype(np.float64) / np.sqrt(d)
                 q[b, h] = np.float32(_bisect_alpha(logits, 64, 0.90)) * base
             else:
                 raise ValueError(spec.query_kind)
-    return f32_to_bf16_bits(q)
+    return round_bits(q, spec.elem)
 
 
 def _bisect_alpha(logits: np.ndarray, top: int, mass: float) -> float:

@@ -17,7 +17,7 @@ from paper_2609_35629_b200 import synth
 
 def geometry(spec: synth.WorkloadSpec) -> sp.Geometry:
     return sp.Geometry(spec.n_seqs, spec.n_q_heads, spec.n_kv_heads, spec.head_dim, spec.parent_size,
-                       spec.reps_per_parent)
+                       spec.reps_per_parent, sp.SANTAPP_FP16 if spec.elem == "fp16" else sp.SANTAPP_BF16)
 
 
 class GpuLayer:
@@ -26,10 +26,10 @@ class GpuLayer:
     def __init__(self, spec, data, device="cuda", builder=None):
         self.spec, self.data = spec, data
         self.geom = geometry(spec)
-        self.k_prompt = sp.bf16_bits_to_cuda(data.k_prompt, device)
-        self.v_prompt = sp.bf16_bits_to_cuda(data.v_prompt, device)
-        self.k_suffix = sp.bf16_bits_to_cuda(data.k_suffix, device)
-        self.v_suffix = sp.bf16_bits_to_cuda(data.v_suffix, device)
+        self.k_prompt = sp.bf16_bits_to_cuda(data.k_prompt, device, self.geom.torch_dtype)
+        self.v_prompt = sp.bf16_bits_to_cuda(data.v_prompt, device, self.geom.torch_dtype)
+        self.k_suffix = sp.bf16_bits_to_cuda(data.k_suffix, device, self.geom.torch_dtype)
+        self.v_suffix = sp.bf16_bits_to_cuda(data.v_suffix, device, self.geom.torch_dtype)
         self.teams = (builder or sp.santapp_build_teams)(self.geom, spec.prompt_len, self.k_prompt, self.v_prompt)
         torch.cuda.synchronize()
         t = self.teams
@@ -49,7 +49,7 @@ class GpuLayer:
         r0, r1 = int(self.seq_row_off[b]), int(self.seq_row_off[b + 1])
         ts = self.team_row_start[j, t0 + b: t1 + b + 1].astype(np.int32)
         tm = self.row_token[j, r0:r1].astype(np.int32)
-        rep = synth.bf16_to_f64(self.rep_bits[j, t0:t1])
+        rep = synth.to_f64(self.rep_bits[j, t0:t1], self.spec.elem)
         return ts, tm, rep
 
     def oracle_inputs(self, b):
@@ -67,8 +67,8 @@ class GpuLayer:
             ts[j, :len(s)] = s
             tm[j] = m
             rk[j, :len(rep)] = rep
-        k = synth.bf16_to_f64(self.data.k_prompt[:, r0:r1])
-        v = synth.bf16_to_f64(self.data.v_prompt[:, r0:r1])
+        k = synth.to_f64(self.data.k_prompt[:, r0:r1], self.spec.elem)
+        v = synth.to_f64(self.data.v_prompt[:, r0:r1], self.spec.elem)
         return dict(k=k, v=v, M=M, ts=ts, tm=tm, rk=rk, N=N)
 
 
@@ -81,9 +81,9 @@ def oracle_step(layer: GpuLayer, q_bits, suffix_len, K, seed, step, stream_base=
     for b in (range(spec.n_seqs) if seqs is None else seqs):
         oi = layer.oracle_inputs(b)
         t = int(suffix_len[b])
-        ks = synth.bf16_to_f64(layer.data.k_suffix[b, :, :t]) if t else None
-        vs = synth.bf16_to_f64(layer.data.v_suffix[b, :, :t]) if t else None
-        q = synth.bf16_to_f64(q_bits[b])
+        ks = synth.to_f64(layer.data.k_suffix[b, :, :t], spec.elem) if t else None
+        vs = synth.to_f64(layer.data.v_suffix[b, :, :t], spec.elem) if t else None
+        q = synth.to_f64(q_bits[b], spec.elem)
         if dense:
             out[b] = orc.dense_step(q, oi["k"], oi["v"], ks, vs, scale, n_threads=n_threads)
         else:
@@ -94,7 +94,7 @@ def oracle_step(layer: GpuLayer, q_bits, suffix_len, K, seed, step, stream_base=
 
 def gpu_step(layer: GpuLayer, q_bits, suffix_len, K, seed, step, stream_base=0, dense=False, debug=True):
     spec = layer.spec
-    q = sp.bf16_bits_to_cuda(q_bits)
+    q = sp.bf16_bits_to_cuda(q_bits, dtype=layer.geom.torch_dtype)
     sl = torch.from_numpy(np.asarray(suffix_len, dtype=np.int32)).cuda()
     if dense:
         out = sp.santapp_dense_decode_attn(layer.geom, layer.teams, q, layer.k_suffix, layer.v_suffix, sl)
@@ -108,4 +108,4 @@ def gpu_step(layer: GpuLayer, q_bits, suffix_len, K, seed, step, stream_base=0, 
 
 
 def max_abs_v(layer: GpuLayer):
-    return float(np.abs(synth.bf16_to_f32(layer.data.v_prompt)).max())
+    return float(np.abs(synth.to_f32(layer.data.v_prompt, layer.spec.elem)).max())

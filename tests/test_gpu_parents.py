@@ -82,7 +82,7 @@ def _check_records(layer, labels, n_parents):
         slots = int(layer.seq_team_off[b + 1] - layer.seq_team_off[b])
         assert slots == min(N, n_parents[b] * spec.reps_per_parent)
         for j in range(spec.n_kv_heads):
-            keys = synth.bf16_to_f64(layer.data.k_prompt[j, r0:r1])
+            keys = synth.to_f64(layer.data.k_prompt[j, r0:r1], spec.elem)
             lab = np.clip(labels[j, r0:r1], 0, n_parents[b] - 1)
             kept = np.unique(lab)
             ps = np.concatenate([[0], np.cumsum([np.count_nonzero(lab == u) for u in kept])]).astype(np.int32)

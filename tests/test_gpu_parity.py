@@ -40,7 +40,7 @@ def check_team_records(layer, seqs=None, kv_heads=None):
     for b in (range(spec.n_seqs) if seqs is None else seqs):
         r0, r1 = int(layer.seq_row_off[b]), int(layer.seq_row_off[b + 1])
         for j in (range(spec.n_kv_heads) if kv_heads is None else kv_heads):
-            keys = synth.bf16_to_f64(layer.data.k_prompt[j, r0:r1])
+            keys = synth.to_f64(layer.data.k_prompt[j, r0:r1], spec.elem)
             ts_o, tm_o, rep_o = orc.build_teams_contiguous(keys, spec.parent_size, spec.reps_per_parent)
             ts_g, tm_g, rep_g = layer.records(b, j)
             assert np.array_equal(ts_g, ts_o)
