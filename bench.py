@@ -57,6 +57,7 @@ def parse_args():
     ap.add_argument("--n-sample", type=int, default=0, help="override K")
     ap.add_argument("--key-layout", default="iid", choices=["iid", "runs"],
                     help="cluster of each prompt row: independent draws, or geometric runs (positional locality)")
+    ap.add_argument("--elem", default="bf16", choices=["bf16", "fp16"], help="16-bit element type of q, K, V")
     ap.add_argument("--parents", default="contiguous", choices=["contiguous", "centres"],
                     help="contiguous: Algorithm 4; centres: the partition Algorithm 3 returns when the fit "
                          "recovers the centres the synthetic keys were drawn around")
@@ -85,6 +86,7 @@ def make_spec(args, seed):
         spec.n_sample = args.n_sample
     spec.key_layout = args.key_layout
     spec.parents = getattr(args, "parents", "contiguous")
+    spec.elem = getattr(args, "elem", "bf16")
     return spec
 
 
@@ -92,7 +94,7 @@ def workload_text(spec, layers):
     return (f"{spec.name}: {spec.n_seqs} seq x {spec.n_q_heads} q heads / {spec.n_kv_heads} KV heads, d={spec.head_dim}, "
             f"prompt {min(spec.prompt_len)}..{max(spec.prompt_len)}, suffix cap {spec.suffix_cap}, "
             f"P={spec.parent_size}, R={spec.reps_per_parent}, K={spec.n_sample}, keys {spec.key_layout}, "
-            f"{getattr(spec, 'parents', 'contiguous')} parents, {layers} layers round-robin")
+            f"{getattr(spec, 'parents', 'contiguous')} parents, {spec.elem} inputs, {layers} layers round-robin")
 
 
 # -------------------------------------------------------------------------------------------
@@ -173,8 +175,8 @@ def run_reference(args):
     scale = 1.0 / math.sqrt(spec.head_dim)
     b = 0
     r0, r1 = int(data.seq_row_off[b]), int(data.seq_row_off[b + 1])
-    k = synth.bf16_to_f64(data.k_prompt[:, r0:r1])
-    v = synth.bf16_to_f64(data.v_prompt[:, r0:r1])
+    k = synth.to_f64(data.k_prompt[:, r0:r1], spec.elem)
+    v = synth.to_f64(data.v_prompt[:, r0:r1], spec.elem)
     recs = [orc.build_teams_contiguous(k[j], spec.parent_size, spec.reps_per_parent)
             for j in range(spec.n_kv_heads)]
     M = np.array([len(r[0]) - 1 for r in recs], dtype=np.int32)
@@ -187,10 +189,10 @@ def run_reference(args):
         rk[j, :len(rep)] = k[j][rep]
 
     def one(step):
-        q = synth.bf16_to_f64(synth.make_queries(spec, data, step)[b])
+        q = synth.to_f64(synth.make_queries(spec, data, step)[b], spec.elem)
         t = int(spec.suffix_len(step)[b])
-        ks = synth.bf16_to_f64(data.k_suffix[b, :, :t]) if t else None
-        vs = synth.bf16_to_f64(data.v_suffix[b, :, :t]) if t else None
+        ks = synth.to_f64(data.k_suffix[b, :, :t], spec.elem) if t else None
+        vs = synth.to_f64(data.v_suffix[b, :, :t], spec.elem) if t else None
         t0 = time.perf_counter()
         orc.decode_step(q, k, v, M, ts, tm, rk, ks, vs, spec.n_sample, 0, step, b, scale, n_threads=cores)
         return time.perf_counter() - t0
@@ -260,7 +262,8 @@ def measure_workload(args, workload, n_layers, n_steps, n_warmup, dev, want_e2e,
     spec = make_spec(wl_args, seed=replicas.replica_seed(0, rank))
     L = n_layers
     geom = sp.Geometry(spec.n_seqs, spec.n_q_heads, spec.n_kv_heads, spec.head_dim, spec.parent_size,
-                       spec.reps_per_parent)
+                       spec.reps_per_parent, sp.SANTAPP_FP16 if spec.elem == "fp16" else sp.SANTAPP_BF16)
+    edt = geom.torch_dtype
     K = spec.n_sample
     B, Hq, Hkv, d = spec.n_seqs, spec.n_q_heads, spec.n_kv_heads, spec.head_dim
     conc = spec.query_kind == "concentrated"
@@ -270,15 +273,15 @@ def measure_workload(args, workload, n_layers, n_steps, n_warmup, dev, want_e2e,
     layers, host_layers = [], []
     q_all = np.empty((N_STEP_INPUTS, L, B, Hq, d), dtype=np.uint16)
     cap = max(spec.suffix_cap, 1)
-    ksuf_all = torch.empty((L, B, Hkv, cap, d), dtype=torch.bfloat16, device=dev)
+    ksuf_all = torch.empty((L, B, Hkv, cap, d), dtype=edt, device=dev)
     vsuf_all = torch.empty_like(ksuf_all)
     for l in range(L):
         by_centres = spec.parents == "centres"
         data = synth.make_layer(spec, layer=l, keep_centres=conc or by_centres)
         for s in range(N_STEP_INPUTS):
             q_all[s, l] = synth.make_queries(spec, data, s)
-        k_prompt = sp.bf16_bits_to_cuda(data.k_prompt, dev)
-        v_prompt = sp.bf16_bits_to_cuda(data.v_prompt, dev)
+        k_prompt = sp.bf16_bits_to_cuda(data.k_prompt, dev, edt)
+        v_prompt = sp.bf16_bits_to_cuda(data.v_prompt, dev, edt)
         if by_centres:
             # Algorithm 3 with the fit replaced by its ideal outcome on these keys: the centres the
             # rows were drawn around, as many as its first line asks for
@@ -294,8 +297,8 @@ def measure_workload(args, workload, n_layers, n_steps, n_warmup, dev, want_e2e,
         torch.cuda.synchronize()
         build_ms = 1e3 * (time.perf_counter() - t_build)
         del k_prompt, v_prompt
-        ksuf_all[l].copy_(sp.bf16_bits_to_cuda(data.k_suffix, dev))
-        vsuf_all[l].copy_(sp.bf16_bits_to_cuda(data.v_suffix, dev))
+        ksuf_all[l].copy_(sp.bf16_bits_to_cuda(data.k_suffix, dev, edt))
+        vsuf_all[l].copy_(sp.bf16_bits_to_cuda(data.v_suffix, dev, edt))
         layers.append(dict(teams=teams, k_suffix=ksuf_all[l], v_suffix=vsuf_all[l]))
         if l == 0:
             host_layers.append(data)
@@ -317,7 +320,7 @@ def measure_workload(args, workload, n_layers, n_steps, n_warmup, dev, want_e2e,
         row[q_bytes + 4 * B:in_bytes] = np.array([step_ids[s]], dtype=np.uint32).view(np.uint8)
     inputs_dev = inputs_host.to(dev)
     cur = torch.zeros(in_bytes_pad, dtype=torch.uint8, device=dev)
-    q_cur = cur[:q_bytes].view(torch.bfloat16).view(L, B, Hq, d)
+    q_cur = cur[:q_bytes].view(edt).view(L, B, Hq, d)
     sl_cur = cur[q_bytes:q_bytes + 4 * B].view(torch.int32)
     step_cur = cur[q_bytes + 4 * B:in_bytes].view(torch.int32)
     out = torch.zeros((L, B, Hq, d), dtype=torch.float32, device=dev)
@@ -482,13 +485,13 @@ def measure_workload(args, workload, n_layers, n_steps, n_warmup, dev, want_e2e,
     # ---- end to end through host buffers ----
     e2e = None
     if want_e2e:
-        new_rows = torch.zeros((N_STEP_INPUTS, 2, B, L, Hkv, d), dtype=torch.bfloat16).pin_memory()
+        new_rows = torch.zeros((N_STEP_INPUTS, 2, B, L, Hkv, d), dtype=edt).pin_memory()
         for s in range(N_STEP_INPUTS):
             for b in range(B):
                 t = max(int(sl_all[s, b]) - 1, 0)
                 new_rows[s, 0, b] = ksuf_all[:, b, :, t].cpu()
                 new_rows[s, 1, b] = vsuf_all[:, b, :, t].cpu()
-        new_dev = torch.zeros((2, B, L, Hkv, d), dtype=torch.bfloat16, device=dev)
+        new_dev = torch.zeros((2, B, L, Hkv, d), dtype=edt, device=dev)
         out_host = torch.zeros((L, B, Hq, d), dtype=torch.float32).pin_memory()
 
         def e2e_step(i):
@@ -518,7 +521,7 @@ def measure_workload(args, workload, n_layers, n_steps, n_warmup, dev, want_e2e,
         line = {
             "metric": METRIC, "value": us_layer, "unit": UNIT, "n_gpus": world, "steps": Kst, "warmup": W,
             "ms_per_step": ms_sparse / Kst, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
-            "dtype": "bf16", "data": "synthetic",
+            "dtype": spec.elem, "data": "synthetic",
             "config": {"workload": workload_text(spec, L), "l2": "inputs larger than L2: layers visited round-robin",
                        "replay": "CUDA graph of one decode step over all layers", "replicas": world},
             "clocks": clocks, "gpu_launches": int(Kst * L * launches_per_layer_step),
@@ -560,18 +563,18 @@ def cpu_baseline_leg(spec, data, teams, seed):
     M = np.ascontiguousarray(teams.team_count.cpu().numpy()[:, b], dtype=np.int32)     # teams of each KV head
     ts = np.ascontiguousarray(trs[:, t0 + b:t1 + b + 1])
     tm = np.ascontiguousarray(tok[:, r0:r1])
-    rk = synth.bf16_to_f64(rep_bits[:, t0:t1])
-    k = synth.bf16_to_f64(data.k_prompt[:, r0:r1])
-    v = synth.bf16_to_f64(data.v_prompt[:, r0:r1])
+    rk = synth.to_f64(rep_bits[:, t0:t1], spec.elem)
+    k = synth.to_f64(data.k_prompt[:, r0:r1], spec.elem)
+    v = synth.to_f64(data.v_prompt[:, r0:r1], spec.elem)
     scale = 1.0 / math.sqrt(d)
     times, n = [], 0
     budget = time.perf_counter() + 12.0
     while time.perf_counter() < budget and n < 4000:
         step = n % spec.n_steps
-        q = synth.bf16_to_f64(synth.make_queries(spec, data, step % N_STEP_INPUTS)[b])
+        q = synth.to_f64(synth.make_queries(spec, data, step % N_STEP_INPUTS)[b], spec.elem)
         t = int(spec.suffix_len(step)[b])
-        ks = synth.bf16_to_f64(data.k_suffix[b, :, :t]) if t else None
-        vs = synth.bf16_to_f64(data.v_suffix[b, :, :t]) if t else None
+        ks = synth.to_f64(data.k_suffix[b, :, :t], spec.elem) if t else None
+        vs = synth.to_f64(data.v_suffix[b, :, :t], spec.elem) if t else None
         s0 = time.perf_counter()
         orc.decode_step(q, k, v, M, ts, tm, rk, ks, vs, spec.n_sample, seed, step, b, scale, n_threads=cores)
         times.append(time.perf_counter() - s0)
@@ -590,10 +593,10 @@ def cpu_baseline_leg(spec, data, teams, seed):
 
     def inputs(i):
         step = i % spec.n_steps
-        q = synth.bf16_to_f64(synth.make_queries(spec, data, step % N_STEP_INPUTS)[b])
+        q = synth.to_f64(synth.make_queries(spec, data, step % N_STEP_INPUTS)[b], spec.elem)
         t = int(spec.suffix_len(step)[b])
-        ks = synth.bf16_to_f64(data.k_suffix[b, :, :t]) if t else None
-        vs = synth.bf16_to_f64(data.v_suffix[b, :, :t]) if t else None
+        ks = synth.to_f64(data.k_suffix[b, :, :t], spec.elem) if t else None
+        vs = synth.to_f64(data.v_suffix[b, :, :t], spec.elem) if t else None
         return q, ks, vs, step
 
     def sparse_1(i):
