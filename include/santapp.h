@@ -12,6 +12,9 @@
  *                              (Algorithm 1) under the GQA rule of the Method section.
  *   santapp_dense_decode_attn  full-cache attention, Eq. (method-attention), over the same
  *                              buffers: the in-library dense baseline.
+ * Beside them: santapp_assign_parents and santapp_build_teams_parents (Algorithm 3 after the fit:
+ * nearest-centre parents, then Algorithm 2 on parents of any size) and santapp_build_groups_mean
+ * (the centroid-guided baseline of the routing diagnostic).
  *
  * Conventions
  *   - "device" pointers address GPU global memory of the current device; "host" pointers
