@@ -251,6 +251,18 @@ int santapp_build_teams_parents(const santapp_geom *geom, const int32_t *prompt_
                                 const void *v_prompt, const int32_t *parent_of, santapp_teams *teams,
                                 void *workspace, size_t workspace_bytes, santapp_stream stream);
 
+/*
+ * Centroid-guided groups on a given parent partition (the paper's baseline forms its groups by
+ * k-means): as santapp_build_groups_mean, but one group per non-empty parent of `parent_of`, in label
+ * order, members in token order. geom->reps_per_parent must be 1; bf16 inputs only. Arguments,
+ * sizes (santapp_parent_teams_sizes) and errors as for santapp_build_teams_parents.
+ */
+int santapp_build_groups_mean_parents(const santapp_geom *geom, const int32_t *prompt_len_host,
+                                      const int32_t *n_parents_host, const void *k_prompt,
+                                      const void *v_prompt, const int32_t *parent_of,
+                                      santapp_teams *teams, void *workspace, size_t workspace_bytes,
+                                      santapp_stream stream);
+
 /* Workspace bytes santapp_decode_attn needs for n_sample = K on these team records. */
 size_t santapp_decode_workspace_bytes(const santapp_geom *geom, const santapp_teams *teams,
                                       int32_t n_sample);

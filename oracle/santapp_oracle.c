@@ -26,6 +26,7 @@
  *   orc_routing_kl            routing-agreement diagnostic, Eq. (diagnostic-kl)
  *   orc_group_mean_keys       centroid-guided baseline of the routing diagnostic: one group per
  *                             parent, routed by the arithmetic mean of its keys
+ *   orc_group_mean_keys_parents   the same baseline on an arbitrary partition (k-means groups)
  *   orc_kmeans_parent_count, orc_nearest_centre_parents
  *                             Algorithm 3 without the fit: the number of centres, and the
  *                             nearest-centre partition with empty parents omitted (the
@@ -670,4 +671,27 @@ int32_t orc_nearest_centre_parents(int32_t N, int d, const double *keys,
         if (filled > before) parent_start[++n_parents] = filled;
     }
     return n_parents;
+}
+
+/* The centroid-guided baseline on an arbitrary parent partition (the paper forms its groups by
+ * k-means): one group per parent, members in increasing token index, routing key = arithmetic
+ * mean of the parent's keys (fp64 sum in token order, one division), stored as a bf16 value
+ * (fp64 -> fp32 to nearest -> bf16 to nearest even) and widened back into out_mean[n_parents][d]. */
+void orc_group_mean_keys_parents(int d, const double *keys, int32_t n_parents, const int32_t *parent_start,
+                                 const int32_t *parent_member, double *out_mean)
+{
+    for (int32_t u = 0; u < n_parents; ++u) {
+        int32_t lo = parent_start[u], hi = parent_start[u + 1];
+        for (int j = 0; j < d; ++j) {
+            double sum = 0.0;
+            for (int32_t a = lo; a < hi; ++a) sum += keys[(int64_t)parent_member[a] * d + j];
+            float f = (float)(sum / (double)(hi - lo));
+            uint32_t bits;
+            memcpy(&bits, &f, sizeof bits);
+            uint32_t rounded = (bits + 0x7FFFu + ((bits >> 16) & 1u)) & 0xFFFF0000u;
+            float back;
+            memcpy(&back, &rounded, sizeof back);
+            out_mean[(int64_t)u * d + j] = (double)back;
+        }
+    }
 }

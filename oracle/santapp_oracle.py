@@ -85,6 +85,8 @@ def lib():
         L.orc_routing_kl.restype = _c.c_double
         L.orc_group_mean_keys.argtypes = [_c.c_int32, _c.c_int, _f64p, _c.c_int32, _f64p]
         L.orc_group_mean_keys.restype = _c.c_int32
+        L.orc_group_mean_keys_parents.argtypes = [_c.c_int, _f64p, _c.c_int32, _i32p, _i32p, _f64p]
+        L.orc_group_mean_keys_parents.restype = None
         L.orc_kmeans_parent_count.argtypes = [_c.c_int32, _c.c_int32]
         L.orc_kmeans_parent_count.restype = _c.c_int32
         L.orc_nearest_centre_parents.argtypes = [_c.c_int32, _c.c_int, _f64p, _c.c_int32, _f64p, _i32p, _i32p, _i32p]
@@ -347,3 +349,14 @@ def nearest_centre_parents(keys, centres):
     parent_member = np.zeros(N, dtype=np.int32)
     n = lib().orc_nearest_centre_parents(N, d, keys, centres.shape[0], centres, label, parent_start, parent_member)
     return label, parent_start[: n + 1].copy(), parent_member
+
+
+def group_mean_keys_parents(keys, parent_start, parent_member):
+    """Centroid-guided groups on a given partition: (team_start, team_member, mean_key), one group
+    per parent, members in token order, the mean key rounded to a bf16 value."""
+    keys = _f64(keys)
+    parent_start, parent_member = _i32(parent_start), _i32(parent_member)
+    n = parent_start.shape[0] - 1
+    mean = np.zeros((n, keys.shape[1]))
+    lib().orc_group_mean_keys_parents(keys.shape[1], keys, n, parent_start, parent_member, mean)
+    return parent_start.copy(), parent_member.copy(), mean

@@ -32,7 +32,7 @@ EXPORTS = [
     "santapp_dense_workspace_bytes", "santapp_dense_decode_attn", "santapp_last_launch_count",
     "santapp_set_stage_mask", "santapp_dense_decode_attn_noalloc", "santapp_build_groups_mean",
     "santapp_kmeans_parent_count", "santapp_assign_parents_workspace_bytes", "santapp_assign_parents",
-    "santapp_parent_teams_sizes", "santapp_build_teams_parents",
+    "santapp_parent_teams_sizes", "santapp_build_teams_parents", "santapp_build_groups_mean_parents",
 ]
 
 STAGE_ROUTE, STAGE_SELECT, STAGE_ATTEND, STAGE_ALL = 1, 2, 4, 7
@@ -110,6 +110,8 @@ def load_library(path: Optional[str] = None):
     L.santapp_build_teams_parents.argtypes = [ctypes.POINTER(CGeom), ctypes.POINTER(i32), ctypes.POINTER(i32), vp, vp,
                                               vp, ctypes.POINTER(CTeams), vp, sz, vp]
     L.santapp_build_teams_parents.restype = ctypes.c_int
+    L.santapp_build_groups_mean_parents.argtypes = L.santapp_build_teams_parents.argtypes
+    L.santapp_build_groups_mean_parents.restype = ctypes.c_int
     L.santapp_decode_workspace_bytes.argtypes = [ctypes.POINTER(CGeom), ctypes.POINTER(CTeams), i32]
     L.santapp_decode_workspace_bytes.restype = sz
     L.santapp_dense_workspace_bytes.argtypes = [ctypes.POINTER(CGeom), ctypes.POINTER(CTeams)]
@@ -286,8 +288,16 @@ def santapp_parent_teams_sizes(geom: Geometry, prompt_len, n_parents) -> Sizes:
                  out.team_row_start_elems, out.build_workspace_bytes)
 
 
+def santapp_build_groups_mean_parents(geom: Geometry, prompt_len, n_parents, k_prompt: torch.Tensor,
+                                      v_prompt: torch.Tensor, parent_of: torch.Tensor, stream=None) -> Teams:
+    """Centroid-guided groups on a given partition (geom.reps_per_parent must be 1)."""
+    return santapp_build_teams_parents(geom, prompt_len, n_parents, k_prompt, v_prompt, parent_of, stream,
+                                       _entry="santapp_build_groups_mean_parents")
+
+
 def santapp_build_teams_parents(geom: Geometry, prompt_len, n_parents, k_prompt: torch.Tensor,
-                                v_prompt: torch.Tensor, parent_of: torch.Tensor, stream=None) -> Teams:
+                                v_prompt: torch.Tensor, parent_of: torch.Tensor, stream=None,
+                                _entry: str = "santapp_build_teams_parents") -> Teams:
     """Team records from a parent label per token (int32 CUDA tensor [n_kv_heads, rows_total])."""
     L = load_library()
     sizes = santapp_parent_teams_sizes(geom, prompt_len, n_parents)
@@ -296,9 +306,9 @@ def santapp_build_teams_parents(geom: Geometry, prompt_len, n_parents, k_prompt:
     g = geom.c()
     if parent_of.dtype != torch.int32:
         raise SantappError(SANTAPP_ERR_INVALID_ARG, "parent_of must be int32")
-    _check(L.santapp_build_teams_parents(ctypes.byref(g), _i32_array(prompt_len), _i32_array(n_parents),
-                                         _ptr(k_prompt), _ptr(v_prompt), _ptr(parent_of), ctypes.byref(teams.c),
-                                         _ptr(ws), ws.numel(), _stream_ptr(stream)))
+    _check(getattr(L, _entry)(ctypes.byref(g), _i32_array(prompt_len), _i32_array(n_parents),
+                              _ptr(k_prompt), _ptr(v_prompt), _ptr(parent_of), ctypes.byref(teams.c),
+                              _ptr(ws), ws.numel(), _stream_ptr(stream)))
     teams._build_ws = ws      # keep alive until the stream has consumed it
     return teams
 

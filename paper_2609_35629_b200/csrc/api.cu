@@ -379,9 +379,10 @@ int santapp_parent_teams_sizes(const santapp_geom *geom, const int32_t *prompt_l
     return SANTAPP_OK;
 }
 
-int santapp_build_teams_parents(const santapp_geom *geom, const int32_t *prompt_len_host, const int32_t *n_parents_host,
-                                const void *k_prompt, const void *v_prompt, const int32_t *parent_of,
-                                santapp_teams *teams, void *workspace, size_t workspace_bytes, santapp_stream stream)
+static int build_parent_records(const santapp_geom *geom, const int32_t *prompt_len_host,
+                                const int32_t *n_parents_host, const void *k_prompt, const void *v_prompt,
+                                const int32_t *parent_of, santapp_teams *teams, void *workspace,
+                                size_t workspace_bytes, santapp_stream stream, bool mean_keys)
 {
     santapp_sizes sz;
     int rc = santapp_parent_teams_sizes(geom, prompt_len_host, n_parents_host, &sz);
@@ -431,6 +432,7 @@ int santapp_build_teams_parents(const santapp_geom *geom, const int32_t *prompt_
     ParentBuildParams p;
     p.bv = make_view(geom, teams);
     p.reps = geom->reps_per_parent;
+    p.mean_keys = mean_keys;
     p.max_labels_per_seq = max_labels;
     p.max_rows_per_seq = sz.max_rows_per_seq;
     p.labels_total = label_off[B];
@@ -459,6 +461,25 @@ int santapp_build_teams_parents(const santapp_geom *geom, const int32_t *prompt_
     err = launch_rep_abs_max(p.bv, p.rep_keys, teams->rep_abs_max, s);
     if (err != cudaSuccess) return cuda_fail(err, "rep_abs_max launch");
     return SANTAPP_OK;
+}
+
+int santapp_build_teams_parents(const santapp_geom *geom, const int32_t *prompt_len_host, const int32_t *n_parents_host,
+                                const void *k_prompt, const void *v_prompt, const int32_t *parent_of,
+                                santapp_teams *teams, void *workspace, size_t workspace_bytes, santapp_stream stream)
+{
+    return build_parent_records(geom, prompt_len_host, n_parents_host, k_prompt, v_prompt, parent_of, teams, workspace,
+                                workspace_bytes, stream, false);
+}
+
+int santapp_build_groups_mean_parents(const santapp_geom *geom, const int32_t *prompt_len_host,
+                                      const int32_t *n_parents_host, const void *k_prompt, const void *v_prompt,
+                                      const int32_t *parent_of, santapp_teams *teams, void *workspace,
+                                      size_t workspace_bytes, santapp_stream stream)
+{
+    if (geom && geom->reps_per_parent != 1) return SANTAPP_ERR_INVALID_ARG;    // one group per parent
+    if (geom && geom->elem_type != SANTAPP_BF16) return SANTAPP_ERR_UNSUPPORTED;
+    return build_parent_records(geom, prompt_len_host, n_parents_host, k_prompt, v_prompt, parent_of, teams, workspace,
+                                workspace_bytes, stream, true);
 }
 
 }  // extern "C"

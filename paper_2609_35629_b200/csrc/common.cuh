@@ -189,6 +189,7 @@ cudaError_t launch_assign_parents(const AssignParams &p, cudaStream_t s);
 struct ParentBuildParams {
     BatchView bv;                           // seq_team_off: team slots per sequence
     int reps, max_labels_per_seq, max_rows_per_seq;
+    bool mean_keys;                         // one group per parent routed by its mean key (reps = 1)
     int64_t labels_total;
     const uint16_t *k_prompt, *v_prompt;    // [n_kv][rows_total][128] token order
     const int32_t *parent_of;               // [n_kv][rows_total] label of each token

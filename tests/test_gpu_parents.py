@@ -210,3 +210,33 @@ def test_centre_parents_paper_point_32k():
     layer, _, _, _ = _centre_layer(spec)
     assert len({int(c) for c in layer.team_count[:, 0]}) > 1
     check_sparse_step(layer, 0, K=31)
+
+
+def test_centroid_groups_on_centre_parents():
+    """The paper's centroid-guided baseline on a clustering's groups (nominal group size 16): one
+    group per non-empty parent routed by its mean key; records equal to the oracle's, decode as usual."""
+    spec = _spec(prompt=(2048, 1100), n_sample=12, R=1, n_clusters=128)
+    spec.parent_size = 16
+    data = synth.make_layer(spec, layer=0, keep_centres=True)
+    n_centres = [sp.santapp_kmeans_parent_count(n, spec.parent_size) for n in spec.prompt_len]     # 128, 68
+    cen = np.ascontiguousarray(np.concatenate([data.centres[:, :n] for n in n_centres], axis=1))
+    labels = _labels_gpu(spec, data, n_centres, cen)
+    lab_dev = torch.from_numpy(labels).cuda()
+
+    def builder(geom, prompt_len, k, v):
+        return sp.santapp_build_groups_mean_parents(geom, prompt_len, n_centres, k, v, lab_dev)
+    layer = pu.GpuLayer(spec, data, builder=builder)
+    for b in range(spec.n_seqs):
+        r0, r1 = int(layer.seq_row_off[b]), int(layer.seq_row_off[b + 1])
+        for j in range(spec.n_kv_heads):
+            keys = synth.bf16_to_f64(data.k_prompt[j, r0:r1])
+            _, ps, pm = orc.nearest_centre_parents(keys, cen[j, sum(n_centres[:b]):sum(n_centres[:b + 1])].astype(np.float64))
+            ts_o, tm_o, mean_o = orc.group_mean_keys_parents(keys, ps, pm)
+            ts_g, tm_g, rep_g = layer.records(b, j)
+            assert np.array_equal(ts_g, ts_o) and np.array_equal(tm_g, tm_o) and np.array_equal(rep_g, mean_o)
+            assert np.array_equal(layer.k_packed_bits[j, r0:r1], data.k_prompt[j, r0:r1][tm_g])
+    for step in range(2):
+        check_sparse_step(layer, step, spec.n_sample)
+    bad = pu.geometry(_spec(prompt=(2048, 1100), R=4))
+    with pytest.raises(sp.SantappError):
+        sp.santapp_build_groups_mean_parents(bad, spec.prompt_len, n_centres, layer.k_prompt, layer.v_prompt, lab_dev)

@@ -51,3 +51,24 @@ def test_decode_with_mean_keys_keeps_the_dense_limit():
     ts, tm, mean = orc.group_mean_keys(k, 8)
     r = orc.decode_head_given_gumbel(q, k, v, ts, tm, mean, None, None, 8, None, 0.25)
     assert np.allclose(r.o, orc.dense_head(q, k, v, 0.25), rtol=0, atol=1e-12)
+
+
+def test_arbitrary_partition_reduces_to_the_contiguous_one():
+    """On the contiguous partition the general routine must give the contiguous routine's keys."""
+    rng = np.random.default_rng(3)
+    k = synth.bf16_to_f64(synth.f32_to_bf16_bits(rng.normal(size=(45, 8)).astype(np.float32)))
+    ts, tm, mean = orc.group_mean_keys(k, 7)
+    ts2, tm2, mean2 = orc.group_mean_keys_parents(k, ts, tm)
+    assert np.array_equal(ts, ts2) and np.array_equal(tm, tm2) and np.array_equal(mean, mean2)
+
+
+def test_arbitrary_partition_hand_worked_and_rounded():
+    k = np.array([[1.0, 10.0], [2.0, 20.0], [4.0, 40.0], [8.0, 80.0], [16.0, 160.0]])
+    ps = np.array([0, 2, 5], dtype=np.int32)
+    pm = np.array([4, 0, 1, 2, 3], dtype=np.int32)                 # parents {4, 0} and {1, 2, 3}
+    _, _, mean = orc.group_mean_keys_parents(k, ps, pm)
+    # (16 + 1) / 2 = 8.5 and (160 + 10) / 2 = 85 are bf16 values; (2 + 4 + 8) / 3 = 4.666..., (20 + 40 + 80) / 3 = 46.66...
+    assert np.array_equal(mean[0], [8.5, 85.0])
+    want = synth.bf16_to_f64(synth.f32_to_bf16_bits(np.array([14.0 / 3.0, 140.0 / 3.0], dtype=np.float32)))
+    assert np.array_equal(mean[1], want)
+    assert mean[1, 0] == 4.65625 and mean[1, 1] == 46.75           # nearest bf16 values, by hand
