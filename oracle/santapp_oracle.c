@@ -27,10 +27,11 @@
  *   orc_group_mean_keys       centroid-guided baseline of the routing diagnostic: one group per
  *                             parent, routed by the arithmetic mean of its keys
  *   orc_group_mean_keys_parents   the same baseline on an arbitrary partition (k-means groups)
+ *   orc_minibatch_kmeans      the fit of Algorithm 3 (minibatch k-means, greedy k-means++ start) in the
+ *                             reading spelled out above the function
  *   orc_kmeans_parent_count, orc_nearest_centre_parents
  *                             Algorithm 3 without the fit: the number of centres, and the
- *                             nearest-centre partition with empty parents omitted (the
- *                             centres are an input)
+ *                             nearest-centre partition with empty parents omitted
  *
  * Parity pins (tests marked "not gpu"): Philox words against an independent
  * library generator; Gumbel law by Kolmogorov-Smirnov and moments; first-draw
@@ -42,7 +43,10 @@
  * figures the paper prints; the routing KL against its closed forms (zero for
  * singleton teams, log N - H(p) for one team holding every key) and against a
  * numpy re-evaluation of the defining sum; the nearest-centre partition against a library
- * vector quantiser, hand-worked ties and empty centres, and brute force over all labellings.
+ * vector quantiser, hand-worked ties and empty centres, and brute force over all labellings; the
+ * fit by recovery of separated blobs, the k = N and k = 1 special cases (the latter against the
+ * mean of the recomputed draws), its step limits, the reassignment of a starved centre, and its
+ * inertia against a library's minibatch and full-batch k-means.
  * Parity unpinned: nothing in this file. (Accuracy of the sampled output
  * against dense attention on real model data is outside what can be pinned
  * here; only the estimator identities are.)
@@ -694,4 +698,178 @@ void orc_group_mean_keys_parents(int d, const double *keys, int32_t n_parents, c
             out_mean[(int64_t)u * d + j] = (double)back;
         }
     }
+}
+
+/* ------------------------------------------------------------------------- */
+/* Algorithm 3, the fit: minibatch k-means with greedy k-means++ start        */
+/* ------------------------------------------------------------------------- */
+
+/* The paper names the routine and its settings (squared-Euclidean centres on the raw keys, greedy
+ * k-means++ initialisation, minibatches sampled with replacement, cumulative-count centre updates,
+ * a no-improvement stopping rule, a reassignment ratio, tolerance zero, a seed) and leaves the
+ * rest to "the implementation default". This is the reading taken here, step by step; every random
+ * choice is a word of the Philox stream with counter (slot, tag, stream, step) and the seed as key,
+ * so the fit is a pure function of its arguments.
+ *
+ *  1. Initialisation sample: n_init = min(N, max(3 * batch, 3 * k)) distinct keys, the head of a
+ *     Fisher-Yates shuffle of 0..N-1 (tag 1: position i swaps with i + floor(word * (N - i) / 2^32)).
+ *  2. Greedy k-means++ on the sample, L = 2 + floor(ln k) trials per centre (tag 2): the first
+ *     centre is a uniform sample point; each later one is the best of L points drawn with
+ *     probability proportional to the squared distance to the nearest centre chosen so far (inverse
+ *     CDF over the sample in order), "best" meaning the smallest resulting potential
+ *     sum_i min(closest_i, |x_i - candidate|^2), ties to the earlier trial.
+ *  3. At most max_iter * ceil(N / batch) minibatch steps. Step t draws `batch` indices uniformly
+ *     with replacement (tag 3), assigns each to its nearest centre (ties to the smaller index),
+ *     then moves every centre that received points to the mean of all points it has received so
+ *     far: c <- (c * count + sum of the new points) / (count + n), count <- count + n.
+ *  4. Reassignment, at steps with (t + 1) divisible by 10 + floor(smallest count): centres whose
+ *     count is below ratio * (largest count), at most batch / 2 of them, in index order, jump onto
+ *     distinct points of the current minibatch (head of a Fisher-Yates shuffle of its slots, tag 4)
+ *     and take the smallest count among the centres that stay.
+ *  5. Stopping: the per-point inertia of each minibatch (measured before its update) feeds an
+ *     exponentially weighted average with alpha = min(1, 2 * batch / (N + 1)); the fit stops after
+ *     `patience` consecutive steps without a new minimum of that average.
+ * Returns the number of steps run; centres[k][d] are the fp64 centres. */
+static uint32_t km_word(uint64_t seed, uint32_t slot, uint32_t tag, uint32_t stream, uint32_t step)
+{
+    uint32_t ctr[4] = {slot, tag, stream, step};
+    uint32_t key[2] = {(uint32_t)(seed & 0xFFFFFFFFu), (uint32_t)(seed >> 32)};
+    uint32_t out[4];
+    orc_philox4x32_10(ctr, key, out);
+    return out[0];
+}
+
+static int32_t km_index(uint32_t word, int32_t n) { return (int32_t)(((uint64_t)word * (uint64_t)n) >> 32); }
+
+int32_t orc_minibatch_kmeans(int32_t N, int d, const double *keys, int32_t k, int32_t batch, int32_t max_iter,
+                             int32_t patience, double ratio, uint64_t seed, uint32_t stream, double *centres)
+{
+    /* 1. initialisation sample */
+    int32_t n_init = 3 * batch > 3 * k ? 3 * batch : 3 * k;
+    if (n_init > N) n_init = N;
+    int32_t *perm = (int32_t *)malloc(sizeof(int32_t) * (size_t)N);
+    for (int32_t i = 0; i < N; ++i) perm[i] = i;
+    for (int32_t i = 0; i < n_init; ++i) {
+        int32_t r = i + km_index(km_word(seed, (uint32_t)i, 1u, stream, 0u), N - i);
+        int32_t t = perm[i]; perm[i] = perm[r]; perm[r] = t;
+    }
+    /* 2. greedy k-means++ */
+    int32_t L = 2 + (int32_t)floor(log((double)k));
+    double *closest = (double *)malloc(sizeof(double) * (size_t)n_init);
+    double *cand = (double *)malloc(sizeof(double) * (size_t)n_init * (size_t)L);
+    int32_t *pick = (int32_t *)malloc(sizeof(int32_t) * (size_t)L);
+    {
+        int32_t first = km_index(km_word(seed, 0u, 2u, stream, 0u), n_init);
+        memcpy(centres, keys + (int64_t)perm[first] * d, sizeof(double) * (size_t)d);
+        for (int32_t i = 0; i < n_init; ++i) closest[i] = sqdist(keys + (int64_t)perm[i] * d, centres, d);
+    }
+    for (int32_t c = 1; c < k; ++c) {
+        double total = 0.0;
+        for (int32_t i = 0; i < n_init; ++i) total += closest[i];
+        for (int32_t l = 0; l < L; ++l) {
+            double target = orc_uniform_open(km_word(seed, (uint32_t)l, 2u, stream, (uint32_t)c)) * total;
+            double cum = 0.0;
+            int32_t at = n_init - 1;
+            for (int32_t i = 0; i < n_init; ++i) {
+                cum += closest[i];
+                if (cum > target) { at = i; break; }
+            }
+            pick[l] = at;
+        }
+        int32_t best = 0;
+        double best_pot = INFINITY;
+        for (int32_t l = 0; l < L; ++l) {
+            const double *x = keys + (int64_t)perm[pick[l]] * d;
+            double pot = 0.0;
+            for (int32_t i = 0; i < n_init; ++i) {
+                double dist = sqdist(keys + (int64_t)perm[i] * d, x, d);
+                cand[(int64_t)l * n_init + i] = dist;
+                pot += dist < closest[i] ? dist : closest[i];
+            }
+            if (pot < best_pot) { best_pot = pot; best = l; }
+        }
+        memcpy(centres + (int64_t)c * d, keys + (int64_t)perm[pick[best]] * d, sizeof(double) * (size_t)d);
+        for (int32_t i = 0; i < n_init; ++i) {
+            double dist = cand[(int64_t)best * n_init + i];
+            if (dist < closest[i]) closest[i] = dist;
+        }
+    }
+    free(pick); free(cand); free(closest); free(perm);
+
+    /* 3.-5. minibatch steps */
+    double *count = (double *)calloc((size_t)k, sizeof(double));
+    int32_t *idx = (int32_t *)malloc(sizeof(int32_t) * (size_t)batch);
+    int32_t *label = (int32_t *)malloc(sizeof(int32_t) * (size_t)batch);
+    int32_t *slots = (int32_t *)malloc(sizeof(int32_t) * (size_t)batch);
+    double *sum = (double *)malloc(sizeof(double) * (size_t)d);
+    int64_t t_max = (int64_t)max_iter * ((N + batch - 1) / batch);
+    double alpha = 2.0 * (double)batch / ((double)N + 1.0);
+    if (alpha > 1.0) alpha = 1.0;
+    double ewa = 0.0, ewa_min = INFINITY;
+    int32_t bad = 0, steps = 0;
+    for (int64_t t = 0; t < t_max; ++t) {
+        double inertia = 0.0;
+        for (int32_t s = 0; s < batch; ++s) {
+            idx[s] = km_index(km_word(seed, (uint32_t)s, 3u, stream, (uint32_t)t), N);
+            double bestd = INFINITY; int32_t arg = 0;
+            for (int32_t u = 0; u < k; ++u) {
+                double dist = sqdist(keys + (int64_t)idx[s] * d, centres + (int64_t)u * d, d);
+                if (dist < bestd) { bestd = dist; arg = u; }
+            }
+            label[s] = arg;
+            inertia += bestd;
+        }
+        /* cumulative-count update */
+        for (int32_t u = 0; u < k; ++u) {
+            int32_t n = 0;
+            for (int j = 0; j < d; ++j) sum[j] = 0.0;
+            for (int32_t s = 0; s < batch; ++s) {
+                if (label[s] != u) continue;
+                ++n;
+                for (int j = 0; j < d; ++j) sum[j] += keys[(int64_t)idx[s] * d + j];
+            }
+            if (n == 0) continue;
+            double grown = count[u] + (double)n;
+            for (int j = 0; j < d; ++j)
+                centres[(int64_t)u * d + j] = (centres[(int64_t)u * d + j] * count[u] + sum[j]) / grown;
+            count[u] = grown;
+        }
+        /* reassignment of starved centres */
+        {
+            double cmin = INFINITY, cmax = 0.0;
+            for (int32_t u = 0; u < k; ++u) { if (count[u] < cmin) cmin = count[u]; if (count[u] > cmax) cmax = count[u]; }
+            int64_t period = 10 + (int64_t)floor(cmin);
+            if (ratio > 0.0 && (t + 1) % period == 0) {
+                double thr = ratio * cmax;
+                int32_t n_move = 0, cap = batch / 2;
+                double keep_min = INFINITY;
+                for (int32_t u = 0; u < k; ++u) {
+                    if (count[u] < thr && n_move < cap) ++n_move;
+                    else if (count[u] < keep_min) keep_min = count[u];
+                }
+                if (n_move > 0) {
+                    for (int32_t s = 0; s < batch; ++s) slots[s] = s;
+                    for (int32_t i = 0; i < n_move; ++i) {
+                        int32_t r = i + km_index(km_word(seed, (uint32_t)i, 4u, stream, (uint32_t)t), batch - i);
+                        int32_t tmp = slots[i]; slots[i] = slots[r]; slots[r] = tmp;
+                    }
+                    int32_t moved = 0;
+                    for (int32_t u = 0; u < k && moved < n_move; ++u) {
+                        if (!(count[u] < thr)) continue;
+                        memcpy(centres + (int64_t)u * d, keys + (int64_t)idx[slots[moved]] * d, sizeof(double) * (size_t)d);
+                        count[u] = keep_min;
+                        ++moved;
+                    }
+                }
+            }
+        }
+        /* stopping rule */
+        ++steps;
+        double per_point = inertia / (double)batch;
+        ewa = t == 0 ? per_point : ewa * (1.0 - alpha) + per_point * alpha;
+        if (ewa < ewa_min) { ewa_min = ewa; bad = 0; }
+        else if (++bad >= patience) break;
+    }
+    free(sum); free(slots); free(label); free(idx); free(count);
+    return steps;
 }

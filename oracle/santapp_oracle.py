@@ -87,6 +87,9 @@ def lib():
         L.orc_group_mean_keys.restype = _c.c_int32
         L.orc_group_mean_keys_parents.argtypes = [_c.c_int, _f64p, _c.c_int32, _i32p, _i32p, _f64p]
         L.orc_group_mean_keys_parents.restype = None
+        L.orc_minibatch_kmeans.argtypes = [_c.c_int32, _c.c_int, _f64p, _c.c_int32, _c.c_int32, _c.c_int32, _c.c_int32,
+                                           _c.c_double, _c.c_uint64, _c.c_uint32, _f64p]
+        L.orc_minibatch_kmeans.restype = _c.c_int32
         L.orc_kmeans_parent_count.argtypes = [_c.c_int32, _c.c_int32]
         L.orc_kmeans_parent_count.restype = _c.c_int32
         L.orc_nearest_centre_parents.argtypes = [_c.c_int32, _c.c_int, _f64p, _c.c_int32, _f64p, _i32p, _i32p, _i32p]
@@ -360,3 +363,12 @@ def group_mean_keys_parents(keys, parent_start, parent_member):
     mean = np.zeros((n, keys.shape[1]))
     lib().orc_group_mean_keys_parents(keys.shape[1], keys, n, parent_start, parent_member, mean)
     return parent_start.copy(), parent_member.copy(), mean
+
+
+def minibatch_kmeans(keys, k, batch=4096, max_iter=100, patience=10, ratio=0.01, seed=0, stream=0):
+    """The fit of Algorithm 3 with the paper's settings as defaults. Returns (centres[k, d] fp64, steps)."""
+    keys = _f64(keys)
+    N, d = keys.shape
+    centres = np.zeros((k, d))
+    steps = lib().orc_minibatch_kmeans(N, d, keys, k, batch, max_iter, patience, ratio, seed, stream, centres)
+    return centres, int(steps)
