@@ -207,10 +207,59 @@ int santapp_build_groups_mean(const santapp_geom *geom, const int32_t *prompt_le
 int32_t santapp_kmeans_parent_count(int32_t prompt_len, int32_t parent_size);
 
 /*
+ * Algorithm 3, the fit: minibatch k-means on the raw keys of each (sequence, KV head), squared
+ * Euclidean distance, fp64 arithmetic. The paper fixes the routine's settings (the defaults named
+ * below) and leaves its details to a library; this is the routine as built here:
+ *   1. Initialisation sample: min(N, max(3 * batch, 3 * k)) distinct keys, the head of a
+ *      Fisher-Yates shuffle of the token indices.
+ *   2. Greedy k-means++ on the sample with 2 + floor(ln k) trials per centre: the first centre is
+ *      a uniform sample point; each later one is the best of the trial points drawn with
+ *      probability proportional to the squared distance to the nearest centre so far, best meaning
+ *      the smallest resulting sum of nearest-centre distances over the sample.
+ *   3. At most max_iter * ceil(N / batch) steps; a step draws `batch` token indices uniformly with
+ *      replacement, assigns each to its nearest centre (ties to the smaller index) and moves every
+ *      centre that received points to the mean of all points it has received so far
+ *      (cumulative count).
+ *   4. At steps t with (t + 1) divisible by 10 + floor(smallest count), centres whose count is
+ *      below reassignment_ratio * (largest count), at most batch / 2 of them, jump onto distinct
+ *      points of the current minibatch and take the smallest count among the centres that stay.
+ *   5. The per-point inertia of each minibatch feeds an exponentially weighted average with
+ *      weight min(1, 2 * batch / (N + 1)); the fit stops after `patience` consecutive steps
+ *      without a new minimum of that average. There is no centre-change criterion (tolerance 0).
+ * Random choices are words of the library's Philox stream (top of this file) with counter
+ * (slot, purpose, stream, step), key = seed, stream = stream_base + b * n_kv_heads + j for
+ * sequence b and KV head j: a fit is a pure function of its arguments.
+ *   n_centres_host   host int32 [n_seqs], in: k of sequence b, 1 <= k <= prompt_len[b]
+ *                    (santapp_kmeans_parent_count gives the paper's choice)
+ *   k_prompt         device [n_kv_heads][rows_total][d], token order, in
+ *   centres          device fp32 [n_kv_heads][sum_b k_b][d], out (the fp64 centres rounded to nearest);
+ *                    the layout santapp_assign_parents takes
+ *   steps_run        device int32 [n_kv_heads][n_seqs] or NULL, out: minibatch steps each fit ran
+ *   workspace        device, >= santapp_kmeans_fit_workspace_bytes(...)
+ * batch_size > 4096: SANTAPP_ERR_UNSUPPORTED. The call enqueues a few kernels per centre and per
+ * step on `stream`; it does not synchronise.
+ */
+typedef struct santapp_kmeans_opts {
+    int32_t batch_size;           /* paper: 4096 */
+    int32_t max_iter;             /* paper: 100 */
+    int32_t patience;             /* paper: 10 */
+    int32_t reserved;             /* set to 0 */
+    double reassignment_ratio;    /* paper: 0.01; 0 switches reassignment off */
+    uint64_t seed;                /* paper: 0 */
+    uint32_t stream_base;
+    uint32_t reserved2;           /* set to 0 */
+} santapp_kmeans_opts;
+size_t santapp_kmeans_fit_workspace_bytes(const santapp_geom *geom, const int32_t *prompt_len_host,
+                                          const int32_t *n_centres_host, const santapp_kmeans_opts *opts);
+int santapp_kmeans_fit(const santapp_geom *geom, const int32_t *prompt_len_host,
+                       const int32_t *n_centres_host, const void *k_prompt,
+                       const santapp_kmeans_opts *opts, float *centres, int32_t *steps_run,
+                       void *workspace, size_t workspace_bytes, santapp_stream stream);
+
+/*
  * Algorithm 3, the assignment that follows the fit: every key joins its nearest centre, squared
  * Euclidean distance evaluated in fp64 on the raw keys, ties going to the smaller centre index.
- * The centres are an input: fitting them (minibatch k-means with the paper's settings) is left to
- * the caller's clustering routine.
+ * The centres are an input: santapp_kmeans_fit's output, or any other clustering's.
  *   n_centres_host   host int32 [n_seqs], in: centres of sequence b (>= 1), the same for every KV head
  *   k_prompt         device bf16 [n_kv_heads][rows_total][d], token order, in
  *   centres          device fp32 [n_kv_heads][sum_b n_centres[b]][d], in: sequence b's centres

@@ -33,6 +33,7 @@ EXPORTS = [
     "santapp_set_stage_mask", "santapp_dense_decode_attn_noalloc", "santapp_build_groups_mean",
     "santapp_kmeans_parent_count", "santapp_assign_parents_workspace_bytes", "santapp_assign_parents",
     "santapp_parent_teams_sizes", "santapp_build_teams_parents", "santapp_build_groups_mean_parents",
+    "santapp_kmeans_fit_workspace_bytes", "santapp_kmeans_fit",
 ]
 
 STAGE_ROUTE, STAGE_SELECT, STAGE_ATTEND, STAGE_ALL = 1, 2, 4, 7
@@ -63,6 +64,12 @@ class CTeams(ctypes.Structure):
                 ("rep_abs_max", ctypes.c_void_p), ("team_count", ctypes.c_void_p),
                 ("rows_total", ctypes.c_int64), ("teams_total", ctypes.c_int64),
                 ("max_teams_per_seq", ctypes.c_int32), ("max_rows_per_seq", ctypes.c_int32)]
+
+
+class CKmeansOpts(ctypes.Structure):
+    _fields_ = [("batch_size", ctypes.c_int32), ("max_iter", ctypes.c_int32), ("patience", ctypes.c_int32),
+                ("reserved", ctypes.c_int32), ("reassignment_ratio", ctypes.c_double), ("seed", ctypes.c_uint64),
+                ("stream_base", ctypes.c_uint32), ("reserved2", ctypes.c_uint32)]
 
 
 class CDebug(ctypes.Structure):
@@ -97,6 +104,12 @@ def load_library(path: Optional[str] = None):
     L.santapp_build_teams.restype = ctypes.c_int
     L.santapp_build_groups_mean.argtypes = L.santapp_build_teams.argtypes
     L.santapp_build_groups_mean.restype = ctypes.c_int
+    L.santapp_kmeans_fit_workspace_bytes.argtypes = [ctypes.POINTER(CGeom), ctypes.POINTER(i32), ctypes.POINTER(i32),
+                                                     ctypes.POINTER(CKmeansOpts)]
+    L.santapp_kmeans_fit_workspace_bytes.restype = sz
+    L.santapp_kmeans_fit.argtypes = [ctypes.POINTER(CGeom), ctypes.POINTER(i32), ctypes.POINTER(i32), vp,
+                                     ctypes.POINTER(CKmeansOpts), vp, vp, vp, sz, vp]
+    L.santapp_kmeans_fit.restype = ctypes.c_int
     L.santapp_kmeans_parent_count.argtypes = [i32, i32]
     L.santapp_kmeans_parent_count.restype = i32
     L.santapp_assign_parents_workspace_bytes.argtypes = [ctypes.POINTER(CGeom)]
@@ -259,6 +272,28 @@ def _i32_array(values):
 def santapp_kmeans_parent_count(prompt_len: int, parent_size: int) -> int:
     """First line of Algorithm 3: min(N, max(2, N // P)); 0 for N < 2 or P < 1."""
     return int(load_library().santapp_kmeans_parent_count(int(prompt_len), int(parent_size)))
+
+
+def santapp_kmeans_fit(geom: Geometry, prompt_len, n_centres, k_prompt: torch.Tensor, batch_size: int = 4096,
+                       max_iter: int = 100, patience: int = 10, reassignment_ratio: float = 0.01, seed: int = 0,
+                       stream_base: int = 0, stream=None):
+    """Minibatch k-means fit per (sequence, KV head); the defaults are the paper's settings.
+    Returns (centres fp32 [n_kv_heads, sum(n_centres), d], steps int32 [n_kv_heads, n_seqs])."""
+    L = load_library()
+    g = geom.c()
+    o = CKmeansOpts(batch_size, max_iter, patience, 0, reassignment_ratio, seed, stream_base, 0)
+    n, c = _i32_array(prompt_len), _i32_array(n_centres)
+    need = int(L.santapp_kmeans_fit_workspace_bytes(ctypes.byref(g), n, c, ctypes.byref(o)))
+    if need == 0:
+        raise SantappError(SANTAPP_ERR_INVALID_ARG, "k-means fit arguments")
+    dev = k_prompt.device
+    ws = torch.empty(need, dtype=torch.uint8, device=dev)
+    centres = torch.empty((geom.n_kv_heads, int(sum(n_centres)), geom.head_dim), dtype=torch.float32, device=dev)
+    steps = torch.zeros((geom.n_kv_heads, geom.n_seqs), dtype=torch.int32, device=dev)
+    _check(L.santapp_kmeans_fit(ctypes.byref(g), n, c, _ptr(k_prompt), ctypes.byref(o), _ptr(centres), _ptr(steps),
+                                _ptr(ws), ws.numel(), _stream_ptr(stream)))
+    centres._ws = ws
+    return centres, steps
 
 
 def santapp_assign_parents(geom: Geometry, prompt_len, n_centres, k_prompt: torch.Tensor, centres: torch.Tensor,

@@ -6,7 +6,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
-SOURCES = ["api.cu", "build_teams.cu", "build_parents.cu", "score.cu", "headplan.cu", "plan.cu", "attend.cu"]
+SOURCES = ["api.cu", "build_teams.cu", "build_parents.cu", "kmeans.cu", "score.cu", "headplan.cu", "plan.cu", "attend.cu"]
 HEADERS = [os.path.join(CSRC, "common.cuh"), os.path.join(CSRC, "pairplan.cuh"), os.path.join(CSRC, "build_util.cuh"), os.path.join(ROOT, "include", "santapp.h")]
 OUT = os.path.join(HERE, "libsantapp.so")
 

@@ -484,6 +484,152 @@ int santapp_build_groups_mean_parents(const santapp_geom *geom, const int32_t *p
 
 }  // extern "C"
 
+namespace {
+
+struct KmeansLayout {
+    size_t row_off, cen_off, tabs, perm, closest, cand, pick, centres64, count, idx, label, dist, state, total;
+    int k_max, n_init_max, trials_max, t_max_max, max_rows;
+    int64_t rows_total, centres_total;
+};
+
+// Per-sequence quantities of the fit and the workspace that holds its state. Returns a status.
+int kmeans_layout(const santapp_geom *geom, const int32_t *prompt_len_host, const int32_t *n_centres_host,
+                  const santapp_kmeans_opts *o, KmeansLayout *L, std::vector<int32_t> *tabs)
+{
+    int rc = check_geom(geom);
+    if (rc != SANTAPP_OK) return rc;
+    if (!prompt_len_host || !n_centres_host || !o) return SANTAPP_ERR_INVALID_ARG;
+    if (o->batch_size < 1 || o->max_iter < 1 || o->patience < 1 || !(o->reassignment_ratio >= 0.0))
+        return SANTAPP_ERR_INVALID_ARG;
+    if (o->batch_size > 4096) return SANTAPP_ERR_UNSUPPORTED;
+    const int B = geom->n_seqs;
+    memset(L, 0, sizeof(*L));
+    if (tabs) tabs->assign(3 * (size_t)B, 0);
+    for (int b = 0; b < B; ++b) {
+        const int N = prompt_len_host[b], k = n_centres_host[b];
+        if (N < 1 || k < 1 || k > N) return SANTAPP_ERR_INVALID_ARG;
+        int64_t n_init = 3 * (int64_t)(o->batch_size > k ? o->batch_size : k);
+        if (n_init > N) n_init = N;
+        const int trials = 2 + (int)floor(log((double)k));
+        const int64_t t_max = (int64_t)o->max_iter * ((N + o->batch_size - 1) / o->batch_size);
+        if (t_max > INT32_MAX) return SANTAPP_ERR_UNSUPPORTED;
+        if (tabs) { (*tabs)[b] = (int32_t)n_init; (*tabs)[B + b] = trials; (*tabs)[2 * B + b] = (int32_t)t_max; }
+        L->rows_total += N;
+        L->centres_total += k;
+        if (k > L->k_max) L->k_max = k;
+        if (n_init > L->n_init_max) L->n_init_max = (int)n_init;
+        if (trials > L->trials_max) L->trials_max = trials;
+        if (t_max > L->t_max_max) L->t_max_max = (int)t_max;
+        if (N > L->max_rows) L->max_rows = N;
+    }
+    if (L->rows_total >= (int64_t)1 << 31) return SANTAPP_ERR_UNSUPPORTED;
+    const size_t H = (size_t)geom->n_kv_heads, pairs = H * (size_t)B;
+    if (pairs > 65535) return SANTAPP_ERR_UNSUPPORTED;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t at = off; off = align_up(off + bytes); return at; };
+    L->row_off = take(sizeof(int64_t) * ((size_t)B + 1));
+    L->cen_off = take(sizeof(int64_t) * ((size_t)B + 1));
+    L->tabs = take(sizeof(int32_t) * 3 * (size_t)B);
+    L->perm = take(sizeof(int32_t) * H * (size_t)L->rows_total);
+    L->closest = take(sizeof(double) * pairs * (size_t)L->n_init_max);
+    L->cand = take(sizeof(double) * pairs * (size_t)L->trials_max * (size_t)L->n_init_max);
+    L->pick = take(sizeof(int32_t) * pairs * (size_t)L->trials_max);
+    L->centres64 = take(sizeof(double) * H * (size_t)L->centres_total * kHeadDim);
+    L->count = take(sizeof(double) * H * (size_t)L->centres_total);
+    L->idx = take(sizeof(int32_t) * pairs * (size_t)o->batch_size);
+    L->label = take(sizeof(int32_t) * pairs * (size_t)o->batch_size);
+    L->dist = take(sizeof(double) * pairs * (size_t)o->batch_size);
+    L->state = take(sizeof(KmeansState) * pairs);
+    L->total = off;
+    return SANTAPP_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t santapp_kmeans_fit_workspace_bytes(const santapp_geom *geom, const int32_t *prompt_len_host,
+                                          const int32_t *n_centres_host, const santapp_kmeans_opts *opts)
+{
+    KmeansLayout L;
+    if (kmeans_layout(geom, prompt_len_host, n_centres_host, opts, &L, nullptr) != SANTAPP_OK) return 0;
+    return L.total;
+}
+
+int santapp_kmeans_fit(const santapp_geom *geom, const int32_t *prompt_len_host, const int32_t *n_centres_host,
+                       const void *k_prompt, const santapp_kmeans_opts *opts, float *centres, int32_t *steps_run,
+                       void *workspace, size_t workspace_bytes, santapp_stream stream)
+{
+    KmeansLayout L;
+    std::vector<int32_t> tabs;
+    int rc = kmeans_layout(geom, prompt_len_host, n_centres_host, opts, &L, &tabs);
+    if (rc != SANTAPP_OK) return rc;
+    if (!k_prompt || !centres || !workspace) return SANTAPP_ERR_INVALID_ARG;
+    if (misaligned(k_prompt, 16) || misaligned(centres, 4) || misaligned(steps_run, 4) || misaligned(workspace, 16))
+        return SANTAPP_ERR_INVALID_ARG;
+    if (workspace_bytes < L.total) return SANTAPP_ERR_WORKSPACE_TOO_SMALL;
+    const int B = geom->n_seqs;
+    std::vector<int64_t> offs(2 * ((size_t)B + 1));
+    int64_t *row_off = offs.data(), *cen_off = row_off + B + 1;
+    row_off[0] = cen_off[0] = 0;
+    for (int b = 0; b < B; ++b) {
+        row_off[b + 1] = row_off[b] + prompt_len_host[b];
+        cen_off[b + 1] = cen_off[b] + n_centres_host[b];
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    g_cuda_error[0] = 0;
+    unsigned char *ws = static_cast<unsigned char *>(workspace);
+    const size_t ob = sizeof(int64_t) * ((size_t)B + 1);
+    cudaError_t err = cudaMemcpyAsync(ws + L.row_off, row_off, ob, cudaMemcpyHostToDevice, s);
+    if (err != cudaSuccess) return cuda_fail(err, "copy row offsets");
+    err = cudaMemcpyAsync(ws + L.cen_off, cen_off, ob, cudaMemcpyHostToDevice, s);
+    if (err != cudaSuccess) return cuda_fail(err, "copy centre offsets");
+    err = cudaMemcpyAsync(ws + L.tabs, tabs.data(), sizeof(int32_t) * tabs.size(), cudaMemcpyHostToDevice, s);
+    if (err != cudaSuccess) return cuda_fail(err, "copy fit tables");
+
+    KmeansParams p;
+    p.n_seqs = B;
+    p.n_kv = geom->n_kv_heads;
+    p.elem = geom->elem_type;
+    p.max_rows_per_seq = L.max_rows;
+    p.batch = opts->batch_size;
+    p.patience = opts->patience;
+    p.ratio = opts->reassignment_ratio;
+    p.seed_lo = (uint32_t)(opts->seed & 0xFFFFFFFFull);
+    p.seed_hi = (uint32_t)(opts->seed >> 32);
+    p.stream_base = opts->stream_base;
+    p.k_max = L.k_max;
+    p.n_init_max = L.n_init_max;
+    p.trials_max = L.trials_max;
+    p.t_max_max = L.t_max_max;
+    p.rows_total = L.rows_total;
+    p.centres_total = L.centres_total;
+    p.seq_row_off = reinterpret_cast<const int64_t *>(ws + L.row_off);
+    p.seq_centre_off = reinterpret_cast<const int64_t *>(ws + L.cen_off);
+    const int32_t *t = reinterpret_cast<const int32_t *>(ws + L.tabs);
+    p.seq_n_init = t;
+    p.seq_trials = t + B;
+    p.seq_t_max = t + 2 * B;
+    p.k_prompt = static_cast<const uint16_t *>(k_prompt);
+    p.centres_out = centres;
+    p.steps_out = steps_run;
+    p.perm = reinterpret_cast<int32_t *>(ws + L.perm);
+    p.closest = reinterpret_cast<double *>(ws + L.closest);
+    p.cand = reinterpret_cast<double *>(ws + L.cand);
+    p.pick = reinterpret_cast<int32_t *>(ws + L.pick);
+    p.centres64 = reinterpret_cast<double *>(ws + L.centres64);
+    p.count = reinterpret_cast<double *>(ws + L.count);
+    p.idx = reinterpret_cast<int32_t *>(ws + L.idx);
+    p.label = reinterpret_cast<int32_t *>(ws + L.label);
+    p.dist = reinterpret_cast<double *>(ws + L.dist);
+    p.state = reinterpret_cast<KmeansState *>(ws + L.state);
+    err = launch_kmeans_fit(p, s);
+    if (err != cudaSuccess) return cuda_fail(err, "kmeans_fit launch");
+    return SANTAPP_OK;
+}
+
+}  // extern "C"
+
 extern "C" {
 
 int santapp_build_teams(const santapp_geom *geom, const int32_t *prompt_len_host, const void *k_prompt,

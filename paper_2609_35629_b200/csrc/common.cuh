@@ -210,6 +210,36 @@ struct ParentBuildParams {
 };
 cudaError_t launch_build_teams_parents(const ParentBuildParams &p, cudaStream_t s);
 
+// Minibatch k-means fit (second line of Algorithm 3), one problem per (sequence, KV head).
+struct KmeansState {
+    double ewa, ewa_min;                    // averaged per-point inertia and its minimum so far
+    int bad, steps, stopped, pad;
+};
+struct KmeansParams {
+    int n_seqs, n_kv, elem, max_rows_per_seq;
+    int batch, patience;
+    double ratio;
+    uint32_t seed_lo, seed_hi, stream_base;
+    int k_max, n_init_max, trials_max, t_max_max;   // maxima over the sequences
+    int64_t rows_total, centres_total;
+    const int64_t *seq_row_off, *seq_centre_off;    // device [n_seqs + 1]
+    const int32_t *seq_n_init, *seq_trials, *seq_t_max;   // device [n_seqs]
+    const uint16_t *k_prompt;               // [n_kv][rows_total][128]
+    float *centres_out;                     // [n_kv][centres_total][128]
+    int32_t *steps_out;                     // [n_kv][n_seqs] or null
+    // workspace; "pairs" arrays are indexed by j * n_seqs + b
+    int32_t *perm;                          // [n_kv][rows_total]
+    double *closest;                        // [pairs][n_init_max]
+    double *cand;                           // [pairs][trials_max][n_init_max]
+    int32_t *pick;                          // [pairs][trials_max]
+    double *centres64;                      // [n_kv][centres_total][128]
+    double *count;                          // [n_kv][centres_total]
+    int32_t *idx, *label;                   // [pairs][batch]
+    double *dist;                           // [pairs][batch]
+    KmeansState *state;                     // [pairs]
+};
+cudaError_t launch_kmeans_fit(const KmeansParams &p, cudaStream_t s);
+
 // ---------------------------------------------------------------------------------------------
 // Device helpers
 // ---------------------------------------------------------------------------------------------

@@ -1,0 +1,419 @@
+// santapp_kmeans_fit: the fit of Algorithm 3 (global minibatch k-means parents), one independent
+// problem per (sequence, KV head). Preparation path, run once after prefill.
+//
+// The paper names the routine and its settings and leaves the rest to its library; the reading
+// taken here is written out in include/santapp.h. Every random choice is a Philox word with
+// counter (slot, tag, stream, step), and every comparison is made on fp64 values obtained by the
+// same operations in the same order wherever the order matters (sums over dimensions, over the
+// sample, over a minibatch; separately rounded multiply and add), so a fit is a pure function
+// of its arguments. Sums whose order matters run on one thread; the distance evaluations around
+// them are spread over the grid.
+#include <limits.h>
+#include <math.h>
+
+#include "common.cuh"
+
+namespace santapp {
+
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kTile = 16;                 // centres staged per shared-memory tile
+constexpr uint32_t kTagSample = 1u, kTagStart = 2u, kTagBatch = 3u, kTagMove = 4u;
+
+struct Pair {
+    int b, j, N, k, n_init, L, t_max;
+    uint32_t stream;
+    int64_t row0, c0;
+    size_t plane;                         // first row of the pair in a [n_kv][rows_total] array
+    size_t cplane;                        // first centre of the pair in a [n_kv][centres_total] array
+    int id;                               // j-major pair index into the per-pair scratch arrays
+};
+
+__device__ __forceinline__ Pair pair_of(const KmeansParams &p, int b, int j)
+{
+    Pair q;
+    q.b = b;
+    q.j = j;
+    q.row0 = p.seq_row_off[b];
+    q.N = (int)(p.seq_row_off[b + 1] - q.row0);
+    q.c0 = p.seq_centre_off[b];
+    q.k = (int)(p.seq_centre_off[b + 1] - q.c0);
+    q.n_init = p.seq_n_init[b];
+    q.L = p.seq_trials[b];
+    q.t_max = p.seq_t_max[b];
+    q.stream = p.stream_base + (uint32_t)(b * p.n_kv + j);
+    q.plane = (size_t)j * p.rows_total + (size_t)q.row0;
+    q.cplane = (size_t)j * p.centres_total + (size_t)q.c0;
+    q.id = j * p.n_seqs + b;
+    return q;
+}
+
+__device__ __forceinline__ uint32_t km_word(const KmeansParams &p, uint32_t slot, uint32_t tag, uint32_t stream, uint32_t step)
+{
+    return philox4x32_10(make_uint4(slot, tag, stream, step), p.seed_lo, p.seed_hi).x;
+}
+__device__ __forceinline__ int km_index(uint32_t word, int n) { return (int)(((unsigned long long)word * (unsigned long long)n) >> 32); }
+
+template <bool kHalf>
+__device__ __forceinline__ double sqdist_rows(const uint4 *a, const uint4 *b)
+{
+    double s = 0.0;
+#pragma unroll 4
+    for (int q = 0; q < 16; ++q) {
+        const uint4 x4 = a[q], y4 = b[q];
+        const uint32_t x[4] = {x4.x, x4.y, x4.z, x4.w}, y[4] = {y4.x, y4.y, y4.z, y4.w};
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+            const double e0 = __dsub_rn((double)elem_lo<kHalf>(x[t]), (double)elem_lo<kHalf>(y[t]));
+            const double e1 = __dsub_rn((double)elem_hi<kHalf>(x[t]), (double)elem_hi<kHalf>(y[t]));
+            s = __dadd_rn(s, __dmul_rn(e0, e0));
+            s = __dadd_rn(s, __dmul_rn(e1, e1));
+        }
+    }
+    return s;
+}
+
+// ---- 1. initialisation sample: head of a Fisher-Yates shuffle ----
+__global__ void __launch_bounds__(kThreads)
+km_perm_identity_kernel(KmeansParams p)
+{
+    const Pair q = pair_of(p, blockIdx.y, blockIdx.z);
+    const int i = blockIdx.x * kThreads + threadIdx.x;
+    if (i < q.N) p.perm[q.plane + i] = i;
+}
+
+__global__ void __launch_bounds__(32)
+km_sample_kernel(KmeansParams p)
+{
+    const Pair q = pair_of(p, blockIdx.x, blockIdx.y);
+    const int lane = threadIdx.x;
+    int32_t *perm = p.perm + q.plane;
+    // the words of 32 positions at a time, the swaps in order on one lane
+    for (int i0 = 0; i0 < q.n_init; i0 += 32) {
+        const int i = i0 + lane;
+        const uint32_t w = i < q.n_init ? km_word(p, (uint32_t)i, kTagSample, q.stream, 0u) : 0u;
+        for (int l = 0; l < 32 && i0 + l < q.n_init; ++l) {
+            const uint32_t wl = __shfl_sync(0xFFFFFFFFu, w, l);
+            if (lane == 0) {
+                const int at = i0 + l;
+                const int r = at + km_index(wl, q.N - at);
+                const int32_t t = perm[at];
+                perm[at] = perm[r];
+                perm[r] = t;
+            }
+        }
+    }
+    if (lane == 0) p.pick[(size_t)q.id * p.trials_max] = km_index(km_word(p, 0u, kTagStart, q.stream, 0u), q.n_init);
+}
+
+// ---- 2. greedy k-means++ on the sample ----
+// Distances of every sample point to the candidate points pick[0..n_cand): cand[l][i].
+template <bool kHalf>
+__global__ void __launch_bounds__(kThreads)
+km_candidate_dist_kernel(KmeansParams p, int c)
+{
+    const Pair q = pair_of(p, blockIdx.z / p.n_kv, blockIdx.z % p.n_kv);
+    const int l = blockIdx.y;
+    if (c >= q.k || l >= (c == 0 ? 1 : q.L)) return;
+    const int i = blockIdx.x * kThreads + threadIdx.x;
+    if (i >= q.n_init) return;
+    const int32_t *perm = p.perm + q.plane;
+    const uint4 *keys = reinterpret_cast<const uint4 *>(p.k_prompt + q.plane * kHeadDim);
+    const int at = p.pick[(size_t)q.id * p.trials_max + l];
+    p.cand[((size_t)q.id * p.trials_max + l) * p.n_init_max + i] =
+        sqdist_rows<kHalf>(keys + (size_t)perm[i] * 16, keys + (size_t)perm[at] * 16);
+}
+
+// One block per pair: potentials of the trials (one lane each, sums in sample order), the best
+// trial becomes centre c, the nearest-centre distances are lowered.
+template <bool kHalf>
+__global__ void __launch_bounds__(kThreads)
+km_accept_kernel(KmeansParams p, int c)
+{
+    __shared__ int best_s;
+    const Pair q = pair_of(p, blockIdx.x, blockIdx.y);
+    if (c >= q.k) return;
+    const int tid = threadIdx.x;
+    const int n_trials = c == 0 ? 1 : q.L;
+    double *closest = p.closest + (size_t)q.id * p.n_init_max;
+    const double *cand = p.cand + (size_t)q.id * p.trials_max * p.n_init_max;
+    if (tid < 32) {
+        double pot = INFINITY;
+        if (c > 0 && tid < n_trials) {
+            const double *mine = cand + (size_t)tid * p.n_init_max;
+            pot = 0.0;
+#pragma unroll 4
+            for (int i = 0; i < q.n_init; ++i) {
+                const double d = mine[i], o = closest[i];
+                pot = __dadd_rn(pot, d < o ? d : o);
+            }
+        }
+        int best = 0;
+        double best_pot = __shfl_sync(0xFFFFFFFFu, pot, 0);
+        for (int l = 1; l < n_trials; ++l) {
+            const double v = __shfl_sync(0xFFFFFFFFu, pot, l);
+            if (v < best_pot) { best_pot = v; best = l; }
+        }
+        if (tid == 0) best_s = best;
+    }
+    __syncthreads();
+    const int best = best_s;
+    const double *win = cand + (size_t)best * p.n_init_max;
+    for (int i = tid; i < q.n_init; i += kThreads) {
+        const double d = win[i];
+        if (c == 0 || d < closest[i]) closest[i] = d;
+    }
+    if (tid < kHeadDim) {
+        const int32_t *perm = p.perm + q.plane;
+        const int at = p.pick[(size_t)q.id * p.trials_max + best];
+        const uint16_t v = p.k_prompt[(q.plane + (size_t)perm[at]) * kHeadDim + tid];
+        p.centres64[(q.cplane + (size_t)c) * kHeadDim + tid] = elem_to_double<kHalf>(v);
+    }
+}
+
+// One warp per pair: the L trial points of centre c, drawn with probability proportional to the
+// distance to the nearest chosen centre (inverse CDF over the sample in order; every lane runs the
+// same running sum and watches for its own target).
+__global__ void __launch_bounds__(32)
+km_draw_trials_kernel(KmeansParams p, int c)
+{
+    const Pair q = pair_of(p, blockIdx.x, blockIdx.y);
+    if (c >= q.k) return;
+    const int lane = threadIdx.x;
+    const double *closest = p.closest + (size_t)q.id * p.n_init_max;
+    double total = 0.0;
+#pragma unroll 8
+    for (int i = 0; i < q.n_init; ++i) total = __dadd_rn(total, closest[i]);
+    const uint32_t w = km_word(p, (uint32_t)lane, kTagStart, q.stream, (uint32_t)c);
+    const double target = __dmul_rn(((double)w + 0.5) * (1.0 / 4294967296.0), total);
+    double cum = 0.0;
+    int at = q.n_init - 1;
+    bool found = false;
+#pragma unroll 8
+    for (int i = 0; i < q.n_init; ++i) {
+        cum = __dadd_rn(cum, closest[i]);
+        if (!found && cum > target) { at = i; found = true; }
+    }
+    if (lane < q.L) p.pick[(size_t)q.id * p.trials_max + lane] = at;
+}
+
+// ---- 3. minibatch steps ----
+__device__ __forceinline__ bool pair_active(const KmeansParams &p, const Pair &q, int t)
+{
+    return t < q.t_max && !p.state[q.id].stopped;
+}
+
+// Draw the minibatch and assign each point to its nearest centre (ties to the smaller index).
+template <bool kHalf>
+__global__ void __launch_bounds__(128)
+km_batch_assign_kernel(KmeansParams p, int t)
+{
+    __shared__ double c[kTile][kHeadDim];
+    const Pair q = pair_of(p, blockIdx.y / p.n_kv, blockIdx.y % p.n_kv);
+    if (!pair_active(p, q, t)) return;
+    const int tid = threadIdx.x;
+    const int s = blockIdx.x * 128 + tid;
+    const bool valid = s < p.batch;
+    const int idx = km_index(km_word(p, (uint32_t)(valid ? s : 0), kTagBatch, q.stream, (uint32_t)t), q.N);
+    uint32_t kw[64];
+    {
+        const uint4 *row = reinterpret_cast<const uint4 *>(p.k_prompt + (q.plane + (size_t)idx) * kHeadDim);
+#pragma unroll
+        for (int v = 0; v < 16; ++v) {
+            const uint4 w = row[v];
+            kw[4 * v] = w.x; kw[4 * v + 1] = w.y; kw[4 * v + 2] = w.z; kw[4 * v + 3] = w.w;
+        }
+    }
+    double best = INFINITY;
+    int arg = 0;
+    const double *cen = p.centres64 + q.cplane * kHeadDim;
+    for (int base = 0; base < q.k; base += kTile) {
+        const int nt = min(kTile, q.k - base);
+        __syncthreads();
+        for (int e = tid; e < nt * kHeadDim; e += 128) c[e >> 7][e & 127] = cen[(size_t)base * kHeadDim + e];
+        __syncthreads();
+        for (int u = 0; u < nt; ++u) {
+            double d = 0.0;
+#pragma unroll
+            for (int w = 0; w < 64; ++w) {
+                const double e0 = __dsub_rn((double)elem_lo<kHalf>(kw[w]), c[u][2 * w]);
+                const double e1 = __dsub_rn((double)elem_hi<kHalf>(kw[w]), c[u][2 * w + 1]);
+                d = __dadd_rn(d, __dmul_rn(e0, e0));
+                d = __dadd_rn(d, __dmul_rn(e1, e1));
+            }
+            if (d < best) { best = d; arg = base + u; }
+        }
+    }
+    if (valid) {
+        const size_t at = (size_t)q.id * p.batch + s;
+        p.idx[at] = idx;
+        p.label[at] = arg;
+        p.dist[at] = best;
+    }
+}
+
+// Cumulative-count update: thread (centre, dimension) adds the centre's new points in minibatch
+// order; c <- (c * count + sum) / (count + n).
+template <bool kHalf>
+__global__ void __launch_bounds__(kThreads)
+km_batch_update_kernel(KmeansParams p, int t)
+{
+    extern __shared__ int32_t batch_tab[];                  // labels, then indices
+    const Pair q = pair_of(p, blockIdx.y / p.n_kv, blockIdx.y % p.n_kv);
+    if (!pair_active(p, q, t)) return;
+    const int u0 = blockIdx.x * (kThreads / kHeadDim);
+    if (u0 >= q.k) return;
+    int32_t *lab = batch_tab, *idx = batch_tab + p.batch;
+    for (int s = threadIdx.x; s < p.batch; s += kThreads) {
+        lab[s] = p.label[(size_t)q.id * p.batch + s];
+        idx[s] = p.idx[(size_t)q.id * p.batch + s];
+    }
+    __syncthreads();
+    const int u = u0 + threadIdx.x / kHeadDim, d = threadIdx.x % kHeadDim;
+    const bool live = u < q.k;
+    double sum = 0.0, count = 0.0;
+    int n = 0;
+    if (live) {
+        count = p.count[q.cplane + u];
+        const uint16_t *col = p.k_prompt + q.plane * kHeadDim + d;
+        for (int s = 0; s < p.batch; ++s) {
+            if (lab[s] != u) continue;
+            ++n;
+            sum = __dadd_rn(sum, elem_to_double<kHalf>(col[(size_t)idx[s] * kHeadDim]));
+        }
+    }
+    __syncthreads();                                        // every thread has read its centre's count
+    if (live && n > 0) {
+        const double grown = __dadd_rn(count, (double)n);
+        double *cd = p.centres64 + (q.cplane + (size_t)u) * kHeadDim + d;
+        *cd = __ddiv_rn(__dadd_rn(__dmul_rn(*cd, count), sum), grown);
+        if (d == 0) p.count[q.cplane + u] = grown;
+    }
+}
+
+// One warp per pair: reassignment of starved centres, averaged inertia, stopping rule.
+template <bool kHalf>
+__global__ void __launch_bounds__(32)
+km_control_kernel(KmeansParams p, int t)
+{
+    extern __shared__ int32_t ctl_tab[];                    // slots[batch], move_centre[batch / 2]
+    __shared__ int n_move_s;
+    const Pair q = pair_of(p, blockIdx.x, blockIdx.y);
+    if (!pair_active(p, q, t)) return;
+    const int lane = threadIdx.x;
+    int32_t *slots = ctl_tab, *move_centre = ctl_tab + p.batch;
+    double *count = p.count + q.cplane;
+    const int32_t *idx = p.idx + (size_t)q.id * p.batch;
+    if (lane == 0) {
+        int n_move = 0;
+        double cmin = INFINITY, cmax = 0.0;
+        for (int u = 0; u < q.k; ++u) {
+            const double v = count[u];
+            if (v < cmin) cmin = v;
+            if (v > cmax) cmax = v;
+        }
+        const long long period = 10 + (long long)floor(cmin);
+        if (p.ratio > 0.0 && ((long long)t + 1) % period == 0) {
+            const double thr = __dmul_rn(p.ratio, cmax);
+            const int cap = p.batch / 2;
+            double keep_min = INFINITY;
+            for (int u = 0; u < q.k; ++u) {
+                const double v = count[u];
+                if (v < thr && n_move < cap) move_centre[n_move++] = u;
+                else if (v < keep_min) keep_min = v;
+            }
+            if (n_move > 0) {
+                for (int s = 0; s < p.batch; ++s) slots[s] = s;
+                for (int i = 0; i < n_move; ++i) {
+                    const int r = i + km_index(km_word(p, (uint32_t)i, kTagMove, q.stream, (uint32_t)t), p.batch - i);
+                    const int tmp = slots[i];
+                    slots[i] = slots[r];
+                    slots[r] = tmp;
+                }
+                for (int i = 0; i < n_move; ++i) count[move_centre[i]] = keep_min;
+            }
+        }
+        n_move_s = n_move;
+    }
+    __syncwarp();
+    const int n_move = n_move_s;
+    for (int i = 0; i < n_move; ++i) {                      // the moved centres jump onto minibatch points
+        const uint16_t *src = p.k_prompt + (q.plane + (size_t)idx[slots[i]]) * kHeadDim;
+        double *dst = p.centres64 + (q.cplane + (size_t)move_centre[i]) * kHeadDim;
+        for (int d = lane; d < kHeadDim; d += 32) dst[d] = elem_to_double<kHalf>(src[d]);
+    }
+    if (lane == 0) {
+        const double *dist = p.dist + (size_t)q.id * p.batch;
+        double inertia = 0.0;
+#pragma unroll 8
+        for (int s = 0; s < p.batch; ++s) inertia = __dadd_rn(inertia, dist[s]);
+        KmeansState &st = p.state[q.id];
+        double alpha = __ddiv_rn(__dmul_rn(2.0, (double)p.batch), __dadd_rn((double)q.N, 1.0));
+        if (alpha > 1.0) alpha = 1.0;
+        const double per_point = __ddiv_rn(inertia, (double)p.batch);
+        const double ewa = t == 0 ? per_point
+                                  : __dadd_rn(__dmul_rn(st.ewa, __dsub_rn(1.0, alpha)), __dmul_rn(per_point, alpha));
+        st.ewa = ewa;
+        st.steps += 1;
+        if (t == 0 || ewa < st.ewa_min) { st.ewa_min = ewa; st.bad = 0; }
+        else if (++st.bad >= p.patience) st.stopped = 1;
+    }
+}
+
+__global__ void __launch_bounds__(kThreads)
+km_finish_kernel(KmeansParams p)
+{
+    const Pair q = pair_of(p, blockIdx.y, blockIdx.z);
+    const int e = blockIdx.x * kThreads + threadIdx.x;
+    if (e < q.k * kHeadDim) p.centres_out[q.cplane * kHeadDim + e] = __double2float_rn(p.centres64[q.cplane * kHeadDim + e]);
+    if (e == 0 && p.steps_out) p.steps_out[q.id] = p.state[q.id].steps;
+}
+
+template <bool kHalf>
+cudaError_t run_fit(const KmeansParams &p, cudaStream_t s)
+{
+    const int B = p.n_seqs, H = p.n_kv, pairs = B * H;
+    cudaError_t err;
+#define KM_CHECK() if ((err = cudaGetLastError()) != cudaSuccess) return err
+    km_perm_identity_kernel<<<dim3((p.max_rows_per_seq + kThreads - 1) / kThreads, B, H), kThreads, 0, s>>>(p);
+    KM_CHECK();
+    km_sample_kernel<<<dim3(B, H), 32, 0, s>>>(p);
+    KM_CHECK();
+    const dim3 dist_grid((p.n_init_max + kThreads - 1) / kThreads, p.trials_max, pairs);
+    for (int c = 0; c < p.k_max; ++c) {
+        if (c > 0) {
+            km_draw_trials_kernel<<<dim3(B, H), 32, 0, s>>>(p, c);
+            KM_CHECK();
+        }
+        km_candidate_dist_kernel<kHalf><<<dist_grid, kThreads, 0, s>>>(p, c);
+        KM_CHECK();
+        km_accept_kernel<kHalf><<<dim3(B, H), kThreads, 0, s>>>(p, c);
+        KM_CHECK();
+    }
+    if ((err = cudaMemsetAsync(p.count, 0, sizeof(double) * (size_t)H * p.centres_total, s)) != cudaSuccess) return err;
+    if ((err = cudaMemsetAsync(p.state, 0, sizeof(KmeansState) * (size_t)pairs, s)) != cudaSuccess) return err;
+    const size_t update_smem = sizeof(int32_t) * 2 * (size_t)p.batch;
+    const size_t control_smem = sizeof(int32_t) * ((size_t)p.batch + (size_t)p.batch / 2 + 1);
+    for (int t = 0; t < p.t_max_max; ++t) {
+        km_batch_assign_kernel<kHalf><<<dim3((p.batch + 127) / 128, pairs), 128, 0, s>>>(p, t);
+        KM_CHECK();
+        km_batch_update_kernel<kHalf><<<dim3((p.k_max + 1) / 2, pairs), kThreads, update_smem, s>>>(p, t);
+        KM_CHECK();
+        km_control_kernel<kHalf><<<dim3(B, H), 32, control_smem, s>>>(p, t);
+        KM_CHECK();
+    }
+    km_finish_kernel<<<dim3((p.k_max * kHeadDim + kThreads - 1) / kThreads, B, H), kThreads, 0, s>>>(p);
+    KM_CHECK();
+#undef KM_CHECK
+    return cudaSuccess;
+}
+
+}  // namespace
+
+cudaError_t launch_kmeans_fit(const KmeansParams &p, cudaStream_t s)
+{
+    return p.elem ? run_fit<true>(p, s) : run_fit<false>(p, s);
+}
+
+}  // namespace santapp

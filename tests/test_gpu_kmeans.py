@@ -1,0 +1,82 @@
+"""GPU parity for the minibatch k-means fit of Algorithm 3: the CUDA fit and the fp64 oracle take
+the same random words and the same fp64 arithmetic in the same order, so centres (rounded to fp32)
+and step counts must be equal, not merely close."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import santapp_oracle as orc
+from paper_2609_35629_b200 import binding as sp
+from paper_2609_35629_b200 import synth
+
+import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+
+def _fit_both(spec, n_centres, **opts):
+    data = synth.make_layer(spec, layer=0, keep_centres=True)
+    geom = pu.geometry(spec)
+    k = sp.bf16_bits_to_cuda(data.k_prompt, dtype=geom.torch_dtype)
+    centres, steps = sp.santapp_kmeans_fit(geom, spec.prompt_len, n_centres, k, **opts)
+    torch.cuda.synchronize()
+    centres, steps = centres.cpu().numpy(), steps.cpu().numpy()
+    base = opts.get("stream_base", 0)
+    o = {kk: v for kk, v in opts.items() if kk != "stream_base"}
+    o = {"batch": o.pop("batch_size", 4096), "ratio": o.pop("reassignment_ratio", 0.01), **o}
+    row0 = c0 = 0
+    for b, kc in enumerate(n_centres):
+        N = spec.prompt_len[b]
+        for j in range(spec.n_kv_heads):
+            keys = synth.to_f64(data.k_prompt[j, row0:row0 + N], spec.elem)
+            want, want_steps = orc.minibatch_kmeans(keys, kc, stream=base + b * spec.n_kv_heads + j, **o)
+            assert int(steps[j, b]) == want_steps, f"steps of pair ({b}, {j})"
+            assert np.array_equal(centres[j, c0:c0 + kc], want.astype(np.float32)), f"centres of pair ({b}, {j})"
+        row0 += N
+        c0 += kc
+    return data, centres, steps
+
+
+def test_fit_matches_the_oracle_on_two_ragged_sequences():
+    spec = synth.spec_small_gqa(prompt=(1536, 1000))
+    spec.n_clusters = 24
+    n_centres = [24, 9]
+    _, _, steps = _fit_both(spec, n_centres, batch_size=256, seed=3, stream_base=11)
+    assert steps.min() >= 10
+
+
+def test_fit_with_reassignment_every_period_and_short_patience():
+    """A high ratio moves centres at every period, a patience of 2 stops early, k is not a multiple of
+    the centres a block updates, and the sample is the whole sequence."""
+    spec = synth.spec_small_gqa(prompt=(700,), n_seqs=1, suffix0=(0,))
+    _fit_both(spec, [13], batch_size=512, reassignment_ratio=0.9, patience=2, max_iter=30, seed=1 << 40)
+    _fit_both(spec, [13], batch_size=64, reassignment_ratio=0.0, patience=10 ** 6, max_iter=2)
+
+
+def test_fit_fp16_inputs():
+    spec = synth.spec_small_gqa(prompt=(900,), n_seqs=1, suffix0=(0,))
+    spec.elem = "fp16"
+    _fit_both(spec, [7], batch_size=128)
+
+
+def test_fit_then_parents_then_decode():
+    """Algorithm 3 end to end on the GPU (count, fit, assignment, omission of empty parents), then
+    Algorithm 2 and a decode step on the result, each against the oracle."""
+    from test_gpu_parents import _check_records, _layer_from_labels
+    from test_gpu_parity import check_sparse_step
+    spec = synth.spec_small_gqa(prompt=(2048, 1200))
+    spec.parent_size, spec.reps_per_parent, spec.n_clusters = 64, 4, 32
+    n_centres = [sp.santapp_kmeans_parent_count(n, spec.parent_size) for n in spec.prompt_len]
+    assert n_centres == [32, 18]
+    data, centres, _ = _fit_both(spec, n_centres, batch_size=512)
+    geom = pu.geometry(spec)
+    k = sp.bf16_bits_to_cuda(data.k_prompt)
+    labels = sp.santapp_assign_parents(geom, spec.prompt_len, n_centres, k, torch.from_numpy(centres).cuda())
+    torch.cuda.synchronize()
+    labels = labels.cpu().numpy()
+    keys = synth.bf16_to_f64(data.k_prompt[2, :2048])
+    want, _, _ = orc.nearest_centre_parents(keys, centres[2, :32].astype(np.float64))
+    assert np.array_equal(labels[2, :2048], want)
+    layer = _layer_from_labels(spec, data, labels, n_centres)
+    _check_records(layer, labels, n_centres)
+    check_sparse_step(layer, 0, spec.n_sample)
