@@ -58,9 +58,9 @@ def parse_args():
     ap.add_argument("--key-layout", default="iid", choices=["iid", "runs"],
                     help="cluster of each prompt row: independent draws, or geometric runs (positional locality)")
     ap.add_argument("--elem", default="bf16", choices=["bf16", "fp16"], help="16-bit element type of q, K, V")
-    ap.add_argument("--parents", default="contiguous", choices=["contiguous", "centres"],
-                    help="contiguous: Algorithm 4; centres: the partition Algorithm 3 returns when the fit "
-                         "recovers the centres the synthetic keys were drawn around")
+    ap.add_argument("--parents", default="contiguous", choices=["contiguous", "centres", "kmeans"],
+                    help="contiguous: Algorithm 4; kmeans: Algorithm 3 with the paper's settings (fit on the GPU); "
+                         "centres: Algorithm 3 with the fit replaced by the centres the synthetic keys were drawn around")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-stages", action="store_true")
@@ -276,20 +276,25 @@ def measure_workload(args, workload, n_layers, n_steps, n_warmup, dev, want_e2e,
     ksuf_all = torch.empty((L, B, Hkv, cap, d), dtype=edt, device=dev)
     vsuf_all = torch.empty_like(ksuf_all)
     for l in range(L):
-        by_centres = spec.parents == "centres"
+        by_centres = spec.parents in ("centres", "kmeans")
         data = synth.make_layer(spec, layer=l, keep_centres=conc or by_centres)
         for s in range(N_STEP_INPUTS):
             q_all[s, l] = synth.make_queries(spec, data, s)
         k_prompt = sp.bf16_bits_to_cuda(data.k_prompt, dev, edt)
         v_prompt = sp.bf16_bits_to_cuda(data.v_prompt, dev, edt)
         if by_centres:
-            # Algorithm 3 with the fit replaced by its ideal outcome on these keys: the centres the
-            # rows were drawn around, as many as its first line asks for
-            n_cen = [min(sp.santapp_kmeans_parent_count(n, spec.parent_size), spec.n_clusters) for n in spec.prompt_len]
-            cen = np.concatenate([data.centres[:, :n] for n in n_cen], axis=1)
+            # Algorithm 3: as many centres as its first line asks for; "kmeans" fits them with the paper's
+            # settings, "centres" takes the fit's ideal outcome on these keys (the centres the rows
+            # were drawn around)
+            n_cen = [sp.santapp_kmeans_parent_count(n, spec.parent_size) for n in spec.prompt_len]
             t_build = time.perf_counter()
-            parent_of = sp.santapp_assign_parents(geom, spec.prompt_len, n_cen, k_prompt,
-                                                  torch.from_numpy(np.ascontiguousarray(cen)).to(dev))
+            if spec.parents == "kmeans":
+                cen_dev, fit_steps = sp.santapp_kmeans_fit(geom, spec.prompt_len, n_cen, k_prompt)
+            else:
+                n_cen = [min(n, spec.n_clusters) for n in n_cen]
+                cen = np.concatenate([data.centres[:, :n] for n in n_cen], axis=1)
+                cen_dev = torch.from_numpy(np.ascontiguousarray(cen)).to(dev)
+            parent_of = sp.santapp_assign_parents(geom, spec.prompt_len, n_cen, k_prompt, cen_dev)
             teams = sp.santapp_build_teams_parents(geom, spec.prompt_len, n_cen, k_prompt, v_prompt, parent_of)
         else:
             t_build = time.perf_counter()

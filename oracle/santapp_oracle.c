@@ -646,8 +646,7 @@ int32_t orc_kmeans_parent_count(int32_t N, int32_t P)
 }
 
 /* Last two lines of Algorithm 3. The centres mu_u are an input (the fit that
- * produces them, MiniBatchKMeans with the paper's settings, is a library
- * routine outside this file). Every key joins its nearest centre in squared
+ * produces them is orc_minibatch_kmeans below). Every key joins its nearest centre in squared
  * Euclidean distance, ties going to the smaller centre index; parents without
  * a key are omitted, the others keep the order of their centres.
  *   keys[N][d], centres[n_centres][d]

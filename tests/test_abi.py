@@ -153,3 +153,30 @@ def test_parent_calls_refuse_null_and_misaligned_arguments(lib):
                                            None) == sp.SANTAPP_ERR_INVALID_ARG
     assert lib.santapp_build_teams_parents(ctypes.byref(g), n, c, A, A, A, ctypes.byref(t), A, 16,
                                            None) == sp.SANTAPP_ERR_WORKSPACE_TOO_SMALL
+
+
+def test_kmeans_fit_argument_checks(lib):
+    g = sp.Geometry(1, 28, 4).c()
+    n = (ctypes.c_int32 * 1)(1024)
+    k = (ctypes.c_int32 * 1)(8)
+    A = 0x10000
+    ok = sp.CKmeansOpts(256, 100, 10, 0, 0.01, 0, 0, 0)
+    need = lib.santapp_kmeans_fit_workspace_bytes(ctypes.byref(g), n, k, ctypes.byref(ok))
+    assert need > 4 * 1024 * 4                                     # at least the shuffle array
+    for bad in (sp.CKmeansOpts(0, 100, 10, 0, 0.01, 0, 0, 0), sp.CKmeansOpts(256, 0, 10, 0, 0.01, 0, 0, 0),
+                sp.CKmeansOpts(256, 100, 0, 0, 0.01, 0, 0, 0), sp.CKmeansOpts(256, 100, 10, 0, -1.0, 0, 0, 0)):
+        assert lib.santapp_kmeans_fit_workspace_bytes(ctypes.byref(g), n, k, ctypes.byref(bad)) == 0
+        assert lib.santapp_kmeans_fit(ctypes.byref(g), n, k, A, ctypes.byref(bad), A, None, A, 1 << 40,
+                                      None) == sp.SANTAPP_ERR_INVALID_ARG
+    big = sp.CKmeansOpts(8192, 100, 10, 0, 0.01, 0, 0, 0)
+    assert lib.santapp_kmeans_fit(ctypes.byref(g), n, k, A, ctypes.byref(big), A, None, A, 1 << 40,
+                                  None) == sp.SANTAPP_ERR_UNSUPPORTED
+    too_many = (ctypes.c_int32 * 1)(2000)                           # more centres than keys
+    assert lib.santapp_kmeans_fit(ctypes.byref(g), n, too_many, A, ctypes.byref(ok), A, None, A, 1 << 40,
+                                  None) == sp.SANTAPP_ERR_INVALID_ARG
+    assert lib.santapp_kmeans_fit(ctypes.byref(g), n, k, None, ctypes.byref(ok), A, None, A, 1 << 40,
+                                  None) == sp.SANTAPP_ERR_INVALID_ARG
+    assert lib.santapp_kmeans_fit(ctypes.byref(g), n, k, A + 2, ctypes.byref(ok), A, None, A, 1 << 40,
+                                  None) == sp.SANTAPP_ERR_INVALID_ARG
+    assert lib.santapp_kmeans_fit(ctypes.byref(g), n, k, A, ctypes.byref(ok), A, None, A, 64,
+                                  None) == sp.SANTAPP_ERR_WORKSPACE_TOO_SMALL

@@ -80,3 +80,30 @@ def test_fit_then_parents_then_decode():
     layer = _layer_from_labels(spec, data, labels, n_centres)
     _check_records(layer, labels, n_centres)
     check_sparse_step(layer, 0, spec.n_sample)
+
+
+def _one_pair_at_full_size(spec, j, **opts):
+    """Fit every pair on the GPU, check one KV head against the oracle (the oracle takes seconds per pair)."""
+    data = synth.make_layer(spec, layer=0)
+    geom = pu.geometry(spec)
+    n_centres = [sp.santapp_kmeans_parent_count(n, spec.parent_size) for n in spec.prompt_len]
+    k = sp.bf16_bits_to_cuda(data.k_prompt)
+    centres, steps = sp.santapp_kmeans_fit(geom, spec.prompt_len, n_centres, k, **opts)
+    torch.cuda.synchronize()
+    keys = synth.bf16_to_f64(data.k_prompt[j, :spec.prompt_len[0]])
+    want, want_steps = orc.minibatch_kmeans(keys, n_centres[0], stream=j)
+    assert int(steps[j, 0]) == want_steps
+    assert np.array_equal(centres[j, :n_centres[0]].cpu().numpy(), want.astype(np.float32))
+    return n_centres
+
+
+def test_fit_config_2_full_size_paper_settings():
+    """32K keys per KV head, 64 centres, the paper's settings (minibatch 4096, 100 iterations,
+    patience 10, ratio 0.01, seed 0): the configuration `bench.py --parents kmeans` prepares."""
+    assert _one_pair_at_full_size(synth.spec_qwen_b1(), j=1) == [64]
+
+
+def test_fit_many_centres_paper_parent_size():
+    """Parents of nominal size 16 (the paper's operating point) on 8K keys: 512 centres, 8 trials per
+    centre, the initialisation sample is the whole sequence."""
+    assert _one_pair_at_full_size(synth.spec_paper_point(prompt=8192), j=3) == [512]
