@@ -125,42 +125,68 @@ km_candidate_dist_kernel(KmeansParams p, int c)
         sqdist_rows<kHalf>(keys + (size_t)perm[i] * 16, keys + (size_t)perm[at] * 16);
 }
 
+constexpr int kAcceptThreads = 512;      // 16 warps: one per trial for up to 65536 centres (2 + ln k <= 13)
+
 // One block per pair: potentials of the trials (one lane each, sums in sample order), the best
 // trial becomes centre c, the nearest-centre distances are lowered.
 template <bool kHalf>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kAcceptThreads)
 km_accept_kernel(KmeansParams p, int c)
 {
+    constexpr int kChunk = 128;
     __shared__ int best_s;
+    __shared__ double pot_s[32];
+    __shared__ double chunk_s[kAcceptThreads / 32][kChunk];
     const Pair q = pair_of(p, blockIdx.x, blockIdx.y);
     if (c >= q.k) return;
     const int tid = threadIdx.x;
     const int n_trials = c == 0 ? 1 : q.L;
     double *closest = p.closest + (size_t)q.id * p.n_init_max;
     const double *cand = p.cand + (size_t)q.id * p.trials_max * p.n_init_max;
-    if (tid < 32) {
-        double pot = INFINITY;
-        if (c > 0 && tid < n_trials) {
-            const double *mine = cand + (size_t)tid * p.n_init_max;
-            pot = 0.0;
-#pragma unroll 4
-            for (int i = 0; i < q.n_init; ++i) {
+    {
+        // warp l sums trial l: the lanes fetch a chunk of 256 terms into shared memory (the next
+        // chunk is in flight meanwhile), then lane 0 adds them in sample order: one chain of
+        // additions, as the order of the sum is part of the result
+        const int warp = tid >> 5, lane = tid & 31;
+        double *buf = chunk_s[warp];
+        for (int l = warp; l < n_trials && c > 0; l += kAcceptThreads / 32) {
+            const double *mine = cand + (size_t)l * p.n_init_max;
+            double pot = 0.0;
+            auto fetch = [&](int i) {                       // term i of the potential (0 past the end)
+                if (i >= q.n_init) return 0.0;
                 const double d = mine[i], o = closest[i];
-                pot = __dadd_rn(pot, d < o ? d : o);
+                return d < o ? d : o;
+            };
+            double term[kChunk / 32];
+#pragma unroll
+            for (int v = 0; v < kChunk / 32; ++v) term[v] = fetch(32 * v + lane);
+            for (int i0 = 0; i0 < q.n_init; i0 += kChunk) {
+                __syncwarp();                               // lane 0 is done with the previous chunk
+#pragma unroll
+                for (int v = 0; v < kChunk / 32; ++v) buf[32 * v + lane] = term[v];
+#pragma unroll
+                for (int v = 0; v < kChunk / 32; ++v) term[v] = fetch(i0 + kChunk + 32 * v + lane);
+                __syncwarp();
+                if (lane == 0) {
+                    const int n = min(kChunk, q.n_init - i0);
+#pragma unroll 8
+                    for (int r = 0; r < n; ++r) pot = __dadd_rn(pot, buf[r]);
+                }
             }
+            if (lane == 0) pot_s[l] = pot;
         }
-        int best = 0;
-        double best_pot = __shfl_sync(0xFFFFFFFFu, pot, 0);
-        for (int l = 1; l < n_trials; ++l) {
-            const double v = __shfl_sync(0xFFFFFFFFu, pot, l);
-            if (v < best_pot) { best_pot = v; best = l; }
+        __syncthreads();
+        if (tid == 0) {
+            int best = 0;
+            for (int l = 1; l < n_trials; ++l)
+                if (pot_s[l] < pot_s[best]) best = l;
+            best_s = best;
         }
-        if (tid == 0) best_s = best;
     }
     __syncthreads();
     const int best = best_s;
     const double *win = cand + (size_t)best * p.n_init_max;
-    for (int i = tid; i < q.n_init; i += kThreads) {
+    for (int i = tid; i < q.n_init; i += kAcceptThreads) {
         const double d = win[i];
         if (c == 0 || d < closest[i]) closest[i] = d;
     }
@@ -172,30 +198,40 @@ km_accept_kernel(KmeansParams p, int c)
     }
 }
 
-// One warp per pair: the L trial points of centre c, drawn with probability proportional to the
-// distance to the nearest chosen centre (inverse CDF over the sample in order; every lane runs the
-// same running sum and watches for its own target).
-__global__ void __launch_bounds__(32)
+// One block per pair: the L trial points of centre c, drawn with probability proportional to the
+// distance to the nearest chosen centre by inverse CDF over the sample in order. The running sums
+// are formed by one thread (their order is part of the result) in shared memory; each trial then
+// finds the first running sum above its target by bisection (the sums never decrease).
+__global__ void __launch_bounds__(kThreads)
 km_draw_trials_kernel(KmeansParams p, int c)
 {
+    extern __shared__ double cum_s[];                       // [n_init]
     const Pair q = pair_of(p, blockIdx.x, blockIdx.y);
     if (c >= q.k) return;
-    const int lane = threadIdx.x;
+    const int tid = threadIdx.x;
     const double *closest = p.closest + (size_t)q.id * p.n_init_max;
-    double total = 0.0;
+    for (int i = tid; i < q.n_init; i += kThreads) cum_s[i] = closest[i];
+    __syncthreads();
+    if (tid == 0) {
+        double cum = 0.0;
 #pragma unroll 8
-    for (int i = 0; i < q.n_init; ++i) total = __dadd_rn(total, closest[i]);
-    const uint32_t w = km_word(p, (uint32_t)lane, kTagStart, q.stream, (uint32_t)c);
-    const double target = __dmul_rn(((double)w + 0.5) * (1.0 / 4294967296.0), total);
-    double cum = 0.0;
-    int at = q.n_init - 1;
-    bool found = false;
-#pragma unroll 8
-    for (int i = 0; i < q.n_init; ++i) {
-        cum = __dadd_rn(cum, closest[i]);
-        if (!found && cum > target) { at = i; found = true; }
+        for (int i = 0; i < q.n_init; ++i) {
+            cum = __dadd_rn(cum, cum_s[i]);
+            cum_s[i] = cum;
+        }
     }
-    if (lane < q.L) p.pick[(size_t)q.id * p.trials_max + lane] = at;
+    __syncthreads();
+    if (tid < q.L) {
+        const double total = cum_s[q.n_init - 1];
+        const uint32_t w = km_word(p, (uint32_t)tid, kTagStart, q.stream, (uint32_t)c);
+        const double target = __dmul_rn(((double)w + 0.5) * (1.0 / 4294967296.0), total);
+        int lo = 0, hi = q.n_init;                          // first i in [lo, hi) with cum_s[i] > target
+        while (lo < hi) {
+            const int mid = (lo + hi) >> 1;
+            if (cum_s[mid] > target) hi = mid; else lo = mid + 1;
+        }
+        p.pick[(size_t)q.id * p.trials_max + tid] = lo < q.n_init ? lo : q.n_init - 1;
+    }
 }
 
 // ---- 3. minibatch steps ----
@@ -381,14 +417,18 @@ cudaError_t run_fit(const KmeansParams &p, cudaStream_t s)
     km_sample_kernel<<<dim3(B, H), 32, 0, s>>>(p);
     KM_CHECK();
     const dim3 dist_grid((p.n_init_max + kThreads - 1) / kThreads, p.trials_max, pairs);
+    const size_t draw_smem = sizeof(double) * (size_t)p.n_init_max;
+    if ((err = cudaFuncSetAttribute(km_draw_trials_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    (int)draw_smem)) != cudaSuccess)
+        return err;
     for (int c = 0; c < p.k_max; ++c) {
         if (c > 0) {
-            km_draw_trials_kernel<<<dim3(B, H), 32, 0, s>>>(p, c);
+            km_draw_trials_kernel<<<dim3(B, H), kThreads, draw_smem, s>>>(p, c);
             KM_CHECK();
         }
         km_candidate_dist_kernel<kHalf><<<dist_grid, kThreads, 0, s>>>(p, c);
         KM_CHECK();
-        km_accept_kernel<kHalf><<<dim3(B, H), kThreads, 0, s>>>(p, c);
+        km_accept_kernel<kHalf><<<dim3(B, H), kAcceptThreads, 0, s>>>(p, c);
         KM_CHECK();
     }
     if ((err = cudaMemsetAsync(p.count, 0, sizeof(double) * (size_t)H * p.centres_total, s)) != cudaSuccess) return err;
