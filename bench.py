@@ -520,7 +520,8 @@ def measure_workload(args, workload, n_layers, n_steps, n_warmup, dev, want_e2e,
     # ---- the oracle on the host cores, bounded sample ----
     cpu_baseline = None
     if rank == 0 and world == 1 and want_cpu:
-        cpu_baseline = cpu_baseline_leg(spec, host_layers[0], layers[0]["teams"], seed)
+        cpu_baseline = cpu_baseline_leg(spec, host_layers[0], layers[0]["teams"], seed,
+                                        kmeans_group_records(spec, host_layers[0], dev))
 
     if rank == 0:
         line = {
@@ -550,7 +551,35 @@ def measure_workload(args, workload, n_layers, n_steps, n_warmup, dev, want_e2e,
     return None
 
 
-def cpu_baseline_leg(spec, data, teams, seed):
+def kmeans_group_records(spec, data, dev):
+    """Records of the paper's centroid-guided baseline for sequence 0: k-means groups of nominal size
+    4 and 16 (Algorithm 3's fit and assignment with the paper's settings, one group per cluster routed
+    by its mean key), built by the library on the GPU. Only for bf16 inputs and prompts where the
+    greedy start of a fit with N / 4 centres stays within seconds."""
+    import torch
+    from paper_2609_35629_b200 import binding as sp
+    N = int(spec.prompt_len[0])
+    if spec.elem != "bf16" or N > 40000 or N < 64:
+        return {}
+    k = sp.bf16_bits_to_cuda(np.ascontiguousarray(data.k_prompt[:, :N]), dev)
+    out = {}
+    for size in (4, 16):
+        geom = sp.Geometry(1, spec.n_q_heads, spec.n_kv_heads, spec.head_dim, size, 1)
+        n_cen = [sp.santapp_kmeans_parent_count(N, size)]
+        centres, _ = sp.santapp_kmeans_fit(geom, [N], n_cen, k)
+        labels = sp.santapp_assign_parents(geom, [N], n_cen, k, centres)
+        t = sp.santapp_build_groups_mean_parents(geom, [N], n_cen, k, k, labels)
+        torch.cuda.synchronize()
+        cnt = t.team_count.cpu().numpy()[:, 0]
+        trs, tok = t.team_row_start.cpu().numpy(), t.row_token.cpu().numpy()
+        rep = t.rep_keys.view(torch.int16).cpu().numpy().view(np.uint16)
+        out[f"centroid_kmeans_groups_of_{size}"] = [
+            (np.ascontiguousarray(trs[j, :cnt[j] + 1]), np.ascontiguousarray(tok[j]), rep[j, :cnt[j]])
+            for j in range(spec.n_kv_heads)]
+    return out
+
+
+def cpu_baseline_leg(spec, data, teams, seed, group_records=None):
     """The fp64 oracle on sequence 0 of layer 0, using the GPU-built team records, timed on
     all host cores for a bounded number of layer-steps."""
     from oracle import santapp_oracle as orc
@@ -618,10 +647,13 @@ def cpu_baseline_leg(spec, data, teams, seed):
              "dense_1_thread_us": few(dense_n(1), 2)}
     # routing agreement with dense attention over the prompt (Eq. diagnostic-kl), no sampling involved:
     # mean over the heads of two of the step inputs, for the workload's teams and for the
-    # centroid-guided baseline (groups of 4 and of 16 contiguous keys routed by their mean key)
-    variants = {"teams": [(ts[j], tm[j], rk[j]) for j in range(n_kv)]}
+    # centroid-guided baseline (groups of 4 and of 16 keys routed by their mean key: contiguous
+    # groups, and the k-means groups the paper's baseline uses)
+    variants = {"teams": [(ts[j][:M[j] + 1], tm[j], rk[j][:M[j]]) for j in range(n_kv)]}
     for size in (4, 16):
         variants[f"centroid_groups_of_{size}"] = [orc.group_mean_keys(k[j], size) for j in range(n_kv)]
+    for name, recs in (group_records or {}).items():              # k-means groups, built by the library
+        variants[name] = [(r[0], r[1], synth.to_f64(r[2], spec.elem)) for r in recs]
     kls = {name: [] for name in variants}
     for i in range(2):
         q, _, _, _ = inputs(i * 100)
