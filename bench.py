@@ -566,6 +566,8 @@ def kmeans_group_records(spec, data, dev):
     for size in (4, 16):
         geom = sp.Geometry(1, spec.n_q_heads, spec.n_kv_heads, spec.head_dim, size, 1)
         n_cen = [sp.santapp_kmeans_parent_count(N, size)]
+        if 3 * max(4096, n_cen[0]) > 28672:                        # the fit's limit on its initialisation sample
+            continue
         centres, _ = sp.santapp_kmeans_fit(geom, [N], n_cen, k)
         labels = sp.santapp_assign_parents(geom, [N], n_cen, k, centres)
         t = sp.santapp_build_groups_mean_parents(geom, [N], n_cen, k, k, labels)

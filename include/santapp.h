@@ -236,7 +236,8 @@ int32_t santapp_kmeans_parent_count(int32_t prompt_len, int32_t parent_size);
  *                    the layout santapp_assign_parents takes
  *   steps_run        device int32 [n_kv_heads][n_seqs] or NULL, out: minibatch steps each fit ran
  *   workspace        device, >= santapp_kmeans_fit_workspace_bytes(...)
- * batch_size > 4096: SANTAPP_ERR_UNSUPPORTED. The call enqueues a few kernels per centre and per
+ * batch_size > 4096, or an initialisation sample above 28672 keys (more than 9557 centres in a
+ * sequence): SANTAPP_ERR_UNSUPPORTED. The call enqueues a few kernels per centre and per
  * step on `stream`; it does not synchronise.
  */
 typedef struct santapp_kmeans_opts {

@@ -486,6 +486,8 @@ int santapp_build_groups_mean_parents(const santapp_geom *geom, const int32_t *p
 
 namespace {
 
+constexpr int kKmeansMaxSample = 28672;     // 224 KB of fp64 running sums: up to 9557 centres per sequence
+
 struct KmeansLayout {
     size_t row_off, cen_off, tabs, perm, closest, cand, pick, centres64, count, idx, label, dist, state, total;
     int k_max, n_init_max, trials_max, t_max_max, max_rows;
@@ -523,6 +525,7 @@ int kmeans_layout(const santapp_geom *geom, const int32_t *prompt_len_host, cons
         if (N > L->max_rows) L->max_rows = N;
     }
     if (L->rows_total >= (int64_t)1 << 31) return SANTAPP_ERR_UNSUPPORTED;
+    if (L->n_init_max > kKmeansMaxSample) return SANTAPP_ERR_UNSUPPORTED;   // its running sums live in shared memory
     const size_t H = (size_t)geom->n_kv_heads, pairs = H * (size_t)B;
     if (pairs > 65535) return SANTAPP_ERR_UNSUPPORTED;
     size_t off = 0;
