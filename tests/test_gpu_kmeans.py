@@ -107,3 +107,18 @@ def test_fit_many_centres_paper_parent_size():
     """Parents of nominal size 16 (the paper's operating point) on 8K keys: 512 centres, 8 trials per
     centre, the initialisation sample is the whole sequence."""
     assert _one_pair_at_full_size(synth.spec_paper_point(prompt=8192), j=3) == [512]
+
+
+@pytest.mark.parametrize("case", range(16))
+def test_fit_random_small_configurations(case):
+    rng = np.random.default_rng(500 + case)
+    n_seqs = int(rng.integers(1, 4))
+    prompt = tuple(int(rng.integers(2, 1500)) for _ in range(n_seqs))
+    spec = synth.spec_small_gqa(n_seqs=n_seqs, prompt=prompt, suffix0=(0,) * n_seqs)
+    spec.n_clusters = int(rng.integers(2, 30))
+    spec.seed = case
+    spec.elem = "fp16" if case % 2 else "bf16"
+    n_centres = [int(rng.integers(1, min(n, 40) + 1)) for n in prompt]
+    _fit_both(spec, n_centres, batch_size=int(rng.choice([16, 100, 512, 4096])), max_iter=int(rng.choice([1, 3, 100])),
+              patience=int(rng.choice([1, 3, 10])), reassignment_ratio=float(rng.choice([0.0, 0.01, 0.5])),
+              seed=int(rng.integers(1 << 62)), stream_base=int(rng.integers(1 << 30)))
