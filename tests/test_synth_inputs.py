@@ -57,3 +57,34 @@ def test_suffix_schedule():
     assert spec.suffix_len(0)[0] == 1 and spec.suffix_len(10)[0] == 11
     assert spec.suffix_len(10_000)[0] == spec.suffix_cap            # clamps at the capacity
     assert synth.spec_paper_point().suffix_len(5)[0] == 0
+
+
+def test_fp16_rounding_and_widening_are_exact_inverses_on_representable_values():
+    import numpy as np
+    from paper_2609_35629_b200 import synth
+    rng = np.random.default_rng(0)
+    x = rng.standard_normal(1000).astype(np.float32) * 3
+    bits = synth.round_bits(x, "fp16")
+    assert bits.dtype == np.uint16
+    back = synth.to_f64(bits, "fp16")
+    assert np.array_equal(back, x.astype(np.float16).astype(np.float64))        # numpy's round-to-nearest-even
+    assert np.array_equal(synth.round_bits(back.astype(np.float32), "fp16"), bits)
+    assert np.max(np.abs(back - x)) <= 2.0 ** -11 * np.max(np.abs(x)) + 1e-12      # 11 significant bits
+    # bf16 stays the default and differs
+    assert np.array_equal(synth.round_bits(x), synth.f32_to_bf16_bits(x))
+    assert not np.array_equal(synth.round_bits(x), bits)
+
+
+def test_spec_element_type_reaches_every_tensor():
+    import numpy as np
+    from paper_2609_35629_b200 import synth
+    a = synth.spec_small_gqa()
+    b = synth.spec_small_gqa()
+    b.elem = "fp16"
+    da, db = synth.make_layer(a), synth.make_layer(b)
+    for name in ("k_prompt", "v_prompt", "k_suffix", "v_suffix"):
+        xa, xb = synth.to_f64(getattr(da, name), "bf16"), synth.to_f64(getattr(db, name), "fp16")
+        assert not np.array_equal(getattr(da, name), getattr(db, name))
+        assert np.max(np.abs(xa - xb)) < 0.05                                   # same draws, other rounding
+    qa, qb = synth.make_queries(a, da, 0), synth.make_queries(b, db, 0)
+    assert qa.shape == qb.shape and not np.array_equal(qa, qb)
