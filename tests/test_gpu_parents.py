@@ -240,3 +240,23 @@ def test_centroid_groups_on_centre_parents():
     bad = pu.geometry(_spec(prompt=(2048, 1100), R=4))
     with pytest.raises(sp.SantappError):
         sp.santapp_build_groups_mean_parents(bad, spec.prompt_len, n_centres, layer.k_prompt, layer.v_prompt, lab_dev)
+
+
+def test_null_team_count_means_every_slot_is_a_team():
+    """Records of the contiguous builder fill every slot, so the decode must give the same bits with
+    team_count left NULL (callers that built their records before the field existed)."""
+    spec = synth.spec_small_gqa()
+    layer = pu.GpuLayer(spec, synth.make_layer(spec, layer=0))
+    q_bits = synth.make_queries(spec, layer.data, 0)
+    sl = spec.suffix_len(0)
+    out_a, dbg_a = pu.gpu_step(layer, q_bits, sl, spec.n_sample, 5, 0)
+    saved = layer.teams.c.team_count
+    layer.teams.c.team_count = None
+    try:
+        out_b, dbg_b = pu.gpu_step(layer, q_bits, sl, spec.n_sample, 5, 0)
+        dense_b, _ = pu.gpu_step(layer, q_bits, sl, 0, 0, 0, dense=True)
+    finally:
+        layer.teams.c.team_count = saved
+    dense_a, _ = pu.gpu_step(layer, q_bits, sl, 0, 0, 0, dense=True)
+    assert np.array_equal(out_a, out_b) and np.array_equal(dense_a, dense_b)
+    assert torch.equal(dbg_a.sel_idx, dbg_b.sel_idx)
