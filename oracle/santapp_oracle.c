@@ -23,6 +23,7 @@
  *                             reading and are documented with the function)
  *   orc_logical_access_*      logical KV-access counter, Eq. (qwen-logical-access)
  *   orc_team_budget           selected-team count, Eq. (method-budget)
+ *   orc_mla_logical_access_pct   shared-row counter of a shared-latent cache, Eq. (mla-logical-access)
  *   orc_routing_kl            routing-agreement diagnostic, Eq. (diagnostic-kl)
  *   orc_group_mean_keys       centroid-guided baseline of the routing diagnostic: one group per
  *                             parent, routed by the arithmetic mean of its keys
@@ -871,4 +872,19 @@ int32_t orc_minibatch_kmeans(int32_t N, int d, const double *keys, int32_t k, in
     }
     free(sum); free(slots); free(label); free(idx); free(count);
     return steps;
+}
+
+/* Shared-row accounting for a shared-latent cache, Eq. (mla-logical-access): per decoding call c,
+ * r[c] routing rows (one per representative), u[c] rows in the union over all heads of the
+ * selected prompt members and the exact suffix, d[c] rows a dense call reads. One row stands for a
+ * token's shared latent and rotary key; a row used in routing and in attention counts in both.
+ * Counts are pooled over the calls before the division. Returns the percentage. */
+double orc_mla_logical_access_pct(int64_t n_calls, const int64_t *r, const int64_t *u, const int64_t *d)
+{
+    double num = 0.0, den = 0.0;
+    for (int64_t c = 0; c < n_calls; ++c) {
+        num += (double)r[c] + (double)u[c];
+        den += (double)d[c];
+    }
+    return 100.0 * num / den;
 }

@@ -87,6 +87,8 @@ def lib():
         L.orc_group_mean_keys.restype = _c.c_int32
         L.orc_group_mean_keys_parents.argtypes = [_c.c_int, _f64p, _c.c_int32, _i32p, _i32p, _f64p]
         L.orc_group_mean_keys_parents.restype = None
+        L.orc_mla_logical_access_pct.argtypes = [_c.c_int64, _i64p, _i64p, _i64p]
+        L.orc_mla_logical_access_pct.restype = _c.c_double
         L.orc_minibatch_kmeans.argtypes = [_c.c_int32, _c.c_int, _f64p, _c.c_int32, _c.c_int32, _c.c_int32, _c.c_int32,
                                            _c.c_double, _c.c_uint64, _c.c_uint32, _f64p]
         L.orc_minibatch_kmeans.restype = _c.c_int32
@@ -372,3 +374,9 @@ def minibatch_kmeans(keys, k, batch=4096, max_iter=100, patience=10, ratio=0.01,
     centres = np.zeros((k, d))
     steps = lib().orc_minibatch_kmeans(N, d, keys, k, batch, max_iter, patience, ratio, seed, stream, centres)
     return centres, int(steps)
+
+
+def mla_logical_access_pct(r, u, d):
+    """Shared-row logical access of Eq. (mla-logical-access), pooled over the calls."""
+    r, u, d = (np.ascontiguousarray(a, dtype=np.int64) for a in (r, u, d))
+    return float(lib().orc_mla_logical_access_pct(r.shape[0], r, u, d))

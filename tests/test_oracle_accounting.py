@@ -59,3 +59,30 @@ def test_union_rows_counts_each_team_once():
     sel = np.array([[0, 2], [2, 3], [0, 3]], dtype=np.int32)
     assert orc.union_rows(ts, sel) == 3 + 5 + 1
     assert orc.union_rows(ts, sel[:1]) == 8
+
+
+def test_shared_row_counter_of_a_shared_latent_cache():
+    """Eq. (mla-logical-access): routing rows and the union over heads are both charged against the
+    dense shared-row count, pooled over calls. The paper prints the two terms and their total for
+    S = 512 and the attention term and the total for S = 1024; the counter must be additive in
+    exactly that way."""
+    g = _golden()
+    d = 100000                                                       # any dense row count: percentages scale
+    r = round(g["mla_S512_routing_pct"] * d / 100)
+    u = round(g["mla_S512_attention_pct"] * d / 100)
+    assert abs(orc.mla_logical_access_pct([r], [u], [d]) - g["mla_S512_total_pct"]) < 0.005
+    assert abs(orc.mla_logical_access_pct([r], [0], [d]) - g["mla_S512_routing_pct"]) < 0.005
+    # S = 1024: the printed total minus the printed attention term leaves a routing term within 0.1 of
+    # S = 512's (the routing scan does not depend on the budget, only the trajectory's length does)
+    routing_1024 = g["mla_S1024_total_pct"] - g["mla_S1024_attention_pct"]
+    assert abs(routing_1024 - g["mla_S512_routing_pct"]) < 0.1
+    u2 = round(g["mla_S1024_attention_pct"] * d / 100)
+    r2 = round(routing_1024 * d / 100)
+    assert abs(orc.mla_logical_access_pct([r2], [u2], [d]) - g["mla_S1024_total_pct"]) < 0.005
+    # above 100 % is possible: a row read in both passes is charged twice
+    assert orc.mla_logical_access_pct([50], [100], [100]) == 150.0
+    # pooled before the division, not a mean of ratios
+    assert orc.mla_logical_access_pct([10, 0], [10, 0], [100, 300]) == 5.0
+    # one counted row per token: no factor 2 for keys and values, unlike the GQA counter
+    assert orc.mla_logical_access_pct([0], [7], [14]) == 50.0
+    assert orc.logical_access_pct([0], [7], [0], [14]) == 50.0
