@@ -32,11 +32,12 @@ struct BatchView {
     int elem;                       // element type of q / K / V / representative keys: 0 bf16, 1 fp16
 };
 
-// Teams of (sequence b, KV head j): the first `pair_team_count` slots of the sequence's range.
+// Teams of (sequence b, KV head j): the first `pair_team_count` slots of the sequence's range (a
+// count outside [0, slots] is clamped, so a corrupt table cannot send a kernel past the records).
 __device__ __forceinline__ int pair_team_count(const BatchView &bv, int b, int j)
 {
-    return bv.team_count ? bv.team_count[(size_t)j * bv.n_seqs + b]
-                         : (int)(bv.seq_team_off[b + 1] - bv.seq_team_off[b]);
+    const int slots = (int)(bv.seq_team_off[b + 1] - bv.seq_team_off[b]);
+    return bv.team_count ? min(max(bv.team_count[(size_t)j * bv.n_seqs + b], 0), slots) : slots;
 }
 
 // Read plan of one (sequence, KV head) pair: the union of the teams its query heads selected,
