@@ -554,17 +554,20 @@ def measure_workload(args, workload, n_layers, n_steps, n_warmup, dev, want_e2e,
 def kmeans_group_records(spec, data, dev):
     """Records of the paper's centroid-guided baseline for sequence 0: k-means groups of nominal size
     4 and 16 (Algorithm 3's fit and assignment with the paper's settings, one group per cluster routed
-    by its mean key), built by the library on the GPU. Only for bf16 inputs and prompts where the
-    greedy start of a fit with N / 4 centres stays within seconds."""
+    by its mean key), built by the library on the GPU. Only for prompts where the greedy start of a
+    fit with N / 4 centres stays within seconds."""
     import torch
     from paper_2609_35629_b200 import binding as sp
     N = int(spec.prompt_len[0])
-    if spec.elem != "bf16" or N > 40000 or N < 64:
+    if N > 40000 or N < 64:
         return {}
-    k = sp.bf16_bits_to_cuda(np.ascontiguousarray(data.k_prompt[:, :N]), dev)
+    half = spec.elem == "fp16"
+    k = sp.bf16_bits_to_cuda(np.ascontiguousarray(data.k_prompt[:, :N]), dev,
+                             torch.float16 if half else torch.bfloat16)
     out = {}
     for size in (4, 16):
-        geom = sp.Geometry(1, spec.n_q_heads, spec.n_kv_heads, spec.head_dim, size, 1)
+        geom = sp.Geometry(1, spec.n_q_heads, spec.n_kv_heads, spec.head_dim, size, 1,
+                           sp.SANTAPP_FP16 if half else sp.SANTAPP_BF16)
         n_cen = [sp.santapp_kmeans_parent_count(N, size)]
         if 3 * max(4096, n_cen[0]) > 28672:                        # the fit's limit on its initialisation sample
             continue
@@ -653,7 +656,7 @@ def cpu_baseline_leg(spec, data, teams, seed, group_records=None):
     # groups, and the k-means groups the paper's baseline uses)
     variants = {"teams": [(ts[j][:M[j] + 1], tm[j], rk[j][:M[j]]) for j in range(n_kv)]}
     for size in (4, 16):
-        variants[f"centroid_groups_of_{size}"] = [orc.group_mean_keys(k[j], size) for j in range(n_kv)]
+        variants[f"centroid_groups_of_{size}"] = [orc.group_mean_keys(k[j], size, elem=spec.elem) for j in range(n_kv)]
     for name, recs in (group_records or {}).items():              # k-means groups, built by the library
         variants[name] = [(r[0], r[1], synth.to_f64(r[2], spec.elem)) for r in recs]
     kls = {name: [] for name in variants}

@@ -64,7 +64,7 @@ typedef void *santapp_stream;            /* cudaStream_t */
 /* 16-bit element type of the inputs. Wherever this header says "bf16" for q, K, V, the suffix or
  * the representative keys, the tensor holds raw 16-bit patterns of this type. Outputs are fp32 and
  * every accumulation is fp32 or fp64 for both. The paper's own runs use fp16 inputs
- * (Appendix "Kernel evaluation protocol and profiling"); santapp_build_groups_mean takes bf16 only. */
+ * (Appendix "Kernel evaluation protocol and profiling"). */
 typedef enum santapp_elem { SANTAPP_BF16 = 0, SANTAPP_FP16 = 1 } santapp_elem;
 
 /* Problem geometry (host struct). */
@@ -190,7 +190,7 @@ int santapp_build_teams(const santapp_geom *geom, const int32_t *prompt_len_host
  * santapp_decode_attn unchanged. The paper forms the groups by k-means; this call uses the
  * contiguous parents of Algorithm 4 (group size = geom->parent_size, last one possibly short).
  * The mean of a parent is the fp64 sum of its keys in token order divided by their number, stored
- * as bf16 (fp64 to fp32 to nearest, fp32 to bf16 to nearest even). Rows keep their token order.
+ * in the element type (fp64 to fp32 to nearest, fp32 to bf16 or fp16 to nearest even). Rows keep their token order.
  * geom->reps_per_parent must be 1 (sizes then come from santapp_build_teams_sizes as usual).
  * Arguments, ownership and errors as for santapp_build_teams.
  */
@@ -304,7 +304,7 @@ int santapp_build_teams_parents(const santapp_geom *geom, const int32_t *prompt_
 /*
  * Centroid-guided groups on a given parent partition (the paper's baseline forms its groups by
  * k-means): as santapp_build_groups_mean, but one group per non-empty parent of `parent_of`, in label
- * order, members in token order. geom->reps_per_parent must be 1; bf16 inputs only. Arguments,
+ * order, members in token order. geom->reps_per_parent must be 1. Arguments,
  * sizes (santapp_parent_teams_sizes) and errors as for santapp_build_teams_parents.
  */
 int santapp_build_groups_mean_parents(const santapp_geom *geom, const int32_t *prompt_len_host,

@@ -603,16 +603,40 @@ double orc_routing_kl(int d, const double *q, int64_t N, const double *k, int32_
     return kl;
 }
 
+/* A real number stored as a 16-bit routing key and read back: fp64 -> fp32 (round to nearest),
+ * then fp32 -> the element type (round to nearest, ties to even). half = 0: bf16 (the upper 16
+ * bits of the fp32 pattern). half = 1: IEEE binary16 (10 fraction bits, smallest normal 2^-14,
+ * gradual underflow in steps of 2^-24, overflow to infinity from 65520). */
+double orc_round_to_elem(double x, int half)
+{
+    float f = (float)x;
+    if (!half) {
+        uint32_t bits;
+        memcpy(&bits, &f, sizeof bits);
+        uint32_t rounded = (bits + 0x7FFFu + ((bits >> 16) & 1u)) & 0xFFFF0000u;
+        float back;
+        memcpy(&back, &rounded, sizeof back);
+        return (double)back;
+    }
+    if (f != f || isinf(f) || f == 0.0f) return (double)f;
+    double a = fabs((double)f);
+    int e;
+    (void)frexp(a, &e);                                   /* a = m * 2^e with m in [0.5, 1) */
+    int ulp_exp = e - 1 < -14 ? -24 : e - 11;             /* spacing of binary16 around a */
+    double v = ldexp(nearbyint(ldexp(a, -ulp_exp)), ulp_exp);   /* nearbyint: ties to even */
+    if (v > 65504.0) v = INFINITY;
+    return f < 0.0f ? -v : v;
+}
+
 /* Centroid-guided baseline (Section "How closely routing follows dense attention" and the
  * appendix on the KL variants): every group is routed by the arithmetic mean of its keys
  * instead of an actual key; the routing logit still adds log n_g, sampling, correction and
- * estimator are unchanged. The paper forms the groups by k-means; here the groups are the
- * contiguous parents of Algorithm 4 (k-means parents are not built in this library).
+ * estimator are unchanged. The paper forms the groups by k-means (orc_group_mean_keys_parents
+ * takes any partition); here the groups are the contiguous parents of Algorithm 4.
  * For parent u: mean_u = (sum over its tokens in index order of k_i) / |C_u| in fp64, then
- * stored as a bf16 value like every other routing key: fp64 -> fp32 (round to nearest) ->
- * bf16 (round to nearest even). out_mean[n_parents][d] receives those values widened back to
- * fp64. Returns n_parents. */
-int32_t orc_group_mean_keys(int32_t N, int d, const double *keys, int32_t P, double *out_mean)
+ * stored as a 16-bit value like every other routing key (orc_round_to_elem).
+ * out_mean[n_parents][d] receives those values widened back to fp64. Returns n_parents. */
+int32_t orc_group_mean_keys(int32_t N, int d, const double *keys, int32_t P, int half, double *out_mean)
 {
     int32_t n_parents = (N + P - 1) / P;
     for (int32_t u = 0; u < n_parents; ++u) {
@@ -620,13 +644,7 @@ int32_t orc_group_mean_keys(int32_t N, int d, const double *keys, int32_t P, dou
         for (int j = 0; j < d; ++j) {
             double sum = 0.0;
             for (int32_t i = lo; i < hi; ++i) sum += keys[(int64_t)i * d + j];
-            float f = (float)(sum / (double)(hi - lo));
-            uint32_t bits;
-            memcpy(&bits, &f, sizeof bits);
-            uint32_t rounded = (bits + 0x7FFFu + ((bits >> 16) & 1u)) & 0xFFFF0000u;
-            float back;
-            memcpy(&back, &rounded, sizeof back);
-            out_mean[(int64_t)u * d + j] = (double)back;
+            out_mean[(int64_t)u * d + j] = orc_round_to_elem(sum / (double)(hi - lo), half);
         }
     }
     return n_parents;
@@ -679,23 +697,17 @@ int32_t orc_nearest_centre_parents(int32_t N, int d, const double *keys,
 
 /* The centroid-guided baseline on an arbitrary parent partition (the paper forms its groups by
  * k-means): one group per parent, members in increasing token index, routing key = arithmetic
- * mean of the parent's keys (fp64 sum in token order, one division), stored as a bf16 value
- * (fp64 -> fp32 to nearest -> bf16 to nearest even) and widened back into out_mean[n_parents][d]. */
+ * mean of the parent's keys (fp64 sum in token order, one division), stored as a 16-bit value
+ * (orc_round_to_elem) and widened back into out_mean[n_parents][d]. */
 void orc_group_mean_keys_parents(int d, const double *keys, int32_t n_parents, const int32_t *parent_start,
-                                 const int32_t *parent_member, double *out_mean)
+                                 const int32_t *parent_member, int half, double *out_mean)
 {
     for (int32_t u = 0; u < n_parents; ++u) {
         int32_t lo = parent_start[u], hi = parent_start[u + 1];
         for (int j = 0; j < d; ++j) {
             double sum = 0.0;
             for (int32_t a = lo; a < hi; ++a) sum += keys[(int64_t)parent_member[a] * d + j];
-            float f = (float)(sum / (double)(hi - lo));
-            uint32_t bits;
-            memcpy(&bits, &f, sizeof bits);
-            uint32_t rounded = (bits + 0x7FFFu + ((bits >> 16) & 1u)) & 0xFFFF0000u;
-            float back;
-            memcpy(&back, &rounded, sizeof back);
-            out_mean[(int64_t)u * d + j] = (double)back;
+            out_mean[(int64_t)u * d + j] = orc_round_to_elem(sum / (double)(hi - lo), half);
         }
     }
 }

@@ -83,9 +83,11 @@ def lib():
         L.orc_dense_kv_bytes.restype = _c.c_double
         L.orc_routing_kl.argtypes = [_c.c_int, _f64p, _c.c_int64, _f64p, _c.c_int32, _i32p, _i32p, _f64p, _c.c_double]
         L.orc_routing_kl.restype = _c.c_double
-        L.orc_group_mean_keys.argtypes = [_c.c_int32, _c.c_int, _f64p, _c.c_int32, _f64p]
+        L.orc_group_mean_keys.argtypes = [_c.c_int32, _c.c_int, _f64p, _c.c_int32, _c.c_int, _f64p]
+        L.orc_round_to_elem.argtypes = [_c.c_double, _c.c_int]
+        L.orc_round_to_elem.restype = _c.c_double
         L.orc_group_mean_keys.restype = _c.c_int32
-        L.orc_group_mean_keys_parents.argtypes = [_c.c_int, _f64p, _c.c_int32, _i32p, _i32p, _f64p]
+        L.orc_group_mean_keys_parents.argtypes = [_c.c_int, _f64p, _c.c_int32, _i32p, _i32p, _c.c_int, _f64p]
         L.orc_group_mean_keys_parents.restype = None
         L.orc_mla_logical_access_pct.argtypes = [_c.c_int64, _i64p, _i64p, _i64p]
         L.orc_mla_logical_access_pct.restype = _c.c_double
@@ -325,15 +327,20 @@ def routing_kl(q, k, team_start, team_member, rep_key, scale):
                                       team_member, rep_key, scale))
 
 
-def group_mean_keys(keys, P):
+def round_to_elem(x, elem="bf16"):
+    """fp64 -> fp32 -> the 16-bit element type (round to nearest even), as a float64 value."""
+    return float(lib().orc_round_to_elem(float(x), 1 if elem == "fp16" else 0))
+
+
+def group_mean_keys(keys, P, elem="bf16"):
     """Centroid-guided baseline on contiguous parents: (team_start, team_member, mean_key) with one
     group per parent, members in token order, and the parent's arithmetic-mean key rounded to a
-    bf16 value as its routing key."""
+    value of the 16-bit element type as its routing key."""
     keys = _f64(keys)
     N, d = keys.shape
     n_parents = (N + P - 1) // P
     mean = np.zeros((n_parents, d))
-    got = lib().orc_group_mean_keys(N, d, keys, P, mean)
+    got = lib().orc_group_mean_keys(N, d, keys, P, 1 if elem == "fp16" else 0, mean)
     assert got == n_parents
     return contiguous_parents(N, P), np.arange(N, dtype=np.int32), mean
 
@@ -356,14 +363,15 @@ def nearest_centre_parents(keys, centres):
     return label, parent_start[: n + 1].copy(), parent_member
 
 
-def group_mean_keys_parents(keys, parent_start, parent_member):
+def group_mean_keys_parents(keys, parent_start, parent_member, elem="bf16"):
     """Centroid-guided groups on a given partition: (team_start, team_member, mean_key), one group
-    per parent, members in token order, the mean key rounded to a bf16 value."""
+    per parent, members in token order, the mean key rounded to a value of the 16-bit element type."""
     keys = _f64(keys)
     parent_start, parent_member = _i32(parent_start), _i32(parent_member)
     n = parent_start.shape[0] - 1
     mean = np.zeros((n, keys.shape[1]))
-    lib().orc_group_mean_keys_parents(keys.shape[1], keys, n, parent_start, parent_member, mean)
+    lib().orc_group_mean_keys_parents(keys.shape[1], keys, n, parent_start, parent_member,
+                                      1 if elem == "fp16" else 0, mean)
     return parent_start.copy(), parent_member.copy(), mean
 
 

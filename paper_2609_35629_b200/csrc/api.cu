@@ -477,7 +477,6 @@ int santapp_build_groups_mean_parents(const santapp_geom *geom, const int32_t *p
                                       size_t workspace_bytes, santapp_stream stream)
 {
     if (geom && geom->reps_per_parent != 1) return SANTAPP_ERR_INVALID_ARG;    // one group per parent
-    if (geom && geom->elem_type != SANTAPP_BF16) return SANTAPP_ERR_UNSUPPORTED;
     return build_parent_records(geom, prompt_len_host, n_parents_host, k_prompt, v_prompt, parent_of, teams, workspace,
                                 workspace_bytes, stream, true);
 }
@@ -647,7 +646,6 @@ int santapp_build_groups_mean(const santapp_geom *geom, const int32_t *prompt_le
                               santapp_stream stream)
 {
     if (geom && geom->reps_per_parent != 1) return SANTAPP_ERR_INVALID_ARG;    // one group per parent
-    if (geom && geom->elem_type != SANTAPP_BF16) return SANTAPP_ERR_UNSUPPORTED;
     return build_records(geom, prompt_len_host, k_prompt, v_prompt, teams, workspace, workspace_bytes, stream, true);
 }
 

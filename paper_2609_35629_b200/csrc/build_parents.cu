@@ -236,18 +236,15 @@ build_parent_general_kernel(ParentBuildParams p)
     __syncthreads();
 
     if (p.mean_keys) {
-        // centroid-guided baseline: the parent is one group, routed by its mean stored as bf16
-        // (fp64 -> fp32 to nearest, fp32 -> bf16 to nearest even)
+        // centroid-guided baseline: the parent is one group, routed by its mean stored as a 16-bit
+        // element (fp64 -> fp32 to nearest, fp32 -> bf16 or fp16 to nearest even)
         const int tb = p.parent_team_base[(size_t)j * p.labels_total + l0 + u_parent];
         const int64_t t0 = p.bv.seq_team_off[b];
         int32_t *tof = p.team_of + plane;
         for (int i = tid; i < nC; i += kThreads) tof[mem[i]] = tb;
         if (tid == 0) p.team_row_start[(size_t)j * (p.bv.teams_total + p.bv.n_seqs) + t0 + b + 1 + tb] = nC;
-        if (tid < kHeadDim) {
-            const uint32_t bits = __float_as_uint(__double2float_rn(mu[tid]));
-            p.rep_keys[((size_t)j * p.bv.teams_total + t0 + tb) * kHeadDim + tid] =
-                (uint16_t)((bits + 0x7FFFu + ((bits >> 16) & 1u)) >> 16);
-        }
+        if (tid < kHeadDim)
+            p.rep_keys[((size_t)j * p.bv.teams_total + t0 + tb) * kHeadDim + tid] = double_to_elem<kHalf>(mu[tid]);
         return;
     }
 

@@ -220,8 +220,9 @@ size_t build_parent_smem(int P)
 // Centroid-guided baseline of the paper's routing diagnostic, on the contiguous parents of
 // Algorithm 4: one group per parent, routed by the arithmetic mean of its keys. A block per
 // (parent, sequence, KV head), a thread per dimension: the mean is the fp64 sum in token order
-// divided by the count, stored like every routing key as bf16 (fp64 -> fp32 to nearest, then
-// fp32 -> bf16 to nearest even). Rows keep their token order, so the packed copies are copies.
+// divided by the count, stored like every routing key as a 16-bit element (fp64 -> fp32 to nearest,
+// then fp32 -> bf16 or fp16 to nearest even). Rows keep their token order, so the packed copies are copies.
+template <bool kHalf>
 __global__ void __launch_bounds__(kHeadDim)
 group_mean_kernel(BuildParams p)
 {
@@ -234,12 +235,10 @@ group_mean_kernel(BuildParams p)
     const size_t plane = (size_t)j * p.bv.rows_total + (size_t)row0;
     const uint16_t *k = p.k_prompt + plane * kHeadDim;
     double sum = 0.0;
-    for (int i = lo; i < hi; ++i) sum = __dadd_rn(sum, bf16_to_double(k[(size_t)i * kHeadDim + d]));
-    const float f = __double2float_rn(__ddiv_rn(sum, (double)(hi - lo)));
-    const uint32_t bits = __float_as_uint(f);
+    for (int i = lo; i < hi; ++i) sum = __dadd_rn(sum, elem_to_double<kHalf>(k[(size_t)i * kHeadDim + d]));
     const int64_t team0 = p.bv.seq_team_off[b];                     // one team per parent
     p.rep_keys[((size_t)j * p.bv.teams_total + (size_t)team0 + parent) * kHeadDim + d] =
-        (uint16_t)((bits + 0x7FFFu + ((bits >> 16) & 1u)) >> 16);
+        double_to_elem<kHalf>(__ddiv_rn(sum, (double)(hi - lo)));
     int32_t *csr = p.team_row_start + (size_t)j * (p.bv.teams_total + p.bv.n_seqs) + team0 + b;
     if (d == 0) {
         csr[parent] = lo;
@@ -262,7 +261,8 @@ group_mean_kernel(BuildParams p)
 cudaError_t launch_build_groups_mean(const BuildParams &p, cudaStream_t s)
 {
     dim3 grid(p.max_parents_per_seq, p.bv.n_seqs, p.bv.n_kv);
-    group_mean_kernel<<<grid, kHeadDim, 0, s>>>(p);
+    if (p.bv.elem) group_mean_kernel<true><<<grid, kHeadDim, 0, s>>>(p);
+    else           group_mean_kernel<false><<<grid, kHeadDim, 0, s>>>(p);
     return cudaGetLastError();
 }
 

@@ -270,6 +270,15 @@ __device__ __forceinline__ float elem_hi(uint32_t w)
 }
 template <bool kHalf>
 __device__ __forceinline__ double elem_to_double(uint16_t b) { return (double)elem_to_float<kHalf>(b); }
+// fp64 -> fp32 (to nearest) -> the 16-bit element type (to nearest even): how a computed routing key is stored.
+template <bool kHalf>
+__device__ __forceinline__ uint16_t double_to_elem(double v)
+{
+    const float f = __double2float_rn(v);
+    if constexpr (kHalf) return __half_as_ushort(__float2half_rn(f));
+    const uint32_t bits = __float_as_uint(f);
+    return (uint16_t)((bits + 0x7FFFu + ((bits >> 16) & 1u)) >> 16);
+}
 
 // Philox4x32-10: 128-bit counter, 64-bit key, four 32-bit words.
 __device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint32_t k0, uint32_t k1)

@@ -107,3 +107,41 @@ def test_fp16_weights_far_below_the_fp16_range_still_count():
     v100 = synth.to_f64(data.v_prompt[0, 100], "fp16")
     assert np.abs(ref[0] - v100).max() > 2 * DENSE_TOL * vmax       # the small weights matter at this tolerance
     assert np.abs(out[0] - ref).max() <= DENSE_TOL * vmax
+
+
+def test_fp16_centroid_groups_contiguous_and_on_labels():
+    """The centroid-guided baseline with fp16 inputs: the mean key is rounded to fp16, records equal the
+    oracle's, and a decode step on them matches."""
+    import dataclasses
+    import torch
+    spec = dataclasses.replace(synth.spec_small_gqa(prompt=(1024, 700)), parent_size=16, reps_per_parent=1,
+                               n_sample=12, elem="fp16")
+    data = synth.make_layer(spec)
+    layer = pu.GpuLayer(spec, data, builder=sp.santapp_build_groups_mean)
+    for b in range(spec.n_seqs):
+        r0, r1 = int(layer.seq_row_off[b]), int(layer.seq_row_off[b + 1])
+        for j in range(spec.n_kv_heads):
+            keys = synth.to_f64(data.k_prompt[j, r0:r1], "fp16")
+            ts_o, tm_o, mean_o = orc.group_mean_keys(keys, spec.parent_size, elem="fp16")
+            ts_g, tm_g, rep_g = layer.records(b, j)
+            assert np.array_equal(ts_g, ts_o) and np.array_equal(tm_g, tm_o) and np.array_equal(rep_g, mean_o)
+    check_sparse_step(layer, 0, K=12)
+    # the same on a random partition per KV head
+    rng = np.random.default_rng(3)
+    n_parents = [50, 33]
+    labels = np.concatenate([rng.integers(0, p, size=(spec.n_kv_heads, n)) for p, n in zip(n_parents, spec.prompt_len)],
+                            axis=1).astype(np.int32)
+    lab_dev = torch.from_numpy(labels).cuda()
+    layer2 = pu.GpuLayer(spec, data, builder=lambda g, n, k, v: sp.santapp_build_groups_mean_parents(g, n, n_parents, k, v, lab_dev))
+    for b in range(spec.n_seqs):
+        r0, r1 = int(layer2.seq_row_off[b]), int(layer2.seq_row_off[b + 1])
+        for j in range(spec.n_kv_heads):
+            keys = synth.to_f64(data.k_prompt[j, r0:r1], "fp16")
+            lab = labels[j, r0:r1]
+            kept = np.unique(lab)
+            ps = np.concatenate([[0], np.cumsum([np.count_nonzero(lab == u) for u in kept])]).astype(np.int32)
+            pm = np.concatenate([np.flatnonzero(lab == u) for u in kept]).astype(np.int32)
+            ts_o, tm_o, mean_o = orc.group_mean_keys_parents(keys, ps, pm, elem="fp16")
+            ts_g, tm_g, rep_g = layer2.records(b, j)
+            assert np.array_equal(ts_g, ts_o) and np.array_equal(tm_g, tm_o) and np.array_equal(rep_g, mean_o)
+    check_sparse_step(layer2, 1, K=12)

@@ -72,3 +72,35 @@ def test_arbitrary_partition_hand_worked_and_rounded():
     want = synth.bf16_to_f64(synth.f32_to_bf16_bits(np.array([14.0 / 3.0, 140.0 / 3.0], dtype=np.float32)))
     assert np.array_equal(mean[1], want)
     assert mean[1, 0] == 4.65625 and mean[1, 1] == 46.75           # nearest bf16 values, by hand
+
+
+def test_rounding_to_fp16_matches_the_library_conversion():
+    """fp64 -> fp32 -> binary16 against numpy's conversions on random values of every magnitude,
+    exact ties, subnormals, the overflow threshold, signed zeros and infinities."""
+    rng = np.random.default_rng(9)
+    xs = np.concatenate([
+        rng.standard_normal(4000) * np.exp(rng.uniform(-20, 12, size=4000)),
+        np.array([0.0, -0.0, 1.0, 1.0 + 2.0 ** -11, 1.0 + 3 * 2.0 ** -11, 2.0 ** -14, 2.0 ** -24, 2.0 ** -25,
+                  1.5 * 2.0 ** -25, 2.0 ** -26, 65504.0, 65519.99, 65520.0, 70000.0, -65520.0, np.inf, -np.inf,
+                  6.1e-5, 5.97e-8, 3.0e-8, 2.98e-8]),
+    ])
+    with np.errstate(over="ignore"):
+        want = xs.astype(np.float32).astype(np.float16).astype(np.float64)
+    got = np.array([orc.round_to_elem(x, "fp16") for x in xs])
+    assert np.array_equal(got, want)
+    assert np.array_equal(np.signbit(got), np.signbit(want))
+    # and bf16 against the generators' helper
+    want_b = synth.bf16_to_f64(synth.f32_to_bf16_bits(xs[np.isfinite(xs)].astype(np.float32)))
+    got_b = np.array([orc.round_to_elem(x, "bf16") for x in xs[np.isfinite(xs)]])
+    assert np.array_equal(got_b, want_b)
+
+
+def test_fp16_mean_keys():
+    rng = np.random.default_rng(10)
+    k = synth.to_f64(synth.round_bits(rng.normal(size=(30, 8)).astype(np.float32), "fp16"), "fp16")
+    ts, _, mean = orc.group_mean_keys(k, 7, elem="fp16")
+    for u in range(len(ts) - 1):
+        exact = k[ts[u]:ts[u + 1]].mean(axis=0)
+        assert np.array_equal(mean[u], exact.astype(np.float32).astype(np.float16).astype(np.float64))
+    _, _, mean2 = orc.group_mean_keys_parents(k, ts, np.arange(30, dtype=np.int32), elem="fp16")
+    assert np.array_equal(mean, mean2)
