@@ -65,3 +65,29 @@ def test_random_configuration(case):
     step = int(rng.integers(0, 3))
     check_sparse_step(layer, step, K, seed=int(rng.integers(1 << 62)), stream_base=int(rng.integers(1 << 20)))
     check_dense_step(layer, step)
+
+
+@pytest.mark.parametrize("case", range(40))
+def test_random_batches_of_many_short_sequences(case):
+    """Many (sequence, KV head) pairs per call: the read plans live in global memory and the rows of
+    all pairs are cut into equal ranges, one per CTA, so CTAs cross pair boundaries all the time."""
+    rng = np.random.default_rng(7000 + case)
+    n_q, n_kv = _GROUPS[rng.integers(len(_GROUPS))]
+    P, R = _PARENTS[rng.integers(len(_PARENTS))]
+    n_seqs = int(rng.integers(8, 49))
+    hi = int(rng.choice([6, 60, 400, 1500]))
+    prompt = [int(rng.integers(1, hi + 1)) for _ in range(n_seqs)]
+    cap = int(rng.choice([0, 3, 16]))
+    spec = synth.WorkloadSpec("fuzz_many", n_seqs, n_q, n_kv, prompt, int(rng.integers(2, 20)), P, R,
+                              int(rng.choice([1, 3, 8, 31, 64])), 2, max(cap, 1),
+                              [int(rng.integers(0, cap + 1)) for _ in range(n_seqs)], 1, seed=int(rng.integers(1 << 30)))
+    spec.elem = "fp16" if case % 2 else "bf16"
+    G = n_q // n_kv
+    slots = max(sum(min(R, min(P, n - s)) for s in range(0, n, P)) for n in prompt)
+    K = spec.n_sample
+    if G * min(K, slots) > 1024:
+        K = spec.n_sample = max(1, 1024 // G)
+    layer = pu.GpuLayer(spec, synth.make_layer(spec, layer=0))
+    check_team_records(layer, seqs=[0, n_seqs - 1])
+    check_sparse_step(layer, 1, K, seed=int(rng.integers(1 << 62)))
+    check_dense_step(layer, 0)
