@@ -60,7 +60,8 @@ def parse_args():
     ap.add_argument("--elem", default="bf16", choices=["bf16", "fp16"], help="16-bit element type of q, K, V")
     ap.add_argument("--parents", default="contiguous", choices=["contiguous", "centres", "kmeans"],
                     help="contiguous: Algorithm 4; kmeans: Algorithm 3 with the paper's settings (fit on the GPU); "
-                         "centres: Algorithm 3 with the fit replaced by the centres the synthetic keys were drawn around")
+                         "centres: Algorithm 3 without the fit, on the first of the centres the synthetic keys were "
+                         "drawn around (uneven parents; not a model of a converged fit)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-stages", action="store_true")
