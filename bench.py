@@ -244,6 +244,18 @@ def run_ours(args):
                     "achieved_frac_of_peak", "dense_achieved_frac_of_peak", "roofline", "stage_us", "paired_rounds",
                     "steps", "warmup")
             line["batched"] = {"workload": big["config"]["workload"], **{k: big[k] for k in keep}}
+        # and the headline workload with the parents of the paper's headline runs: Algorithm 3
+        # (minibatch k-means with the paper's settings, fitted by the library), four layers
+        if args.parents == "contiguous" and args.elem == "bf16":
+            gc.collect()
+            torch.cuda.empty_cache()
+            km_args = argparse.Namespace(**{**vars(args), "parents": "kmeans"})
+            km = measure_workload(km_args, args.workload, 4, 40, 5, dev, want_e2e=False, want_cpu=False, want_stages=True)
+            if rank == 0:
+                keep = ("value", "unit", "dense_us_per_layer_step", "speedup_vs_dense", "read_reduction",
+                        "logical_access_pct", "roofline", "stage_us", "paired_rounds", "team_build_ms_last_layer",
+                        "steps", "warmup")
+                line["kmeans_parents"] = {"workload": km["config"]["workload"], **{k: km[k] for k in keep}}
     if rank == 0:
         print(json.dumps(line), flush=True)
     if world > 1:
