@@ -238,7 +238,9 @@ int32_t santapp_kmeans_parent_count(int32_t prompt_len, int32_t parent_size);
  *   workspace        device, >= santapp_kmeans_fit_workspace_bytes(...)
  * batch_size > 4096, or an initialisation sample above 28672 keys (more than 9557 centres in a
  * sequence): SANTAPP_ERR_UNSUPPORTED. The call enqueues a few kernels per centre and per
- * step on `stream`; it does not synchronise.
+ * step on `stream`, and every 16 steps waits for the stream to learn whether any fit is still
+ * running (most stop long before the step limit): it blocks the calling thread for most of the
+ * fit and must not be issued during a stream capture.
  */
 typedef struct santapp_kmeans_opts {
     int32_t batch_size;           /* paper: 4096 */

@@ -488,7 +488,7 @@ namespace {
 constexpr int kKmeansMaxSample = 28672;     // 224 KB of fp64 running sums: up to 9557 centres per sequence
 
 struct KmeansLayout {
-    size_t row_off, cen_off, tabs, perm, closest, cand, pick, centres64, count, idx, label, dist, state, total;
+    size_t row_off, cen_off, tabs, perm, closest, cand, pick, centres64, count, idx, label, dist, state, active, total;
     int k_max, n_init_max, trials_max, t_max_max, max_rows;
     int64_t rows_total, centres_total;
 };
@@ -542,6 +542,7 @@ int kmeans_layout(const santapp_geom *geom, const int32_t *prompt_len_host, cons
     L->label = take(sizeof(int32_t) * pairs * (size_t)o->batch_size);
     L->dist = take(sizeof(double) * pairs * (size_t)o->batch_size);
     L->state = take(sizeof(KmeansState) * pairs);
+    L->active = take(sizeof(int));
     L->total = off;
     return SANTAPP_OK;
 }
@@ -625,6 +626,7 @@ int santapp_kmeans_fit(const santapp_geom *geom, const int32_t *prompt_len_host,
     p.label = reinterpret_cast<int32_t *>(ws + L.label);
     p.dist = reinterpret_cast<double *>(ws + L.dist);
     p.state = reinterpret_cast<KmeansState *>(ws + L.state);
+    p.active = reinterpret_cast<int *>(ws + L.active);
     err = launch_kmeans_fit(p, s);
     if (err != cudaSuccess) return cuda_fail(err, "kmeans_fit launch");
     return SANTAPP_OK;

@@ -238,6 +238,7 @@ struct KmeansParams {
     int32_t *idx, *label;                   // [pairs][batch]
     double *dist;                           // [pairs][batch]
     KmeansState *state;                     // [pairs]
+    int *active;                            // [1] fits that still have steps to run
 };
 cudaError_t launch_kmeans_fit(const KmeansParams &p, cudaStream_t s);
 

@@ -19,6 +19,7 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kTile = 16;                 // centres staged per shared-memory tile
+constexpr int kPollEvery = 16;            // steps between two looks at the fits' stop flags
 constexpr uint32_t kTagSample = 1u, kTagStart = 2u, kTagBatch = 3u, kTagMove = 4u;
 
 struct Pair {
@@ -397,6 +398,25 @@ km_control_kernel(KmeansParams p, int t)
     }
 }
 
+// How many fits still have steps to run after step t (one block; the host reads it now and then
+// and stops enqueuing steps once it is zero).
+__global__ void __launch_bounds__(kThreads)
+km_count_active_kernel(KmeansParams p, int t)
+{
+    __shared__ int n_s;
+    if (threadIdx.x == 0) n_s = 0;
+    __syncthreads();
+    const int pairs = p.n_seqs * p.n_kv;
+    int n = 0;
+    for (int i = threadIdx.x; i < pairs; i += kThreads) {
+        const int b = i % p.n_seqs;                         // state is indexed j * n_seqs + b
+        n += (t + 1 < p.seq_t_max[b] && !p.state[i].stopped) ? 1 : 0;
+    }
+    if (n) atomicAdd(&n_s, n);
+    __syncthreads();
+    if (threadIdx.x == 0) *p.active = n_s;
+}
+
 __global__ void __launch_bounds__(kThreads)
 km_finish_kernel(KmeansParams p)
 {
@@ -442,6 +462,16 @@ cudaError_t run_fit(const KmeansParams &p, cudaStream_t s)
         KM_CHECK();
         km_control_kernel<kHalf><<<dim3(B, H), 32, control_smem, s>>>(p, t);
         KM_CHECK();
+        if ((t + 1) % kPollEvery == 0 && t + 1 < p.t_max_max) {
+            // most fits stop long before the step limit: ask the device how many are still running
+            // (the copy into pageable memory returns when it has completed)
+            int active = 1;
+            km_count_active_kernel<<<1, kThreads, 0, s>>>(p, t);
+            KM_CHECK();
+            if ((err = cudaMemcpyAsync(&active, p.active, sizeof(int), cudaMemcpyDeviceToHost, s)) != cudaSuccess) return err;
+            if ((err = cudaStreamSynchronize(s)) != cudaSuccess) return err;
+            if (active == 0) break;
+        }
     }
     km_finish_kernel<<<dim3((p.k_max * kHeadDim + kThreads - 1) / kThreads, B, H), kThreads, 0, s>>>(p);
     KM_CHECK();
