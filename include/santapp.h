@@ -139,7 +139,13 @@ typedef struct santapp_debug {
                                   comparable routing scores (non-finite q or keys): its sample was
                                   completed with arbitrary teams, the output is meaningless;
                                   bit 2: a bounded wait for an asynchronous copy expired in the
-                                  scorer (never expected; the step's result is not valid)           */
+                                  scorer (never expected; the step's result is not valid).
+                                  Cleared by the call itself before its first kernel                */
+    uint64_t *trace;           /* uint64 [5][256][16] or NULL: device-timer readings (ns) that thread 0
+                                  of the first 256 blocks of each kernel of the call notes at fixed
+                                  points, [kernel][block][mark]; kernels in launch order: scoring,
+                                  sampling, read plans, attention, merge. For latency breakdowns;
+                                  not a stable interface                                             */
 } santapp_debug;
 
 /* Library version: major * 10000 + minor * 100 + patch. */
@@ -339,7 +345,7 @@ size_t santapp_decode_workspace_bytes(const santapp_geom *geom, const santapp_te
  *   suffix_len_dev  device int32 [n_seqs], in: visible suffix rows per sequence (clamped to
  *                   [0, suffix_cap]); NULL means 0 everywhere
  *   n_sample        1 <= K <= 128, and (query heads per KV head) * min(K, M_b) <= 1024
- *                   (SANTAPP_ERR_UNSUPPORTED beyond; likewise for more than 65536 (sequence, KV
+ *                   (SANTAPP_ERR_UNSUPPORTED beyond; likewise for more than 65535 (sequence, KV
  *                   head) pairs in one call or more than 65536 teams in a sequence)
  *   seed, step, stream_base   random-stream key and counters (see top of file)
  *   step_dev        device uint32 [1] or NULL: when given, its value is added to `step` on the

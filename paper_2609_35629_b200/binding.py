@@ -74,7 +74,7 @@ class CKmeansOpts(ctypes.Structure):
 
 class CDebug(ctypes.Structure):
     _fields_ = [("sel_idx", ctypes.c_void_p), ("sel_logc", ctypes.c_void_p), ("tau", ctypes.c_void_p),
-                ("union_rows", ctypes.c_void_p), ("status", ctypes.c_void_p)]
+                ("union_rows", ctypes.c_void_p), ("status", ctypes.c_void_p), ("trace", ctypes.c_void_p)]
 
 
 _lib = None
@@ -361,15 +361,17 @@ def santapp_dense_workspace_bytes(geom: Geometry, teams: Teams) -> int:
 class DebugBuffers:
     """Optional per-step diagnostics (device tensors)."""
 
-    def __init__(self, geom: Geometry, n_sample: int, device):
+    def __init__(self, geom: Geometry, n_sample: int, device, trace: bool = False):
         B, Hq, Hkv = geom.n_seqs, geom.n_q_heads, geom.n_kv_heads
+        self.trace = torch.zeros((5, 256, 16), dtype=torch.int64, device=device) if trace else None
         self.sel_idx = torch.full((B, Hq, n_sample), -1, dtype=torch.int32, device=device)
         self.sel_logc = torch.zeros((B, Hq, n_sample), dtype=torch.float32, device=device)
         self.tau = torch.zeros((B, Hq), dtype=torch.float64, device=device)
         self.union_rows = torch.zeros((B, Hkv), dtype=torch.int32, device=device)
         self.status = torch.zeros(1, dtype=torch.int32, device=device)
         self.c = CDebug(self.sel_idx.data_ptr(), self.sel_logc.data_ptr(), self.tau.data_ptr(),
-                        self.union_rows.data_ptr(), self.status.data_ptr())
+                        self.union_rows.data_ptr(), self.status.data_ptr(),
+                        self.trace.data_ptr() if trace else None)
 
 
 def santapp_decode_attn(geom: Geometry, teams: Teams, q: torch.Tensor, k_suffix: Optional[torch.Tensor],

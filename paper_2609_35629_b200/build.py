@@ -7,7 +7,8 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 SOURCES = ["api.cu", "build_teams.cu", "build_parents.cu", "kmeans.cu", "score.cu", "headplan.cu", "plan.cu", "attend.cu"]
-HEADERS = [os.path.join(CSRC, "common.cuh"), os.path.join(CSRC, "pairplan.cuh"), os.path.join(CSRC, "build_util.cuh"), os.path.join(ROOT, "include", "santapp.h")]
+HEADERS = [os.path.join(CSRC, h) for h in ("common.cuh", "pairplan.cuh", "headplan.cuh", "score_tile.cuh", "build_util.cuh")] \
+    + [os.path.join(ROOT, "include", "santapp.h")]
 OUT = os.path.join(HERE, "libsantapp.so")
 
 
@@ -27,6 +28,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
     cmd = [_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
            "-Xcompiler", "-fPIC", "-shared", "-I", os.path.join(ROOT, "include"), "-I", CSRC,
            "-o", OUT] + srcs
+    if os.environ.get("SANTAPP_TUNE"):
+        cmd.insert(1, "-DSANTAPP_TUNE")
     if verbose:
         cmd.insert(1, "-Xptxas")
         cmd.insert(2, "-v")

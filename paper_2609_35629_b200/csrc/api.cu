@@ -1,6 +1,7 @@
 // C ABI of the SANTA++ decode-attention library: argument checks, workspace carving, launches.
 #include <math.h>
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <mutex>
@@ -83,8 +84,9 @@ BatchView make_view(const santapp_geom *g, const santapp_teams *t)
 
 // Workspace layout shared by the sparse and the dense call. Offsets in bytes.
 struct DecodeLayout {
-    size_t ctl, y32, ymax, sel_team, sel_logc, sel_rows, seg_prefix, seg_row, seg_mask, seg_logc, pair_nseg, pair_rows, pair_prefix, partials, total;
-    int seg_cap, grid, n_pairs, ctas_per_pair, ymax_stride;
+    size_t y32, sel_team, sel_logc, sel_rows, seg_prefix, seg_row, seg_mask, seg_logc, pair_nseg, pair_rows, pair_prefix, partials, total;
+    int seg_cap, grid, n_pairs, ctas_per_pair, tile_stride;
+    int64_t y_stride;
     bool static_split;
 };
 
@@ -103,10 +105,9 @@ DecodeLayout decode_layout(const santapp_geom *g, const santapp_teams *t, int K,
     L.seg_cap = (int)cap + 1;                                   // + the suffix segment
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
-    L.ctl = take(sizeof(int32_t) * ((size_t)L.n_pairs + 2));
-    L.y32 = take(dense ? 0 : sizeof(float) * (size_t)g->n_q_heads * (size_t)t->teams_total);
-    L.ymax_stride = (int)(t->teams_total / 16 + g->n_seqs + 1);
-    L.ymax = take(dense ? 0 : sizeof(float) * (size_t)g->n_q_heads * (size_t)L.ymax_stride);
+    L.y_stride = score_row_stride(t->max_teams_per_seq);
+    L.y32 = take(dense ? 0 : sizeof(float) * (size_t)g->n_q_heads * (size_t)g->n_seqs * (size_t)L.y_stride);
+    L.tile_stride = (int)(t->teams_total / 16 + g->n_seqs + 1);
     L.sel_team = take(dense ? 0 : sizeof(int32_t) * (size_t)g->n_seqs * g->n_q_heads * K);
     L.sel_logc = take(dense ? 0 : sizeof(float) * (size_t)g->n_seqs * g->n_q_heads * K);
     L.sel_rows = take(dense ? 0 : sizeof(int2) * (size_t)g->n_seqs * g->n_q_heads * K);
@@ -122,11 +123,8 @@ DecodeLayout decode_layout(const santapp_geom *g, const santapp_teams *t, int K,
     return L;
 }
 
-void fill_plan(const DecodeLayout &L, char *ws, PlanView &plan, Control &ctl)
+void fill_plan(const DecodeLayout &L, char *ws, PlanView &plan)
 {
-    int32_t *c = reinterpret_cast<int32_t *>(ws + L.ctl);
-    ctl.attend_ticket = c;
-    ctl.plan_ticket = c + L.n_pairs;
     plan.seg_cap = L.seg_cap;
     plan.seg_prefix = reinterpret_cast<int32_t *>(ws + L.seg_prefix);
     plan.seg_row = reinterpret_cast<int32_t *>(ws + L.seg_row);
@@ -692,8 +690,7 @@ int santapp_decode_attn(const santapp_geom *geom, const santapp_teams *teams, co
     const double sc = scale == 0.f ? 1.0 / sqrt((double)geom->head_dim) : (double)scale;
 
     PlanView plan;
-    Control ctl;
-    fill_plan(L, ws, plan, ctl);
+    fill_plan(L, ws, plan);
 
     ScoreParams rp;
     rp.bv = make_view(geom, teams);
@@ -701,8 +698,8 @@ int santapp_decode_attn(const santapp_geom *geom, const santapp_teams *teams, co
     rp.team_row_start = teams->team_row_start;
     rp.q = static_cast<const uint16_t *>(q);
     rp.y32 = reinterpret_cast<float *>(ws + L.y32);
-    rp.ymax = reinterpret_cast<float *>(ws + L.ymax);
-    rp.ymax_stride = L.ymax_stride;
+    rp.y_stride = L.y_stride;
+    rp.tile_stride = L.tile_stride;
     rp.n_sample = n_sample;
     rp.seed_lo = (uint32_t)(seed & 0xFFFFFFFFull);
     rp.seed_hi = (uint32_t)(seed >> 32);
@@ -710,10 +707,15 @@ int santapp_decode_attn(const santapp_geom *geom, const santapp_teams *teams, co
     rp.step_dev = step_dev;
     rp.stream_base = stream_base;
     rp.scale = sc;
-    rp.ctl = ctl;
     rp.n_pairs = L.n_pairs;
     rp.status = dbg ? dbg->status : nullptr;
+    rp.trace = dbg ? reinterpret_cast<unsigned long long *>(dbg->trace) : nullptr;
     cudaError_t err = cudaSuccess;
+    if (rp.status && g_stage_mask == SANTAPP_STAGE_ALL) {
+        // diagnostics only: a node of its own, so that no kernel both clears and raises the flags
+        err = cudaMemsetAsync(rp.status, 0, sizeof(int32_t), s);
+        if (err != cudaSuccess) return cuda_fail(err, "status memset");
+    }
     if (g_stage_mask & SANTAPP_STAGE_ROUTE) {
         err = launch_score32(rp, teams->max_teams_per_seq, s);
         if (err != cudaSuccess) return cuda_fail(err, "score launch");
@@ -723,8 +725,7 @@ int santapp_decode_attn(const santapp_geom *geom, const santapp_teams *teams, co
     PlanParams pp;
     pp.in.bv = rp.bv;
     pp.in.y32 = rp.y32;
-    pp.in.ymax = rp.ymax;
-    pp.in.ymax_stride = L.ymax_stride;
+    pp.in.y_stride = L.y_stride;
     pp.in.rep_keys = rp.rep_keys;
     pp.in.team_row_start = teams->team_row_start;
     pp.in.rep_abs_max = teams->rep_abs_max;
@@ -746,18 +747,24 @@ int santapp_decode_attn(const santapp_geom *geom, const santapp_teams *teams, co
     pp.in.dbg_sel_logc = dbg ? dbg->sel_logc : nullptr;
     pp.in.dbg_tau = dbg ? dbg->tau : nullptr;
     pp.in.dbg_union_rows = dbg ? dbg->union_rows : nullptr;
+    pp.in.trace = rp.trace;
     pp.plan = plan;
-    pp.ctl = ctl;
     pp.n_pairs = L.n_pairs;
     if (g_stage_mask & SANTAPP_STAGE_SELECT) {
         err = launch_headplan(pp.in, s);
         if (err != cudaSuccess) return cuda_fail(err, "headplan launch");
         ++g_launches;
     }
+    // few pairs: the plan is built inside the attention kernel (fixed CTAs per pair)
     if (!L.static_split && (g_stage_mask & SANTAPP_STAGE_SELECT)) {
-        err = launch_plan(pp, s);
+        err = launch_plan(pp, teams->max_teams_per_seq, s);
         if (err != cudaSuccess) return cuda_fail(err, "plan launch");
         ++g_launches;
+        if (L.n_pairs > attend_pairs_staged()) {                // else the attention kernel sums the pairs' rows itself
+            err = launch_pair_prefix(pp, s);
+            if (err != cudaSuccess) return cuda_fail(err, "pair prefix launch");
+            ++g_launches;
+        }
     }
 
     AttendParams ap;
@@ -770,18 +777,24 @@ int santapp_decode_attn(const santapp_geom *geom, const santapp_teams *teams, co
     ap.qk_scale_log2 = (float)(sc * 1.4426950408889634);
     ap.plan = plan;
     ap.in = pp.in;
-    ap.ctl = ctl;
     ap.n_pairs = L.n_pairs;
     ap.partials = reinterpret_cast<float *>(ws + L.partials);
     ap.out = out;
     ap.status = rp.status;
     ap.min_rows_per_cta = 64;
     ap.span_penalty_rows = 640;                                 // measured: a second span costs about 8 us of one SM's bandwidth
+#ifdef SANTAPP_TUNE
+    if (const char *e = getenv("SANTAPP_SPAN_PENALTY")) ap.span_penalty_rows = atoi(e);
+#endif
     ap.ctas_per_pair = L.ctas_per_pair;
+    ap.max_words = (teams->max_teams_per_seq + 31) / 32;
     if (g_stage_mask & SANTAPP_STAGE_ATTEND) {
         const int launch_grid = L.static_split ? L.n_pairs * L.ctas_per_pair : grid;
         err = launch_attend(ap, false, L.static_split, launch_grid, s);
         if (err != cudaSuccess) return cuda_fail(err, "attend launch");
+        ++g_launches;
+        err = launch_merge(ap, L.static_split, launch_grid, s);
+        if (err != cudaSuccess) return cuda_fail(err, "merge launch");
         ++g_launches;
     }
     return SANTAPP_OK;
@@ -814,8 +827,7 @@ int santapp_dense_decode_attn(const santapp_geom *geom, const santapp_teams *tea
     const double sc = scale == 0.f ? 1.0 / sqrt((double)geom->head_dim) : (double)scale;
 
     PlanView plan;
-    Control ctl;
-    fill_plan(L, ws, plan, ctl);
+    fill_plan(L, ws, plan);
 
     PlanParams pp;
     memset(&pp, 0, sizeof(pp));
@@ -823,17 +835,17 @@ int santapp_dense_decode_attn(const santapp_geom *geom, const santapp_teams *tea
     pp.in.suffix_len = suffix_len_dev;
     pp.in.suffix_cap = suffix_cap;
     pp.plan = plan;
-    pp.ctl = ctl;
     pp.n_pairs = L.n_pairs;
     cudaError_t err;
-    if (L.static_split) {
-        // the plan is trivial and built inside the kernel; only the merge tickets need clearing
-        err = cudaMemsetAsync(ctl.attend_ticket, 0, sizeof(int32_t) * (size_t)L.n_pairs, s);
-        if (err != cudaSuccess) return cuda_fail(err, "ticket memset");
-    } else {
+    if (!L.static_split) {                                      // else the plan is trivial and built inside the kernel
         err = launch_dense_plan(pp, s);
         if (err != cudaSuccess) return cuda_fail(err, "dense_plan launch");
         ++g_launches;
+        if (L.n_pairs > attend_pairs_staged()) {
+            err = launch_pair_prefix(pp, s);
+            if (err != cudaSuccess) return cuda_fail(err, "pair prefix launch");
+            ++g_launches;
+        }
     }
 
     AttendParams ap;
@@ -846,17 +858,22 @@ int santapp_dense_decode_attn(const santapp_geom *geom, const santapp_teams *tea
     ap.qk_scale_log2 = (float)(sc * 1.4426950408889634);
     ap.plan = plan;
     ap.in = pp.in;
-    ap.ctl = ctl;
     ap.n_pairs = L.n_pairs;
     ap.partials = reinterpret_cast<float *>(ws + L.partials);
     ap.out = out;
     ap.status = nullptr;
     ap.min_rows_per_cta = 64;
     ap.span_penalty_rows = 1040;                                // measured on the dense path: about 13 us
+#ifdef SANTAPP_TUNE
+    if (const char *e = getenv("SANTAPP_SPAN_PENALTY_DENSE")) ap.span_penalty_rows = atoi(e);
+#endif
     ap.ctas_per_pair = L.ctas_per_pair;
     const int launch_grid = L.static_split ? L.n_pairs * L.ctas_per_pair : grid;
     err = launch_attend(ap, true, L.static_split, launch_grid, s);
     if (err != cudaSuccess) return cuda_fail(err, "attend launch");
+    ++g_launches;
+    err = launch_merge(ap, L.static_split, launch_grid, s);
+    if (err != cudaSuccess) return cuda_fail(err, "merge launch");
     ++g_launches;
     return SANTAPP_OK;
 }

@@ -5,9 +5,10 @@
 //
 // Work split, two ways (split-K by rows, never by teams; one CTA per SM):
 //   static   a fixed number of CTAs per (sequence, KV head) pair. Every CTA of a pair first
-//            runs the pair's sampling and builds its read plan in shared memory (pairplan.cuh;
+//            builds the pair's read plan in shared memory from the heads' samples (pairplan.cuh;
 //            the dense kernel's plan is trivial), then takes its share of the pair's rows. No
-//            plan kernel, no global plan: the shortest path for few pairs.
+//            plan kernel, no global plan: the shortest path for few pairs (a kernel boundary or
+//            a counter in global memory costs about a microsecond, the redundant build less).
 //   dynamic  the rows of all pairs form one global row space cut into equal contiguous ranges;
 //            plans come from a plan kernel through global memory. Best balance for many pairs.
 // Inside a CTA each warp takes a contiguous run of 16-row blocks and streams them through a
@@ -22,9 +23,9 @@
 // selected it (mask), with the head's own correction. The weights are split into two bf16
 // terms (p = p_hi + p_lo) so that O^T += V^T P^T keeps fp32-level accuracy.
 //
-// Each CTA leaves one online-softmax partial per pair it touched; the last CTA to finish a
-// pair stages that pair's partials in shared memory and merges them by log-sum-exp (the
-// split-softmax reduction).
+// Each CTA leaves one online-softmax partial per pair it touched; a second, small kernel merges
+// every pair's partials by log-sum-exp (the split-softmax reduction). A kernel boundary costs less
+// here than any counter the CTAs of one launch could meet at, and it needs no state between calls.
 #include <math_constants.h>
 
 #include "common.cuh"
@@ -34,8 +35,8 @@ namespace santapp {
 
 namespace {
 
-constexpr int kWarps = kPlanWarps;                          // 12
-constexpr int kAttendThreads = kPlanThreads;
+constexpr int kWarps = 12;
+constexpr int kAttendThreads = kWarps * 32;
 constexpr int kBlockRows = 16;                              // rows per block (one warp, one MMA K step)
 constexpr int kSlots = 2;                                   // ring slots per warp
 constexpr int kRowBytes = kHeadDim * 2;                     // one bf16 row
@@ -116,8 +117,8 @@ struct Smem {
     static constexpr size_t seg_mask = seg_row + (kSegMax + 3) * 4;             // uint [kSegMax]
     static constexpr size_t pair_prefix = (seg_mask + (kSegMax + 3) * 4 + 15) / 16 * 16;   // int64 [kPairMax + 1]
     static constexpr size_t pair_nseg = pair_prefix + (kPairMax + 1) * 8;       // int [kPairMax]
-    static constexpr size_t misc = pair_nseg + kPairMax * 4;                    // flags
-    static constexpr size_t total = misc + 64;
+    static constexpr size_t misc = pair_nseg + kPairMax * 4;                    // flags, then scan scratch [40]
+    static constexpr size_t total = misc + 64 + 160;
     // aliases of the ring: plan scratch before a pair's rows are streamed, merge scratch after
     static_assert(sizeof(PlanScratch) <= ring_bytes, "plan scratch must fit in the ring");
     static constexpr int red_pitch = kHeadDim + 4;                              // floats per (warp, head) row: the 4 extra
@@ -126,8 +127,6 @@ struct Smem {
     static constexpr size_t red_m = red_acc + (size_t)kWarps * G * red_pitch * 4;  // float [warps][G]
     static constexpr size_t red_l = red_m + (size_t)kWarps * G * 4;
     static_assert(red_l + (size_t)kWarps * G * 4 <= ring_bytes, "merge scratch must fit in the ring");
-    static constexpr int merge_fit = (int)(ring_bytes / ((size_t)G * kPartialStride * 4));
-    static constexpr int merge_chunk = merge_fit < 64 ? merge_fit : 64;         // partials staged at once (two per lane)
     static_assert(total <= 227 * 1024, "shared memory budget");
 };
 
@@ -143,12 +142,12 @@ attend_kernel(AttendParams p)
     int64_t *pair_prefix = reinterpret_cast<int64_t *>(smem + S::pair_prefix);
     int *pair_nseg = reinterpret_cast<int *>(smem + S::pair_nseg);
     int *misc = reinterpret_cast<int *>(smem + S::misc);
-    int *last_flag = misc;
+    int *scan_scratch = misc + 16;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = lane >> 2, c = lane & 3;                 // MMA fragment coordinates
     const int hw = lane >> 4, chunk = lane & 15;           // copy coordinates: row parity, 16-byte chunk
-
+    trace_mark(p.in.trace, 3, 0);
     const uint32_t ring_w = smem_u32(smem + S::ring) + (uint32_t)warp * kSlots * kSlotBytes;
     float *logc_w = reinterpret_cast<float *>(smem + S::logc_tab) + warp * kSlots * kBlockRows * kMaxGroup;
     unsigned char *mask_w = smem + S::mask_tab + warp * kSlots * kBlockRows;
@@ -165,6 +164,27 @@ attend_kernel(AttendParams p)
         __syncthreads();
         pair_base = base;
     };
+    // Batches of at most kPairMax pairs: the row prefix over the pairs is summed here from the
+    // pairs' row counts (thread t owns pairs 2t and 2t + 1); block 0 leaves it in global memory
+    // for the merge kernel.
+    auto stage_all_pairs = [&]() {
+        static_assert(2 * kAttendThreads >= kPairMax, "two pairs per thread");
+        const int i0 = 2 * tid, i1 = 2 * tid + 1;
+        const int v0 = i0 < p.n_pairs ? __ldcg(p.plan.pair_rows + i0) : 0;
+        const int v1 = i1 < p.n_pairs ? __ldcg(p.plan.pair_rows + i1) : 0;
+        if (i0 < p.n_pairs) pair_nseg[i0] = __ldcg(p.plan.pair_nseg + i0);
+        if (i1 < p.n_pairs) pair_nseg[i1] = __ldcg(p.plan.pair_nseg + i1);
+        int total;
+        const int excl = block_exclusive_scan(v0 + v1, scan_scratch, total);
+        if (i0 <= p.n_pairs) pair_prefix[i0] = excl;
+        if (i1 <= p.n_pairs) pair_prefix[i1] = excl + v0;
+        if (blockIdx.x == 0) {
+            if (i0 <= p.n_pairs) p.plan.pair_row_prefix[i0] = excl;
+            if (i1 <= p.n_pairs) p.plan.pair_row_prefix[i1] = excl + v0;
+        }
+        __syncthreads();
+        pair_base = 0;
+    };
     int64_t r0 = 0, r1 = 0, rows_per_cta = 0;              // dynamic split: global row range
     if (kStatic) {
         pair = blockIdx.x / p.ctas_per_pair;
@@ -174,7 +194,7 @@ attend_kernel(AttendParams p)
         // pair_prefix / pair_nseg hold a window of kPairMax pairs starting at pair_base; batches of up
         // to kPairMax pairs are staged whole, before anything else is waited for
         const bool windowed = p.n_pairs > kPairMax;
-        if (!windowed) stage_pairs(0);
+        if (!windowed) stage_all_pairs();
         const int64_t all_rows = windowed ? p.plan.pair_row_prefix[p.n_pairs] : pair_prefix[p.n_pairs];
         // Rows of all pairs laid end to end, with a gap of span_penalty_rows after every pair: a CTA
         // whose range crosses from one pair into the next pays the fixed cost of a second span
@@ -198,7 +218,7 @@ attend_kernel(AttendParams p)
     }
 
     while (true) {
-        int a, bnd, nseg, n_ctas, first_slot, slot_id;
+        int a, bnd, nseg, slot_id;
         int64_t pb = 0, pe = 0;
         const int b = pair / p.bv.n_kv, j = pair - b * p.bv.n_kv;
         const float *g_logc = p.plan.seg_logc + (size_t)pair * cap * kMaxGroup;
@@ -217,7 +237,11 @@ attend_kernel(AttendParams p)
 
         if (kStatic) {
             int rows;
-            if (kAll) {
+            if (!kAll) {
+                PlanScratch &scratch = *reinterpret_cast<PlanScratch *>(smem + S::ring);
+                build_pair_plan<kAttendThreads>(p.in, pair, p.max_words, scratch, seg_prefix, seg_row, seg_mask,
+                                                p.plan.seg_logc + (size_t)pair * cap * kMaxGroup, nseg, rows, sub == 0);
+            } else {
                 __syncthreads();
                 if (tid == 0) {
                     const int64_t row0 = p.bv.seq_row_off[b];
@@ -244,22 +268,18 @@ attend_kernel(AttendParams p)
                 __syncthreads();
                 nseg = misc[2];
                 rows = misc[3];
-            } else {
-                PlanScratch &scratch = *reinterpret_cast<PlanScratch *>(smem + S::ring);
-                build_pair_plan<G>(p.in, pair, scratch, seg_prefix, seg_row, seg_mask,
-                                   p.plan.seg_logc + (size_t)pair * cap * kMaxGroup, nseg, rows, sub == 0);
             }
             const int per_cta = max((rows + p.ctas_per_pair - 1) / p.ctas_per_pair, p.min_rows_per_cta);
-            n_ctas = (rows + per_cta - 1) / per_cta;
             a = sub * per_cta;
             bnd = min(a + per_cta, rows);
-            first_slot = pair * p.ctas_per_pair;
-            slot_id = first_slot + sub;
-            if (a >= rows) {                               // more CTAs than this pair needs
-                if (p.ctas_per_pair > 1) return;
-                pair += gridDim.x;
-                if (pair >= p.n_pairs) return;
-                continue;
+            slot_id = pair * p.ctas_per_pair + sub;
+            if (a >= rows) {                               // more CTAs than this pair needs: an empty partial
+                if (tid < G) {
+                    float *part = p.partials + ((size_t)slot_id * G + tid) * kPartialStride;
+                    part[0] = -CUDART_INF_F;
+                    part[1] = 0.f;
+                }
+                return;
             }
         } else {
             // this pair's rows occupy [pb, pe) of the padded row line
@@ -275,10 +295,7 @@ attend_kernel(AttendParams p)
                 continue;
             }
             nseg = pair_nseg[pair - pair_base];
-            const int c_lo = (int)(pb / rows_per_cta), c_hi = (int)((pe - 1) / rows_per_cta);
-            n_ctas = c_hi - c_lo + 1;
-            first_slot = c_lo + pair;
-            slot_id = blockIdx.x + pair;
+            slot_id = blockIdx.x + pair;                   // CTA c's partial of pair i lives in slot c + i
             __syncthreads();                               // the previous span is done with the tables
             // one round trip: every load is issued before the first store
             const int32_t *g_prefix = p.plan.seg_prefix + (size_t)pair * (cap + 1);
@@ -295,6 +312,7 @@ attend_kernel(AttendParams p)
             }
         }
         __syncthreads();
+        trace_mark(p.in.trace, 3, 1);
 
         const unsigned char *k_plane = reinterpret_cast<const unsigned char *>(p.k_packed)
                                        + (size_t)j * p.bv.rows_total * kRowBytes;
@@ -376,6 +394,7 @@ attend_kernel(AttendParams p)
             issue(i + 1);
             cp_async_wait_group<1>();                      // block i has landed (this lane's copies)
             __syncwarp();                                  // ... and every other lane's
+            if (i == 0) trace_mark(p.in.trace, 3, 2);
             const int slot = i % kSlots;
             const uint32_t k_addr = ring_w + slot * kSlotBytes;
             const uint32_t v_addr = k_addr + kTileBytes;
@@ -453,6 +472,7 @@ attend_kernel(AttendParams p)
         }
         cp_async_wait_group<0>();
         __syncthreads();                                   // every block of the span is consumed
+        trace_mark(p.in.trace, 3, 3);
 
         // ---- merge the warps into one partial (the ring is free: reuse it) ----
         float(*red_acc)[G][S::red_pitch] = reinterpret_cast<float(*)[G][S::red_pitch]>(smem + S::red_acc);
@@ -498,95 +518,10 @@ attend_kernel(AttendParams p)
             if (lane == 0) { part[h * kPartialStride] = mh; part[h * kPartialStride + 1] = den; }
         }
 
-        // ---- last CTA of the pair: log-sum-exp merge of the pair's partials ----
-        __threadfence();
-        __syncthreads();
-        if (tid == 0) *last_flag = (atomicAdd(p.ctl.attend_ticket + pair, 1) == n_ctas - 1);
-        __syncthreads();
-        if (*last_flag) {
-            __threadfence();
-            if (tid == 0) p.ctl.attend_ticket[pair] = 0;              // every CTA of the pair has arrived
-            // The pair's partials are contiguous in memory. Stage them in shared memory a chunk
-            // at a time with asynchronous copies, then merge from there: thread (h, lane) owns
-            // four output columns of head h.
-            const float *first = p.partials + (size_t)first_slot * G * kPartialStride;
-            float *stage = reinterpret_cast<float *>(smem + S::ring);
-            constexpr int kPer = G * kPartialStride;                   // floats per partial
-            const int h = tid >> 5;
-            float m_acc = -CUDART_INF_F, l_acc = 0.f;
-            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-            for (int c0 = 0; c0 < n_ctas; c0 += S::merge_chunk) {
-                const int nc = min(S::merge_chunk, n_ctas - c0);
-                __syncthreads();                           // the previous chunk has been read
-                const int n16 = nc * kPer / 4;             // 16-byte pieces
-                const float *src = first + (size_t)c0 * kPer;
-                for (int i = tid; i < n16; i += kAttendThreads)
-                    cp_async16(smem_u32(stage + 4 * i), src + 4 * i, 16u);
-                cp_async_commit();
-                cp_async_wait_group<0>();
-                __syncthreads();
-                if (h < G) {
-                    // this warp's head: lane l holds the maxima and sums of partials l and l + 32
-                    float mv[2], lv[2];
-#pragma unroll
-                    for (int u = 0; u < 2; ++u) {
-                        const int cc = lane + 32 * u;
-                        mv[u] = cc < nc ? stage[(cc * G + h) * kPartialStride] : -CUDART_INF_F;
-                        lv[u] = cc < nc ? stage[(cc * G + h) * kPartialStride + 1] : 0.f;
-                    }
-                    float mc = fmaxf(mv[0], mv[1]);
-#pragma unroll
-                    for (int o = 16; o > 0; o >>= 1) mc = fmaxf(mc, __shfl_xor_sync(0xFFFFFFFFu, mc, o));
-                    const float m_new = fmaxf(m_acc, mc);
-                    if (m_new > -CUDART_INF_F) {
-                        const float f = m_acc > -CUDART_INF_F ? exp2f(m_acc - m_new) : 0.f;
-                        acc.x *= f; acc.y *= f; acc.z *= f; acc.w *= f;
-                        // one weight per partial, computed once and handed round by shuffle
-                        float w[2];
-#pragma unroll
-                        for (int u = 0; u < 2; ++u) w[u] = mv[u] > -CUDART_INF_F ? exp2f(mv[u] - m_new) : 0.f;
-                        float lsum = fmaf(w[0], lv[0], w[1] * lv[1]);
-#pragma unroll
-                        for (int o = 16; o > 0; o >>= 1) lsum += __shfl_xor_sync(0xFFFFFFFFu, lsum, o);
-                        l_acc = fmaf(l_acc, f, lsum);
-                        const float *col = stage + h * kPartialStride + 4 + lane * 4;
-                        const int n_lo = min(nc, 32);
-#pragma unroll 4
-                        for (int cc = 0; cc < n_lo; ++cc) {
-                            const float wgt = __shfl_sync(0xFFFFFFFFu, w[0], cc);
-                            const float4 v = *reinterpret_cast<const float4 *>(col + (size_t)cc * kPer);
-                            acc.x = fmaf(wgt, v.x, acc.x);
-                            acc.y = fmaf(wgt, v.y, acc.y);
-                            acc.z = fmaf(wgt, v.z, acc.z);
-                            acc.w = fmaf(wgt, v.w, acc.w);
-                        }
-#pragma unroll 4
-                        for (int cc = 32; cc < nc; ++cc) {
-                            const float wgt = __shfl_sync(0xFFFFFFFFu, w[1], cc - 32);
-                            const float4 v = *reinterpret_cast<const float4 *>(col + (size_t)cc * kPer);
-                            acc.x = fmaf(wgt, v.x, acc.x);
-                            acc.y = fmaf(wgt, v.y, acc.y);
-                            acc.z = fmaf(wgt, v.z, acc.z);
-                            acc.w = fmaf(wgt, v.w, acc.w);
-                        }
-                        m_acc = m_new;
-                    }
-                }
-            }
-            if (h < G) {
-                const float inv = 1.f / l_acc;
-                const float4 ov = make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
-                *reinterpret_cast<float4 *>(p.out + ((size_t)b * p.bv.n_q + (size_t)j * G + h) * kHeadDim + lane * 4) = ov;
-                if (p.status && !(isfinite(ov.x) && isfinite(ov.y) && isfinite(ov.z) && isfinite(ov.w)))
-                    atomicOr(p.status, 1);
-            }
-        }
-
         // ---- next span ----
         if (kStatic) {
-            if (p.ctas_per_pair > 1) return;
-            pair += gridDim.x;                             // more pairs than CTAs: whole pairs, round robin
-            if (pair >= p.n_pairs) return;
+            trace_mark(p.in.trace, 3, 5);
+            return;                                        // one span per CTA
         } else {
             if (pb + bnd < pe) return;                     // the range ended inside this pair
             r0 = pe + p.span_penalty_rows;                 // first row of the next pair
@@ -594,6 +529,99 @@ attend_kernel(AttendParams p)
             ++pair;
         }
     }
+}
+
+// Log-sum-exp merge of a pair's partials (the split-softmax reduction): one block per (query head
+// of the group, pair). Thread (part, lane) takes the partials part, part + kParts, ...
+// (at most kDepth of them in flight at once) for four output columns. Every step is laid out
+// for a short dependent chain: all loads first, one block-wide maximum, weights relative to it
+// (independent of each other), sums across the parts by the first four warps.
+template <int kParts, bool kStatic>
+__global__ void __launch_bounds__(kParts * 32)
+merge_kernel(AttendParams p, int attend_grid)
+{
+    __shared__ float red_m[kParts], red_l[kParts];
+    __shared__ __align__(16) float red_acc[kParts][kHeadDim];
+    const int G = p.bv.group;
+    const int h = blockIdx.x, pair = blockIdx.y;
+    const int b = pair / p.bv.n_kv, j = pair - b * p.bv.n_kv;
+    const int part = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    trace_mark(p.in.trace, 4, 0);
+    int first_slot, n;
+    if (kStatic) {
+        first_slot = pair * p.ctas_per_pair;
+        n = p.ctas_per_pair;
+    } else {
+        // the attention kernel's split: rows of all pairs end to end with a gap behind each
+        // (all below 2^32: rows_total < 2^31 and the gaps add at most 2^26 * 16)
+        const int64_t pre0 = p.plan.pair_row_prefix[pair], pre1 = p.plan.pair_row_prefix[pair + 1];
+        const int64_t all_rows = p.plan.pair_row_prefix[p.n_pairs];
+        const uint32_t total = (uint32_t)(all_rows + (int64_t)p.span_penalty_rows * (p.n_pairs - 1));
+        uint32_t rows_per_cta = (total + (uint32_t)attend_grid - 1u) / (uint32_t)attend_grid;
+        if (rows_per_cta < (uint32_t)p.min_rows_per_cta) rows_per_cta = (uint32_t)p.min_rows_per_cta;
+        const uint32_t pb = (uint32_t)(pre0 + (int64_t)p.span_penalty_rows * pair);
+        const uint32_t pe = pb + (uint32_t)(pre1 - pre0);
+        const int c_lo = (int)(pb / rows_per_cta), c_hi = (int)((max(pe, pb + 1u) - 1u) / rows_per_cta);
+        first_slot = c_lo + pair;
+        n = pe > pb ? c_hi - c_lo + 1 : 0;
+    }
+    const size_t stride = (size_t)G * kPartialStride;
+    const float *base = p.partials + ((size_t)first_slot * G + h) * kPartialStride;
+    constexpr int kDepth = 4;                              // partials a thread has in flight: one round trip for n <= 4 kParts
+    float m_run = -CUDART_INF_F, l_run = 0.f;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int i0 = part; i0 < n; i0 += kParts * kDepth) {   // one trip unless n > kDepth * kParts
+        float2 ml[kDepth];
+        float4 v[kDepth];
+#pragma unroll
+        for (int u = 0; u < kDepth; ++u) {
+            const int i = i0 + u * kParts;
+            ml[u] = make_float2(-CUDART_INF_F, 0.f);
+            v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (i < n) {
+                ml[u] = __ldcg(reinterpret_cast<const float2 *>(base + (size_t)i * stride));
+                v[u] = __ldcg(reinterpret_cast<const float4 *>(base + (size_t)i * stride + 4) + lane);
+            }
+        }
+        float m_new = m_run;
+#pragma unroll
+        for (int u = 0; u < kDepth; ++u) m_new = fmaxf(m_new, ml[u].x);
+        if (m_new > -CUDART_INF_F) {
+            const float f = exp2f(m_run - m_new);          // 0 on the first trip
+            acc.x *= f; acc.y *= f; acc.z *= f; acc.w *= f;
+            l_run *= f;
+#pragma unroll
+            for (int u = 0; u < kDepth; ++u) {
+                // a partial without rows for this head (m = -inf) holds no data
+                const float w = ml[u].x > -CUDART_INF_F ? exp2f(ml[u].x - m_new) : 0.f;
+                acc.x = fmaf(w, ml[u].x > -CUDART_INF_F ? v[u].x : 0.f, acc.x);
+                acc.y = fmaf(w, ml[u].x > -CUDART_INF_F ? v[u].y : 0.f, acc.y);
+                acc.z = fmaf(w, ml[u].x > -CUDART_INF_F ? v[u].z : 0.f, acc.z);
+                acc.w = fmaf(w, ml[u].x > -CUDART_INF_F ? v[u].w : 0.f, acc.w);
+                l_run = fmaf(w, ml[u].y, l_run);
+            }
+            m_run = m_new;
+        }
+    }
+    if (lane == 0) red_m[part] = m_run;
+    __syncthreads();
+    float m_all = -CUDART_INF_F;
+#pragma unroll
+    for (int i = 0; i < kParts; ++i) m_all = fmaxf(m_all, red_m[i]);
+    const float f = m_run > -CUDART_INF_F ? exp2f(m_run - m_all) : 0.f;
+    *reinterpret_cast<float4 *>(&red_acc[part][4 * lane]) = make_float4(acc.x * f, acc.y * f, acc.z * f, acc.w * f);
+    if (lane == 0) red_l[part] = l_run * f;
+    __syncthreads();
+    if (threadIdx.x < kHeadDim) {
+        const int d = threadIdx.x;
+        float num = 0.f, den = 0.f;
+#pragma unroll
+        for (int i = 0; i < kParts; ++i) { num += red_acc[i][d]; den += red_l[i]; }
+        const float ov = num / den;
+        p.out[((size_t)b * p.bv.n_q + (size_t)j * G + h) * kHeadDim + d] = ov;
+        if (p.status && !isfinite(ov)) atomicOr(p.status, 1);
+    }
+    trace_mark(p.in.trace, 4, 1);
 }
 
 template <int G, bool kHalf>
@@ -607,13 +635,11 @@ cudaError_t launch_attend_g(const AttendParams &p, bool all_heads, bool static_s
     cudaError_t err = ensure_dynamic_smem(fns[which], (int)smem, done[which]);
     if (err != cudaSuccess) return err;
     if (all_heads) {
-        if (static_split) attend_kernel<G, true, true, kHalf><<<grid, kAttendThreads, smem, s>>>(p);
-        else              attend_kernel<G, true, false, kHalf><<<grid, kAttendThreads, smem, s>>>(p);
-    } else {
-        if (static_split) attend_kernel<G, false, true, kHalf><<<grid, kAttendThreads, smem, s>>>(p);
-        else              attend_kernel<G, false, false, kHalf><<<grid, kAttendThreads, smem, s>>>(p);
+        if (static_split) return launch_kernel(attend_kernel<G, true, true, kHalf>, dim3(grid), dim3(kAttendThreads), smem, s, p);
+        return launch_kernel(attend_kernel<G, true, false, kHalf>, dim3(grid), dim3(kAttendThreads), smem, s, p);
     }
-    return cudaGetLastError();
+    if (static_split) return launch_kernel(attend_kernel<G, false, true, kHalf>, dim3(grid), dim3(kAttendThreads), smem, s, p);
+    return launch_kernel(attend_kernel<G, false, false, kHalf>, dim3(grid), dim3(kAttendThreads), smem, s, p);
 }
 
 }  // namespace
@@ -626,7 +652,18 @@ int attend_grid_size()
 }
 
 int attend_max_segments() { return kSegMax; }
-int attend_max_pairs() { return 1 << 16; }
+int attend_max_pairs() { return 65535; }                   // a grid dimension of the merge kernel
+int attend_pairs_staged() { return kPairMax; }
+
+cudaError_t launch_merge(const AttendParams &p, bool static_split, int attend_grid, cudaStream_t s)
+{
+    // few pairs: many partials each (16 warps share them); many pairs: a handful each
+    const dim3 blocks(p.bv.group, p.n_pairs);
+    const bool wide = static_split || p.n_pairs * 8 <= attend_grid;
+    if (static_split) return launch_kernel(merge_kernel<16, true>, blocks, dim3(16 * 32), 0, s, p, attend_grid);
+    if (wide) return launch_kernel(merge_kernel<16, false>, blocks, dim3(16 * 32), 0, s, p, attend_grid);
+    return launch_kernel(merge_kernel<4, false>, blocks, dim3(4 * 32), 0, s, p, attend_grid);
+}
 
 cudaError_t launch_attend(const AttendParams &p, bool all_heads, bool static_split, int grid, cudaStream_t s)
 {

@@ -18,6 +18,8 @@ constexpr int kMaxTeamsPerSeq = 65536;  // the union plan keeps one bit and a pr
 constexpr uint32_t kSrcSuffix = 0x80000000u;   // segment flag: rows live in the suffix buffers
 
 constexpr int kPartialStride = 132;     // floats per (slot, head): m, l, 2 pad, acc[128]
+constexpr int kTraceSlots = 16;         // device-timer marks per block (diagnostic trace)
+constexpr int kTraceBlocks = 256;       // blocks of a kernel that leave marks; kernel k writes from block slot k * kTraceBlocks
 
 // ---------------------------------------------------------------------------------------------
 // Device-side views. Plain structs passed by value to kernels.
@@ -55,35 +57,37 @@ struct PlanView {
     int64_t *pair_row_prefix;       // [n_pairs + 1] exclusive prefix of pair_rows over pairs
 };
 
-struct Control {
-    int32_t *plan_ticket;           // [1]
-    int32_t *attend_ticket;         // [n_pairs]
-};
+// Scores of one (query head, sequence) form a row of y_stride floats, y_stride = the longest
+// sequence's team slots rounded up to a multiple of 4: rows are 16-byte aligned and their address
+// needs nothing that lives in device memory.
+__host__ __device__ __forceinline__ int64_t score_row_stride(int max_teams_per_seq)
+{
+    return ((int64_t)max_teams_per_seq + 3) & ~(int64_t)3;
+}
 
 struct ScoreParams {
     BatchView bv;
     const uint16_t *rep_keys;       // [n_kv][teams_total][128]
     const int32_t *team_row_start;  // [n_kv][teams_total + n_seqs]
     const uint16_t *q;              // [n_seqs][n_q][128]
-    float *y32;                     // [n_q][teams_total] fp32 perturbed routing scores
-    float *ymax;                    // [n_q][ymax_stride] largest score of each 16-team block: sequence b's
-                                    //   blocks start at seq_team_off[b] / 16 + b
-    int ymax_stride;
+    float *y32;                     // [n_q][n_seqs][y_stride] fp32 perturbed routing scores (see score_row_stride)
+    int64_t y_stride;
+    int tile_stride;                // tile slots per KV head: sequence b's 16-team tiles start at
+                                    //   seq_team_off[b] / 16 + b
     int n_sample;
     uint32_t seed_lo, seed_hi, step, stream_base;
     const uint32_t *step_dev;       // nullable: added to step
     double scale;
-    Control ctl;
     int n_pairs;
     int32_t *status;                // nullable
+    unsigned long long *trace;      // nullable, see trace_mark
 };
 
 // What the sampling step (headplan.cu) and the union step (pairplan.cuh) read and write.
 struct PlanInputs {
     BatchView bv;
-    const float *y32;               // [n_q][teams_total]
-    const float *ymax;              // [n_q][ymax_stride], see ScoreParams
-    int ymax_stride;
+    const float *y32;               // [n_q][n_seqs][y_stride], see ScoreParams
+    int64_t y_stride;
     const uint16_t *rep_keys;       // [n_kv][teams_total][128]
     const int32_t *team_row_start;  // [n_kv][teams_total + n_seqs]
     const float *rep_abs_max;       // [n_kv][n_seqs]
@@ -103,12 +107,12 @@ struct PlanInputs {
     float *dbg_sel_logc;
     double *dbg_tau;
     int32_t *dbg_union_rows;
+    unsigned long long *trace;      // nullable: device-timer marks, kTraceSlots per block of a kernel
 };
 
 struct PlanParams {
     PlanInputs in;
     PlanView plan;
-    Control ctl;
     int n_pairs;
 };
 
@@ -120,7 +124,6 @@ struct AttendParams {
     float qk_scale_log2;            // scale * log2(e)
     PlanView plan;                  // plan in global memory (dynamic split); seg_logc in both modes
     PlanInputs in;                  // static split: the plan is built inside the kernel
-    Control ctl;
     int n_pairs;
     float *partials;                // [slots][group][kPartialStride]
     float *out;                     // [n_seqs][n_q][128]
@@ -128,6 +131,7 @@ struct AttendParams {
     int min_rows_per_cta;
     int span_penalty_rows;          // equal-range split: rows a second span costs a CTA (see attend.cu)
     int ctas_per_pair;              // static split: CTAs that share one (sequence, KV head) pair
+    int max_words;                  // static split: 32-team words that cover the longest sequence's teams
 };
 
 // Kernels that need more than the default dynamic shared memory opt in once per device (the
@@ -145,20 +149,36 @@ inline cudaError_t ensure_dynamic_smem(const void *fn, int bytes, std::atomic<un
     return err;
 }
 
+// Launch through cudaLaunchKernelEx so that the launch's own status comes back (no sticky-error read).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // ---------------------------------------------------------------------------------------------
 // Host launchers (each returns the cudaError_t of its launches).
 // ---------------------------------------------------------------------------------------------
 cudaError_t launch_score32(const ScoreParams &p, int max_teams_per_seq, cudaStream_t s);
 cudaError_t launch_rep_abs_max(const BatchView &bv, const uint16_t *rep_keys, float *rep_abs_max, cudaStream_t s);
 cudaError_t launch_headplan(const PlanInputs &in, cudaStream_t s);
-cudaError_t launch_plan(const PlanParams &p, cudaStream_t s);
+cudaError_t launch_plan(const PlanParams &p, int max_teams_per_seq, cudaStream_t s);
+cudaError_t launch_pair_prefix(const PlanParams &p, cudaStream_t s);
 cudaError_t launch_dense_plan(const PlanParams &p, cudaStream_t s);
 // split: 0 = rows of all pairs cut into equal ranges (plan read from global memory),
 //        1 = a fixed number of CTAs per pair (plan built in the kernel; dense: trivial plan)
 cudaError_t launch_attend(const AttendParams &p, bool all_heads, bool static_split, int grid, cudaStream_t s);
+// log-sum-exp merge of the partials the attention kernel left (launched with `attend_grid` blocks)
+cudaError_t launch_merge(const AttendParams &p, bool static_split, int attend_grid, cudaStream_t s);
 int attend_grid_size();
 int attend_max_segments();
 int attend_max_pairs();
+int attend_pairs_staged();
 
 struct BuildParams {
     BatchView bv;
@@ -305,6 +325,17 @@ __device__ __forceinline__ double gumbel_from_word(uint32_t x)
 __device__ __forceinline__ uint32_t pick_word(const uint4 &w, int i)
 {
     return i == 0 ? w.x : (i == 1 ? w.y : (i == 2 ? w.z : w.w));
+}
+
+// Diagnostic: thread 0 of a block notes the device timer (ns) in slot `slot` of its block's marks.
+__device__ __forceinline__ void trace_mark(unsigned long long *trace, int kernel, int slot)
+{
+    const unsigned blk = blockIdx.x + blockIdx.y * gridDim.x;
+    if (trace != nullptr && threadIdx.x == 0 && blk < (unsigned)kTraceBlocks) {
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+        trace[((size_t)kernel * kTraceBlocks + blk) * kTraceSlots + slot] = t;
+    }
 }
 
 // Order-preserving map from a double to an unsigned 64-bit key (larger double <=> larger key).
