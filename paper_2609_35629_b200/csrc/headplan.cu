@@ -7,14 +7,15 @@ namespace santapp {
 namespace {
 
 // Few heads: 512 threads each, so that every per-thread loop is short (the kernel is a chain of
-// dependent steps, not a throughput problem); many heads: 128 threads and more resident blocks.
+// dependent steps, not a throughput problem); more heads: 256 threads and four resident blocks per
+// SM, then 128 threads and eight.
 template <int kHeadThreads, bool kHalf>
-__global__ void __launch_bounds__(kHeadThreads, 512 / kHeadThreads)
+__global__ void __launch_bounds__(kHeadThreads, kHeadThreads >= 512 ? 1 : 1024 / kHeadThreads)
 headplan_kernel(PlanInputs in)
 {
     __shared__ HeadSmem sm;
     trace_mark(in.trace, 1, 0);
-    select_head<kHeadThreads, kHeadThreads >= 512 ? 4 : 8, kHalf>(in, blockIdx.x, sm);
+    select_head<kHeadThreads, kHeadThreads >= 512 ? 4 : 2, kHalf>(in, blockIdx.x, sm);
     trace_mark(in.trace, 1, 1);
 }
 
@@ -23,12 +24,14 @@ headplan_kernel(PlanInputs in)
 cudaError_t launch_headplan(const PlanInputs &in, cudaStream_t s)
 {
     const int n_heads = in.bv.n_seqs * in.bv.n_q;
-    const bool wide = n_heads <= attend_grid_size();
+    const int sms = attend_grid_size();
     if (in.bv.elem) {
-        if (wide) return launch_kernel(headplan_kernel<512, true>, dim3(n_heads), dim3(512), 0, s, in);
+        if (n_heads <= sms) return launch_kernel(headplan_kernel<512, true>, dim3(n_heads), dim3(512), 0, s, in);
+        if (n_heads <= 4 * sms) return launch_kernel(headplan_kernel<256, true>, dim3(n_heads), dim3(256), 0, s, in);
         return launch_kernel(headplan_kernel<128, true>, dim3(n_heads), dim3(128), 0, s, in);
     }
-    if (wide) return launch_kernel(headplan_kernel<512, false>, dim3(n_heads), dim3(512), 0, s, in);
+    if (n_heads <= sms) return launch_kernel(headplan_kernel<512, false>, dim3(n_heads), dim3(512), 0, s, in);
+    if (n_heads <= 4 * sms) return launch_kernel(headplan_kernel<256, false>, dim3(n_heads), dim3(256), 0, s, in);
     return launch_kernel(headplan_kernel<128, false>, dim3(n_heads), dim3(128), 0, s, in);
 }
 

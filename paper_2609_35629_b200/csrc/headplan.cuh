@@ -159,13 +159,9 @@ __device__ __forceinline__ void select_head(const PlanInputs &in, int hq, HeadSm
                 for (int i = tid; i < 256; i += kT) sm.hist[i] = 0;
                 __syncthreads();
             }
-            int below = 0;
             auto count = [&](float x) {
                 const int gb = score_bin(top, x);
-                if (gb >= win) {
-                    if (gb - win < kWindow) atomicAdd(&sm.hist[gb - win], 1);
-                    else ++below;
-                }
+                if (gb >= win) atomicAdd(&sm.hist[min(gb - win, kWindow)], 1);
             };
             float grp = -CUDART_INF_F;
             bool any = false;
@@ -187,9 +183,6 @@ __device__ __forceinline__ void select_head(const PlanInputs &in, int hq, HeadSm
                     }
                 }
             });
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) below += __shfl_xor_sync(0xFFFFFFFFu, below, o);
-            if (lane == 0 && below > 0) atomicAdd(&sm.hist[kWindow], below);
             trace_mark(in.trace, 1, 9);
             __syncthreads();
             trace_mark(in.trace, 1, 10);
@@ -270,7 +263,7 @@ __device__ __forceinline__ void select_head(const PlanInputs &in, int hq, HeadSm
             const double *qs = sm.q64[sub];
             // four candidates per thread group at a time: all their key pieces are requested before
             // the first product, so a chunk costs one memory round trip
-            constexpr int kPerPass = kDotWarps * 32 / kDotLanes, kChunk = kT >= 512 ? 1 : 4;
+            constexpr int kPerPass = kDotWarps * 32 / kDotLanes, kChunk = kT >= 512 ? 2 : 4;
             for (int c0 = 0; c0 < n_cand; c0 += kPerPass * kChunk) {
                 uint4 w[kChunk][2];
 #pragma unroll
@@ -348,17 +341,27 @@ __device__ __forceinline__ void select_head(const PlanInputs &in, int hq, HeadSm
                     if (e < n_list) { y = sm.list_y[cur][e]; phi = sm.list_phi[cur][e]; id = sm.list_id[cur][e]; rows = sm.list_rows[cur][e]; }
                     else { y = sm.cand_y[e - n_list]; phi = sm.cand_phi[e - n_list]; id = sm.cand_id[e - n_list]; rows = sm.cand_rows[e - n_list]; }
                 }
-                // rank = entries ahead of this one (larger score, or the same score and a smaller id)
-                int rank = 0;
+                // rank = entries ahead of this one (larger score, or the same score and a smaller id);
+                // ids are looked at only when some other entry has exactly the same score
+                int rank = 0, same = 0;
                 if (live) {
                     for (int a = sub; a < n_list; a += 8) {
                         const double w = sm.list_y[cur][a];
-                        rank += (w > y) || (w == y && sm.list_id[cur][a] < id);
+                        rank += (w > y);
+                        same += (w == y);
                     }
                     for (int a = sub; a < n_cand; a += 8) {
                         const double w = sm.cand_y[a];
-                        rank += (w > y) || (w == y && sm.cand_id[a] < id);
+                        rank += (w > y);
+                        same += (w == y);
                     }
+                }
+                same += __shfl_xor_sync(0xFFFFFFFFu, same, 1);
+                same += __shfl_xor_sync(0xFFFFFFFFu, same, 2);
+                same += __shfl_xor_sync(0xFFFFFFFFu, same, 4);
+                if (live && same > 1) {
+                    for (int a = sub; a < n_list; a += 8) rank += (sm.list_y[cur][a] == y && sm.list_id[cur][a] < id);
+                    for (int a = sub; a < n_cand; a += 8) rank += (sm.cand_y[a] == y && sm.cand_id[a] < id);
                 }
                 rank += __shfl_xor_sync(0xFFFFFFFFu, rank, 1);
                 rank += __shfl_xor_sync(0xFFFFFFFFu, rank, 2);

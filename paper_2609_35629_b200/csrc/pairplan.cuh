@@ -119,9 +119,35 @@ __device__ __forceinline__ void build_pair_plan(const PlanInputs &in, int pair, 
         if (ok) atomicOr(&sc.bitmap[ent_team[u] >> 5], 1u << (ent_team[u] & 31));
     }
     __syncthreads();
-    // word prefix of the bitmap: segment index of a team = selected teams before it.
-    // Thread t owns the contiguous words [t * wpt, (t + 1) * wpt).
-    {
+    // Segment index of a team = selected teams before it: prefix over the bitmap's words.
+    int ent_seg[kEntPerThread];
+    int nseg_prompt;
+    if (n_words <= 64) {
+        // every warp sums the (at most 64) words for itself, two per lane: no table, no barrier
+        const int lane = tid & 31;
+        const uint32_t w0 = 2 * lane < n_words ? sc.bitmap[2 * lane] : 0u;
+        const uint32_t w1 = 2 * lane + 1 < n_words ? sc.bitmap[2 * lane + 1] : 0u;
+        const int c0 = __popc(w0), c1 = __popc(w1);
+        int incl = c0 + c1;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+            if (lane >= o) incl += t;
+        }
+        nseg_prompt = __shfl_sync(0xFFFFFFFFu, incl, 31);
+        const int excl = incl - c0 - c1;
+#pragma unroll
+        for (int u = 0; u < kEntPerThread; ++u) {
+            const int team = ent_key[u] >= 0 ? ent_key[u] >> 3 : 0;
+            const int word = team >> 5, src = word >> 1;
+            // every lane takes part in every exchange; the choice between a lane's two words comes after
+            const int s_excl = __shfl_sync(0xFFFFFFFFu, excl, src), s_c0 = __shfl_sync(0xFFFFFFFFu, c0, src);
+            const uint32_t s_w0 = __shfl_sync(0xFFFFFFFFu, w0, src), s_w1 = __shfl_sync(0xFFFFFFFFu, w1, src);
+            const uint32_t bits = (word & 1) ? s_w1 : s_w0;
+            ent_seg[u] = s_excl + ((word & 1) ? s_c0 : 0) + __popc(bits & ((1u << (team & 31)) - 1u));
+        }
+    } else {
+        // thread t owns the contiguous words [t * wpt, (t + 1) * wpt)
         const int wpt = (n_words + kPlanThreads - 1) / kPlanThreads;
         const int lo = min(tid * wpt, n_words), hi = min(lo + wpt, n_words);
         int sum = 0;
@@ -129,15 +155,18 @@ __device__ __forceinline__ void build_pair_plan(const PlanInputs &in, int pair, 
         int total;
         int run = block_exclusive_scan(sum, sc.scan, total);
         for (int w = lo; w < hi; ++w) { sc.wprefix[w] = run; run += __popc(sc.bitmap[w]); }
-        if (tid == 0) sc.misc[0] = total;                             // segments of the prompt
+        __syncthreads();
+        nseg_prompt = total;
+#pragma unroll
+        for (int u = 0; u < kEntPerThread; ++u) {
+            const int team = ent_key[u] >= 0 ? ent_key[u] >> 3 : 0;
+            ent_seg[u] = sc.wprefix[team >> 5] + __popc(sc.bitmap[team >> 5] & ((1u << (team & 31)) - 1u));
+        }
     }
-    __syncthreads();
-    const int nseg_prompt = sc.misc[0];
 #pragma unroll
     for (int u = 0; u < kEntPerThread; ++u) {
         if (ent_key[u] >= 0) {
-            const int team = ent_key[u] >> 3, h = ent_key[u] & 7;
-            const int seg = sc.wprefix[team >> 5] + __popc(sc.bitmap[team >> 5] & ((1u << (team & 31)) - 1u));
+            const int h = ent_key[u] & 7, seg = ent_seg[u];
             atomicOr(&seg_mask[seg], 1u << h);
             g_logc[(size_t)seg * kMaxGroup + h] = kLog2e * ent_logc[u];
             seg_row[seg] = (int32_t)(row0 + ent_rows[u].x);           // same value from every selecting head
