@@ -36,12 +36,14 @@ METRIC = "decode_attn_us_per_layer_step"
 UNIT = "us"
 N_STEP_INPUTS = 8          # distinct (query, suffix length, step) inputs cycled through
 
-# DRAM bytes (read + write) of one attend_kernel launch from an ncu capture of the same per-launch
-# work (summaries under profiles/, named for the kernel and workload); None where none was taken.
+# DRAM bytes (read + write) of one attend_kernel launch, recorded from an ncu capture of this
+# kernel on the same per-launch work (default seed, independent keys, contiguous parents). A
+# recorded figure, not one measured by this run: it is reported as `traffic` together with
+# `traffic_kind`, and left out (null) for any other variant of the workload.
 NCU_TRAFFIC_BYTES = {
-    "qwen7b_b1_32k": 34.61e6,      # profiles/attend_kernel_qwen7b_b1_32k.md (mean of two launches)
-    "qwen7b_b8_32k": 409.0e6,      # profiles/attend_kernel_qwen7b_b8_32k.md
-    "ragged": 1036.2e6,            # profiles/all_kernels_ragged.md (mean of two launches)
+    "qwen7b_b1_32k": 34.61e6,
+    "qwen7b_b8_32k": 409.0e6,
+    "ragged": 1036.2e6,
 }
 
 
@@ -244,6 +246,15 @@ def run_ours(args):
                     "achieved_frac_of_peak", "dense_achieved_frac_of_peak", "roofline", "stage_us", "paired_rounds",
                     "steps", "warmup")
             line["batched"] = {"workload": big["config"]["workload"], **{k: big[k] for k in keep}}
+        # the two mid-size workloads: eight 32K sequences with 64 sampled teams, and four 128K
+        # sequences with 32 (a few layers and steps each)
+        for key, wl, n_lay, k_over in (("mid_batch", "qwen7b_b8_32k", 4, 0), ("long_context", "long_128k", 2, 32)):
+            gc.collect()
+            torch.cuda.empty_cache()
+            wl_args = argparse.Namespace(**{**vars(args), "n_sample": k_over})
+            res = measure_workload(wl_args, wl, n_lay, 10, 3, dev, want_e2e=False, want_cpu=False, want_stages=True)
+            if rank == 0:
+                line[key] = {"workload": res["config"]["workload"], **{k: res[k] for k in keep}}
         # and the headline workload with the parents of the paper's headline runs: Algorithm 3
         # (minibatch k-means with the paper's settings, fitted by the library), four layers
         if args.parents == "contiguous" and args.elem == "bf16":
@@ -475,7 +486,8 @@ def measure_workload(args, workload, n_layers, n_steps, n_warmup, dev, want_e2e,
         g_sparse.replay()
         torch.cuda.synchronize()
         for name, mask in (("route_score", sp.STAGE_ROUTE), ("select_plan", sp.STAGE_SELECT),
-                           ("route_and_select", sp.STAGE_ROUTE | sp.STAGE_SELECT), ("attend", sp.STAGE_ATTEND)):
+                           ("route_and_select", sp.STAGE_ROUTE | sp.STAGE_SELECT), ("attend", sp.STAGE_ATTEND),
+                           ("merge", sp.STAGE_MERGE), ("attend_and_merge", sp.STAGE_ATTEND | sp.STAGE_MERGE)):
             sp.santapp_set_stage_mask(mask)
             g = capture(sparse_layer)
             sp.santapp_set_stage_mask(sp.STAGE_ALL)
@@ -498,7 +510,9 @@ def measure_workload(args, workload, n_layers, n_steps, n_warmup, dev, want_e2e,
                     "traffic": (NCU_TRAFFIC_BYTES.get(spec.name)
                                 if not args.n_sample and spec.key_layout == "iid" and spec.parents == "contiguous" else None),
                     "peak_kind": peak_kind,
-                    "algorithmic_bytes_per_launch": attend_bytes_1, "us_per_launch": stages["attend"]}
+                    "traffic_kind": "recorded from an earlier ncu capture of this kernel and workload, not measured in this run",
+                    "algorithmic_bytes_per_launch": attend_bytes_1, "us_per_launch": stages["attend"],
+                    "launches_timed": "attend_kernel alone (the merge kernel that follows it is stage_us.merge)"}
 
     # ---- end to end through host buffers ----
     e2e = None

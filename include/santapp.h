@@ -18,9 +18,11 @@
  *
  * Conventions
  *   - "device" pointers address GPU global memory of the current device; "host" pointers
- *     address CPU memory. The library allocates no device memory and keeps no state: the
- *     caller owns every buffer, including workspaces, whose sizes come from the *_sizes /
- *     *_workspace_bytes queries. Buffers should be 256-byte aligned; a bf16 / fp32 array or a
+ *     address CPU memory. The library allocates no device memory and keeps no state between
+ *     calls (one exception, stated with it: santapp_dense_decode_attn_noalloc and its built-in
+ *     array): the caller owns every buffer, including workspaces, whose sizes come from the
+ *     *_sizes / *_workspace_bytes queries. A workspace needs no initialisation: every word a
+ *     kernel reads was written earlier in the same call. Buffers should be 256-byte aligned; a bf16 / fp32 array or a
  *     workspace that is not at least 16-byte aligned (64-bit offset arrays: 8, 32-bit tables: 4)
  *     is refused with SANTAPP_ERR_INVALID_ARG.
  *   - bf16 tensors are raw 16-bit patterns. head_dim is 128. Query head h uses KV head
@@ -398,11 +400,13 @@ int santapp_dense_decode_attn(const santapp_geom *geom, const santapp_teams *tea
  *     santapp_last_cuda_error says how many bytes were needed). On a 148-SM GPU with 7 query
  *     heads per KV head the 2 MiB array covers about 400 (sequence, KV head) pairs.
  *   - Set-up: the first call on each device looks up the array's device address (the device
- *     must be current, as for every call) and remembers it. Make that first call outside any
- *     stream capture.
+ *     must be current, as for every call) and remembers it for the life of the process. Make
+ *     that first call outside any stream capture. The remembered address belongs to the
+ *     device's context: after a cudaDeviceReset it is stale, and the library must be reloaded
+ *     before this entry point is used again on that device.
  *   - Sharing: every call on a device uses the same array, which keeps whatever the previous
- *     call left in it. Nothing in it has to be cleared between calls: the kernels initialise
- *     every counter and table they read. Two calls that can overlap on the GPU (different
+ *     call left in it. Nothing in it has to be cleared between calls: the kernels write every
+ *     table they read, and there are no counters. Two calls that can overlap on the GPU (different
  *     streams without an ordering between them) race on the array and must not be issued.
  */
 #define SANTAPP_STATIC_SCRATCH_BYTES (2u << 20)
@@ -423,11 +427,13 @@ int santapp_last_launch_count(void);
  * Bit 0: representative scoring and perturbation; bit 1: sampling per query head, and the
  * read plans as a kernel of their own for batches of many (sequence, KV head) pairs (for few
  * pairs the union of the heads' samples is the first phase of the attention kernel);
- * bit 2: exact attention and merge. A stage that is skipped reuses what an earlier full call
- * with the same arguments left in the same workspace. The default, and the only setting that
- * computes a decode step, is SANTAPP_STAGE_ALL.
+ * bit 2: exact attention (each block leaves a partial result); bit 3: the merge of the partials
+ * into the output. A stage that is skipped reuses what an earlier full call with the same
+ * arguments left in the same workspace. The default, and the only setting that computes a
+ * decode step, is SANTAPP_STAGE_ALL.
  */
-enum { SANTAPP_STAGE_ROUTE = 1, SANTAPP_STAGE_SELECT = 2, SANTAPP_STAGE_ATTEND = 4, SANTAPP_STAGE_ALL = 7 };
+enum { SANTAPP_STAGE_ROUTE = 1, SANTAPP_STAGE_SELECT = 2, SANTAPP_STAGE_ATTEND = 4, SANTAPP_STAGE_MERGE = 8,
+       SANTAPP_STAGE_ALL = 15 };
 void santapp_set_stage_mask(int mask);
 
 #ifdef __cplusplus

@@ -36,7 +36,7 @@ EXPORTS = [
     "santapp_kmeans_fit_workspace_bytes", "santapp_kmeans_fit",
 ]
 
-STAGE_ROUTE, STAGE_SELECT, STAGE_ATTEND, STAGE_ALL = 1, 2, 4, 7
+STAGE_ROUTE, STAGE_SELECT, STAGE_ATTEND, STAGE_MERGE, STAGE_ALL = 1, 2, 4, 8, 15
 
 
 class SantappError(RuntimeError):

@@ -793,6 +793,9 @@ int santapp_decode_attn(const santapp_geom *geom, const santapp_teams *teams, co
         err = launch_attend(ap, false, L.static_split, launch_grid, s);
         if (err != cudaSuccess) return cuda_fail(err, "attend launch");
         ++g_launches;
+    }
+    if (g_stage_mask & SANTAPP_STAGE_MERGE) {
+        const int launch_grid = L.static_split ? L.n_pairs * L.ctas_per_pair : grid;
         err = launch_merge(ap, L.static_split, launch_grid, s);
         if (err != cudaSuccess) return cuda_fail(err, "merge launch");
         ++g_launches;

@@ -522,12 +522,72 @@ def test_stage_mask_reruns_one_stage_on_the_same_workspace():
     try:
         # each stage alone, in pipeline order, reusing what the full call left in the workspace;
         # only the last stage writes the output
-        for mask in (sp.STAGE_ATTEND, sp.STAGE_ROUTE, sp.STAGE_SELECT, sp.STAGE_ATTEND):
+        for mask in (sp.STAGE_ATTEND | sp.STAGE_MERGE, sp.STAGE_ROUTE, sp.STAGE_SELECT, sp.STAGE_ATTEND, sp.STAGE_MERGE):
             sp.santapp_set_stage_mask(mask)
             again = sp.santapp_decode_attn(*args, workspace=ws)
             assert sp.santapp_last_launch_count() <= 3
             torch.cuda.synchronize()
-            if mask == sp.STAGE_ATTEND:
+            if mask & sp.STAGE_MERGE:
                 assert torch.allclose(full, again, rtol=0, atol=1e-6)
     finally:
         sp.santapp_set_stage_mask(sp.STAGE_ALL)
+
+
+def test_guard_words_around_the_workspaces_survive_every_call():
+    """The decode, dense and build workspaces sit between guard words (a known pattern in the 4 KB
+    before and after each): a kernel writing outside the sizes the library asked for would change
+    them. One small batch with the plan inside the attention kernel, one ragged batch with plans in
+    global memory."""
+    def guarded(n_bytes):
+        pad = 4096
+        buf = torch.full((n_bytes + 2 * pad + 256,), 0xA5, dtype=torch.uint8, device="cuda")
+        off = (-buf.data_ptr()) % 256                     # the workspace itself 256-byte aligned
+        return buf, buf[off + pad: off + pad + n_bytes], (off, pad, n_bytes)
+
+    def intact(buf, where):
+        off, pad, n = where
+        head, tail = buf[:off + pad], buf[off + pad + n:]
+        return bool((head == 0xA5).all()) and bool((tail == 0xA5).all())
+
+    cases = [synth.spec_small_gqa(seed=21),
+             synth.spec_small_gqa(seed=22, n_seqs=24, prompt=tuple(200 + 97 * (i % 7) for i in range(24)), parent_size=64,
+                                  reps=8, n_sample=8, suffix0=tuple(i % 5 for i in range(24)))]
+    for spec in cases:
+        layer = pu.GpuLayer(spec, synth.make_layer(spec))
+        q_bits = synth.make_queries(spec, layer.data, 1)
+        q = sp.bf16_bits_to_cuda(q_bits)
+        sl_np = spec.suffix_len(1)
+        sl = torch.from_numpy(sl_np).cuda()
+        K = spec.n_sample
+        buf, ws, where = guarded(sp.santapp_decode_workspace_bytes(layer.geom, layer.teams, K))
+        dbg = sp.DebugBuffers(layer.geom, K, "cuda")
+        out = sp.santapp_decode_attn(layer.geom, layer.teams, q, layer.k_suffix, layer.v_suffix, sl, K, 77, 1, debug=dbg,
+                                     workspace=ws)
+        torch.cuda.synchronize()
+        assert intact(buf, where), "decode wrote outside its workspace"
+        ref = pu.oracle_step(layer, q_bits, sl_np, K, 77, 1)
+        vmax = pu.max_abs_v(layer)
+        for b, r in ref.items():
+            assert np.array_equal(dbg.sel_idx.cpu().numpy()[b][:, :r.sel.shape[1]], r.sel)
+            assert np.abs(out[b].cpu().numpy() - r.o).max() <= SPARSE_TOL * vmax
+        buf, ws, where = guarded(sp.santapp_dense_workspace_bytes(layer.geom, layer.teams))
+        dense = sp.santapp_dense_decode_attn(layer.geom, layer.teams, q, layer.k_suffix, layer.v_suffix, sl, workspace=ws)
+        torch.cuda.synchronize()
+        assert intact(buf, where), "dense decode wrote outside its workspace"
+        dref = pu.oracle_step(layer, q_bits, sl_np, 0, 0, 1, dense=True)
+        for b, o in dref.items():
+            assert np.abs(dense[b].cpu().numpy() - o).max() <= DENSE_TOL * vmax
+        # the team builder's workspace, through the C ABI with a guarded buffer
+        sizes = sp.santapp_build_teams_sizes(layer.geom, spec.prompt_len)
+        buf, ws, where = guarded(max(sizes.build_workspace_bytes, 256))
+        teams = sp.Teams(layer.geom, sizes, "cuda")
+        import ctypes
+        g = layer.geom.c()
+        arr = (ctypes.c_int32 * spec.n_seqs)(*[int(x) for x in spec.prompt_len])
+        rc = sp.load_library().santapp_build_teams(ctypes.byref(g), arr, ctypes.c_void_p(layer.k_prompt.data_ptr()),
+                                                   ctypes.c_void_p(layer.v_prompt.data_ptr()), ctypes.byref(teams.c),
+                                                   ctypes.c_void_p(ws.data_ptr()), ws.numel(), None)
+        torch.cuda.synchronize()
+        assert rc == 0 and intact(buf, where), "team build wrote outside its workspace"
+        assert torch.equal(teams.team_row_start, layer.teams.team_row_start)
+        assert torch.equal(teams.k_packed.view(torch.int16), layer.teams.k_packed.view(torch.int16))
