@@ -84,7 +84,7 @@ BatchView make_view(const santapp_geom *g, const santapp_teams *t)
 
 // Workspace layout shared by the sparse and the dense call. Offsets in bytes.
 struct DecodeLayout {
-    size_t y32, sel_team, sel_logc, sel_rows, seg_prefix, seg_row, seg_mask, seg_logc, pair_nseg, pair_rows, pair_prefix, partials, total;
+    size_t counter, y32, sel_team, sel_logc, sel_rows, seg_prefix, seg_row, seg_mask, seg_logc, pair_nseg, pair_rows, pair_prefix, partials, total;
     int seg_cap, grid, n_pairs, ctas_per_pair, tile_stride;
     int64_t y_stride;
     bool static_split;
@@ -98,13 +98,18 @@ DecodeLayout decode_layout(const santapp_geom *g, const santapp_teams *t, int K,
     L.grid = grid;
     // few pairs: a fixed number of CTAs per pair and the plan built inside the attention kernel;
     // many pairs: equal row ranges over a plan in global memory
-    L.static_split = (int64_t)L.n_pairs * 9 <= grid;
+    int static_factor = 9;
+#ifdef SANTAPP_TUNE
+    if (const char *e = getenv("SANTAPP_STATIC_FACTOR")) static_factor = atoi(e);
+#endif
+    L.static_split = (int64_t)L.n_pairs * static_factor <= grid;
     L.ctas_per_pair = L.static_split ? grid / L.n_pairs : 1;
     int64_t cap = dense ? 1 : (int64_t)G * K;
     if (cap > t->max_teams_per_seq) cap = t->max_teams_per_seq;
     L.seg_cap = (int)cap + 1;                                   // + the suffix segment
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
+    L.counter = take(sizeof(int32_t) * 2);
     L.y_stride = score_row_stride(t->max_teams_per_seq);
     L.y32 = take(dense ? 0 : sizeof(float) * (size_t)g->n_q_heads * (size_t)g->n_seqs * (size_t)L.y_stride);
     L.tile_stride = (int)(t->teams_total / 16 + g->n_seqs + 1);
@@ -118,7 +123,8 @@ DecodeLayout decode_layout(const santapp_geom *g, const santapp_teams *t, int K,
     L.pair_nseg = take(sizeof(int32_t) * (size_t)L.n_pairs);
     L.pair_rows = take(sizeof(int32_t) * (size_t)L.n_pairs);
     L.pair_prefix = take(sizeof(int64_t) * ((size_t)L.n_pairs + 1));
-    L.partials = take(sizeof(float) * ((size_t)grid + L.n_pairs) * G * kPartialStride);
+    // one partial per (block or tail chunk, pair it touches)
+    L.partials = take(sizeof(float) * ((size_t)grid * (1 + kMaxTailChunksPerBlock) + 1 + L.n_pairs) * G * kPartialStride);
     L.total = off;
     return L;
 }
@@ -134,6 +140,7 @@ void fill_plan(const DecodeLayout &L, char *ws, PlanView &plan)
     plan.pair_rows = reinterpret_cast<int32_t *>(ws + L.pair_rows);
     plan.pair_union_rows = nullptr;
     plan.pair_row_prefix = reinterpret_cast<int64_t *>(ws + L.pair_prefix);
+    plan.tail_counter = reinterpret_cast<int32_t *>(ws + L.counter);
 }
 
 }  // namespace

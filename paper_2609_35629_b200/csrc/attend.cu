@@ -185,7 +185,11 @@ attend_kernel(AttendParams p)
         __syncthreads();
         pair_base = 0;
     };
-    int64_t r0 = 0, r1 = 0, rows_per_cta = 0;              // dynamic split: global row range
+    uint32_t r0 = 0, r1 = 0;                               // dynamic split: this item's range of the padded row line (< 2^32)
+    int item = blockIdx.x;                                 // dynamic split: fixed range (< gridDim.x) or tail chunk
+    int next_chunk = 0;                                    // thread 0: the tail chunk taken from the counter for later
+    RangeSplit &sp = *reinterpret_cast<RangeSplit *>(misc + 8);   // the same in every thread: kept in shared memory
+    const bool windowed = p.n_pairs > kPairMax;
     if (kStatic) {
         pair = blockIdx.x / p.ctas_per_pair;
         sub = blockIdx.x - pair * p.ctas_per_pair;
@@ -193,25 +197,37 @@ attend_kernel(AttendParams p)
     } else {
         // pair_prefix / pair_nseg hold a window of kPairMax pairs starting at pair_base; batches of up
         // to kPairMax pairs are staged whole, before anything else is waited for
-        const bool windowed = p.n_pairs > kPairMax;
         if (!windowed) stage_all_pairs();
         const int64_t all_rows = windowed ? p.plan.pair_row_prefix[p.n_pairs] : pair_prefix[p.n_pairs];
         // Rows of all pairs laid end to end, with a gap of span_penalty_rows after every pair: a CTA
         // whose range crosses from one pair into the next pays the fixed cost of a second span
         // (tables, pipeline refill, merge) out of its row budget, so ranges cost about equal time.
-        const int64_t total = all_rows + (int64_t)p.span_penalty_rows * (p.n_pairs - 1);
-        rows_per_cta = (total + gridDim.x - 1) / gridDim.x;
-        if (rows_per_cta < p.min_rows_per_cta) rows_per_cta = p.min_rows_per_cta;
-        r0 = (int64_t)blockIdx.x * rows_per_cta;
-        if (r0 >= total) return;
-        r1 = min(r0 + rows_per_cta, total);
+        __syncthreads();
+        if (tid == 0) sp = make_range_split(all_rows, p.n_pairs, p.span_penalty_rows, p.min_rows_per_cta, (int)gridDim.x);
+        __syncthreads();
+    }
+
+  for (;;) {                                               // items of this block (one, for the fixed split)
+    if (!kStatic) {
+        // the next tail chunk is asked for now and looked at when this item is done
+        if (tid == 0 && sp.n_tail > 0) next_chunk = atomicAdd(p.plan.tail_counter, 1);
+        {
+            const bool fixed = item < (int)gridDim.x;
+            const uint64_t lo64 = fixed ? (uint64_t)item * sp.fixed_rows
+                                        : (uint64_t)sp.fixed_end + (uint64_t)(item - (int)gridDim.x) * sp.chunk_rows;
+            const uint64_t end = fixed ? sp.fixed_end : sp.total;
+            const uint64_t hi64 = min(lo64 + (fixed ? sp.fixed_rows : sp.chunk_rows), end);
+            if (lo64 >= hi64) goto item_done;
+            r0 = (uint32_t)lo64;
+            r1 = (uint32_t)hi64;
+        }
         // first pair of the range: the largest i with prefix[i] + penalty * i <= r0
         int lo = 0, hi = p.n_pairs;
         while (hi - lo > 1) {
             const int mid = (lo + hi) >> 1;
             const int64_t start = (windowed ? p.plan.pair_row_prefix[mid] : pair_prefix[mid])
                                   + (int64_t)p.span_penalty_rows * mid;
-            if (start <= r0) lo = mid; else hi = mid;
+            if (start <= (int64_t)r0) lo = mid; else hi = mid;
         }
         if (windowed) stage_pairs(lo);
         pair = lo;
@@ -219,7 +235,7 @@ attend_kernel(AttendParams p)
 
     while (true) {
         int a, bnd, nseg, slot_id;
-        int64_t pb = 0, pe = 0;
+        uint32_t pb = 0, pe = 0;
         const int b = pair / p.bv.n_kv, j = pair - b * p.bv.n_kv;
         const float *g_logc = p.plan.seg_logc + (size_t)pair * cap * kMaxGroup;
         // A fragments of q for the 8 k-steps: head g (zero rows for g >= G and for M rows 8..15);
@@ -284,18 +300,18 @@ attend_kernel(AttendParams p)
         } else {
             // this pair's rows occupy [pb, pe) of the padded row line
             if (pair - pair_base >= kPairMax) stage_pairs(pair);           // walked off the staged window
-            pb = pair_prefix[pair - pair_base] + (int64_t)p.span_penalty_rows * pair;
-            pe = pb + (pair_prefix[pair - pair_base + 1] - pair_prefix[pair - pair_base]);
+            pb = (uint32_t)(pair_prefix[pair - pair_base] + (int64_t)p.span_penalty_rows * pair);
+            pe = pb + (uint32_t)(pair_prefix[pair - pair_base + 1] - pair_prefix[pair - pair_base]);
             a = (int)(max(r0, pb) - pb);
             bnd = (int)(min(r1, pe) - pb);
             if (a >= bnd) {                                // the range starts in the gap behind this pair
                 r0 = pe + p.span_penalty_rows;
-                if (r0 >= r1 || pair + 1 >= p.n_pairs) return;
+                if (r0 >= r1 || pair + 1 >= p.n_pairs) goto item_done;
                 ++pair;
                 continue;
             }
             nseg = pair_nseg[pair - pair_base];
-            slot_id = blockIdx.x + pair;                   // CTA c's partial of pair i lives in slot c + i
+            slot_id = item + pair;                         // item c's partial of pair i lives in slot c + i
             __syncthreads();                               // the previous span is done with the tables
             // one round trip: every load is issued before the first store
             const int32_t *g_prefix = p.plan.seg_prefix + (size_t)pair * (cap + 1);
@@ -523,12 +539,32 @@ attend_kernel(AttendParams p)
             trace_mark(p.in.trace, 3, 5);
             return;                                        // one span per CTA
         } else {
-            if (pb + bnd < pe) return;                     // the range ended inside this pair
+            if (pb + bnd < pe) goto item_done;             // the range ended inside this pair
             r0 = pe + p.span_penalty_rows;                 // first row of the next pair
-            if (r0 >= r1 || pair + 1 >= p.n_pairs) return;
+            if (r0 >= r1 || pair + 1 >= p.n_pairs) goto item_done;
             ++pair;
         }
     }
+item_done:
+    if (kStatic) return;
+    if (sp.n_tail == 0) return;
+    __syncthreads();                                       // also: every warp is done with the previous span's scratch
+    if (tid == 0) misc[5] = next_chunk;
+    __syncthreads();
+    if (misc[5] >= sp.n_tail) {
+        // Out of chunks: the block leaves. The last block to leave resets both counters, so that the
+        // kernel can be launched again on the same plans.
+        if (tid == 0) {
+            const int left = atomicAdd(p.plan.tail_counter + 1, 1);
+            if (left == (int)gridDim.x - 1) {
+                p.plan.tail_counter[0] = 0;
+                p.plan.tail_counter[1] = 0;
+            }
+        }
+        return;
+    }
+    item = (int)gridDim.x + misc[5];
+  }
 }
 
 // Log-sum-exp merge of a pair's partials (the split-softmax reduction): one block per (query head
@@ -547,26 +583,37 @@ merge_kernel(AttendParams p, int attend_grid)
     const int b = pair / p.bv.n_kv, j = pair - b * p.bv.n_kv;
     const int part = threadIdx.x >> 5, lane = threadIdx.x & 31;
     trace_mark(p.in.trace, 4, 0);
-    int first_slot, n;
+    // the pair's partials: slots [first_slot, first_slot + n_fixed), then [tail_slot, tail_slot + n - n_fixed)
+    int first_slot, n, n_fixed, tail_slot = 0;
     if (kStatic) {
         first_slot = pair * p.ctas_per_pair;
-        n = p.ctas_per_pair;
+        n = n_fixed = p.ctas_per_pair;
     } else {
-        // the attention kernel's split: rows of all pairs end to end with a gap behind each
-        // (all below 2^32: rows_total < 2^31 and the gaps add at most 2^26 * 16)
+        // the attention kernel's split: rows of all pairs end to end with a gap behind each; item c
+        // (fixed range or tail chunk) left its partial of pair i in slot c + i
         const int64_t pre0 = p.plan.pair_row_prefix[pair], pre1 = p.plan.pair_row_prefix[pair + 1];
-        const int64_t all_rows = p.plan.pair_row_prefix[p.n_pairs];
-        const uint32_t total = (uint32_t)(all_rows + (int64_t)p.span_penalty_rows * (p.n_pairs - 1));
-        uint32_t rows_per_cta = (total + (uint32_t)attend_grid - 1u) / (uint32_t)attend_grid;
-        if (rows_per_cta < (uint32_t)p.min_rows_per_cta) rows_per_cta = (uint32_t)p.min_rows_per_cta;
+        const RangeSplit sp = make_range_split(p.plan.pair_row_prefix[p.n_pairs], p.n_pairs, p.span_penalty_rows,
+                                               p.min_rows_per_cta, attend_grid);
         const uint32_t pb = (uint32_t)(pre0 + (int64_t)p.span_penalty_rows * pair);
         const uint32_t pe = pb + (uint32_t)(pre1 - pre0);
-        const int c_lo = (int)(pb / rows_per_cta), c_hi = (int)((max(pe, pb + 1u) - 1u) / rows_per_cta);
-        first_slot = c_lo + pair;
-        n = pe > pb ? c_hi - c_lo + 1 : 0;
+        n_fixed = 0;
+        first_slot = pair;
+        if (pe > pb && pb < sp.fixed_end) {
+            const int c_lo = (int)(pb / sp.fixed_rows), c_hi = (int)((min(pe, sp.fixed_end) - 1u) / sp.fixed_rows);
+            first_slot = c_lo + pair;
+            n_fixed = c_hi - c_lo + 1;
+        }
+        n = n_fixed;
+        if (pe > pb && pe > sp.fixed_end) {
+            const int j_lo = (int)((max(pb, sp.fixed_end) - sp.fixed_end) / sp.chunk_rows);
+            const int j_hi = (int)((pe - 1u - sp.fixed_end) / sp.chunk_rows);
+            tail_slot = attend_grid + j_lo + pair;
+            n += j_hi - j_lo + 1;
+        }
     }
     const size_t stride = (size_t)G * kPartialStride;
-    const float *base = p.partials + ((size_t)first_slot * G + h) * kPartialStride;
+    const float *base = p.partials + (size_t)h * kPartialStride;
+    auto slot_of = [&](int i) { return (size_t)(i < n_fixed ? first_slot + i : tail_slot + (i - n_fixed)); };
     constexpr int kDepth = 4;                              // partials a thread has in flight: one round trip for n <= 4 kParts
     float m_run = -CUDART_INF_F, l_run = 0.f;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -579,8 +626,8 @@ merge_kernel(AttendParams p, int attend_grid)
             ml[u] = make_float2(-CUDART_INF_F, 0.f);
             v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
             if (i < n) {
-                ml[u] = __ldcg(reinterpret_cast<const float2 *>(base + (size_t)i * stride));
-                v[u] = __ldcg(reinterpret_cast<const float4 *>(base + (size_t)i * stride + 4) + lane);
+                ml[u] = __ldcg(reinterpret_cast<const float2 *>(base + slot_of(i) * stride));
+                v[u] = __ldcg(reinterpret_cast<const float4 *>(base + slot_of(i) * stride + 4) + lane);
             }
         }
         float m_new = m_run;

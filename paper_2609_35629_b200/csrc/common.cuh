@@ -55,7 +55,47 @@ struct PlanView {
     int32_t *pair_rows;             // [n_pairs] rows of the pair's plan (prompt union + suffix)
     int32_t *pair_union_rows;       // [n_pairs] prompt rows only
     int64_t *pair_row_prefix;       // [n_pairs + 1] exclusive prefix of pair_rows over pairs
+    int32_t *tail_counter;          // [2] equal-range split: next tail chunk to hand out, and the count of
+                                    //   blocks that have left; zeroed with the plans, both reset themselves
 };
+
+// Equal-range split of the attention kernel: the padded row line [0, total) is cut into one fixed
+// range per block over its first part and, when the ranges are long enough to pay for it, into
+// small chunks over its last part (about a sixth), which blocks take from a counter as they
+// finish: blocks do not all stream at the same speed, and the chunks even out their finish.
+struct RangeSplit {
+    uint32_t total;                 // rows of the padded line (< 2^32: rows_total < 2^31, gaps add at most 2^26 * 16)
+    uint32_t fixed_rows;            // rows per fixed range
+    uint32_t fixed_end;             // the fixed ranges cover [0, fixed_end)
+    uint32_t chunk_rows;            // rows per tail chunk
+    int n_tail;                     // tail chunks covering [fixed_end, total)
+};
+__host__ __device__ __forceinline__ RangeSplit make_range_split(int64_t all_rows, int n_pairs, int span_penalty_rows,
+                                                                int min_rows_per_cta, int grid)
+{
+    RangeSplit sp;
+    sp.total = (uint32_t)(all_rows + (int64_t)span_penalty_rows * (n_pairs - 1));
+    uint32_t per = (sp.total + (uint32_t)grid - 1u) / (uint32_t)grid;
+    if (per < (uint32_t)min_rows_per_cta) per = (uint32_t)min_rows_per_cta;
+    if (per < 2048u) {                                      // short ranges: a chunk's fixed cost would not pay
+        sp.fixed_rows = per;
+        sp.fixed_end = sp.total;
+        sp.chunk_rows = 1u;
+        sp.n_tail = 0;
+        return sp;
+    }
+    sp.fixed_rows = per - per / 6u;
+    const uint64_t covered = (uint64_t)sp.fixed_rows * (uint32_t)grid;
+    sp.fixed_end = covered < sp.total ? (uint32_t)covered : sp.total;
+    const uint32_t tail = sp.total - sp.fixed_end;
+    uint32_t chunk = (tail + 2u * (uint32_t)grid - 1u) / (2u * (uint32_t)grid);
+    if (chunk < 256u) chunk = 256u;
+    sp.chunk_rows = chunk;
+    sp.n_tail = (int)((tail + chunk - 1u) / chunk);
+    return sp;
+}
+constexpr int kMaxTailChunksPerBlock = 2;                   // n_tail <= 2 * grid (+ 1 by rounding)
+
 
 // Scores of one (query head, sequence) form a row of y_stride floats, y_stride = the longest
 // sequence's team slots rounded up to a multiple of 4: rows are 16-byte aligned and their address

@@ -37,6 +37,7 @@ plan_kernel(PlanParams p, int max_words)
     for (int i = tid; i <= nseg; i += kPlanThreads) g_prefix[i] = sm.seg_prefix[i];
     for (int i = tid; i < nseg; i += kPlanThreads) { g_row[i] = sm.seg_row[i]; g_mask[i] = sm.seg_mask[i]; }
     if (tid == 0) { p.plan.pair_nseg[pair] = nseg; p.plan.pair_rows[pair] = rows; }
+    if (pair == 0 && tid < 2) p.plan.tail_counter[tid] = 0;
     trace_mark(p.in.trace, 2, 1);
 }
 
@@ -46,6 +47,7 @@ dense_plan_kernel(PlanParams p)
 {
     const uint32_t all_heads = (1u << p.in.bv.group) - 1u;
     const int pair = blockIdx.x * blockDim.x + threadIdx.x;
+    if (pair < 2) p.plan.tail_counter[pair] = 0;
     if (pair >= p.n_pairs) return;
     const int b = pair / p.in.bv.n_kv;
     const int cap = p.plan.seg_cap;
