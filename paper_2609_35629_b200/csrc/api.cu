@@ -717,6 +717,10 @@ int santapp_decode_attn(const santapp_geom *geom, const santapp_teams *teams, co
     rp.n_pairs = L.n_pairs;
     rp.status = dbg ? dbg->status : nullptr;
     rp.trace = dbg ? reinterpret_cast<unsigned long long *>(dbg->trace) : nullptr;
+    rp.tune_flags = 0;
+#ifdef SANTAPP_TUNE
+    if (const char *e = getenv("SANTAPP_SCORE_FLAGS")) rp.tune_flags = atoi(e);
+#endif
     cudaError_t err = cudaSuccess;
     if (rp.status && g_stage_mask == SANTAPP_STAGE_ALL) {
         // diagnostics only: a node of its own, so that no kernel both clears and raises the flags

@@ -121,6 +121,7 @@ struct ScoreParams {
     int n_pairs;
     int32_t *status;                // nullable
     unsigned long long *trace;      // nullable, see trace_mark
+    int tune_flags;                 // diagnostic builds only
 };
 
 // What the sampling step (headplan.cu) and the union step (pairplan.cuh) read and write.

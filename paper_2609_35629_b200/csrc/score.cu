@@ -71,6 +71,7 @@ __device__ __forceinline__ ScoreCtx score_ctx(const ScoreParams &p)
     c.seed_lo = p.seed_lo;
     c.seed_hi = p.seed_hi;
     c.stream_base = p.stream_base;
+    c.tune_flags = p.tune_flags;
     return c;
 }
 
@@ -79,6 +80,7 @@ template <int G, bool kHalf>
 __global__ void __launch_bounds__(kScoreThreads, 2)
 score32_kernel(ScoreParams p)
 {
+    __shared__ uint4 philox_words[kScoreThreads / 32][32];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = lane >> 2, c = lane & 3;
     const int pair = blockIdx.y;
@@ -98,7 +100,11 @@ score32_kernel(ScoreParams p)
     load_key_pieces(rep, base, M, g, c, kb);
     const uint32_t step = p.step + (p.step_dev ? *p.step_dev : 0u);
     const int32_t *csr = p.team_row_start + (size_t)j * (p.bv.teams_total + p.bv.n_seqs) + team0 + b;
-    score_tile<G, kHalf>(ctx, b, j, team0, M, base, csr + base, kb, qa, step, (float)p.scale, g, c);
+    TileScores ts;
+    uint32_t *words = reinterpret_cast<uint32_t *>(philox_words[warp]);
+    score_tile_front<G, kHalf>(ctx, b, j, M, base, csr + base, kb, qa, step, g, c, words, ts);
+    __syncwarp();                                      // every lane's Philox words are in shared memory
+    score_tile_back<G>(ts, (float)p.scale, g, c, words);
     trace_mark(p.trace, 0, 1);
 }
 
@@ -159,6 +165,7 @@ __global__ void __launch_bounds__(kScoreThreads, 2)
 score32_flat_kernel(ScoreParams p)
 {
     extern __shared__ uint4 score_ring[];
+    __shared__ uint4 philox_words[kScoreThreads / 32][32];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = lane >> 2, c = lane & 3;
     const long long n_tiles = (long long)p.bv.n_kv * p.tile_stride;
@@ -194,9 +201,11 @@ score32_flat_kernel(ScoreParams p)
     }
     TileCursor ahead = cursor_at(p, t_lo), here = ahead;
     long long t_ahead = t_lo;                                   // tile index under `ahead`
+    uint32_t pending = 0u;                                       // bit s: a bulk copy into stage s is in flight
     auto issue_tile = [&](int s) {
         int base;
         if (t_ahead < t_hi && locate_tile(p, seq_slot, ahead, base)) {
+            pending |= 1u << s;
             // the tile's keys are one contiguous run: a single bulk copy by lane 0
             if (lane == 0) {
                 const uint16_t *src = p.rep_keys + ((size_t)ahead.j * p.bv.teams_total + ahead.team0 + base) * kHeadDim;
@@ -222,6 +231,13 @@ score32_flat_kernel(ScoreParams p)
     int q_b = -1, q_j = -1;
     int stage = 0;
     uint32_t phases = 0u;                                        // bit s: parity of the next completion of stage s
+    uint32_t *words = reinterpret_cast<uint32_t *>(philox_words[warp]);
+#ifdef SANTAPP_TUNE
+    long long tk[4] = {0, 0, 0, 0}, tk0 = clock64();
+#define SCORE_TICK(i) { const long long now = clock64(); tk[i] += now - tk0; tk0 = now; }
+#else
+#define SCORE_TICK(i)
+#endif
     for (long long ti = t_lo; ti < t_hi; ++ti) {
         cp_async_wait_group<kScoreStages - 1>();                 // this lane's row offset of tile ti has landed
         __syncwarp();                                            // the row offsets come from other lanes
@@ -233,10 +249,20 @@ score32_flat_kernel(ScoreParams p)
                 if (++polls >= kScoreWaitPolls) break;
             }
             if (polls >= kScoreWaitPolls) {
+                // Never expected. The step is marked invalid; before the warp leaves it waits (again
+                // with a limit) for the copies it still has in flight, so that none of them lands
+                // in shared memory that no longer belongs to this block.
                 if (lane == 0 && p.status) atomicOr(p.status, 4);
+                for (int s = 0; s < kScoreStages; ++s) {
+                    if (!((pending >> s) & 1u)) continue;
+                    for (int again = 0; again < kScoreWaitPolls; ++again)
+                        if (mbar_try_wait(bars + 8 * s, (phases >> s) & 1u)) break;
+                }
                 break;
             }
+            pending &= ~(1u << stage);
             phases ^= 1u << stage;
+            SCORE_TICK(0)
             if (here.b != q_b || here.j != q_j) {
                 load_q_fragments<G>(ctx, here.b, here.j, g, c, qa);
                 q_b = here.b;
@@ -247,15 +273,28 @@ score32_flat_kernel(ScoreParams p)
             for (int t = 0; t < 2; ++t)
 #pragma unroll
                 for (int i = 0; i < 4; ++i) kb[t][i] = tile_of(stage)[(8 * t + g) * 16 + c + 4 * i];
-            score_tile<G, kHalf>(ctx, here.b, here.j, here.team0, here.M, base, csr_ring + stage * 32, kb, qa, step, scale, g, c);
+            SCORE_TICK(1)
+            TileScores ts;
+            score_tile_front<G, kHalf>(ctx, here.b, here.j, here.M, base, csr_ring + stage * 32, kb, qa, step, g, c, words, ts);
+            __syncwarp();                                        // every lane's Philox words are in shared memory
+            score_tile_back<G>(ts, scale, g, c, words);
+            SCORE_TICK(2)
         }
-        __syncwarp();                                            // every lane is done with the stage's row offsets
+        __syncwarp();                                            // every lane is done with the stage's row offsets and the words
         // refill the stage just consumed (its pieces are in registers and already used above)
         issue_tile(stage);
         advance(p, here);
         stage = stage + 1 == kScoreStages ? 0 : stage + 1;
+        SCORE_TICK(3)
     }
     cp_async_wait_group<0>();
+#ifdef SANTAPP_TUNE
+    if (p.trace && lane == 0 && blockIdx.x < 8) {
+        unsigned long long *o = p.trace + ((size_t)blockIdx.x * 8 + warp) * 8;
+        o[0] = (unsigned long long)(t_hi - t_lo);
+        for (int i = 0; i < 4; ++i) o[1 + i] = (unsigned long long)tk[i];
+    }
+#endif
 }
 
 // One block per (sequence, KV head): largest |element| among the pair's representative keys.

@@ -24,22 +24,23 @@ struct ScoreCtx {
     int n_q, n_seqs;
     const uint16_t *q;              // [n_seqs][n_q][128]
     uint32_t seed_lo, seed_hi, stream_base;
+    int tune_flags;                 // diagnostic builds only: bits switch parts of the tile off
 };
 
+// D (16 teams x 8 heads) += A (16 teams x 16 dims, row) * B (16 dims x 8 heads, col), fp32 accumulation.
 template <bool kHalf>
-__device__ __forceinline__ void mma_score(float (&d)[4], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1)
+__device__ __forceinline__ void mma_score(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1)
 {
-    // A rows 8..15 are zero (a1 = a3 = 0): only heads 0..7 exist
     if constexpr (kHalf)
         asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
                      "{%0,%1,%2,%3};"
                      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-                     : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1));
+                     : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
     else
         asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
                      "{%0,%1,%2,%3};"
                      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-                     : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1));
+                     : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
 // Gumbel(0,1) in fp32 from a 32-bit word: u = (x + 0.5) / 2^32, G = -log(-log u), to an absolute
@@ -90,62 +91,83 @@ __device__ __forceinline__ void load_key_pieces(const uint16_t *rep, int base, i
     }
 }
 
-// Scores of one tile of 16 teams (two n-tiles of 8; B row n = team base + 8 t + g) from the key
-// pieces kb of this lane: writes Y32 for the G heads.
-// csr_tile points at the 17 row offsets of the tile's teams (global or shared memory).
+// What the first half of a tile's work leaves for the second half (all in registers).
+struct TileScores {
+    float dot[4];                   // q . l for (team g, head 2c), (g, 2c+1), (g+8, 2c), (g+8, 2c+1)
+    float log_lo, log_hi;           // log n of teams g and g + 8
+    float *y_row[2];                // score rows of heads 2c and 2c + 1 for the tile's sequence
+    int t_lo;                       // team base + g; -1 when the tile is empty
+    int M;
+};
+
+// Scores of one tile of 16 teams from the key pieces kb of this lane (kb[t][i]: 16-byte piece
+// c + 4 i of the key of team base + 8 t + g), in two halves so that a kernel walking many tiles can
+// run the tensor-core instructions of one tile beside the arithmetic of the previous one.
+// The 16 teams are the M rows of the tensor-core tile and the query heads its 8 columns, so one
+// instruction per 16 dimensions covers the whole tile (the legacy tensor-core instruction is slow
+// on this GPU, and a tile's time is mostly spent waiting for them). A lane ends up with the
+// scores of teams g and g + 8 for heads 2 c and 2 c + 1.
+// csr_tile points at the 17 row offsets of the tile's teams (global or shared memory);
+// words_smem: 128 words of this warp's own shared memory (the tile's Philox words, [head][team]);
+// the caller orders writes and reads of that buffer (__syncwarp) between the two halves.
 template <int G, bool kHalf>
-__device__ __forceinline__ void score_tile(const ScoreCtx &p, int b, int j, int64_t team0, int M, int base,
-                                           const int32_t *csr_tile, const uint4 (&kb)[2][4], const uint32_t (&qa)[8][2],
-                                           uint32_t step, float scale, int g, int c)
+__device__ __forceinline__ void score_tile_front(const ScoreCtx &p, int b, int j, int M, int base, const int32_t *csr_tile,
+                                                 const uint4 (&kb)[2][4], const uint32_t (&qa)[8][2], uint32_t step, int g,
+                                                 int c, uint32_t *words_smem, TileScores &out)
 {
-    const uint32_t head = (uint32_t)(j * G + (g < G ? g : 0));
-    float *y = p.y32 + ((size_t)head * p.n_seqs + b) * p.y_stride;
-    // team sizes of this lane's four teams (teams base + 8 t + 2 c, + 1)
-    int n_team[2][2];
-#pragma unroll
-    for (int t = 0; t < 2; ++t) {
-        const int t0 = base + 8 * t + 2 * c, o = 8 * t + 2 * c;
-        const int r0 = t0 < M ? csr_tile[o] : 0, r1 = t0 < M ? csr_tile[o + 1] : 1, r2 = t0 + 1 < M ? csr_tile[o + 2] : 2;
-        n_team[t][0] = r1 - r0;
-        n_team[t][1] = r2 - r1;
-    }
-    float acc[2][4];
-#pragma unroll
-    for (int t = 0; t < 2; ++t) {
-        acc[t][0] = acc[t][1] = acc[t][2] = acc[t][3] = 0.f;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            mma_score<kHalf>(acc[t], qa[2 * i][0], qa[2 * i][1], kb[t][i].x, kb[t][i].y);
-            mma_score<kHalf>(acc[t], qa[2 * i + 1][0], qa[2 * i + 1][1], kb[t][i].z, kb[t][i].w);
-        }
-    }
-    // One Philox block covers four consecutive teams of a head: teams base + 8 t + {0..3} belong
-    // to thread columns 0 and 1, + {4..7} to columns 2 and 3. The even column computes the block
-    // of n-tile 0, the odd one that of n-tile 1, and the two exchange halves.
-    const int my_t = c & 1;
-    const uint4 words = philox4x32_10(
-        make_uint4((uint32_t)(base + 8 * my_t + 4 * (c >> 1)) >> 2, step, head, p.stream_base + (uint32_t)b),
-        p.seed_lo, p.seed_hi);
-    // this lane needs words {2 (c & 1), 2 (c & 1) + 1} of both n-tiles' blocks
-    uint32_t w[2][2];
+    const int lane = 4 * g + c;
+    // One Philox block covers four consecutive teams of a head: 4 blocks per head and tile, lane
+    // 4 h + tb computes the block of head h, teams base + 4 tb .. + 3, and leaves its words in
+    // shared memory at [h][4 tb .. 4 tb + 3].
     {
-        const uint32_t give0 = (c & 1) ? words.x : words.z, give1 = (c & 1) ? words.y : words.w;
-        const uint32_t got0 = __shfl_xor_sync(0xFFFFFFFFu, give0, 1), got1 = __shfl_xor_sync(0xFFFFFFFFu, give1, 1);
-        const uint32_t keep0 = (c & 1) ? words.z : words.x, keep1 = (c & 1) ? words.w : words.y;
-        w[0][0] = my_t ? got0 : keep0;
-        w[0][1] = my_t ? got1 : keep1;
-        w[1][0] = my_t ? keep0 : got0;
-        w[1][1] = my_t ? keep1 : got1;
+        const int h = lane >> 2, tb = lane & 3;
+        uint4 words = make_uint4((uint32_t)(base >> 2) + (uint32_t)tb, step, (uint32_t)(j * G + (h < G ? h : 0)),
+                                 p.stream_base + (uint32_t)b);
+#ifdef SANTAPP_TUNE
+        if (!(p.tune_flags & 2))
+#endif
+        words = philox4x32_10(words, p.seed_lo, p.seed_hi);
+        reinterpret_cast<uint4 *>(words_smem)[lane] = words;
     }
-    // acc[t][0], acc[t][1]: head g, teams base + 8 t + 2 c, + 1
-    if (g < G) {
+    // sizes of this lane's two teams
+    const int t_lo = base + g, t_hi = base + g + 8;
+    const int n_lo = t_lo < M ? csr_tile[g + 1] - csr_tile[g] : 1;
+    const int n_hi = t_hi < M ? csr_tile[g + 9] - csr_tile[g + 8] : 1;
+    out.log_lo = __logf((float)n_lo);
+    out.log_hi = __logf((float)n_hi);
+    out.t_lo = t_lo;
+    out.M = M;
 #pragma unroll
-        for (int t = 0; t < 2; ++t) {
-            const int t0 = base + 8 * t + 2 * c;
-            const float y0 = __logf((float)n_team[t][0]) + acc[t][0] * scale + gumbel32_from_word(w[t][0]);
-            const float y1 = __logf((float)n_team[t][1]) + acc[t][1] * scale + gumbel32_from_word(w[t][1]);
-            if (t0 + 1 < M) *reinterpret_cast<float2 *>(y + t0) = make_float2(y0, y1);      // t0 is even, the row 16-byte aligned
-            else if (t0 < M) y[t0] = y0;
+    for (int e = 0; e < 2; ++e) {
+        const int h = min(2 * c + e, G - 1);
+        out.y_row[e] = p.y32 + ((size_t)(j * G + h) * p.n_seqs + b) * p.y_stride;
+    }
+    // two accumulators (even and odd steps of 16 dimensions)
+    float acc0[4] = {0.f, 0.f, 0.f, 0.f}, acc1[4] = {0.f, 0.f, 0.f, 0.f};
+#ifdef SANTAPP_TUNE
+    if (p.tune_flags & 1) { acc0[0] = __uint_as_float(kb[0][0].x ^ kb[1][1].y); acc0[2] = __uint_as_float(kb[0][2].z ^ kb[1][3].w); } else
+#endif
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        mma_score<kHalf>(acc0, kb[0][i].x, kb[1][i].x, kb[0][i].y, kb[1][i].y, qa[2 * i][0], qa[2 * i][1]);
+        mma_score<kHalf>(acc1, kb[0][i].z, kb[1][i].z, kb[0][i].w, kb[1][i].w, qa[2 * i + 1][0], qa[2 * i + 1][1]);
+    }
+#pragma unroll
+    for (int e = 0; e < 4; ++e) out.dot[e] = acc0[e] + acc1[e];
+}
+
+template <int G>
+__device__ __forceinline__ void score_tile_back(const TileScores &t, float scale, int g, int c, const uint32_t *words_smem)
+{
+    if (t.t_lo < 0) return;
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {                          // head 2 c + e
+        const int h = 2 * c + e;
+        if (h < G) {
+            const float y_lo = t.log_lo + t.dot[e] * scale + gumbel32_from_word(words_smem[h * 16 + g]);
+            const float y_hi = t.log_hi + t.dot[2 + e] * scale + gumbel32_from_word(words_smem[h * 16 + g + 8]);
+            if (t.t_lo < t.M) t.y_row[e][t.t_lo] = y_lo;
+            if (t.t_lo + 8 < t.M) t.y_row[e][t.t_lo + 8] = y_hi;
         }
     }
 }
