@@ -384,6 +384,37 @@ def minibatch_kmeans(keys, k, batch=4096, max_iter=100, patience=10, ratio=0.01,
     return centres, int(steps)
 
 
+def shared_latent_records(rows, d_latent, P, R):
+    """Teams of a shared-latent cache (appendix "Token sparsity after latent compression"): rows
+    [N, d_latent + d_rope] hold a content latent followed by a rotary key; contiguous parents
+    (Algorithm 4) and Algorithm 2 run on the content latents alone, and a team's routing key is
+    its representative's whole row. Returns (team_start, team_member, rep_rows)."""
+    rows = _f64(rows)
+    ts, tm, rep = build_teams_contiguous(np.ascontiguousarray(rows[:, :d_latent]), P, R)
+    return ts, tm, np.ascontiguousarray(rows[rep])
+
+
+def shared_latent_step(q, rows, d_latent, team_start, team_member, rep_rows, suffix_rows, K, seed, step, stream,
+                       scale, n_threads=1):
+    """Algorithm 1 for the n_q heads that share one row per token: a head's logit is its query
+    against the whole row (latent and rotary part), its value the row's latent part. Argument
+    marshalling only: one KV "head", keys = rows, values = rows with the rotary columns zeroed
+    (they add exact zeros to every sum). Returns the StepResult with o [n_q, d_latent]."""
+    rows, q = _f64(rows), _f64(q)
+    vals = rows.copy()
+    vals[:, d_latent:] = 0.0
+    ks = vs = None
+    if suffix_rows is not None and len(suffix_rows):
+        ks = _f64(suffix_rows)[None]
+        vs = ks.copy()
+        vs[:, :, d_latent:] = 0.0
+    M = np.array([len(team_start) - 1], dtype=np.int32)
+    r = decode_step(q, rows[None], vals[None], M, _i32(team_start)[None], _i32(team_member)[None], _f64(rep_rows)[None],
+                    ks, vs, K, seed, step, stream, scale, n_threads=n_threads)
+    r.o = np.ascontiguousarray(r.o[:, :d_latent])
+    return r
+
+
 def mla_logical_access_pct(r, u, d):
     """Shared-row logical access of Eq. (mla-logical-access), pooled over the calls."""
     r, u, d = (np.ascontiguousarray(a, dtype=np.int64) for a in (r, u, d))
