@@ -41,9 +41,9 @@ N_STEP_INPUTS = 8          # distinct (query, suffix length, step) inputs cycled
 # recorded figure, not one measured by this run: it is reported as `traffic` together with
 # `traffic_kind`, and left out (null) for any other variant of the workload.
 NCU_TRAFFIC_BYTES = {
-    "qwen7b_b1_32k": 34.61e6,
-    "qwen7b_b8_32k": 409.0e6,
-    "ragged": 1036.2e6,
+    "qwen7b_b1_32k": 34.57e6,
+    "qwen7b_b8_32k": 405.3e6,
+    "ragged": 1037.1e6,
 }
 
 

@@ -246,15 +246,18 @@ int32_t santapp_kmeans_parent_count(int32_t prompt_len, int32_t parent_size);
  *   workspace        device, >= santapp_kmeans_fit_workspace_bytes(...)
  * batch_size > 4096, or an initialisation sample above 28672 keys (more than 9557 centres in a
  * sequence): SANTAPP_ERR_UNSUPPORTED. The call enqueues a few kernels per centre and per
- * step on `stream`, and every 16 steps waits for the stream to learn whether any fit is still
- * running (most stop long before the step limit): it blocks the calling thread for most of the
- * fit and must not be issued during a stream capture.
+ * step on `stream`. By default it waits for the stream every 16 steps to learn whether any fit
+ * is still running (most stop long before the step limit), so it blocks the calling thread for
+ * most of the fit; with opts->no_host_poll = 1 it never waits and enqueues every step up to the
+ * limit instead (the result is the same: a stopped fit's later steps do nothing).
  */
 typedef struct santapp_kmeans_opts {
     int32_t batch_size;           /* paper: 4096 */
     int32_t max_iter;             /* paper: 100 */
     int32_t patience;             /* paper: 10 */
-    int32_t reserved;             /* set to 0 */
+    int32_t no_host_poll;         /* 0: the call looks at the fits' stop flags every 16 steps (and waits for
+                                     the stream to do so); 1: it never waits: every step up to the limit is
+                                     enqueued, steps of a fit that has stopped return at once */
     double reassignment_ratio;    /* paper: 0.01; 0 switches reassignment off */
     uint64_t seed;                /* paper: 0 */
     uint32_t stream_base;
@@ -398,7 +401,7 @@ int santapp_dense_decode_attn(const santapp_geom *geom, const santapp_teams *tea
  *   - Limit: if santapp_dense_workspace_bytes(geom, teams) exceeds SANTAPP_STATIC_SCRATCH_BYTES
  *     the call returns SANTAPP_ERR_STATIC_SCRATCH and launches nothing (the text of
  *     santapp_last_cuda_error says how many bytes were needed). On a 148-SM GPU with 7 query
- *     heads per KV head the 2 MiB array covers about 400 (sequence, KV head) pairs.
+ *     heads per KV head the 2 MiB array covers about 110 (sequence, KV head) pairs.
  *   - Set-up: the first call on each device looks up the array's device address (the device
  *     must be current, as for every call) and remembers it for the life of the process. Make
  *     that first call outside any stream capture. The remembered address belongs to the

@@ -68,7 +68,7 @@ class CTeams(ctypes.Structure):
 
 class CKmeansOpts(ctypes.Structure):
     _fields_ = [("batch_size", ctypes.c_int32), ("max_iter", ctypes.c_int32), ("patience", ctypes.c_int32),
-                ("reserved", ctypes.c_int32), ("reassignment_ratio", ctypes.c_double), ("seed", ctypes.c_uint64),
+                ("no_host_poll", ctypes.c_int32), ("reassignment_ratio", ctypes.c_double), ("seed", ctypes.c_uint64),
                 ("stream_base", ctypes.c_uint32), ("reserved2", ctypes.c_uint32)]
 
 
@@ -276,12 +276,12 @@ def santapp_kmeans_parent_count(prompt_len: int, parent_size: int) -> int:
 
 def santapp_kmeans_fit(geom: Geometry, prompt_len, n_centres, k_prompt: torch.Tensor, batch_size: int = 4096,
                        max_iter: int = 100, patience: int = 10, reassignment_ratio: float = 0.01, seed: int = 0,
-                       stream_base: int = 0, stream=None):
+                       stream_base: int = 0, stream=None, no_host_poll: bool = False):
     """Minibatch k-means fit per (sequence, KV head); the defaults are the paper's settings.
     Returns (centres fp32 [n_kv_heads, sum(n_centres), d], steps int32 [n_kv_heads, n_seqs])."""
     L = load_library()
     g = geom.c()
-    o = CKmeansOpts(batch_size, max_iter, patience, 0, reassignment_ratio, seed, stream_base, 0)
+    o = CKmeansOpts(batch_size, max_iter, patience, 1 if no_host_poll else 0, reassignment_ratio, seed, stream_base, 0)
     n, c = _i32_array(prompt_len), _i32_array(n_centres)
     need = int(L.santapp_kmeans_fit_workspace_bytes(ctypes.byref(g), n, c, ctypes.byref(o)))
     if need == 0:

@@ -602,6 +602,7 @@ int santapp_kmeans_fit(const santapp_geom *geom, const int32_t *prompt_len_host,
     p.max_rows_per_seq = L.max_rows;
     p.batch = opts->batch_size;
     p.patience = opts->patience;
+    p.no_host_poll = opts->no_host_poll != 0;
     p.ratio = opts->reassignment_ratio;
     p.seed_lo = (uint32_t)(opts->seed & 0xFFFFFFFFull);
     p.seed_hi = (uint32_t)(opts->seed >> 32);

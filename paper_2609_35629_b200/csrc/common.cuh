@@ -280,6 +280,7 @@ struct KmeansState {
 struct KmeansParams {
     int n_seqs, n_kv, elem, max_rows_per_seq;
     int batch, patience;
+    int no_host_poll;                       // never wait for the stream inside the call
     double ratio;
     uint32_t seed_lo, seed_hi, stream_base;
     int k_max, n_init_max, trials_max, t_max_max;   // maxima over the sequences

@@ -462,7 +462,7 @@ cudaError_t run_fit(const KmeansParams &p, cudaStream_t s)
         KM_CHECK();
         km_control_kernel<kHalf><<<dim3(B, H), 32, control_smem, s>>>(p, t);
         KM_CHECK();
-        if ((t + 1) % kPollEvery == 0 && t + 1 < p.t_max_max) {
+        if (!p.no_host_poll && (t + 1) % kPollEvery == 0 && t + 1 < p.t_max_max) {
             // most fits stop long before the step limit: ask the device how many are still running
             // (the copy into pageable memory returns when it has completed)
             int active = 1;

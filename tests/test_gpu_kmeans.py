@@ -22,7 +22,7 @@ def _fit_both(spec, n_centres, **opts):
     torch.cuda.synchronize()
     centres, steps = centres.cpu().numpy(), steps.cpu().numpy()
     base = opts.get("stream_base", 0)
-    o = {kk: v for kk, v in opts.items() if kk != "stream_base"}
+    o = {kk: v for kk, v in opts.items() if kk not in ("stream_base", "no_host_poll")}
     o = {"batch": o.pop("batch_size", 4096), "ratio": o.pop("reassignment_ratio", 0.01), **o}
     row0 = c0 = 0
     for b, kc in enumerate(n_centres):
@@ -51,6 +51,17 @@ def test_fit_with_reassignment_every_period_and_short_patience():
     spec = synth.spec_small_gqa(prompt=(700,), n_seqs=1, suffix0=(0,))
     _fit_both(spec, [13], batch_size=512, reassignment_ratio=0.9, patience=2, max_iter=30, seed=1 << 40)
     _fit_both(spec, [13], batch_size=64, reassignment_ratio=0.0, patience=10 ** 6, max_iter=2)
+
+
+def test_fit_without_host_polling_gives_the_same_centres():
+    """With no_host_poll the call never waits for the stream: every step up to the limit is enqueued
+    and the steps of a fit that has already stopped do nothing, so centres and step counts stay
+    those of the oracle (two sequences whose fits stop at different steps)."""
+    spec = synth.spec_small_gqa(prompt=(1536, 1000))
+    spec.n_clusters = 24
+    _, _, steps = _fit_both(spec, [24, 9], batch_size=256, seed=3, stream_base=11, max_iter=20, no_host_poll=True)
+    assert len(set(steps.ravel().tolist())) > 1
+    assert steps.max() < 20 * 6                                 # the fits stopped before the limit
 
 
 def test_fit_fp16_inputs():
