@@ -5,7 +5,7 @@ merge) runs in the library's CUDA kernels. PyTorch is used for device memory and
 streams. There is no CPU fallback: if the library is missing or cannot be loaded
 the first call raises.
 
-The functions keep the names of the C entry points (include/santapp.h).
+The functions keep the names of the C entry points (include/santapp.h, include/santapp_latent.h).
 """
 import ctypes
 import os
@@ -34,7 +34,10 @@ EXPORTS = [
     "santapp_kmeans_parent_count", "santapp_assign_parents_workspace_bytes", "santapp_assign_parents",
     "santapp_parent_teams_sizes", "santapp_build_teams_parents", "santapp_build_groups_mean_parents",
     "santapp_kmeans_fit_workspace_bytes", "santapp_kmeans_fit",
+    "santapp_latent_sizes", "santapp_latent_build_teams", "santapp_latent_decode_workspace_bytes",
+    "santapp_latent_decode_attn", "santapp_latent_dense_workspace_bytes", "santapp_latent_dense_decode_attn",
 ]
+LATENT_DIM, LATENT_ROPE_DIM, LATENT_ROW = 512, 64, 576
 
 STAGE_ROUTE, STAGE_SELECT, STAGE_ATTEND, STAGE_MERGE, STAGE_ALL = 1, 2, 4, 8, 15
 
@@ -78,6 +81,18 @@ class CDebug(ctypes.Structure):
 
 
 _lib = None
+
+
+class CLatentGeom(ctypes.Structure):
+    _fields_ = [("n_seqs", ctypes.c_int32), ("n_heads", ctypes.c_int32), ("parent_size", ctypes.c_int32),
+                ("reps_per_parent", ctypes.c_int32)]
+
+
+class CLatentTeams(ctypes.Structure):
+    _fields_ = [("rows_packed", ctypes.c_void_p), ("rep_rows", ctypes.c_void_p), ("team_row_start", ctypes.c_void_p),
+                ("row_token", ctypes.c_void_p), ("seq_row_off", ctypes.c_void_p), ("seq_team_off", ctypes.c_void_p),
+                ("rep_abs_max", ctypes.c_void_p), ("rows_total", ctypes.c_int64), ("teams_total", ctypes.c_int64),
+                ("max_teams_per_seq", ctypes.c_int32), ("max_rows_per_seq", ctypes.c_int32)]
 
 
 def load_library(path: Optional[str] = None):
@@ -140,6 +155,20 @@ def load_library(path: Optional[str] = None):
     L.santapp_dense_decode_attn_noalloc.argtypes = [ctypes.POINTER(CGeom), ctypes.POINTER(CTeams), vp, vp, vp, vp,
                                                     i32, f32, vp, vp]
     L.santapp_dense_decode_attn_noalloc.restype = ctypes.c_int
+    LG, LT = ctypes.POINTER(CLatentGeom), ctypes.POINTER(CLatentTeams)
+    L.santapp_latent_sizes.argtypes = [LG, ctypes.POINTER(i32), ctypes.POINTER(CSizes)]
+    L.santapp_latent_sizes.restype = ctypes.c_int
+    L.santapp_latent_build_teams.argtypes = [LG, ctypes.POINTER(i32), vp, LT, vp, sz, vp]
+    L.santapp_latent_build_teams.restype = ctypes.c_int
+    L.santapp_latent_decode_workspace_bytes.argtypes = [LG, LT, i32, i32]
+    L.santapp_latent_decode_workspace_bytes.restype = sz
+    L.santapp_latent_dense_workspace_bytes.argtypes = [LG, LT]
+    L.santapp_latent_dense_workspace_bytes.restype = sz
+    L.santapp_latent_decode_attn.argtypes = [LG, LT, vp, vp, vp, i32, i32, u64, u32, vp, u32, f32, vp,
+                                             ctypes.POINTER(CDebug), vp, sz, vp]
+    L.santapp_latent_decode_attn.restype = ctypes.c_int
+    L.santapp_latent_dense_decode_attn.argtypes = [LG, LT, vp, vp, vp, i32, f32, vp, vp, sz, vp]
+    L.santapp_latent_dense_decode_attn.restype = ctypes.c_int
     if path is None:
         _lib = L
     return L
@@ -432,6 +461,119 @@ def santapp_dense_decode_attn_noalloc(geom: Geometry, teams: Teams, q: torch.Ten
     _check(L.santapp_dense_decode_attn_noalloc(ctypes.byref(g), ctypes.byref(teams.c), _ptr(q), _ptr(k_suffix),
                                                _ptr(v_suffix), _ptr(suffix_len), cap, scale, _ptr(out),
                                                _stream_ptr(stream)))
+    return out
+
+
+# ------------------------------------------------------------------------------------------------
+# Shared-latent rows (include/santapp_latent.h)
+# ------------------------------------------------------------------------------------------------
+@dataclass
+class LatentGeometry:
+    n_seqs: int
+    n_heads: int = 16
+    parent_size: int = 16
+    reps_per_parent: int = 4
+
+    def c(self) -> CLatentGeom:
+        return CLatentGeom(self.n_seqs, self.n_heads, self.parent_size, self.reps_per_parent)
+
+
+class LatentTeams:
+    """Team records of shared-latent rows: device tensors plus the C struct that points at them."""
+
+    def __init__(self, geom: LatentGeometry, sizes: Sizes, device):
+        self.geom = geom
+        self.sizes = sizes
+        self.rows_packed = torch.empty((sizes.rows_total, LATENT_ROW), dtype=torch.bfloat16, device=device)
+        self.rep_rows = torch.empty((sizes.teams_total, LATENT_ROW), dtype=torch.bfloat16, device=device)
+        self.team_row_start = torch.empty(sizes.teams_total + geom.n_seqs, dtype=torch.int32, device=device)
+        self.row_token = torch.empty(sizes.rows_total, dtype=torch.int32, device=device)
+        self.seq_row_off = torch.empty(geom.n_seqs + 1, dtype=torch.int64, device=device)
+        self.seq_team_off = torch.empty(geom.n_seqs + 1, dtype=torch.int64, device=device)
+        self.rep_abs_max = torch.empty(geom.n_seqs, dtype=torch.float32, device=device)
+        self.c = CLatentTeams(self.rows_packed.data_ptr(), self.rep_rows.data_ptr(), self.team_row_start.data_ptr(),
+                              self.row_token.data_ptr(), self.seq_row_off.data_ptr(), self.seq_team_off.data_ptr(),
+                              self.rep_abs_max.data_ptr(), sizes.rows_total, sizes.teams_total,
+                              sizes.max_teams_per_seq, sizes.max_rows_per_seq)
+
+
+def santapp_latent_sizes(geom: LatentGeometry, prompt_len) -> Sizes:
+    L = load_library()
+    out = CSizes()
+    g = geom.c()
+    _check(L.santapp_latent_sizes(ctypes.byref(g), _i32_array(prompt_len), ctypes.byref(out)))
+    return Sizes(out.rows_total, out.teams_total, out.max_teams_per_seq, out.max_rows_per_seq,
+                 out.team_row_start_elems, out.build_workspace_bytes)
+
+
+def santapp_latent_build_teams(geom: LatentGeometry, prompt_len, rows_prompt: torch.Tensor, stream=None) -> LatentTeams:
+    """rows_prompt: bf16 CUDA tensor [rows_total, 576] in token order (512 latent values, 64 rotary)."""
+    L = load_library()
+    sizes = santapp_latent_sizes(geom, prompt_len)
+    teams = LatentTeams(geom, sizes, rows_prompt.device)
+    ws = torch.empty(max(sizes.build_workspace_bytes, 256), dtype=torch.uint8, device=rows_prompt.device)
+    g = geom.c()
+    _check(L.santapp_latent_build_teams(ctypes.byref(g), _i32_array(prompt_len), _ptr(rows_prompt), ctypes.byref(teams.c),
+                                        _ptr(ws), ws.numel(), _stream_ptr(stream)))
+    teams._build_ws = ws
+    return teams
+
+
+def santapp_latent_decode_workspace_bytes(geom: LatentGeometry, teams: LatentTeams, n_sample: int, suffix_cap: int) -> int:
+    g = geom.c()
+    return int(load_library().santapp_latent_decode_workspace_bytes(ctypes.byref(g), ctypes.byref(teams.c), n_sample,
+                                                                    suffix_cap))
+
+
+def santapp_latent_dense_workspace_bytes(geom: LatentGeometry, teams: LatentTeams) -> int:
+    g = geom.c()
+    return int(load_library().santapp_latent_dense_workspace_bytes(ctypes.byref(g), ctypes.byref(teams.c)))
+
+
+class LatentDebugBuffers(DebugBuffers):
+    """Diagnostics of a shared-latent step: per (sequence, head) samples, per sequence union rows."""
+
+    def __init__(self, geom: LatentGeometry, n_sample: int, device):
+        super().__init__(Geometry(geom.n_seqs, geom.n_heads, 1), n_sample, device)
+
+
+def santapp_latent_decode_attn(geom: LatentGeometry, teams: LatentTeams, q: torch.Tensor,
+                               suffix_rows: Optional[torch.Tensor], suffix_len: Optional[torch.Tensor], n_sample: int,
+                               seed: int, step: int, scale: float, stream_base: int = 0,
+                               out: Optional[torch.Tensor] = None, debug: Optional[DebugBuffers] = None,
+                               workspace: Optional[torch.Tensor] = None, stream=None,
+                               step_dev: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """q bf16 [B, H, 576]; suffix_rows bf16 [B, cap, 576]; suffix_len int32 [B] (device). Returns fp32 [B, H, 512]."""
+    L = load_library()
+    cap = 0 if suffix_rows is None else int(suffix_rows.shape[1])
+    if out is None:
+        out = torch.empty((geom.n_seqs, geom.n_heads, LATENT_DIM), dtype=torch.float32, device=q.device)
+    if workspace is None:
+        workspace = torch.empty(santapp_latent_decode_workspace_bytes(geom, teams, n_sample, cap), dtype=torch.uint8,
+                                device=q.device)
+    g = geom.c()
+    _check(L.santapp_latent_decode_attn(ctypes.byref(g), ctypes.byref(teams.c), _ptr(q), _ptr(suffix_rows),
+                                        _ptr(suffix_len), cap, n_sample, ctypes.c_uint64(seed), step, _ptr(step_dev),
+                                        stream_base, scale, _ptr(out),
+                                        ctypes.byref(debug.c) if debug is not None else None, _ptr(workspace),
+                                        workspace.numel(), _stream_ptr(stream)))
+    return out
+
+
+def santapp_latent_dense_decode_attn(geom: LatentGeometry, teams: LatentTeams, q: torch.Tensor,
+                                     suffix_rows: Optional[torch.Tensor], suffix_len: Optional[torch.Tensor],
+                                     scale: float, out: Optional[torch.Tensor] = None,
+                                     workspace: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    L = load_library()
+    cap = 0 if suffix_rows is None else int(suffix_rows.shape[1])
+    if out is None:
+        out = torch.empty((geom.n_seqs, geom.n_heads, LATENT_DIM), dtype=torch.float32, device=q.device)
+    if workspace is None:
+        workspace = torch.empty(santapp_latent_dense_workspace_bytes(geom, teams), dtype=torch.uint8, device=q.device)
+    g = geom.c()
+    _check(L.santapp_latent_dense_decode_attn(ctypes.byref(g), ctypes.byref(teams.c), _ptr(q), _ptr(suffix_rows),
+                                              _ptr(suffix_len), cap, scale, _ptr(out), _ptr(workspace),
+                                              workspace.numel(), _stream_ptr(stream)))
     return out
 
 

@@ -25,6 +25,17 @@ int cuda_fail(cudaError_t err, const char *where)
 
 inline size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
 
+}  // namespace
+
+// The same bookkeeping for entry points that live in other files.
+namespace santapp {
+int note_cuda_failure(cudaError_t err, const char *where) { return cuda_fail(err, where); }
+void note_launch_count(int n) { g_launches = n; }
+int current_stage_mask() { return g_stage_mask; }
+}  // namespace santapp
+
+namespace {
+
 // Device arrays are read and written 16 bytes at a time (8 for the 64-bit offsets, 4 for the 32-bit
 // tables): a pointer that is not aligned accordingly would fault on the device, so it is refused here.
 inline bool misaligned(const void *p, size_t a) { return p != nullptr && (reinterpret_cast<uintptr_t>(p) % a) != 0; }

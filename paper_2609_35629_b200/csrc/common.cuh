@@ -202,6 +202,12 @@ inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block
     return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
+// Per-thread bookkeeping behind santapp_last_cuda_error / santapp_last_launch_count / santapp_set_stage_mask
+// (api.cu), for entry points defined in other files.
+int note_cuda_failure(cudaError_t err, const char *where);     // records the text, returns SANTAPP_ERR_CUDA
+void note_launch_count(int n);
+int current_stage_mask();
+
 // ---------------------------------------------------------------------------------------------
 // Host launchers (each returns the cudaError_t of its launches).
 // ---------------------------------------------------------------------------------------------

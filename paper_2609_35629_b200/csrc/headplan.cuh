@@ -28,8 +28,10 @@ constexpr int kListCap = 132;           // running top list: K + 1 <= 129 entrie
 constexpr int kDotLanes = 8;            // threads that share one candidate's dot product
 constexpr int kWindow = 255;            // histogram bins per pass of the bound
 
-struct alignas(16) HeadSmem {
-    double q64[kDotLanes][18];          // query in fp64: [16-dim slice][16 + pad] (pad: conflict-free LDS.128)
+// kDim: values per routing key (128 for K rows, 576 for shared-latent rows); a multiple of 64.
+template <int kDim>
+struct alignas(16) HeadSmemT {
+    double q64[kDotLanes][kDim / kDotLanes + 2];   // query in fp64: [slice of kDim / 8 dims][+ pad] (pad: conflict-free LDS.128)
     double cand_y[kCandCap + 2];        // dot products, then exact Y; read in pairs
     double cand_phi[kCandCap];          // log n_g, then phi_g
     double cand_g[kCandCap];            // Gumbel term
@@ -43,6 +45,7 @@ struct alignas(16) HeadSmem {
     float red_max[kMaxHeadWarps], red_sum[kMaxHeadWarps];
     int n_cand, bound_bin, bound_below, bound_total;
 };
+using HeadSmem = HeadSmemT<kHeadDim>;
 
 // Guard on |Y32 - Y|: tensor-core accumulation of exact 16-bit products in fp32 (relative to the sum
 // of magnitudes, bounded by scale * |q|_1 * max|l|), plus the fp32 logarithm and Gumbel terms.
@@ -62,10 +65,14 @@ __device__ __forceinline__ int score_bin(float top, float v)
 // block's warps compute dot products, the second half the Gumbel terms. Nothing is done (and
 // nothing written) when K >= M: every team is then read with c = 1 and nothing is drawn.
 // kScoreRegs: 16-byte pieces of the score row a thread keeps in registers.
-template <int kT, int kScoreRegs, bool kHalf>
-__device__ __forceinline__ void select_head(const PlanInputs &in, int hq, HeadSmem &sm)
+template <int kT, int kScoreRegs, bool kHalf, int kDim = kHeadDim>
+__device__ __forceinline__ void select_head(const PlanInputs &in, int hq, HeadSmemT<kDim> &sm)
 {
+    static_assert(kDim % 64 == 0, "eight lanes share a key, each takes whole 16-byte pieces");
     constexpr int kHeadWarps = kT / 32, kDotWarps = kHeadWarps / 2;
+    constexpr int kSlice = kDim / kDotLanes;                          // dims per lane of a dot product
+    constexpr int kPieces = kSlice / 8;                               // 16-byte pieces per lane
+    constexpr int kQRegs = (kDim + kT - 1) / kT;                      // query values a thread converts
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int b = hq / in.bv.n_q, hh = hq - b * in.bv.n_q;            // hh = j * G + h
     const int j = hh / in.bv.group;
@@ -84,7 +91,10 @@ __device__ __forceinline__ void select_head(const PlanInputs &in, int hq, HeadSm
         const int at = tid + i * kT;
         yv[i] = at < n4_row ? __ldcg(y4 + at) : kNone;
     }
-    const float q_val = tid < kHeadDim ? elem_to_float<kHalf>(in.q[(size_t)hq * kHeadDim + tid]) : 0.f;
+    float q_val[kQRegs];
+#pragma unroll
+    for (int i = 0; i < kQRegs; ++i)
+        q_val[i] = tid + i * kT < kDim ? elem_to_float<kHalf>(in.q[(size_t)hq * kDim + tid + i * kT]) : 0.f;
     const float k_abs_max = in.rep_abs_max[(size_t)j * in.bv.n_seqs + b];
 
     const int64_t team0 = in.bv.seq_team_off[b];
@@ -93,7 +103,7 @@ __device__ __forceinline__ void select_head(const PlanInputs &in, int hq, HeadSm
     if (K >= M) return;
     trace_mark(in.trace, 1, 7);
     const uint32_t step = in.step + (in.step_dev ? *in.step_dev : 0u);
-    const uint16_t *rep = in.rep_keys + ((size_t)j * in.bv.teams_total + team0) * kHeadDim;
+    const uint16_t *rep = in.rep_keys + ((size_t)j * in.bv.teams_total + team0) * kDim;
     const int32_t *csr = in.team_row_start + (size_t)j * (in.bv.teams_total + in.bv.n_seqs) + team0 + b;
     const int n4 = (M + 3) >> 2;                                      // 16-byte pieces that hold teams
     const int need = K + 1;
@@ -121,7 +131,9 @@ __device__ __forceinline__ void select_head(const PlanInputs &in, int hq, HeadSm
         }
     };
     {
-        float a = fabsf(q_val), top = -CUDART_INF_F;
+        float a = 0.f, top = -CUDART_INF_F;
+#pragma unroll
+        for (int i = 0; i < kQRegs; ++i) a += fabsf(q_val[i]);
         each_score([&](float x, int, bool) { top = fmaxf(top, x); });
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
@@ -130,7 +142,11 @@ __device__ __forceinline__ void select_head(const PlanInputs &in, int hq, HeadSm
         }
         trace_mark(in.trace, 1, 8);
         __syncthreads();                                              // the shared structure is free (block reuse)
-        if (tid < kHeadDim) sm.q64[tid >> 4][tid & 15] = (double)q_val;
+#pragma unroll
+        for (int i = 0; i < kQRegs; ++i) {
+            const int d = tid + i * kT;
+            if (d < kDim) sm.q64[d / kSlice][d % kSlice] = (double)q_val[i];
+        }
         if (lane == 0) { sm.red_sum[warp] = a; sm.red_max[warp] = top; }
         if (tid == 0) sm.n_cand = 0;
         for (int i = tid; i < 256; i += kT) sm.hist[i] = 0;
@@ -256,48 +272,44 @@ __device__ __forceinline__ void select_head(const PlanInputs &in, int hq, HeadSm
         }
         const int n_cand = sm.n_cand;
 
-        // ---- 3a. exact terms: dot products on the first half of the warps (8 lanes per candidate, 16 dims each),
+        // ---- 3a. exact terms: dot products on the first half of the warps (8 lanes per candidate, kDim / 8 dims each),
         //          log n_g and the Gumbel term on the other warps (one thread per candidate) ----
         if (warp < kDotWarps) {
             const int sub = lane & (kDotLanes - 1);
             const double *qs = sm.q64[sub];
-            // four candidates per thread group at a time: all their key pieces are requested before
+            // a few candidates per thread group at a time: all their key pieces are requested before
             // the first product, so a chunk costs one memory round trip
-            constexpr int kPerPass = kDotWarps * 32 / kDotLanes, kChunk = kT >= 512 ? 2 : 4;
+            constexpr int kPerPass = kDotWarps * 32 / kDotLanes, kChunk = kPieces > 2 ? 1 : (kT >= 512 ? 2 : 4);
             for (int c0 = 0; c0 < n_cand; c0 += kPerPass * kChunk) {
-                uint4 w[kChunk][2];
+                uint4 w[kChunk][kPieces];
 #pragma unroll
                 for (int u = 0; u < kChunk; ++u) {
                     const int cand = c0 + u * kPerPass + (tid >> 3);
                     if (cand < n_cand) {
-                        const uint4 *kr = reinterpret_cast<const uint4 *>(rep + (size_t)sm.cand_id[cand] * kHeadDim) + sub * 2;
-                        w[u][0] = __ldg(kr);
-                        w[u][1] = __ldg(kr + 1);
+                        const uint4 *kr = reinterpret_cast<const uint4 *>(rep + (size_t)sm.cand_id[cand] * kDim) + sub * kPieces;
+#pragma unroll
+                        for (int pc = 0; pc < kPieces; ++pc) w[u][pc] = __ldg(kr + pc);
                     } else {
-                        w[u][0] = w[u][1] = make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+                        for (int pc = 0; pc < kPieces; ++pc) w[u][pc] = make_uint4(0u, 0u, 0u, 0u);
                     }
                 }
 #pragma unroll
                 for (int u = 0; u < kChunk; ++u) {
                     const int cand = c0 + u * kPerPass + (tid >> 3);
-                    const uint4 w0 = w[u][0], w1 = w[u][1];
-                    double d0 = 0.0, d1 = 0.0;
-                    d0 = fma((double)elem_lo<kHalf>(w0.x), qs[0], d0);
-                    d1 = fma((double)elem_hi<kHalf>(w0.x), qs[1], d1);
-                    d0 = fma((double)elem_lo<kHalf>(w0.y), qs[2], d0);
-                    d1 = fma((double)elem_hi<kHalf>(w0.y), qs[3], d1);
-                    d0 = fma((double)elem_lo<kHalf>(w0.z), qs[4], d0);
-                    d1 = fma((double)elem_hi<kHalf>(w0.z), qs[5], d1);
-                    d0 = fma((double)elem_lo<kHalf>(w0.w), qs[6], d0);
-                    d1 = fma((double)elem_hi<kHalf>(w0.w), qs[7], d1);
-                    d0 = fma((double)elem_lo<kHalf>(w1.x), qs[8], d0);
-                    d1 = fma((double)elem_hi<kHalf>(w1.x), qs[9], d1);
-                    d0 = fma((double)elem_lo<kHalf>(w1.y), qs[10], d0);
-                    d1 = fma((double)elem_hi<kHalf>(w1.y), qs[11], d1);
-                    d0 = fma((double)elem_lo<kHalf>(w1.z), qs[12], d0);
-                    d1 = fma((double)elem_hi<kHalf>(w1.z), qs[13], d1);
-                    d0 = fma((double)elem_lo<kHalf>(w1.w), qs[14], d0);
-                    d1 = fma((double)elem_hi<kHalf>(w1.w), qs[15], d1);
+                    double d0 = 0.0, d1 = 0.0;                        // even and odd dims of the slice, in order
+#pragma unroll
+                    for (int pc = 0; pc < kPieces; ++pc) {
+                        const uint4 wv = w[u][pc];
+                        d0 = fma((double)elem_lo<kHalf>(wv.x), qs[8 * pc + 0], d0);
+                        d1 = fma((double)elem_hi<kHalf>(wv.x), qs[8 * pc + 1], d1);
+                        d0 = fma((double)elem_lo<kHalf>(wv.y), qs[8 * pc + 2], d0);
+                        d1 = fma((double)elem_hi<kHalf>(wv.y), qs[8 * pc + 3], d1);
+                        d0 = fma((double)elem_lo<kHalf>(wv.z), qs[8 * pc + 4], d0);
+                        d1 = fma((double)elem_hi<kHalf>(wv.z), qs[8 * pc + 5], d1);
+                        d0 = fma((double)elem_lo<kHalf>(wv.w), qs[8 * pc + 6], d0);
+                        d1 = fma((double)elem_hi<kHalf>(wv.w), qs[8 * pc + 7], d1);
+                    }
                     double d = d0 + d1;
                     d += __shfl_xor_sync(0xFFFFFFFFu, d, 1);
                     d += __shfl_xor_sync(0xFFFFFFFFu, d, 2);

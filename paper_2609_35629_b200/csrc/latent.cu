@@ -1,0 +1,1222 @@
+// Shared-latent rows (appendix "Token sparsity after latent compression"): one stored row per
+// token, a 512-value content latent followed by a 64-value rotary key, shared by up to 16 query
+// heads. Teams come from the latents alone (Algorithm 4 + Algorithm 2), every head runs
+// Algorithm 1 on the shared teams with its own query against the whole row, a row is read once
+// when any head selected its team, and its latent part is the value.
+//
+// Kernels of one decode step:
+//   latent_score_kernel    fp32 routing scores of all 16 heads for 16 teams per warp (mma.sync,
+//                          teams as the M tile, heads as two N tiles, 36 k-steps), Gumbel added
+//   latent_select_kernel   Algorithm 1's sample per (sequence, head): select_head over 576 values
+//   latent_plan_kernel     union of the heads' samples per sequence, written row by row: source
+//                          row and segment of every row to read, per-segment log c (or -inf) per head
+//   latent_attend_kernel   one block per SM, two groups of four warps on alternating 32-row tiles;
+//                          S = Q K^T with the contraction split over the group's warps, P V with
+//                          the 512 value columns split over them; one partial per (block, sequence)
+//   latent_merge_kernel    log-sum-exp merge of the partials
+#include <cuda_bf16.h>
+#include <limits.h>
+#include <math_constants.h>
+
+#include <algorithm>
+#include <vector>
+
+#include "build_util.cuh"
+#include "common.cuh"
+#include "headplan.cuh"
+#include "santapp_latent.h"
+#include "score_tile.cuh"
+
+using namespace santapp;
+
+namespace {
+
+constexpr int kRowDim = SANTAPP_LATENT_ROW;          // 576 values per row
+constexpr int kLatDim = SANTAPP_LATENT_DIM;          // 512: distances, means and values use these
+constexpr int kRowBytes = kRowDim * 2;               // 1152
+constexpr int kRowChunks = kRowBytes / 16;           // 72 16-byte pieces
+constexpr int kHeads = SANTAPP_LATENT_MAX_HEADS;     // 16: the M tile of the attention MMAs
+constexpr int kMaxP = SANTAPP_LATENT_MAX_PARENT;
+constexpr int kLatPartialStride = 4 + kLatDim;       // floats per (slot, head): m, l, 2 pad, acc[512]
+constexpr int kMaxLatentSeqs = 4096;
+
+struct LatentView {
+    int n_seqs, n_heads;
+    const int64_t *seq_row_off, *seq_team_off;
+    int64_t rows_total, teams_total;
+};
+
+// ---------------------------------------------------------------------------------------------
+// Records: contiguous parents, Algorithm 2 on the latent columns
+// ---------------------------------------------------------------------------------------------
+struct LatentBuildParams {
+    LatentView lv;
+    int parent_size, reps, teams_per_full_parent;
+    const uint16_t *rows_prompt;
+    uint16_t *rows_packed, *rep_rows;
+    int32_t *team_row_start, *row_token;
+    float *rep_abs_max;
+    uint8_t *owner;                 // workspace [rows_total]
+    int max_parents_per_seq;
+};
+
+constexpr int kLbThreads = 128;
+
+// Squared distance between two rows' latent parts in fp64: dims in increasing order, multiply
+// and add rounded separately (the order the records are defined with).
+__device__ __forceinline__ double latent_sqdist(const uint32_t *a, const uint32_t *b)
+{
+    double s = 0.0;
+#pragma unroll 8
+    for (int w = 0; w < kLatDim / 2; ++w) {
+        const uint32_t x = a[w], y = b[w];
+        const double e0 = __dsub_rn((double)bf16_lo(x), (double)bf16_lo(y));
+        const double e1 = __dsub_rn((double)bf16_hi(x), (double)bf16_hi(y));
+        s = __dadd_rn(s, __dmul_rn(e0, e0));
+        s = __dadd_rn(s, __dmul_rn(e1, e1));
+    }
+    return s;
+}
+
+// One block per (parent, sequence).
+__global__ void __launch_bounds__(kLbThreads)
+latent_build_parent_kernel(LatentBuildParams p)
+{
+    constexpr int kPitch = kRowDim / 2 + 1;                 // words per staged row (+1: conflict-free column walks)
+    __shared__ uint32_t rows[kMaxP * kPitch];
+    __shared__ double mu[kLatDim];
+    __shared__ double mind[kMaxP];
+    __shared__ ValIdx scratch[33];
+    __shared__ int owner[kMaxP], count[kMaxP], rep_of[kMaxP];
+    __shared__ unsigned char is_rep[kMaxP];
+
+    const int parent = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
+    const int64_t row0 = p.lv.seq_row_off[b];
+    const int N = (int)(p.lv.seq_row_off[b + 1] - row0);
+    const int P = p.parent_size;
+    const int first = parent * P;
+    if (first >= N) return;
+    const int nC = min(P, N - first);
+    const int r = min(p.reps, nC);
+
+    const uint32_t *src = reinterpret_cast<const uint32_t *>(p.rows_prompt) + (size_t)(row0 + first) * (kRowDim / 2);
+    for (int e = tid; e < nC * (kRowDim / 2); e += kLbThreads) rows[(e / (kRowDim / 2)) * kPitch + e % (kRowDim / 2)] = src[e];
+    for (int i = tid; i < nC; i += kLbThreads) { is_rep[i] = 0; count[i] = 0; }
+    __syncthreads();
+
+    // parent mean of the latent columns: rows added in token order, then one division
+    for (int d = tid; d < kLatDim; d += kLbThreads) {
+        double s = 0.0;
+        for (int i = 0; i < nC; ++i) {
+            const uint32_t word = rows[i * kPitch + (d >> 1)];
+            s = __dadd_rn(s, (double)((d & 1) ? bf16_hi(word) : bf16_lo(word)));
+        }
+        mu[d] = __ddiv_rn(s, (double)nC);
+    }
+    __syncthreads();
+
+    // first representative: the row whose latent is nearest the mean
+    {
+        ValIdx best = {INFINITY, INT_MAX};
+        for (int i = tid; i < nC; i += kLbThreads) {
+            double s = 0.0;
+            const uint32_t *row = rows + i * kPitch;
+            for (int w = 0; w < kLatDim / 2; ++w) {
+                const uint32_t word = row[w];
+                const double e0 = __dsub_rn((double)bf16_lo(word), mu[2 * w]);
+                const double e1 = __dsub_rn((double)bf16_hi(word), mu[2 * w + 1]);
+                s = __dadd_rn(s, __dmul_rn(e0, e0));
+                s = __dadd_rn(s, __dmul_rn(e1, e1));
+            }
+            ValIdx c = {s, i};
+            best = pick<true>(best, c);
+        }
+        best = block_arg<true>(best, scratch);
+        if (tid == 0) { rep_of[0] = best.i; is_rep[best.i] = 1; }
+    }
+    __syncthreads();
+
+    // farthest-first representatives with the running nearest-representative assignment
+    for (int i = tid; i < nC; i += kLbThreads) { mind[i] = INFINITY; owner[i] = 0; }
+    for (int u = 0; u < r; ++u) {
+        const uint32_t *ref = rows + rep_of[u] * kPitch;
+        ValIdx far = {-2.0, INT_MAX};
+        for (int i = tid; i < nC; i += kLbThreads) {
+            const double dist = latent_sqdist(rows + i * kPitch, ref);
+            if (dist < mind[i]) { mind[i] = dist; owner[i] = u; }
+            ValIdx c = {is_rep[i] ? -1.0 : mind[i], i};
+            far = pick<false>(far, c);
+        }
+        if (u + 1 < r) {
+            far = block_arg<false>(far, scratch);
+            if (tid == 0) { rep_of[u + 1] = far.i; is_rep[far.i] = 1; }
+            __syncthreads();
+        }
+    }
+    __syncthreads();
+    for (int u = tid; u < r; u += kLbThreads) owner[rep_of[u]] = u;      // a representative owns its own row
+    __syncthreads();
+    for (int i = tid; i < nC; i += kLbThreads) atomicAdd(&count[owner[i]], 1);
+    __syncthreads();
+
+    uint8_t *owner_out = p.owner + row0 + first;
+    for (int i = tid; i < nC; i += kLbThreads) owner_out[i] = (uint8_t)owner[i];
+    const int64_t team0 = p.lv.seq_team_off[b];
+    const int team_local0 = parent * p.teams_per_full_parent;
+    int32_t *csr = p.team_row_start + team0 + b;
+    if (parent == 0 && tid == 0) csr[0] = 0;
+    for (int u = tid; u < r; u += kLbThreads) csr[1 + team_local0 + u] = count[u];    // sizes; scanned next
+    uint32_t *rep_dst = reinterpret_cast<uint32_t *>(p.rep_rows) + (size_t)(team0 + team_local0) * (kRowDim / 2);
+    for (int e = tid; e < r * (kRowDim / 2); e += kLbThreads)
+        rep_dst[e] = rows[rep_of[e / (kRowDim / 2)] * kPitch + e % (kRowDim / 2)];
+}
+
+// One block per sequence: team sizes -> CSR offsets, and the largest |value| of the representatives.
+__global__ void __launch_bounds__(256)
+latent_scan_kernel(LatentBuildParams p)
+{
+    __shared__ int scratch[33];
+    __shared__ uint32_t red[8];
+    const int b = blockIdx.x;
+    const int64_t team0 = p.lv.seq_team_off[b];
+    const int M = (int)(p.lv.seq_team_off[b + 1] - team0);
+    int32_t *csr = p.team_row_start + team0 + b + 1;
+    int carry = 0;
+    for (int base = 0; base < M; base += 256) {
+        const int g = base + threadIdx.x;
+        const int v = g < M ? csr[g] : 0;
+        int total;
+        const int excl = block_exclusive_scan(v, scratch, total);
+        if (g < M) csr[g] = carry + excl + v;
+        carry += total;
+    }
+    const uint32_t *w = reinterpret_cast<const uint32_t *>(p.rep_rows) + (size_t)team0 * (kRowDim / 2);
+    const int64_t n = (int64_t)M * (kRowDim / 2);
+    uint32_t m = 0u;                                        // bf16 magnitudes order like integers
+    for (int64_t i = threadIdx.x; i < n; i += 256) {
+        const uint32_t v = w[i];
+        m = max(m, max(v & 0x7FFFu, (v >> 16) & 0x7FFFu));
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = m;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int i = 1; i < 8; ++i) m = max(m, red[i]);
+        p.rep_abs_max[b] = __uint_as_float(m << 16);
+    }
+}
+
+// One block per (parent, sequence): stable partition of the parent's rows by team, row copies.
+__global__ void __launch_bounds__(kLbThreads)
+latent_pack_kernel(LatentBuildParams p)
+{
+    __shared__ uint8_t owner[kMaxP];
+    __shared__ int dest[kMaxP];
+    const int parent = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
+    const int64_t row0 = p.lv.seq_row_off[b];
+    const int N = (int)(p.lv.seq_row_off[b + 1] - row0);
+    const int first = parent * p.parent_size;
+    if (first >= N) return;
+    const int nC = min(p.parent_size, N - first);
+    for (int i = tid; i < nC; i += kLbThreads) owner[i] = p.owner[row0 + first + i];
+    __syncthreads();
+    const int32_t *csr = p.team_row_start + p.lv.seq_team_off[b] + b;
+    const int team_local0 = parent * p.teams_per_full_parent;
+    for (int i = tid; i < nC; i += kLbThreads) {
+        const int u = owner[i];
+        int rank = 0;
+        for (int a = 0; a < i; ++a) rank += (owner[a] == u);
+        dest[i] = csr[team_local0 + u] + rank;              // members in increasing token index
+    }
+    __syncthreads();
+    const uint4 *src = reinterpret_cast<const uint4 *>(p.rows_prompt) + (size_t)(row0 + first) * kRowChunks;
+    uint4 *dst = reinterpret_cast<uint4 *>(p.rows_packed) + (size_t)row0 * kRowChunks;
+    for (int e = tid; e < nC * kRowChunks; e += kLbThreads) {
+        const int i = e / kRowChunks, c = e - i * kRowChunks;
+        dst[(size_t)dest[i] * kRowChunks + c] = src[e];
+    }
+    for (int i = tid; i < nC; i += kLbThreads) p.row_token[row0 + dest[i]] = first + i;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Routing scores (Eq. method-routing plus the Gumbel term), fp32 on tensor cores
+// ---------------------------------------------------------------------------------------------
+struct LatentScoreParams {
+    LatentView lv;
+    const uint16_t *rep_rows;       // [teams_total][576]
+    const int32_t *team_row_start;  // [teams_total + n_seqs]
+    const uint16_t *q;              // [n_seqs][n_heads][576]
+    float *y32;                     // [n_heads][n_seqs][y_stride]
+    int64_t y_stride;
+    int n_sample;
+    uint32_t seed_lo, seed_hi, step, stream_base;
+    const uint32_t *step_dev;
+    float scale;
+};
+
+constexpr int kLsThreads = 256;
+constexpr int kLsTeamsPerBlock = (kLsThreads / 32) * 16;
+
+__device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1)
+{
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// Grid (ceil(max teams / 128), sequences); a warp scores 16 teams for all heads: the teams are the
+// MMA's 16 rows, the heads its columns (two tiles of 8), the 576 values 36 k-steps. Both operands
+// use the same permutation of the contraction index inside every block of 32 values, so a lane
+// feeds the tensor core 16-byte pieces of a representative row (and of a query) as they lie in
+// memory: piece t of the block supplies k-slots {2t, 2t+1, 2t+8, 2t+9} of the block's two MMAs.
+__global__ void __launch_bounds__(kLsThreads)
+latent_score_kernel(LatentScoreParams p)
+{
+    constexpr int kQPitchW = (kRowBytes + 16) / 4;                  // words per staged query (+16 bytes: conflict-free LDS.128)
+    __shared__ __align__(16) uint32_t q_s[kHeads * kQPitchW];
+    __shared__ __align__(16) uint32_t words_s[kLsThreads / 32][kHeads][16];
+    const int b = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int64_t team0 = p.lv.seq_team_off[b];
+    const int M = (int)(p.lv.seq_team_off[b + 1] - team0);
+    if (p.n_sample >= M || (int)blockIdx.x * kLsTeamsPerBlock >= M) return;      // nothing is drawn / no team here
+    const int H = p.lv.n_heads;
+    const uint4 *qg = reinterpret_cast<const uint4 *>(p.q + (size_t)b * H * kRowDim);
+    for (int e = tid; e < kHeads * kRowChunks; e += kLsThreads) {
+        const int h = e / kRowChunks, c = e - h * kRowChunks;
+        const uint4 v = h < H ? __ldg(qg + (size_t)h * kRowChunks + c) : make_uint4(0u, 0u, 0u, 0u);
+        *reinterpret_cast<uint4 *>(q_s + h * kQPitchW + c * 4) = v;
+    }
+    __syncthreads();
+    const int t0 = ((int)blockIdx.x * (kLsThreads / 32) + warp) * 16;
+    if (t0 >= M) return;
+    const uint32_t step = p.step + (p.step_dev ? *p.step_dev : 0u);
+    const int r = lane >> 2, t = lane & 3;
+    const int ga = t0 + r, gb = t0 + r + 8;                         // the lane's two teams (rows r and r + 8 of the tile)
+    const uint4 *ka = reinterpret_cast<const uint4 *>(p.rep_rows + (size_t)(team0 + min(ga, M - 1)) * kRowDim) + t;
+    const uint4 *kb = reinterpret_cast<const uint4 *>(p.rep_rows + (size_t)(team0 + min(gb, M - 1)) * kRowDim) + t;
+    const int32_t *csr = p.team_row_start + team0 + b;
+    const int na = ga < M ? csr[ga + 1] - csr[ga] : 1, nb = gb < M ? csr[gb + 1] - csr[gb] : 1;
+
+    // Philox words of the tile: lane computes the blocks of head (lane & 15) for two groups of four teams
+    {
+        const int h = lane & 15, tg = (lane >> 4) * 2;
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const uint4 w = philox4x32_10(make_uint4((uint32_t)(t0 >> 2) + tg + u, step, (uint32_t)h, p.stream_base + (uint32_t)b),
+                                          p.seed_lo, p.seed_hi);
+            *reinterpret_cast<uint4 *>(&words_s[warp][h][(tg + u) * 4]) = w;
+        }
+    }
+
+    float acc[2][4] = {};
+    constexpr int kBatch = 6;                                       // blocks of 32 values requested together
+#pragma unroll 1
+    for (int blk0 = 0; blk0 < kRowDim / 32; blk0 += kBatch) {
+        uint4 wa[kBatch], wb[kBatch];
+#pragma unroll
+        for (int i = 0; i < kBatch; ++i) { wa[i] = __ldg(ka + (blk0 + i) * 4); wb[i] = __ldg(kb + (blk0 + i) * 4); }
+#pragma unroll
+        for (int i = 0; i < kBatch; ++i) {
+            const int piece = (blk0 + i) * 4 + t;
+            const uint4 q0 = *reinterpret_cast<const uint4 *>(q_s + r * kQPitchW + piece * 4);
+            const uint4 q1 = *reinterpret_cast<const uint4 *>(q_s + (r + 8) * kQPitchW + piece * 4);
+            mma_bf16(acc[0], wa[i].x, wb[i].x, wa[i].y, wb[i].y, q0.x, q0.y);
+            mma_bf16(acc[0], wa[i].z, wb[i].z, wa[i].w, wb[i].w, q0.z, q0.w);
+            mma_bf16(acc[1], wa[i].x, wb[i].x, wa[i].y, wb[i].y, q1.x, q1.y);
+            mma_bf16(acc[1], wa[i].z, wb[i].z, wa[i].w, wb[i].w, q1.z, q1.w);
+        }
+    }
+    __syncwarp();
+    const float log_a = __logf((float)na), log_b = __logf((float)nb);
+#pragma unroll
+    for (int n = 0; n < 2; ++n) {
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+            const int h = 8 * n + 2 * t + e;
+            if (h < H) {
+                float *row = p.y32 + ((size_t)h * p.lv.n_seqs + b) * p.y_stride;
+                if (ga < M) row[ga] = log_a + acc[n][e] * p.scale + gumbel32_from_word(words_s[warp][h][r]);
+                if (gb < M) row[gb] = log_b + acc[n][2 + e] * p.scale + gumbel32_from_word(words_s[warp][h][r + 8]);
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Sampling per (sequence, head): Algorithm 1 on 576-value routing keys
+// ---------------------------------------------------------------------------------------------
+template <int kT>
+__global__ void __launch_bounds__(kT, kT >= 512 ? 1 : 1024 / kT)
+latent_select_kernel(PlanInputs in)
+{
+    __shared__ HeadSmemT<kRowDim> sm;
+    select_head<kT, kT >= 512 ? 4 : 2, false, kRowDim>(in, blockIdx.x, sm);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Union of the heads' samples per sequence, written row by row
+// ---------------------------------------------------------------------------------------------
+struct LatentPlanParams {
+    LatentView lv;
+    const int32_t *sel_team;        // [n_seqs][n_heads][K]
+    const float *sel_logc;
+    const int2 *sel_rows;
+    const int32_t *suffix_len;      // nullable
+    int suffix_cap, n_sample, seg_cap;
+    int2 *row_meta;                 // [rows_total + n_seqs * suffix_cap] {source row, segment}: sequence b's rows to
+                                    //   read, in team order then suffix, start at seq_row_off[b] + b * suffix_cap
+    float *seg_bias;                // [n_seqs][seg_cap][16] -log2(e) log c_g of each head (a row's weight is e^s / c_g),
+                                    //   -inf where the head did not select the team
+    int32_t *pair_rows;             // [n_seqs] rows to read
+    int32_t *dbg_sel_idx;
+    float *dbg_sel_logc;
+    double *dbg_tau;
+    int32_t *dbg_union_rows;
+};
+
+constexpr int kLpThreads = 512;
+constexpr int kLatSegMax = kHeads * 128 + 1;                // 16 heads x K <= 128 teams, + the suffix
+
+struct LatentPlanSmem {
+    uint32_t bitmap[kMaxTeamsPerSeq / 32];
+    int wprefix[kMaxTeamsPerSeq / 32];
+    int seg_start[kLatSegMax], seg_n[kLatSegMax], seg_prefix[kLatSegMax + 1];
+    int scan[40];
+};
+
+__global__ void __launch_bounds__(kLpThreads)
+latent_plan_kernel(LatentPlanParams p)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    LatentPlanSmem &sm = *reinterpret_cast<LatentPlanSmem *>(smem_raw);
+    const int b = blockIdx.x, tid = threadIdx.x;
+    const int H = p.lv.n_heads, K = p.n_sample;
+    const int64_t row0 = p.lv.seq_row_off[b];
+    const int N = (int)(p.lv.seq_row_off[b + 1] - row0);
+    const int M = (int)(p.lv.seq_team_off[b + 1] - p.lv.seq_team_off[b]);
+    int t_suffix = 0;
+    if (p.suffix_len != nullptr && p.suffix_cap > 0) t_suffix = max(0, min(p.suffix_len[b], p.suffix_cap));
+    int2 *line = p.row_meta + row0 + (int64_t)b * p.suffix_cap;
+    float *bias = p.seg_bias + (size_t)b * p.seg_cap * kHeads;
+    const size_t head0 = (size_t)b * H;
+    const float kLog2e = 1.4426950408889634f;
+
+    if (K >= M) {
+        // every team is read with correction one; nothing was drawn
+        for (int i = tid; i < N; i += kLpThreads) line[i] = make_int2((int)(row0 + i), 0);
+        for (int i = tid; i < t_suffix; i += kLpThreads) line[N + i] = make_int2((int)(kSrcSuffix | (uint32_t)(b * p.suffix_cap + i)), 0);
+        if (tid < kHeads) bias[tid] = 0.f;
+        if (tid == 0) {
+            p.pair_rows[b] = N + t_suffix;
+            if (p.dbg_union_rows) p.dbg_union_rows[b] = N;
+        }
+        for (int e = tid; e < H * K; e += kLpThreads) {
+            const int a = e % K;
+            if (p.dbg_sel_idx) p.dbg_sel_idx[head0 * K + e] = a < M ? a : -1;
+            if (p.dbg_sel_logc) p.dbg_sel_logc[head0 * K + e] = 0.f;
+        }
+        if (tid < H && p.dbg_tau) p.dbg_tau[head0 + tid] = __longlong_as_double(0x7FF8000000000000ll);
+        return;
+    }
+
+    const int n_words = (M + 31) / 32, E = H * K;
+    for (int i = tid; i < n_words; i += kLpThreads) sm.bitmap[i] = 0u;
+    __syncthreads();
+    for (int e = tid; e < E; e += kLpThreads) {
+        const int team = __ldcg(p.sel_team + head0 * K + e);
+        if (team >= 0 && team < M) atomicOr(&sm.bitmap[team >> 5], 1u << (team & 31));
+    }
+    __syncthreads();
+    int nseg;
+    {
+        const int wpt = (n_words + kLpThreads - 1) / kLpThreads;
+        const int lo = min(tid * wpt, n_words), hi = min(lo + wpt, n_words);
+        int sum = 0;
+        for (int w = lo; w < hi; ++w) sum += __popc(sm.bitmap[w]);
+        int run = block_exclusive_scan(sum, sm.scan, nseg);
+        for (int w = lo; w < hi; ++w) { sm.wprefix[w] = run; run += __popc(sm.bitmap[w]); }
+    }
+    for (int i = tid; i < nseg * kHeads; i += kLpThreads) bias[i] = -CUDART_INF_F;
+    if (tid < kHeads) bias[(size_t)nseg * kHeads + tid] = 0.f;              // the suffix segment
+    __syncthreads();
+    for (int e = tid; e < E; e += kLpThreads) {
+        const int team = __ldcg(p.sel_team + head0 * K + e);
+        if (team < 0 || team >= M) continue;                                   // cannot come from the sampler
+        const int seg = sm.wprefix[team >> 5] + __popc(sm.bitmap[team >> 5] & ((1u << (team & 31)) - 1u));
+        const int2 rows = __ldcg(p.sel_rows + head0 * K + e);
+        bias[(size_t)seg * kHeads + e / K] = -kLog2e * __ldcg(p.sel_logc + head0 * K + e);   // weight e^s / c_g
+        sm.seg_start[seg] = rows.x;                                            // the same from every selecting head
+        sm.seg_n[seg] = rows.y;
+    }
+    __syncthreads();
+    int total;
+    {
+        const int spt = (nseg + kLpThreads - 1) / kLpThreads;
+        const int lo = min(tid * spt, nseg), hi = min(lo + spt, nseg);
+        int sum = 0;
+        for (int sg = lo; sg < hi; ++sg) sum += sm.seg_n[sg];
+        int run = block_exclusive_scan(sum, sm.scan, total);
+        for (int sg = lo; sg < hi; ++sg) { sm.seg_prefix[sg] = run; run += sm.seg_n[sg]; }
+    }
+    __syncthreads();
+    total = min(total, N);                                                     // distinct teams cannot hold more rows
+    for (int sg = tid; sg < nseg; sg += kLpThreads) {
+        const int at = sm.seg_prefix[sg], n = sm.seg_n[sg], start = sm.seg_start[sg];
+        for (int i = 0; i < n && at + i < N; ++i) line[at + i] = make_int2((int)(row0 + min(start + i, N - 1)), sg);
+    }
+    for (int i = tid; i < t_suffix; i += kLpThreads)
+        line[total + i] = make_int2((int)(kSrcSuffix | (uint32_t)(b * p.suffix_cap + i)), nseg);
+    if (tid == 0) {
+        p.pair_rows[b] = total + t_suffix;
+        if (p.dbg_union_rows) p.dbg_union_rows[b] = total;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Attention over the rows to read, and the merge of the blocks' partial results
+// ---------------------------------------------------------------------------------------------
+struct LatentAttendParams {
+    LatentView lv;
+    const uint16_t *rows_packed;    // [rows_total][576]
+    const uint16_t *suffix_rows;    // [n_seqs][suffix_cap][576]
+    const uint16_t *q;              // [n_seqs][n_heads][576]
+    const int2 *row_meta;           // see LatentPlanParams (not read by the dense variant)
+    const float *seg_bias;
+    const int32_t *pair_rows;
+    const int32_t *suffix_len;      // nullable
+    int suffix_cap, seg_cap;
+    float qk_scale_log2;            // scale * log2(e)
+    float *partials;                // [grid + n_seqs][16][kLatPartialStride]: block c leaves sequence b's share in slot c + b
+    uint32_t *pair_prefix;          // [n_seqs + 1] rows to read before each sequence; written by block 0 for the merge
+};
+
+constexpr int kLaThreads = 256;
+constexpr int kTileRows = 32;
+constexpr int kTileBytes = kTileRows * kRowBytes;                   // 36864
+constexpr int kBiasPitch = 20;                                      // floats per tile row (16 heads + pad: conflict-free reads)
+constexpr int kOffBias = 2 * 2 * kTileBytes;                        // two groups x two stages of rows
+constexpr int kOffXch = kOffBias + 2 * 2 * kTileRows * kBiasPitch * 4;
+constexpr int kOffPrefix = kOffXch + 2 * 4 * 4 * 32 * 16;           // per group: 4 warps x 4 float4 x 32 lanes
+constexpr int kOffScan = kOffPrefix + (kMaxLatentSeqs + 4) * 4;
+constexpr int kLaSmemBytes = kOffScan + 48 * 4;
+
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, int bytes)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void ldmatrix_x4(uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3, uint32_t addr)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3, uint32_t addr)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void group_barrier(int grp)
+{
+    asm volatile("bar.sync %0, 128;" ::"r"(grp + 1) : "memory");
+}
+__device__ __forceinline__ float ex2(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
+{
+    const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t *>(&v);
+}
+
+// One block per SM. The rows to read of all sequences form one line, cut into equal ranges, one
+// per block; a block walks the sequences its range touches. Inside a sequence the block's two
+// groups of four warps take alternate tiles of 32 rows, each group with its own two-stage ring of
+// asynchronous copies (16-byte pieces, XOR-swizzled by the row so that ldmatrix is conflict-free)
+// and its own running softmax; the groups' states are merged when the sequence's share is done.
+// Per tile and group: every warp multiplies the 16 heads' queries (A fragments, kept in registers
+// for the warp's 144 of the 576 values) by all 32 rows, the four partial S tiles are summed
+// through shared memory, every warp forms the same P, and multiplies it with its 128 of the 512
+// value columns (P split into two bf16 terms, so the weights keep 16 bits).
+template <bool kAll>
+__global__ void __launch_bounds__(kLaThreads, 1)
+latent_attend_kernel(LatentAttendParams p)
+{
+    extern __shared__ __align__(128) unsigned char smem[];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, grp = warp >> 2, gw = warp & 3, gt = tid & 127;
+    const int r = lane >> 2, t = lane & 3;
+    uint32_t *prefix = reinterpret_cast<uint32_t *>(smem + kOffPrefix);
+    int *scan = reinterpret_cast<int *>(smem + kOffScan);
+    const int n = p.lv.n_seqs, H = p.lv.n_heads;
+    {
+        uint32_t carry = 0;
+        for (int base = 0; base < n; base += kLaThreads) {
+            const int i = base + tid;
+            int v = 0;
+            if (i < n) {
+                if (kAll) {
+                    v = (int)(p.lv.seq_row_off[i + 1] - p.lv.seq_row_off[i]);
+                    if (p.suffix_len != nullptr && p.suffix_cap > 0) v += max(0, min(p.suffix_len[i], p.suffix_cap));
+                } else {
+                    v = __ldcg(p.pair_rows + i);
+                }
+            }
+            int total;
+            const int excl = block_exclusive_scan(v, scan, total);
+            if (i < n) prefix[i] = carry + (uint32_t)excl;
+            carry += (uint32_t)total;
+        }
+        if (tid == 0) prefix[n] = carry;
+        __syncthreads();
+    }
+    if (blockIdx.x == 0)
+        for (int i = tid; i <= n; i += kLaThreads) p.pair_prefix[i] = prefix[i];
+    const uint32_t total = prefix[n];
+    const uint32_t per = (total + gridDim.x - 1) / gridDim.x;
+    const uint32_t lo = min(total, blockIdx.x * per), hi = min(total, lo + per);
+    if (lo >= hi) return;
+    int pr = 0;
+    {
+        int a = 0, c = n;                                   // largest pr with prefix[pr] <= lo
+        while (c - a > 1) {
+            const int mid = (a + c) >> 1;
+            if (prefix[mid] <= lo) a = mid; else c = mid;
+        }
+        pr = a;
+    }
+    const uint32_t smem_base = (uint32_t)__cvta_generic_to_shared(smem);
+    const uint32_t tiles_addr = smem_base + grp * 2 * kTileBytes;
+    float *bias_grp = reinterpret_cast<float *>(smem + kOffBias) + grp * 2 * kTileRows * kBiasPitch;
+    float4 *xch = reinterpret_cast<float4 *>(smem + kOffXch) + grp * (4 * 4 * 32);
+    const uint4 *rows_g = reinterpret_cast<const uint4 *>(p.rows_packed);
+    const uint4 *suffix_g = reinterpret_cast<const uint4 *>(p.suffix_rows);
+
+    for (; pr < n && prefix[pr] < hi; ++pr) {
+        if (prefix[pr + 1] <= lo) continue;
+        const int b = pr;
+        const int s_lo = (int)(max(lo, prefix[pr]) - prefix[pr]), s_hi = (int)(min(hi, prefix[pr + 1]) - prefix[pr]);
+        const int64_t row0 = p.lv.seq_row_off[b];
+        const int N = (int)(p.lv.seq_row_off[b + 1] - row0);
+        const int2 *line = kAll ? nullptr : p.row_meta + row0 + (int64_t)b * p.suffix_cap;
+        const float *bias_g = kAll ? nullptr : p.seg_bias + (size_t)b * p.seg_cap * kHeads;
+
+        // the warp's share of the queries as A fragments: values [144 gw, 144 gw + 144)
+        uint32_t qa[9][4];
+        {
+            const uint32_t *q32 = reinterpret_cast<const uint32_t *>(p.q + (size_t)b * H * kRowDim);
+#pragma unroll
+            for (int ks = 0; ks < 9; ++ks) {
+                const int d0 = 16 * (9 * gw + ks) + 2 * t;
+                qa[ks][0] = r < H ? __ldg(q32 + (r * kRowDim + d0) / 2) : 0u;
+                qa[ks][1] = r + 8 < H ? __ldg(q32 + ((r + 8) * kRowDim + d0) / 2) : 0u;
+                qa[ks][2] = r < H ? __ldg(q32 + (r * kRowDim + d0 + 8) / 2) : 0u;
+                qa[ks][3] = r + 8 < H ? __ldg(q32 + ((r + 8) * kRowDim + d0 + 8) / 2) : 0u;
+            }
+        }
+        const int n_tiles = (s_hi - s_lo + kTileRows - 1) / kTileRows;
+        const int my_tiles = (n_tiles - grp + 1) / 2;       // tiles grp, grp + 2, ...
+        float m0 = -CUDART_INF_F, m1 = -CUDART_INF_F, l0 = 0.f, l1 = 0.f;
+        float o[16][4];
+#pragma unroll
+        for (int j2 = 0; j2 < 16; ++j2) o[j2][0] = o[j2][1] = o[j2][2] = o[j2][3] = 0.f;
+
+        // source row (and segment) of this thread's row of the group's j-th tile; x = -1: no row
+        auto load_meta = [&](int j) -> int2 {
+            const int pos = s_lo + kTileRows * (grp + 2 * j) + (gt >> 2);
+            if (j >= my_tiles || pos >= s_hi) return make_int2(-1, 0);
+            if (kAll)
+                return make_int2(pos < N ? (int)(row0 + pos) : (int)(kSrcSuffix | (uint32_t)(b * p.suffix_cap + pos - N)), 0);
+            return __ldcg(line + pos);
+        };
+        // four threads copy a row (18 pieces each); rows past the share's end are zero-filled
+        auto issue = [&](int j, int2 meta) {
+            if (j < my_tiles) {
+                const int i = gt >> 2, qd = gt & 3, stage = j & 1;
+                const bool valid = meta.x != -1;
+                const uint32_t src = (uint32_t)meta.x;
+                const uint4 *g = !valid ? rows_g
+                                        : ((src & kSrcSuffix) ? suffix_g + (size_t)(src & 0x7FFFFFFFu) * kRowChunks
+                                                              : rows_g + (size_t)src * kRowChunks);
+                const uint32_t dst = tiles_addr + stage * kTileBytes + i * kRowBytes;
+                const int bytes = valid ? 16 : 0;
+#pragma unroll
+                for (int c = 0; c < kRowChunks / 4; ++c) {
+                    const int chunk = 4 * c + qd;
+                    cp_async16(dst + ((chunk ^ (i & 7)) << 4), g + chunk, bytes);
+                }
+                if (!kAll) {
+                    const uint32_t bdst = smem_base + kOffBias + ((grp * 2 + stage) * kTileRows * kBiasPitch + i * kBiasPitch + 4 * qd) * 4;
+                    cp_async16(bdst, valid ? bias_g + (size_t)meta.y * kHeads + 4 * qd : reinterpret_cast<const float *>(rows_g), bytes);
+                }
+            }
+            asm volatile("cp.async.commit_group;" ::: "memory");
+        };
+
+        if (my_tiles > 0) {
+            issue(0, load_meta(0));
+            issue(1, load_meta(1));
+        }
+        int2 meta_next = load_meta(2);
+#pragma unroll 1
+        for (int j = 0; j < my_tiles; ++j) {
+            const int2 meta_cur = meta_next;                // of the tile issued at the end of this round
+            meta_next = load_meta(j + 3);
+            asm volatile("cp.async.wait_group 1;" ::: "memory");
+            group_barrier(grp);                             // tile j is in shared memory for every warp of the group
+            const uint32_t tile_addr = tiles_addr + (j & 1) * kTileBytes;
+            const float *bias_s = bias_grp + (j & 1) * kTileRows * kBiasPitch;
+            const int nv = min(kTileRows, s_hi - (s_lo + kTileRows * (grp + 2 * j)));
+
+            // ---- partial S (16 heads x 32 rows) over the warp's 144 values ----
+            float x[4][4];
+#pragma unroll
+            for (int nt = 0; nt < 4; ++nt) x[nt][0] = x[nt][1] = x[nt][2] = x[nt][3] = 0.f;
+#pragma unroll
+            for (int ks = 0; ks < 9; ++ks) {
+#pragma unroll
+                for (int ntp = 0; ntp < 2; ++ntp) {
+                    const int row = 16 * ntp + ((lane >> 4) << 3) + (lane & 7);
+                    const int chunk = 18 * gw + 2 * ks + ((lane >> 3) & 1);
+                    uint32_t r0, r1, r2, r3;
+                    ldmatrix_x4(r0, r1, r2, r3, tile_addr + row * kRowBytes + ((chunk ^ (lane & 7)) << 4));
+                    mma_bf16(x[2 * ntp], qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3], r0, r1);
+                    mma_bf16(x[2 * ntp + 1], qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3], r2, r3);
+                }
+            }
+#pragma unroll
+            for (int nt = 0; nt < 4; ++nt) xch[(gw * 4 + nt) * 32 + lane] = make_float4(x[nt][0], x[nt][1], x[nt][2], x[nt][3]);
+            group_barrier(grp);
+#pragma unroll
+            for (int nt = 0; nt < 4; ++nt) {
+                float4 s = xch[nt * 32 + lane];
+#pragma unroll
+                for (int w = 1; w < 4; ++w) {
+                    const float4 v = xch[(w * 4 + nt) * 32 + lane];
+                    s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+                }
+                x[nt][0] = s.x; x[nt][1] = s.y; x[nt][2] = s.z; x[nt][3] = s.w;
+            }
+
+            // ---- softmax step (log2 domain): heads r (c = 0, 1) and r + 8 (c = 2, 3), rows 8 nt + 2 t + (c & 1) ----
+            float mx0 = -CUDART_INF_F, mx1 = -CUDART_INF_F;
+#pragma unroll
+            for (int nt = 0; nt < 4; ++nt) {
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const int row = 8 * nt + 2 * t + (c & 1), head = r + ((c >> 1) << 3);
+                    const float bia = kAll ? 0.f : bias_s[row * kBiasPitch + head];
+                    x[nt][c] = row < nv ? fmaf(x[nt][c], p.qk_scale_log2, bia) : -CUDART_INF_F;
+                }
+                mx0 = fmaxf(mx0, fmaxf(x[nt][0], x[nt][1]));
+                mx1 = fmaxf(mx1, fmaxf(x[nt][2], x[nt][3]));
+            }
+            mx0 = fmaxf(mx0, __shfl_xor_sync(0xFFFFFFFFu, mx0, 1));
+            mx0 = fmaxf(mx0, __shfl_xor_sync(0xFFFFFFFFu, mx0, 2));
+            mx1 = fmaxf(mx1, __shfl_xor_sync(0xFFFFFFFFu, mx1, 1));
+            mx1 = fmaxf(mx1, __shfl_xor_sync(0xFFFFFFFFu, mx1, 2));
+            const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);
+            const float mu0 = mn0 == -CUDART_INF_F ? 0.f : mn0, mu1 = mn1 == -CUDART_INF_F ? 0.f : mn1;
+            const float a0 = ex2(m0 - mu0), a1 = ex2(m1 - mu1);
+            m0 = mn0;
+            m1 = mn1;
+            float ps0 = 0.f, ps1 = 0.f;
+#pragma unroll
+            for (int nt = 0; nt < 4; ++nt) {
+                x[nt][0] = ex2(x[nt][0] - mu0);
+                x[nt][1] = ex2(x[nt][1] - mu0);
+                x[nt][2] = ex2(x[nt][2] - mu1);
+                x[nt][3] = ex2(x[nt][3] - mu1);
+                ps0 += x[nt][0] + x[nt][1];
+                ps1 += x[nt][2] + x[nt][3];
+            }
+            l0 = l0 * a0 + ps0;
+            l1 = l1 * a1 + ps1;
+#pragma unroll
+            for (int j2 = 0; j2 < 16; ++j2) { o[j2][0] *= a0; o[j2][1] *= a0; o[j2][2] *= a1; o[j2][3] *= a1; }
+            uint32_t ph[2][4], pl[2][4];
+#pragma unroll
+            for (int ks2 = 0; ks2 < 2; ++ks2) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int nt = 2 * ks2 + (i >> 1), c = (i & 1) * 2;
+                    const float v0 = x[nt][c], v1 = x[nt][c + 1];
+                    const uint32_t hi16 = pack_bf16(v0, v1);
+                    ph[ks2][i] = hi16;
+                    pl[ks2][i] = pack_bf16(v0 - bf16_lo(hi16), v1 - bf16_hi(hi16));
+                }
+            }
+
+            // ---- O (16 heads x the warp's 128 value columns) += P V ----
+#pragma unroll
+            for (int j2 = 0; j2 < 8; ++j2) {
+#pragma unroll
+                for (int ks2 = 0; ks2 < 2; ++ks2) {
+                    const int mi = lane >> 3;
+                    const int row = 16 * ks2 + ((mi & 1) << 3) + (lane & 7);
+                    const int chunk = 16 * gw + 2 * j2 + (mi >> 1);
+                    uint32_t r0, r1, r2, r3;
+                    ldmatrix_x4_trans(r0, r1, r2, r3, tile_addr + row * kRowBytes + ((chunk ^ (lane & 7)) << 4));
+                    mma_bf16(o[2 * j2], ph[ks2][0], ph[ks2][1], ph[ks2][2], ph[ks2][3], r0, r1);
+                    mma_bf16(o[2 * j2 + 1], ph[ks2][0], ph[ks2][1], ph[ks2][2], ph[ks2][3], r2, r3);
+                    mma_bf16(o[2 * j2], pl[ks2][0], pl[ks2][1], pl[ks2][2], pl[ks2][3], r0, r1);
+                    mma_bf16(o[2 * j2 + 1], pl[ks2][0], pl[ks2][1], pl[ks2][2], pl[ks2][3], r2, r3);
+                }
+            }
+            group_barrier(grp);                             // every warp is done with this stage
+            issue(j + 2, meta_cur);
+        }
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        l0 += __shfl_xor_sync(0xFFFFFFFFu, l0, 1);
+        l0 += __shfl_xor_sync(0xFFFFFFFFu, l0, 2);
+        l1 += __shfl_xor_sync(0xFFFFFFFFu, l1, 1);
+        l1 += __shfl_xor_sync(0xFFFFFFFFu, l1, 2);
+
+        // ---- the two groups' states into one partial ----
+        __syncthreads();
+        float4 *comb = reinterpret_cast<float4 *>(smem);            // the rings are idle
+        float *comb_ml = reinterpret_cast<float *>(smem + 4 * 16 * 32 * 16);
+        if (grp == 1) {
+#pragma unroll
+            for (int j2 = 0; j2 < 16; ++j2) comb[(gw * 16 + j2) * 32 + lane] = make_float4(o[j2][0], o[j2][1], o[j2][2], o[j2][3]);
+            if (gw == 0 && t == 0) {
+                comb_ml[r] = m0;
+                comb_ml[r + 8] = m1;
+                comb_ml[16 + r] = l0;
+                comb_ml[16 + r + 8] = l1;
+            }
+        }
+        __syncthreads();
+        if (grp == 0) {
+            const float n0 = comb_ml[r], n1 = comb_ml[r + 8], k0 = comb_ml[16 + r], k1 = comb_ml[16 + r + 8];
+            const float M0 = fmaxf(m0, n0), M1 = fmaxf(m1, n1);
+            const float u0 = M0 == -CUDART_INF_F ? 0.f : M0, u1 = M1 == -CUDART_INF_F ? 0.f : M1;
+            const float w0 = ex2(m0 - u0), v0 = ex2(n0 - u0), w1 = ex2(m1 - u1), v1 = ex2(n1 - u1);
+            float *out0 = p.partials + ((size_t)(blockIdx.x + b) * kHeads + r) * kLatPartialStride;
+            float *out1 = out0 + 8 * kLatPartialStride;
+            if (gw == 0 && t == 0) {
+                out0[0] = M0;
+                out0[1] = w0 * l0 + v0 * k0;
+                out1[0] = M1;
+                out1[1] = w1 * l1 + v1 * k1;
+            }
+#pragma unroll
+            for (int j2 = 0; j2 < 16; ++j2) {
+                const float4 c = comb[(gw * 16 + j2) * 32 + lane];
+                const int col = 4 + 128 * gw + 8 * j2 + 2 * t;
+                *reinterpret_cast<float2 *>(out0 + col) = make_float2(w0 * o[j2][0] + v0 * c.x, w0 * o[j2][1] + v0 * c.y);
+                *reinterpret_cast<float2 *>(out1 + col) = make_float2(w1 * o[j2][2] + v1 * c.z, w1 * o[j2][3] + v1 * c.w);
+            }
+        }
+        __syncthreads();
+    }
+}
+
+// One block per (head, sequence): out = sum_c w_c acc_c / sum_c w_c l_c over the blocks that read
+// rows of the sequence, w_c = 2^(m_c - max m). Thread i owns value columns 4 i .. 4 i + 3.
+__global__ void __launch_bounds__(128)
+latent_merge_kernel(const float *partials, const uint32_t *pair_prefix, int n_seqs, int n_heads, int grid, float *out, int32_t *status)
+{
+    const int h = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
+    const uint32_t total = pair_prefix[n_seqs], per = (total + grid - 1) / grid;
+    const uint32_t lo = pair_prefix[b], hi = pair_prefix[b + 1];
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    float L = 0.f;
+    if (hi > lo) {
+        const int c_lo = (int)(lo / per), c_hi = (int)((hi - 1) / per);
+        float M = -CUDART_INF_F;
+        for (int c = c_lo; c <= c_hi; ++c) M = fmaxf(M, __ldcg(partials + ((size_t)(c + b) * kHeads + h) * kLatPartialStride));
+        const float Mu = M == -CUDART_INF_F ? 0.f : M;
+        for (int c = c_lo; c <= c_hi; ++c) {
+            const float *ps = partials + ((size_t)(c + b) * kHeads + h) * kLatPartialStride;
+            const float w = ex2(__ldcg(ps) - Mu);
+            const float4 v = __ldcg(reinterpret_cast<const float4 *>(ps + 4) + tid);
+            L += w * __ldcg(ps + 1);
+            acc.x += w * v.x; acc.y += w * v.y; acc.z += w * v.z; acc.w += w * v.w;
+        }
+    }
+    const float inv = 1.f / L;
+    const float4 res = make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
+    reinterpret_cast<float4 *>(out + ((size_t)b * n_heads + h) * kLatDim)[tid] = res;
+    if (status != nullptr && !(isfinite(res.x) && isfinite(res.y) && isfinite(res.z) && isfinite(res.w))) atomicOr(status, 1);
+}
+
+}  // namespace
+
+// ---------------------------------------------------------------------------------------------
+// C ABI
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+inline size_t lat_align(size_t x) { return (x + 255) / 256 * 256; }
+inline bool lat_misaligned(const void *p, size_t a) { return p != nullptr && (reinterpret_cast<uintptr_t>(p) % a) != 0; }
+
+int check_latent_geom(const santapp_latent_geom *g)
+{
+    if (!g) return SANTAPP_ERR_INVALID_ARG;
+    if (g->n_seqs < 1 || g->n_heads < 1 || g->parent_size < 1 || g->reps_per_parent < 1) return SANTAPP_ERR_INVALID_ARG;
+    if (g->parent_size % g->reps_per_parent != 0) return SANTAPP_ERR_INVALID_ARG;
+    if (g->n_heads > kHeads || g->parent_size > kMaxP || g->n_seqs > kMaxLatentSeqs) return SANTAPP_ERR_UNSUPPORTED;
+    return SANTAPP_OK;
+}
+
+int latent_teams_in_sequence(int N, int P, int R)
+{
+    const int full = N / P, tail = N % P;
+    return full * (R < P ? R : P) + (tail ? (R < tail ? R : tail) : 0);
+}
+
+int check_latent_teams(const santapp_latent_geom *g, const santapp_latent_teams *t)
+{
+    if (!t) return SANTAPP_ERR_INVALID_ARG;
+    if (!t->rows_packed || !t->rep_rows || !t->team_row_start || !t->seq_row_off || !t->seq_team_off || !t->rep_abs_max)
+        return SANTAPP_ERR_INVALID_ARG;
+    if (lat_misaligned(t->rows_packed, 16) || lat_misaligned(t->rep_rows, 16) || lat_misaligned(t->team_row_start, 4)
+        || lat_misaligned(t->row_token, 4) || lat_misaligned(t->seq_row_off, 8) || lat_misaligned(t->seq_team_off, 8)
+        || lat_misaligned(t->rep_abs_max, 4))
+        return SANTAPP_ERR_INVALID_ARG;
+    if (t->rows_total < g->n_seqs || t->teams_total < g->n_seqs || t->max_teams_per_seq < 1) return SANTAPP_ERR_INVALID_ARG;
+    if (t->rows_total >= (int64_t)1 << 31) return SANTAPP_ERR_UNSUPPORTED;
+    if (t->max_teams_per_seq > kMaxTeamsPerSeq) return SANTAPP_ERR_UNSUPPORTED;
+    return SANTAPP_OK;
+}
+
+LatentView make_latent_view(const santapp_latent_geom *g, const santapp_latent_teams *t)
+{
+    LatentView lv;
+    lv.n_seqs = g->n_seqs;
+    lv.n_heads = g->n_heads;
+    lv.seq_row_off = t->seq_row_off;
+    lv.seq_team_off = t->seq_team_off;
+    lv.rows_total = t->rows_total;
+    lv.teams_total = t->teams_total;
+    return lv;
+}
+
+// Workspace of the decode calls. Offsets in bytes.
+struct LatentLayout {
+    size_t y32, sel_team, sel_logc, sel_rows, row_meta, seg_bias, pair_rows, pair_prefix, partials, total;
+    int seg_cap, grid;
+    int64_t y_stride;
+};
+
+LatentLayout latent_layout(const santapp_latent_geom *g, const santapp_latent_teams *t, int K, int suffix_cap, bool dense)
+{
+    LatentLayout L;
+    L.grid = attend_grid_size();
+    int64_t cap = (int64_t)g->n_heads * K;
+    if (cap > t->max_teams_per_seq) cap = t->max_teams_per_seq;
+    L.seg_cap = (int)cap + 1;
+    L.y_stride = score_row_stride(t->max_teams_per_seq);
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = lat_align(off + bytes); return o; };
+    const size_t heads = (size_t)g->n_seqs * g->n_heads;
+    L.y32 = take(dense ? 0 : sizeof(float) * (size_t)g->n_heads * g->n_seqs * (size_t)L.y_stride);
+    L.sel_team = take(dense ? 0 : sizeof(int32_t) * heads * K);
+    L.sel_logc = take(dense ? 0 : sizeof(float) * heads * K);
+    L.sel_rows = take(dense ? 0 : sizeof(int2) * heads * K);
+    L.row_meta = take(dense ? 0 : sizeof(int2) * ((size_t)t->rows_total + (size_t)g->n_seqs * suffix_cap));
+    L.seg_bias = take(dense ? 0 : sizeof(float) * (size_t)g->n_seqs * L.seg_cap * kHeads);
+    L.pair_rows = take(sizeof(int32_t) * (size_t)g->n_seqs);
+    L.pair_prefix = take(sizeof(uint32_t) * ((size_t)g->n_seqs + 1));
+    L.partials = take(sizeof(float) * ((size_t)L.grid + g->n_seqs) * kHeads * kLatPartialStride);
+    L.total = off;
+    return L;
+}
+
+int latent_attend_and_merge(const santapp_latent_geom *geom, const santapp_latent_teams *teams, const LatentLayout &L, char *ws,
+                            const void *q, const void *suffix_rows, const int32_t *suffix_len_dev, int suffix_cap, float scale,
+                            float *out, int32_t *status, bool dense, int mask, int &launches, cudaStream_t s)
+{
+    LatentAttendParams ap;
+    ap.lv = make_latent_view(geom, teams);
+    ap.rows_packed = static_cast<const uint16_t *>(teams->rows_packed);
+    ap.suffix_rows = static_cast<const uint16_t *>(suffix_rows);
+    ap.q = static_cast<const uint16_t *>(q);
+    ap.row_meta = reinterpret_cast<const int2 *>(ws + L.row_meta);
+    ap.seg_bias = reinterpret_cast<const float *>(ws + L.seg_bias);
+    ap.pair_rows = reinterpret_cast<const int32_t *>(ws + L.pair_rows);
+    ap.suffix_len = suffix_cap > 0 ? suffix_len_dev : nullptr;
+    ap.suffix_cap = suffix_cap;
+    ap.seg_cap = L.seg_cap;
+    ap.qk_scale_log2 = (float)((double)scale * 1.4426950408889634);
+    ap.partials = reinterpret_cast<float *>(ws + L.partials);
+    ap.pair_prefix = reinterpret_cast<uint32_t *>(ws + L.pair_prefix);
+    cudaError_t err;
+    if (mask & SANTAPP_STAGE_ATTEND) {
+        static std::atomic<unsigned long long> done_all, done_sel;
+        if (dense) {
+            if ((err = ensure_dynamic_smem((const void *)latent_attend_kernel<true>, kLaSmemBytes, done_all)) != cudaSuccess)
+                return note_cuda_failure(err, "latent attend attribute");
+            err = launch_kernel(latent_attend_kernel<true>, dim3(L.grid), dim3(kLaThreads), kLaSmemBytes, s, ap);
+        } else {
+            if ((err = ensure_dynamic_smem((const void *)latent_attend_kernel<false>, kLaSmemBytes, done_sel)) != cudaSuccess)
+                return note_cuda_failure(err, "latent attend attribute");
+            err = launch_kernel(latent_attend_kernel<false>, dim3(L.grid), dim3(kLaThreads), kLaSmemBytes, s, ap);
+        }
+        if (err != cudaSuccess) return note_cuda_failure(err, "latent attend launch");
+        ++launches;
+    }
+    if (mask & SANTAPP_STAGE_MERGE) {
+        err = launch_kernel(latent_merge_kernel, dim3(geom->n_heads, geom->n_seqs), dim3(128), 0, s,
+                            (const float *)ap.partials, (const uint32_t *)ap.pair_prefix, geom->n_seqs, geom->n_heads, L.grid, out,
+                            status);
+        if (err != cudaSuccess) return note_cuda_failure(err, "latent merge launch");
+        ++launches;
+    }
+    return SANTAPP_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int santapp_latent_sizes(const santapp_latent_geom *geom, const int32_t *prompt_len_host, santapp_sizes *out)
+{
+    const int rc = check_latent_geom(geom);
+    if (rc != SANTAPP_OK) return rc;
+    if (!prompt_len_host || !out) return SANTAPP_ERR_INVALID_ARG;
+    int64_t rows = 0, tms = 0;
+    int max_t = 0, max_r = 0;
+    for (int b = 0; b < geom->n_seqs; ++b) {
+        const int N = prompt_len_host[b];
+        if (N < 1) return SANTAPP_ERR_INVALID_ARG;
+        const int M = latent_teams_in_sequence(N, geom->parent_size, geom->reps_per_parent);
+        rows += N;
+        tms += M;
+        if (M > max_t) max_t = M;
+        if (N > max_r) max_r = N;
+    }
+    if (rows >= (int64_t)1 << 31) return SANTAPP_ERR_UNSUPPORTED;
+    if (max_t > kMaxTeamsPerSeq) return SANTAPP_ERR_UNSUPPORTED;
+    out->rows_total = rows;
+    out->teams_total = tms;
+    out->max_teams_per_seq = max_t;
+    out->max_rows_per_seq = max_r;
+    out->team_row_start_elems = tms + geom->n_seqs;
+    out->build_workspace_bytes = lat_align((size_t)rows);
+    return SANTAPP_OK;
+}
+
+int santapp_latent_build_teams(const santapp_latent_geom *geom, const int32_t *prompt_len_host, const void *rows_prompt,
+                               santapp_latent_teams *teams, void *workspace, size_t workspace_bytes, santapp_stream stream)
+{
+    santapp_sizes sz;
+    const int rc = santapp_latent_sizes(geom, prompt_len_host, &sz);
+    if (rc != SANTAPP_OK) return rc;
+    if (!rows_prompt || !teams || !workspace) return SANTAPP_ERR_INVALID_ARG;
+    if (!teams->rows_packed || !teams->rep_rows || !teams->team_row_start || !teams->row_token || !teams->seq_row_off
+        || !teams->seq_team_off || !teams->rep_abs_max)
+        return SANTAPP_ERR_INVALID_ARG;
+    if (lat_misaligned(rows_prompt, 16) || lat_misaligned(workspace, 16) || lat_misaligned(teams->rows_packed, 16)
+        || lat_misaligned(teams->rep_rows, 16) || lat_misaligned(teams->team_row_start, 4) || lat_misaligned(teams->row_token, 4)
+        || lat_misaligned(teams->seq_row_off, 8) || lat_misaligned(teams->seq_team_off, 8) || lat_misaligned(teams->rep_abs_max, 4))
+        return SANTAPP_ERR_INVALID_ARG;
+    if (workspace_bytes < sz.build_workspace_bytes) return SANTAPP_ERR_WORKSPACE_TOO_SMALL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+
+    std::vector<int64_t> offs(2 * ((size_t)geom->n_seqs + 1));
+    int64_t *row_off = offs.data(), *team_off = offs.data() + geom->n_seqs + 1;
+    row_off[0] = team_off[0] = 0;
+    int max_parents = 0;
+    for (int b = 0; b < geom->n_seqs; ++b) {
+        const int N = prompt_len_host[b];
+        row_off[b + 1] = row_off[b] + N;
+        team_off[b + 1] = team_off[b] + latent_teams_in_sequence(N, geom->parent_size, geom->reps_per_parent);
+        max_parents = std::max(max_parents, (N + geom->parent_size - 1) / geom->parent_size);
+    }
+    const size_t ob = sizeof(int64_t) * ((size_t)geom->n_seqs + 1);
+    cudaError_t err = cudaMemcpyAsync(teams->seq_row_off, row_off, ob, cudaMemcpyHostToDevice, s);
+    if (err != cudaSuccess) return note_cuda_failure(err, "copy seq_row_off");
+    err = cudaMemcpyAsync(teams->seq_team_off, team_off, ob, cudaMemcpyHostToDevice, s);
+    if (err != cudaSuccess) return note_cuda_failure(err, "copy seq_team_off");
+    teams->rows_total = sz.rows_total;
+    teams->teams_total = sz.teams_total;
+    teams->max_teams_per_seq = sz.max_teams_per_seq;
+    teams->max_rows_per_seq = sz.max_rows_per_seq;
+
+    LatentBuildParams p;
+    p.lv = make_latent_view(geom, teams);
+    p.parent_size = geom->parent_size;
+    p.reps = geom->reps_per_parent;
+    p.teams_per_full_parent = std::min(geom->reps_per_parent, geom->parent_size);
+    p.rows_prompt = static_cast<const uint16_t *>(rows_prompt);
+    p.rows_packed = static_cast<uint16_t *>(teams->rows_packed);
+    p.rep_rows = static_cast<uint16_t *>(teams->rep_rows);
+    p.team_row_start = teams->team_row_start;
+    p.row_token = teams->row_token;
+    p.rep_abs_max = teams->rep_abs_max;
+    p.owner = static_cast<uint8_t *>(workspace);
+    p.max_parents_per_seq = max_parents;
+    const dim3 grid(max_parents, geom->n_seqs);
+    if ((err = launch_kernel(latent_build_parent_kernel, grid, dim3(kLbThreads), 0, s, p)) != cudaSuccess)
+        return note_cuda_failure(err, "latent build launch");
+    if ((err = launch_kernel(latent_scan_kernel, dim3(geom->n_seqs), dim3(256), 0, s, p)) != cudaSuccess)
+        return note_cuda_failure(err, "latent scan launch");
+    if ((err = launch_kernel(latent_pack_kernel, grid, dim3(kLbThreads), 0, s, p)) != cudaSuccess)
+        return note_cuda_failure(err, "latent pack launch");
+    return SANTAPP_OK;
+}
+
+size_t santapp_latent_decode_workspace_bytes(const santapp_latent_geom *geom, const santapp_latent_teams *teams, int32_t n_sample,
+                                             int32_t suffix_cap)
+{
+    if (check_latent_geom(geom) != SANTAPP_OK || !teams || n_sample < 1 || n_sample > 128 || suffix_cap < 0) return 0;
+    return latent_layout(geom, teams, n_sample, suffix_cap, false).total;
+}
+
+size_t santapp_latent_dense_workspace_bytes(const santapp_latent_geom *geom, const santapp_latent_teams *teams)
+{
+    if (check_latent_geom(geom) != SANTAPP_OK || !teams) return 0;
+    return latent_layout(geom, teams, 1, 0, true).total;
+}
+
+int santapp_latent_decode_attn(const santapp_latent_geom *geom, const santapp_latent_teams *teams, const void *q,
+                               const void *suffix_rows, const int32_t *suffix_len_dev, int32_t suffix_cap, int32_t n_sample,
+                               uint64_t seed, uint32_t step, const uint32_t *step_dev, uint32_t stream_base, float scale,
+                               float *out, const santapp_debug *dbg, void *workspace, size_t workspace_bytes,
+                               santapp_stream stream)
+{
+    note_launch_count(0);
+    int rc = check_latent_geom(geom);
+    if (rc != SANTAPP_OK) return rc;
+    if ((rc = check_latent_teams(geom, teams)) != SANTAPP_OK) return rc;
+    if (!q || !out || !workspace) return SANTAPP_ERR_INVALID_ARG;
+    if (lat_misaligned(q, 16) || lat_misaligned(out, 16) || lat_misaligned(workspace, 16) || lat_misaligned(suffix_rows, 16)
+        || lat_misaligned(suffix_len_dev, 4))
+        return SANTAPP_ERR_INVALID_ARG;
+    if (n_sample < 1 || suffix_cap < 0) return SANTAPP_ERR_INVALID_ARG;
+    if (n_sample > 128) return SANTAPP_ERR_UNSUPPORTED;
+    if (suffix_cap > 0 && suffix_len_dev && !suffix_rows) return SANTAPP_ERR_INVALID_ARG;
+    if (!(scale > 0.f) || isinf(scale)) return SANTAPP_ERR_INVALID_ARG;
+    if ((int64_t)geom->n_seqs * (int64_t)suffix_cap + teams->rows_total >= (int64_t)1 << 31) return SANTAPP_ERR_UNSUPPORTED;
+    const LatentLayout L = latent_layout(geom, teams, n_sample, suffix_cap, false);
+    if (workspace_bytes < L.total) return SANTAPP_ERR_WORKSPACE_TOO_SMALL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    char *ws = static_cast<char *>(workspace);
+    const int mask = current_stage_mask();
+    int launches = 0;
+    cudaError_t err;
+    int32_t *status = dbg ? dbg->status : nullptr;
+    if (status) {
+        if ((err = cudaMemsetAsync(status, 0, sizeof(int32_t), s)) != cudaSuccess) return note_cuda_failure(err, "clear status");
+    }
+    const LatentView lv = make_latent_view(geom, teams);
+
+    if (mask & SANTAPP_STAGE_ROUTE) {
+        LatentScoreParams sp;
+        sp.lv = lv;
+        sp.rep_rows = static_cast<const uint16_t *>(teams->rep_rows);
+        sp.team_row_start = teams->team_row_start;
+        sp.q = static_cast<const uint16_t *>(q);
+        sp.y32 = reinterpret_cast<float *>(ws + L.y32);
+        sp.y_stride = L.y_stride;
+        sp.n_sample = n_sample;
+        sp.seed_lo = (uint32_t)(seed & 0xFFFFFFFFull);
+        sp.seed_hi = (uint32_t)(seed >> 32);
+        sp.step = step;
+        sp.step_dev = step_dev;
+        sp.stream_base = stream_base;
+        sp.scale = scale;
+        const dim3 grid((teams->max_teams_per_seq + kLsTeamsPerBlock - 1) / kLsTeamsPerBlock, geom->n_seqs);
+        if ((err = launch_kernel(latent_score_kernel, grid, dim3(kLsThreads), 0, s, sp)) != cudaSuccess)
+            return note_cuda_failure(err, "latent score launch");
+        ++launches;
+    }
+    if (mask & SANTAPP_STAGE_SELECT) {
+        PlanInputs in = {};
+        in.bv.n_seqs = geom->n_seqs;
+        in.bv.n_q = geom->n_heads;
+        in.bv.n_kv = 1;
+        in.bv.group = geom->n_heads;
+        in.bv.seq_row_off = teams->seq_row_off;
+        in.bv.seq_team_off = teams->seq_team_off;
+        in.bv.team_count = nullptr;
+        in.bv.rows_total = teams->rows_total;
+        in.bv.teams_total = teams->teams_total;
+        in.bv.elem = 0;
+        in.y32 = reinterpret_cast<const float *>(ws + L.y32);
+        in.y_stride = L.y_stride;
+        in.rep_keys = static_cast<const uint16_t *>(teams->rep_rows);
+        in.team_row_start = teams->team_row_start;
+        in.rep_abs_max = teams->rep_abs_max;
+        in.q = static_cast<const uint16_t *>(q);
+        in.n_sample = n_sample;
+        in.seed_lo = (uint32_t)(seed & 0xFFFFFFFFull);
+        in.seed_hi = (uint32_t)(seed >> 32);
+        in.step = step;
+        in.step_dev = step_dev;
+        in.stream_base = stream_base;
+        in.scale = (double)scale;
+        in.suffix_len = suffix_cap > 0 ? suffix_len_dev : nullptr;
+        in.suffix_cap = suffix_cap;
+        in.sel_team = reinterpret_cast<int32_t *>(ws + L.sel_team);
+        in.sel_logc = reinterpret_cast<float *>(ws + L.sel_logc);
+        in.sel_rows = reinterpret_cast<int2 *>(ws + L.sel_rows);
+        in.status = status;
+        in.dbg_sel_idx = dbg ? dbg->sel_idx : nullptr;
+        in.dbg_sel_logc = dbg ? dbg->sel_logc : nullptr;
+        in.dbg_tau = dbg ? dbg->tau : nullptr;
+        in.dbg_union_rows = nullptr;
+        in.trace = nullptr;
+        const int n_heads = geom->n_seqs * geom->n_heads;
+        if (n_heads <= L.grid) err = launch_kernel(latent_select_kernel<512>, dim3(n_heads), dim3(512), 0, s, in);
+        else                   err = launch_kernel(latent_select_kernel<256>, dim3(n_heads), dim3(256), 0, s, in);
+        if (err != cudaSuccess) return note_cuda_failure(err, "latent select launch");
+        ++launches;
+
+        LatentPlanParams pp;
+        pp.lv = lv;
+        pp.sel_team = in.sel_team;
+        pp.sel_logc = in.sel_logc;
+        pp.sel_rows = in.sel_rows;
+        pp.suffix_len = in.suffix_len;
+        pp.suffix_cap = suffix_cap;
+        pp.n_sample = n_sample;
+        pp.seg_cap = L.seg_cap;
+        pp.row_meta = reinterpret_cast<int2 *>(ws + L.row_meta);
+        pp.seg_bias = reinterpret_cast<float *>(ws + L.seg_bias);
+        pp.pair_rows = reinterpret_cast<int32_t *>(ws + L.pair_rows);
+        pp.dbg_sel_idx = in.dbg_sel_idx;
+        pp.dbg_sel_logc = in.dbg_sel_logc;
+        pp.dbg_tau = in.dbg_tau;
+        pp.dbg_union_rows = dbg ? dbg->union_rows : nullptr;
+        static std::atomic<unsigned long long> done_plan;
+        if ((err = ensure_dynamic_smem((const void *)latent_plan_kernel, (int)sizeof(LatentPlanSmem), done_plan)) != cudaSuccess)
+            return note_cuda_failure(err, "latent plan attribute");
+        if ((err = launch_kernel(latent_plan_kernel, dim3(geom->n_seqs), dim3(kLpThreads), sizeof(LatentPlanSmem), s, pp)) != cudaSuccess)
+            return note_cuda_failure(err, "latent plan launch");
+        ++launches;
+    }
+    rc = latent_attend_and_merge(geom, teams, L, ws, q, suffix_rows, suffix_len_dev, suffix_cap, scale, out, status, false, mask,
+                                 launches, s);
+    note_launch_count(launches);
+    return rc;
+}
+
+int santapp_latent_dense_decode_attn(const santapp_latent_geom *geom, const santapp_latent_teams *teams, const void *q,
+                                     const void *suffix_rows, const int32_t *suffix_len_dev, int32_t suffix_cap, float scale,
+                                     float *out, void *workspace, size_t workspace_bytes, santapp_stream stream)
+{
+    note_launch_count(0);
+    int rc = check_latent_geom(geom);
+    if (rc != SANTAPP_OK) return rc;
+    if ((rc = check_latent_teams(geom, teams)) != SANTAPP_OK) return rc;
+    if (!q || !out || !workspace) return SANTAPP_ERR_INVALID_ARG;
+    if (lat_misaligned(q, 16) || lat_misaligned(out, 16) || lat_misaligned(workspace, 16) || lat_misaligned(suffix_rows, 16)
+        || lat_misaligned(suffix_len_dev, 4))
+        return SANTAPP_ERR_INVALID_ARG;
+    if (suffix_cap < 0) return SANTAPP_ERR_INVALID_ARG;
+    if (suffix_cap > 0 && suffix_len_dev && !suffix_rows) return SANTAPP_ERR_INVALID_ARG;
+    if (!(scale > 0.f) || isinf(scale)) return SANTAPP_ERR_INVALID_ARG;
+    if ((int64_t)geom->n_seqs * (int64_t)suffix_cap + teams->rows_total >= (int64_t)1 << 31) return SANTAPP_ERR_UNSUPPORTED;
+    const LatentLayout L = latent_layout(geom, teams, 1, 0, true);
+    if (workspace_bytes < L.total) return SANTAPP_ERR_WORKSPACE_TOO_SMALL;
+    int launches = 0;
+    rc = latent_attend_and_merge(geom, teams, L, static_cast<char *>(workspace), q, suffix_rows, suffix_len_dev, suffix_cap, scale,
+                                 out, nullptr, true, SANTAPP_STAGE_ATTEND | SANTAPP_STAGE_MERGE, launches,
+                                 static_cast<cudaStream_t>(stream));
+    note_launch_count(launches);
+    return rc;
+}
+
+}  // extern "C"

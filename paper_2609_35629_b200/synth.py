@@ -262,3 +262,96 @@ def _bisect_alpha(logits: np.ndarray, top: int, mass: float) -> float:
         else:
             hi = mid
     return 0.5 * (lo + hi)
+
+
+# ------------------------------------------------------------------------------------------------
+# Shared-latent rows (the paper's appendix "Token sparsity after latent compression": one row per
+# token, 512 content-latent values followed by 64 rotary-key values, shared by 16 heads). Stand-in
+# for the DeepSeek-V2-Lite cache of that study, which is not available. Recipe:
+#   latent part  n_clusters centres ~ N(0, I_512), row = centre + 0.3 * eps (cluster per row drawn
+#                uniformly at random), the first four rows multiplied by 4 ("sinks")
+#   rotary part  N(0, I_64)
+#   suffix rows  drawn like prompt rows (no sinks)
+#   queries      per (step, sequence, head): q = 0.55 * (row_j + 0.5 * eps) for a uniformly random
+#                prompt row j, over all 576 values; used with logit scale 1 / sqrt(192) (128 content
+#                + 64 rotary query values before absorption), the largest logit is then about 25
+# ------------------------------------------------------------------------------------------------
+LATENT_DIM, LATENT_ROPE_DIM = 512, 64
+LATENT_ROW = LATENT_DIM + LATENT_ROPE_DIM
+LATENT_SCALE = float(np.float32(1.0 / np.sqrt(192.0)))   # an fp32 value: the C ABI takes the scale as a float
+
+
+@dataclass
+class LatentSpec:
+    name: str
+    prompt_len: List[int]
+    n_heads: int = 16
+    n_clusters: int = 512
+    parent_size: int = 16
+    reps_per_parent: int = 4
+    n_sample: int = 128              # K teams per head (the paper's S = 512 rows at team size 4)
+    suffix_cap: int = 16
+    suffix_len0: Optional[List[int]] = None
+    suffix_growth: int = 1
+    seed: int = 0
+
+    @property
+    def n_seqs(self) -> int:
+        return len(self.prompt_len)
+
+    @property
+    def rows_total(self) -> int:
+        return int(sum(self.prompt_len))
+
+    def suffix_len(self, step: int) -> np.ndarray:
+        s0 = np.zeros(self.n_seqs, dtype=np.int64) if self.suffix_len0 is None else np.asarray(self.suffix_len0, dtype=np.int64)
+        return np.minimum(s0 + self.suffix_growth * step, self.suffix_cap).astype(np.int32)
+
+
+def spec_latent_8k(seed: int = 0, n_seqs: int = 32, n_sample: int = 128, prompt: int = 8192) -> LatentSpec:
+    """The paper's shared-latent study point: 8K context, P = 16, R = 4, 16 heads; a batch of sequences."""
+    return LatentSpec("latent_8k", [prompt] * n_seqs, n_sample=n_sample, seed=seed)
+
+
+@dataclass
+class LatentLayerData:
+    spec: LatentSpec
+    layer: int
+    rows: np.ndarray                 # [rows_total, 576] bf16 bits, token order, sequences concatenated
+    suffix: np.ndarray               # [n_seqs, suffix_cap, 576]
+    seq_row_off: np.ndarray
+
+
+def make_latent_layer(spec: LatentSpec, layer: int = 0) -> LatentLayerData:
+    off = np.zeros(spec.n_seqs + 1, dtype=np.int64)
+    off[1:] = np.cumsum(spec.prompt_len)
+    rows = np.empty((spec.rows_total, LATENT_ROW), dtype=np.uint16)
+    cap = max(spec.suffix_cap, 1)
+    suffix = np.empty((spec.n_seqs, cap, LATENT_ROW), dtype=np.uint16)
+    rng = np.random.default_rng([spec.seed, layer, 0, 11])
+    centres = rng.standard_normal((spec.n_clusters, LATENT_DIM), dtype=np.float32)
+    for b in range(spec.n_seqs):
+        n = spec.prompt_len[b]
+        x = np.empty((n, LATENT_ROW), dtype=np.float32)
+        x[:, :LATENT_DIM] = _clustered_rows(rng, n, centres)
+        x[:, LATENT_DIM:] = rng.standard_normal((n, LATENT_ROPE_DIM), dtype=np.float32)
+        x[: min(4, n)] *= np.float32(4.0)
+        rows[off[b]:off[b + 1]] = round_bits(x)
+        s = np.empty((cap, LATENT_ROW), dtype=np.float32)
+        s[:, :LATENT_DIM] = _clustered_rows(rng, cap, centres)
+        s[:, LATENT_DIM:] = rng.standard_normal((cap, LATENT_ROPE_DIM), dtype=np.float32)
+        suffix[b] = round_bits(s)
+    return LatentLayerData(spec, layer, rows, suffix, off)
+
+
+def make_latent_queries(spec: LatentSpec, data: LatentLayerData, step: int) -> np.ndarray:
+    """bf16 bits [n_seqs, n_heads, 576]."""
+    rng = np.random.default_rng([spec.seed, data.layer, step, 12])
+    q = np.empty((spec.n_seqs, spec.n_heads, LATENT_ROW), dtype=np.float32)
+    for b in range(spec.n_seqs):
+        lo, hi = int(data.seq_row_off[b]), int(data.seq_row_off[b + 1])
+        for h in range(spec.n_heads):
+            eps = rng.standard_normal(LATENT_ROW, dtype=np.float32)
+            row = to_f32(data.rows[int(rng.integers(lo, hi))])
+            q[b, h] = np.float32(0.55) * (row + np.float32(0.5) * eps)
+    return round_bits(q)

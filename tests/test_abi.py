@@ -1,4 +1,4 @@
-"""The C-ABI library loads and exports every symbol include/santapp.h declares; host-side
+"""The C-ABI library loads and exports every symbol include/*.h declares; host-side
 argument checks and size queries work without a GPU (no compute call is made here)."""
 import ctypes
 import os
@@ -19,7 +19,8 @@ def lib():
 
 
 def test_header_symbols_are_exported(lib):
-    header = open(os.path.join(ROOT, "include", "santapp.h")).read()
+    inc = os.path.join(ROOT, "include")
+    header = "".join(open(os.path.join(inc, f)).read() for f in sorted(os.listdir(inc)) if f.endswith(".h"))
     header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
     declared = set(re.findall(r"\b(santapp_[a-z_]+)\s*\(", header))
     assert declared, "no declarations found"
