@@ -55,8 +55,9 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--layers", type=int, default=28)
     ap.add_argument("--workload", default="qwen7b_b1_32k",
-                    choices=["qwen7b_b1_32k", "qwen7b_b8_32k", "ragged", "long_128k", "paper_point_32k", "small_gqa"])
+                    choices=["qwen7b_b1_32k", "qwen7b_b8_32k", "ragged", "long_128k", "paper_point_32k", "small_gqa", "latent_8k"])
     ap.add_argument("--n-sample", type=int, default=0, help="override K")
+    ap.add_argument("--latent-seqs", type=int, default=32, help="sequences of the latent_8k workload")
     ap.add_argument("--key-layout", default="iid", choices=["iid", "runs"],
                     help="cluster of each prompt row: independent draws, or geometric runs (positional locality)")
     ap.add_argument("--elem", default="bf16", choices=["bf16", "fp16"], help="16-bit element type of q, K, V")
@@ -232,6 +233,16 @@ def run_ours(args):
     replicas.init_replicas("nccl", dev)
     sp.load_library()
 
+    if args.workload == "latent_8k":
+        res = measure_latent(args, min(args.layers, 4), min(args.steps, 20), args.warmup, dev, n_seqs=args.latent_seqs,
+                             n_sample=args.n_sample or 128)
+        if rank == 0:
+            print(json.dumps({"metric": METRIC, "unit": UNIT, "n_gpus": world, "higher_is_better": False, "scaling": "weak",
+                              "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": {"workload": res["workload"]},
+                              **res}), flush=True)
+        if world > 1:
+            dist.destroy_process_group()
+        return
     line = measure_workload(args, args.workload, args.layers, args.steps, args.warmup, dev,
                             want_e2e=not args.no_e2e, want_cpu=not args.no_cpu_baseline, want_stages=not args.no_stages)
     # Beside the headline workload (batch 1, latency-bound on this GPU), the same measurement on a
@@ -255,6 +266,12 @@ def run_ours(args):
             res = measure_workload(wl_args, wl, n_lay, 10, 3, dev, want_e2e=False, want_cpu=False, want_stages=True)
             if rank == 0:
                 line[key] = {"workload": res["config"]["workload"], **{k: res[k] for k in keep}}
+        # shared-latent rows (one 576-value row per token, 16 heads) at the paper's 8K study point, 32 sequences
+        gc.collect()
+        torch.cuda.empty_cache()
+        lat = measure_latent(args, 4, 10, 3, dev)
+        if rank == 0:
+            line["shared_latent"] = lat
         # and the headline workload with the parents of the paper's headline runs: Algorithm 3
         # (minibatch k-means with the paper's settings, fitted by the library), four layers
         if args.parents == "contiguous" and args.elem == "bf16":
@@ -576,6 +593,162 @@ def measure_workload(args, workload, n_layers, n_steps, n_warmup, dev, want_e2e,
         }
         return line
     return None
+
+
+def measure_latent(args, n_layers, n_steps, n_warmup, dev, n_seqs=32, n_sample=128):
+    """Shared-latent rows (one 512 + 64 value row per token, 16 heads): the same measurement as
+    measure_workload on the paper's study point (8K context, P = 16, R = 4) as a batch of sequences.
+    Returns a dict on rank 0 (None elsewhere)."""
+    import torch
+    from paper_2609_35629_b200 import binding as sp
+    from paper_2609_35629_b200 import replicas, synth
+
+    rank, world, local_rank = replicas.env_rank_world()
+    spec = synth.spec_latent_8k(seed=replicas.replica_seed(0, rank), n_seqs=n_seqs, n_sample=n_sample)
+    L, B, H, K = n_layers, spec.n_seqs, spec.n_heads, spec.n_sample
+    geom = sp.LatentGeometry(B, H, spec.parent_size, spec.reps_per_parent)
+    ROW, DV = synth.LATENT_ROW, synth.LATENT_DIM
+    scale = synth.LATENT_SCALE
+    S = 4                                                   # distinct step inputs cycled through
+    layers = []
+    q_all = np.empty((S, L, B, H, ROW), dtype=np.uint16)
+    for l in range(L):
+        data = synth.make_latent_layer(spec, layer=l)
+        for s in range(S):
+            q_all[s, l] = synth.make_latent_queries(spec, data, s)
+        rows = sp.bf16_bits_to_cuda(data.rows, dev)
+        t0 = time.perf_counter()
+        teams = sp.santapp_latent_build_teams(geom, spec.prompt_len, rows)
+        torch.cuda.synchronize()
+        build_ms = 1e3 * (time.perf_counter() - t0)
+        del rows
+        layers.append(dict(teams=teams, suffix=sp.bf16_bits_to_cuda(data.suffix, dev)))
+    step_ids = [0, 5, 10, 15]
+    sl_all = np.stack([spec.suffix_len(st) for st in step_ids]).astype(np.int32)
+    q_dev = sp.bf16_bits_to_cuda(q_all, dev)
+    sl_dev = torch.from_numpy(sl_all).to(dev)
+    step_dev_all = torch.tensor(step_ids, dtype=torch.int32, device=dev)
+    q_cur = torch.empty_like(q_dev[0])
+    sl_cur = torch.empty_like(sl_dev[0])
+    step_cur = torch.zeros(1, dtype=torch.int32, device=dev)
+    out = torch.zeros((L, B, H, DV), dtype=torch.float32, device=dev)
+    out_dense = torch.zeros_like(out)
+    cap = spec.suffix_cap
+    ws = [torch.empty(sp.santapp_latent_decode_workspace_bytes(geom, layers[l]["teams"], K, cap), dtype=torch.uint8, device=dev)
+          for l in range(L)]
+    wsd = torch.empty(sp.santapp_latent_dense_workspace_bytes(geom, layers[0]["teams"]), dtype=torch.uint8, device=dev)
+    seed = replicas.replica_seed(1234, rank)
+
+    def sparse_layer(l, debug=None):
+        ly = layers[l]
+        sp.santapp_latent_decode_attn(geom, ly["teams"], q_cur[l], ly["suffix"], sl_cur, K, seed, 0, scale, stream_base=l * B,
+                                      out=out[l], debug=debug, workspace=ws[l], step_dev=step_cur)
+
+    def dense_layer(l):
+        ly = layers[l]
+        sp.santapp_latent_dense_decode_attn(geom, ly["teams"], q_cur[l], ly["suffix"], sl_cur, scale, out=out_dense[l], workspace=wsd)
+
+    def set_inputs(s):
+        q_cur.copy_(q_dev[s], non_blocking=True)
+        sl_cur.copy_(sl_dev[s], non_blocking=True)
+        step_cur.copy_(step_dev_all[s:s + 1], non_blocking=True)
+
+    dbg = sp.LatentDebugBuffers(geom, K, dev)
+    union = np.zeros((S, L), dtype=np.int64)
+    for s in range(S):
+        set_inputs(s)
+        for l in range(L):
+            sparse_layer(l, debug=dbg)
+            torch.cuda.synchronize()
+            union[s, l] = int(dbg.union_rows.sum().item())
+            assert int(dbg.status.item()) == 0, "non-finite output"
+    launches = sp.santapp_last_launch_count()
+    M_total = int(layers[0]["teams"].sizes.teams_total)
+    N_total = int(layers[0]["teams"].sizes.rows_total)
+    suffix_rows = sl_all.sum(axis=1).astype(np.int64)
+    io_bytes = B * H * (ROW * 2 + DV * 4)
+    attend_bytes = 2 * ROW * (union + suffix_rows[:, None]) + io_bytes              # one 1152-byte row per row read
+    route_bytes = M_total * ROW * 2 + (M_total + B) * 4
+    sparse_bytes = attend_bytes + route_bytes
+    dense_bytes = 2 * ROW * (N_total + suffix_rows) + io_bytes
+
+    def capture(fn):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            for l in range(L):
+                fn(l)
+        return g
+
+    set_inputs(0)
+    for l in range(L):
+        dense_layer(l)
+    torch.cuda.synchronize()
+    g_sparse, g_dense = capture(sparse_layer), capture(dense_layer)
+
+    def timed(run_step, steps, warmup):
+        for i in range(warmup):
+            run_step(i)
+        replicas.barrier(dev)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(steps):
+            run_step(warmup + i)
+        e1.record()
+        torch.cuda.synchronize()
+        ms = replicas.max_over_ranks(e0.elapsed_time(e1), dev)
+        replicas.barrier(dev)
+        return ms
+
+    def sparse_step(i):
+        set_inputs(i % S)
+        g_sparse.replay()
+
+    def dense_step(i):
+        set_inputs(i % S)
+        g_dense.replay()
+
+    W = max(n_warmup, 3)
+    us_sparse = replicas.us_per_layer_step(timed(sparse_step, n_steps, W), n_steps, L, world)
+    us_dense = replicas.us_per_layer_step(timed(dense_step, n_steps, W), n_steps, L, world)
+    used = np.array([(W + i) % S for i in range(n_steps)])
+    mean_sparse, mean_dense = float(sparse_bytes[used].mean()), float(dense_bytes[used].mean())
+    stages = {}
+    set_inputs(1)
+    g_sparse.replay()
+    torch.cuda.synchronize()
+    for name, mask in (("route_score", sp.STAGE_ROUTE), ("select_plan", sp.STAGE_SELECT), ("attend", sp.STAGE_ATTEND),
+                       ("merge", sp.STAGE_MERGE)):
+        sp.santapp_set_stage_mask(mask)
+        g = capture(sparse_layer)
+        sp.santapp_set_stage_mask(sp.STAGE_ALL)
+        reps = max(n_steps, 10)
+        stages[name] = 1e3 * timed(lambda i: g.replay(), reps, 3) / (reps * L)
+    peaks = {}
+    try:
+        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+    except Exception:
+        pass
+    peak_gbs = float(peaks.get("hbm_gbs", 6650.0))
+    attend_1 = float(attend_bytes[1].mean())
+    achieved = attend_1 / (stages["attend"] * 1e-6) / 1e9
+    if rank != 0:
+        return None
+    return {
+        "workload": (f"{spec.name}: {B} seq x {H} heads sharing one {ROW}-value row per token, prompt {spec.prompt_len[0]}, "
+                     f"suffix cap {cap}, P={spec.parent_size}, R={spec.reps_per_parent}, K={K}, contiguous parents, bf16, "
+                     f"{L} layers round-robin"),
+        "value": us_sparse, "unit": UNIT, "steps": n_steps, "warmup": W, "gpu_launches_per_layer_step": launches,
+        "dense_us_per_layer_step": us_dense, "speedup_vs_dense": us_dense / us_sparse,
+        "read_reduction": mean_dense / mean_sparse,
+        "achieved_frac_of_peak": mean_sparse / (us_sparse * 1e-6) / 1e9 / peak_gbs,
+        "dense_achieved_frac_of_peak": mean_dense / (us_dense * 1e-6) / 1e9 / peak_gbs,
+        "logical_access_pct": 100.0 * float((M_total + union[used].mean() + suffix_rows[used].mean())
+                                            / (N_total + suffix_rows[used].mean())),
+        "roofline": {"bound": "hbm", "kernel": "latent_attend_kernel", "achieved": achieved, "peak": peak_gbs, "unit": "GB/s",
+                     "frac": achieved / peak_gbs, "traffic": NCU_TRAFFIC_BYTES.get(spec.name) if (n_seqs, n_sample) == (32, 128) else None,
+                     "algorithmic_bytes_per_launch": attend_1, "us_per_launch": stages["attend"]},
+        "stage_us": stages, "team_build_ms_last_layer": build_ms,
+    }
 
 
 def kmeans_group_records(spec, data, dev):

@@ -7,7 +7,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 SOURCES = ["api.cu", "build_teams.cu", "build_parents.cu", "kmeans.cu", "score.cu", "headplan.cu", "plan.cu", "attend.cu", "latent.cu"]
-HEADERS = [os.path.join(CSRC, h) for h in ("common.cuh", "pairplan.cuh", "headplan.cuh", "score_tile.cuh", "build_util.cuh")] \
+HEADERS = [os.path.join(CSRC, h) for h in ("common.cuh", "pairplan.cuh", "headplan.cuh", "score_tile.cuh", "build_util.cuh", "latent_tc.cuh")] \
     + [os.path.join(ROOT, "include", h) for h in ("santapp.h", "santapp_latent.h")]
 OUT = os.path.join(HERE, "libsantapp.so")
 

@@ -69,7 +69,8 @@ template <int kT, int kScoreRegs, bool kHalf, int kDim = kHeadDim>
 __device__ __forceinline__ void select_head(const PlanInputs &in, int hq, HeadSmemT<kDim> &sm)
 {
     static_assert(kDim % 64 == 0, "eight lanes share a key, each takes whole 16-byte pieces");
-    constexpr int kHeadWarps = kT / 32, kDotWarps = kHeadWarps / 2;
+    constexpr bool kAllDot = kDim > 128;
+    constexpr int kHeadWarps = kT / 32, kDotWarps = kAllDot ? kHeadWarps : kHeadWarps / 2;
     constexpr int kSlice = kDim / kDotLanes;                          // dims per lane of a dot product
     constexpr int kPieces = kSlice / 8;                               // 16-byte pieces per lane
     constexpr int kQRegs = (kDim + kT - 1) / kT;                      // query values a thread converts
@@ -274,7 +275,9 @@ __device__ __forceinline__ void select_head(const PlanInputs &in, int hq, HeadSm
 
         // ---- 3a. exact terms: dot products on the first half of the warps (8 lanes per candidate, kDim / 8 dims each),
         //          log n_g and the Gumbel term on the other warps (one thread per candidate) ----
-        if (warp < kDotWarps) {
+        // Long keys (kAllDot): every warp takes part in the dot products (their round trips to memory
+        // are the longest chain of the kernel), then every thread takes a candidate's other terms.
+        if (kAllDot || warp < kDotWarps) {
             const int sub = lane & (kDotLanes - 1);
             const double *qs = sm.q64[sub];
             // a few candidates per thread group at a time: all their key pieces are requested before
@@ -317,8 +320,9 @@ __device__ __forceinline__ void select_head(const PlanInputs &in, int hq, HeadSm
                     if (cand < n_cand && sub == 0) sm.cand_y[cand] = d;
                 }
             }
-        } else {
-            for (int i = tid - kDotWarps * 32; i < n_cand; i += kT - kDotWarps * 32) {
+        }
+        if (kAllDot || warp >= kDotWarps) {
+            for (int i = kAllDot ? tid : tid - kDotWarps * 32; i < n_cand; i += kAllDot ? kT : kT - kDotWarps * 32) {
                 const int id = sm.cand_id[i];
                 const int r_lo = csr[id];
                 const int n_g = csr[id + 1] - r_lo;

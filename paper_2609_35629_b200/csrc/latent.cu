@@ -18,6 +18,9 @@
 #include <limits.h>
 #include <math_constants.h>
 
+#include <stdlib.h>
+#include <string.h>
+
 #include <algorithm>
 #include <vector>
 
@@ -489,6 +492,7 @@ struct LatentAttendParams {
     float qk_scale_log2;            // scale * log2(e)
     float *partials;                // [grid + n_seqs][16][kLatPartialStride]: block c leaves sequence b's share in slot c + b
     uint32_t *pair_prefix;          // [n_seqs + 1] rows to read before each sequence; written by block 0 for the merge
+    unsigned long long *trace;      // nullable: device-timer marks of the third tile of a block's first share (diagnostic)
 };
 
 constexpr int kLaThreads = 256;
@@ -811,33 +815,67 @@ latent_attend_kernel(LatentAttendParams p)
     }
 }
 
+}  // namespace
+
+#include "latent_tc.cuh"
+
+namespace {
+
 // One block per (head, sequence): out = sum_c w_c acc_c / sum_c w_c l_c over the blocks that read
-// rows of the sequence, w_c = 2^(m_c - max m). Thread i owns value columns 4 i .. 4 i + 3.
-__global__ void __launch_bounds__(128)
+// rows of the sequence, w_c = 2^(m_c - max m). Four thread groups take every fourth partial; thread
+// i of a group owns value columns 4 i .. 4 i + 3; the groups' sums meet in shared memory.
+constexpr int kLmThreads = 512;
+__global__ void __launch_bounds__(kLmThreads)
 latent_merge_kernel(const float *partials, const uint32_t *pair_prefix, int n_seqs, int n_heads, int grid, float *out, int32_t *status)
 {
-    const int h = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
+    __shared__ float red[kLmThreads / 32];
+    __shared__ float4 part_acc[3][128];
+    __shared__ float part_l[3][128];
+    const int h = blockIdx.x, b = blockIdx.y, tid = threadIdx.x, part = tid >> 7, col = tid & 127;
     const uint32_t total = pair_prefix[n_seqs], per = (total + grid - 1) / grid;
     const uint32_t lo = pair_prefix[b], hi = pair_prefix[b + 1];
+    const int c_lo = (int)(lo / per), c_hi = hi > lo ? (int)((hi - 1) / per) : c_lo - 1;
+    const float *base = partials + ((size_t)b * kHeads + h) * kLatPartialStride;      // slot c + b
+    const size_t slot = (size_t)kHeads * kLatPartialStride;
+    float M = -CUDART_INF_F;
+    for (int c = c_lo + tid; c <= c_hi; c += kLmThreads) M = fmaxf(M, __ldcg(base + c * slot));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xFFFFFFFFu, M, o));
+    if ((tid & 31) == 0) red[tid >> 5] = M;
+    __syncthreads();
+#pragma unroll
+    for (int w = 0; w < kLmThreads / 32; ++w) M = fmaxf(M, red[w]);
+    const float Mu = M == -CUDART_INF_F ? 0.f : M;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     float L = 0.f;
-    if (hi > lo) {
-        const int c_lo = (int)(lo / per), c_hi = (int)((hi - 1) / per);
-        float M = -CUDART_INF_F;
-        for (int c = c_lo; c <= c_hi; ++c) M = fmaxf(M, __ldcg(partials + ((size_t)(c + b) * kHeads + h) * kLatPartialStride));
-        const float Mu = M == -CUDART_INF_F ? 0.f : M;
-        for (int c = c_lo; c <= c_hi; ++c) {
-            const float *ps = partials + ((size_t)(c + b) * kHeads + h) * kLatPartialStride;
-            const float w = ex2(__ldcg(ps) - Mu);
-            const float4 v = __ldcg(reinterpret_cast<const float4 *>(ps + 4) + tid);
-            L += w * __ldcg(ps + 1);
-            acc.x += w * v.x; acc.y += w * v.y; acc.z += w * v.z; acc.w += w * v.w;
-        }
+    for (int c = c_lo + part; c <= c_hi; c += 8) {
+        const float *p0 = base + c * slot, *p1 = p0 + 4 * slot;
+        const bool two = c + 4 <= c_hi;
+        const float m0 = __ldcg(p0), l0 = __ldcg(p0 + 1);
+        const float4 v0 = __ldcg(reinterpret_cast<const float4 *>(p0 + 4) + col);
+        const float m1 = two ? __ldcg(p1) : -CUDART_INF_F, l1 = two ? __ldcg(p1 + 1) : 0.f;
+        const float4 v1 = two ? __ldcg(reinterpret_cast<const float4 *>(p1 + 4) + col) : make_float4(0.f, 0.f, 0.f, 0.f);
+        const float w0 = ex2(m0 - Mu), w1 = ex2(m1 - Mu);
+        L += w0 * l0 + w1 * l1;
+        acc.x += w0 * v0.x + w1 * v1.x;
+        acc.y += w0 * v0.y + w1 * v1.y;
+        acc.z += w0 * v0.z + w1 * v1.z;
+        acc.w += w0 * v0.w + w1 * v1.w;
     }
-    const float inv = 1.f / L;
-    const float4 res = make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
-    reinterpret_cast<float4 *>(out + ((size_t)b * n_heads + h) * kLatDim)[tid] = res;
-    if (status != nullptr && !(isfinite(res.x) && isfinite(res.y) && isfinite(res.z) && isfinite(res.w))) atomicOr(status, 1);
+    if (part > 0) { part_acc[part - 1][col] = acc; part_l[part - 1][col] = L; }
+    __syncthreads();
+    if (part == 0) {
+#pragma unroll
+        for (int g = 0; g < 3; ++g) {
+            const float4 v = part_acc[g][col];
+            acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+            L += part_l[g][col];
+        }
+        const float inv = 1.f / L;
+        const float4 res = make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
+        reinterpret_cast<float4 *>(out + ((size_t)b * n_heads + h) * kLatDim)[col] = res;
+        if (status != nullptr && !(isfinite(res.x) && isfinite(res.y) && isfinite(res.z) && isfinite(res.w))) atomicOr(status, 1);
+    }
 }
 
 }  // namespace
@@ -925,7 +963,8 @@ LatentLayout latent_layout(const santapp_latent_geom *g, const santapp_latent_te
 
 int latent_attend_and_merge(const santapp_latent_geom *geom, const santapp_latent_teams *teams, const LatentLayout &L, char *ws,
                             const void *q, const void *suffix_rows, const int32_t *suffix_len_dev, int suffix_cap, float scale,
-                            float *out, int32_t *status, bool dense, int mask, int &launches, cudaStream_t s)
+                            float *out, int32_t *status, bool dense, int mask, int &launches, cudaStream_t s,
+                            unsigned long long *trace = nullptr)
 {
     LatentAttendParams ap;
     ap.lv = make_latent_view(geom, teams);
@@ -941,23 +980,39 @@ int latent_attend_and_merge(const santapp_latent_geom *geom, const santapp_laten
     ap.qk_scale_log2 = (float)((double)scale * 1.4426950408889634);
     ap.partials = reinterpret_cast<float *>(ws + L.partials);
     ap.pair_prefix = reinterpret_cast<uint32_t *>(ws + L.pair_prefix);
+    ap.trace = trace;
     cudaError_t err;
     if (mask & SANTAPP_STAGE_ATTEND) {
-        static std::atomic<unsigned long long> done_all, done_sel;
-        if (dense) {
-            if ((err = ensure_dynamic_smem((const void *)latent_attend_kernel<true>, kLaSmemBytes, done_all)) != cudaSuccess)
+        static std::atomic<unsigned long long> done_all, done_sel, done_tc_all, done_tc_sel;
+        // The tcgen05 variant (latent_tc.cuh) computes the same thing on the 5th-generation tensor cores; it is
+        // slower here (a tcgen05.mma of N = 16 columns costs as much as one of 64, and one thread issues 68 of
+        // them per 64 rows), so the mma.sync kernel is the default and the other is chosen by the environment.
+        const char *which = getenv("SANTAPP_LATENT_ATTEND");
+        const bool legacy = !(which != nullptr && strcmp(which, "tcgen05") == 0);
+        if (legacy) {
+            if (dense) {
+                if ((err = ensure_dynamic_smem((const void *)latent_attend_kernel<true>, kLaSmemBytes, done_all)) != cudaSuccess)
+                    return note_cuda_failure(err, "latent attend attribute");
+                err = launch_kernel(latent_attend_kernel<true>, dim3(L.grid), dim3(kLaThreads), kLaSmemBytes, s, ap);
+            } else {
+                if ((err = ensure_dynamic_smem((const void *)latent_attend_kernel<false>, kLaSmemBytes, done_sel)) != cudaSuccess)
+                    return note_cuda_failure(err, "latent attend attribute");
+                err = launch_kernel(latent_attend_kernel<false>, dim3(L.grid), dim3(kLaThreads), kLaSmemBytes, s, ap);
+            }
+        } else if (dense) {
+            if ((err = ensure_dynamic_smem((const void *)latent_attend_tc_kernel<true>, kTcSmemBytes, done_tc_all)) != cudaSuccess)
                 return note_cuda_failure(err, "latent attend attribute");
-            err = launch_kernel(latent_attend_kernel<true>, dim3(L.grid), dim3(kLaThreads), kLaSmemBytes, s, ap);
+            err = launch_kernel(latent_attend_tc_kernel<true>, dim3(L.grid), dim3(kTcThreads), kTcSmemBytes, s, ap, status);
         } else {
-            if ((err = ensure_dynamic_smem((const void *)latent_attend_kernel<false>, kLaSmemBytes, done_sel)) != cudaSuccess)
+            if ((err = ensure_dynamic_smem((const void *)latent_attend_tc_kernel<false>, kTcSmemBytes, done_tc_sel)) != cudaSuccess)
                 return note_cuda_failure(err, "latent attend attribute");
-            err = launch_kernel(latent_attend_kernel<false>, dim3(L.grid), dim3(kLaThreads), kLaSmemBytes, s, ap);
+            err = launch_kernel(latent_attend_tc_kernel<false>, dim3(L.grid), dim3(kTcThreads), kTcSmemBytes, s, ap, status);
         }
         if (err != cudaSuccess) return note_cuda_failure(err, "latent attend launch");
         ++launches;
     }
     if (mask & SANTAPP_STAGE_MERGE) {
-        err = launch_kernel(latent_merge_kernel, dim3(geom->n_heads, geom->n_seqs), dim3(128), 0, s,
+        err = launch_kernel(latent_merge_kernel, dim3(geom->n_heads, geom->n_seqs), dim3(kLmThreads), 0, s,
                             (const float *)ap.partials, (const uint32_t *)ap.pair_prefix, geom->n_seqs, geom->n_heads, L.grid, out,
                             status);
         if (err != cudaSuccess) return note_cuda_failure(err, "latent merge launch");
@@ -1188,7 +1243,7 @@ int santapp_latent_decode_attn(const santapp_latent_geom *geom, const santapp_la
         ++launches;
     }
     rc = latent_attend_and_merge(geom, teams, L, ws, q, suffix_rows, suffix_len_dev, suffix_cap, scale, out, status, false, mask,
-                                 launches, s);
+                                 launches, s, dbg ? reinterpret_cast<unsigned long long *>(dbg->trace) : nullptr);
     note_launch_count(launches);
     return rc;
 }

@@ -197,6 +197,21 @@ def test_step_full_bench_batch_sampled_sequences():
     check_dense(layer, 0, seqs=[0, 31])
 
 
+def test_tcgen05_variant_of_the_attention_kernel(small, monkeypatch):
+    """The tensor-memory variant (chosen by the environment) against the oracle: sparse with a ragged
+    tail and a suffix, dense, and a sequence of the full batch shape; its bounded waits must not expire."""
+    monkeypatch.setenv("SANTAPP_LATENT_ATTEND", "tcgen05")
+    check_step(small, 3)
+    check_dense(small, 9)
+    layer = LatentLayer(synth.LatentSpec("8k", [8192, 5000], suffix_cap=16, suffix_len0=[0, 5]))
+    check_step(layer, 1, K=128)
+    check_dense(layer, 1)
+    for H, lens in ((5, [1, 17, 1000]), (9, [31, 33])):
+        odd = LatentLayer(synth.LatentSpec(f"h{H}", lens, n_heads=H, n_sample=7, suffix_cap=3, suffix_len0=[1] * len(lens)))
+        check_step(odd, 2)
+        check_dense(odd, 2)
+
+
 def test_same_seed_same_bits_and_step_changes_the_sample(small):
     q_bits = synth.make_latent_queries(small.spec, small.data, 0)
     sl = small.spec.suffix_len(0)
