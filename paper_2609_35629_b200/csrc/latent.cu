@@ -354,7 +354,9 @@ __global__ void __launch_bounds__(kT, kT >= 512 ? 1 : 1024 / kT)
 latent_select_kernel(PlanInputs in)
 {
     __shared__ HeadSmemT<kRowDim> sm;
+    trace_mark(in.trace, 1, 0);
     select_head<kT, kT >= 512 ? 4 : 2, false, kRowDim>(in, blockIdx.x, sm);
+    trace_mark(in.trace, 1, 1);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -624,33 +626,44 @@ latent_attend_kernel(LatentAttendParams p)
 #pragma unroll
         for (int j2 = 0; j2 < 16; ++j2) o[j2][0] = o[j2][1] = o[j2][2] = o[j2][3] = 0.f;
 
-        // source row (and segment) of this thread's row of the group's j-th tile; x = -1: no row
-        auto load_meta = [&](int j) -> int2 {
-            const int pos = s_lo + kTileRows * (grp + 2 * j) + (gt >> 2);
-            if (j >= my_tiles || pos >= s_hi) return make_int2(-1, 0);
-            if (kAll)
-                return make_int2(pos < N ? (int)(row0 + pos) : (int)(kSrcSuffix | (uint32_t)(b * p.suffix_cap + pos - N)), 0);
-            return __ldcg(line + pos);
+        // source rows (and segments) of this thread's two rows of the group's j-th tile, rows gt / 8 and
+        // gt / 8 + 16; source -1: no row
+        auto load_meta = [&](int j) -> int4 {
+            int4 m = make_int4(-1, 0, -1, 0);
+            if (j >= my_tiles) return m;
+            const int pos = s_lo + kTileRows * (grp + 2 * j) + (gt >> 3);
+            if (kAll) {
+                if (pos < s_hi) m.x = pos < N ? (int)(row0 + pos) : (int)(kSrcSuffix | (uint32_t)(b * p.suffix_cap + pos - N));
+                if (pos + 16 < s_hi)
+                    m.z = pos + 16 < N ? (int)(row0 + pos + 16) : (int)(kSrcSuffix | (uint32_t)(b * p.suffix_cap + pos + 16 - N));
+                return m;
+            }
+            if (pos < s_hi) { const int2 v = __ldcg(line + pos); m.x = v.x; m.y = v.y; }
+            if (pos + 16 < s_hi) { const int2 v = __ldcg(line + pos + 16); m.z = v.x; m.w = v.y; }
+            return m;
         };
-        // four threads copy a row (18 pieces each); rows past the share's end are zero-filled
-        auto issue = [&](int j, int2 meta) {
+        // eight threads copy a row, 128 bytes per instruction (one line of shared memory: the swizzle only
+        // permutes pieces inside it), nine instructions per row; rows past the share's end are zero-filled
+        auto issue = [&](int j, int4 meta) {
             if (j < my_tiles) {
-                const int i = gt >> 2, qd = gt & 3, stage = j & 1;
-                const bool valid = meta.x != -1;
-                const uint32_t src = (uint32_t)meta.x;
-                const uint4 *g = !valid ? rows_g
-                                        : ((src & kSrcSuffix) ? suffix_g + (size_t)(src & 0x7FFFFFFFu) * kRowChunks
-                                                              : rows_g + (size_t)src * kRowChunks);
-                const uint32_t dst = tiles_addr + stage * kTileBytes + i * kRowBytes;
-                const int bytes = valid ? 16 : 0;
+                const int jl = gt & 7, stage = j & 1;
 #pragma unroll
-                for (int c = 0; c < kRowChunks / 4; ++c) {
-                    const int chunk = 4 * c + qd;
-                    cp_async16(dst + ((chunk ^ (i & 7)) << 4), g + chunk, bytes);
-                }
-                if (!kAll) {
-                    const uint32_t bdst = smem_base + kOffBias + ((grp * 2 + stage) * kTileRows * kBiasPitch + i * kBiasPitch + 4 * qd) * 4;
-                    cp_async16(bdst, valid ? bias_g + (size_t)meta.y * kHeads + 4 * qd : reinterpret_cast<const float *>(rows_g), bytes);
+                for (int half = 0; half < 2; ++half) {
+                    const int i = (gt >> 3) + 16 * half;
+                    const int msrc = half ? meta.z : meta.x, mseg = half ? meta.w : meta.y;
+                    const bool valid = msrc != -1;
+                    const uint32_t src = (uint32_t)msrc;
+                    const uint4 *g = !valid ? rows_g
+                                            : ((src & kSrcSuffix) ? suffix_g + (size_t)(src & 0x7FFFFFFFu) * kRowChunks
+                                                                  : rows_g + (size_t)src * kRowChunks);
+                    const uint32_t dst = tiles_addr + stage * kTileBytes + i * kRowBytes + ((jl ^ (i & 7)) << 4);
+                    const int bytes = valid ? 16 : 0;
+#pragma unroll
+                    for (int c = 0; c < kRowChunks / 8; ++c) cp_async16(dst + c * 128, g + 8 * c + jl, bytes);
+                    if (!kAll && jl < 4) {
+                        const uint32_t bdst = smem_base + kOffBias + ((grp * 2 + stage) * kTileRows * kBiasPitch + i * kBiasPitch + 4 * jl) * 4;
+                        cp_async16(bdst, valid ? bias_g + (size_t)mseg * kHeads + 4 * jl : reinterpret_cast<const float *>(rows_g), bytes);
+                    }
                 }
             }
             asm volatile("cp.async.commit_group;" ::: "memory");
@@ -660,10 +673,10 @@ latent_attend_kernel(LatentAttendParams p)
             issue(0, load_meta(0));
             issue(1, load_meta(1));
         }
-        int2 meta_next = load_meta(2);
+        int4 meta_next = load_meta(2);
 #pragma unroll 1
         for (int j = 0; j < my_tiles; ++j) {
-            const int2 meta_cur = meta_next;                // of the tile issued at the end of this round
+            const int4 meta_cur = meta_next;                // of the tile issued at the end of this round
             meta_next = load_meta(j + 3);
             asm volatile("cp.async.wait_group 1;" ::: "memory");
             group_barrier(grp);                             // tile j is in shared memory for every warp of the group
@@ -735,8 +748,10 @@ latent_attend_kernel(LatentAttendParams p)
             }
             l0 = l0 * a0 + ps0;
             l1 = l1 * a1 + ps1;
+            if (__any_sync(0xFFFFFFFFu, a0 != 1.f || a1 != 1.f)) {       // most tiles leave the maxima where they were
 #pragma unroll
-            for (int j2 = 0; j2 < 16; ++j2) { o[j2][0] *= a0; o[j2][1] *= a0; o[j2][2] *= a1; o[j2][3] *= a1; }
+                for (int j2 = 0; j2 < 16; ++j2) { o[j2][0] *= a0; o[j2][1] *= a0; o[j2][2] *= a1; o[j2][3] *= a1; }
+            }
             uint32_t ph[2][4], pl[2][4];
 #pragma unroll
             for (int ks2 = 0; ks2 < 2; ++ks2) {
@@ -1212,7 +1227,7 @@ int santapp_latent_decode_attn(const santapp_latent_geom *geom, const santapp_la
         in.dbg_sel_logc = dbg ? dbg->sel_logc : nullptr;
         in.dbg_tau = dbg ? dbg->tau : nullptr;
         in.dbg_union_rows = nullptr;
-        in.trace = nullptr;
+        in.trace = dbg ? reinterpret_cast<unsigned long long *>(dbg->trace) : nullptr;
         const int n_heads = geom->n_seqs * geom->n_heads;
         if (n_heads <= L.grid) err = launch_kernel(latent_select_kernel<512>, dim3(n_heads), dim3(512), 0, s, in);
         else                   err = launch_kernel(latent_select_kernel<256>, dim3(n_heads), dim3(256), 0, s, in);

@@ -1,14 +1,14 @@
 // Attention over shared-latent rows on the 5th-generation tensor cores (tcgen05, accumulators in
 // tensor memory). Included by latent.cu, which defines the parameter struct and the constants.
 //
-// One block per SM, nine warps with fixed roles:
+// One block per SM, thirteen warps with fixed roles:
 //   warps 0-3   softmax: read S^T (rows x heads) from tensor memory, keep the running reference
 //               maximum and the row sums, write P^T (two bf16 terms) to shared memory, rescale
 //               O^T when the maximum has grown by more than 2^8, write the block's partial result
 //   warp 4      one lane issues every tcgen05.mma: S^T = Rows Q^T (M = 64 rows, N = 16 heads,
 //               36 steps of K = 16), then O^T += V^T P^T (M = 128 value columns x 4, N = 16 heads,
 //               K = 64 rows, for both terms of P)
-//   warps 5-6 / 7-8   copy the even / odd 64-row tiles from global to shared memory (cp.async,
+//   warps 5-8 / 9-12  copy the even / odd 64-row tiles from global to shared memory (cp.async,
 //               16-byte pieces laid out as the MMA's canonical no-swizzle layout, see below)
 // The roles meet on mbarriers; every wait is bounded, and a wait that expires raises bit 2 of the
 // status word, after which all waits return at once (the control flow never depends on data, so the
@@ -28,7 +28,7 @@
 
 namespace {
 
-constexpr int kTcThreads = 288;
+constexpr int kTcThreads = 416;
 constexpr int kTcRows = 64;                                          // rows per tile = M of the S^T MMA
 constexpr int kTcColBytes = (kTcRows / 8) * 1024;                    // 8192: one block of 64 values of all 64 rows
 constexpr int kTcStageBytes = (kRowDim / 64) * kTcColBytes;          // 73728
@@ -41,7 +41,7 @@ constexpr int kTcOffRed = kTcOffPrefix + (kMaxLatentSeqs + 4) * 4;   // [2][4 wa
 constexpr int kTcOffBar = kTcOffRed + (2 * 4 * 16 + 4 * 16) * 4;     // 10 mbarriers
 constexpr int kTcOffMisc = kTcOffBar + 10 * 8;                       // tensor-memory base, abort flag, scan scratch
 constexpr int kTcSmemBytes = kTcOffMisc + 8 + 48 * 4;
-constexpr uint32_t kTcColumns = 256;                                 // tensor-memory columns: S^T 2 x (4 partial sums x 16), O^T 4 x 16 from column 128
+constexpr uint32_t kTcColumns = 256;                                 // tensor-memory columns: S^T at columns 0 and 64, O^T 4 x 16 from column 128
 constexpr uint32_t kTcColO = 128;
 constexpr int kTcWaitLimit = 1 << 22;
 
@@ -151,7 +151,7 @@ latent_attend_tc_kernel(LatentAttendParams p, int32_t *status)
     // ---- set-up: barriers, tensor memory, the sequences' row prefix ----
     if (tid == 0) {
         *abort_flag = 0;
-        const uint32_t counts[10] = {64, 64, 1, 1, 1, 1, 128, 128, 128, 128};
+        const uint32_t counts[10] = {128, 128, 1, 1, 1, 1, 128, 128, 128, 128};
         for (int i = 0; i < 10; ++i) asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar0 + 8 * i), "r"(counts[i]));
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -225,8 +225,8 @@ latent_attend_tc_kernel(LatentAttendParams p, int32_t *status)
         tc_fence_after();
 
         if (warp >= 5) {
-            // ================= copies: warps 5-6 take even tiles, 7-8 odd tiles =================
-            const int par = (warp - 5) >> 1, pw = (warp - 5) & 1, pt = pw * 32 + lane;      // pt: 0..63 inside the pair of warps
+            // ================= copies: warps 5-8 take even tiles, 9-12 odd tiles =================
+            const int par = (warp - 5) >> 2, pw = (warp - 5) & 3, pt = pw * 32 + lane;      // pt: 0..127 inside the four warps
             const int jl = lane & 7, rl = lane >> 3;        // a warp instruction copies 128 bytes of each of four rows
             const int2 *line = kAll ? nullptr : p.row_meta + row0 + (int64_t)b * p.suffix_cap;
             const float *bias_g = kAll ? nullptr : p.seg_bias + (size_t)b * p.seg_cap * kHeads;
@@ -234,40 +234,40 @@ latent_attend_tc_kernel(LatentAttendParams p, int32_t *status)
                 const uint32_t g = gt0 + i;
                 if ((int)(g & 1u) != par) continue;
                 const int pos0 = s_lo + kTcRows * i;
-                // source rows of this thread: rows 32 pw + 4 u + rl, u < 8, and row pt for the bias copy
-                int src[8], seg_pt = 0;
+                // source rows of this thread: rows 16 pw + 4 u + rl, u < 4, and row pt / 2 for the bias copy
+                int src[4], seg_pt = 0;
 #pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    const int pos = pos0 + 32 * pw + 4 * u + rl;
+                for (int u = 0; u < 4; ++u) {
+                    const int pos = pos0 + 16 * pw + 4 * u + rl;
                     if (pos >= s_hi) src[u] = -1;
                     else if (kAll) src[u] = pos < N ? (int)(row0 + pos) : (int)(kSrcSuffix | (uint32_t)(b * p.suffix_cap + pos - N));
                     else src[u] = __ldcg(line + pos).x;
                 }
-                const bool ok_pt = pos0 + pt < s_hi;
-                if (!kAll && ok_pt) seg_pt = __ldcg(line + pos0 + pt).y;
+                const bool ok_pt = pos0 + (pt >> 1) < s_hi;
+                if (!kAll && ok_pt) seg_pt = __ldcg(line + pos0 + (pt >> 1)).y;
                 const bool tr = gt0 == 0 && i == 2 && pt == 0;
                 tc_mark(p.trace, tr, 0);
                 if (g >= 2) mbar_wait(bar0 + 8 * (kBarPvDone + par), (g >> 1) - 1, abort_flag, status);     // the stage is free
                 tc_mark(p.trace, tr, 1);
                 const uint32_t stage = smem_base + par * kTcStageBytes;
 #pragma unroll
-                for (int u = 0; u < 8; ++u) {
+                for (int u = 0; u < 4; ++u) {
                     const bool valid = src[u] != -1;
                     const uint32_t s = (uint32_t)src[u];
                     const uint4 *gp = !valid ? rows_g
                                              : ((s & kSrcSuffix) ? suffix_g + (size_t)(s & 0x7FFFFFFFu) * kRowChunks
                                                                  : rows_g + (size_t)s * kRowChunks);
-                    const int r = 32 * pw + 4 * u + rl;
+                    const int r = 16 * pw + 4 * u + rl;
                     const uint32_t dst = stage + (r >> 3) * 1024 + (r & 7) * 128 + ((jl ^ (r & 7)) << 4);
                     const int bytes = valid ? 16 : 0;
 #pragma unroll
                     for (int ac = 0; ac < kRowDim / 64; ++ac) cp_async16(dst + ac * kTcColBytes, gp + 8 * ac + jl, bytes);
                 }
-                if (!kAll) {
-                    const uint32_t bdst = smem_base + kTcOffBias + (par * kTcRows + pt) * kBiasPitch * 4;
-                    const float *bsrc = ok_pt ? bias_g + (size_t)seg_pt * kHeads : reinterpret_cast<const float *>(rows_g);
+                if (!kAll) {                                // two threads copy a row's 16 corrections
+                    const uint32_t bdst = smem_base + kTcOffBias + ((par * kTcRows + (pt >> 1)) * kBiasPitch + 8 * (pt & 1)) * 4;
+                    const float *bsrc = ok_pt ? bias_g + (size_t)seg_pt * kHeads + 8 * (pt & 1) : reinterpret_cast<const float *>(rows_g);
 #pragma unroll
-                    for (int u = 0; u < 4; ++u) cp_async16(bdst + 16 * u, bsrc + 4 * u, ok_pt ? 16 : 0);
+                    for (int u = 0; u < 2; ++u) cp_async16(bdst + 16 * u, bsrc + 4 * u, ok_pt ? 16 : 0);
                 }
                 asm volatile("cp.async.commit_group;" ::: "memory");
                 tc_mark(p.trace, tr, 2);
@@ -294,13 +294,10 @@ latent_attend_tc_kernel(LatentAttendParams p, int32_t *status)
                             // thread issues everything, so the instructions between two MMAs are what this costs)
                             const uint64_t da = tc_desc_sw128(smem_base + bpar * kTcStageBytes, 16, 1024);
                             const uint64_t dq = tc_desc_sw128(smem_base + kTcOffQ, 16, 1024);
-                            // consecutive instructions add into different accumulators (four partial sums of S^T,
-                            // added up by the softmax warps): an instruction into the same accumulator as the one
-                            // before it has to wait for that one's result
 #pragma unroll
                             for (int ks = 0; ks < kRowDim / 16; ++ks)
-                                tc_mma(tmem + 64 * bpar + 16 * (ks & 3), da + (uint64_t)(((ks >> 2) * kTcColBytes + (ks & 3) * 32) >> 4),
-                                       dq + (uint64_t)(((ks >> 2) * kTcQColBytes + (ks & 3) * 32) >> 4), idesc_s, ks > 3 ? 1u : 0u);
+                                tc_mma(tmem + 64 * bpar, da + (uint64_t)(((ks >> 2) * kTcColBytes + (ks & 3) * 32) >> 4),
+                                       dq + (uint64_t)(((ks >> 2) * kTcQColBytes + (ks & 3) * 32) >> 4), idesc_s, ks > 0 ? 1u : 0u);
                             tc_commit(bar0 + 8 * (kBarSReady + bpar));
                             tc_mark(p.trace, gt0 == 0 && s_next == 2, 4);
                             ++s_next;
@@ -355,13 +352,6 @@ latent_attend_tc_kernel(LatentAttendParams p, int32_t *status)
                 tc_fence_after();
                 uint32_t sv[16];
                 tc_ld16(lane_addr + 64 * bpar, sv);
-#pragma unroll
-                for (int part = 1; part < 4; ++part) {
-                    uint32_t sw[16];
-                    tc_ld16(lane_addr + 64 * bpar + 16 * part, sw);
-#pragma unroll
-                    for (int h = 0; h < kHeads; ++h) sv[h] = __float_as_uint(__uint_as_float(sv[h]) + __uint_as_float(sw[h]));
-                }
                 tc_fence_before();
                 mbar_arrive(bar0 + 8 * (kBarSFree + bpar));
                 float x[kHeads], mx[kHeads];
