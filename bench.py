@@ -14,7 +14,9 @@ in HBM, replayed from CUDA graphs; `e2e` is the same through host buffers (pinne
 device copies of the step's queries, new suffix rows and counters, device to host read of the
 outputs, inside the timed region). With the default workload the line also carries `batched`:
 the same measurement on the ragged 32-sequence batch (two layers, a few steps), the size at which
-the operator is bandwidth-bound rather than latency-bound (`--no-batched` skips it).
+the operator is bandwidth-bound rather than latency-bound (`--no-batched` skips it), `mid_batch` and
+`long_context` (configs 3 and 5), `shared_latent` (rows of 512 + 64 values shared by 16 heads, 32
+sequences of 8K, `--workload latent_8k` on its own) and `kmeans_parents`.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--layers L]
 """
@@ -269,9 +271,13 @@ def run_ours(args):
         # shared-latent rows (one 576-value row per token, 16 heads) at the paper's 8K study point, 32 sequences
         gc.collect()
         torch.cuda.empty_cache()
-        lat = measure_latent(args, 4, 10, 3, dev)
-        if rank == 0:
-            line["shared_latent"] = lat
+        # (budgets of the paper's study: S = 512 rows per head is K = 128 teams, S = 128 is K = 32)
+        for key, k_lat in (("shared_latent", 128), ("shared_latent_k32", 32)):
+            gc.collect()
+            torch.cuda.empty_cache()
+            lat = measure_latent(args, 2, 10, 3, dev, n_sample=k_lat)
+            if rank == 0:
+                line[key] = lat
         # and the headline workload with the parents of the paper's headline runs: Algorithm 3
         # (minibatch k-means with the paper's settings, fitted by the library), four layers
         if args.parents == "contiguous" and args.elem == "bf16":

@@ -192,3 +192,27 @@ def test_kmeans_fit_refuses_a_sample_that_does_not_fit_in_shared_memory(lib):
     assert lib.santapp_kmeans_fit_workspace_bytes(ctypes.byref(g), n, fits, ctypes.byref(ok)) > 0
     assert lib.santapp_kmeans_fit(ctypes.byref(g), n, too_many, 0x10000, ctypes.byref(ok), 0x10000, None, 0x10000,
                                   1 << 40, None) == sp.SANTAPP_ERR_UNSUPPORTED
+
+
+def test_latent_sizes_follow_algorithms_4_and_2(lib):
+    g = sp.LatentGeometry(3, 16, 16, 4)
+    s = sp.santapp_latent_sizes(g, [8192, 100, 5])
+    assert s.rows_total == 8192 + 100 + 5
+    assert s.teams_total == 512 * 4 + (6 * 4 + 4) + 4          # a tail of 4 rows gives 4 teams, of 5 rows min(R, 5)
+    assert s.max_teams_per_seq == 2048 and s.max_rows_per_seq == 8192
+    assert s.team_row_start_elems == s.teams_total + 3
+    assert s.build_workspace_bytes >= s.rows_total
+
+
+@pytest.mark.parametrize("geom,lens,status", [
+    (sp.LatentGeometry(0, 16, 16, 4), [], sp.SANTAPP_ERR_INVALID_ARG),
+    (sp.LatentGeometry(1, 0, 16, 4), [8], sp.SANTAPP_ERR_INVALID_ARG),
+    (sp.LatentGeometry(1, 16, 16, 5), [8], sp.SANTAPP_ERR_INVALID_ARG),          # R must divide P
+    (sp.LatentGeometry(1, 17, 16, 4), [8], sp.SANTAPP_ERR_UNSUPPORTED),          # more than 16 heads per row
+    (sp.LatentGeometry(1, 16, 64, 4), [8], sp.SANTAPP_ERR_UNSUPPORTED),          # parents above 32 rows
+    (sp.LatentGeometry(1, 16, 16, 4), [0], sp.SANTAPP_ERR_INVALID_ARG),
+])
+def test_bad_latent_geometry_is_rejected_on_the_host(lib, geom, lens, status):
+    with pytest.raises(sp.SantappError) as e:
+        sp.santapp_latent_sizes(geom, lens)
+    assert e.value.status == status

@@ -88,3 +88,21 @@ def test_spec_element_type_reaches_every_tensor():
         assert np.max(np.abs(xa - xb)) < 0.05                                   # same draws, other rounding
     qa, qb = synth.make_queries(a, da, 0), synth.make_queries(b, db, 0)
     assert qa.shape == qb.shape and not np.array_equal(qa, qb)
+
+
+def test_shared_latent_inputs_are_seeded_and_shaped():
+    spec = synth.LatentSpec("t", [100, 37], suffix_cap=5, suffix_len0=[0, 4])
+    a, b = synth.make_latent_layer(spec), synth.make_latent_layer(spec)
+    assert a.rows.shape == (137, synth.LATENT_ROW) and a.rows.dtype == np.uint16
+    assert a.suffix.shape == (2, 5, synth.LATENT_ROW)
+    assert np.array_equal(a.rows, b.rows) and np.array_equal(a.suffix, b.suffix)
+    assert not np.array_equal(a.rows, synth.make_latent_layer(spec, layer=1).rows)
+    q0, q1 = synth.make_latent_queries(spec, a, 0), synth.make_latent_queries(spec, a, 1)
+    assert q0.shape == (2, 16, synth.LATENT_ROW) and not np.array_equal(q0, q1)
+    assert np.array_equal(q0, synth.make_latent_queries(spec, b, 0))
+    assert list(spec.suffix_len(3)) == [3, 5]
+    # the scale is handed to the C ABI as a float: it must survive that conversion unchanged
+    assert float(np.float32(synth.LATENT_SCALE)) == synth.LATENT_SCALE
+    # sinks: the first four rows are four times larger
+    x = synth.to_f32(a.rows)
+    assert np.abs(x[:4]).mean() > 3.0 * np.abs(x[4:100]).mean()
