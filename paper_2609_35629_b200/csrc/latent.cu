@@ -10,9 +10,10 @@
 //   latent_select_kernel   Algorithm 1's sample per (sequence, head): select_head over 576 values
 //   latent_plan_kernel     union of the heads' samples per sequence, written row by row: source
 //                          row and segment of every row to read, per-segment log c (or -inf) per head
-//   latent_attend_kernel   one block per SM, two groups of four warps on alternating 32-row tiles;
-//                          S = Q K^T with the contraction split over the group's warps, P V with
-//                          the 512 value columns split over them; one partial per (block, sequence)
+//   latent_attend_kernel   one block per SM, 32-row tiles: four warps compute S = Q K^T (contraction
+//                          split between them), softmax and P, four copy the rows and accumulate
+//                          O += P V (value columns split between them); one partial per (block, sequence)
+//                          (latent_tc.cuh: the same operator on tcgen05, chosen by the environment)
 //   latent_merge_kernel    log-sum-exp merge of the partials
 #include <cuda_bf16.h>
 #include <limits.h>
@@ -497,15 +498,9 @@ struct LatentAttendParams {
     unsigned long long *trace;      // nullable: device-timer marks of the third tile of a block's first share (diagnostic)
 };
 
-constexpr int kLaThreads = 256;
 constexpr int kTileRows = 32;
 constexpr int kTileBytes = kTileRows * kRowBytes;                   // 36864
 constexpr int kBiasPitch = 20;                                      // floats per tile row (16 heads + pad: conflict-free reads)
-constexpr int kOffBias = 2 * 2 * kTileBytes;                        // two groups x two stages of rows
-constexpr int kOffXch = kOffBias + 2 * 2 * kTileRows * kBiasPitch * 4;
-constexpr int kOffPrefix = kOffXch + 2 * 4 * 4 * 32 * 16;           // per group: 4 warps x 4 float4 x 32 lanes
-constexpr int kOffScan = kOffPrefix + (kMaxLatentSeqs + 4) * 4;
-constexpr int kLaSmemBytes = kOffScan + 48 * 4;
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, int bytes)
 {
@@ -519,10 +514,6 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t &r0, uint32_t &r1, ui
 {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
 }
-__device__ __forceinline__ void group_barrier(int grp)
-{
-    asm volatile("bar.sync %0, 128;" ::"r"(grp + 1) : "memory");
-}
 __device__ __forceinline__ float ex2(float x)
 {
     float y;
@@ -535,28 +526,57 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
     return *reinterpret_cast<const uint32_t *>(&v);
 }
 
-// One block per SM. The rows to read of all sequences form one line, cut into equal ranges, one
-// per block; a block walks the sequences its range touches. Inside a sequence the block's two
-// groups of four warps take alternate tiles of 32 rows, each group with its own two-stage ring of
-// asynchronous copies (16-byte pieces, XOR-swizzled by the row so that ldmatrix is conflict-free)
-// and its own running softmax; the groups' states are merged when the sequence's share is done.
-// Per tile and group: every warp multiplies the 16 heads' queries (A fragments, kept in registers
-// for the warp's 144 of the 576 values) by all 32 rows, the four partial S tiles are summed
-// through shared memory, every warp forms the same P, and multiplies it with its 128 of the 512
-// value columns (P split into two bf16 terms, so the weights keep 16 bits).
+// One block per SM. The rows to read of all sequences form one line, cut into equal ranges, one per
+// block; a block walks the sequences its range touches, 32 rows (a tile) at a time, and leaves one
+// partial result per sequence. Eight warps in two roles. Four compute S = Q Rows^T of a tile with
+// the contraction split between them (each keeps its 144 of the 576 query values as A fragments in
+// registers), add the four partial S tiles up through shared memory, take a quarter of the tile's
+// rows each through the softmax step (tile maxima exchanged through shared memory) and hand P (two
+// bf16 terms, already laid out as the A fragments of the next product) and the factors by which the
+// running maxima moved over through shared memory. The other four copy the rows from global memory
+// into a ring of four tiles (eight lanes copy 128 contiguous bytes of a row into one XOR-swizzled
+// line, so ldmatrix is conflict-free and a global sector lands in one piece) and accumulate
+// O += P V for their 128 of the 512 value columns. S of a tile runs beside P V of the tile before it
+// while two more tiles are on their way from memory; named barriers order the hand-overs.
+constexpr int kLfThreads = 256;
+constexpr int kLfStages = 4;
+constexpr int kLfOffBias = kLfStages * kTileBytes;                              // [stage][32 rows][kBiasPitch] floats
+constexpr int kLfOffXch = kLfOffBias + kLfStages * kTileRows * kBiasPitch * 4;  // [tile parity][4 warps][4][32 lanes] float4
+constexpr int kLfOffP = kLfOffXch + 2 * 4 * 4 * 32 * 16 + 2 * 64 * 4;            // (+ the warps' tile maxima [parity][4][16]); P: [tile parity][16 registers][32 lanes]
+constexpr int kLfOffAlpha = kLfOffP + 2 * 16 * 32 * 4;                          // [tile parity][16 heads]
+constexpr int kLfOffMl = kLfOffAlpha + 2 * 16 * 4;                              // [m 16 | l of each S warp 4 x 16]
+constexpr int kLfOffPrefix = kLfOffMl + 80 * 4;
+constexpr int kLfOffScan = kLfOffPrefix + (kMaxLatentSeqs + 4) * 4;
+constexpr int kLfSmemBytes = kLfOffScan + 48 * 4;
+
+__device__ __forceinline__ void named_sync(int id, int count) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory"); }
+__device__ __forceinline__ void named_arrive(int id, int count) { asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(count) : "memory"); }
+// named barriers: rows of a tile are in shared memory (by tile parity), P of a tile is in shared
+// memory (by parity), the S warps among themselves, the P V warps among themselves
+enum { kLfBarData = 1, kLfBarP = 3, kLfBarS = 5, kLfBarV = 6, kLfBarS2 = 7 };
+
+// Diagnostic: the calling thread notes its SM's cycle counter in mark `slot` of its block (kernel 3 of the trace).
+__device__ __forceinline__ void lf_mark(unsigned long long *trace, bool on, int slot)
+{
+    if (trace != nullptr && on && blockIdx.x < (unsigned)kTraceBlocks) {
+        trace[((size_t)3 * kTraceBlocks + blockIdx.x) * kTraceSlots + slot] = (unsigned long long)clock64();   // SM cycles
+    }
+}
+
 template <bool kAll>
-__global__ void __launch_bounds__(kLaThreads, 1)
+__global__ void __launch_bounds__(kLfThreads, 1)
 latent_attend_kernel(LatentAttendParams p)
 {
     extern __shared__ __align__(128) unsigned char smem[];
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, grp = warp >> 2, gw = warp & 3, gt = tid & 127;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int pv_role = warp >> 2, gw = warp & 3, gt = gw * 32 + lane;
     const int r = lane >> 2, t = lane & 3;
-    uint32_t *prefix = reinterpret_cast<uint32_t *>(smem + kOffPrefix);
-    int *scan = reinterpret_cast<int *>(smem + kOffScan);
+    uint32_t *prefix = reinterpret_cast<uint32_t *>(smem + kLfOffPrefix);
+    int *scan = reinterpret_cast<int *>(smem + kLfOffScan);
     const int n = p.lv.n_seqs, H = p.lv.n_heads;
     {
         uint32_t carry = 0;
-        for (int base = 0; base < n; base += kLaThreads) {
+        for (int base = 0; base < n; base += kLfThreads) {
             const int i = base + tid;
             int v = 0;
             if (i < n) {
@@ -576,7 +596,7 @@ latent_attend_kernel(LatentAttendParams p)
         __syncthreads();
     }
     if (blockIdx.x == 0)
-        for (int i = tid; i <= n; i += kLaThreads) p.pair_prefix[i] = prefix[i];
+        for (int i = tid; i <= n; i += kLfThreads) p.pair_prefix[i] = prefix[i];
     const uint32_t total = prefix[n];
     const uint32_t per = (total + gridDim.x - 1) / gridDim.x;
     const uint32_t lo = min(total, blockIdx.x * per), hi = min(total, lo + per);
@@ -591,9 +611,11 @@ latent_attend_kernel(LatentAttendParams p)
         pr = a;
     }
     const uint32_t smem_base = (uint32_t)__cvta_generic_to_shared(smem);
-    const uint32_t tiles_addr = smem_base + grp * 2 * kTileBytes;
-    float *bias_grp = reinterpret_cast<float *>(smem + kOffBias) + grp * 2 * kTileRows * kBiasPitch;
-    float4 *xch = reinterpret_cast<float4 *>(smem + kOffXch) + grp * (4 * 4 * 32);
+    const float *bias_all = reinterpret_cast<const float *>(smem + kLfOffBias);
+    float4 *xch_all = reinterpret_cast<float4 *>(smem + kLfOffXch);
+    uint32_t *p_all = reinterpret_cast<uint32_t *>(smem + kLfOffP);
+    float *alpha_all = reinterpret_cast<float *>(smem + kLfOffAlpha);
+    float *ml = reinterpret_cast<float *>(smem + kLfOffMl);
     const uint4 *rows_g = reinterpret_cast<const uint4 *>(p.rows_packed);
     const uint4 *suffix_g = reinterpret_cast<const uint4 *>(p.suffix_rows);
 
@@ -603,230 +625,264 @@ latent_attend_kernel(LatentAttendParams p)
         const int s_lo = (int)(max(lo, prefix[pr]) - prefix[pr]), s_hi = (int)(min(hi, prefix[pr + 1]) - prefix[pr]);
         const int64_t row0 = p.lv.seq_row_off[b];
         const int N = (int)(p.lv.seq_row_off[b + 1] - row0);
-        const int2 *line = kAll ? nullptr : p.row_meta + row0 + (int64_t)b * p.suffix_cap;
-        const float *bias_g = kAll ? nullptr : p.seg_bias + (size_t)b * p.seg_cap * kHeads;
-
-        // the warp's share of the queries as A fragments: values [144 gw, 144 gw + 144)
-        uint32_t qa[9][4];
-        {
-            const uint32_t *q32 = reinterpret_cast<const uint32_t *>(p.q + (size_t)b * H * kRowDim);
-#pragma unroll
-            for (int ks = 0; ks < 9; ++ks) {
-                const int d0 = 16 * (9 * gw + ks) + 2 * t;
-                qa[ks][0] = r < H ? __ldg(q32 + (r * kRowDim + d0) / 2) : 0u;
-                qa[ks][1] = r + 8 < H ? __ldg(q32 + ((r + 8) * kRowDim + d0) / 2) : 0u;
-                qa[ks][2] = r < H ? __ldg(q32 + (r * kRowDim + d0 + 8) / 2) : 0u;
-                qa[ks][3] = r + 8 < H ? __ldg(q32 + ((r + 8) * kRowDim + d0 + 8) / 2) : 0u;
-            }
-        }
         const int n_tiles = (s_hi - s_lo + kTileRows - 1) / kTileRows;
-        const int my_tiles = (n_tiles - grp + 1) / 2;       // tiles grp, grp + 2, ...
-        float m0 = -CUDART_INF_F, m1 = -CUDART_INF_F, l0 = 0.f, l1 = 0.f;
-        float o[16][4];
-#pragma unroll
-        for (int j2 = 0; j2 < 16; ++j2) o[j2][0] = o[j2][1] = o[j2][2] = o[j2][3] = 0.f;
 
-        // source rows (and segments) of this thread's two rows of the group's j-th tile, rows gt / 8 and
-        // gt / 8 + 16; source -1: no row
-        auto load_meta = [&](int j) -> int4 {
-            int4 m = make_int4(-1, 0, -1, 0);
-            if (j >= my_tiles) return m;
-            const int pos = s_lo + kTileRows * (grp + 2 * j) + (gt >> 3);
-            if (kAll) {
-                if (pos < s_hi) m.x = pos < N ? (int)(row0 + pos) : (int)(kSrcSuffix | (uint32_t)(b * p.suffix_cap + pos - N));
-                if (pos + 16 < s_hi)
-                    m.z = pos + 16 < N ? (int)(row0 + pos + 16) : (int)(kSrcSuffix | (uint32_t)(b * p.suffix_cap + pos + 16 - N));
-                return m;
+        if (!pv_role) {
+            // ================= S, softmax, P =================
+            float m0 = -CUDART_INF_F, m1 = -CUDART_INF_F, l0 = 0.f, l1 = 0.f;       // heads r and r + 8
+            uint32_t qa[9][4];                              // the warp's share of the queries: values [144 gw, 144 gw + 144)
+            {
+                const uint32_t *q32 = reinterpret_cast<const uint32_t *>(p.q + (size_t)b * H * kRowDim);
+#pragma unroll
+                for (int ks = 0; ks < 9; ++ks) {
+                    const int d0 = 16 * (9 * gw + ks) + 2 * t;
+                    qa[ks][0] = r < H ? __ldg(q32 + (r * kRowDim + d0) / 2) : 0u;
+                    qa[ks][1] = r + 8 < H ? __ldg(q32 + ((r + 8) * kRowDim + d0) / 2) : 0u;
+                    qa[ks][2] = r < H ? __ldg(q32 + (r * kRowDim + d0 + 8) / 2) : 0u;
+                    qa[ks][3] = r + 8 < H ? __ldg(q32 + ((r + 8) * kRowDim + d0 + 8) / 2) : 0u;
+                }
             }
-            if (pos < s_hi) { const int2 v = __ldcg(line + pos); m.x = v.x; m.y = v.y; }
-            if (pos + 16 < s_hi) { const int2 v = __ldcg(line + pos + 16); m.z = v.x; m.w = v.y; }
-            return m;
-        };
-        // eight threads copy a row, 128 bytes per instruction (one line of shared memory: the swizzle only
-        // permutes pieces inside it), nine instructions per row; rows past the share's end are zero-filled
-        auto issue = [&](int j, int4 meta) {
-            if (j < my_tiles) {
-                const int jl = gt & 7, stage = j & 1;
+#pragma unroll 1
+            for (int j = 0; j < n_tiles; ++j) {
+                const int par = j & 1, stage = j & (kLfStages - 1);
+                const bool tr = j >= 4 && j <= 5 && gt == 0;
+                lf_mark(p.trace, tr && j == 4, 0);
+                named_sync(kLfBarData + par, 256);          // the tile's rows (and corrections) have landed
+                lf_mark(p.trace, tr && j == 4, 1);
+                const uint32_t tile_addr = smem_base + stage * kTileBytes;
+                const float *bias_s = bias_all + stage * kTileRows * kBiasPitch;
+                const int nv = min(kTileRows, s_hi - (s_lo + kTileRows * j));
+                float x[4][4];
 #pragma unroll
-                for (int half = 0; half < 2; ++half) {
-                    const int i = (gt >> 3) + 16 * half;
-                    const int msrc = half ? meta.z : meta.x, mseg = half ? meta.w : meta.y;
-                    const bool valid = msrc != -1;
-                    const uint32_t src = (uint32_t)msrc;
-                    const uint4 *g = !valid ? rows_g
-                                            : ((src & kSrcSuffix) ? suffix_g + (size_t)(src & 0x7FFFFFFFu) * kRowChunks
-                                                                  : rows_g + (size_t)src * kRowChunks);
-                    const uint32_t dst = tiles_addr + stage * kTileBytes + i * kRowBytes + ((jl ^ (i & 7)) << 4);
-                    const int bytes = valid ? 16 : 0;
+                for (int nt = 0; nt < 4; ++nt) x[nt][0] = x[nt][1] = x[nt][2] = x[nt][3] = 0.f;
+                {
+                    // all of the warp's key fragments first (the loads pipeline; an MMA right behind its own
+                    // load would wait out the load's latency every time), then the 36 MMAs
+                    uint32_t kb[9][2][4];
 #pragma unroll
-                    for (int c = 0; c < kRowChunks / 8; ++c) cp_async16(dst + c * 128, g + 8 * c + jl, bytes);
-                    if (!kAll && jl < 4) {
-                        const uint32_t bdst = smem_base + kOffBias + ((grp * 2 + stage) * kTileRows * kBiasPitch + i * kBiasPitch + 4 * jl) * 4;
-                        cp_async16(bdst, valid ? bias_g + (size_t)mseg * kHeads + 4 * jl : reinterpret_cast<const float *>(rows_g), bytes);
+                    for (int ks = 0; ks < 9; ++ks) {
+#pragma unroll
+                        for (int ntp = 0; ntp < 2; ++ntp) {
+                            const int row = 16 * ntp + ((lane >> 4) << 3) + (lane & 7);
+                            const int chunk = 18 * gw + 2 * ks + ((lane >> 3) & 1);
+                            ldmatrix_x4(kb[ks][ntp][0], kb[ks][ntp][1], kb[ks][ntp][2], kb[ks][ntp][3],
+                                        tile_addr + row * kRowBytes + ((chunk ^ (lane & 7)) << 4));
+                        }
+                    }
+#pragma unroll
+                    for (int ks = 0; ks < 9; ++ks) {
+#pragma unroll
+                        for (int ntp = 0; ntp < 2; ++ntp) {
+                            mma_bf16(x[2 * ntp], qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3], kb[ks][ntp][0], kb[ks][ntp][1]);
+                            mma_bf16(x[2 * ntp + 1], qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3], kb[ks][ntp][2], kb[ks][ntp][3]);
+                        }
                     }
                 }
+                float4 *xch = xch_all + par * (4 * 4 * 32);
+                lf_mark(p.trace, tr && j == 4, 2);
+#pragma unroll
+                for (int nt = 0; nt < 4; ++nt) xch[(gw * 4 + nt) * 32 + lane] = make_float4(x[nt][0], x[nt][1], x[nt][2], x[nt][3]);
+                named_sync(kLfBarS, 128);
+                lf_mark(p.trace, tr && j == 4, 3);
+                // from here on the warp owns rows 8 gw .. 8 gw + 7 of the tile: its four values per lane are
+                // heads r (y0, y1) and r + 8 (y2, y3) for rows 8 gw + 2 t and + 1
+                float y0, y1, y2, y3;
+                {
+                    float4 sacc = xch[gw * 32 + lane];
+#pragma unroll
+                    for (int w = 1; w < 4; ++w) {
+                        const float4 v = xch[(w * 4 + gw) * 32 + lane];
+                        sacc.x += v.x; sacc.y += v.y; sacc.z += v.z; sacc.w += v.w;
+                    }
+                    const int row = 8 * gw + 2 * t;
+                    const float b00 = kAll ? 0.f : bias_s[row * kBiasPitch + r], b01 = kAll ? 0.f : bias_s[(row + 1) * kBiasPitch + r];
+                    const float b10 = kAll ? 0.f : bias_s[row * kBiasPitch + r + 8], b11 = kAll ? 0.f : bias_s[(row + 1) * kBiasPitch + r + 8];
+                    y0 = row < nv ? fmaf(sacc.x, p.qk_scale_log2, b00) : -CUDART_INF_F;
+                    y1 = row + 1 < nv ? fmaf(sacc.y, p.qk_scale_log2, b01) : -CUDART_INF_F;
+                    y2 = row < nv ? fmaf(sacc.z, p.qk_scale_log2, b10) : -CUDART_INF_F;
+                    y3 = row + 1 < nv ? fmaf(sacc.w, p.qk_scale_log2, b11) : -CUDART_INF_F;
+                }
+                float mx0 = fmaxf(y0, y1), mx1 = fmaxf(y2, y3);
+                mx0 = fmaxf(mx0, __shfl_xor_sync(0xFFFFFFFFu, mx0, 1));
+                mx0 = fmaxf(mx0, __shfl_xor_sync(0xFFFFFFFFu, mx0, 2));
+                mx1 = fmaxf(mx1, __shfl_xor_sync(0xFFFFFFFFu, mx1, 1));
+                mx1 = fmaxf(mx1, __shfl_xor_sync(0xFFFFFFFFu, mx1, 2));
+                float *mxw = reinterpret_cast<float *>(xch_all) + 2 * (4 * 4 * 32) * 4 + par * 64;   // [parity][4 warps][16 heads]
+                if (t == 0) {
+                    mxw[gw * 16 + r] = mx0;
+                    mxw[gw * 16 + r + 8] = mx1;
+                }
+                named_sync(kLfBarS2, 128);
+                mx0 = fmaxf(fmaxf(mxw[r], mxw[16 + r]), fmaxf(mxw[32 + r], mxw[48 + r]));
+                mx1 = fmaxf(fmaxf(mxw[r + 8], mxw[16 + r + 8]), fmaxf(mxw[32 + r + 8], mxw[48 + r + 8]));
+                const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);
+                const float mu0 = mn0 == -CUDART_INF_F ? 0.f : mn0, mu1 = mn1 == -CUDART_INF_F ? 0.f : mn1;
+                const float a0 = ex2(m0 - mu0), a1 = ex2(m1 - mu1);
+                m0 = mn0;
+                m1 = mn1;
+                y0 = ex2(y0 - mu0);
+                y1 = ex2(y1 - mu0);
+                y2 = ex2(y2 - mu1);
+                y3 = ex2(y3 - mu1);
+                l0 = l0 * a0 + y0 + y1;                     // the warp's rows only: the four warps' sums are added at the end
+                l1 = l1 * a1 + y2 + y3;
+                {
+                    // P as the A fragments of P V: n-tile gw is registers (gw / 2) * 4 + (gw % 2) * 2 and + 1 of a lane
+                    uint32_t *pb = p_all + par * (16 * 32);
+                    const int reg = (gw >> 1) * 4 + (gw & 1) * 2;
+                    const uint32_t h0 = pack_bf16(y0, y1), h1 = pack_bf16(y2, y3);
+                    pb[reg * 32 + lane] = h0;
+                    pb[(reg + 1) * 32 + lane] = h1;
+                    pb[(8 + reg) * 32 + lane] = pack_bf16(y0 - bf16_lo(h0), y1 - bf16_hi(h0));
+                    pb[(8 + reg + 1) * 32 + lane] = pack_bf16(y2 - bf16_lo(h1), y3 - bf16_hi(h1));
+                    if (gw == 0 && t == 0) {
+                        alpha_all[par * 16 + r] = a0;
+                        alpha_all[par * 16 + r + 8] = a1;
+                    }
+                }
+                named_arrive(kLfBarP + par, 256);
+                lf_mark(p.trace, tr && j == 4, 4);
+                lf_mark(p.trace, tr && j == 5, 5);
             }
-            asm volatile("cp.async.commit_group;" ::: "memory");
-        };
-
-        if (my_tiles > 0) {
-            issue(0, load_meta(0));
-            issue(1, load_meta(1));
-        }
-        int4 meta_next = load_meta(2);
+            l0 += __shfl_xor_sync(0xFFFFFFFFu, l0, 1);
+            l0 += __shfl_xor_sync(0xFFFFFFFFu, l0, 2);
+            l1 += __shfl_xor_sync(0xFFFFFFFFu, l1, 1);
+            l1 += __shfl_xor_sync(0xFFFFFFFFu, l1, 2);
+            if (t == 0) {
+                if (gw == 0) { ml[r] = m0; ml[r + 8] = m1; }
+                ml[16 + gw * 16 + r] = l0;                  // [4 warps][16 heads]
+                ml[16 + gw * 16 + r + 8] = l1;
+            }
+            __syncthreads();                                // m and l are in shared memory
+        } else {
+            // ================= copies and O += P V =================
+            float o[16][4];                                 // 16 heads x the warp's 128 value columns
+#pragma unroll
+            for (int j2 = 0; j2 < 16; ++j2) o[j2][0] = o[j2][1] = o[j2][2] = o[j2][3] = 0.f;
+            const int2 *line = kAll ? nullptr : p.row_meta + row0 + (int64_t)b * p.suffix_cap;
+            const float *bias_g = kAll ? nullptr : p.seg_bias + (size_t)b * p.seg_cap * kHeads;
+            // source rows (and segments) of this thread's two rows of tile j, rows gt / 8 and gt / 8 + 16; -1: no row
+            auto load_meta = [&](int j) -> int4 {
+                int4 m = make_int4(-1, 0, -1, 0);
+                if (j >= n_tiles) return m;
+                const int pos = s_lo + kTileRows * j + (gt >> 3);
+                if (kAll) {
+                    if (pos < s_hi) m.x = pos < N ? (int)(row0 + pos) : (int)(kSrcSuffix | (uint32_t)(b * p.suffix_cap + pos - N));
+                    if (pos + 16 < s_hi)
+                        m.z = pos + 16 < N ? (int)(row0 + pos + 16) : (int)(kSrcSuffix | (uint32_t)(b * p.suffix_cap + pos + 16 - N));
+                    return m;
+                }
+                if (pos < s_hi) { const int2 v = __ldcg(line + pos); m.x = v.x; m.y = v.y; }
+                if (pos + 16 < s_hi) { const int2 v = __ldcg(line + pos + 16); m.z = v.x; m.w = v.y; }
+                return m;
+            };
+            // eight threads copy a row, 128 bytes per instruction (one line of shared memory: the swizzle only
+            // permutes pieces inside it); rows past the share's end are zero-filled
+            auto issue = [&](int j, int4 meta) {
+                if (j < n_tiles) {
+                    const int jl = gt & 7, stage = j & (kLfStages - 1);
+#pragma unroll
+                    for (int half = 0; half < 2; ++half) {
+                        const int i = (gt >> 3) + 16 * half;
+                        const int msrc = half ? meta.z : meta.x, mseg = half ? meta.w : meta.y;
+                        const bool valid = msrc != -1;
+                        const uint32_t src = (uint32_t)msrc;
+                        const uint4 *g = !valid ? rows_g
+                                                : ((src & kSrcSuffix) ? suffix_g + (size_t)(src & 0x7FFFFFFFu) * kRowChunks
+                                                                      : rows_g + (size_t)src * kRowChunks);
+                        const uint32_t dst = smem_base + stage * kTileBytes + i * kRowBytes + ((jl ^ (i & 7)) << 4);
+                        const int bytes = valid ? 16 : 0;
+#pragma unroll
+                        for (int c = 0; c < kRowChunks / 8; ++c) cp_async16(dst + c * 128, g + 8 * c + jl, bytes);
+                        if (!kAll && jl < 4) {
+                            const uint32_t bdst = smem_base + kLfOffBias + (stage * kTileRows * kBiasPitch + i * kBiasPitch + 4 * jl) * 4;
+                            cp_async16(bdst, valid ? bias_g + (size_t)mseg * kHeads + 4 * jl : reinterpret_cast<const float *>(rows_g), bytes);
+                        }
+                    }
+                }
+                asm volatile("cp.async.commit_group;" ::: "memory");
+            };
+#pragma unroll
+            for (int j = 0; j < kLfStages; ++j) issue(j, load_meta(j));
+            asm volatile("cp.async.wait_group 3;" ::: "memory");
+            named_arrive(kLfBarData, 256);                  // tile 0 is there
+            int4 meta_next = load_meta(kLfStages);
 #pragma unroll 1
-        for (int j = 0; j < my_tiles; ++j) {
-            const int4 meta_cur = meta_next;                // of the tile issued at the end of this round
-            meta_next = load_meta(j + 3);
-            asm volatile("cp.async.wait_group 1;" ::: "memory");
-            group_barrier(grp);                             // tile j is in shared memory for every warp of the group
-            const uint32_t tile_addr = tiles_addr + (j & 1) * kTileBytes;
-            const float *bias_s = bias_grp + (j & 1) * kTileRows * kBiasPitch;
-            const int nv = min(kTileRows, s_hi - (s_lo + kTileRows * (grp + 2 * j)));
-
-            // ---- partial S (16 heads x 32 rows) over the warp's 144 values ----
-            float x[4][4];
-#pragma unroll
-            for (int nt = 0; nt < 4; ++nt) x[nt][0] = x[nt][1] = x[nt][2] = x[nt][3] = 0.f;
-#pragma unroll
-            for (int ks = 0; ks < 9; ++ks) {
-#pragma unroll
-                for (int ntp = 0; ntp < 2; ++ntp) {
-                    const int row = 16 * ntp + ((lane >> 4) << 3) + (lane & 7);
-                    const int chunk = 18 * gw + 2 * ks + ((lane >> 3) & 1);
-                    uint32_t r0, r1, r2, r3;
-                    ldmatrix_x4(r0, r1, r2, r3, tile_addr + row * kRowBytes + ((chunk ^ (lane & 7)) << 4));
-                    mma_bf16(x[2 * ntp], qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3], r0, r1);
-                    mma_bf16(x[2 * ntp + 1], qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3], r2, r3);
+            for (int j = 0; j < n_tiles; ++j) {
+                const int par = j & 1;
+                const int4 meta_cur = meta_next;            // of the tile issued at the end of this round
+                meta_next = load_meta(j + kLfStages + 1);
+                const bool tr = j == 4 && gt == 0;
+                lf_mark(p.trace, tr, 6);
+                if (j + 1 < n_tiles) {                      // tile j + 1 was requested three rounds ago: tell the S warps
+                    asm volatile("cp.async.wait_group 2;" ::: "memory");
+                    named_arrive(kLfBarData + (par ^ 1), 256);
                 }
-            }
+                lf_mark(p.trace, tr, 7);
+                named_sync(kLfBarP + par, 256);             // P of tile j is there
+                lf_mark(p.trace, tr, 8);
+                uint32_t pf[16];
+                const uint32_t *pb = p_all + par * (16 * 32);
 #pragma unroll
-            for (int nt = 0; nt < 4; ++nt) xch[(gw * 4 + nt) * 32 + lane] = make_float4(x[nt][0], x[nt][1], x[nt][2], x[nt][3]);
-            group_barrier(grp);
+                for (int i = 0; i < 16; ++i) pf[i] = pb[i * 32 + lane];
+                const float a0 = alpha_all[par * 16 + r], a1 = alpha_all[par * 16 + r + 8];
+                if (__any_sync(0xFFFFFFFFu, a0 != 1.f || a1 != 1.f)) {        // most tiles leave the maxima where they were
 #pragma unroll
-            for (int nt = 0; nt < 4; ++nt) {
-                float4 s = xch[nt * 32 + lane];
-#pragma unroll
-                for (int w = 1; w < 4; ++w) {
-                    const float4 v = xch[(w * 4 + nt) * 32 + lane];
-                    s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+                    for (int j2 = 0; j2 < 16; ++j2) { o[j2][0] *= a0; o[j2][1] *= a0; o[j2][2] *= a1; o[j2][3] *= a1; }
                 }
-                x[nt][0] = s.x; x[nt][1] = s.y; x[nt][2] = s.z; x[nt][3] = s.w;
-            }
-
-            // ---- softmax step (log2 domain): heads r (c = 0, 1) and r + 8 (c = 2, 3), rows 8 nt + 2 t + (c & 1) ----
-            float mx0 = -CUDART_INF_F, mx1 = -CUDART_INF_F;
+                const uint32_t tile_addr = smem_base + (j & (kLfStages - 1)) * kTileBytes;
+                {
+                    uint32_t vb[2][8][4];                   // V fragments of the 16 column tiles, both k-steps: all loads first
 #pragma unroll
-            for (int nt = 0; nt < 4; ++nt) {
+                    for (int ks2 = 0; ks2 < 2; ++ks2) {
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    const int row = 8 * nt + 2 * t + (c & 1), head = r + ((c >> 1) << 3);
-                    const float bia = kAll ? 0.f : bias_s[row * kBiasPitch + head];
-                    x[nt][c] = row < nv ? fmaf(x[nt][c], p.qk_scale_log2, bia) : -CUDART_INF_F;
+                        for (int j2 = 0; j2 < 8; ++j2) {
+                            const int mi = lane >> 3;
+                            const int row = 16 * ks2 + ((mi & 1) << 3) + (lane & 7);
+                            const int chunk = 16 * gw + 2 * j2 + (mi >> 1);
+                            ldmatrix_x4_trans(vb[ks2][j2][0], vb[ks2][j2][1], vb[ks2][j2][2], vb[ks2][j2][3],
+                                              tile_addr + row * kRowBytes + ((chunk ^ (lane & 7)) << 4));
+                        }
+                    }
+#pragma unroll
+                    for (int ks2 = 0; ks2 < 2; ++ks2) {
+#pragma unroll
+                        for (int term = 0; term < 2; ++term) {      // 16 independent accumulators per term
+#pragma unroll
+                            for (int j2 = 0; j2 < 8; ++j2) {
+                                mma_bf16(o[2 * j2], pf[8 * term + 4 * ks2], pf[8 * term + 4 * ks2 + 1], pf[8 * term + 4 * ks2 + 2],
+                                         pf[8 * term + 4 * ks2 + 3], vb[ks2][j2][0], vb[ks2][j2][1]);
+                                mma_bf16(o[2 * j2 + 1], pf[8 * term + 4 * ks2], pf[8 * term + 4 * ks2 + 1], pf[8 * term + 4 * ks2 + 2],
+                                         pf[8 * term + 4 * ks2 + 3], vb[ks2][j2][2], vb[ks2][j2][3]);
+                            }
+                        }
+                    }
                 }
-                mx0 = fmaxf(mx0, fmaxf(x[nt][0], x[nt][1]));
-                mx1 = fmaxf(mx1, fmaxf(x[nt][2], x[nt][3]));
+                lf_mark(p.trace, tr, 9);
+                named_sync(kLfBarV, 128);                   // every P V warp is done with this stage
+                lf_mark(p.trace, tr, 10);
+                issue(j + kLfStages, meta_cur);
+                lf_mark(p.trace, tr, 11);
             }
-            mx0 = fmaxf(mx0, __shfl_xor_sync(0xFFFFFFFFu, mx0, 1));
-            mx0 = fmaxf(mx0, __shfl_xor_sync(0xFFFFFFFFu, mx0, 2));
-            mx1 = fmaxf(mx1, __shfl_xor_sync(0xFFFFFFFFu, mx1, 1));
-            mx1 = fmaxf(mx1, __shfl_xor_sync(0xFFFFFFFFu, mx1, 2));
-            const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);
-            const float mu0 = mn0 == -CUDART_INF_F ? 0.f : mn0, mu1 = mn1 == -CUDART_INF_F ? 0.f : mn1;
-            const float a0 = ex2(m0 - mu0), a1 = ex2(m1 - mu1);
-            m0 = mn0;
-            m1 = mn1;
-            float ps0 = 0.f, ps1 = 0.f;
-#pragma unroll
-            for (int nt = 0; nt < 4; ++nt) {
-                x[nt][0] = ex2(x[nt][0] - mu0);
-                x[nt][1] = ex2(x[nt][1] - mu0);
-                x[nt][2] = ex2(x[nt][2] - mu1);
-                x[nt][3] = ex2(x[nt][3] - mu1);
-                ps0 += x[nt][0] + x[nt][1];
-                ps1 += x[nt][2] + x[nt][3];
-            }
-            l0 = l0 * a0 + ps0;
-            l1 = l1 * a1 + ps1;
-            if (__any_sync(0xFFFFFFFFu, a0 != 1.f || a1 != 1.f)) {       // most tiles leave the maxima where they were
-#pragma unroll
-                for (int j2 = 0; j2 < 16; ++j2) { o[j2][0] *= a0; o[j2][1] *= a0; o[j2][2] *= a1; o[j2][3] *= a1; }
-            }
-            uint32_t ph[2][4], pl[2][4];
-#pragma unroll
-            for (int ks2 = 0; ks2 < 2; ++ks2) {
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int nt = 2 * ks2 + (i >> 1), c = (i & 1) * 2;
-                    const float v0 = x[nt][c], v1 = x[nt][c + 1];
-                    const uint32_t hi16 = pack_bf16(v0, v1);
-                    ph[ks2][i] = hi16;
-                    pl[ks2][i] = pack_bf16(v0 - bf16_lo(hi16), v1 - bf16_hi(hi16));
-                }
-            }
-
-            // ---- O (16 heads x the warp's 128 value columns) += P V ----
-#pragma unroll
-            for (int j2 = 0; j2 < 8; ++j2) {
-#pragma unroll
-                for (int ks2 = 0; ks2 < 2; ++ks2) {
-                    const int mi = lane >> 3;
-                    const int row = 16 * ks2 + ((mi & 1) << 3) + (lane & 7);
-                    const int chunk = 16 * gw + 2 * j2 + (mi >> 1);
-                    uint32_t r0, r1, r2, r3;
-                    ldmatrix_x4_trans(r0, r1, r2, r3, tile_addr + row * kRowBytes + ((chunk ^ (lane & 7)) << 4));
-                    mma_bf16(o[2 * j2], ph[ks2][0], ph[ks2][1], ph[ks2][2], ph[ks2][3], r0, r1);
-                    mma_bf16(o[2 * j2 + 1], ph[ks2][0], ph[ks2][1], ph[ks2][2], ph[ks2][3], r2, r3);
-                    mma_bf16(o[2 * j2], pl[ks2][0], pl[ks2][1], pl[ks2][2], pl[ks2][3], r0, r1);
-                    mma_bf16(o[2 * j2 + 1], pl[ks2][0], pl[ks2][1], pl[ks2][2], pl[ks2][3], r2, r3);
-                }
-            }
-            group_barrier(grp);                             // every warp is done with this stage
-            issue(j + 2, meta_cur);
-        }
-        asm volatile("cp.async.wait_group 0;" ::: "memory");
-        l0 += __shfl_xor_sync(0xFFFFFFFFu, l0, 1);
-        l0 += __shfl_xor_sync(0xFFFFFFFFu, l0, 2);
-        l1 += __shfl_xor_sync(0xFFFFFFFFu, l1, 1);
-        l1 += __shfl_xor_sync(0xFFFFFFFFu, l1, 2);
-
-        // ---- the two groups' states into one partial ----
-        __syncthreads();
-        float4 *comb = reinterpret_cast<float4 *>(smem);            // the rings are idle
-        float *comb_ml = reinterpret_cast<float *>(smem + 4 * 16 * 32 * 16);
-        if (grp == 1) {
-#pragma unroll
-            for (int j2 = 0; j2 < 16; ++j2) comb[(gw * 16 + j2) * 32 + lane] = make_float4(o[j2][0], o[j2][1], o[j2][2], o[j2][3]);
-            if (gw == 0 && t == 0) {
-                comb_ml[r] = m0;
-                comb_ml[r + 8] = m1;
-                comb_ml[16 + r] = l0;
-                comb_ml[16 + r + 8] = l1;
-            }
-        }
-        __syncthreads();
-        if (grp == 0) {
-            const float n0 = comb_ml[r], n1 = comb_ml[r + 8], k0 = comb_ml[16 + r], k1 = comb_ml[16 + r + 8];
-            const float M0 = fmaxf(m0, n0), M1 = fmaxf(m1, n1);
-            const float u0 = M0 == -CUDART_INF_F ? 0.f : M0, u1 = M1 == -CUDART_INF_F ? 0.f : M1;
-            const float w0 = ex2(m0 - u0), v0 = ex2(n0 - u0), w1 = ex2(m1 - u1), v1 = ex2(n1 - u1);
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
+            __syncthreads();                                // m and l are in shared memory
+            const float M0 = ml[r], M1 = ml[r + 8];
             float *out0 = p.partials + ((size_t)(blockIdx.x + b) * kHeads + r) * kLatPartialStride;
             float *out1 = out0 + 8 * kLatPartialStride;
             if (gw == 0 && t == 0) {
                 out0[0] = M0;
-                out0[1] = w0 * l0 + v0 * k0;
+                out0[1] = ml[16 + r] + ml[32 + r] + ml[48 + r] + ml[64 + r];
                 out1[0] = M1;
-                out1[1] = w1 * l1 + v1 * k1;
+                out1[1] = ml[16 + r + 8] + ml[32 + r + 8] + ml[48 + r + 8] + ml[64 + r + 8];
             }
 #pragma unroll
             for (int j2 = 0; j2 < 16; ++j2) {
-                const float4 c = comb[(gw * 16 + j2) * 32 + lane];
                 const int col = 4 + 128 * gw + 8 * j2 + 2 * t;
-                *reinterpret_cast<float2 *>(out0 + col) = make_float2(w0 * o[j2][0] + v0 * c.x, w0 * o[j2][1] + v0 * c.y);
-                *reinterpret_cast<float2 *>(out1 + col) = make_float2(w1 * o[j2][2] + v1 * c.z, w1 * o[j2][3] + v1 * c.w);
+                *reinterpret_cast<float2 *>(out0 + col) = make_float2(o[j2][0], o[j2][1]);
+                *reinterpret_cast<float2 *>(out1 + col) = make_float2(o[j2][2], o[j2][3]);
             }
         }
-        __syncthreads();
+        __syncthreads();                                    // the share is done: shared memory may be reused
     }
 }
 
@@ -998,21 +1054,23 @@ int latent_attend_and_merge(const santapp_latent_geom *geom, const santapp_laten
     ap.trace = trace;
     cudaError_t err;
     if (mask & SANTAPP_STAGE_ATTEND) {
-        static std::atomic<unsigned long long> done_all, done_sel, done_tc_all, done_tc_sel;
+        static std::atomic<unsigned long long> done_tc_all, done_tc_sel;
         // The tcgen05 variant (latent_tc.cuh) computes the same thing on the 5th-generation tensor cores; it is
         // slower here (a tcgen05.mma of N = 16 columns costs as much as one of 64, and one thread issues 68 of
-        // them per 64 rows), so the mma.sync kernel is the default and the other is chosen by the environment.
+        // them per 64 rows), so the mma.sync kernel is the default and the other is chosen by the environment
+        // (SANTAPP_LATENT_ATTEND=tcgen05).
         const char *which = getenv("SANTAPP_LATENT_ATTEND");
-        const bool legacy = !(which != nullptr && strcmp(which, "tcgen05") == 0);
-        if (legacy) {
+        const bool tc = which != nullptr && strcmp(which, "tcgen05") == 0;
+        static std::atomic<unsigned long long> done_sp_all, done_sp_sel;
+        if (!tc) {
             if (dense) {
-                if ((err = ensure_dynamic_smem((const void *)latent_attend_kernel<true>, kLaSmemBytes, done_all)) != cudaSuccess)
+                if ((err = ensure_dynamic_smem((const void *)latent_attend_kernel<true>, kLfSmemBytes, done_sp_all)) != cudaSuccess)
                     return note_cuda_failure(err, "latent attend attribute");
-                err = launch_kernel(latent_attend_kernel<true>, dim3(L.grid), dim3(kLaThreads), kLaSmemBytes, s, ap);
+                err = launch_kernel(latent_attend_kernel<true>, dim3(L.grid), dim3(kLfThreads), kLfSmemBytes, s, ap);
             } else {
-                if ((err = ensure_dynamic_smem((const void *)latent_attend_kernel<false>, kLaSmemBytes, done_sel)) != cudaSuccess)
+                if ((err = ensure_dynamic_smem((const void *)latent_attend_kernel<false>, kLfSmemBytes, done_sp_sel)) != cudaSuccess)
                     return note_cuda_failure(err, "latent attend attribute");
-                err = launch_kernel(latent_attend_kernel<false>, dim3(L.grid), dim3(kLaThreads), kLaSmemBytes, s, ap);
+                err = launch_kernel(latent_attend_kernel<false>, dim3(L.grid), dim3(kLfThreads), kLfSmemBytes, s, ap);
             }
         } else if (dense) {
             if ((err = ensure_dynamic_smem((const void *)latent_attend_tc_kernel<true>, kTcSmemBytes, done_tc_all)) != cudaSuccess)
