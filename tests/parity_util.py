@@ -109,3 +109,16 @@ def gpu_step(layer: GpuLayer, q_bits, suffix_len, K, seed, step, stream_base=0, 
 
 def max_abs_v(layer: GpuLayer):
     return float(np.abs(synth.to_f32(layer.data.v_prompt, layer.spec.elem)).max())
+
+
+def assert_same_sample(sel_gpu, logc_gpu, sel_ref, logc_ref, what=""):
+    """Sampled teams of one head: the same set, the same log c per team, and the same order by
+    perturbed score -- except that two neighbours in that order may have changed places (both
+    sides sum the fp64 routing dot product in a different order, so a near-tie between two
+    SELECTED teams may fall either way; the sample, tau and every correction are the same then)."""
+    sel_gpu, sel_ref = np.asarray(sel_gpu), np.asarray(sel_ref)
+    assert sorted(sel_gpu.tolist()) == sorted(sel_ref.tolist()), f"sampled teams differ {what}"
+    pos = {int(g): i for i, g in enumerate(sel_ref)}
+    for i, g in enumerate(sel_gpu):
+        assert abs(pos[int(g)] - i) <= 1, f"order of the sample differs by more than a swap of neighbours {what}"
+        assert abs(float(logc_gpu[i]) - float(logc_ref[pos[int(g)]])) <= 1e-5, f"log c differs {what}"

@@ -9,6 +9,8 @@ from oracle import santapp_oracle as orc
 from paper_2609_35629_b200 import binding as sp
 from paper_2609_35629_b200 import synth
 
+import parity_util as pu
+
 pytestmark = pytest.mark.gpu
 
 SPARSE_TOL = 2e-3       # |out - oracle| <= tol * max |value|, as for the K/V path
@@ -94,9 +96,9 @@ def check_step(layer, step, K=None, seed=1234, suffix_len=None, seqs=None, strea
             assert np.allclose(tau[b], r.tau, rtol=0, atol=1e-9)
         else:
             assert np.all(np.isnan(tau[b]))
-        assert np.array_equal(sel[b, :, :Ke], r.sel[:, :Ke]), f"sampled teams differ (seq {b}, step {step})"
+        for h in range(spec.n_heads):
+            pu.assert_same_sample(sel[b, h, :Ke], logc[b, h, :Ke], r.sel[h, :Ke], r.logc[h, :Ke], f"(seq {b}, head {h}, step {step})")
         assert np.all(sel[b, :, Ke:] == -1)
-        assert np.allclose(logc[b, :, :Ke], r.logc[:, :Ke], rtol=0, atol=1e-5)
         assert union[b, 0] == orc.union_rows(ts, r.sel[:, :Ke])
         vmax = np.abs(rows_b[:, :D]).max()
         err = np.abs(out[b] - r.o).max()

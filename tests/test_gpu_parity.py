@@ -73,9 +73,9 @@ def check_sparse_step(layer, step, K, seed=1234, stream_base=0, suffix_len=None,
             hs = slice(j * G, (j + 1) * G)
             if Ke < M:
                 assert np.all(r.margin[hs] > 1e-9), "seeded workload too close to a selection boundary"
-            assert np.array_equal(sel[b, hs, :Ke], r.sel[hs, :Ke]), f"sampled teams differ (seq {b}, step {step})"
+            for h in range(j * G, (j + 1) * G):
+                pu.assert_same_sample(sel[b, h, :Ke], logc[b, h, :Ke], r.sel[h, :Ke], r.logc[h, :Ke], f"(seq {b}, head {h}, step {step})")
             assert np.all(sel[b, hs, Ke:] == -1)
-            assert np.allclose(logc[b, hs, :Ke], r.logc[hs, :Ke], rtol=0, atol=1e-5)
             if Ke < M:
                 assert np.allclose(tau[b, hs], r.tau[hs], rtol=0, atol=1e-9)
             else:
