@@ -177,6 +177,18 @@ def test_step_fewer_heads_and_odd_sizes():
         check_dense(layer, 2)
 
 
+def test_step_many_short_sequences_blocks_span_several():
+    """200 sequences of 5 to 300 rows: every block's range covers several sequences, most shares are
+    shorter than a tile or than the copy ring, sequences with fewer teams than the budget sit beside
+    sequences that sample."""
+    rng = np.random.default_rng(3)
+    lens = [int(x) for x in rng.integers(5, 300, size=200)]
+    layer = LatentLayer(synth.LatentSpec("short", lens, n_sample=9, suffix_cap=6, suffix_len0=[int(x) for x in rng.integers(0, 7, size=200)],
+                                         suffix_growth=0))
+    check_step(layer, 0)
+    check_dense(layer, 0)
+
+
 def test_step_paper_point_8k_all_budgets():
     """8K context, P = 16, R = 4, 16 heads; the study's budgets S = 128, 256, 512 rows are K = 32, 64, 128 teams."""
     layer = LatentLayer(synth.LatentSpec("8k", [8192, 8192], suffix_cap=16, suffix_len0=[0, 5]))
@@ -212,6 +224,11 @@ def test_tcgen05_variant_of_the_attention_kernel(small, monkeypatch):
         odd = LatentLayer(synth.LatentSpec(f"h{H}", lens, n_heads=H, n_sample=7, suffix_cap=3, suffix_len0=[1] * len(lens)))
         check_step(odd, 2)
         check_dense(odd, 2)
+    rng = np.random.default_rng(4)
+    lens = [int(x) for x in rng.integers(5, 300, size=200)]
+    short = LatentLayer(synth.LatentSpec("short", lens, n_sample=9, suffix_cap=6, suffix_len0=[3] * 200, suffix_growth=0))
+    check_step(short, 0)
+    check_dense(short, 0)
 
 
 def test_same_seed_same_bits_and_step_changes_the_sample(small):
