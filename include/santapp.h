@@ -223,7 +223,9 @@ int32_t santapp_kmeans_parent_count(int32_t prompt_len, int32_t parent_size);
  *   2. Greedy k-means++ on the sample with 2 + floor(ln k) trials per centre: the first centre is
  *      a uniform sample point; each later one is the best of the trial points drawn with
  *      probability proportional to the squared distance to the nearest centre so far, best meaning
- *      the smallest resulting sum of nearest-centre distances over the sample.
+ *      the smallest resulting sum of nearest-centre distances over the sample. Sums over the
+ *      sample (that potential, and the running sums of the draw) are taken in blocks of 128
+ *      consecutive sample points: inside a block in order, then the block sums in order.
  *   3. At most max_iter * ceil(N / batch) steps; a step draws `batch` token indices uniformly with
  *      replacement, assigns each to its nearest centre (ties to the smaller index) and moves every
  *      centre that received points to the mean of all points it has received so far
@@ -244,7 +246,7 @@ int32_t santapp_kmeans_parent_count(int32_t prompt_len, int32_t parent_size);
  *                    the layout santapp_assign_parents takes
  *   steps_run        device int32 [n_kv_heads][n_seqs] or NULL, out: minibatch steps each fit ran
  *   workspace        device, >= santapp_kmeans_fit_workspace_bytes(...)
- * batch_size > 4096, or an initialisation sample above 28672 keys (more than 9557 centres in a
+ * batch_size > 4096, or an initialisation sample above 28544 keys (more than 9514 centres in a
  * sequence): SANTAPP_ERR_UNSUPPORTED. The call enqueues a few kernels per centre and per
  * step on `stream`. By default it waits for the stream every 16 steps to learn whether any fit
  * is still running (most stop long before the step limit), so it blocks the calling thread for

@@ -730,6 +730,11 @@ void orc_group_mean_keys_parents(int d, const double *keys, int32_t n_parents, c
  *     probability proportional to the squared distance to the nearest centre chosen so far (inverse
  *     CDF over the sample in order), "best" meaning the smallest resulting potential
  *     sum_i min(closest_i, |x_i - candidate|^2), ties to the earlier trial.
+ *     Sums over the sample (the potential of a trial, the running sums of the inverse CDF) are
+ *     taken in blocks of 128 consecutive sample points: the points of a block are added in order,
+ *     the block sums are added in order, and a running sum is (sum of the earlier blocks) + (sum
+ *     inside its block so far). The paper leaves the order open; this one lets the blocks be
+ *     summed side by side.
  *  3. At most max_iter * ceil(N / batch) minibatch steps. Step t draws `batch` indices uniformly
  *     with replacement (tag 3), assigns each to its nearest centre (ties to the smaller index),
  *     then moves every centre that received points to the mean of all points it has received so
@@ -753,6 +758,23 @@ static uint32_t km_word(uint64_t seed, uint32_t slot, uint32_t tag, uint32_t str
 
 static int32_t km_index(uint32_t word, int32_t n) { return (int32_t)(((uint64_t)word * (uint64_t)n) >> 32); }
 
+/* Sum of x[0..n) in blocks of 128 (see step 2 above); cum, when given, receives the running sums. */
+#define KM_SUM_BLOCK 128
+static double km_blocked_sum(const double *x, int32_t n, double *cum)
+{
+    double off = 0.0;
+    for (int32_t b0 = 0; b0 < n; b0 += KM_SUM_BLOCK) {
+        int32_t e = b0 + KM_SUM_BLOCK < n ? b0 + KM_SUM_BLOCK : n;
+        double w = 0.0;
+        for (int32_t i = b0; i < e; ++i) {
+            w += x[i];
+            if (cum) cum[i] = off + w;
+        }
+        off += w;
+    }
+    return off;
+}
+
 int32_t orc_minibatch_kmeans(int32_t N, int d, const double *keys, int32_t k, int32_t batch, int32_t max_iter,
                              int32_t patience, double ratio, uint64_t seed, uint32_t stream, double *centres)
 {
@@ -775,16 +797,15 @@ int32_t orc_minibatch_kmeans(int32_t N, int d, const double *keys, int32_t k, in
         memcpy(centres, keys + (int64_t)perm[first] * d, sizeof(double) * (size_t)d);
         for (int32_t i = 0; i < n_init; ++i) closest[i] = sqdist(keys + (int64_t)perm[i] * d, centres, d);
     }
+    double *cum = (double *)malloc(sizeof(double) * (size_t)n_init);
+    double *term = (double *)malloc(sizeof(double) * (size_t)n_init);
     for (int32_t c = 1; c < k; ++c) {
-        double total = 0.0;
-        for (int32_t i = 0; i < n_init; ++i) total += closest[i];
+        double total = km_blocked_sum(closest, n_init, cum);
         for (int32_t l = 0; l < L; ++l) {
             double target = orc_uniform_open(km_word(seed, (uint32_t)l, 2u, stream, (uint32_t)c)) * total;
-            double cum = 0.0;
             int32_t at = n_init - 1;
             for (int32_t i = 0; i < n_init; ++i) {
-                cum += closest[i];
-                if (cum > target) { at = i; break; }
+                if (cum[i] > target) { at = i; break; }
             }
             pick[l] = at;
         }
@@ -792,12 +813,12 @@ int32_t orc_minibatch_kmeans(int32_t N, int d, const double *keys, int32_t k, in
         double best_pot = INFINITY;
         for (int32_t l = 0; l < L; ++l) {
             const double *x = keys + (int64_t)perm[pick[l]] * d;
-            double pot = 0.0;
             for (int32_t i = 0; i < n_init; ++i) {
                 double dist = sqdist(keys + (int64_t)perm[i] * d, x, d);
                 cand[(int64_t)l * n_init + i] = dist;
-                pot += dist < closest[i] ? dist : closest[i];
+                term[i] = dist < closest[i] ? dist : closest[i];
             }
+            double pot = km_blocked_sum(term, n_init, NULL);
             if (pot < best_pot) { best_pot = pot; best = l; }
         }
         memcpy(centres + (int64_t)c * d, keys + (int64_t)perm[pick[best]] * d, sizeof(double) * (size_t)d);
@@ -806,7 +827,7 @@ int32_t orc_minibatch_kmeans(int32_t N, int d, const double *keys, int32_t k, in
             if (dist < closest[i]) closest[i] = dist;
         }
     }
-    free(pick); free(cand); free(closest); free(perm);
+    free(term); free(cum); free(pick); free(cand); free(closest); free(perm);
 
     /* 3.-5. minibatch steps */
     double *count = (double *)calloc((size_t)k, sizeof(double));

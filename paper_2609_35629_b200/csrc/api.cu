@@ -501,11 +501,11 @@ int santapp_build_groups_mean_parents(const santapp_geom *geom, const int32_t *p
 
 namespace {
 
-constexpr int kKmeansMaxSample = 28672;     // 224 KB of fp64 running sums: up to 9557 centres per sequence
+constexpr int kKmeansMaxSample = 28544;     // 223 KB of fp64 running sums (plus their block offsets): up to 9514 centres per sequence
 
 struct KmeansLayout {
-    size_t row_off, cen_off, tabs, perm, closest, cand, pick, centres64, count, idx, label, dist, state, active, total;
-    int k_max, n_init_max, trials_max, t_max_max, max_rows;
+    size_t row_off, cen_off, tabs, perm, closest, cand, part, pick, centres64, count, idx, label, dist, dist_part, label_part, state, active, total;
+    int k_max, n_init_max, trials_max, t_max_max, max_rows, assign_split;
     int64_t rows_total, centres_total;
 };
 
@@ -551,12 +551,17 @@ int kmeans_layout(const santapp_geom *geom, const int32_t *prompt_len_host, cons
     L->perm = take(sizeof(int32_t) * H * (size_t)L->rows_total);
     L->closest = take(sizeof(double) * pairs * (size_t)L->n_init_max);
     L->cand = take(sizeof(double) * pairs * (size_t)L->trials_max * (size_t)L->n_init_max);
+    L->part = take(sizeof(double) * pairs * (size_t)L->trials_max * (((size_t)L->n_init_max + 127) / 128));
     L->pick = take(sizeof(int32_t) * pairs * (size_t)L->trials_max);
     L->centres64 = take(sizeof(double) * H * (size_t)L->centres_total * kHeadDim);
     L->count = take(sizeof(double) * H * (size_t)L->centres_total);
     L->idx = take(sizeof(int32_t) * pairs * (size_t)o->batch_size);
     L->label = take(sizeof(int32_t) * pairs * (size_t)o->batch_size);
     L->dist = take(sizeof(double) * pairs * (size_t)o->batch_size);
+    // the nearest-centre search of a minibatch is cut into slices of the centres (about 128 each, at most 16)
+    L->assign_split = L->k_max / 128 < 1 ? 1 : (L->k_max / 128 > 16 ? 16 : L->k_max / 128);
+    L->dist_part = take(sizeof(double) * pairs * (size_t)L->assign_split * (size_t)o->batch_size);
+    L->label_part = take(sizeof(int32_t) * pairs * (size_t)L->assign_split * (size_t)o->batch_size);
     L->state = take(sizeof(KmeansState) * pairs);
     L->active = take(sizeof(int));
     L->total = off;
@@ -636,12 +641,16 @@ int santapp_kmeans_fit(const santapp_geom *geom, const int32_t *prompt_len_host,
     p.perm = reinterpret_cast<int32_t *>(ws + L.perm);
     p.closest = reinterpret_cast<double *>(ws + L.closest);
     p.cand = reinterpret_cast<double *>(ws + L.cand);
+    p.part = reinterpret_cast<double *>(ws + L.part);
     p.pick = reinterpret_cast<int32_t *>(ws + L.pick);
     p.centres64 = reinterpret_cast<double *>(ws + L.centres64);
     p.count = reinterpret_cast<double *>(ws + L.count);
     p.idx = reinterpret_cast<int32_t *>(ws + L.idx);
     p.label = reinterpret_cast<int32_t *>(ws + L.label);
     p.dist = reinterpret_cast<double *>(ws + L.dist);
+    p.dist_part = reinterpret_cast<double *>(ws + L.dist_part);
+    p.label_part = reinterpret_cast<int32_t *>(ws + L.label_part);
+    p.assign_split = L.assign_split;
     p.state = reinterpret_cast<KmeansState *>(ws + L.state);
     p.active = reinterpret_cast<int *>(ws + L.active);
     err = launch_kmeans_fit(p, s);

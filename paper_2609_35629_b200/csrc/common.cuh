@@ -300,11 +300,15 @@ struct KmeansParams {
     int32_t *perm;                          // [n_kv][rows_total]
     double *closest;                        // [pairs][n_init_max]
     double *cand;                           // [pairs][trials_max][n_init_max]
+    double *part;                           // [pairs][trials_max][ceil(n_init_max / 128)] block sums of the trials' potentials
     int32_t *pick;                          // [pairs][trials_max]
     double *centres64;                      // [n_kv][centres_total][128]
     double *count;                          // [n_kv][centres_total]
     int32_t *idx, *label;                   // [pairs][batch]
     double *dist;                           // [pairs][batch]
+    double *dist_part;                      // [pairs][assign_split][batch] nearest centre inside each slice of the centres
+    int32_t *label_part;                    // [pairs][assign_split][batch]
+    int assign_split;                       // slices the centres are cut into for the nearest-centre search
     KmeansState *state;                     // [pairs]
     int *active;                            // [1] fits that still have steps to run
 };

@@ -109,35 +109,60 @@ km_sample_kernel(KmeansParams p)
 }
 
 // ---- 2. greedy k-means++ on the sample ----
-// Distances of every sample point to the candidate points pick[0..n_cand): cand[l][i].
+constexpr int kSumBlock = 128;           // sums over the initialisation sample are taken in blocks of this many points
+constexpr int kMaxSumBlocks = 224;       // an initialisation sample holds at most 28544 points (223 blocks)
+static_assert(kThreads == 2 * kSumBlock, "a block of the distance kernel covers two blocks of the sums");
+
+// Distances of every sample point to the candidate points pick[0..n_cand): cand[l][i]; and, for c > 0,
+// the sums of min(closest_i, cand[l][i]) over each block of kSumBlock consecutive sample points, added
+// in order by one thread per block (the potential of a trial is the sum of its block sums in order).
 template <bool kHalf>
 __global__ void __launch_bounds__(kThreads)
 km_candidate_dist_kernel(KmeansParams p, int c)
 {
+    __shared__ double term_s[kThreads];
     const Pair q = pair_of(p, blockIdx.z / p.n_kv, blockIdx.z % p.n_kv);
     const int l = blockIdx.y;
     if (c >= q.k || l >= (c == 0 ? 1 : q.L)) return;
-    const int i = blockIdx.x * kThreads + threadIdx.x;
-    if (i >= q.n_init) return;
-    const int32_t *perm = p.perm + q.plane;
-    const uint4 *keys = reinterpret_cast<const uint4 *>(p.k_prompt + q.plane * kHeadDim);
-    const int at = p.pick[(size_t)q.id * p.trials_max + l];
-    p.cand[((size_t)q.id * p.trials_max + l) * p.n_init_max + i] =
-        sqdist_rows<kHalf>(keys + (size_t)perm[i] * 16, keys + (size_t)perm[at] * 16);
+    const int tid = threadIdx.x, i = blockIdx.x * kThreads + tid;
+    if (blockIdx.x * kThreads >= q.n_init) return;
+    double term = -1.0;                                     // marks a point past the end of the sample
+    if (i < q.n_init) {
+        const int32_t *perm = p.perm + q.plane;
+        const uint4 *keys = reinterpret_cast<const uint4 *>(p.k_prompt + q.plane * kHeadDim);
+        const int at = p.pick[(size_t)q.id * p.trials_max + l];
+        const double d = sqdist_rows<kHalf>(keys + (size_t)perm[i] * 16, keys + (size_t)perm[at] * 16);
+        p.cand[((size_t)q.id * p.trials_max + l) * p.n_init_max + i] = d;
+        if (c > 0) {
+            const double o = p.closest[(size_t)q.id * p.n_init_max + i];
+            term = d < o ? d : o;
+        }
+    }
+    if (c == 0) return;
+    term_s[tid] = term;
+    __syncthreads();
+    if ((tid & (kSumBlock - 1)) == 0) {
+        double w = 0.0;
+        for (int u = 0; u < kSumBlock; ++u) {
+            const double v = term_s[tid + u];
+            if (v >= 0.0) w = __dadd_rn(w, v);
+        }
+        const int n_part = (p.n_init_max + kSumBlock - 1) / kSumBlock;
+        const int blk = blockIdx.x * 2 + (tid >> 7);
+        if (blk * kSumBlock < q.n_init) p.part[((size_t)q.id * p.trials_max + l) * n_part + blk] = w;
+    }
 }
 
 constexpr int kAcceptThreads = 512;      // 16 warps: one per trial for up to 65536 centres (2 + ln k <= 13)
 
-// One block per pair: potentials of the trials (one lane each, sums in sample order), the best
+// One block per pair: potentials of the trials (sums in blocks of kSumBlock sample points), the best
 // trial becomes centre c, the nearest-centre distances are lowered.
 template <bool kHalf>
 __global__ void __launch_bounds__(kAcceptThreads)
 km_accept_kernel(KmeansParams p, int c)
 {
-    constexpr int kChunk = 128;
     __shared__ int best_s;
     __shared__ double pot_s[32];
-    __shared__ double chunk_s[kAcceptThreads / 32][kChunk];
     const Pair q = pair_of(p, blockIdx.x, blockIdx.y);
     if (c >= q.k) return;
     const int tid = threadIdx.x;
@@ -145,36 +170,13 @@ km_accept_kernel(KmeansParams p, int c)
     double *closest = p.closest + (size_t)q.id * p.n_init_max;
     const double *cand = p.cand + (size_t)q.id * p.trials_max * p.n_init_max;
     {
-        // warp l sums trial l: the lanes fetch a chunk of 256 terms into shared memory (the next
-        // chunk is in flight meanwhile), then lane 0 adds them in sample order: one chain of
-        // additions, as the order of the sum is part of the result
-        const int warp = tid >> 5, lane = tid & 31;
-        double *buf = chunk_s[warp];
-        for (int l = warp; l < n_trials && c > 0; l += kAcceptThreads / 32) {
-            const double *mine = cand + (size_t)l * p.n_init_max;
+        // the potential of a trial: its block sums (left by the distance kernel) added in order
+        const int n_blocks = (q.n_init + kSumBlock - 1) / kSumBlock, n_part = (p.n_init_max + kSumBlock - 1) / kSumBlock;
+        if (tid < n_trials && c > 0) {
+            const double *part = p.part + ((size_t)q.id * p.trials_max + tid) * n_part;
             double pot = 0.0;
-            auto fetch = [&](int i) {                       // term i of the potential (0 past the end)
-                if (i >= q.n_init) return 0.0;
-                const double d = mine[i], o = closest[i];
-                return d < o ? d : o;
-            };
-            double term[kChunk / 32];
-#pragma unroll
-            for (int v = 0; v < kChunk / 32; ++v) term[v] = fetch(32 * v + lane);
-            for (int i0 = 0; i0 < q.n_init; i0 += kChunk) {
-                __syncwarp();                               // lane 0 is done with the previous chunk
-#pragma unroll
-                for (int v = 0; v < kChunk / 32; ++v) buf[32 * v + lane] = term[v];
-#pragma unroll
-                for (int v = 0; v < kChunk / 32; ++v) term[v] = fetch(i0 + kChunk + 32 * v + lane);
-                __syncwarp();
-                if (lane == 0) {
-                    const int n = min(kChunk, q.n_init - i0);
-#pragma unroll 8
-                    for (int r = 0; r < n; ++r) pot = __dadd_rn(pot, buf[r]);
-                }
-            }
-            if (lane == 0) pot_s[l] = pot;
+            for (int blk = 0; blk < n_blocks; ++blk) pot = __dadd_rn(pot, part[blk]);
+            pot_s[tid] = pot;
         }
         __syncthreads();
         if (tid == 0) {
@@ -201,35 +203,56 @@ km_accept_kernel(KmeansParams p, int c)
 
 // One block per pair: the L trial points of centre c, drawn with probability proportional to the
 // distance to the nearest chosen centre by inverse CDF over the sample in order. The running sums
-// are formed by one thread (their order is part of the result) in shared memory; each trial then
-// finds the first running sum above its target by bisection (the sums never decrease).
+// are formed in blocks of kSumBlock points (inside a block in order, then the block sums in order: the
+// order is part of the result) in shared memory; each trial then finds the first running sum above its
+// target by bisection (the sums never decrease).
 __global__ void __launch_bounds__(kThreads)
 km_draw_trials_kernel(KmeansParams p, int c)
 {
-    extern __shared__ double cum_s[];                       // [n_init]
+    extern __shared__ double cum_s[];                       // [n_init] running sums, then [blocks] block offsets
     const Pair q = pair_of(p, blockIdx.x, blockIdx.y);
     if (c >= q.k) return;
     const int tid = threadIdx.x;
     const double *closest = p.closest + (size_t)q.id * p.n_init_max;
-    for (int i = tid; i < q.n_init; i += kThreads) cum_s[i] = closest[i];
-    __syncthreads();
-    if (tid == 0) {
-        double cum = 0.0;
-#pragma unroll 8
-        for (int i = 0; i < q.n_init; ++i) {
-            cum = __dadd_rn(cum, cum_s[i]);
-            cum_s[i] = cum;
+    const int n_blocks = (q.n_init + kSumBlock - 1) / kSumBlock;
+    double *off_s = cum_s + p.n_init_max + kMaxSumBlocks;
+    // cum_s holds one pad word per block (point i at i + i / kSumBlock), so that threads that walk
+    // different blocks do not meet in one bank
+    for (int blk = tid; blk < n_blocks; blk += kThreads) {  // running sums inside each block, in order
+        const int lo = blk * kSumBlock;
+        double w = 0.0;
+        for (int u = 0; u < kSumBlock; u += 8) {
+            double term[8];
+#pragma unroll
+            for (int v = 0; v < 8; ++v) term[v] = lo + u + v < q.n_init ? closest[lo + u + v] : -1.0;
+#pragma unroll
+            for (int v = 0; v < 8; ++v) {
+                if (term[v] >= 0.0) {
+                    w = __dadd_rn(w, term[v]);
+                    cum_s[lo + u + v + blk] = w;
+                }
+            }
         }
     }
     __syncthreads();
+    if (tid == 0) {                                         // sums of the earlier blocks, in order
+        double off = 0.0;
+        for (int blk = 0; blk < n_blocks; ++blk) {
+            off_s[blk] = off;
+            off = __dadd_rn(off, cum_s[min((blk + 1) * kSumBlock, q.n_init) - 1 + blk]);
+        }
+    }
+    __syncthreads();
+    for (int i = tid; i < q.n_init; i += kThreads) cum_s[i + i / kSumBlock] = __dadd_rn(off_s[i / kSumBlock], cum_s[i + i / kSumBlock]);
+    __syncthreads();
     if (tid < q.L) {
-        const double total = cum_s[q.n_init - 1];
+        const double total = cum_s[q.n_init - 1 + (q.n_init - 1) / kSumBlock];
         const uint32_t w = km_word(p, (uint32_t)tid, kTagStart, q.stream, (uint32_t)c);
         const double target = __dmul_rn(((double)w + 0.5) * (1.0 / 4294967296.0), total);
         int lo = 0, hi = q.n_init;                          // first i in [lo, hi) with cum_s[i] > target
         while (lo < hi) {
             const int mid = (lo + hi) >> 1;
-            if (cum_s[mid] > target) hi = mid; else lo = mid + 1;
+            if (cum_s[mid + mid / kSumBlock] > target) hi = mid; else lo = mid + 1;
         }
         p.pick[(size_t)q.id * p.trials_max + tid] = lo < q.n_init ? lo : q.n_init - 1;
     }
@@ -265,8 +288,13 @@ km_batch_assign_kernel(KmeansParams p, int t)
     double best = INFINITY;
     int arg = 0;
     const double *cen = p.centres64 + q.cplane * kHeadDim;
-    for (int base = 0; base < q.k; base += kTile) {
-        const int nt = min(kTile, q.k - base);
+    // this block searches one slice of the centres (a multiple of kTile each); the slices' results are
+    // compared in slice order afterwards, so ties still go to the smaller centre index
+    const int slice = blockIdx.z;
+    const int per = ((q.k + p.assign_split - 1) / p.assign_split + kTile - 1) / kTile * kTile;
+    const int k_lo = min(slice * per, q.k), k_hi = min(k_lo + per, q.k);
+    for (int base = k_lo; base < k_hi; base += kTile) {
+        const int nt = min(kTile, k_hi - base);
         __syncthreads();
         for (int e = tid; e < nt * kHeadDim; e += 128) c[e >> 7][e & 127] = cen[(size_t)base * kHeadDim + e];
         __syncthreads();
@@ -284,10 +312,37 @@ km_batch_assign_kernel(KmeansParams p, int t)
     }
     if (valid) {
         const size_t at = (size_t)q.id * p.batch + s;
-        p.idx[at] = idx;
-        p.label[at] = arg;
-        p.dist[at] = best;
+        if (slice == 0) p.idx[at] = idx;
+        if (p.assign_split == 1) {
+            p.label[at] = arg;
+            p.dist[at] = best;
+        } else {
+            const size_t pa = ((size_t)q.id * p.assign_split + slice) * p.batch + s;
+            p.label_part[pa] = arg;
+            p.dist_part[pa] = best;
+        }
     }
+}
+
+// The nearest centre of each minibatch point over all slices (strictly smaller distance wins, slices in
+// order of the centre index).
+__global__ void __launch_bounds__(128)
+km_assign_reduce_kernel(KmeansParams p, int t)
+{
+    const Pair q = pair_of(p, blockIdx.y / p.n_kv, blockIdx.y % p.n_kv);
+    if (!pair_active(p, q, t)) return;
+    const int s = blockIdx.x * 128 + threadIdx.x;
+    if (s >= p.batch) return;
+    double best = INFINITY;
+    int arg = 0;
+    for (int slice = 0; slice < p.assign_split; ++slice) {
+        const size_t pa = ((size_t)q.id * p.assign_split + slice) * p.batch + s;
+        const double d = p.dist_part[pa];
+        if (d < best) { best = d; arg = p.label_part[pa]; }
+    }
+    const size_t at = (size_t)q.id * p.batch + s;
+    p.label[at] = arg;
+    p.dist[at] = best;
 }
 
 // Cumulative-count update: thread (centre, dimension) adds the centre's new points in minibatch
@@ -437,7 +492,7 @@ cudaError_t run_fit(const KmeansParams &p, cudaStream_t s)
     km_sample_kernel<<<dim3(B, H), 32, 0, s>>>(p);
     KM_CHECK();
     const dim3 dist_grid((p.n_init_max + kThreads - 1) / kThreads, p.trials_max, pairs);
-    const size_t draw_smem = sizeof(double) * (size_t)p.n_init_max;
+    const size_t draw_smem = sizeof(double) * ((size_t)p.n_init_max + 2 * kMaxSumBlocks);
     if ((err = cudaFuncSetAttribute(km_draw_trials_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     (int)draw_smem)) != cudaSuccess)
         return err;
@@ -456,8 +511,12 @@ cudaError_t run_fit(const KmeansParams &p, cudaStream_t s)
     const size_t update_smem = sizeof(int32_t) * 2 * (size_t)p.batch;
     const size_t control_smem = sizeof(int32_t) * ((size_t)p.batch + (size_t)p.batch / 2 + 1);
     for (int t = 0; t < p.t_max_max; ++t) {
-        km_batch_assign_kernel<kHalf><<<dim3((p.batch + 127) / 128, pairs), 128, 0, s>>>(p, t);
+        km_batch_assign_kernel<kHalf><<<dim3((p.batch + 127) / 128, pairs, p.assign_split), 128, 0, s>>>(p, t);
         KM_CHECK();
+        if (p.assign_split > 1) {
+            km_assign_reduce_kernel<<<dim3((p.batch + 127) / 128, pairs), 128, 0, s>>>(p, t);
+            KM_CHECK();
+        }
         km_batch_update_kernel<kHalf><<<dim3((p.k_max + 1) / 2, pairs), kThreads, update_smem, s>>>(p, t);
         KM_CHECK();
         km_control_kernel<kHalf><<<dim3(B, H), 32, control_smem, s>>>(p, t);

@@ -187,8 +187,8 @@ def test_kmeans_fit_refuses_a_sample_that_does_not_fit_in_shared_memory(lib):
     g = sp.Geometry(1, 28, 4).c()
     n = (ctypes.c_int32 * 1)(200000)
     ok = sp.CKmeansOpts(4096, 100, 10, 0, 0.01, 0, 0, 0)
-    fits = (ctypes.c_int32 * 1)(9557)
-    too_many = (ctypes.c_int32 * 1)(9558)
+    fits = (ctypes.c_int32 * 1)(9514)
+    too_many = (ctypes.c_int32 * 1)(9515)
     assert lib.santapp_kmeans_fit_workspace_bytes(ctypes.byref(g), n, fits, ctypes.byref(ok)) > 0
     assert lib.santapp_kmeans_fit(ctypes.byref(g), n, too_many, 0x10000, ctypes.byref(ok), 0x10000, None, 0x10000,
                                   1 << 40, None) == sp.SANTAPP_ERR_UNSUPPORTED
