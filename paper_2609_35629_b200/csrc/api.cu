@@ -504,7 +504,7 @@ namespace {
 constexpr int kKmeansMaxSample = 28544;     // 223 KB of fp64 running sums (plus their block offsets): up to 9514 centres per sequence
 
 struct KmeansLayout {
-    size_t row_off, cen_off, tabs, perm, closest, cand, part, pick, centres64, count, idx, label, dist, dist_part, label_part, state, active, total;
+    size_t row_off, cen_off, tabs, perm, closest, cand, part, pick, centres64, count, idx, label, dist, dist_part, label_part, sorted, state, active, total;
     int k_max, n_init_max, trials_max, t_max_max, max_rows, assign_split;
     int64_t rows_total, centres_total;
 };
@@ -562,6 +562,7 @@ int kmeans_layout(const santapp_geom *geom, const int32_t *prompt_len_host, cons
     L->assign_split = L->k_max / 128 < 1 ? 1 : (L->k_max / 128 > 16 ? 16 : L->k_max / 128);
     L->dist_part = take(sizeof(double) * pairs * (size_t)L->assign_split * (size_t)o->batch_size);
     L->label_part = take(sizeof(int32_t) * pairs * (size_t)L->assign_split * (size_t)o->batch_size);
+    L->sorted = take(sizeof(uint32_t) * pairs * 4096);
     L->state = take(sizeof(KmeansState) * pairs);
     L->active = take(sizeof(int));
     L->total = off;
@@ -651,6 +652,7 @@ int santapp_kmeans_fit(const santapp_geom *geom, const int32_t *prompt_len_host,
     p.dist_part = reinterpret_cast<double *>(ws + L.dist_part);
     p.label_part = reinterpret_cast<int32_t *>(ws + L.label_part);
     p.assign_split = L.assign_split;
+    p.sorted = reinterpret_cast<uint32_t *>(ws + L.sorted);
     p.state = reinterpret_cast<KmeansState *>(ws + L.state);
     p.active = reinterpret_cast<int *>(ws + L.active);
     err = launch_kmeans_fit(p, s);

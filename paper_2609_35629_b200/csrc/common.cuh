@@ -309,6 +309,7 @@ struct KmeansParams {
     double *dist_part;                      // [pairs][assign_split][batch] nearest centre inside each slice of the centres
     int32_t *label_part;                    // [pairs][assign_split][batch]
     int assign_split;                       // slices the centres are cut into for the nearest-centre search
+    uint32_t *sorted;                       // [pairs][4096] minibatch slots ordered by (label, slot): label << 12 | slot, padded with ~0
     KmeansState *state;                     // [pairs]
     int *active;                            // [1] fits that still have steps to run
 };

@@ -153,101 +153,117 @@ km_candidate_dist_kernel(KmeansParams p, int c)
     }
 }
 
-constexpr int kAcceptThreads = 512;      // 16 warps: one per trial for up to 65536 centres (2 + ln k <= 13)
+constexpr int kAcceptThreads = 1024;
 
 // One block per pair: potentials of the trials (sums in blocks of kSumBlock sample points), the best
-// trial becomes centre c, the nearest-centre distances are lowered.
+// trial becomes centre c, the nearest-centre distances are lowered, and the trial points of centre
+// c + 1 are drawn. Every serial sum runs over shared memory with its loads ahead of its additions.
 template <bool kHalf>
 __global__ void __launch_bounds__(kAcceptThreads)
 km_accept_kernel(KmeansParams p, int c)
 {
+    extern __shared__ double cum_s[];                       // [n_init + blocks] running sums, then [blocks] block offsets
     __shared__ int best_s;
     __shared__ double pot_s[32];
     const Pair q = pair_of(p, blockIdx.x, blockIdx.y);
     if (c >= q.k) return;
     const int tid = threadIdx.x;
     const int n_trials = c == 0 ? 1 : q.L;
+    const int n_blocks = (q.n_init + kSumBlock - 1) / kSumBlock, n_part = (p.n_init_max + kSumBlock - 1) / kSumBlock;
     double *closest = p.closest + (size_t)q.id * p.n_init_max;
     const double *cand = p.cand + (size_t)q.id * p.trials_max * p.n_init_max;
-    {
+    double *off_s = cum_s + p.n_init_max + kMaxSumBlocks;
+    if (c > 0) {
         // the potential of a trial: its block sums (left by the distance kernel) added in order
-        const int n_blocks = (q.n_init + kSumBlock - 1) / kSumBlock, n_part = (p.n_init_max + kSumBlock - 1) / kSumBlock;
-        if (tid < n_trials && c > 0) {
-            const double *part = p.part + ((size_t)q.id * p.trials_max + tid) * n_part;
-            double pot = 0.0;
-            for (int blk = 0; blk < n_blocks; ++blk) pot = __dadd_rn(pot, part[blk]);
-            pot_s[tid] = pot;
+        for (int e = tid; e < n_trials * n_blocks; e += kAcceptThreads) {
+            const int l = e / n_blocks;
+            cum_s[e] = p.part[((size_t)q.id * p.trials_max + l) * n_part + (e - l * n_blocks)];
         }
         __syncthreads();
-        if (tid == 0) {
-            int best = 0;
-            for (int l = 1; l < n_trials; ++l)
-                if (pot_s[l] < pot_s[best]) best = l;
-            best_s = best;
+        if (tid < n_trials) {
+            double pot = 0.0;
+#pragma unroll 8
+            for (int blk = 0; blk < n_blocks; ++blk) pot = __dadd_rn(pot, cum_s[tid * n_blocks + blk]);
+            pot_s[tid] = pot;
         }
+    }
+    __syncthreads();
+    if (tid == 0) {
+        int best = 0;
+        for (int l = 1; l < n_trials; ++l)
+            if (pot_s[l] < pot_s[best]) best = l;
+        best_s = best;
     }
     __syncthreads();
     const int best = best_s;
     const double *win = cand + (size_t)best * p.n_init_max;
-    for (int i = tid; i < q.n_init; i += kAcceptThreads) {
-        const double d = win[i];
-        if (c == 0 || d < closest[i]) closest[i] = d;
-    }
     if (tid < kHeadDim) {
         const int32_t *perm = p.perm + q.plane;
         const int at = p.pick[(size_t)q.id * p.trials_max + best];
         const uint16_t v = p.k_prompt[(q.plane + (size_t)perm[at]) * kHeadDim + tid];
         p.centres64[(q.cplane + (size_t)c) * kHeadDim + tid] = elem_to_double<kHalf>(v);
     }
-}
-
-// One block per pair: the L trial points of centre c, drawn with probability proportional to the
-// distance to the nearest chosen centre by inverse CDF over the sample in order. The running sums
-// are formed in blocks of kSumBlock points (inside a block in order, then the block sums in order: the
-// order is part of the result) in shared memory; each trial then finds the first running sum above its
-// target by bisection (the sums never decrease).
-__global__ void __launch_bounds__(kThreads)
-km_draw_trials_kernel(KmeansParams p, int c)
-{
-    extern __shared__ double cum_s[];                       // [n_init] running sums, then [blocks] block offsets
-    const Pair q = pair_of(p, blockIdx.x, blockIdx.y);
-    if (c >= q.k) return;
-    const int tid = threadIdx.x;
-    const double *closest = p.closest + (size_t)q.id * p.n_init_max;
-    const int n_blocks = (q.n_init + kSumBlock - 1) / kSumBlock;
-    double *off_s = cum_s + p.n_init_max + kMaxSumBlocks;
-    // cum_s holds one pad word per block (point i at i + i / kSumBlock), so that threads that walk
-    // different blocks do not meet in one bank
-    for (int blk = tid; blk < n_blocks; blk += kThreads) {  // running sums inside each block, in order
-        const int lo = blk * kSumBlock;
-        double w = 0.0;
-        for (int u = 0; u < kSumBlock; u += 8) {
-            double term[8];
+    // The nearest-centre distances are lowered and kept in shared memory for the draw of the next
+    // centre's trial points (inverse CDF over the sample in order). cum_s holds one pad word per
+    // block of the sums (point i at i + i / kSumBlock), so that threads that walk different blocks do
+    // not meet in one bank.
+    for (int i0 = 0; i0 < q.n_init; i0 += 8 * kAcceptThreads) {
+        double d[8], o[8];
 #pragma unroll
-            for (int v = 0; v < 8; ++v) term[v] = lo + u + v < q.n_init ? closest[lo + u + v] : -1.0;
+        for (int v = 0; v < 8; ++v) {
+            const int i = i0 + v * kAcceptThreads + tid;
+            if (i < q.n_init) {
+                d[v] = win[i];
+                o[v] = c == 0 ? 0.0 : closest[i];
+            }
+        }
+#pragma unroll
+        for (int v = 0; v < 8; ++v) {
+            const int i = i0 + v * kAcceptThreads + tid;
+            if (i < q.n_init) {
+                const double t = (c == 0 || d[v] < o[v]) ? d[v] : o[v];
+                closest[i] = t;
+                cum_s[i + i / kSumBlock] = t;
+            }
+        }
+    }
+    if (c + 1 >= q.k) return;                               // the pair's last centre draws nothing
+    __syncthreads();
+    // running sums inside each block (a thread per block), the block offsets in order, offset + running sum
+    if (tid < n_blocks) {
+        const int lo = tid * kSumBlock, cnt = min(kSumBlock, q.n_init - lo);
+        double *blk_s = cum_s + lo + tid;
+        double w = 0.0;
+        for (int u = 0; u < cnt; u += 8) {
+            double t[8];
+#pragma unroll
+            for (int v = 0; v < 8; ++v) t[v] = u + v < cnt ? blk_s[u + v] : 0.0;
 #pragma unroll
             for (int v = 0; v < 8; ++v) {
-                if (term[v] >= 0.0) {
-                    w = __dadd_rn(w, term[v]);
-                    cum_s[lo + u + v + blk] = w;
+                if (u + v < cnt) {
+                    w = __dadd_rn(w, t[v]);
+                    blk_s[u + v] = w;
                 }
             }
         }
+        off_s[tid] = w;
     }
     __syncthreads();
     if (tid == 0) {                                         // sums of the earlier blocks, in order
         double off = 0.0;
+#pragma unroll 8
         for (int blk = 0; blk < n_blocks; ++blk) {
+            const double t = off_s[blk];
             off_s[blk] = off;
-            off = __dadd_rn(off, cum_s[min((blk + 1) * kSumBlock, q.n_init) - 1 + blk]);
+            off = __dadd_rn(off, t);
         }
     }
     __syncthreads();
-    for (int i = tid; i < q.n_init; i += kThreads) cum_s[i + i / kSumBlock] = __dadd_rn(off_s[i / kSumBlock], cum_s[i + i / kSumBlock]);
+    for (int i = tid; i < q.n_init; i += kAcceptThreads) cum_s[i + i / kSumBlock] = __dadd_rn(off_s[i / kSumBlock], cum_s[i + i / kSumBlock]);
     __syncthreads();
     if (tid < q.L) {
         const double total = cum_s[q.n_init - 1 + (q.n_init - 1) / kSumBlock];
-        const uint32_t w = km_word(p, (uint32_t)tid, kTagStart, q.stream, (uint32_t)c);
+        const uint32_t w = km_word(p, (uint32_t)tid, kTagStart, q.stream, (uint32_t)(c + 1));
         const double target = __dmul_rn(((double)w + 0.5) * (1.0 / 4294967296.0), total);
         int lo = 0, hi = q.n_init;                          // first i in [lo, hi) with cum_s[i] > target
         while (lo < hi) {
@@ -345,35 +361,58 @@ km_assign_reduce_kernel(KmeansParams p, int t)
     p.dist[at] = best;
 }
 
+// The minibatch's slots ordered by (label, slot), one block per pair: a bitonic sort of the keys
+// label << 12 | slot in shared memory (batch <= 4096; the keys are distinct, so the order is the
+// minibatch order inside every label).
+constexpr int kSortThreads = 1024, kSortKeys = 4096;
+__global__ void __launch_bounds__(kSortThreads)
+km_sort_batch_kernel(KmeansParams p, int t)
+{
+    __shared__ uint32_t key_s[kSortKeys];
+    const Pair q = pair_of(p, blockIdx.x / p.n_kv, blockIdx.x % p.n_kv);
+    if (!pair_active(p, q, t)) return;
+    const int tid = threadIdx.x;
+    for (int s = tid; s < kSortKeys; s += kSortThreads)
+        key_s[s] = s < p.batch ? ((uint32_t)p.label[(size_t)q.id * p.batch + s] << 12) | (uint32_t)s : 0xFFFFFFFFu;
+    __syncthreads();
+    for (int size = 2; size <= kSortKeys; size <<= 1) {
+        for (int stride = size >> 1; stride > 0; stride >>= 1) {
+            for (int e = tid; e < kSortKeys / 2; e += kSortThreads) {
+                const int lo = 2 * e - (e & (stride - 1)), hi = lo + stride;       // partners of this compare-exchange
+                const bool up = (lo & size) == 0;
+                const uint32_t a = key_s[lo], b = key_s[hi];
+                if ((a > b) == up) { key_s[lo] = b; key_s[hi] = a; }
+            }
+            __syncthreads();
+        }
+    }
+    for (int s = tid; s < kSortKeys; s += kSortThreads) p.sorted[(size_t)q.id * kSortKeys + s] = key_s[s];
+}
+
 // Cumulative-count update: thread (centre, dimension) adds the centre's new points in minibatch
-// order; c <- (c * count + sum) / (count + n).
+// order (it finds them in the sorted slots); c <- (c * count + sum) / (count + n).
 template <bool kHalf>
 __global__ void __launch_bounds__(kThreads)
 km_batch_update_kernel(KmeansParams p, int t)
 {
-    extern __shared__ int32_t batch_tab[];                  // labels, then indices
     const Pair q = pair_of(p, blockIdx.y / p.n_kv, blockIdx.y % p.n_kv);
     if (!pair_active(p, q, t)) return;
-    const int u0 = blockIdx.x * (kThreads / kHeadDim);
-    if (u0 >= q.k) return;
-    int32_t *lab = batch_tab, *idx = batch_tab + p.batch;
-    for (int s = threadIdx.x; s < p.batch; s += kThreads) {
-        lab[s] = p.label[(size_t)q.id * p.batch + s];
-        idx[s] = p.idx[(size_t)q.id * p.batch + s];
-    }
-    __syncthreads();
-    const int u = u0 + threadIdx.x / kHeadDim, d = threadIdx.x % kHeadDim;
+    const int u = blockIdx.x * (kThreads / kHeadDim) + threadIdx.x / kHeadDim, d = threadIdx.x % kHeadDim;
     const bool live = u < q.k;
     double sum = 0.0, count = 0.0;
     int n = 0;
     if (live) {
+        const uint32_t *sorted = p.sorted + (size_t)q.id * kSortKeys;
+        int lo = 0, hi = kSortKeys;                         // first position with label >= u
+        while (lo < hi) {
+            const int mid = (lo + hi) >> 1;
+            if ((sorted[mid] >> 12) >= (uint32_t)u) hi = mid; else lo = mid + 1;
+        }
         count = p.count[q.cplane + u];
         const uint16_t *col = p.k_prompt + q.plane * kHeadDim + d;
-        for (int s = 0; s < p.batch; ++s) {
-            if (lab[s] != u) continue;
-            ++n;
-            sum = __dadd_rn(sum, elem_to_double<kHalf>(col[(size_t)idx[s] * kHeadDim]));
-        }
+        const int32_t *idx = p.idx + (size_t)q.id * p.batch;
+        for (int at = lo; at < kSortKeys && (sorted[at] >> 12) == (uint32_t)u; ++at, ++n)
+            sum = __dadd_rn(sum, elem_to_double<kHalf>(col[(size_t)idx[sorted[at] & 4095u] * kHeadDim]));
     }
     __syncthreads();                                        // every thread has read its centre's count
     if (live && n > 0) {
@@ -493,22 +532,16 @@ cudaError_t run_fit(const KmeansParams &p, cudaStream_t s)
     KM_CHECK();
     const dim3 dist_grid((p.n_init_max + kThreads - 1) / kThreads, p.trials_max, pairs);
     const size_t draw_smem = sizeof(double) * ((size_t)p.n_init_max + 2 * kMaxSumBlocks);
-    if ((err = cudaFuncSetAttribute(km_draw_trials_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                    (int)draw_smem)) != cudaSuccess)
+    if ((err = cudaFuncSetAttribute(km_accept_kernel<kHalf>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)draw_smem)) != cudaSuccess)
         return err;
     for (int c = 0; c < p.k_max; ++c) {
-        if (c > 0) {
-            km_draw_trials_kernel<<<dim3(B, H), kThreads, draw_smem, s>>>(p, c);
-            KM_CHECK();
-        }
         km_candidate_dist_kernel<kHalf><<<dist_grid, kThreads, 0, s>>>(p, c);
         KM_CHECK();
-        km_accept_kernel<kHalf><<<dim3(B, H), kAcceptThreads, 0, s>>>(p, c);
+        km_accept_kernel<kHalf><<<dim3(B, H), kAcceptThreads, draw_smem, s>>>(p, c);     // ... and the trial points of centre c + 1
         KM_CHECK();
     }
     if ((err = cudaMemsetAsync(p.count, 0, sizeof(double) * (size_t)H * p.centres_total, s)) != cudaSuccess) return err;
     if ((err = cudaMemsetAsync(p.state, 0, sizeof(KmeansState) * (size_t)pairs, s)) != cudaSuccess) return err;
-    const size_t update_smem = sizeof(int32_t) * 2 * (size_t)p.batch;
     const size_t control_smem = sizeof(int32_t) * ((size_t)p.batch + (size_t)p.batch / 2 + 1);
     for (int t = 0; t < p.t_max_max; ++t) {
         km_batch_assign_kernel<kHalf><<<dim3((p.batch + 127) / 128, pairs, p.assign_split), 128, 0, s>>>(p, t);
@@ -517,7 +550,9 @@ cudaError_t run_fit(const KmeansParams &p, cudaStream_t s)
             km_assign_reduce_kernel<<<dim3((p.batch + 127) / 128, pairs), 128, 0, s>>>(p, t);
             KM_CHECK();
         }
-        km_batch_update_kernel<kHalf><<<dim3((p.k_max + 1) / 2, pairs), kThreads, update_smem, s>>>(p, t);
+        km_sort_batch_kernel<<<dim3(pairs), kSortThreads, 0, s>>>(p, t);
+        KM_CHECK();
+        km_batch_update_kernel<kHalf><<<dim3((p.k_max + 1) / 2, pairs), kThreads, 0, s>>>(p, t);
         KM_CHECK();
         km_control_kernel<kHalf><<<dim3(B, H), 32, control_smem, s>>>(p, t);
         KM_CHECK();
