@@ -111,45 +111,141 @@ km_sample_kernel(KmeansParams p)
 // ---- 2. greedy k-means++ on the sample ----
 constexpr int kSumBlock = 128;           // sums over the initialisation sample are taken in blocks of this many points
 constexpr int kMaxSumBlocks = 224;       // an initialisation sample holds at most 28544 points (223 blocks)
-static_assert(kThreads == 2 * kSumBlock, "a block of the distance kernel covers two blocks of the sums");
+// fp32 -> fp64 where it is written (the compiler would otherwise widen all of a point's values ahead of
+// a loop over centres and keep them in local memory)
+__device__ __forceinline__ double widen_here(float x)
+{
+    double r;
+    asm volatile("cvt.f64.f32 %0, %1;" : "=d"(r) : "f"(x));
+    return r;
+}
+
+constexpr int kDistThreads = 64;         // a block covers one block of the sums: two points per thread
+constexpr int kDistTrials = 6;           // candidate points per block
+
+// Squared distances (fp64, the 128 terms added in order) of two points (rows of packed words in global
+// memory, read eight values at a time, one read ahead) to kN candidate points held as doubles in
+// shared memory: a candidate value serves both points and a point value is widened once for all
+// candidates (widening runs at a quarter of the fp64 add rate). The loop is kept rolled: a warp runs
+// it once, and a body unrolled over the whole row is fetched from instruction memory slower than it runs.
+template <bool kHalf, int kN>
+__device__ __forceinline__ void dist_two_points(const uint4 *row0, const uint4 *row1, const double (*y_s)[kHeadDim],
+                                                double (&d)[2][kDistTrials])
+{
+    uint4 nxt0 = row0[0], nxt1 = row1[0];
+#pragma unroll 1
+    for (int qd = 0; qd < 16; ++qd) {
+        const uint32_t xw[2][4] = {{nxt0.x, nxt0.y, nxt0.z, nxt0.w}, {nxt1.x, nxt1.y, nxt1.z, nxt1.w}};
+        if (qd + 1 < 16) {
+            nxt0 = row0[qd + 1];
+            nxt1 = row1[qd + 1];
+        }
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+            double2 y[kN];
+#pragma unroll
+            for (int v = 0; v < kN; ++v) y[v] = *reinterpret_cast<const double2 *>(&y_s[v][8 * qd + 2 * t]);
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                const double x0 = widen_here(elem_lo<kHalf>(xw[j][t])), x1 = widen_here(elem_hi<kHalf>(xw[j][t]));
+#pragma unroll
+                for (int v = 0; v < kN; ++v) {
+                    const double e = __dsub_rn(x0, y[v].x);
+                    d[j][v] = __dadd_rn(d[j][v], __dmul_rn(e, e));
+                }
+#pragma unroll
+                for (int v = 0; v < kN; ++v) {
+                    const double e = __dsub_rn(x1, y[v].y);
+                    d[j][v] = __dadd_rn(d[j][v], __dmul_rn(e, e));
+                }
+            }
+        }
+    }
+}
 
 // Distances of every sample point to the candidate points pick[0..n_cand): cand[l][i]; and, for c > 0,
 // the sums of min(closest_i, cand[l][i]) over each block of kSumBlock consecutive sample points, added
-// in order by one thread per block (the potential of a trial is the sum of its block sums in order).
+// in order by one thread per candidate (the potential of a trial is the sum of its block sums in order).
 template <bool kHalf>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kDistThreads)
 km_candidate_dist_kernel(KmeansParams p, int c)
 {
-    __shared__ double term_s[kThreads];
+    __shared__ __align__(16) double y_s[kDistTrials][kHeadDim];
+    __shared__ double term_s[kDistTrials][kSumBlock];
     const Pair q = pair_of(p, blockIdx.z / p.n_kv, blockIdx.z % p.n_kv);
-    const int l = blockIdx.y;
-    if (c >= q.k || l >= (c == 0 ? 1 : q.L)) return;
-    const int tid = threadIdx.x, i = blockIdx.x * kThreads + tid;
-    if (blockIdx.x * kThreads >= q.n_init) return;
-    double term = -1.0;                                     // marks a point past the end of the sample
-    if (i < q.n_init) {
-        const int32_t *perm = p.perm + q.plane;
-        const uint4 *keys = reinterpret_cast<const uint4 *>(p.k_prompt + q.plane * kHeadDim);
-        const int at = p.pick[(size_t)q.id * p.trials_max + l];
-        const double d = sqdist_rows<kHalf>(keys + (size_t)perm[i] * 16, keys + (size_t)perm[at] * 16);
-        p.cand[((size_t)q.id * p.trials_max + l) * p.n_init_max + i] = d;
-        if (c > 0) {
-            const double o = p.closest[(size_t)q.id * p.n_init_max + i];
-            term = d < o ? d : o;
+    if (c >= q.k || blockIdx.x * kSumBlock >= q.n_init) return;
+    const int L = c == 0 ? 1 : q.L;
+    const int n_chunks = (L + kDistTrials - 1) / kDistTrials, per = (L + n_chunks - 1) / n_chunks;
+    const int l0 = blockIdx.y * per, cn = min(per, L - l0);
+    if (cn <= 0) return;
+    const int tid = threadIdx.x;
+    const int32_t *perm = p.perm + q.plane;
+    const uint16_t *keys = p.k_prompt + q.plane * kHeadDim;
+    __shared__ int row_s[kDistTrials];
+    if (tid < cn) row_s[tid] = perm[p.pick[(size_t)q.id * p.trials_max + l0 + tid]];
+    int i[2];
+    const uint4 *row[2];
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+        i[j] = blockIdx.x * kSumBlock + j * kDistThreads + tid;
+        row[j] = reinterpret_cast<const uint4 *>(keys + (size_t)perm[min(i[j], q.n_init - 1)] * kHeadDim);
+    }
+    __syncthreads();
+    {
+        // the candidates' rows as doubles: a thread widens one packed word (two values) of every row
+        uint32_t yw[kDistTrials];
+#pragma unroll
+        for (int v = 0; v < kDistTrials; ++v)
+            yw[v] = v < cn ? reinterpret_cast<const uint32_t *>(keys + (size_t)row_s[v] * kHeadDim)[tid] : 0u;
+#pragma unroll
+        for (int v = 0; v < kDistTrials; ++v) {
+            if (v < cn) {
+                y_s[v][2 * tid] = (double)elem_lo<kHalf>(yw[v]);
+                y_s[v][2 * tid + 1] = (double)elem_hi<kHalf>(yw[v]);
+            }
+        }
+    }
+    __syncthreads();
+    double d[2][kDistTrials];
+#pragma unroll
+    for (int j = 0; j < 2; ++j)
+#pragma unroll
+        for (int v = 0; v < kDistTrials; ++v) d[j][v] = 0.0;
+    switch (cn) {
+    case 1: dist_two_points<kHalf, 1>(row[0], row[1], y_s, d); break;
+    case 2: dist_two_points<kHalf, 2>(row[0], row[1], y_s, d); break;
+    case 3: dist_two_points<kHalf, 3>(row[0], row[1], y_s, d); break;
+    case 4: dist_two_points<kHalf, 4>(row[0], row[1], y_s, d); break;
+    case 5: dist_two_points<kHalf, 5>(row[0], row[1], y_s, d); break;
+    default: dist_two_points<kHalf, 6>(row[0], row[1], y_s, d); break;
+    }
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+#pragma unroll
+        for (int v = 0; v < kDistTrials; ++v) {
+            if (v >= cn) continue;
+            double term = -1.0;                             // marks a point past the end of the sample
+            if (i[j] < q.n_init) {
+                p.cand[((size_t)q.id * p.trials_max + l0 + v) * p.n_init_max + i[j]] = d[j][v];
+                if (c > 0) {
+                    const double o = p.closest[(size_t)q.id * p.n_init_max + i[j]];
+                    term = d[j][v] < o ? d[j][v] : o;
+                }
+            }
+            term_s[v][j * kDistThreads + tid] = term;
         }
     }
     if (c == 0) return;
-    term_s[tid] = term;
     __syncthreads();
-    if ((tid & (kSumBlock - 1)) == 0) {
+    if (tid < cn) {
         double w = 0.0;
+#pragma unroll 8
         for (int u = 0; u < kSumBlock; ++u) {
-            const double v = term_s[tid + u];
+            const double v = term_s[tid][u];
             if (v >= 0.0) w = __dadd_rn(w, v);
         }
         const int n_part = (p.n_init_max + kSumBlock - 1) / kSumBlock;
-        const int blk = blockIdx.x * 2 + (tid >> 7);
-        if (blk * kSumBlock < q.n_init) p.part[((size_t)q.id * p.trials_max + l) * n_part + blk] = w;
+        p.part[((size_t)q.id * p.trials_max + l0 + tid) * n_part + blockIdx.x] = w;
     }
 }
 
@@ -280,29 +376,38 @@ __device__ __forceinline__ bool pair_active(const KmeansParams &p, const Pair &q
     return t < q.t_max && !p.state[q.id].stopped;
 }
 
-// Draw the minibatch and assign each point to its nearest centre (ties to the smaller index).
+// Draw the minibatch and assign each point to its nearest centre (ties to the smaller index). A thread
+// holds two points and takes four centres at a time: a centre value read from shared memory serves
+// two sums and a point value is widened once for four, so that neither the shared-memory path nor
+// the conversions hold up the fp64 pipe; every sum still adds its 128 terms in order.
+constexpr int kAssignPts = 2;             // points per thread
+
+constexpr int kAssignBlock = 128 * kAssignPts;
 template <bool kHalf>
 __global__ void __launch_bounds__(128)
 km_batch_assign_kernel(KmeansParams p, int t)
 {
-    __shared__ double c[kTile][kHeadDim];
+    __shared__ __align__(16) double c[kTile][kHeadDim];
     const Pair q = pair_of(p, blockIdx.y / p.n_kv, blockIdx.y % p.n_kv);
     if (!pair_active(p, q, t)) return;
     const int tid = threadIdx.x;
-    const int s = blockIdx.x * 128 + tid;
-    const bool valid = s < p.batch;
-    const int idx = km_index(km_word(p, (uint32_t)(valid ? s : 0), kTagBatch, q.stream, (uint32_t)t), q.N);
-    uint32_t kw[64];
-    {
-        const uint4 *row = reinterpret_cast<const uint4 *>(p.k_prompt + (q.plane + (size_t)idx) * kHeadDim);
+    int s[kAssignPts], idx[kAssignPts];
+    uint32_t kw[kAssignPts][64];
+#pragma unroll
+    for (int j = 0; j < kAssignPts; ++j) {
+        s[j] = blockIdx.x * kAssignBlock + j * 128 + tid;
+        idx[j] = km_index(km_word(p, (uint32_t)(s[j] < p.batch ? s[j] : 0), kTagBatch, q.stream, (uint32_t)t), q.N);
+        const uint4 *row = reinterpret_cast<const uint4 *>(p.k_prompt + (q.plane + (size_t)idx[j]) * kHeadDim);
 #pragma unroll
         for (int v = 0; v < 16; ++v) {
             const uint4 w = row[v];
-            kw[4 * v] = w.x; kw[4 * v + 1] = w.y; kw[4 * v + 2] = w.z; kw[4 * v + 3] = w.w;
+            kw[j][4 * v] = w.x; kw[j][4 * v + 1] = w.y; kw[j][4 * v + 2] = w.z; kw[j][4 * v + 3] = w.w;
         }
     }
-    double best = INFINITY;
-    int arg = 0;
+    double best[kAssignPts];
+    int arg[kAssignPts];
+#pragma unroll
+    for (int j = 0; j < kAssignPts; ++j) { best[j] = INFINITY; arg[j] = 0; }
     const double *cen = p.centres64 + q.cplane * kHeadDim;
     // this block searches one slice of the centres (a multiple of kTile each); the slices' results are
     // compared in slice order afterwards, so ties still go to the smaller centre index
@@ -314,28 +419,52 @@ km_batch_assign_kernel(KmeansParams p, int t)
         __syncthreads();
         for (int e = tid; e < nt * kHeadDim; e += 128) c[e >> 7][e & 127] = cen[(size_t)base * kHeadDim + e];
         __syncthreads();
-        for (int u = 0; u < nt; ++u) {
-            double d = 0.0;
+        for (int u = 0; u < nt; u += 4) {
+            const double *cu[4] = {c[u], c[min(u + 1, nt - 1)], c[min(u + 2, nt - 1)], c[min(u + 3, nt - 1)]};
+            double d[kAssignPts][4];
+#pragma unroll
+            for (int j = 0; j < kAssignPts; ++j)
+#pragma unroll
+                for (int v = 0; v < 4; ++v) d[j][v] = 0.0;
 #pragma unroll
             for (int w = 0; w < 64; ++w) {
-                const double e0 = __dsub_rn((double)elem_lo<kHalf>(kw[w]), c[u][2 * w]);
-                const double e1 = __dsub_rn((double)elem_hi<kHalf>(kw[w]), c[u][2 * w + 1]);
-                d = __dadd_rn(d, __dmul_rn(e0, e0));
-                d = __dadd_rn(d, __dmul_rn(e1, e1));
+                double2 y[4];
+#pragma unroll
+                for (int v = 0; v < 4; ++v) y[v] = *reinterpret_cast<const double2 *>(cu[v] + 2 * w);
+#pragma unroll
+                for (int j = 0; j < kAssignPts; ++j) {
+                    const double x0 = widen_here(elem_lo<kHalf>(kw[j][w])), x1 = widen_here(elem_hi<kHalf>(kw[j][w]));
+#pragma unroll
+                    for (int v = 0; v < 4; ++v) {
+                        const double e = __dsub_rn(x0, y[v].x);
+                        d[j][v] = __dadd_rn(d[j][v], __dmul_rn(e, e));
+                    }
+#pragma unroll
+                    for (int v = 0; v < 4; ++v) {
+                        const double e = __dsub_rn(x1, y[v].y);
+                        d[j][v] = __dadd_rn(d[j][v], __dmul_rn(e, e));
+                    }
+                }
             }
-            if (d < best) { best = d; arg = base + u; }
+#pragma unroll
+            for (int j = 0; j < kAssignPts; ++j)
+#pragma unroll
+                for (int v = 0; v < 4; ++v)
+                    if (u + v < nt && d[j][v] < best[j]) { best[j] = d[j][v]; arg[j] = base + u + v; }
         }
     }
-    if (valid) {
-        const size_t at = (size_t)q.id * p.batch + s;
-        if (slice == 0) p.idx[at] = idx;
+#pragma unroll
+    for (int j = 0; j < kAssignPts; ++j) {
+        if (s[j] >= p.batch) continue;
+        const size_t at = (size_t)q.id * p.batch + s[j];
+        if (slice == 0) p.idx[at] = idx[j];
         if (p.assign_split == 1) {
-            p.label[at] = arg;
-            p.dist[at] = best;
+            p.label[at] = arg[j];
+            p.dist[at] = best[j];
         } else {
-            const size_t pa = ((size_t)q.id * p.assign_split + slice) * p.batch + s;
-            p.label_part[pa] = arg;
-            p.dist_part[pa] = best;
+            const size_t pa = ((size_t)q.id * p.assign_split + slice) * p.batch + s[j];
+            p.label_part[pa] = arg[j];
+            p.dist_part[pa] = best[j];
         }
     }
 }
@@ -530,12 +659,12 @@ cudaError_t run_fit(const KmeansParams &p, cudaStream_t s)
     KM_CHECK();
     km_sample_kernel<<<dim3(B, H), 32, 0, s>>>(p);
     KM_CHECK();
-    const dim3 dist_grid((p.n_init_max + kThreads - 1) / kThreads, p.trials_max, pairs);
+    const dim3 dist_grid((p.n_init_max + kSumBlock - 1) / kSumBlock, (p.trials_max + kDistTrials - 1) / kDistTrials, pairs);
     const size_t draw_smem = sizeof(double) * ((size_t)p.n_init_max + 2 * kMaxSumBlocks);
     if ((err = cudaFuncSetAttribute(km_accept_kernel<kHalf>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)draw_smem)) != cudaSuccess)
         return err;
     for (int c = 0; c < p.k_max; ++c) {
-        km_candidate_dist_kernel<kHalf><<<dist_grid, kThreads, 0, s>>>(p, c);
+        km_candidate_dist_kernel<kHalf><<<dist_grid, kDistThreads, 0, s>>>(p, c);
         KM_CHECK();
         km_accept_kernel<kHalf><<<dim3(B, H), kAcceptThreads, draw_smem, s>>>(p, c);     // ... and the trial points of centre c + 1
         KM_CHECK();
@@ -544,7 +673,7 @@ cudaError_t run_fit(const KmeansParams &p, cudaStream_t s)
     if ((err = cudaMemsetAsync(p.state, 0, sizeof(KmeansState) * (size_t)pairs, s)) != cudaSuccess) return err;
     const size_t control_smem = sizeof(int32_t) * ((size_t)p.batch + (size_t)p.batch / 2 + 1);
     for (int t = 0; t < p.t_max_max; ++t) {
-        km_batch_assign_kernel<kHalf><<<dim3((p.batch + 127) / 128, pairs, p.assign_split), 128, 0, s>>>(p, t);
+        km_batch_assign_kernel<kHalf><<<dim3((p.batch + kAssignBlock - 1) / kAssignBlock, pairs, p.assign_split), 128, 0, s>>>(p, t);
         KM_CHECK();
         if (p.assign_split > 1) {
             km_assign_reduce_kernel<<<dim3((p.batch + 127) / 128, pairs), 128, 0, s>>>(p, t);
