@@ -120,25 +120,29 @@ __device__ __forceinline__ double widen_here(float x)
     return r;
 }
 
-constexpr int kDistThreads = 64;         // a block covers one block of the sums: two points per thread
+constexpr int kDistPts = 1;              // points per thread
+constexpr int kDistThreads = kSumBlock / kDistPts;   // a block covers one block of the sums
+static_assert(kDistThreads % 64 == 0, "64 threads widen one candidate row");
 constexpr int kDistTrials = 6;           // candidate points per block
 
-// Squared distances (fp64, the 128 terms added in order) of two points (rows of packed words in global
+// Squared distances (fp64, the 128 terms added in order) of kP points (rows of packed words in global
 // memory, read eight values at a time, one read ahead) to kN candidate points held as doubles in
-// shared memory: a candidate value serves both points and a point value is widened once for all
+// shared memory: a candidate value serves all kP points and a point value is widened once for all
 // candidates (widening runs at a quarter of the fp64 add rate). The loop is kept rolled: a warp runs
 // it once, and a body unrolled over the whole row is fetched from instruction memory slower than it runs.
-template <bool kHalf, int kN>
-__device__ __forceinline__ void dist_two_points(const uint4 *row0, const uint4 *row1, const double (*y_s)[kHeadDim],
-                                                double (&d)[2][kDistTrials])
+template <bool kHalf, int kP, int kN, int kD>
+__device__ __forceinline__ void dist_points(const uint4 *const (&row)[kP], const double (*y_s)[kHeadDim], double (&d)[kP][kD])
 {
-    uint4 nxt0 = row0[0], nxt1 = row1[0];
+    uint4 nxt[kP];
+#pragma unroll
+    for (int j = 0; j < kP; ++j) nxt[j] = row[j][0];
 #pragma unroll 1
     for (int qd = 0; qd < 16; ++qd) {
-        const uint32_t xw[2][4] = {{nxt0.x, nxt0.y, nxt0.z, nxt0.w}, {nxt1.x, nxt1.y, nxt1.z, nxt1.w}};
-        if (qd + 1 < 16) {
-            nxt0 = row0[qd + 1];
-            nxt1 = row1[qd + 1];
+        uint32_t xw[kP][4];
+#pragma unroll
+        for (int j = 0; j < kP; ++j) {
+            xw[j][0] = nxt[j].x; xw[j][1] = nxt[j].y; xw[j][2] = nxt[j].z; xw[j][3] = nxt[j].w;
+            if (qd + 1 < 16) nxt[j] = row[j][qd + 1];
         }
 #pragma unroll
         for (int t = 0; t < 4; ++t) {
@@ -146,7 +150,7 @@ __device__ __forceinline__ void dist_two_points(const uint4 *row0, const uint4 *
 #pragma unroll
             for (int v = 0; v < kN; ++v) y[v] = *reinterpret_cast<const double2 *>(&y_s[v][8 * qd + 2 * t]);
 #pragma unroll
-            for (int j = 0; j < 2; ++j) {
+            for (int j = 0; j < kP; ++j) {
                 const double x0 = widen_here(elem_lo<kHalf>(xw[j][t])), x1 = widen_here(elem_hi<kHalf>(xw[j][t]));
 #pragma unroll
                 for (int v = 0; v < kN; ++v) {
@@ -183,44 +187,50 @@ km_candidate_dist_kernel(KmeansParams p, int c)
     const uint16_t *keys = p.k_prompt + q.plane * kHeadDim;
     __shared__ int row_s[kDistTrials];
     if (tid < cn) row_s[tid] = perm[p.pick[(size_t)q.id * p.trials_max + l0 + tid]];
-    int i[2];
-    const uint4 *row[2];
+    int i[kDistPts];
+    const uint4 *row[kDistPts];
 #pragma unroll
-    for (int j = 0; j < 2; ++j) {
+    for (int j = 0; j < kDistPts; ++j) {
         i[j] = blockIdx.x * kSumBlock + j * kDistThreads + tid;
         row[j] = reinterpret_cast<const uint4 *>(keys + (size_t)perm[min(i[j], q.n_init - 1)] * kHeadDim);
     }
     __syncthreads();
     {
-        // the candidates' rows as doubles: a thread widens one packed word (two values) of every row
-        uint32_t yw[kDistTrials];
+        // the candidates' rows as doubles: a thread widens one packed word (two values) of every
+        // kGroups-th row
+        constexpr int kGroups = kDistThreads / 64, kMine = (kDistTrials + kGroups - 1) / kGroups;
+        const int wi = tid & 63, v0 = tid >> 6;
+        uint32_t yw[kMine];
 #pragma unroll
-        for (int v = 0; v < kDistTrials; ++v)
-            yw[v] = v < cn ? reinterpret_cast<const uint32_t *>(keys + (size_t)row_s[v] * kHeadDim)[tid] : 0u;
+        for (int m = 0; m < kMine; ++m) {
+            const int v = v0 + m * kGroups;
+            yw[m] = v < cn ? reinterpret_cast<const uint32_t *>(keys + (size_t)row_s[v] * kHeadDim)[wi] : 0u;
+        }
 #pragma unroll
-        for (int v = 0; v < kDistTrials; ++v) {
+        for (int m = 0; m < kMine; ++m) {
+            const int v = v0 + m * kGroups;
             if (v < cn) {
-                y_s[v][2 * tid] = (double)elem_lo<kHalf>(yw[v]);
-                y_s[v][2 * tid + 1] = (double)elem_hi<kHalf>(yw[v]);
+                y_s[v][2 * wi] = (double)elem_lo<kHalf>(yw[m]);
+                y_s[v][2 * wi + 1] = (double)elem_hi<kHalf>(yw[m]);
             }
         }
     }
     __syncthreads();
-    double d[2][kDistTrials];
+    double d[kDistPts][kDistTrials];
 #pragma unroll
-    for (int j = 0; j < 2; ++j)
+    for (int j = 0; j < kDistPts; ++j)
 #pragma unroll
         for (int v = 0; v < kDistTrials; ++v) d[j][v] = 0.0;
     switch (cn) {
-    case 1: dist_two_points<kHalf, 1>(row[0], row[1], y_s, d); break;
-    case 2: dist_two_points<kHalf, 2>(row[0], row[1], y_s, d); break;
-    case 3: dist_two_points<kHalf, 3>(row[0], row[1], y_s, d); break;
-    case 4: dist_two_points<kHalf, 4>(row[0], row[1], y_s, d); break;
-    case 5: dist_two_points<kHalf, 5>(row[0], row[1], y_s, d); break;
-    default: dist_two_points<kHalf, 6>(row[0], row[1], y_s, d); break;
+    case 1: dist_points<kHalf, kDistPts, 1, kDistTrials>(row, y_s, d); break;
+    case 2: dist_points<kHalf, kDistPts, 2, kDistTrials>(row, y_s, d); break;
+    case 3: dist_points<kHalf, kDistPts, 3, kDistTrials>(row, y_s, d); break;
+    case 4: dist_points<kHalf, kDistPts, 4, kDistTrials>(row, y_s, d); break;
+    case 5: dist_points<kHalf, kDistPts, 5, kDistTrials>(row, y_s, d); break;
+    default: dist_points<kHalf, kDistPts, 6, kDistTrials>(row, y_s, d); break;
     }
 #pragma unroll
-    for (int j = 0; j < 2; ++j) {
+    for (int j = 0; j < kDistPts; ++j) {
 #pragma unroll
         for (int v = 0; v < kDistTrials; ++v) {
             if (v >= cn) continue;
@@ -377,12 +387,12 @@ __device__ __forceinline__ bool pair_active(const KmeansParams &p, const Pair &q
 }
 
 // Draw the minibatch and assign each point to its nearest centre (ties to the smaller index). A thread
-// holds two points and takes four centres at a time: a centre value read from shared memory serves
-// two sums and a point value is widened once for four, so that neither the shared-memory path nor
-// the conversions hold up the fp64 pipe; every sum still adds its 128 terms in order.
+// holds two points and takes eight centres at a time (dist_points); every sum still adds its 128
+// terms in order.
 constexpr int kAssignPts = 2;             // points per thread
-
 constexpr int kAssignBlock = 128 * kAssignPts;
+constexpr int kAssignGroup = 8;           // centres per pass
+static_assert(kTile % kAssignGroup == 0, "a tile of centres is a whole number of passes");
 template <bool kHalf>
 __global__ void __launch_bounds__(128)
 km_batch_assign_kernel(KmeansParams p, int t)
@@ -392,22 +402,17 @@ km_batch_assign_kernel(KmeansParams p, int t)
     if (!pair_active(p, q, t)) return;
     const int tid = threadIdx.x;
     int s[kAssignPts], idx[kAssignPts];
-    uint32_t kw[kAssignPts][64];
+    const uint4 *row[kAssignPts];
+    double best[kAssignPts];
+    int arg[kAssignPts];
 #pragma unroll
     for (int j = 0; j < kAssignPts; ++j) {
         s[j] = blockIdx.x * kAssignBlock + j * 128 + tid;
         idx[j] = km_index(km_word(p, (uint32_t)(s[j] < p.batch ? s[j] : 0), kTagBatch, q.stream, (uint32_t)t), q.N);
-        const uint4 *row = reinterpret_cast<const uint4 *>(p.k_prompt + (q.plane + (size_t)idx[j]) * kHeadDim);
-#pragma unroll
-        for (int v = 0; v < 16; ++v) {
-            const uint4 w = row[v];
-            kw[j][4 * v] = w.x; kw[j][4 * v + 1] = w.y; kw[j][4 * v + 2] = w.z; kw[j][4 * v + 3] = w.w;
-        }
+        row[j] = reinterpret_cast<const uint4 *>(p.k_prompt + (q.plane + (size_t)idx[j]) * kHeadDim);
+        best[j] = INFINITY;
+        arg[j] = 0;
     }
-    double best[kAssignPts];
-    int arg[kAssignPts];
-#pragma unroll
-    for (int j = 0; j < kAssignPts; ++j) { best[j] = INFINITY; arg[j] = 0; }
     const double *cen = p.centres64 + q.cplane * kHeadDim;
     // this block searches one slice of the centres (a multiple of kTile each); the slices' results are
     // compared in slice order afterwards, so ties still go to the smaller centre index
@@ -419,37 +424,18 @@ km_batch_assign_kernel(KmeansParams p, int t)
         __syncthreads();
         for (int e = tid; e < nt * kHeadDim; e += 128) c[e >> 7][e & 127] = cen[(size_t)base * kHeadDim + e];
         __syncthreads();
-        for (int u = 0; u < nt; u += 4) {
-            const double *cu[4] = {c[u], c[min(u + 1, nt - 1)], c[min(u + 2, nt - 1)], c[min(u + 3, nt - 1)]};
-            double d[kAssignPts][4];
+        for (int u = 0; u < nt; u += kAssignGroup) {
+            // (rows of the tile past nt hold older values; their sums are not looked at)
+            double d[kAssignPts][kAssignGroup];
 #pragma unroll
             for (int j = 0; j < kAssignPts; ++j)
 #pragma unroll
-                for (int v = 0; v < 4; ++v) d[j][v] = 0.0;
-#pragma unroll
-            for (int w = 0; w < 64; ++w) {
-                double2 y[4];
-#pragma unroll
-                for (int v = 0; v < 4; ++v) y[v] = *reinterpret_cast<const double2 *>(cu[v] + 2 * w);
-#pragma unroll
-                for (int j = 0; j < kAssignPts; ++j) {
-                    const double x0 = widen_here(elem_lo<kHalf>(kw[j][w])), x1 = widen_here(elem_hi<kHalf>(kw[j][w]));
-#pragma unroll
-                    for (int v = 0; v < 4; ++v) {
-                        const double e = __dsub_rn(x0, y[v].x);
-                        d[j][v] = __dadd_rn(d[j][v], __dmul_rn(e, e));
-                    }
-#pragma unroll
-                    for (int v = 0; v < 4; ++v) {
-                        const double e = __dsub_rn(x1, y[v].y);
-                        d[j][v] = __dadd_rn(d[j][v], __dmul_rn(e, e));
-                    }
-                }
-            }
+                for (int v = 0; v < kAssignGroup; ++v) d[j][v] = 0.0;
+            dist_points<kHalf, kAssignPts, kAssignGroup, kAssignGroup>(row, c + u, d);
 #pragma unroll
             for (int j = 0; j < kAssignPts; ++j)
 #pragma unroll
-                for (int v = 0; v < 4; ++v)
+                for (int v = 0; v < kAssignGroup; ++v)
                     if (u + v < nt && d[j][v] < best[j]) { best[j] = d[j][v]; arg[j] = base + u + v; }
         }
     }
@@ -552,26 +538,45 @@ km_batch_update_kernel(KmeansParams p, int t)
     }
 }
 
-// One warp per pair: reassignment of starved centres, averaged inertia, stopping rule.
+// One block per pair: reassignment of starved centres, averaged inertia, stopping rule. The serial
+// parts (the inertia is the sum of the minibatch distances in order) run on one thread over shared
+// memory that all threads filled.
 template <bool kHalf>
-__global__ void __launch_bounds__(32)
+__global__ void __launch_bounds__(kThreads)
 km_control_kernel(KmeansParams p, int t)
 {
-    extern __shared__ int32_t ctl_tab[];                    // slots[batch], move_centre[batch / 2]
+    extern __shared__ double ctl_dist[];                    // dist[batch], then int32 slots[batch], move_centre[batch / 2]
     __shared__ int n_move_s;
+    __shared__ double cmin_s[kThreads / 32], cmax_s[kThreads / 32];
     const Pair q = pair_of(p, blockIdx.x, blockIdx.y);
     if (!pair_active(p, q, t)) return;
-    const int lane = threadIdx.x;
-    int32_t *slots = ctl_tab, *move_centre = ctl_tab + p.batch;
+    const int tid = threadIdx.x;
+    int32_t *slots = reinterpret_cast<int32_t *>(ctl_dist + p.batch), *move_centre = slots + p.batch;
     double *count = p.count + q.cplane;
     const int32_t *idx = p.idx + (size_t)q.id * p.batch;
-    if (lane == 0) {
-        int n_move = 0;
-        double cmin = INFINITY, cmax = 0.0;
-        for (int u = 0; u < q.k; ++u) {
+    {
+        const double *dist = p.dist + (size_t)q.id * p.batch;
+        for (int s = tid; s < p.batch; s += kThreads) ctl_dist[s] = dist[s];
+        double cmin = INFINITY, cmax = 0.0;                 // smallest and largest count: any order gives the same
+        for (int u = tid; u < q.k; u += kThreads) {
             const double v = count[u];
             if (v < cmin) cmin = v;
             if (v > cmax) cmax = v;
+        }
+        for (int o = 16; o > 0; o >>= 1) {
+            const double a = __shfl_xor_sync(0xffffffffu, cmin, o), b = __shfl_xor_sync(0xffffffffu, cmax, o);
+            if (a < cmin) cmin = a;
+            if (b > cmax) cmax = b;
+        }
+        if ((tid & 31) == 0) { cmin_s[tid >> 5] = cmin; cmax_s[tid >> 5] = cmax; }
+    }
+    __syncthreads();
+    if (tid == 0) {
+        int n_move = 0;
+        double cmin = INFINITY, cmax = 0.0;
+        for (int w = 0; w < kThreads / 32; ++w) {
+            if (cmin_s[w] < cmin) cmin = cmin_s[w];
+            if (cmax_s[w] > cmax) cmax = cmax_s[w];
         }
         const long long period = 10 + (long long)floor(cmin);
         if (p.ratio > 0.0 && ((long long)t + 1) % period == 0) {
@@ -596,18 +601,17 @@ km_control_kernel(KmeansParams p, int t)
         }
         n_move_s = n_move;
     }
-    __syncwarp();
+    __syncthreads();
     const int n_move = n_move_s;
-    for (int i = 0; i < n_move; ++i) {                      // the moved centres jump onto minibatch points
+    for (int e = tid; e < n_move * kHeadDim; e += kThreads) {   // the moved centres jump onto minibatch points
+        const int i = e >> 7, d = e & (kHeadDim - 1);
         const uint16_t *src = p.k_prompt + (q.plane + (size_t)idx[slots[i]]) * kHeadDim;
-        double *dst = p.centres64 + (q.cplane + (size_t)move_centre[i]) * kHeadDim;
-        for (int d = lane; d < kHeadDim; d += 32) dst[d] = elem_to_double<kHalf>(src[d]);
+        p.centres64[(q.cplane + (size_t)move_centre[i]) * kHeadDim + d] = elem_to_double<kHalf>(src[d]);
     }
-    if (lane == 0) {
-        const double *dist = p.dist + (size_t)q.id * p.batch;
+    if (tid == 0) {
         double inertia = 0.0;
 #pragma unroll 8
-        for (int s = 0; s < p.batch; ++s) inertia = __dadd_rn(inertia, dist[s]);
+        for (int s = 0; s < p.batch; ++s) inertia = __dadd_rn(inertia, ctl_dist[s]);
         KmeansState &st = p.state[q.id];
         double alpha = __ddiv_rn(__dmul_rn(2.0, (double)p.batch), __dadd_rn((double)q.N, 1.0));
         if (alpha > 1.0) alpha = 1.0;
@@ -671,7 +675,9 @@ cudaError_t run_fit(const KmeansParams &p, cudaStream_t s)
     }
     if ((err = cudaMemsetAsync(p.count, 0, sizeof(double) * (size_t)H * p.centres_total, s)) != cudaSuccess) return err;
     if ((err = cudaMemsetAsync(p.state, 0, sizeof(KmeansState) * (size_t)pairs, s)) != cudaSuccess) return err;
-    const size_t control_smem = sizeof(int32_t) * ((size_t)p.batch + (size_t)p.batch / 2 + 1);
+    const size_t control_smem = sizeof(double) * (size_t)p.batch + sizeof(int32_t) * ((size_t)p.batch + (size_t)p.batch / 2 + 1);
+    if ((err = cudaFuncSetAttribute(km_control_kernel<kHalf>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)control_smem)) != cudaSuccess)
+        return err;
     for (int t = 0; t < p.t_max_max; ++t) {
         km_batch_assign_kernel<kHalf><<<dim3((p.batch + kAssignBlock - 1) / kAssignBlock, pairs, p.assign_split), 128, 0, s>>>(p, t);
         KM_CHECK();
@@ -683,7 +689,7 @@ cudaError_t run_fit(const KmeansParams &p, cudaStream_t s)
         KM_CHECK();
         km_batch_update_kernel<kHalf><<<dim3((p.k_max + 1) / 2, pairs), kThreads, 0, s>>>(p, t);
         KM_CHECK();
-        km_control_kernel<kHalf><<<dim3(B, H), 32, control_smem, s>>>(p, t);
+        km_control_kernel<kHalf><<<dim3(B, H), kThreads, control_smem, s>>>(p, t);
         KM_CHECK();
         if (!p.no_host_poll && (t + 1) % kPollEvery == 0 && t + 1 < p.t_max_max) {
             // most fits stop long before the step limit: ask the device how many are still running
