@@ -23,33 +23,34 @@ __device__ __forceinline__ int clamp_label(int v, int n) { return min(max(v, 0),
 
 // ---- Algorithm 3, assignment step: b_i = argmin_u |k_i - mu_u|^2, ties to the smaller u ----
 constexpr int kAssignThreads = 128;
+constexpr int kAssignPts = 2;             // tokens per thread
+constexpr int kAssignGroup = 8;           // centres per pass
 constexpr int kCentreTile = 16;
+static_assert(kCentreTile % kAssignGroup == 0, "a tile of centres is a whole number of passes");
 
+// A thread holds two tokens and takes eight centres at a time (dist_points: a centre value read from
+// shared memory serves both tokens, a token value is widened once for the eight centres).
 template <bool kHalf>
 __global__ void __launch_bounds__(kAssignThreads)
 assign_parents_kernel(AssignParams p)
 {
-    __shared__ double c[kCentreTile][kHeadDim];
+    __shared__ __align__(16) double c[kCentreTile][kHeadDim];
     const int b = blockIdx.y, j = blockIdx.z, tid = threadIdx.x;
     const int64_t row0 = p.seq_row_off[b];
     const int N = (int)(p.seq_row_off[b + 1] - row0);
-    if ((int)(blockIdx.x * kAssignThreads) >= N) return;
-    const int i = blockIdx.x * kAssignThreads + tid;
-    const bool valid = i < N;
+    if ((int)(blockIdx.x * kAssignThreads * kAssignPts) >= N) return;
     const int64_t c0off = p.seq_centre_off[b];
     const int n_centres = (int)(p.seq_centre_off[b + 1] - c0off);
-
-    uint32_t kw[64];
-    {
-        const uint4 *row = reinterpret_cast<const uint4 *>(p.k_prompt + ((size_t)j * p.rows_total + row0 + (valid ? i : 0)) * kHeadDim);
+    int i[kAssignPts], arg[kAssignPts];
+    const uint4 *row[kAssignPts];
+    double best[kAssignPts];
 #pragma unroll
-        for (int q = 0; q < 16; ++q) {
-            const uint4 w = row[q];
-            kw[4 * q] = w.x; kw[4 * q + 1] = w.y; kw[4 * q + 2] = w.z; kw[4 * q + 3] = w.w;
-        }
+    for (int u = 0; u < kAssignPts; ++u) {
+        i[u] = (blockIdx.x * kAssignPts + u) * kAssignThreads + tid;
+        row[u] = reinterpret_cast<const uint4 *>(p.k_prompt + ((size_t)j * p.rows_total + row0 + min(i[u], N - 1)) * kHeadDim);
+        best[u] = INFINITY;
+        arg[u] = 0;
     }
-    double best = INFINITY;
-    int arg = 0;
     const float *cen = p.centres + ((size_t)j * p.centres_total + c0off) * kHeadDim;
     for (int base = 0; base < n_centres; base += kCentreTile) {
         const int nt = min(kCentreTile, n_centres - base);
@@ -57,19 +58,24 @@ assign_parents_kernel(AssignParams p)
         for (int e = tid; e < nt * kHeadDim; e += kAssignThreads)
             c[e >> 7][e & 127] = (double)cen[(size_t)base * kHeadDim + e];
         __syncthreads();
-        for (int t = 0; t < nt; ++t) {
-            double s = 0.0;
+        for (int t = 0; t < nt; t += kAssignGroup) {
+            // (rows of the tile past nt hold older values; their sums are not looked at)
+            double s[kAssignPts][kAssignGroup];
 #pragma unroll
-            for (int w = 0; w < 64; ++w) {
-                const double e0 = __dsub_rn((double)elem_lo<kHalf>(kw[w]), c[t][2 * w]);
-                const double e1 = __dsub_rn((double)elem_hi<kHalf>(kw[w]), c[t][2 * w + 1]);
-                s = __dadd_rn(s, __dmul_rn(e0, e0));
-                s = __dadd_rn(s, __dmul_rn(e1, e1));
-            }
-            if (s < best) { best = s; arg = base + t; }
+            for (int u = 0; u < kAssignPts; ++u)
+#pragma unroll
+                for (int v = 0; v < kAssignGroup; ++v) s[u][v] = 0.0;
+            dist_points<kHalf, kAssignPts, kAssignGroup, kAssignGroup>(row, c + t, s);
+#pragma unroll
+            for (int u = 0; u < kAssignPts; ++u)
+#pragma unroll
+                for (int v = 0; v < kAssignGroup; ++v)
+                    if (t + v < nt && s[u][v] < best[u]) { best[u] = s[u][v]; arg[u] = base + t + v; }
         }
     }
-    if (valid) p.parent_of[(size_t)j * p.rows_total + row0 + i] = arg;
+#pragma unroll
+    for (int u = 0; u < kAssignPts; ++u)
+        if (i[u] < N) p.parent_of[(size_t)j * p.rows_total + row0 + i[u]] = arg[u];
 }
 
 // ---- token counts per label ----
@@ -350,7 +356,7 @@ pack_rows_kernel(ParentBuildParams p)
 
 cudaError_t launch_assign_parents(const AssignParams &p, cudaStream_t s)
 {
-    dim3 grid((p.max_rows_per_seq + kAssignThreads - 1) / kAssignThreads, p.n_seqs, p.n_kv);
+    dim3 grid((p.max_rows_per_seq + kAssignThreads * kAssignPts - 1) / (kAssignThreads * kAssignPts), p.n_seqs, p.n_kv);
     if (p.elem) assign_parents_kernel<true><<<grid, kAssignThreads, 0, s>>>(p);
     else        assign_parents_kernel<false><<<grid, kAssignThreads, 0, s>>>(p);
     return cudaGetLastError();

@@ -342,6 +342,58 @@ __device__ __forceinline__ float elem_hi(uint32_t w)
     if constexpr (kHalf) return __half2float(__ushort_as_half((unsigned short)(w >> 16)));
     else return bf16_hi(w);
 }
+
+// fp32 -> fp64 where it is written (the compiler would otherwise widen all of a point's values ahead of
+// a loop over centres and keep them in local memory)
+__device__ __forceinline__ double widen_here(float x)
+{
+    double r;
+    asm volatile("cvt.f64.f32 %0, %1;" : "=d"(r) : "f"(x));
+    return r;
+}
+
+// Squared distances (fp64, the 128 terms added in order) of kP points (rows of packed words in global
+// memory, read eight values at a time, one read ahead) to kN candidate points held as doubles in
+// shared memory: a candidate value serves all kP points and a point value is widened once for all
+// candidates (widening runs at a quarter of the fp64 add rate). The loop is kept rolled: a warp runs
+// it once, and a body unrolled over the whole row is fetched from instruction memory slower than it runs.
+template <bool kHalf, int kP, int kN, int kD>
+__device__ __forceinline__ void dist_points(const uint4 *const (&row)[kP], const double (*y_s)[kHeadDim], double (&d)[kP][kD])
+{
+    uint4 nxt[kP];
+#pragma unroll
+    for (int j = 0; j < kP; ++j) nxt[j] = row[j][0];
+#pragma unroll 1
+    for (int qd = 0; qd < 16; ++qd) {
+        uint32_t xw[kP][4];
+#pragma unroll
+        for (int j = 0; j < kP; ++j) {
+            xw[j][0] = nxt[j].x; xw[j][1] = nxt[j].y; xw[j][2] = nxt[j].z; xw[j][3] = nxt[j].w;
+            if (qd + 1 < 16) nxt[j] = row[j][qd + 1];
+        }
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+            double2 y[kN];
+#pragma unroll
+            for (int v = 0; v < kN; ++v) y[v] = *reinterpret_cast<const double2 *>(&y_s[v][8 * qd + 2 * t]);
+#pragma unroll
+            for (int j = 0; j < kP; ++j) {
+                const double x0 = widen_here(elem_lo<kHalf>(xw[j][t])), x1 = widen_here(elem_hi<kHalf>(xw[j][t]));
+#pragma unroll
+                for (int v = 0; v < kN; ++v) {
+                    const double e = __dsub_rn(x0, y[v].x);
+                    d[j][v] = __dadd_rn(d[j][v], __dmul_rn(e, e));
+                }
+#pragma unroll
+                for (int v = 0; v < kN; ++v) {
+                    const double e = __dsub_rn(x1, y[v].y);
+                    d[j][v] = __dadd_rn(d[j][v], __dmul_rn(e, e));
+                }
+            }
+        }
+    }
+}
+
 template <bool kHalf>
 __device__ __forceinline__ double elem_to_double(uint16_t b) { return (double)elem_to_float<kHalf>(b); }
 // fp64 -> fp32 (to nearest) -> the 16-bit element type (to nearest even): how a computed routing key is stored.

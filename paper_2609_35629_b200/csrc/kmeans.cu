@@ -111,61 +111,10 @@ km_sample_kernel(KmeansParams p)
 // ---- 2. greedy k-means++ on the sample ----
 constexpr int kSumBlock = 128;           // sums over the initialisation sample are taken in blocks of this many points
 constexpr int kMaxSumBlocks = 224;       // an initialisation sample holds at most 28544 points (223 blocks)
-// fp32 -> fp64 where it is written (the compiler would otherwise widen all of a point's values ahead of
-// a loop over centres and keep them in local memory)
-__device__ __forceinline__ double widen_here(float x)
-{
-    double r;
-    asm volatile("cvt.f64.f32 %0, %1;" : "=d"(r) : "f"(x));
-    return r;
-}
-
 constexpr int kDistPts = 1;              // points per thread
 constexpr int kDistThreads = kSumBlock / kDistPts;   // a block covers one block of the sums
 static_assert(kDistThreads % 64 == 0, "64 threads widen one candidate row");
 constexpr int kDistTrials = 6;           // candidate points per block
-
-// Squared distances (fp64, the 128 terms added in order) of kP points (rows of packed words in global
-// memory, read eight values at a time, one read ahead) to kN candidate points held as doubles in
-// shared memory: a candidate value serves all kP points and a point value is widened once for all
-// candidates (widening runs at a quarter of the fp64 add rate). The loop is kept rolled: a warp runs
-// it once, and a body unrolled over the whole row is fetched from instruction memory slower than it runs.
-template <bool kHalf, int kP, int kN, int kD>
-__device__ __forceinline__ void dist_points(const uint4 *const (&row)[kP], const double (*y_s)[kHeadDim], double (&d)[kP][kD])
-{
-    uint4 nxt[kP];
-#pragma unroll
-    for (int j = 0; j < kP; ++j) nxt[j] = row[j][0];
-#pragma unroll 1
-    for (int qd = 0; qd < 16; ++qd) {
-        uint32_t xw[kP][4];
-#pragma unroll
-        for (int j = 0; j < kP; ++j) {
-            xw[j][0] = nxt[j].x; xw[j][1] = nxt[j].y; xw[j][2] = nxt[j].z; xw[j][3] = nxt[j].w;
-            if (qd + 1 < 16) nxt[j] = row[j][qd + 1];
-        }
-#pragma unroll
-        for (int t = 0; t < 4; ++t) {
-            double2 y[kN];
-#pragma unroll
-            for (int v = 0; v < kN; ++v) y[v] = *reinterpret_cast<const double2 *>(&y_s[v][8 * qd + 2 * t]);
-#pragma unroll
-            for (int j = 0; j < kP; ++j) {
-                const double x0 = widen_here(elem_lo<kHalf>(xw[j][t])), x1 = widen_here(elem_hi<kHalf>(xw[j][t]));
-#pragma unroll
-                for (int v = 0; v < kN; ++v) {
-                    const double e = __dsub_rn(x0, y[v].x);
-                    d[j][v] = __dadd_rn(d[j][v], __dmul_rn(e, e));
-                }
-#pragma unroll
-                for (int v = 0; v < kN; ++v) {
-                    const double e = __dsub_rn(x1, y[v].y);
-                    d[j][v] = __dadd_rn(d[j][v], __dmul_rn(e, e));
-                }
-            }
-        }
-    }
-}
 
 // Distances of every sample point to the candidate points pick[0..n_cand): cand[l][i]; and, for c > 0,
 // the sums of min(closest_i, cand[l][i]) over each block of kSumBlock consecutive sample points, added
