@@ -329,23 +329,31 @@ def measure_workload(args, workload, n_layers, n_steps, n_warmup, dev, want_e2e,
             q_all[s, l] = synth.make_queries(spec, data, s)
         k_prompt = sp.bf16_bits_to_cuda(data.k_prompt, dev, edt)
         v_prompt = sp.bf16_bits_to_cuda(data.v_prompt, dev, edt)
-        if by_centres:
+        def build_records():
+            if not by_centres:
+                return sp.santapp_build_teams(geom, spec.prompt_len, k_prompt, v_prompt)
             # Algorithm 3: as many centres as its first line asks for; "kmeans" fits them with the paper's
             # settings, "centres" takes the fit's ideal outcome on these keys (the centres the rows
             # were drawn around)
             n_cen = [sp.santapp_kmeans_parent_count(n, spec.parent_size) for n in spec.prompt_len]
-            t_build = time.perf_counter()
             if spec.parents == "kmeans":
-                cen_dev, fit_steps = sp.santapp_kmeans_fit(geom, spec.prompt_len, n_cen, k_prompt)
+                cen_dev, _ = sp.santapp_kmeans_fit(geom, spec.prompt_len, n_cen, k_prompt)
             else:
                 n_cen = [min(n, spec.n_clusters) for n in n_cen]
                 cen = np.concatenate([data.centres[:, :n] for n in n_cen], axis=1)
                 cen_dev = torch.from_numpy(np.ascontiguousarray(cen)).to(dev)
             parent_of = sp.santapp_assign_parents(geom, spec.prompt_len, n_cen, k_prompt, cen_dev)
-            teams = sp.santapp_build_teams_parents(geom, spec.prompt_len, n_cen, k_prompt, v_prompt, parent_of)
-        else:
-            t_build = time.perf_counter()
-            teams = sp.santapp_build_teams(geom, spec.prompt_len, k_prompt, v_prompt)
+            return sp.santapp_build_teams_parents(geom, spec.prompt_len, n_cen, k_prompt, v_prompt, parent_of)
+
+        if l == L - 1:
+            # the timed build is a second one, whose buffers come out of torch's cache: a first
+            # build's wall clock is mostly that of fresh device allocations, which vary from run to run
+            teams = build_records()
+            torch.cuda.synchronize()
+            del teams
+        torch.cuda.synchronize()                            # the copies above are not part of the build
+        t_build = time.perf_counter()
+        teams = build_records()
         torch.cuda.synchronize()
         build_ms = 1e3 * (time.perf_counter() - t_build)
         del k_prompt, v_prompt
@@ -623,6 +631,13 @@ def measure_latent(args, n_layers, n_steps, n_warmup, dev, n_seqs=32, n_sample=1
         for s in range(S):
             q_all[s, l] = synth.make_latent_queries(spec, data, s)
         rows = sp.bf16_bits_to_cuda(data.rows, dev)
+        if l == L - 1:
+            # the timed build is a second one, whose buffers come out of torch's cache: the first
+            # build's time is mostly that of fresh device allocations (3 to 190 ms from run to run)
+            teams = sp.santapp_latent_build_teams(geom, spec.prompt_len, rows)
+            torch.cuda.synchronize()
+            del teams
+        torch.cuda.synchronize()
         t0 = time.perf_counter()
         teams = sp.santapp_latent_build_teams(geom, spec.prompt_len, rows)
         torch.cuda.synchronize()
@@ -775,7 +790,7 @@ def kmeans_group_records(spec, data, dev):
         geom = sp.Geometry(1, spec.n_q_heads, spec.n_kv_heads, spec.head_dim, size, 1,
                            sp.SANTAPP_FP16 if half else sp.SANTAPP_BF16)
         n_cen = [sp.santapp_kmeans_parent_count(N, size)]
-        if 3 * max(4096, n_cen[0]) > 28672:                        # the fit's limit on its initialisation sample
+        if 3 * max(4096, n_cen[0]) > 28544:                        # the fit's limit on its initialisation sample
             continue
         centres, _ = sp.santapp_kmeans_fit(geom, [N], n_cen, k)
         labels = sp.santapp_assign_parents(geom, [N], n_cen, k, centres)
