@@ -383,6 +383,8 @@ struct LatentPlanParams {
 
 constexpr int kLpThreads = 512;
 constexpr int kLatSegMax = kHeads * 128 + 1;                // 16 heads x K <= 128 teams, + the suffix
+constexpr int kLpPerThread = kHeads * 128 / kLpThreads;     // sampled teams of a sequence per thread
+static_assert(kLpPerThread * kLpThreads == kHeads * 128, "a block holds a sequence's samples in registers");
 
 struct LatentPlanSmem {
     uint32_t bitmap[kMaxTeamsPerSeq / 32];
@@ -427,12 +429,26 @@ latent_plan_kernel(LatentPlanParams p)
     }
 
     const int n_words = (M + 31) / 32, E = H * K;
+    // a thread's share of the samples (at most kLpPerThread entries), all requested at once
+    int my_team[kLpPerThread];
+    int2 my_rows[kLpPerThread];
+    float my_logc[kLpPerThread];
+#pragma unroll
+    for (int u = 0; u < kLpPerThread; ++u) {
+        const int e = tid + u * kLpThreads;
+        my_team[u] = -1;
+        if (e < E) {
+            my_team[u] = __ldcg(p.sel_team + head0 * K + e);
+            my_rows[u] = __ldcg(p.sel_rows + head0 * K + e);
+            my_logc[u] = __ldcg(p.sel_logc + head0 * K + e);
+            if (my_team[u] >= M) my_team[u] = -1;                              // cannot come from the sampler
+        }
+    }
     for (int i = tid; i < n_words; i += kLpThreads) sm.bitmap[i] = 0u;
     __syncthreads();
-    for (int e = tid; e < E; e += kLpThreads) {
-        const int team = __ldcg(p.sel_team + head0 * K + e);
-        if (team >= 0 && team < M) atomicOr(&sm.bitmap[team >> 5], 1u << (team & 31));
-    }
+#pragma unroll
+    for (int u = 0; u < kLpPerThread; ++u)
+        if (my_team[u] >= 0) atomicOr(&sm.bitmap[my_team[u] >> 5], 1u << (my_team[u] & 31));
     __syncthreads();
     int nseg;
     {
@@ -446,14 +462,14 @@ latent_plan_kernel(LatentPlanParams p)
     for (int i = tid; i < nseg * kHeads; i += kLpThreads) bias[i] = -CUDART_INF_F;
     if (tid < kHeads) bias[(size_t)nseg * kHeads + tid] = 0.f;              // the suffix segment
     __syncthreads();
-    for (int e = tid; e < E; e += kLpThreads) {
-        const int team = __ldcg(p.sel_team + head0 * K + e);
-        if (team < 0 || team >= M) continue;                                   // cannot come from the sampler
+#pragma unroll
+    for (int u = 0; u < kLpPerThread; ++u) {
+        const int team = my_team[u], e = tid + u * kLpThreads;
+        if (team < 0) continue;
         const int seg = sm.wprefix[team >> 5] + __popc(sm.bitmap[team >> 5] & ((1u << (team & 31)) - 1u));
-        const int2 rows = __ldcg(p.sel_rows + head0 * K + e);
-        bias[(size_t)seg * kHeads + e / K] = -kLog2e * __ldcg(p.sel_logc + head0 * K + e);   // weight e^s / c_g
-        sm.seg_start[seg] = rows.x;                                            // the same from every selecting head
-        sm.seg_n[seg] = rows.y;
+        bias[(size_t)seg * kHeads + e / K] = -kLog2e * my_logc[u];             // weight e^s / c_g
+        sm.seg_start[seg] = my_rows[u].x;                                      // the same from every selecting head
+        sm.seg_n[seg] = my_rows[u].y;
     }
     __syncthreads();
     int total;
