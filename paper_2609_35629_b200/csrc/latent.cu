@@ -253,7 +253,7 @@ struct LatentScoreParams {
     const uint16_t *q;              // [n_seqs][n_heads][576]
     float *y32;                     // [n_heads][n_seqs][y_stride]
     int64_t y_stride;
-    int n_sample;
+    int n_sample, tiles_per_warp;
     uint32_t seed_lo, seed_hi, step, stream_base;
     const uint32_t *step_dev;
     float scale;
@@ -269,11 +269,13 @@ __device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-// Grid (ceil(max teams / 128), sequences); a warp scores 16 teams for all heads: the teams are the
-// MMA's 16 rows, the heads its columns (two tiles of 8), the 576 values 36 k-steps. Both operands
-// use the same permutation of the contraction index inside every block of 32 values, so a lane
-// feeds the tensor core 16-byte pieces of a representative row (and of a query) as they lie in
-// memory: piece t of the block supplies k-slots {2t, 2t+1, 2t+8, 2t+9} of the block's two MMAs.
+// Grid (ceil(max teams / (128 tiles_per_warp)), sequences); a warp scores tiles_per_warp consecutive
+// tiles of 16 teams for all heads: the teams are the MMA's 16 rows, the heads its columns (two tiles
+// of 8), the 576 values 36 k-steps. Both operands use the same permutation of the contraction index
+// inside every block of 32 values, so a lane feeds the tensor core 16-byte pieces of a
+// representative row (and of a query) as they lie in memory: piece t of the block supplies k-slots
+// {2t, 2t+1, 2t+8, 2t+9} of the block's two MMAs. The host picks tiles_per_warp so that all blocks
+// are resident at once (two per SM): a second, partly filled wave of blocks costs as much as a full one.
 __global__ void __launch_bounds__(kLsThreads)
 latent_score_kernel(LatentScoreParams p)
 {
@@ -283,67 +285,102 @@ latent_score_kernel(LatentScoreParams p)
     const int b = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int64_t team0 = p.lv.seq_team_off[b];
     const int M = (int)(p.lv.seq_team_off[b + 1] - team0);
-    if (p.n_sample >= M || (int)blockIdx.x * kLsTeamsPerBlock >= M) return;      // nothing is drawn / no team here
+    const int tpw = p.tiles_per_warp;
+    if (p.n_sample >= M || (int)blockIdx.x * kLsTeamsPerBlock * tpw >= M) return;    // nothing is drawn / no team here
     const int H = p.lv.n_heads;
-    const uint4 *qg = reinterpret_cast<const uint4 *>(p.q + (size_t)b * H * kRowDim);
-    for (int e = tid; e < kHeads * kRowChunks; e += kLsThreads) {
-        const int h = e / kRowChunks, c = e - h * kRowChunks;
-        const uint4 v = h < H ? __ldg(qg + (size_t)h * kRowChunks + c) : make_uint4(0u, 0u, 0u, 0u);
-        *reinterpret_cast<uint4 *>(q_s + h * kQPitchW + c * 4) = v;
+    // the warp's first pieces of its representatives' rows are requested before anything else: they
+    // do not depend on the queries, and the block's set-up (queries into shared memory) runs while
+    // they are on their way
+    constexpr int kBatch = 6;                                       // blocks of 32 values requested together
+    const int t_first = ((int)blockIdx.x * (kLsThreads / 32) + warp) * tpw * 16;
+    const bool live = t_first < M;
+    const int r = lane >> 2, t = lane & 3;
+    const uint16_t *rep = p.rep_rows + (size_t)team0 * kRowDim;
+    auto row_ptr = [&](int team) { return reinterpret_cast<const uint4 *>(rep + (size_t)min(team, M - 1) * kRowDim) + t; };
+    uint4 wa[kBatch], wb[kBatch];
+    if (live) {
+        const uint4 *ka = row_ptr(t_first + r), *kb = row_ptr(t_first + r + 8);
+#pragma unroll
+        for (int i = 0; i < kBatch; ++i) { wa[i] = __ldg(ka + i * 4); wb[i] = __ldg(kb + i * 4); }
+    }
+    const int32_t *csr = p.team_row_start + team0 + b;
+    const uint32_t step = p.step + (p.step_dev ? *p.step_dev : 0u);
+    {
+        const uint4 *qg = reinterpret_cast<const uint4 *>(p.q + (size_t)b * H * kRowDim);
+        constexpr int kMine = (kHeads * kRowChunks + kLsThreads - 1) / kLsThreads;
+        uint4 v[kMine];
+#pragma unroll
+        for (int u = 0; u < kMine; ++u) {                           // all of a thread's pieces in flight at once
+            const int e = tid + u * kLsThreads, h = e / kRowChunks, c = e - h * kRowChunks;
+            v[u] = (e < kHeads * kRowChunks && h < H) ? __ldg(qg + (size_t)h * kRowChunks + c) : make_uint4(0u, 0u, 0u, 0u);
+        }
+#pragma unroll
+        for (int u = 0; u < kMine; ++u) {
+            const int e = tid + u * kLsThreads, h = e / kRowChunks, c = e - h * kRowChunks;
+            if (e < kHeads * kRowChunks) *reinterpret_cast<uint4 *>(q_s + h * kQPitchW + c * 4) = v[u];
+        }
     }
     __syncthreads();
-    const int t0 = ((int)blockIdx.x * (kLsThreads / 32) + warp) * 16;
-    if (t0 >= M) return;
-    const uint32_t step = p.step + (p.step_dev ? *p.step_dev : 0u);
-    const int r = lane >> 2, t = lane & 3;
-    const int ga = t0 + r, gb = t0 + r + 8;                         // the lane's two teams (rows r and r + 8 of the tile)
-    const uint4 *ka = reinterpret_cast<const uint4 *>(p.rep_rows + (size_t)(team0 + min(ga, M - 1)) * kRowDim) + t;
-    const uint4 *kb = reinterpret_cast<const uint4 *>(p.rep_rows + (size_t)(team0 + min(gb, M - 1)) * kRowDim) + t;
-    const int32_t *csr = p.team_row_start + team0 + b;
-    const int na = ga < M ? csr[ga + 1] - csr[ga] : 1, nb = gb < M ? csr[gb + 1] - csr[gb] : 1;
+    if (!live) return;
 
-    // Philox words of the tile: lane computes the blocks of head (lane & 15) for two groups of four teams
-    {
-        const int h = lane & 15, tg = (lane >> 4) * 2;
-#pragma unroll
-        for (int u = 0; u < 2; ++u) {
-            const uint4 w = philox4x32_10(make_uint4((uint32_t)(t0 >> 2) + tg + u, step, (uint32_t)h, p.stream_base + (uint32_t)b),
-                                          p.seed_lo, p.seed_hi);
-            *reinterpret_cast<uint4 *>(&words_s[warp][h][(tg + u) * 4]) = w;
-        }
-    }
-
-    float acc[2][4] = {};
-    constexpr int kBatch = 6;                                       // blocks of 32 values requested together
 #pragma unroll 1
-    for (int blk0 = 0; blk0 < kRowDim / 32; blk0 += kBatch) {
-        uint4 wa[kBatch], wb[kBatch];
+    for (int it = 0; it < tpw; ++it) {
+        const int t0 = t_first + it * 16;
+        if (t0 >= M) break;
+        const int ga = t0 + r, gb = t0 + r + 8;                     // the lane's two teams (rows r and r + 8 of the tile)
+        const uint4 *ka = row_ptr(ga), *kb = row_ptr(gb);
+        const bool more = it + 1 < tpw && t0 + 16 < M;              // the next tile's first pieces follow this tile's last
+        const uint4 *ka_next = row_ptr(ga + 16), *kb_next = row_ptr(gb + 16);
+        int na = 1, nb = 1;
+        if (ga < M) na = csr[ga + 1] - csr[ga];
+        if (gb < M) nb = csr[gb + 1] - csr[gb];
+        // Philox words of the tile: lane computes the blocks of head (lane & 15) for two groups of four teams
+        {
+            const int h = lane & 15, tg = (lane >> 4) * 2;
 #pragma unroll
-        for (int i = 0; i < kBatch; ++i) { wa[i] = __ldg(ka + (blk0 + i) * 4); wb[i] = __ldg(kb + (blk0 + i) * 4); }
-#pragma unroll
-        for (int i = 0; i < kBatch; ++i) {
-            const int piece = (blk0 + i) * 4 + t;
-            const uint4 q0 = *reinterpret_cast<const uint4 *>(q_s + r * kQPitchW + piece * 4);
-            const uint4 q1 = *reinterpret_cast<const uint4 *>(q_s + (r + 8) * kQPitchW + piece * 4);
-            mma_bf16(acc[0], wa[i].x, wb[i].x, wa[i].y, wb[i].y, q0.x, q0.y);
-            mma_bf16(acc[0], wa[i].z, wb[i].z, wa[i].w, wb[i].w, q0.z, q0.w);
-            mma_bf16(acc[1], wa[i].x, wb[i].x, wa[i].y, wb[i].y, q1.x, q1.y);
-            mma_bf16(acc[1], wa[i].z, wb[i].z, wa[i].w, wb[i].w, q1.z, q1.w);
-        }
-    }
-    __syncwarp();
-    const float log_a = __logf((float)na), log_b = __logf((float)nb);
-#pragma unroll
-    for (int n = 0; n < 2; ++n) {
-#pragma unroll
-        for (int e = 0; e < 2; ++e) {
-            const int h = 8 * n + 2 * t + e;
-            if (h < H) {
-                float *row = p.y32 + ((size_t)h * p.lv.n_seqs + b) * p.y_stride;
-                if (ga < M) row[ga] = log_a + acc[n][e] * p.scale + gumbel32_from_word(words_s[warp][h][r]);
-                if (gb < M) row[gb] = log_b + acc[n][2 + e] * p.scale + gumbel32_from_word(words_s[warp][h][r + 8]);
+            for (int u = 0; u < 2; ++u) {
+                const uint4 w = philox4x32_10(make_uint4((uint32_t)(t0 >> 2) + tg + u, step, (uint32_t)h, p.stream_base + (uint32_t)b),
+                                              p.seed_lo, p.seed_hi);
+                *reinterpret_cast<uint4 *>(&words_s[warp][h][(tg + u) * 4]) = w;
             }
         }
+        float acc[2][4] = {};
+#pragma unroll 1
+        for (int blk0 = 0; blk0 < kRowDim / 32; blk0 += kBatch) {
+            const bool last = blk0 + kBatch >= kRowDim / 32;
+#pragma unroll
+            for (int i = 0; i < kBatch; ++i) {
+                const int piece = (blk0 + i) * 4 + t;
+                const uint4 q0 = *reinterpret_cast<const uint4 *>(q_s + r * kQPitchW + piece * 4);
+                const uint4 q1 = *reinterpret_cast<const uint4 *>(q_s + (r + 8) * kQPitchW + piece * 4);
+                mma_bf16(acc[0], wa[i].x, wb[i].x, wa[i].y, wb[i].y, q0.x, q0.y);
+                mma_bf16(acc[0], wa[i].z, wb[i].z, wa[i].w, wb[i].w, q0.z, q0.w);
+                mma_bf16(acc[1], wa[i].x, wb[i].x, wa[i].y, wb[i].y, q1.x, q1.y);
+                mma_bf16(acc[1], wa[i].z, wb[i].z, wa[i].w, wb[i].w, q1.z, q1.w);
+                if (!last) {                                        // the same piece of the next batch
+                    wa[i] = __ldg(ka + (blk0 + kBatch + i) * 4);
+                    wb[i] = __ldg(kb + (blk0 + kBatch + i) * 4);
+                } else if (more) {
+                    wa[i] = __ldg(ka_next + i * 4);
+                    wb[i] = __ldg(kb_next + i * 4);
+                }
+            }
+        }
+        __syncwarp();
+        const float log_a = __logf((float)na), log_b = __logf((float)nb);
+#pragma unroll
+        for (int n = 0; n < 2; ++n) {
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const int h = 8 * n + 2 * t + e;
+                if (h < H) {
+                    float *row = p.y32 + ((size_t)h * p.lv.n_seqs + b) * p.y_stride;
+                    if (ga < M) row[ga] = log_a + acc[n][e] * p.scale + gumbel32_from_word(words_s[warp][h][r]);
+                    if (gb < M) row[gb] = log_b + acc[n][2 + e] * p.scale + gumbel32_from_word(words_s[warp][h][r + 8]);
+                }
+            }
+        }
+        __syncwarp();                                               // the words are rewritten for the next tile
     }
 }
 
@@ -1261,7 +1298,12 @@ int santapp_latent_decode_attn(const santapp_latent_geom *geom, const santapp_la
         sp.step_dev = step_dev;
         sp.stream_base = stream_base;
         sp.scale = scale;
-        const dim3 grid((teams->max_teams_per_seq + kLsTeamsPerBlock - 1) / kLsTeamsPerBlock, geom->n_seqs);
+        // as many tiles per warp as it takes for all blocks to be resident at once (two per SM)
+        const long long blocks1 = (long long)((teams->max_teams_per_seq + kLsTeamsPerBlock - 1) / kLsTeamsPerBlock) * geom->n_seqs;
+        const long long slots = 2ll * attend_grid_size();
+        sp.tiles_per_warp = (int)std::min<long long>(std::max<long long>((blocks1 + slots - 1) / slots, 1), 64);
+        const dim3 grid((teams->max_teams_per_seq + kLsTeamsPerBlock * sp.tiles_per_warp - 1) / (kLsTeamsPerBlock * sp.tiles_per_warp),
+                        geom->n_seqs);
         if ((err = launch_kernel(latent_score_kernel, grid, dim3(kLsThreads), 0, s, sp)) != cudaSuccess)
             return note_cuda_failure(err, "latent score launch");
         ++launches;
