@@ -211,6 +211,18 @@ def test_step_full_bench_batch_sampled_sequences():
     check_dense(layer, 0, seqs=[0, 31])
 
 
+def test_step_ragged_batch_with_several_tiles_per_scoring_warp():
+    """72 sequences of 3000 to 5500 rows: more 128-team blocks of the scorer than fit on the GPU at
+    once, so every scoring warp takes three tiles in a row, the last of them ragged or empty; four
+    sequences (the shortest and the longest among them) against the oracle."""
+    rng = np.random.default_rng(5)
+    lens = [int(x) for x in rng.integers(3000, 5500, size=72)]
+    lens[7], lens[40] = 3000, 5499
+    layer = LatentLayer(synth.LatentSpec("ragged72", lens, n_sample=48, suffix_cap=4,
+                                         suffix_len0=[int(x) for x in rng.integers(0, 5, size=72)], suffix_growth=0))
+    check_step(layer, 0, seqs=[0, 7, 40, 71])
+
+
 def test_tcgen05_variant_of_the_attention_kernel(small, monkeypatch):
     """The tensor-memory variant (chosen by the environment) against the oracle: sparse with a ragged
     tail and a suffix, dense, and a sequence of the full batch shape; its bounded waits must not expire."""
