@@ -251,7 +251,11 @@ int32_t santapp_kmeans_parent_count(int32_t prompt_len, int32_t parent_size);
  * step on `stream`. By default it waits for the stream every 16 steps to learn whether any fit
  * is still running (most stop long before the step limit), so it blocks the calling thread for
  * most of the fit; with opts->no_host_poll = 1 it never waits and enqueues every step up to the
- * limit instead (the result is the same: a stopped fit's later steps do nothing).
+ * limit instead (the result is the same: a stopped fit's later steps do nothing). In that mode the
+ * call may be issued during a stream capture and the graph replayed: the per-sequence tables made
+ * from the host arrays travel inside kernel arguments, nothing is copied from host memory. (The
+ * other preparation calls that take host arrays -- the builders and santapp_assign_parents -- copy
+ * their tables from host memory that is gone when they return: they must not be captured.)
  */
 typedef struct santapp_kmeans_opts {
     int32_t batch_size;           /* paper: 4096 */

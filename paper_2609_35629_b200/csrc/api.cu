@@ -604,13 +604,28 @@ int santapp_kmeans_fit(const santapp_geom *geom, const int32_t *prompt_len_host,
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     g_cuda_error[0] = 0;
     unsigned char *ws = static_cast<unsigned char *>(workspace);
-    const size_t ob = sizeof(int64_t) * ((size_t)B + 1);
-    cudaError_t err = cudaMemcpyAsync(ws + L.row_off, row_off, ob, cudaMemcpyHostToDevice, s);
-    if (err != cudaSuccess) return cuda_fail(err, "copy row offsets");
-    err = cudaMemcpyAsync(ws + L.cen_off, cen_off, ob, cudaMemcpyHostToDevice, s);
-    if (err != cudaSuccess) return cuda_fail(err, "copy centre offsets");
-    err = cudaMemcpyAsync(ws + L.tabs, tabs.data(), sizeof(int32_t) * tabs.size(), cudaMemcpyHostToDevice, s);
-    if (err != cudaSuccess) return cuda_fail(err, "copy fit tables");
+    cudaError_t err = cudaSuccess;
+    {
+        // the tables travel inside kernel arguments, a chunk of sequences per launch
+        int32_t *t_dev = reinterpret_cast<int32_t *>(ws + L.tabs);
+        for (int first = 0; first < B; first += kKmTableChunk) {
+            KmTableChunk c;
+            c.first = first;
+            c.n = std::min(kKmTableChunk, B - first);
+            for (int i = 0; i <= c.n; ++i) {
+                c.row_off[i] = row_off[first + i];
+                c.centre_off[i] = cen_off[first + i];
+            }
+            for (int i = 0; i < c.n; ++i) {
+                c.n_init[i] = tabs[first + i];
+                c.trials[i] = tabs[(size_t)B + first + i];
+                c.t_max[i] = tabs[2 * (size_t)B + first + i];
+            }
+            err = launch_kmeans_tables(c, reinterpret_cast<int64_t *>(ws + L.row_off), reinterpret_cast<int64_t *>(ws + L.cen_off),
+                                       t_dev, t_dev + B, t_dev + 2 * (size_t)B, s);
+            if (err != cudaSuccess) return cuda_fail(err, "fit tables");
+        }
+    }
 
     KmeansParams p;
     p.n_seqs = B;

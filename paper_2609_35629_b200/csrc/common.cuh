@@ -315,6 +315,17 @@ struct KmeansParams {
 };
 cudaError_t launch_kmeans_fit(const KmeansParams &p, cudaStream_t s);
 
+// Per-sequence tables of the fit, handed to the device inside kernel arguments (a copy from host
+// memory that is gone after the call would be read again by every replay of a captured graph).
+constexpr int kKmTableChunk = 128;
+struct KmTableChunk {
+    int32_t first, n;                               // sequences [first, first + n); offsets also get entry first + n
+    int64_t row_off[kKmTableChunk + 1], centre_off[kKmTableChunk + 1];
+    int32_t n_init[kKmTableChunk], trials[kKmTableChunk], t_max[kKmTableChunk];
+};
+cudaError_t launch_kmeans_tables(const KmTableChunk &c, int64_t *row_off, int64_t *centre_off, int32_t *n_init,
+                                 int32_t *trials, int32_t *t_max, cudaStream_t s);
+
 // ---------------------------------------------------------------------------------------------
 // Device helpers
 // ---------------------------------------------------------------------------------------------

@@ -659,6 +659,31 @@ cudaError_t run_fit(const KmeansParams &p, cudaStream_t s)
 
 }  // namespace
 
+namespace {
+__global__ void __launch_bounds__(kKmTableChunk + 32)
+km_tables_kernel(const __grid_constant__ KmTableChunk c, int64_t *row_off, int64_t *centre_off, int32_t *n_init,
+                 int32_t *trials, int32_t *t_max)
+{
+    const int i = threadIdx.x;
+    if (i <= c.n) {
+        row_off[c.first + i] = c.row_off[i];
+        centre_off[c.first + i] = c.centre_off[i];
+    }
+    if (i < c.n) {
+        n_init[c.first + i] = c.n_init[i];
+        trials[c.first + i] = c.trials[i];
+        t_max[c.first + i] = c.t_max[i];
+    }
+}
+}  // namespace
+
+cudaError_t launch_kmeans_tables(const KmTableChunk &c, int64_t *row_off, int64_t *centre_off, int32_t *n_init,
+                                 int32_t *trials, int32_t *t_max, cudaStream_t s)
+{
+    km_tables_kernel<<<1, kKmTableChunk + 32, 0, s>>>(c, row_off, centre_off, n_init, trials, t_max);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_kmeans_fit(const KmeansParams &p, cudaStream_t s)
 {
     return p.elem ? run_fit<true>(p, s) : run_fit<false>(p, s);

@@ -64,6 +64,29 @@ def test_fit_without_host_polling_gives_the_same_centres():
     assert steps.max() < 20 * 6                                 # the fits stopped before the limit
 
 
+def test_fit_without_host_polling_can_be_captured_in_a_cuda_graph():
+    """With no_host_poll the call only enqueues work: captured in a CUDA graph on a side stream and
+    replayed twice, it leaves the centres and step counts of the plain call (which the test above
+    compares with the oracle)."""
+    spec = synth.spec_small_gqa(prompt=(1536, 1000))
+    spec.n_clusters = 24
+    data = synth.make_layer(spec, layer=0, keep_centres=True)
+    geom = pu.geometry(spec)
+    k = sp.bf16_bits_to_cuda(data.k_prompt, dtype=geom.torch_dtype)
+    opts = dict(batch_size=256, seed=3, stream_base=11, max_iter=20, no_host_poll=True)
+    want_c, want_s = sp.santapp_kmeans_fit(geom, spec.prompt_len, [24, 9], k, **opts)
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        got_c, got_s = sp.santapp_kmeans_fit(geom, spec.prompt_len, [24, 9], k, **opts)
+    for _ in range(2):
+        got_c.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(got_c, want_c) and torch.equal(got_s, want_s)
+
+
 def test_fit_fp16_inputs():
     spec = synth.spec_small_gqa(prompt=(900,), n_seqs=1, suffix0=(0,))
     spec.elem = "fp16"
