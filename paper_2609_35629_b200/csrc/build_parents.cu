@@ -10,6 +10,8 @@
 // scatter of the tokens by team; copy K/V rows into the team-contiguous layout.
 #include <limits.h>
 
+#include <algorithm>
+
 #include "build_util.cuh"
 #include "common.cuh"
 
@@ -126,18 +128,23 @@ scan_parents_kernel(ParentBuildParams p)
     }
 }
 
-// One warp per (sequence, KV head): position of every token in the list ordered by (label, token
-// index). Tokens are taken 32 at a time in increasing index; lanes with the same label form a
-// group whose lowest lane reserves the group's slots at the label's cursor, and each lane takes
-// the slot of its rank inside the group. The full-warp shuffle that hands the reserved base round
-// also makes every reservation of one step complete before the next step begins.
+// One block per (sequence, KV head): position of every token in the list ordered by (label, token
+// index). One warp takes the tokens 32 at a time in increasing index; lanes with the same label
+// form a group whose lowest lane reserves the group's slots at the label's cursor, and each lane
+// takes the slot of its rank inside the group. The full-warp shuffle that hands the reserved base
+// round also makes every reservation of one step complete before the next step begins. The
+// cursors are copied into shared memory by the whole block when they fit (smem_labels of them: a
+// step then costs a shared-memory atomic instead of a round trip to L2; they are not needed
+// afterwards), and a step's labels are requested one step ahead.
 //   kInverse: out[position] = token (member lists); otherwise out[token] = position.
+constexpr int kScatterSmemLabels = 50 * 1024;               // cursors that fit in shared memory (200 KB)
 template <bool kInverse>
-__global__ void __launch_bounds__(32)
+__global__ void __launch_bounds__(kThreads)
 stable_scatter_kernel(const int32_t *labels, int32_t *cursors, int32_t *out, const int64_t *seq_row_off,
-                      const int64_t *seq_label_off, int64_t rows_total, int64_t labels_total)
+                      const int64_t *seq_label_off, int64_t rows_total, int64_t labels_total, int smem_labels)
 {
-    const int b = blockIdx.x, j = blockIdx.y, lane = threadIdx.x;
+    extern __shared__ int32_t cur_s[];
+    const int b = blockIdx.x, j = blockIdx.y, tid = threadIdx.x, lane = tid & 31;
     const int64_t row0 = seq_row_off[b];
     const int N = (int)(seq_row_off[b + 1] - row0);
     const int64_t l0 = seq_label_off[b];
@@ -145,15 +152,23 @@ stable_scatter_kernel(const int32_t *labels, int32_t *cursors, int32_t *out, con
     const int32_t *lab = labels + (size_t)j * rows_total + row0;
     int32_t *cur = cursors + (size_t)j * labels_total + l0;
     int32_t *dst = out + (size_t)j * rows_total + row0;
+    const bool in_smem = n_labels <= smem_labels;
+    if (in_smem)
+        for (int u = tid; u < n_labels; u += kThreads) cur_s[u] = cur[u];
+    __syncthreads();
+    if (tid >= 32) return;
+    int next = lane < N ? lab[lane] : 0;
     for (int i0 = 0; i0 < N; i0 += 32) {
         const int i = i0 + lane;
         const bool valid = i < N;
-        const int u = valid ? clamp_label(lab[i], n_labels) : -1 - lane;       // idle lanes stay alone
+        const int mine = next;
+        if (i + 32 < N) next = lab[i + 32];
+        const int u = valid ? clamp_label(mine, n_labels) : -1 - lane;         // idle lanes stay alone
         const unsigned group = __match_any_sync(0xFFFFFFFFu, u);
         const int leader = __ffs(group) - 1;
         const int rank = __popc(group & ((1u << lane) - 1u));
         int base = 0;
-        if (valid && lane == leader) base = atomicAdd(cur + u, __popc(group));
+        if (valid && lane == leader) base = in_smem ? atomicAdd(cur_s + u, __popc(group)) : atomicAdd(cur + u, __popc(group));
         base = __shfl_sync(0xFFFFFFFFu, base, leader);
         if (valid) {
             if (kInverse) dst[base + rank] = i;
@@ -374,16 +389,24 @@ cudaError_t launch_build_teams_parents(const ParentBuildParams &p, cudaStream_t 
     if ((err = cudaGetLastError()) != cudaSuccess) return err;
     scan_parents_kernel<<<dim3(B, H), kThreads, 0, s>>>(p);
     if ((err = cudaGetLastError()) != cudaSuccess) return err;
-    stable_scatter_kernel<true><<<dim3(B, H), 32, 0, s>>>(p.parent_of, p.parent_cursor, p.members, p.bv.seq_row_off,
-                                                          p.seq_label_off, p.bv.rows_total, p.labels_total);
+    // cursors in shared memory when a sequence's labels (teams: at most reps per label) fit
+    const int lab_smem = std::min(p.max_labels_per_seq, kScatterSmemLabels);
+    const long long max_teams = (long long)p.max_labels_per_seq * p.reps;
+    const int team_smem = (int)std::min<long long>(max_teams, kScatterSmemLabels);
+    if ((err = cudaFuncSetAttribute(stable_scatter_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    (int)sizeof(int32_t) * kScatterSmemLabels)) != cudaSuccess) return err;
+    if ((err = cudaFuncSetAttribute(stable_scatter_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    (int)sizeof(int32_t) * kScatterSmemLabels)) != cudaSuccess) return err;
+    stable_scatter_kernel<true><<<dim3(B, H), kThreads, sizeof(int32_t) * (size_t)lab_smem, s>>>(
+        p.parent_of, p.parent_cursor, p.members, p.bv.seq_row_off, p.seq_label_off, p.bv.rows_total, p.labels_total, lab_smem);
     if ((err = cudaGetLastError()) != cudaSuccess) return err;
     if (p.bv.elem) build_parent_general_kernel<true><<<dim3(p.max_labels_per_seq, B, H), kThreads, 0, s>>>(p);
     else           build_parent_general_kernel<false><<<dim3(p.max_labels_per_seq, B, H), kThreads, 0, s>>>(p);
     if ((err = cudaGetLastError()) != cudaSuccess) return err;
     scan_teams_kernel<<<dim3(B, H), kThreads, 0, s>>>(p);
     if ((err = cudaGetLastError()) != cudaSuccess) return err;
-    stable_scatter_kernel<false><<<dim3(B, H), 32, 0, s>>>(p.team_of, p.team_cursor, p.dest, p.bv.seq_row_off,
-                                                           p.bv.seq_team_off, p.bv.rows_total, p.bv.teams_total);
+    stable_scatter_kernel<false><<<dim3(B, H), kThreads, sizeof(int32_t) * (size_t)team_smem, s>>>(
+        p.team_of, p.team_cursor, p.dest, p.bv.seq_row_off, p.bv.seq_team_off, p.bv.rows_total, p.bv.teams_total, team_smem);
     if ((err = cudaGetLastError()) != cudaSuccess) return err;
     pack_rows_kernel<<<dim3((p.max_rows_per_seq + kThreads / 32 - 1) / (kThreads / 32), B, H), kThreads, 0, s>>>(p);
     return cudaGetLastError();

@@ -11,6 +11,8 @@
 #include <limits.h>
 #include <math.h>
 
+#include <algorithm>
+
 #include "common.cuh"
 
 namespace santapp {
@@ -84,28 +86,43 @@ km_perm_identity_kernel(KmeansParams p)
     if (i < q.N) p.perm[q.plane + i] = i;
 }
 
-__global__ void __launch_bounds__(32)
-km_sample_kernel(KmeansParams p)
+// One block per pair. The swaps run in order on one lane; when the sequence's index list fits in
+// shared memory (smem_rows entries) it lives there for the shuffle -- a swap then costs two
+// shared-memory round trips instead of two to L2 -- and only the head, the sample, is written out.
+constexpr int kSampleSmemRows = 50 * 1024;
+__global__ void __launch_bounds__(kThreads)
+km_sample_kernel(KmeansParams p, int smem_rows)
 {
+    extern __shared__ int32_t perm_s[];
     const Pair q = pair_of(p, blockIdx.x, blockIdx.y);
-    const int lane = threadIdx.x;
-    int32_t *perm = p.perm + q.plane;
-    // the words of 32 positions at a time, the swaps in order on one lane
-    for (int i0 = 0; i0 < q.n_init; i0 += 32) {
-        const int i = i0 + lane;
-        const uint32_t w = i < q.n_init ? km_word(p, (uint32_t)i, kTagSample, q.stream, 0u) : 0u;
-        for (int l = 0; l < 32 && i0 + l < q.n_init; ++l) {
-            const uint32_t wl = __shfl_sync(0xFFFFFFFFu, w, l);
-            if (lane == 0) {
-                const int at = i0 + l;
-                const int r = at + km_index(wl, q.N - at);
-                const int32_t t = perm[at];
-                perm[at] = perm[r];
-                perm[r] = t;
+    const int tid = threadIdx.x, lane = tid & 31;
+    int32_t *perm_g = p.perm + q.plane;                       // (holds the identity when it is used for the shuffle)
+    const bool in_smem = q.N <= smem_rows;
+    if (in_smem)
+        for (int i = tid; i < q.N; i += kThreads) perm_s[i] = i;
+    __syncthreads();
+    if (tid < 32) {
+        int32_t *perm = in_smem ? perm_s : perm_g;
+        // the words of 32 positions at a time, the swaps in order on one lane
+        for (int i0 = 0; i0 < q.n_init; i0 += 32) {
+            const int i = i0 + lane;
+            const uint32_t w = i < q.n_init ? km_word(p, (uint32_t)i, kTagSample, q.stream, 0u) : 0u;
+            for (int l = 0; l < 32 && i0 + l < q.n_init; ++l) {
+                const uint32_t wl = __shfl_sync(0xFFFFFFFFu, w, l);
+                if (lane == 0) {
+                    const int at = i0 + l;
+                    const int r = at + km_index(wl, q.N - at);
+                    const int32_t t = perm[at];
+                    perm[at] = perm[r];
+                    perm[r] = t;
+                }
             }
         }
     }
-    if (lane == 0) p.pick[(size_t)q.id * p.trials_max] = km_index(km_word(p, 0u, kTagStart, q.stream, 0u), q.n_init);
+    __syncthreads();
+    if (in_smem)
+        for (int i = tid; i < q.n_init; i += kThreads) perm_g[i] = perm_s[i];
+    if (tid == 0) p.pick[(size_t)q.id * p.trials_max] = km_index(km_word(p, 0u, kTagStart, q.stream, 0u), q.n_init);
 }
 
 // ---- 2. greedy k-means++ on the sample ----
@@ -608,9 +625,14 @@ cudaError_t run_fit(const KmeansParams &p, cudaStream_t s)
     const int B = p.n_seqs, H = p.n_kv, pairs = B * H;
     cudaError_t err;
 #define KM_CHECK() if ((err = cudaGetLastError()) != cudaSuccess) return err
-    km_perm_identity_kernel<<<dim3((p.max_rows_per_seq + kThreads - 1) / kThreads, B, H), kThreads, 0, s>>>(p);
-    KM_CHECK();
-    km_sample_kernel<<<dim3(B, H), 32, 0, s>>>(p);
+    const int sample_smem_rows = std::min(p.max_rows_per_seq, kSampleSmemRows);
+    if (p.max_rows_per_seq > sample_smem_rows) {              // some sequence shuffles its index list in global memory
+        km_perm_identity_kernel<<<dim3((p.max_rows_per_seq + kThreads - 1) / kThreads, B, H), kThreads, 0, s>>>(p);
+        KM_CHECK();
+    }
+    if ((err = cudaFuncSetAttribute(km_sample_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    (int)sizeof(int32_t) * kSampleSmemRows)) != cudaSuccess) return err;
+    km_sample_kernel<<<dim3(B, H), kThreads, sizeof(int32_t) * (size_t)sample_smem_rows, s>>>(p, sample_smem_rows);
     KM_CHECK();
     const dim3 dist_grid((p.n_init_max + kSumBlock - 1) / kSumBlock, (p.trials_max + kDistTrials - 1) / kDistTrials, pairs);
     const size_t draw_smem = sizeof(double) * ((size_t)p.n_init_max + 2 * kMaxSumBlocks);
