@@ -87,6 +87,14 @@ def test_fit_without_host_polling_can_be_captured_in_a_cuda_graph():
         assert torch.equal(got_c, want_c) and torch.equal(got_s, want_s)
 
 
+def test_fit_on_a_sequence_too_long_for_the_shared_memory_shuffle():
+    """52000 keys beside 900: the long sequence's index list does not fit in shared memory, so its
+    initialisation sample is shuffled in global memory, the short one's in shared memory."""
+    spec = synth.spec_small_gqa(prompt=(52000, 900), suffix0=(0, 0))
+    spec.n_clusters = 16
+    _fit_both(spec, [11, 6], batch_size=192, seed=5, max_iter=3, patience=4)
+
+
 def test_fit_fp16_inputs():
     spec = synth.spec_small_gqa(prompt=(900,), n_seqs=1, suffix0=(0,))
     spec.elem = "fp16"
