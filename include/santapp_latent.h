@@ -97,8 +97,8 @@ size_t santapp_latent_decode_workspace_bytes(const santapp_latent_geom *geom,
  *   suffix_rows   device bf16 [n_seqs][suffix_cap][576] or NULL when suffix_cap == 0: rows of the
  *                 generated tokens, attended exactly by every head
  *   suffix_len_dev device int32 [n_seqs] or NULL (= 0): visible suffix rows, clamped to [0, suffix_cap]
- *   n_sample      1 <= K <= 128 teams per head (the paper's budgets S = 128, 256, 512 with P = 16,
- *                 R = 4 are K = 32, 64, 128)
+ *   n_sample      1 <= K <= 256 teams per head (the paper's budgets S = 128, 256, 512, 1024 with
+ *                 P = 16, R = 4 are K = 32, 64, 128, 256)
  *   scale         logit scale, > 0 (the model's; there is no default for this row format)
  *   out           device fp32 [n_seqs][n_heads][512]
  *   dbg           as in santapp_decode_attn with n_q_heads = n_heads and one KV head; `trace` is

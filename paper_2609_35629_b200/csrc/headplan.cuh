@@ -24,7 +24,7 @@ namespace santapp {
 
 constexpr int kMaxHeadWarps = 32;        // blocks of up to 1024 threads
 constexpr int kCandCap = 512;           // candidates refined at a time
-constexpr int kListCap = 132;           // running top list: K + 1 <= 129 entries (+ one pad)
+constexpr int kListCap = 260;           // running top list: K + 1 <= 257 entries (+ pad); K <= 128 for K/V rows, <= 256 for shared-latent rows
 constexpr int kDotLanes = 8;            // threads that share one candidate's dot product
 constexpr int kWindow = 255;            // histogram bins per pass of the bound
 

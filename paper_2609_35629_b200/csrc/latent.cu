@@ -419,9 +419,10 @@ struct LatentPlanParams {
 };
 
 constexpr int kLpThreads = 512;
-constexpr int kLatSegMax = kHeads * 128 + 1;                // 16 heads x K <= 128 teams, + the suffix
-constexpr int kLpPerThread = kHeads * 128 / kLpThreads;     // sampled teams of a sequence per thread
-static_assert(kLpPerThread * kLpThreads == kHeads * 128, "a block holds a sequence's samples in registers");
+constexpr int kLatMaxSample = 256;                          // K: the paper's largest budget, S = 1024 rows at R / P = 1 / 4
+constexpr int kLatSegMax = kHeads * kLatMaxSample + 1;      // 16 heads x K teams, + the suffix
+constexpr int kLpPerThread = kHeads * kLatMaxSample / kLpThreads;     // sampled teams of a sequence per thread
+static_assert(kLpPerThread * kLpThreads == kHeads * kLatMaxSample, "a block holds a sequence's samples in registers");
 
 struct LatentPlanSmem {
     uint32_t bitmap[kMaxTeamsPerSeq / 32];
@@ -1241,7 +1242,7 @@ int santapp_latent_build_teams(const santapp_latent_geom *geom, const int32_t *p
 size_t santapp_latent_decode_workspace_bytes(const santapp_latent_geom *geom, const santapp_latent_teams *teams, int32_t n_sample,
                                              int32_t suffix_cap)
 {
-    if (check_latent_geom(geom) != SANTAPP_OK || !teams || n_sample < 1 || n_sample > 128 || suffix_cap < 0) return 0;
+    if (check_latent_geom(geom) != SANTAPP_OK || !teams || n_sample < 1 || n_sample > kLatMaxSample || suffix_cap < 0) return 0;
     return latent_layout(geom, teams, n_sample, suffix_cap, false).total;
 }
 
@@ -1266,7 +1267,7 @@ int santapp_latent_decode_attn(const santapp_latent_geom *geom, const santapp_la
         || lat_misaligned(suffix_len_dev, 4))
         return SANTAPP_ERR_INVALID_ARG;
     if (n_sample < 1 || suffix_cap < 0) return SANTAPP_ERR_INVALID_ARG;
-    if (n_sample > 128) return SANTAPP_ERR_UNSUPPORTED;
+    if (n_sample > kLatMaxSample) return SANTAPP_ERR_UNSUPPORTED;
     if (suffix_cap > 0 && suffix_len_dev && !suffix_rows) return SANTAPP_ERR_INVALID_ARG;
     if (!(scale > 0.f) || isinf(scale)) return SANTAPP_ERR_INVALID_ARG;
     if ((int64_t)geom->n_seqs * (int64_t)suffix_cap + teams->rows_total >= (int64_t)1 << 31) return SANTAPP_ERR_UNSUPPORTED;

@@ -190,10 +190,11 @@ def test_step_many_short_sequences_blocks_span_several():
 
 
 def test_step_paper_point_8k_all_budgets():
-    """8K context, P = 16, R = 4, 16 heads; the study's budgets S = 128, 256, 512 rows are K = 32, 64, 128 teams."""
+    """8K context, P = 16, R = 4, 16 heads; the study's budgets S = 128, 256, 512, 1024 rows are
+    K = 32, 64, 128, 256 teams."""
     layer = LatentLayer(synth.LatentSpec("8k", [8192, 8192], suffix_cap=16, suffix_len0=[0, 5]))
     check_records(layer)
-    for K in (32, 64, 128):
+    for K in (32, 64, 128, 256):
         worst, union = check_step(layer, 1, K=K)
         # shared-row accounting on the kernel's own counts (Eq. mla-logical-access)
         sl = layer.spec.suffix_len(1)
@@ -257,7 +258,7 @@ def test_bad_arguments_are_refused_on_the_host(small):
     q = sp.bf16_bits_to_cuda(synth.make_latent_queries(small.spec, small.data, 0))
     ws = torch.empty(1 << 20, dtype=torch.uint8, device="cuda")
     with pytest.raises(sp.SantappError) as e:
-        sp.santapp_latent_decode_attn(small.geom, small.teams, q, None, None, 129, 0, 0, synth.LATENT_SCALE, workspace=ws)
+        sp.santapp_latent_decode_attn(small.geom, small.teams, q, None, None, 257, 0, 0, synth.LATENT_SCALE, workspace=ws)
     assert e.value.status == sp.SANTAPP_ERR_UNSUPPORTED
     with pytest.raises(sp.SantappError) as e:
         sp.santapp_latent_decode_attn(small.geom, small.teams, q, None, None, 8, 0, 0, 0.0)
