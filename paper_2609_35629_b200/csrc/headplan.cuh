@@ -18,6 +18,8 @@
 
 #include <math_constants.h>
 
+#include <stddef.h>
+
 #include "common.cuh"
 
 namespace santapp {
@@ -44,8 +46,12 @@ struct alignas(16) HeadSmemT {
     int hist[256];
     float red_max[kMaxHeadWarps], red_sum[kMaxHeadWarps];
     int n_cand, bound_bin, bound_below, bound_total;
+    uint32_t taken[(kListCap + 31) / 32];   // ranks handed out by the integer ranking pass
+    int need_exact;                     // two entries met on one rank: rank again on whole scores
 };
 using HeadSmem = HeadSmemT<kHeadDim>;
+static_assert(offsetof(HeadSmemT<128>, cand_g) % 16 == 0 && offsetof(HeadSmemT<576>, cand_g) % 16 == 0,
+              "the ranking pass reads the keys kept in cand_g sixteen bytes at a time");
 
 // Guard on |Y32 - Y|: tensor-core accumulation of exact 16-bit products in fp32 (relative to the sum
 // of magnitudes, bounded by scale * |q|_1 * max|l|), plus the fp32 logarithm and Gumbel terms.
@@ -343,10 +349,51 @@ __device__ __forceinline__ void select_head(const PlanInputs &in, int hq, HeadSm
         __syncthreads();
 
         // ---- 3b. merge with the running list: keep the K + 1 largest by (Y descending, id ascending) ----
-        // eight lanes share an entry: each counts the entries ahead of it in its share of the scores
-        {
+        // Ranking is all comparisons, and the count of them is what this step costs. First pass, on
+        // integers: every entry (list, then candidates) gets the upper half of its score's integer
+        // key (same order as the score); a thread holds one entry and walks all keys, four per
+        // broadcast load, counting the larger ones. Two entries whose scores agree in the upper half
+        // of the key land on the same rank; the second one to arrive sees the rank taken and asks for
+        // the exact pass below, which ranks on whole scores and ids as the paper's order says.
+        const int n_all = n_list + n_cand;
+        uint32_t *key_hi = reinterpret_cast<uint32_t *>(sm.cand_g);   // (the Gumbel terms are used up)
+        const int n_pad = (n_all + 3) & ~3;
+        for (int e = tid; e < n_pad; e += kT) {
+            uint32_t h = 0u;                                          // padding: below every key
+            if (e < n_all) h = (uint32_t)(sortable_key(e < n_list ? sm.list_y[cur][e] : sm.cand_y[e - n_list]) >> 32);
+            key_hi[e] = h;
+        }
+        if (tid < (kListCap + 31) / 32) sm.taken[tid] = 0u;
+        if (tid == 0) sm.need_exact = 0;
+        __syncthreads();
+        for (int e = tid; e < n_all; e += kT) {
+            const uint32_t yh = key_hi[e];
+            int rank = 0;
+#pragma unroll 2
+            for (int a = 0; a < n_pad; a += 4) {
+                const uint4 w = *reinterpret_cast<const uint4 *>(key_hi + a);
+                rank += (w.x > yh) + (w.y > yh) + (w.z > yh) + (w.w > yh);
+            }
+            if (rank <= K) {
+                const uint32_t bit = 1u << (rank & 31);
+                if (atomicOr(&sm.taken[rank >> 5], bit) & bit) sm.need_exact = 1;
+                else if (e < n_list) {
+                    sm.list_y[cur ^ 1][rank] = sm.list_y[cur][e];
+                    sm.list_phi[cur ^ 1][rank] = sm.list_phi[cur][e];
+                    sm.list_id[cur ^ 1][rank] = sm.list_id[cur][e];
+                    sm.list_rows[cur ^ 1][rank] = sm.list_rows[cur][e];
+                } else {
+                    sm.list_y[cur ^ 1][rank] = sm.cand_y[e - n_list];
+                    sm.list_phi[cur ^ 1][rank] = sm.cand_phi[e - n_list];
+                    sm.list_id[cur ^ 1][rank] = sm.cand_id[e - n_list];
+                    sm.list_rows[cur ^ 1][rank] = sm.cand_rows[e - n_list];
+                }
+            }
+        }
+        __syncthreads();
+        if (sm.need_exact) {
+            // eight lanes share an entry: each counts the entries ahead of it in its share of the scores
             const int sub = lane & 7;
-            const int n_all = n_list + n_cand;
             for (int e0 = 0; e0 < n_all; e0 += kT / 8) {                  // uniform trip count: the votes below are warp-wide
                 const int e = e0 + (tid >> 3);
                 const bool live = e < n_all;
