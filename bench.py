@@ -13,7 +13,7 @@ Prints ONE JSON line (rank 0). `value` is microseconds per layer-step with all i
 in HBM, replayed from CUDA graphs; `e2e` is the same through host buffers (pinned host to
 device copies of the step's queries, new suffix rows and counters, device to host read of the
 outputs, inside the timed region). With the default workload the line also carries `batched`:
-the same measurement on the ragged 32-sequence batch (two layers, a few steps), the size at which
+the same measurement on the ragged 32-sequence batch (two layers, 30 steps), the size at which
 the operator is bandwidth-bound rather than latency-bound (`--no-batched` skips it), `mid_batch` and
 `long_context` (configs 3 and 5), `shared_latent` (rows of 512 + 64 values shared by 16 heads, 32
 sequences of 8K, `--workload latent_8k` on its own) and `kmeans_parents`.
@@ -253,7 +253,7 @@ def run_ours(args):
         import gc
         gc.collect()
         torch.cuda.empty_cache()
-        big = measure_workload(args, "ragged", 2, 10, 3, dev, want_e2e=False, want_cpu=False, want_stages=True)
+        big = measure_workload(args, "ragged", 2, 30, 3, dev, want_e2e=False, want_cpu=False, want_stages=True)
         if rank == 0:
             keep = ("value", "unit", "dense_us_per_layer_step", "speedup_vs_dense", "read_reduction",
                     "achieved_frac_of_peak", "dense_achieved_frac_of_peak", "roofline", "stage_us", "paired_rounds",
@@ -265,7 +265,7 @@ def run_ours(args):
             gc.collect()
             torch.cuda.empty_cache()
             wl_args = argparse.Namespace(**{**vars(args), "n_sample": k_over})
-            res = measure_workload(wl_args, wl, n_lay, 10, 3, dev, want_e2e=False, want_cpu=False, want_stages=True)
+            res = measure_workload(wl_args, wl, n_lay, 30, 3, dev, want_e2e=False, want_cpu=False, want_stages=True)
             if rank == 0:
                 line[key] = {"workload": res["config"]["workload"], **{k: res[k] for k in keep}}
         # shared-latent rows (one 576-value row per token, 16 heads) at the paper's 8K study point, 32 sequences
@@ -275,7 +275,7 @@ def run_ours(args):
         for key, k_lat in (("shared_latent", 128), ("shared_latent_k32", 32)):
             gc.collect()
             torch.cuda.empty_cache()
-            lat = measure_latent(args, 2, 10, 3, dev, n_sample=k_lat)
+            lat = measure_latent(args, 2, 30, 3, dev, n_sample=k_lat)
             if rank == 0:
                 line[key] = lat
         # and the headline workload with the parents of the paper's headline runs: Algorithm 3
