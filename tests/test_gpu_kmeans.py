@@ -95,6 +95,15 @@ def test_fit_on_a_sequence_too_long_for_the_shared_memory_shuffle():
     _fit_both(spec, [11, 6], batch_size=192, seed=5, max_iter=3, patience=4)
 
 
+def test_fit_of_150_short_sequences_takes_its_tables_in_two_chunks():
+    """More sequences than one kernel-argument chunk of the per-sequence tables holds (128)."""
+    rng = np.random.default_rng(9)
+    lens = tuple(int(x) for x in rng.integers(30, 70, size=150))
+    spec = synth.spec_small_gqa(n_seqs=150, prompt=lens, suffix0=(0,) * 150)
+    spec.n_clusters = 4
+    _fit_both(spec, [2 + (i % 3) for i in range(150)], batch_size=16, seed=2, max_iter=2, patience=3)
+
+
 def test_fit_fp16_inputs():
     spec = synth.spec_small_gqa(prompt=(900,), n_seqs=1, suffix0=(0,))
     spec.elem = "fp16"
