@@ -224,6 +224,15 @@ def test_step_ragged_batch_with_several_tiles_per_scoring_warp():
     check_step(layer, 0, seqs=[0, 7, 40, 71])
 
 
+def test_two_hundred_steps_of_the_sampler():
+    """Many draws on one layer (a different seed every step, K = 96 of 512 and 375 teams): now and
+    then two candidates' scores agree in the upper half of their integer keys, which sends a head
+    through the exact ranking pass; every sample must still be the oracle's."""
+    layer = LatentLayer(synth.LatentSpec("soak", [2048, 1500], n_sample=96, suffix_cap=12, suffix_len0=[0, 3]))
+    for step in range(200):
+        check_step(layer, step, seed=step * 7 + 1)
+
+
 def test_tcgen05_variant_of_the_attention_kernel(small, monkeypatch):
     """The tensor-memory variant (chosen by the environment) against the oracle: sparse with a ragged
     tail and a suffix, dense, and a sequence of the full batch shape; its bounded waits must not expire."""
