@@ -54,7 +54,8 @@ typedef struct santapp_latent_teams {
     void *rows_packed;         /* bf16 [rows_total][576]: each team's members contiguous, teams in
                                   id order, members by token index                               */
     void *rep_rows;            /* bf16 [teams_total][576]: the representatives' rows (frozen
-                                  routing keys)                                                  */
+                                  routing keys); 32-byte aligned (the scorer reads 32 bytes at a
+                                  time), every other array as in santapp.h                       */
     int32_t *team_row_start;   /* int32 [teams_total + n_seqs]: sequence b's M_b + 1 CSR offsets
                                   start at seq_team_off[b] + b; values are local to the sequence */
     int32_t *row_token;        /* int32 [rows_total]: token index (local) of each packed row      */

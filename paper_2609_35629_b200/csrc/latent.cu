@@ -269,12 +269,27 @@ __device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
+// 32 bytes from global memory in one instruction (read-only path; the address is 32-byte aligned).
+struct Words8 { uint32_t v[8]; };
+__device__ __forceinline__ Words8 ldg256(const void *p)
+{
+    Words8 w;
+    asm volatile("ld.global.nc.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(w.v[0]), "=r"(w.v[1]), "=r"(w.v[2]), "=r"(w.v[3]), "=r"(w.v[4]), "=r"(w.v[5]), "=r"(w.v[6]), "=r"(w.v[7])
+                 : "l"(p));
+    return w;
+}
+
 // Grid (ceil(max teams / (128 tiles_per_warp)), sequences); a warp scores tiles_per_warp consecutive
 // tiles of 16 teams for all heads: the teams are the MMA's 16 rows, the heads its columns (two tiles
 // of 8), the 576 values 36 k-steps. Both operands use the same permutation of the contraction index
-// inside every block of 32 values, so a lane feeds the tensor core 16-byte pieces of a
-// representative row (and of a query) as they lie in memory: piece t of the block supplies k-slots
-// {2t, 2t+1, 2t+8, 2t+9} of the block's two MMAs. The host picks tiles_per_warp so that all blocks
+// inside every segment of 64 values (128 bytes), so a lane feeds the tensor core 32-byte pieces of a
+// representative row (and of a query) as they lie in memory: lane t of a row's four lanes takes bytes
+// [32 t, 32 t + 32) of the segment with one 256-bit load, and the s-th eight bytes of its piece are
+// its k-slots {2t, 2t+1, 2t+8, 2t+9} of the segment's s-th MMA. One load instruction of a warp then
+// touches eight whole 128-byte lines (with 16-byte pieces it touched eight half lines, and the kernel
+// was bound by the number of line accesses in L1: 70 % of its peak at 48 % of the DRAM bandwidth).
+// The host picks tiles_per_warp so that all blocks
 // are resident at once (two per SM): a second, partly filled wave of blocks costs as much as a full one.
 __global__ void __launch_bounds__(kLsThreads)
 latent_score_kernel(LatentScoreParams p)
@@ -291,17 +306,18 @@ latent_score_kernel(LatentScoreParams p)
     // the warp's first pieces of its representatives' rows are requested before anything else: they
     // do not depend on the queries, and the block's set-up (queries into shared memory) runs while
     // they are on their way
-    constexpr int kBatch = 6;                                       // blocks of 32 values requested together
+    constexpr int kBatch = 3;                                       // segments of 64 values requested together
+    constexpr int kSegs = kRowDim / 64;                             // 9 segments of 128 bytes per row
     const int t_first = ((int)blockIdx.x * (kLsThreads / 32) + warp) * tpw * 16;
     const bool live = t_first < M;
     const int r = lane >> 2, t = lane & 3;
     const uint16_t *rep = p.rep_rows + (size_t)team0 * kRowDim;
-    auto row_ptr = [&](int team) { return reinterpret_cast<const uint4 *>(rep + (size_t)min(team, M - 1) * kRowDim) + t; };
-    uint4 wa[kBatch], wb[kBatch];
+    auto row_ptr = [&](int team) { return reinterpret_cast<const unsigned char *>(rep + (size_t)min(team, M - 1) * kRowDim) + 32 * t; };
+    Words8 wa[kBatch], wb[kBatch];
     if (live) {
-        const uint4 *ka = row_ptr(t_first + r), *kb = row_ptr(t_first + r + 8);
+        const unsigned char *ka = row_ptr(t_first + r), *kb = row_ptr(t_first + r + 8);
 #pragma unroll
-        for (int i = 0; i < kBatch; ++i) { wa[i] = __ldg(ka + i * 4); wb[i] = __ldg(kb + i * 4); }
+        for (int i = 0; i < kBatch; ++i) { wa[i] = ldg256(ka + i * 128); wb[i] = ldg256(kb + i * 128); }
     }
     const int32_t *csr = p.team_row_start + team0 + b;
     const uint32_t step = p.step + (p.step_dev ? *p.step_dev : 0u);
@@ -328,9 +344,9 @@ latent_score_kernel(LatentScoreParams p)
         const int t0 = t_first + it * 16;
         if (t0 >= M) break;
         const int ga = t0 + r, gb = t0 + r + 8;                     // the lane's two teams (rows r and r + 8 of the tile)
-        const uint4 *ka = row_ptr(ga), *kb = row_ptr(gb);
+        const unsigned char *ka = row_ptr(ga), *kb = row_ptr(gb);
         const bool more = it + 1 < tpw && t0 + 16 < M;              // the next tile's first pieces follow this tile's last
-        const uint4 *ka_next = row_ptr(ga + 16), *kb_next = row_ptr(gb + 16);
+        const unsigned char *ka_next = row_ptr(ga + 16), *kb_next = row_ptr(gb + 16);
         int na = 1, nb = 1;
         if (ga < M) na = csr[ga + 1] - csr[ga];
         if (gb < M) nb = csr[gb + 1] - csr[gb];
@@ -346,23 +362,28 @@ latent_score_kernel(LatentScoreParams p)
         }
         float acc[2][4] = {};
 #pragma unroll 1
-        for (int blk0 = 0; blk0 < kRowDim / 32; blk0 += kBatch) {
-            const bool last = blk0 + kBatch >= kRowDim / 32;
+        for (int sg0 = 0; sg0 < kSegs; sg0 += kBatch) {
+            const bool last = sg0 + kBatch >= kSegs;
 #pragma unroll
             for (int i = 0; i < kBatch; ++i) {
-                const int piece = (blk0 + i) * 4 + t;
-                const uint4 q0 = *reinterpret_cast<const uint4 *>(q_s + r * kQPitchW + piece * 4);
-                const uint4 q1 = *reinterpret_cast<const uint4 *>(q_s + (r + 8) * kQPitchW + piece * 4);
-                mma_bf16(acc[0], wa[i].x, wb[i].x, wa[i].y, wb[i].y, q0.x, q0.y);
-                mma_bf16(acc[0], wa[i].z, wb[i].z, wa[i].w, wb[i].w, q0.z, q0.w);
-                mma_bf16(acc[1], wa[i].x, wb[i].x, wa[i].y, wb[i].y, q1.x, q1.y);
-                mma_bf16(acc[1], wa[i].z, wb[i].z, wa[i].w, wb[i].w, q1.z, q1.w);
+                // the lane's 32 bytes of the two queries (heads r and r + 8) for this segment
+                const uint32_t *qa = q_s + r * kQPitchW + (sg0 + i) * 32 + 8 * t;
+                const uint32_t *qb = qa + 8 * kQPitchW;
+                const uint4 qa0 = *reinterpret_cast<const uint4 *>(qa), qa1 = *reinterpret_cast<const uint4 *>(qa + 4);
+                const uint4 qb0 = *reinterpret_cast<const uint4 *>(qb), qb1 = *reinterpret_cast<const uint4 *>(qb + 4);
+                const uint32_t q0[8] = {qa0.x, qa0.y, qa0.z, qa0.w, qa1.x, qa1.y, qa1.z, qa1.w};
+                const uint32_t q1[8] = {qb0.x, qb0.y, qb0.z, qb0.w, qb1.x, qb1.y, qb1.z, qb1.w};
+#pragma unroll
+                for (int s4 = 0; s4 < 4; ++s4) {
+                    mma_bf16(acc[0], wa[i].v[2 * s4], wb[i].v[2 * s4], wa[i].v[2 * s4 + 1], wb[i].v[2 * s4 + 1], q0[2 * s4], q0[2 * s4 + 1]);
+                    mma_bf16(acc[1], wa[i].v[2 * s4], wb[i].v[2 * s4], wa[i].v[2 * s4 + 1], wb[i].v[2 * s4 + 1], q1[2 * s4], q1[2 * s4 + 1]);
+                }
                 if (!last) {                                        // the same piece of the next batch
-                    wa[i] = __ldg(ka + (blk0 + kBatch + i) * 4);
-                    wb[i] = __ldg(kb + (blk0 + kBatch + i) * 4);
+                    wa[i] = ldg256(ka + (sg0 + kBatch + i) * 128);
+                    wb[i] = ldg256(kb + (sg0 + kBatch + i) * 128);
                 } else if (more) {
-                    wa[i] = __ldg(ka_next + i * 4);
-                    wb[i] = __ldg(kb_next + i * 4);
+                    wa[i] = ldg256(ka_next + i * 128);
+                    wb[i] = ldg256(kb_next + i * 128);
                 }
             }
         }
@@ -1033,7 +1054,7 @@ int check_latent_teams(const santapp_latent_geom *g, const santapp_latent_teams 
     if (!t) return SANTAPP_ERR_INVALID_ARG;
     if (!t->rows_packed || !t->rep_rows || !t->team_row_start || !t->seq_row_off || !t->seq_team_off || !t->rep_abs_max)
         return SANTAPP_ERR_INVALID_ARG;
-    if (lat_misaligned(t->rows_packed, 16) || lat_misaligned(t->rep_rows, 16) || lat_misaligned(t->team_row_start, 4)
+    if (lat_misaligned(t->rows_packed, 16) || lat_misaligned(t->rep_rows, 32) || lat_misaligned(t->team_row_start, 4)
         || lat_misaligned(t->row_token, 4) || lat_misaligned(t->seq_row_off, 8) || lat_misaligned(t->seq_team_off, 8)
         || lat_misaligned(t->rep_abs_max, 4))
         return SANTAPP_ERR_INVALID_ARG;
@@ -1190,7 +1211,7 @@ int santapp_latent_build_teams(const santapp_latent_geom *geom, const int32_t *p
         || !teams->seq_team_off || !teams->rep_abs_max)
         return SANTAPP_ERR_INVALID_ARG;
     if (lat_misaligned(rows_prompt, 16) || lat_misaligned(workspace, 16) || lat_misaligned(teams->rows_packed, 16)
-        || lat_misaligned(teams->rep_rows, 16) || lat_misaligned(teams->team_row_start, 4) || lat_misaligned(teams->row_token, 4)
+        || lat_misaligned(teams->rep_rows, 32) || lat_misaligned(teams->team_row_start, 4) || lat_misaligned(teams->row_token, 4)
         || lat_misaligned(teams->seq_row_off, 8) || lat_misaligned(teams->seq_team_off, 8) || lat_misaligned(teams->rep_abs_max, 4))
         return SANTAPP_ERR_INVALID_ARG;
     if (workspace_bytes < sz.build_workspace_bytes) return SANTAPP_ERR_WORKSPACE_TOO_SMALL;
